@@ -1,0 +1,145 @@
+"""Dithered backward products in fp64 (test infrastructure).
+
+The method reaches exactly the dense products with the quantized gradient
+delta~ = q * Delta (sparsity only skips zeros), so the oracle is the plain definition:
+
+  linear (row-major batch form of Eqs. (qda), (qdw)):
+      dX[b,k] = sum_j delta~[b,j] W[j,k]          (delta_a^{l-1} = W^T delta~_z)
+      dW[j,k] = sum_b delta~[b,j] X[b,k]          (delta_W = delta~_z a^T)
+      db[j]   = sum_b delta~[b,j]
+  convolution ("analogous for convolutional layers", Section 3): cross-correlation,
+  stride 1, zero padding p = (k-1)/2, NCHW,
+      z[b,co,y,x]      = sum_{ci,ky,kx} W[co,ci,ky,kx] X[b,ci,y+ky-p,x+kx-p]
+      dW[co,ci,ky,kx]  = sum_{b,y,x} delta~[b,co,y,x] X[b,ci,y+ky-p,x+kx-p]
+      dX[b,ci,y',x']   = sum_{co,ky,kx} delta~[b,co,y'-ky+p,x'-kx+p] W[co,ci,ky,kx]
+
+Each routine can also return S = sum |term| per output, the scale of the elementwise
+error bound |err| <= tol * S.
+"""
+import numpy as np
+
+
+def _dq(codes, Delta):
+    return np.asarray(codes, dtype=np.float64) * float(np.float32(Delta))
+
+
+def linear_backward(codes, Delta, X, W, with_abs=False):
+    """codes [B,N] int, X [B,K], W [N,K] -> dict(dW [N,K], dX [B,K], db [N]) in fp64."""
+    d = _dq(codes, Delta)
+    X = np.asarray(X, dtype=np.float64)
+    W = np.asarray(W, dtype=np.float64)
+    out = {"dW": d.T @ X, "dX": d @ W, "db": d.sum(axis=0)}
+    if with_abs:
+        a = np.abs(d)
+        out["S_dW"] = a.T @ np.abs(X)
+        out["S_dX"] = a @ np.abs(W)
+        out["S_db"] = a.sum(axis=0)
+    return out
+
+
+def _pad_hw(a, p):
+    return np.pad(a, ((0, 0), (0, 0), (p, p), (p, p)))
+
+
+def conv_forward(X, W):
+    """z = W * X (cross-correlation, stride 1, pad (k-1)/2), fp64."""
+    X = np.asarray(X, dtype=np.float64)
+    W = np.asarray(W, dtype=np.float64)
+    B, Ci, H, Wd = X.shape
+    Co, Ci2, k, k2 = W.shape
+    assert Ci == Ci2 and k == k2 and k % 2 == 1
+    p = (k - 1) // 2
+    Xp = _pad_hw(X, p)
+    z = np.zeros((B, Co, H, Wd))
+    for ky in range(k):
+        for kx in range(k):
+            z += np.einsum("bchw,oc->bohw", Xp[:, :, ky:ky + H, kx:kx + Wd], W[:, :, ky, kx],
+                           optimize=True)
+    return z
+
+
+def conv_backward(codes, Delta, X, W, with_abs=False):
+    """codes [B,Co,H,W], X [B,Ci,H,W], W [Co,Ci,k,k] -> dict(dW, dX, db) in fp64."""
+    d = _dq(codes, Delta)
+    X = np.asarray(X, dtype=np.float64)
+    W = np.asarray(W, dtype=np.float64)
+    B, Co, H, Wd = d.shape
+    _, Ci, _, _ = X.shape
+    k = W.shape[2]
+    assert W.shape == (Co, Ci, k, k) and k % 2 == 1 and X.shape == (B, Ci, H, Wd)
+    p = (k - 1) // 2
+
+    def both(dd, XX, WW):
+        Xp = _pad_hw(XX, p)
+        dp = _pad_hw(dd, p)
+        dW = np.zeros((Co, Ci, k, k))
+        dX = np.zeros((B, Ci, H, Wd))
+        for ky in range(k):
+            for kx in range(k):
+                # dW[co,ci,ky,kx] = sum_{b,y,x} d[b,co,y,x] X[b,ci,y+ky-p,x+kx-p]
+                dW[:, :, ky, kx] = np.einsum("bohw,bchw->oc", dd,
+                                             Xp[:, :, ky:ky + H, kx:kx + Wd], optimize=True)
+                # dX[b,ci,y',x'] += sum_co d[b,co,y'-ky+p,x'-kx+p] W[co,ci,ky,kx]
+                # padded index of d: (y'-ky+p)+p = y' + (2p-ky)
+                oy, ox = 2 * p - ky, 2 * p - kx
+                dX += np.einsum("bohw,oc->bchw", dp[:, :, oy:oy + H, ox:ox + Wd],
+                                WW[:, :, ky, kx], optimize=True)
+        return dW, dX
+
+    dW, dX = both(d, X, W)
+    out = {"dW": dW, "dX": dX, "db": d.sum(axis=(0, 2, 3))}
+    if with_abs:
+        sW, sX = both(np.abs(d), np.abs(X), np.abs(W))
+        out["S_dW"], out["S_dX"] = sW, sX
+        out["S_db"] = np.abs(d).sum(axis=(0, 2, 3))
+    return out
+
+
+# ---- brute force on tiny shapes: the definitions as nested loops, no library contraction ----
+
+def linear_backward_bruteforce(codes, Delta, X, W):
+    D = float(np.float32(Delta))
+    B, N = np.shape(codes)
+    K = np.shape(X)[1]
+    dW = [[0.0] * K for _ in range(N)]
+    dX = [[0.0] * K for _ in range(B)]
+    db = [0.0] * N
+    for b in range(B):
+        for j in range(N):
+            t = float(codes[b][j]) * D
+            db[j] += t
+            for k in range(K):
+                dW[j][k] += t * float(X[b][k])
+                dX[b][k] += t * float(W[j][k])
+    return {"dW": np.array(dW), "dX": np.array(dX), "db": np.array(db)}
+
+
+def conv_backward_bruteforce(codes, Delta, X, W):
+    D = float(np.float32(Delta))
+    codes = np.asarray(codes)
+    X = np.asarray(X, dtype=np.float64)
+    W = np.asarray(W, dtype=np.float64)
+    B, Co, H, Wd = codes.shape
+    Ci = X.shape[1]
+    k = W.shape[2]
+    p = (k - 1) // 2
+    dW = np.zeros((Co, Ci, k, k))
+    dX = np.zeros((B, Ci, H, Wd))
+    db = np.zeros(Co)
+    for b in range(B):
+        for co in range(Co):
+            for y in range(H):
+                for x in range(Wd):
+                    t = float(codes[b, co, y, x]) * D
+                    if t == 0.0:
+                        continue
+                    db[co] += t
+                    for ci in range(Ci):
+                        for ky in range(k):
+                            for kx in range(k):
+                                yy, xx = y + ky - p, x + kx - p
+                                if 0 <= yy < H and 0 <= xx < Wd:
+                                    # forward term z[b,co,y,x] += W[co,ci,ky,kx] X[b,ci,yy,xx]
+                                    dW[co, ci, ky, kx] += t * X[b, ci, yy, xx]
+                                    dX[b, ci, yy, xx] += t * W[co, ci, ky, kx]
+    return {"dW": dW, "dX": dX, "db": db}
