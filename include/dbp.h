@@ -1,0 +1,179 @@
+/*
+ * dbp.h -- C ABI of the dithered-backprop library for NVIDIA B200 (sm_100a).
+ *
+ * The library computes the backward pass of linear and convolution layers in which the
+ * preactivation gradient delta_z is first quantized by non-subtractive dither (NSD) and the
+ * resulting sparse tensor of small-integer codes drives both backward products
+ * (Wiedemann et al., "Dithered backprop", Section 3: Eq. (nsd), Algorithm 1,
+ * Eqs. (qdz), (qda), (qdw)).
+ *
+ * Conventions for every call
+ *   - Unless a function name ends in `_host`, every data pointer is a DEVICE pointer owned by
+ *     the caller, to contiguous row-major memory whose base is 16-byte aligned. The library
+ *     allocates only its own per-context workspace.
+ *   - Calls enqueue work on the context's CUDA stream and return without synchronising
+ *     (the `_host` variants and dbp_last_device_status synchronise the stream).
+ *   - Return value: DBP_OK or a negative dbp_status. Errors the host can see (null or
+ *     misaligned pointers, bad sizes, unsupported kernel size) return before anything is
+ *     enqueued. Conditions only the device can see (non-finite delta, codes clipped to
+ *     +-127) leave all outputs defined and are reported by dbp_last_device_status.
+ *   - There is no CPU fallback: every step runs in the library's CUDA kernels.
+ *   - One context per host thread and stream; calls on one context are not re-entrant.
+ */
+#ifndef DBP_H_
+#define DBP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dbp_ctx dbp_ctx;
+
+typedef enum { DBP_F32 = 0, DBP_BF16 = 1 } dbp_dtype;
+
+typedef enum {
+    DBP_OK = 0,
+    DBP_EINVAL = -1,        /* null / misaligned pointer, non-positive size, bad enum */
+    DBP_EUNSUPPORTED = -2,  /* kernel size, stride or padding outside {1x1, 3x3; 1; (k-1)/2} */
+    DBP_ECUDA = -3,         /* a CUDA runtime call failed */
+    DBP_ENOMEM = -4,        /* workspace allocation failed */
+    DBP_ENONFINITE = -5,    /* device: delta holds NaN or Inf (all codes were set to 0) */
+    DBP_ESATURATED = -6,    /* device: some codes were clipped to +-127 */
+    DBP_ECAPACITY = -7      /* a caller-provided size is smaller than required */
+} dbp_status;
+
+/* flags for the backward calls */
+#define DBP_FORCE_SPARSE 1u /* always use the sparse gather kernels */
+#define DBP_FORCE_DENSE  2u /* always use the dense tensor-core path (where it exists) */
+#define DBP_DX_F32       4u /* with io = DBP_BF16: write dX as fp32 instead of bf16 */
+
+/* Elements per segment of the sparse structure (see dbp_sparse). */
+#define DBP_SEGMENT 1024
+
+/*
+ * Sparse form of the quantized gradient delta~ = Delta * q (the "sparse tensors with low
+ * precision non-zero values" of Section 1; the paper fixes no storage format, this one is
+ * the library's). The tensor is taken flat, element i at its row-major offset.
+ *   bitmap  : bit (i & 31) of word (i >> 5) is 1 iff q_i != 0.
+ *   values  : the non-zero int8 codes of segment g (elements g*1024 ... g*1024+1023) in
+ *             element order, packed from values[g*1024]; bytes past the segment's count
+ *             are unspecified.
+ *   offsets : offsets[w] = number of non-zero codes of word w's segment that precede word w.
+ *             So code i lives at values[(i>>10)*1024 + offsets[i>>5] + popc(bitmap[i>>5] &
+ *             ((1u << (i&31)) - 1))].
+ *   delta   : device scalar, the step size Delta used.
+ *   nnz     : device scalar, number of non-zero codes.
+ * Buffer sizes for a given numel come from dbp_sparse_bytes.
+ */
+typedef struct dbp_sparse {
+    uint32_t *bitmap;
+    uint16_t *offsets;
+    int8_t *values;
+    float *delta;
+    long long *nnz;
+    long long numel;
+} dbp_sparse;
+
+/* Context. `device` is a CUDA ordinal; `cuda_stream` is a cudaStream_t (NULL = default
+ * stream). The context owns its workspace and frees it in dbp_destroy. */
+int dbp_create(dbp_ctx **out, int device, void *cuda_stream);
+int dbp_destroy(dbp_ctx *ctx);
+int dbp_set_stream(dbp_ctx *ctx, void *cuda_stream);
+const char *dbp_status_string(int status);
+
+/* Synchronises the stream, then reports the device-side condition of the calls since the
+ * previous report (DBP_OK, DBP_ENONFINITE or DBP_ESATURATED) and the number of clipped
+ * codes; both outputs may be NULL. Clears the record. */
+int dbp_last_device_status(dbp_ctx *ctx, int *status, long long *saturated);
+
+/* Bytes the caller must allocate for each array of a dbp_sparse over `numel` elements. */
+int dbp_sparse_bytes(long long numel, size_t *bitmap_bytes, size_t *offsets_bytes,
+                     size_t *values_bytes);
+
+/*
+ * Algorithm 1 (NSD): sigma = population std of delta over all `numel` elements,
+ * Delta = scale * sigma, q_i = floor(delta_i / Delta + u_i) (Eq. (nsd) with the dither
+ * nu_i = (u_i - 1/2) Delta), clipped to [-127, 127].
+ *   delta    : numel elements of `dtype`.
+ *   seed     : u_i comes from output (i >> 1) of the SplitMix64 sequence started at `seed`
+ *              (low 32 bits for even i, high for odd); its top 23 bits k give
+ *              u_i = (2k+1) 2^-24.
+ *   scale    : s > 0. If scale <= 0 the step is read from the device scalar *delta_in.
+ *   out      : arrays sized by dbp_sparse_bytes; out->numel is set by the call;
+ *              *out->delta and *out->nnz are written on the device.
+ * sigma = 0 is not an error (Delta = 0, every code 0).
+ */
+int nsd_quantize(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
+                 unsigned long long seed, float scale, const float *delta_in, dbp_sparse *out);
+
+/* Expands a dbp_sparse to one int8 code per element (codes: numel bytes, device). */
+int nsd_decode_dense(dbp_ctx *ctx, const dbp_sparse *q, int8_t *codes);
+
+/*
+ * Dithered backward of a linear layer z = a W^T (Eqs. (qdz), (qda), (qdw), row-major batch
+ * form): quantizes delta [B,N] as in nsd_quantize, then
+ *     dX[b,k] = Delta sum_j q[b,j] W[j,k]      dW[j,k] = Delta sum_b q[b,j] X[b,k]
+ *     db[j]   = Delta sum_b q[b,j]
+ * X [B,K], W [N,K], delta [B,N] are of dtype `io`; dW [N,K] and db [N] are fp32; dX [B,K]
+ * is of dtype `io` (fp32 with DBP_DX_F32). Any of dW, dX, db may be NULL (skipped).
+ * q_out may be NULL; otherwise it receives the sparse structure (arrays sized for B*N).
+ * Outputs are overwritten, not accumulated.
+ */
+int dithered_linear_backward(dbp_ctx *ctx, const void *delta, const void *X, const void *W,
+                             int io, long long B, long long N, long long K,
+                             unsigned long long seed, float scale, const float *delta_in,
+                             dbp_sparse *q_out, float *dW, void *dX, float *db,
+                             unsigned flags);
+
+/*
+ * The same for a convolution layer ("analogous for convolutional layers", Section 3):
+ * cross-correlation, NCHW, square kernel k in {1, 3}, stride 1, zero padding (k-1)/2.
+ * delta [B,Cout,H,W], X [B,Cin,H,W], W [Cout,Cin,k,k]:
+ *     dX[b,ci,y,x]     = Delta sum_{co,ky,kx} q[b,co,y-ky+p,x-kx+p] W[co,ci,ky,kx]
+ *     dW[co,ci,ky,kx]  = Delta sum_{b,y,x}    q[b,co,y,x] X[b,ci,y+ky-p,x+kx-p]
+ *     db[co]           = Delta sum_{b,y,x}    q[b,co,y,x]
+ * Other k, stride or pad return DBP_EUNSUPPORTED.
+ */
+int dithered_conv_backward(dbp_ctx *ctx, const void *delta, const void *X, const void *W,
+                           int io, long long B, long long Cin, long long Cout, long long H,
+                           long long Wd, int k, int stride, int pad,
+                           unsigned long long seed, float scale, const float *delta_in,
+                           dbp_sparse *q_out, float *dW, void *dX, float *db, unsigned flags);
+
+/*
+ * Host-buffer variants: every pointer (delta, X, W, dW, dX, db, and the two scalars) is a
+ * HOST pointer. The call copies the inputs to the device workspace, runs the same kernels,
+ * copies the results back and synchronises. delta_out / nnz_out (may be NULL) receive the
+ * step size and the number of non-zero codes.
+ */
+int dithered_linear_backward_host(dbp_ctx *ctx, const void *delta, const void *X, const void *W,
+                                  int io, long long B, long long N, long long K,
+                                  unsigned long long seed, float scale,
+                                  float *dW, void *dX, float *db, unsigned flags,
+                                  float *delta_out, long long *nnz_out);
+int dithered_conv_backward_host(dbp_ctx *ctx, const void *delta, const void *X, const void *W,
+                                int io, long long B, long long Cin, long long Cout, long long H,
+                                long long Wd, int k, int stride, int pad,
+                                unsigned long long seed, float scale,
+                                float *dW, void *dX, float *db, unsigned flags,
+                                float *delta_out, long long *nnz_out);
+
+/*
+ * Elementwise steps between layers of a network's backward pass (Section 3, backward
+ * equations): delta_z = delta_a (.) f'(z) for ReLU, with the derivative given as one byte
+ * per element (0 or 1), and the 2x2 max-pool routing of a pooled gradient g [planes,h,w] to
+ * out [planes,2h,2w], argmax in {0,1,2,3} being the row-major position of the forward
+ * maximum inside each window. fp32 device arrays.
+ */
+int dbp_relu_backward(dbp_ctx *ctx, const float *delta_a, const uint8_t *mask, float *delta_z,
+                      long long numel);
+int dbp_maxpool2x2_backward(dbp_ctx *ctx, const float *g, const int8_t *argmax, float *out,
+                            long long planes, long long h, long long w);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DBP_H_ */

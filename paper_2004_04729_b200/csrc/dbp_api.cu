@@ -1,0 +1,326 @@
+// C ABI entry points (see include/dbp.h): argument checks, workspace, kernel sequencing.
+#include <new>
+
+#include "dbp_internal.cuh"
+
+namespace dbp {
+
+int ws_reserve(dbp_ctx *ctx, Workspace &w, size_t bytes) {
+    if (bytes <= w.bytes) return DBP_OK;
+    // the stream may still be using the old block
+    if (w.ptr) {
+        if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return DBP_ECUDA;
+        cudaFree(w.ptr);
+        w.ptr = nullptr;
+        w.bytes = 0;
+    }
+    const size_t want = (bytes + (size_t(1) << 20) - 1) & ~((size_t(1) << 20) - 1);
+    if (cudaMalloc(&w.ptr, want) != cudaSuccess) {
+        cudaGetLastError();
+        w.ptr = nullptr;
+        return DBP_ENOMEM;
+    }
+    w.bytes = want;
+    return DBP_OK;
+}
+
+namespace {
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+size_t elem_size(int dtype) { return dtype == DBP_F32 ? 4 : 2; }
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+// Quantize delta into `sp` (caller's arrays, or the context's internal ones) and into the
+// context's dense code buffer, which the product kernels read.
+int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
+                          unsigned long long seed, float scale, const float *delta_in,
+                          dbp_sparse *q_out, const float **delta_p, const int8_t **codes) {
+    size_t bb, ob, vb;
+    int rc = dbp_sparse_bytes(numel, &bb, &ob, &vb);
+    if (rc) return rc;
+    dbp_sparse sp;
+    if (q_out) {
+        if (!q_out->bitmap || !q_out->offsets || !q_out->values || !q_out->delta || !q_out->nnz) return DBP_EINVAL;
+        if (!aligned16(q_out->bitmap) || !aligned16(q_out->offsets) || !aligned16(q_out->values)) return DBP_EINVAL;
+        q_out->numel = numel;
+        sp = *q_out;
+    } else {
+        if ((rc = ws_reserve(ctx, ctx->sp_bitmap, bb)) || (rc = ws_reserve(ctx, ctx->sp_offsets, ob)) ||
+            (rc = ws_reserve(ctx, ctx->sp_values, vb)))
+            return rc;
+        sp.bitmap = static_cast<uint32_t *>(ctx->sp_bitmap.ptr);
+        sp.offsets = static_cast<uint16_t *>(ctx->sp_offsets.ptr);
+        sp.values = static_cast<int8_t *>(ctx->sp_values.ptr);
+        sp.delta = nullptr;
+        sp.nnz = nullptr;
+        sp.numel = numel;
+    }
+    if ((rc = ws_reserve(ctx, ctx->dense_codes, static_cast<size_t>(numel) + 16))) return rc;
+    int8_t *dense = static_cast<int8_t *>(ctx->dense_codes.ptr);
+    if ((rc = launch_statistics(ctx, delta, dtype, numel, scale, delta_in, sp.delta,
+                                reinterpret_cast<unsigned long long *>(sp.nnz))))
+        return rc;
+    if ((rc = launch_quantize(ctx, delta, dtype, numel, seed, &ctx->state->delta, sp.bitmap, sp.offsets,
+                              sp.values, dense, reinterpret_cast<unsigned long long *>(sp.nnz))))
+        return rc;
+    *delta_p = &ctx->state->delta;
+    *codes = dense;
+    return DBP_OK;
+}
+
+int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const void *W, int io,
+                       const ConvShape &s, unsigned long long seed, float scale,
+                       const float *delta_in, dbp_sparse *q_out, float *dW, void *dX, float *db,
+                       unsigned flags) {
+    if (!ctx || !delta) return DBP_EINVAL;
+    if (io != DBP_F32 && io != DBP_BF16) return DBP_EINVAL;
+    if (s.B <= 0 || s.Cin <= 0 || s.Cout <= 0 || s.H <= 0 || s.W <= 0) return DBP_EINVAL;
+    if (s.B > 65535 * 32 || s.Cin > (1 << 20) || s.Cout > (1 << 20) || s.H > 4096 || s.W > 4096) return DBP_EINVAL;
+    if (!(scale > 0.f) && !delta_in) return DBP_EINVAL;
+    if ((dW && !X) || (dX && !W)) return DBP_EINVAL;
+    if (!aligned16(delta) || !aligned16(X) || !aligned16(W) || !aligned16(dW) || !aligned16(dX)) return DBP_EINVAL;
+    if ((flags & DBP_FORCE_SPARSE) && (flags & DBP_FORCE_DENSE)) return DBP_EINVAL;
+    if (flags & DBP_FORCE_DENSE) return DBP_EUNSUPPORTED;   // no dense tensor-core path yet
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DBP_ECUDA;
+    const long long numel = s.B * s.Cout * s.H * s.W;
+    const float *delta_p = nullptr;
+    const int8_t *codes = nullptr;
+    int rc = quantize_for_products(ctx, delta, io, numel, seed, scale, delta_in, q_out, &delta_p, &codes);
+    if (rc) return rc;
+    if (dX) {
+        const size_t wb = sizeof(float) * static_cast<size_t>(s.Cout) * s.Cin * s.k * s.k;
+        if ((rc = ws_reserve(ctx, ctx->w_taps, wb))) return rc;
+        float *wt = static_cast<float *>(ctx->w_taps.ptr);
+        if ((rc = launch_weight_taps(ctx, W, io, s, wt))) return rc;
+        const bool dx_bf16 = (io == DBP_BF16) && !(flags & DBP_DX_F32);
+        if ((rc = launch_conv_dx(ctx, codes, wt, delta_p, s, dX, dx_bf16))) return rc;
+    }
+    if (dW && (rc = launch_conv_dw(ctx, codes, X, io, delta_p, s, dW))) return rc;
+    if (db && (rc = launch_bias_grad(ctx, codes, delta_p, s, db))) return rc;
+    return DBP_OK;
+}
+
+}  // namespace
+}  // namespace dbp
+
+using namespace dbp;
+
+extern "C" {
+
+int dbp_create(dbp_ctx **out, int device, void *cuda_stream) {
+    if (!out) return DBP_EINVAL;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+        cudaGetLastError();
+        return DBP_ECUDA;
+    }
+    DeviceGuard guard(device);
+    if (!guard.ok) return DBP_ECUDA;
+    dbp_ctx *ctx = new (std::nothrow) dbp_ctx();
+    if (!ctx) return DBP_ENOMEM;
+    ctx->device = device;
+    ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) == cudaSuccess) ctx->sm_count = prop.multiProcessorCount;
+    ctx->partial_blocks = ctx->sm_count * 8;
+    if (cudaMalloc(&ctx->state, sizeof(DeviceState)) != cudaSuccess ||
+        cudaMalloc(&ctx->partials, sizeof(double) * 2 * ctx->partial_blocks) != cudaSuccess ||
+        cudaMemset(ctx->state, 0, sizeof(DeviceState)) != cudaSuccess) {
+        cudaGetLastError();
+        dbp_destroy(ctx);
+        return DBP_ENOMEM;
+    }
+    *out = ctx;
+    return DBP_OK;
+}
+
+int dbp_destroy(dbp_ctx *ctx) {
+    if (!ctx) return DBP_EINVAL;
+    DeviceGuard guard(ctx->device);
+    cudaStreamSynchronize(ctx->stream);
+    Workspace *all[] = {&ctx->dense_codes, &ctx->w_taps, &ctx->sp_bitmap, &ctx->sp_offsets, &ctx->sp_values};
+    for (Workspace *w : all) if (w->ptr) cudaFree(w->ptr);
+    for (Workspace &w : ctx->io) if (w.ptr) cudaFree(w.ptr);
+    if (ctx->state) cudaFree(ctx->state);
+    if (ctx->partials) cudaFree(ctx->partials);
+    delete ctx;
+    return DBP_OK;
+}
+
+int dbp_set_stream(dbp_ctx *ctx, void *cuda_stream) {
+    if (!ctx) return DBP_EINVAL;
+    ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+    return DBP_OK;
+}
+
+const char *dbp_status_string(int status) {
+    switch (status) {
+        case DBP_OK: return "ok";
+        case DBP_EINVAL: return "invalid argument";
+        case DBP_EUNSUPPORTED: return "unsupported configuration";
+        case DBP_ECUDA: return "CUDA runtime error";
+        case DBP_ENOMEM: return "out of memory";
+        case DBP_ENONFINITE: return "non-finite value in delta";
+        case DBP_ESATURATED: return "codes clipped to +-127";
+        case DBP_ECAPACITY: return "buffer too small";
+        default: return "unknown status";
+    }
+}
+
+int dbp_last_device_status(dbp_ctx *ctx, int *status, long long *saturated) {
+    if (!ctx) return DBP_EINVAL;
+    DeviceGuard guard(ctx->device);
+    DeviceState h;
+    if (cudaMemcpyAsync(&h, ctx->state, sizeof(h), cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess ||
+        cudaStreamSynchronize(ctx->stream) != cudaSuccess)
+        return DBP_ECUDA;
+    if (status) *status = h.nonfinite ? DBP_ENONFINITE : (h.saturated ? DBP_ESATURATED : DBP_OK);
+    if (saturated) *saturated = static_cast<long long>(h.saturated);
+    if (h.nonfinite || h.saturated) {
+        if (cudaMemsetAsync(&ctx->state->nonfinite, 0, sizeof(int), ctx->stream) != cudaSuccess ||
+            cudaMemsetAsync(&ctx->state->saturated, 0, sizeof(unsigned long long), ctx->stream) != cudaSuccess)
+            return DBP_ECUDA;
+    }
+    return DBP_OK;
+}
+
+int dbp_sparse_bytes(long long numel, size_t *bitmap_bytes, size_t *offsets_bytes, size_t *values_bytes) {
+    if (numel <= 0) return DBP_EINVAL;
+    const size_t nseg = (static_cast<size_t>(numel) + kSegment - 1) / kSegment;
+    if (bitmap_bytes) *bitmap_bytes = nseg * kWordsPerSegment * sizeof(uint32_t);
+    if (offsets_bytes) *offsets_bytes = nseg * kWordsPerSegment * sizeof(uint16_t);
+    if (values_bytes) *values_bytes = nseg * kSegment;
+    return DBP_OK;
+}
+
+int nsd_quantize(dbp_ctx *ctx, const void *delta, int dtype, long long numel, unsigned long long seed,
+                 float scale, const float *delta_in, dbp_sparse *out) {
+    if (!ctx || !delta || !out || numel <= 0) return DBP_EINVAL;
+    if (dtype != DBP_F32 && dtype != DBP_BF16) return DBP_EINVAL;
+    if (!(scale > 0.f) && !delta_in) return DBP_EINVAL;
+    if (!out->bitmap || !out->offsets || !out->values || !out->delta || !out->nnz) return DBP_EINVAL;
+    if (!aligned16(delta) || !aligned16(out->bitmap) || !aligned16(out->offsets) || !aligned16(out->values))
+        return DBP_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DBP_ECUDA;
+    out->numel = numel;
+    int rc = launch_statistics(ctx, delta, dtype, numel, scale, delta_in, out->delta,
+                               reinterpret_cast<unsigned long long *>(out->nnz));
+    if (rc) return rc;
+    return launch_quantize(ctx, delta, dtype, numel, seed, &ctx->state->delta, out->bitmap, out->offsets,
+                           out->values, nullptr, reinterpret_cast<unsigned long long *>(out->nnz));
+}
+
+int nsd_decode_dense(dbp_ctx *ctx, const dbp_sparse *q, int8_t *codes) {
+    if (!ctx || !q || !codes || q->numel <= 0 || !q->bitmap || !q->offsets || !q->values) return DBP_EINVAL;
+    if (!aligned16(codes)) return DBP_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DBP_ECUDA;
+    return launch_decode(ctx, q->bitmap, q->offsets, q->values, q->numel, codes);
+}
+
+int dithered_linear_backward(dbp_ctx *ctx, const void *delta, const void *X, const void *W, int io,
+                             long long B, long long N, long long K, unsigned long long seed, float scale,
+                             const float *delta_in, dbp_sparse *q_out, float *dW, void *dX, float *db,
+                             unsigned flags) {
+    // [B,N] x [N,K]: the 1x1 convolution with one position per image has the same layout
+    ConvShape s{B, K, N, 1, 1, 1};
+    return conv_backward_impl(ctx, delta, X, W, io, s, seed, scale, delta_in, q_out, dW, dX, db, flags);
+}
+
+int dithered_conv_backward(dbp_ctx *ctx, const void *delta, const void *X, const void *W, int io,
+                           long long B, long long Cin, long long Cout, long long H, long long Wd, int k,
+                           int stride, int pad, unsigned long long seed, float scale,
+                           const float *delta_in, dbp_sparse *q_out, float *dW, void *dX, float *db,
+                           unsigned flags) {
+    if ((k != 1 && k != 3) || stride != 1 || pad != (k - 1) / 2) return DBP_EUNSUPPORTED;
+    ConvShape s{B, Cin, Cout, H, Wd, k};
+    return conv_backward_impl(ctx, delta, X, W, io, s, seed, scale, delta_in, q_out, dW, dX, db, flags);
+}
+
+static int host_backward(dbp_ctx *ctx, const void *delta, const void *X, const void *W, int io,
+                         const ConvShape &s, unsigned long long seed, float scale, float *dW, void *dX,
+                         float *db, unsigned flags, float *delta_out, long long *nnz_out) {
+    if (!ctx || !delta) return DBP_EINVAL;
+    if (io != DBP_F32 && io != DBP_BF16) return DBP_EINVAL;
+    if (s.B <= 0 || s.Cin <= 0 || s.Cout <= 0 || s.H <= 0 || s.W <= 0) return DBP_EINVAL;
+    if ((dW && !X) || (dX && !W)) return DBP_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DBP_ECUDA;
+    const size_t es = elem_size(io);
+    const size_t nd = static_cast<size_t>(s.B) * s.Cout * s.H * s.W;
+    const size_t nx = static_cast<size_t>(s.B) * s.Cin * s.H * s.W;
+    const size_t nw = static_cast<size_t>(s.Cout) * s.Cin * s.k * s.k;
+    const size_t dx_es = (io == DBP_BF16 && !(flags & DBP_DX_F32)) ? 2 : 4;
+    int rc;
+    if ((rc = ws_reserve(ctx, ctx->io[0], nd * es)) || (rc = ws_reserve(ctx, ctx->io[1], X ? nx * es : 16)) ||
+        (rc = ws_reserve(ctx, ctx->io[2], W ? nw * es : 16)) || (rc = ws_reserve(ctx, ctx->io[3], dW ? nw * 4 : 16)) ||
+        (rc = ws_reserve(ctx, ctx->io[4], dX ? nx * dx_es : 16)) || (rc = ws_reserve(ctx, ctx->io[5], db ? s.Cout * 4 : 16)))
+        return rc;
+    cudaStream_t st = ctx->stream;
+    if (cudaMemcpyAsync(ctx->io[0].ptr, delta, nd * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return DBP_ECUDA;
+    if (X && cudaMemcpyAsync(ctx->io[1].ptr, X, nx * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return DBP_ECUDA;
+    if (W && cudaMemcpyAsync(ctx->io[2].ptr, W, nw * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return DBP_ECUDA;
+    rc = conv_backward_impl(ctx, ctx->io[0].ptr, X ? ctx->io[1].ptr : nullptr, W ? ctx->io[2].ptr : nullptr, io, s,
+                            seed, scale, nullptr, nullptr, dW ? static_cast<float *>(ctx->io[3].ptr) : nullptr,
+                            dX ? ctx->io[4].ptr : nullptr, db ? static_cast<float *>(ctx->io[5].ptr) : nullptr, flags);
+    if (rc) return rc;
+    if (dW && cudaMemcpyAsync(dW, ctx->io[3].ptr, nw * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DBP_ECUDA;
+    if (dX && cudaMemcpyAsync(dX, ctx->io[4].ptr, nx * dx_es, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DBP_ECUDA;
+    if (db && cudaMemcpyAsync(db, ctx->io[5].ptr, s.Cout * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DBP_ECUDA;
+    DeviceState h;
+    if (cudaMemcpyAsync(&h, ctx->state, sizeof(h), cudaMemcpyDeviceToHost, st) != cudaSuccess) return DBP_ECUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return DBP_ECUDA;
+    if (delta_out) *delta_out = h.delta;
+    if (nnz_out) *nnz_out = static_cast<long long>(h.nnz);
+    return DBP_OK;
+}
+
+int dithered_linear_backward_host(dbp_ctx *ctx, const void *delta, const void *X, const void *W, int io,
+                                  long long B, long long N, long long K, unsigned long long seed,
+                                  float scale, float *dW, void *dX, float *db, unsigned flags,
+                                  float *delta_out, long long *nnz_out) {
+    if (!(scale > 0.f)) return DBP_EINVAL;
+    ConvShape s{B, K, N, 1, 1, 1};
+    return host_backward(ctx, delta, X, W, io, s, seed, scale, dW, dX, db, flags, delta_out, nnz_out);
+}
+
+int dithered_conv_backward_host(dbp_ctx *ctx, const void *delta, const void *X, const void *W, int io,
+                                long long B, long long Cin, long long Cout, long long H, long long Wd,
+                                int k, int stride, int pad, unsigned long long seed, float scale,
+                                float *dW, void *dX, float *db, unsigned flags, float *delta_out,
+                                long long *nnz_out) {
+    if ((k != 1 && k != 3) || stride != 1 || pad != (k - 1) / 2) return DBP_EUNSUPPORTED;
+    if (!(scale > 0.f)) return DBP_EINVAL;
+    ConvShape s{B, Cin, Cout, H, Wd, k};
+    return host_backward(ctx, delta, X, W, io, s, seed, scale, dW, dX, db, flags, delta_out, nnz_out);
+}
+
+int dbp_relu_backward(dbp_ctx *ctx, const float *delta_a, const uint8_t *mask, float *delta_z, long long numel) {
+    if (!ctx || !delta_a || !mask || !delta_z || numel <= 0) return DBP_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DBP_ECUDA;
+    return launch_relu_backward(ctx, delta_a, mask, delta_z, numel);
+}
+
+int dbp_maxpool2x2_backward(dbp_ctx *ctx, const float *g, const int8_t *argmax, float *out, long long planes,
+                            long long h, long long w) {
+    if (!ctx || !g || !argmax || !out || planes <= 0 || h <= 0 || w <= 0) return DBP_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DBP_ECUDA;
+    return launch_maxpool_backward(ctx, g, argmax, out, planes, h, w);
+}
+
+}  // extern "C"

@@ -1,0 +1,78 @@
+// Internal declarations shared by the library's translation units (not part of the ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dbp.h"
+
+namespace dbp {
+
+constexpr int kSegment = DBP_SEGMENT;          // elements per sparse segment
+constexpr int kWordsPerSegment = kSegment / 32;
+
+// Device-side scalars of one context.
+struct DeviceState {
+    float delta;                        // step size of the internal quantization
+    int nonfinite;                      // set when delta_z held NaN/Inf
+    unsigned int ticket;                // last-block election of the statistics kernel
+    int pad0;
+    unsigned long long nnz;             // non-zero codes of the internal quantization
+    unsigned long long saturated;       // clipped codes since the last report
+};
+
+struct Workspace {
+    void *ptr = nullptr;
+    size_t bytes = 0;
+};
+
+}  // namespace dbp
+
+struct dbp_ctx {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    int sm_count = 148;
+    dbp::DeviceState *state = nullptr;  // device
+    double *partials = nullptr;         // device, statistics partial sums
+    int partial_blocks = 0;
+    dbp::Workspace dense_codes;         // int8 per element of delta
+    dbp::Workspace w_taps;              // fp32 weights as [Cout][k*k][Cin]
+    dbp::Workspace sp_bitmap, sp_offsets, sp_values;  // internal dbp_sparse
+    dbp::Workspace io[8];               // staging for the *_host entry points
+};
+
+namespace dbp {
+
+int ws_reserve(dbp_ctx *ctx, Workspace &w, size_t bytes);
+
+// ---- nsd_kernels.cu
+int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long numel, float scale,
+                      const float *delta_in, float *delta_out, unsigned long long *nnz_out);
+int launch_quantize(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
+                    unsigned long long seed, const float *delta_p, uint32_t *bitmap,
+                    uint16_t *offsets, int8_t *values, int8_t *dense,
+                    unsigned long long *nnz_out);
+int launch_decode(dbp_ctx *ctx, const uint32_t *bitmap, const uint16_t *offsets,
+                  const int8_t *values, long long numel, int8_t *dense);
+
+// ---- product_kernels.cu
+struct ConvShape {
+    long long B, Cin, Cout, H, W;
+    int k;
+};
+int launch_weight_taps(dbp_ctx *ctx, const void *W, int dtype, const ConvShape &s, float *w_taps);
+int launch_conv_dx(dbp_ctx *ctx, const int8_t *codes, const float *w_taps, const float *delta_p,
+                   const ConvShape &s, void *dX, bool dx_bf16);
+int launch_conv_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, int dtype,
+                   const float *delta_p, const ConvShape &s, float *dW);
+int launch_bias_grad(dbp_ctx *ctx, const int8_t *codes, const float *delta_p, const ConvShape &s,
+                     float *db);
+int launch_relu_backward(dbp_ctx *ctx, const float *da, const uint8_t *mask, float *dz,
+                         long long n);
+int launch_maxpool_backward(dbp_ctx *ctx, const float *g, const int8_t *argmax, float *out,
+                            long long planes, long long h, long long w);
+
+inline int cuda_ok(cudaError_t e) { return e == cudaSuccess ? DBP_OK : DBP_ECUDA; }
+
+}  // namespace dbp

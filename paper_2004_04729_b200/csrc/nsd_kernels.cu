@@ -1,0 +1,351 @@
+// NSD quantization kernels: one-pass statistics (Algorithm 1, std line), dither + quantize +
+// compaction (Section 3.1, Eq. (nsd)), and expansion of the sparse structure to dense codes.
+//
+// Both streaming kernels are bound by HBM bandwidth: 128-bit loads of delta_z, 128-bit stores
+// of the packed codes, bitmap words and offsets assembled with warp shuffles.
+#include "dbp_internal.cuh"
+
+namespace dbp {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr unsigned kFull = 0xffffffffu;
+
+template <typename T>
+struct Elem;
+
+template <>
+struct Elem<float> {
+    static constexpr int EPT = 4;  // elements per 128-bit load
+    __device__ static void load(const float *p, float (&v)[4]) {
+        float4 q = __ldg(reinterpret_cast<const float4 *>(p));
+        v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+    }
+    __device__ static float one(const float *p) { return __ldg(p); }
+};
+
+template <>
+struct Elem<__nv_bfloat16> {
+    static constexpr int EPT = 8;
+    __device__ static void load(const __nv_bfloat16 *p, float (&v)[8]) {
+        uint4 q = __ldg(reinterpret_cast<const uint4 *>(p));
+        const unsigned w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[2 * i] = __uint_as_float(w[i] << 16);           // bf16 -> fp32 is exact
+            v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    }
+    __device__ static float one(const __nv_bfloat16 *p) {
+        return __uint_as_float(static_cast<unsigned>(__ldg(reinterpret_cast<const unsigned short *>(p))) << 16);
+    }
+};
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+    return v;
+}
+
+// ---------------------------------------------------------------- statistics (sigma, Delta)
+// Sum and sum of squares of every element: fp32 inside one 128-bit chunk, fp64 across
+// chunks, per-block partials combined in a fixed order by the last block to finish, so the
+// step size does not depend on scheduling. sigma is the population standard deviation about
+// the mean; Delta = scale * sigma rounded once to fp32.
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ partials,
+                  DeviceState *__restrict__ st, float scale, float *__restrict__ delta_out,
+                  unsigned long long *__restrict__ nnz_out) {
+    constexpr int EPT = Elem<T>::EPT;
+    const long long nvec = n / EPT;
+    double d1 = 0.0, d2 = 0.0;
+    const long long stride = static_cast<long long>(gridDim.x) * kThreads;
+    for (long long i = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x; i < nvec; i += stride) {
+        float v[EPT];
+        Elem<T>::load(x + i * EPT, v);
+        float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+        for (int j = 0; j < EPT; ++j) {
+            s1 += v[j];
+            s2 = fmaf(v[j], v[j], s2);
+        }
+        d1 += static_cast<double>(s1);
+        d2 += static_cast<double>(s2);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (long long i = nvec * EPT; i < n; ++i) {
+            const float v = Elem<T>::one(x + i);
+            d1 += static_cast<double>(v);
+            d2 += static_cast<double>(v) * static_cast<double>(v);
+        }
+    }
+    __shared__ double sh1[kThreads / 32], sh2[kThreads / 32];
+    __shared__ bool is_last;
+    d1 = warp_sum(d1);
+    d2 = warp_sum(d2);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) { sh1[warp] = d1; sh2[warp] = d2; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double a = 0.0, b = 0.0;
+        for (int w = 0; w < kThreads / 32; ++w) { a += sh1[w]; b += sh2[w]; }
+        partials[2 * blockIdx.x] = a;
+        partials[2 * blockIdx.x + 1] = b;
+        __threadfence();
+        const unsigned t = atomicAdd(&st->ticket, 1u);
+        is_last = (t == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last || warp != 0) return;
+    __threadfence();
+    double a = 0.0, b = 0.0;
+    for (int blk = lane; blk < static_cast<int>(gridDim.x); blk += 32) {
+        a += __ldcg(partials + 2 * blk);
+        b += __ldcg(partials + 2 * blk + 1);
+    }
+    a = warp_sum(a);
+    b = warp_sum(b);
+    if (lane == 0) {
+        float delta = 0.f;
+        if (!isfinite(a) || !isfinite(b)) {
+            st->nonfinite = 1;                      // every code becomes 0
+        } else {
+            const double mean = a / static_cast<double>(n);
+            double var = b / static_cast<double>(n) - mean * mean;
+            if (var < 0.0) var = 0.0;
+            delta = static_cast<float>(static_cast<double>(scale) * sqrt(var));
+        }
+        st->delta = delta;
+        st->nnz = 0ull;
+        st->ticket = 0u;
+        if (delta_out) *delta_out = delta;
+        if (nnz_out) *nnz_out = 0ull;
+    }
+}
+
+__global__ void set_step_kernel(const float *__restrict__ delta_in, DeviceState *st,
+                                float *delta_out, unsigned long long *nnz_out) {
+    const float d = *delta_in;
+    st->delta = d;
+    st->nnz = 0ull;
+    if (delta_out) *delta_out = d;
+    if (nnz_out) *nnz_out = 0ull;
+}
+
+// ---------------------------------------------------------------- dither + quantize + compact
+// SplitMix64 output number c of the sequence started at `seed` (counter-based: no state).
+__device__ __forceinline__ unsigned long long splitmix64_mix(unsigned long long z) {
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+// u = (2k+1) 2^-24 from the top 23 bits k of h: (1 + k 2^-23) - (1 - 2^-24), exact.
+__device__ __forceinline__ float dither_from_bits(unsigned h) {
+    return __uint_as_float(0x3f800000u | (h >> 9)) - 0.99999994f;
+}
+
+// q = floor(x / Delta + u) with one rounding, clipped to [-127, 127].
+__device__ __forceinline__ int quantize_one(float x, float inv, float u, unsigned &sat) {
+    const float f = floorf(__fmaf_rn(x, inv, u));
+    int q;
+    if (f > 127.f) { q = 127; ++sat; }
+    else if (f < -127.f) { q = -127; ++sat; }
+    else q = __float2int_rz(f);
+    return q;
+}
+
+// One warp owns one 1024-element segment at a time: ITER 128-bit loads per lane, codes
+// packed through a per-warp shared staging line, one coalesced store each of the 32 bitmap
+// words, the 32 offsets and the packed codes.
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+quantize_kernel(const T *__restrict__ x, long long n, unsigned long long seed,
+                const float *__restrict__ delta_p, uint32_t *__restrict__ bitmap,
+                uint16_t *__restrict__ offsets, int8_t *__restrict__ values,
+                int8_t *__restrict__ dense, DeviceState *__restrict__ st,
+                unsigned long long *__restrict__ nnz_out) {
+    constexpr int EPT = Elem<T>::EPT;
+    constexpr int ITER = kSegment / (32 * EPT);  // 8 (fp32) or 4 (bf16)
+    constexpr int LPW = 32 / EPT;                // lanes that share one bitmap word
+    __shared__ __align__(16) int8_t stage[kThreads / 32][kSegment];
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long nseg = (n + kSegment - 1) / kSegment;
+    const long long nwarps = static_cast<long long>(gridDim.x) * (kThreads / 32);
+    const float delta = *delta_p;
+    const bool live = (delta > 0.f) && (delta < __int_as_float(0x7f800000));
+    const float inv = live ? __fdiv_rn(1.0f, delta) : 0.f;
+    const int sub = lane % LPW;                  // my position inside the word
+    const unsigned below = (1u << (EPT * sub)) - 1u;
+    unsigned long long nnz_local = 0ull;
+    unsigned sat = 0;
+
+    for (long long seg = static_cast<long long>(blockIdx.x) * (kThreads / 32) + warp; seg < nseg; seg += nwarps) {
+        unsigned running = 0, my_word = 0, my_off = 0;
+#pragma unroll
+        for (int it = 0; it < ITER; ++it) {
+            const long long e0 = seg * kSegment + it * (32 * EPT) + lane * EPT;
+            float v[EPT];
+            if (e0 + EPT <= n) {
+                Elem<T>::load(x + e0, v);
+            } else {
+#pragma unroll
+                for (int j = 0; j < EPT; ++j) v[j] = (e0 + j < n) ? Elem<T>::one(x + e0 + j) : 0.f;
+            }
+            int q[EPT];
+            unsigned bits = 0;
+            unsigned long long z = seed + (static_cast<unsigned long long>(e0 >> 1) + 1ull) * 0x9E3779B97F4A7C15ull;
+#pragma unroll
+            for (int j = 0; j < EPT; j += 2) {
+                const unsigned long long r = splitmix64_mix(z);
+                z += 0x9E3779B97F4A7C15ull;
+                q[j] = live ? quantize_one(v[j], inv, dither_from_bits(static_cast<unsigned>(r)), sat) : 0;
+                q[j + 1] = live ? quantize_one(v[j + 1], inv, dither_from_bits(static_cast<unsigned>(r >> 32)), sat) : 0;
+                if (e0 + j >= n) q[j] = 0;
+                if (e0 + j + 1 >= n) q[j + 1] = 0;
+                bits |= (q[j] != 0 ? 1u : 0u) << j;
+                bits |= (q[j + 1] != 0 ? 1u : 0u) << (j + 1);
+            }
+            // bitmap word shared by LPW consecutive lanes
+            unsigned word = bits << (EPT * sub);
+#pragma unroll
+            for (int o = 1; o < LPW; o <<= 1) word |= __shfl_xor_sync(kFull, word, o);
+            const unsigned pc = __popc(word);
+            // exclusive prefix over the EPT words of this iteration
+            unsigned before = 0, total = 0;
+            const int my_w = lane / LPW;
+#pragma unroll
+            for (int w = 0; w < EPT; ++w) {
+                const unsigned c = __shfl_sync(kFull, pc, w * LPW);
+                before += (w < my_w) ? c : 0u;
+                total += c;
+            }
+            const unsigned word_off = running + before;
+            unsigned rank = word_off + __popc(word & below);
+#pragma unroll
+            for (int j = 0; j < EPT; ++j)
+                if (q[j] != 0) stage[warp][rank++] = static_cast<int8_t>(q[j]);
+            if (dense != nullptr) {
+                if (e0 + EPT <= n) {
+                    unsigned pk[EPT / 4];
+#pragma unroll
+                    for (int j = 0; j < EPT; j += 4)
+                        pk[j / 4] = (q[j] & 0xff) | ((q[j + 1] & 0xff) << 8) | ((q[j + 2] & 0xff) << 16) |
+                                    (static_cast<unsigned>(q[j + 3] & 0xff) << 24);
+                    if (EPT == 4) *reinterpret_cast<unsigned *>(dense + e0) = pk[0];
+                    else *reinterpret_cast<uint2 *>(dense + e0) = make_uint2(pk[0], pk[EPT / 4 - 1]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < EPT; ++j)
+                        if (e0 + j < n) dense[e0 + j] = static_cast<int8_t>(q[j]);
+                }
+            }
+            // lane (it*EPT + w) keeps word w of this iteration and its offset
+            const unsigned wv = __shfl_sync(kFull, word, (lane % EPT) * LPW);
+            const unsigned ov = __shfl_sync(kFull, word_off, (lane % EPT) * LPW);
+            if (lane / EPT == it) { my_word = wv; my_off = ov; }
+            running += total;
+        }
+        __syncwarp();
+        bitmap[seg * kWordsPerSegment + lane] = my_word;
+        offsets[seg * kWordsPerSegment + lane] = static_cast<uint16_t>(my_off);
+        for (unsigned i = lane * 16; i < running; i += 512)
+            *reinterpret_cast<uint4 *>(values + seg * kSegment + i) =
+                *reinterpret_cast<const uint4 *>(&stage[warp][i]);
+        __syncwarp();
+        nnz_local += running;
+    }
+    sat = __reduce_add_sync(kFull, sat);
+    if (lane == 0) {
+        if (nnz_local) {
+            atomicAdd(&st->nnz, nnz_local);
+            if (nnz_out) atomicAdd(nnz_out, nnz_local);
+        }
+        if (sat) atomicAdd(&st->saturated, static_cast<unsigned long long>(sat));
+    }
+}
+
+// One warp per segment, one lane per bitmap word: 32 codes written as two 128-bit stores.
+__global__ void __launch_bounds__(kThreads)
+decode_kernel(const uint32_t *__restrict__ bitmap, const uint16_t *__restrict__ offsets,
+              const int8_t *__restrict__ values, long long n, int8_t *__restrict__ dense) {
+    const int lane = threadIdx.x & 31;
+    const long long nseg = (n + kSegment - 1) / kSegment;
+    const long long nwarps = static_cast<long long>(gridDim.x) * (kThreads / 32);
+    for (long long seg = static_cast<long long>(blockIdx.x) * (kThreads / 32) + (threadIdx.x >> 5); seg < nseg; seg += nwarps) {
+        const long long w = seg * kWordsPerSegment + lane;
+        unsigned word = bitmap[w];
+        const int8_t *src = values + seg * kSegment + offsets[w];
+        unsigned pk[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        while (word) {
+            const int b = __ffs(word) - 1;
+            word &= word - 1;
+            pk[b >> 2] |= (static_cast<unsigned>(*src++) & 0xffu) << (8 * (b & 3));
+        }
+        const long long e0 = w * 32;
+        if (e0 + 32 <= n) {
+            uint4 *dst = reinterpret_cast<uint4 *>(dense + e0);
+            dst[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            dst[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+        } else {
+            for (int j = 0; j < 32; ++j)
+                if (e0 + j < n) dense[e0 + j] = static_cast<int8_t>((pk[j >> 2] >> (8 * (j & 3))) & 0xff);
+        }
+    }
+}
+
+}  // namespace
+
+int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long numel, float scale,
+                      const float *delta_in, float *delta_out, unsigned long long *nnz_out) {
+    if (!(scale > 0.f)) {
+        set_step_kernel<<<1, 1, 0, ctx->stream>>>(delta_in, ctx->state, delta_out, nnz_out);
+        return cuda_ok(cudaGetLastError());
+    }
+    const int ept = dtype == DBP_F32 ? 4 : 8;
+    long long blocks = (numel / ept + kThreads * 4 - 1) / (kThreads * 4);
+    if (blocks < 1) blocks = 1;
+    if (blocks > ctx->partial_blocks) blocks = ctx->partial_blocks;
+    if (dtype == DBP_F32)
+        statistics_kernel<float><<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(
+            static_cast<const float *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out);
+    else
+        statistics_kernel<__nv_bfloat16><<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(
+            static_cast<const __nv_bfloat16 *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out);
+    return cuda_ok(cudaGetLastError());
+}
+
+int launch_quantize(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
+                    unsigned long long seed, const float *delta_p, uint32_t *bitmap,
+                    uint16_t *offsets, int8_t *values, int8_t *dense,
+                    unsigned long long *nnz_out) {
+    const long long nseg = (numel + kSegment - 1) / kSegment;
+    long long blocks = (nseg + kThreads / 32 - 1) / (kThreads / 32);
+    const long long cap = static_cast<long long>(ctx->sm_count) * 8;
+    if (blocks > cap) blocks = cap;
+    if (dtype == DBP_F32)
+        quantize_kernel<float><<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(
+            static_cast<const float *>(delta), numel, seed, delta_p, bitmap, offsets, values, dense,
+            ctx->state, nnz_out);
+    else
+        quantize_kernel<__nv_bfloat16><<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(
+            static_cast<const __nv_bfloat16 *>(delta), numel, seed, delta_p, bitmap, offsets, values,
+            dense, ctx->state, nnz_out);
+    return cuda_ok(cudaGetLastError());
+}
+
+int launch_decode(dbp_ctx *ctx, const uint32_t *bitmap, const uint16_t *offsets,
+                  const int8_t *values, long long numel, int8_t *dense) {
+    const long long nseg = (numel + kSegment - 1) / kSegment;
+    long long blocks = (nseg + kThreads / 32 - 1) / (kThreads / 32);
+    const long long cap = static_cast<long long>(ctx->sm_count) * 8;
+    if (blocks > cap) blocks = cap;
+    decode_kernel<<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(bitmap, offsets, values,
+                                                                            numel, dense);
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace dbp
