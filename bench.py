@@ -1,0 +1,386 @@
+#!/usr/bin/env python
+"""Benchmark of the dithered-backprop hot path on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--config 5|3|1] [--impl reference]
+
+One *step* is one pass of the whole path (statistics -> NSD quantize/compact -> dX -> dW)
+over every layer of the workload, on seeded synthetic inputs already resident in HBM.
+The metric is dense-equivalent backward throughput: the FLOPs a dense backward of the same
+layers would do (2 per MAC, both products) divided by the measured time.
+
+Default workload (config 5): the ResNet-50 ImageNet-shaped bottleneck layer set, batch 64,
+bf16 storage with fp32 accumulation, Delta = 5 std(delta) (about 90 % zeros after NSD).
+With N > 1 every rank runs the same layer set on its own batch shard (weak scaling; the
+path has no data-path exchange between ranks).
+
+`--impl reference` times the CPU oracle (the plain fp64 definition used for parity checks)
+on a bounded sample of the same workload, on the host cores.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+METRIC = "dithered backward dense-equiv GFLOP/s and % HBM roofline vs cuBLAS dense"
+UNIT = "GFLOP/s (dense-equivalent, dW+dX)"
+FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # fp32 FMA lanes x 2 flop x max SM clock
+
+
+def measured_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+# ------------------------------------------------------------------ workloads
+
+def layer_specs(config, batch):
+    """[(Layer factory, multiplicity)] in network order."""
+    if config == 1:
+        return [(lambda: wl.config1(batch or 128), 1)], "config1: linear 784->300, B128, fp32, s=2"
+    if config == 3:
+        return [(lambda: wl.config3(batch or 128), 1)], "config3: conv3x3 64->64 @32x32, B128, fp32, s=2"
+    if config == 5:
+        b = batch or 64
+        specs = [((lambda i=i: wl.config5_layer(i, batch=b)), wl.RESNET50_SET[i][5])
+                 for i in range(len(wl.RESNET50_SET))]
+        return specs, f"config5: ResNet-50 bottleneck layer set (48 convs, 16 shapes), B{b}, bf16, s=5"
+    raise SystemExit("--config must be 1, 3 or 5")
+
+
+def algorithmic_bytes(L):
+    """Bytes one layer's backward must move at least: delta read twice (statistics, then
+    quantize), sparse structure written once and read by both products, X and W read, dX and
+    dW written."""
+    e = 2 if L.dtype == "bf16" else 4
+    nd, nx, nw = L.delta.size, L.X.size, L.W.size
+    return 2 * nd * e + nx * e + nw * e + nx * e + nw * 4
+
+
+# ------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm = [float(r[0]) for r in self.rows if r and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for j, n in enumerate(names)
+                   if any(len(r) > 3 + j and r[3 + j].lower().startswith("active") for r in self.rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": reasons,
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------ CPU oracle arm
+
+def oracle_sample(config, budget_s=20.0):
+    """Times the oracle (NSD + fp64 products, as it stands) on a bounded sample of the
+    workload; returns (dense-equivalent GFLOP/s, seconds, description, threads)."""
+    import oracle
+    if config == 1:
+        layers, what = [wl.config1()], "the whole layer (B128)"
+    elif config == 3:
+        layers, what = [wl.config3(batch=8)], "batch 8 of 128"
+    else:
+        idx = [2, 6, 10, 14, 1, 15]
+        layers = [wl.config5_layer(i, batch=2) for i in idx]
+        what = "batch 2 of 64 of shapes " + ",".join(wl.RESNET50_SET[i][0] for i in idx)
+    t0 = time.perf_counter()
+    flops = 0.0
+    for L in layers:
+        D = oracle.step_size(L.delta, L.scale)
+        codes, _, _ = oracle.nsd_codes(L.delta, L.seed, D)
+        fn = oracle.linear_backward if L.kind == "linear" else oracle.conv_backward
+        fn(codes, D, L.X, L.W)
+        flops += L.dense_flops
+        if time.perf_counter() - t0 > budget_s:
+            break
+    dt = time.perf_counter() - t0
+    try:
+        cores = len(os.sched_getaffinity(0))
+    except Exception:
+        cores = os.cpu_count()
+    return flops / dt / 1e9, dt, what, cores
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    _, name = layer_specs(args.config, args.batch)
+    for _ in range(max(0, min(args.warmup, 1))):
+        oracle_sample(args.config, budget_s=2.0)
+    t0 = time.perf_counter()
+    vals = []
+    for _ in range(args.steps):
+        v, dt, what, cores = oracle_sample(args.config, budget_s=12.0)
+        vals.append(v)
+    total = time.perf_counter() - t0
+    v = float(np.mean(vals))
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": total / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": name, "sample": what},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------ CUDA arm
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=5)
+    ap.add_argument("--batch", type=int, default=0, help="override the config's batch size")
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--no-dense", action="store_true", help="skip the cuDNN/cuBLAS dense comparison")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl != "reference":
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    import paper_2004_04729_b200 as dbp
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    ctx = dbp.Context(local)
+
+    specs, name = layer_specs(args.config, args.batch)
+    tdt = lambda L: torch.bfloat16 if L.dtype == "bf16" else torch.float32
+    layers = []          # one entry per layer instance: (Layer, delta, X, W, dW, dX)
+    hosts = []           # one entry per distinct shape: pinned host tensors
+    dense_flops = alg_bytes = 0.0
+    for make, mult in specs:
+        L = make()
+        hd, hX, hW = (torch.from_numpy(a).to(tdt(L)).pin_memory() for a in (L.delta, L.X, L.W))
+        hosts.append((L, mult, hd, hX, hW,
+                      torch.empty(L.W.shape, dtype=torch.float32).pin_memory(),
+                      torch.empty(L.X.shape, dtype=tdt(L)).pin_memory()))
+        for _ in range(mult):
+            d, X, W = hd.to(dev), hX.to(dev), hW.to(dev)
+            layers.append((L, d, X, W,
+                           torch.empty(L.W.shape, dtype=torch.float32, device=dev),
+                           torch.empty(L.X.shape, dtype=tdt(L), device=dev)))
+            dense_flops += L.dense_flops
+            alg_bytes += algorithmic_bytes(L)
+    lib = dbp.load_library()
+    import ctypes
+
+    def run_layer(L, d, X, W, dW, dX):
+        code = 1 if L.dtype == "bf16" else 0
+        if L.kind == "linear":
+            B, N = d.shape
+            rc = lib.dithered_linear_backward(ctx._h, d.data_ptr(), X.data_ptr(), W.data_ptr(), code,
+                                              B, N, X.shape[1], L.seed, L.scale, None, None,
+                                              dW.data_ptr(), dX.data_ptr(), None, 0)
+        else:
+            B, Co, H, Wd = d.shape
+            rc = lib.dithered_conv_backward(ctx._h, d.data_ptr(), X.data_ptr(), W.data_ptr(), code,
+                                            B, X.shape[1], Co, H, Wd, L.k, 1, (L.k - 1) // 2, L.seed,
+                                            L.scale, None, None, dW.data_ptr(), dX.data_ptr(), None, 0)
+        if rc != 0:
+            raise RuntimeError(f"library call failed on {L.name}: {rc}")
+
+    def step():
+        for item in layers:
+            run_layer(*item)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    ctx.profile_enable(True)
+    ctx.profile_read()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms = e0.elapsed_time(e1) / args.steps
+    prof = ctx.profile_read()
+    ctx.profile_enable(False)
+    if world > 1:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = t.item()
+    value = dense_flops * world / (ms * 1e-3) / 1e9
+
+    # non-zero work actually done (for the arithmetic roofline of the sparse products)
+    nnz_flops = 0.0
+    for (L, d, X, W, dW, dX) in layers:
+        q = dbp.nsd_quantize(ctx, d, L.seed, L.scale)
+        nnz_flops += (q.nnz.item() / d.numel()) * L.dense_flops
+    torch.cuda.synchronize()
+    density = nnz_flops / dense_flops
+
+    # ---- end to end through the host entry points (H2D + kernels + D2H every step)
+    e2e = None
+    if not args.no_e2e:
+        h2d = d2h = 0
+        def host_step():
+            for (L, mult, hd, hX, hW, odW, odX) in hosts:
+                fn = dbp.dithered_linear_backward_host if L.kind == "linear" else dbp.dithered_conv_backward_host
+                for _ in range(mult):
+                    fn(ctx, hd, hX, hW, L.seed, L.scale, odW, odX)
+        for (L, mult, hd, hX, hW, odW, odX) in hosts:
+            h2d += mult * (hd.numel() * hd.element_size() + hX.numel() * hX.element_size() + hW.numel() * hW.element_size())
+            d2h += mult * (odW.numel() * 4 + odX.numel() * odX.element_size())
+        host_step()
+        ksteps = max(1, min(args.steps, 3))
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(ksteps):
+            host_step()
+        barrier()
+        dt = (time.perf_counter() - t0) / ksteps
+        if world > 1:
+            t = torch.tensor([dt], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = t.item()
+        e2e = {"value": dense_flops * world / dt / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": dt * 1e3, "steps": ksteps}
+
+    # ---- dense library backward on the same shapes (context, not the product path)
+    dense = None
+    if not args.no_dense and rank == 0:
+        import torch.nn.functional as F
+        def dense_step(allow_tf32):
+            torch.backends.cudnn.allow_tf32 = allow_tf32
+            torch.backends.cuda.matmul.allow_tf32 = allow_tf32
+            for (L, d, X, W, dW, dX) in layers:
+                if L.kind == "linear":
+                    torch.matmul(d.t(), X)
+                    torch.matmul(d, W)
+                else:
+                    p = (L.k - 1) // 2
+                    torch.ops.aten.convolution_backward(d, X, W, None, [1, 1], [p, p], [1, 1], False,
+                                                        [0, 0], 1, [True, True, False])
+        dense = {}
+        for label, tf32 in (("tf32_off", False), ("tf32_on", True)):
+            for _ in range(3):
+                dense_step(tf32)
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(max(3, args.steps // 2)):
+                dense_step(tf32)
+            b.record()
+            torch.cuda.synchronize()
+            dms = a.elapsed_time(b) / max(3, args.steps // 2)
+            dense[label] = {"ms_per_step": dms, "gflops": dense_flops / (dms * 1e-3) / 1e9}
+        dense["what"] = "torch cuDNN/cuBLAS backward-data + backward-filter on the unquantized delta, same buffers"
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    hbm_peak, peak_src = measured_peaks()
+    kern = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps}
+            for k, v in prof.items() if v[1]}
+    top = max(("dx", "dw", "quantize", "statistics"), key=lambda k: prof[k][0])
+    launches = sum(v[1] for v in prof.values())
+    if top in ("dx", "dw"):
+        per_launch_ms = prof[top][0] / prof[top][1]
+        flops_per_launch = nnz_flops / 2 / len(layers)
+        ach = flops_per_launch / (per_launch_ms * 1e-3) / 1e12
+        roof = {"kernel": f"conv_{top}_kernel", "bound": "alu", "achieved": ach, "peak": FMA_PEAK_TFLOPS,
+                "unit": "TFLOP/s", "frac": ach / FMA_PEAK_TFLOPS, "traffic": None,
+                "peak_source": "148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
+                "note": "non-zero-code FMAs only (2*nnz*K_eff flops per product), mean over layers"}
+    else:
+        e = 2 if layers[0][0].dtype == "bf16" else 4
+        nd = sum(l[1].numel() for l in layers)
+        per = (e + (0.1875 + density + 1.0)) if top == "quantize" else e
+        ach = nd * per / (prof[top][0] / args.steps * 1e-3) / 1e9
+        roof = {"kernel": f"{top}_kernel", "bound": "hbm", "achieved": ach, "peak": hbm_peak, "unit": "GB/s",
+                "frac": ach / hbm_peak, "traffic": None, "peak_source": peak_src}
+    path_gbs = alg_bytes / (ms * 1e-3) / 1e9
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 storage, f32 accumulate" if layers[0][0].dtype == "bf16" else "f32",
+        "data": "synthetic",
+        "config": {"workload": name, "layers_per_step": len(layers), "l2": "inputs larger than L2 (distinct buffers per layer instance)"
+                   if alg_bytes > 2.5e8 else "working set smaller than L2 (warm)", "nsd_density": density},
+        "clocks": clocks, "gpu_launches": launches, "e2e": e2e,
+        "roofline": roof,
+        "hbm_path": {"algorithmic_gb_per_step": alg_bytes / 1e9, "achieved_gbs": path_gbs,
+                     "frac_of_measured_hbm": path_gbs / hbm_peak, "peak": hbm_peak, "peak_source": peak_src},
+        "kernels": kern, "dense_baseline": dense,
+    }
+    if not args.no_cpu and world == 1:
+        v, dt, what, cores = oracle_sample(args.config)
+        out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what,
+                               "seconds": dt}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -89,6 +89,27 @@ const char *dbp_status_string(int status);
  * codes; both outputs may be NULL. Clears the record. */
 int dbp_last_device_status(dbp_ctx *ctx, int *status, long long *saturated);
 
+/*
+ * Per-kernel device timing (a measurement aid, off by default). While enabled, every kernel
+ * the library launches is bracketed by CUDA events on the context's stream.
+ * dbp_profile_read synchronises the stream and returns, for one kernel kind, the summed
+ * device time in milliseconds and the number of launches since the previous read of that
+ * kind (either output may be NULL).
+ */
+typedef enum {
+    DBP_K_STATISTICS = 0, /* sigma / Delta reduction */
+    DBP_K_QUANTIZE = 1,   /* dither + quantize + compact */
+    DBP_K_WEIGHT_TAPS = 2,/* weight re-layout for dX */
+    DBP_K_DX = 3,         /* sparse input-gradient product */
+    DBP_K_DW = 4,         /* sparse weight-gradient product */
+    DBP_K_DB = 5,         /* bias gradient */
+    DBP_K_DECODE = 6,     /* sparse -> dense codes */
+    DBP_K_GLUE = 7,       /* ReLU derivative / max-pool routing */
+    DBP_K_COUNT = 8
+} dbp_kernel_kind;
+int dbp_profile_enable(dbp_ctx *ctx, int on);
+int dbp_profile_read(dbp_ctx *ctx, int kind, double *milliseconds, long long *launches);
+
 /* Bytes the caller must allocate for each array of a dbp_sparse over `numel` elements. */
 int dbp_sparse_bytes(long long numel, size_t *bitmap_bytes, size_t *offsets_bytes,
                      size_t *values_bytes);

@@ -20,7 +20,10 @@ EXPORTED_SYMBOLS = [
     "dbp_last_device_status", "dbp_sparse_bytes", "nsd_quantize", "nsd_decode_dense",
     "dithered_linear_backward", "dithered_conv_backward", "dithered_linear_backward_host",
     "dithered_conv_backward_host", "dbp_relu_backward", "dbp_maxpool2x2_backward",
+    "dbp_profile_enable", "dbp_profile_read",
 ]
+
+KERNEL_KINDS = ["statistics", "quantize", "weight_taps", "dx", "dw", "db", "decode", "glue"]
 
 
 class DbpError(RuntimeError):
@@ -72,6 +75,8 @@ def load_library():
     lib.dithered_conv_backward_host.argtypes = [vp, vp, vp, vp, i32, ll, ll, ll, ll, ll, i32, i32,
                                                 i32, ull, f32, vp, vp, vp, u32,
                                                 ctypes.POINTER(f32), ctypes.POINTER(ll)]
+    lib.dbp_profile_enable.argtypes = [vp, i32]
+    lib.dbp_profile_read.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ll)]
     lib.dbp_relu_backward.argtypes = [vp, vp, vp, vp, ll]
     lib.dbp_maxpool2x2_backward.argtypes = [vp, vp, vp, vp, ll, ll, ll]
     for name in EXPORTED_SYMBOLS:
@@ -134,6 +139,19 @@ class Context:
         _check(load_library().dbp_last_device_status(self._h, ctypes.byref(st), ctypes.byref(sat)),
                "dbp_last_device_status")
         return st.value, sat.value
+
+    def profile_enable(self, on: bool = True):
+        _check(load_library().dbp_profile_enable(self._h, int(bool(on))), "dbp_profile_enable")
+
+    def profile_read(self):
+        """{kernel kind: (milliseconds, launches)} since the previous read."""
+        out = {}
+        for i, name in enumerate(KERNEL_KINDS):
+            ms, n = ctypes.c_double(), ctypes.c_longlong()
+            _check(load_library().dbp_profile_read(self._h, i, ctypes.byref(ms), ctypes.byref(n)),
+                   "dbp_profile_read")
+            out[name] = (ms.value, n.value)
+        return out
 
     def close(self):
         if getattr(self, "_h", None) is not None and self._h.value:

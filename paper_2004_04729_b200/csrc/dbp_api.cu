@@ -67,12 +67,18 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
     }
     if ((rc = ws_reserve(ctx, ctx->dense_codes, static_cast<size_t>(numel) + 16))) return rc;
     int8_t *dense = static_cast<int8_t *>(ctx->dense_codes.ptr);
-    if ((rc = launch_statistics(ctx, delta, dtype, numel, scale, delta_in, sp.delta,
-                                reinterpret_cast<unsigned long long *>(sp.nnz))))
-        return rc;
-    if ((rc = launch_quantize(ctx, delta, dtype, numel, seed, &ctx->state->delta, sp.bitmap, sp.offsets,
-                              sp.values, dense, reinterpret_cast<unsigned long long *>(sp.nnz))))
-        return rc;
+    {
+        KernelTimer t(ctx, DBP_K_STATISTICS);
+        rc = launch_statistics(ctx, delta, dtype, numel, scale, delta_in, sp.delta,
+                               reinterpret_cast<unsigned long long *>(sp.nnz));
+    }
+    if (rc) return rc;
+    {
+        KernelTimer t(ctx, DBP_K_QUANTIZE);
+        rc = launch_quantize(ctx, delta, dtype, numel, seed, &ctx->state->delta, sp.bitmap, sp.offsets,
+                             sp.values, dense, reinterpret_cast<unsigned long long *>(sp.nnz));
+    }
+    if (rc) return rc;
     *delta_p = &ctx->state->delta;
     *codes = dense;
     return DBP_OK;
@@ -102,12 +108,28 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
         const size_t wb = sizeof(float) * static_cast<size_t>(s.Cout) * s.Cin * s.k * s.k;
         if ((rc = ws_reserve(ctx, ctx->w_taps, wb))) return rc;
         float *wt = static_cast<float *>(ctx->w_taps.ptr);
-        if ((rc = launch_weight_taps(ctx, W, io, s, wt))) return rc;
+        {
+            KernelTimer t(ctx, DBP_K_WEIGHT_TAPS);
+            rc = launch_weight_taps(ctx, W, io, s, wt);
+        }
+        if (rc) return rc;
         const bool dx_bf16 = (io == DBP_BF16) && !(flags & DBP_DX_F32);
-        if ((rc = launch_conv_dx(ctx, codes, wt, delta_p, s, dX, dx_bf16))) return rc;
+        {
+            KernelTimer t(ctx, DBP_K_DX);
+            rc = launch_conv_dx(ctx, codes, wt, delta_p, s, dX, dx_bf16);
+        }
+        if (rc) return rc;
     }
-    if (dW && (rc = launch_conv_dw(ctx, codes, X, io, delta_p, s, dW))) return rc;
-    if (db && (rc = launch_bias_grad(ctx, codes, delta_p, s, db))) return rc;
+    if (dW) {
+        KernelTimer t(ctx, DBP_K_DW);
+        rc = launch_conv_dw(ctx, codes, X, io, delta_p, s, dW);
+        if (rc) return rc;
+    }
+    if (db) {
+        KernelTimer t(ctx, DBP_K_DB);
+        rc = launch_bias_grad(ctx, codes, delta_p, s, db);
+        if (rc) return rc;
+    }
     return DBP_OK;
 }
 
@@ -153,6 +175,7 @@ int dbp_destroy(dbp_ctx *ctx) {
     Workspace *all[] = {&ctx->dense_codes, &ctx->w_taps, &ctx->sp_bitmap, &ctx->sp_offsets, &ctx->sp_values};
     for (Workspace *w : all) if (w->ptr) cudaFree(w->ptr);
     for (Workspace &w : ctx->io) if (w.ptr) cudaFree(w.ptr);
+    for (ProfSlot &p : ctx->prof) { cudaEventDestroy(p.begin); cudaEventDestroy(p.end); }
     if (ctx->state) cudaFree(ctx->state);
     if (ctx->partials) cudaFree(ctx->partials);
     delete ctx;
@@ -196,6 +219,33 @@ int dbp_last_device_status(dbp_ctx *ctx, int *status, long long *saturated) {
     return DBP_OK;
 }
 
+int dbp_profile_enable(dbp_ctx *ctx, int on) {
+    if (!ctx) return DBP_EINVAL;
+    ctx->profiling = on != 0;
+    return DBP_OK;
+}
+
+int dbp_profile_read(dbp_ctx *ctx, int kind, double *milliseconds, long long *launches) {
+    if (!ctx || kind < 0 || kind >= DBP_K_COUNT) return DBP_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return DBP_ECUDA;
+    for (size_t i = 0; i < ctx->prof_used; ++i) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, ctx->prof[i].begin, ctx->prof[i].end) != cudaSuccess) {
+            cudaGetLastError();
+            continue;
+        }
+        ctx->prof_ms[ctx->prof[i].kind] += ms;
+        ctx->prof_launches[ctx->prof[i].kind] += 1;
+    }
+    ctx->prof_used = 0;
+    if (milliseconds) *milliseconds = ctx->prof_ms[kind];
+    if (launches) *launches = ctx->prof_launches[kind];
+    ctx->prof_ms[kind] = 0.0;
+    ctx->prof_launches[kind] = 0;
+    return DBP_OK;
+}
+
 int dbp_sparse_bytes(long long numel, size_t *bitmap_bytes, size_t *offsets_bytes, size_t *values_bytes) {
     if (numel <= 0) return DBP_EINVAL;
     const size_t nseg = (static_cast<size_t>(numel) + kSegment - 1) / kSegment;
@@ -216,9 +266,14 @@ int nsd_quantize(dbp_ctx *ctx, const void *delta, int dtype, long long numel, un
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DBP_ECUDA;
     out->numel = numel;
-    int rc = launch_statistics(ctx, delta, dtype, numel, scale, delta_in, out->delta,
+    int rc;
+    {
+        KernelTimer t(ctx, DBP_K_STATISTICS);
+        rc = launch_statistics(ctx, delta, dtype, numel, scale, delta_in, out->delta,
                                reinterpret_cast<unsigned long long *>(out->nnz));
+    }
     if (rc) return rc;
+    KernelTimer t(ctx, DBP_K_QUANTIZE);
     return launch_quantize(ctx, delta, dtype, numel, seed, &ctx->state->delta, out->bitmap, out->offsets,
                            out->values, nullptr, reinterpret_cast<unsigned long long *>(out->nnz));
 }
@@ -228,6 +283,7 @@ int nsd_decode_dense(dbp_ctx *ctx, const dbp_sparse *q, int8_t *codes) {
     if (!aligned16(codes)) return DBP_EINVAL;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DBP_ECUDA;
+    KernelTimer t(ctx, DBP_K_DECODE);
     return launch_decode(ctx, q->bitmap, q->offsets, q->values, q->numel, codes);
 }
 
@@ -312,6 +368,7 @@ int dbp_relu_backward(dbp_ctx *ctx, const float *delta_a, const uint8_t *mask, f
     if (!ctx || !delta_a || !mask || !delta_z || numel <= 0) return DBP_EINVAL;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DBP_ECUDA;
+    KernelTimer t(ctx, DBP_K_GLUE);
     return launch_relu_backward(ctx, delta_a, mask, delta_z, numel);
 }
 
@@ -320,6 +377,7 @@ int dbp_maxpool2x2_backward(dbp_ctx *ctx, const float *g, const int8_t *argmax, 
     if (!ctx || !g || !argmax || !out || planes <= 0 || h <= 0 || w <= 0) return DBP_EINVAL;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DBP_ECUDA;
+    KernelTimer t(ctx, DBP_K_GLUE);
     return launch_maxpool_backward(ctx, g, argmax, out, planes, h, w);
 }
 

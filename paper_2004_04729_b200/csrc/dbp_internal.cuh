@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "dbp.h"
 
 namespace dbp {
@@ -20,6 +22,11 @@ struct DeviceState {
     int pad0;
     unsigned long long nnz;             // non-zero codes of the internal quantization
     unsigned long long saturated;       // clipped codes since the last report
+};
+
+struct ProfSlot {
+    cudaEvent_t begin, end;
+    int kind;
 };
 
 struct Workspace {
@@ -40,6 +47,11 @@ struct dbp_ctx {
     dbp::Workspace w_taps;              // fp32 weights as [Cout][k*k][Cin]
     dbp::Workspace sp_bitmap, sp_offsets, sp_values;  // internal dbp_sparse
     dbp::Workspace io[8];               // staging for the *_host entry points
+    bool profiling = false;
+    std::vector<dbp::ProfSlot> prof;    // event pairs, reused after every read
+    size_t prof_used = 0;
+    double prof_ms[DBP_K_COUNT] = {0};
+    long long prof_launches[DBP_K_COUNT] = {0};
 };
 
 namespace dbp {
@@ -72,6 +84,28 @@ int launch_relu_backward(dbp_ctx *ctx, const float *da, const uint8_t *mask, flo
                          long long n);
 int launch_maxpool_backward(dbp_ctx *ctx, const float *g, const int8_t *argmax, float *out,
                             long long planes, long long h, long long w);
+
+// Brackets one kernel launch with events while profiling is on.
+struct KernelTimer {
+    dbp_ctx *ctx;
+    ProfSlot *slot = nullptr;
+    KernelTimer(dbp_ctx *c, int kind) : ctx(c) {
+        if (!c->profiling) return;
+        if (c->prof_used == c->prof.size()) {
+            ProfSlot s;
+            if (cudaEventCreate(&s.begin) != cudaSuccess) return;
+            if (cudaEventCreate(&s.end) != cudaSuccess) { cudaEventDestroy(s.begin); return; }
+            s.kind = kind;
+            c->prof.push_back(s);
+        }
+        slot = &c->prof[c->prof_used++];
+        slot->kind = kind;
+        cudaEventRecord(slot->begin, c->stream);
+    }
+    ~KernelTimer() {
+        if (slot) cudaEventRecord(slot->end, ctx->stream);
+    }
+};
 
 inline int cuda_ok(cudaError_t e) { return e == cudaSuccess ? DBP_OK : DBP_ECUDA; }
 
