@@ -107,22 +107,26 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     if (dX) {
         const size_t wb = sizeof(float) * static_cast<size_t>(s.Cout) * s.Cin * s.k * s.k;
         if ((rc = ws_reserve(ctx, ctx->w_taps, wb))) return rc;
-        float *wt = static_cast<float *>(ctx->w_taps.ptr);
+        void *wt = ctx->w_taps.ptr;
+        const bool dx_bf16 = (io == DBP_BF16) && !(flags & DBP_DX_F32);
+        // streamed kernel: weight rows must be 16-byte multiples; otherwise the generic one
+        const bool streamed = (s.Cin * static_cast<long long>(elem_size(io))) % 16 == 0;
         {
             KernelTimer t(ctx, DBP_K_WEIGHT_TAPS);
-            rc = launch_weight_taps(ctx, W, io, s, wt);
+            rc = launch_weight_taps(ctx, W, io, s, wt, !streamed);
         }
         if (rc) return rc;
-        const bool dx_bf16 = (io == DBP_BF16) && !(flags & DBP_DX_F32);
         {
             KernelTimer t(ctx, DBP_K_DX);
-            rc = launch_conv_dx(ctx, codes, wt, delta_p, s, dX, dx_bf16);
+            rc = streamed ? launch_conv_dx_streamed(ctx, codes, wt, io, delta_p, s, dX, dx_bf16)
+                          : launch_conv_dx(ctx, codes, static_cast<const float *>(wt), delta_p, s, dX, dx_bf16);
         }
         if (rc) return rc;
     }
     if (dW) {
         KernelTimer t(ctx, DBP_K_DW);
-        rc = launch_conv_dw(ctx, codes, X, io, delta_p, s, dW);
+        rc = launch_conv_dw_streamed(ctx, codes, X, io, delta_p, s, dW);
+        if (rc == DBP_EUNSUPPORTED) rc = launch_conv_dw(ctx, codes, X, io, delta_p, s, dW);
         if (rc) return rc;
     }
     if (db) {

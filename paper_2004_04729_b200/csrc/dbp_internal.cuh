@@ -73,11 +73,17 @@ struct ConvShape {
     long long B, Cin, Cout, H, W;
     int k;
 };
-int launch_weight_taps(dbp_ctx *ctx, const void *W, int dtype, const ConvShape &s, float *w_taps);
+// weights as [Cout][k*k][Cin]; kept in their own dtype unless to_f32
+int launch_weight_taps(dbp_ctx *ctx, const void *W, int dtype, const ConvShape &s, void *w_taps,
+                       bool to_f32);
+int launch_conv_dx_streamed(dbp_ctx *ctx, const int8_t *codes, const void *w_taps, int w_dtype,
+                            const float *delta_p, const ConvShape &s, void *dX, bool dx_bf16);
 int launch_conv_dx(dbp_ctx *ctx, const int8_t *codes, const float *w_taps, const float *delta_p,
                    const ConvShape &s, void *dX, bool dx_bf16);
 int launch_conv_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, int dtype,
                    const float *delta_p, const ConvShape &s, float *dW);
+int launch_conv_dw_streamed(dbp_ctx *ctx, const int8_t *codes, const void *X, int dtype,
+                            const float *delta_p, const ConvShape &s, float *dW);
 int launch_bias_grad(dbp_ctx *ctx, const int8_t *codes, const float *delta_p, const ConvShape &s,
                      float *db);
 int launch_relu_backward(dbp_ctx *ctx, const float *da, const uint8_t *mask, float *dz,

@@ -16,8 +16,11 @@ __device__ __forceinline__ float to_f32(float v) { return v; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
 
 // ------------------------------------------------------------------ weights as [Cout][tap][Cin]
-template <typename T>
-__global__ void weight_taps_kernel(const T *__restrict__ W, float *__restrict__ out, long long Cout,
+__device__ __forceinline__ void store_as(float *p, float v) { *p = v; }
+__device__ __forceinline__ void store_as(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
+
+template <typename T, typename O>
+__global__ void weight_taps_kernel(const T *__restrict__ W, O *__restrict__ out, long long Cout,
                                    long long Cin, int KK) {
     const long long n = Cout * Cin * KK;
     for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < n;
@@ -25,7 +28,7 @@ __global__ void weight_taps_kernel(const T *__restrict__ W, float *__restrict__ 
         const long long ci = i % Cin;
         const long long t = (i / Cin) % KK;
         const long long co = i / (Cin * KK);
-        out[i] = to_f32(W[(co * Cin + ci) * KK + t]);
+        store_as(out + i, to_f32(W[(co * Cin + ci) * KK + t]));
     }
 }
 
@@ -348,14 +351,20 @@ int blocks_for(long long n, int threads, int cap) {
 
 }  // namespace
 
-int launch_weight_taps(dbp_ctx *ctx, const void *W, int dtype, const ConvShape &s, float *w_taps) {
+int launch_weight_taps(dbp_ctx *ctx, const void *W, int dtype, const ConvShape &s, void *w_taps,
+                       bool to_f32) {
     const int KK = s.k * s.k;
     const long long n = s.Cout * s.Cin * KK;
     const int blocks = blocks_for(n, 256, ctx->sm_count * 8);
     if (dtype == DBP_F32)
-        weight_taps_kernel<float><<<blocks, 256, 0, ctx->stream>>>(static_cast<const float *>(W), w_taps, s.Cout, s.Cin, KK);
+        weight_taps_kernel<float, float><<<blocks, 256, 0, ctx->stream>>>(
+            static_cast<const float *>(W), static_cast<float *>(w_taps), s.Cout, s.Cin, KK);
+    else if (to_f32)
+        weight_taps_kernel<__nv_bfloat16, float><<<blocks, 256, 0, ctx->stream>>>(
+            static_cast<const __nv_bfloat16 *>(W), static_cast<float *>(w_taps), s.Cout, s.Cin, KK);
     else
-        weight_taps_kernel<__nv_bfloat16><<<blocks, 256, 0, ctx->stream>>>(static_cast<const __nv_bfloat16 *>(W), w_taps, s.Cout, s.Cin, KK);
+        weight_taps_kernel<__nv_bfloat16, __nv_bfloat16><<<blocks, 256, 0, ctx->stream>>>(
+            static_cast<const __nv_bfloat16 *>(W), static_cast<__nv_bfloat16 *>(w_taps), s.Cout, s.Cin, KK);
     return cuda_ok(cudaGetLastError());
 }
 
