@@ -42,13 +42,25 @@ typedef enum {
     DBP_ENOMEM = -4,        /* workspace allocation failed */
     DBP_ENONFINITE = -5,    /* device: delta holds NaN or Inf (all codes were set to 0) */
     DBP_ESATURATED = -6,    /* device: some codes were clipped to +-127 */
-    DBP_ECAPACITY = -7      /* a caller-provided size is smaller than required */
+    DBP_ECAPACITY = -7,     /* a caller-provided size is smaller than required */
+    DBP_ETIMEOUT = -8       /* device: a bounded wait inside a kernel expired (results undefined) */
 } dbp_status;
 
 /* flags for the backward calls */
 #define DBP_FORCE_SPARSE 1u /* always use the sparse gather kernels */
-#define DBP_FORCE_DENSE  2u /* always use the dense tensor-core path (where it exists) */
+#define DBP_FORCE_DENSE  2u /* always use the dense tensor-core path; DBP_EUNSUPPORTED where it
+                               does not exist (it covers bf16 linear and 1x1 layers, Cin % 8 == 0) */
 #define DBP_DX_F32       4u /* with io = DBP_BF16: write dX as fp32 instead of bf16 */
+
+/*
+ * Density crossover (Section 3.4: the sparse products cost O(p_nz m k n), a dense product
+ * O(m k n) at a much higher arithmetic rate on tensor cores). Without a FORCE flag a layer
+ * that the dense path supports uses it when the context's estimate of p_nz exceeds
+ * `crossover`; the estimate is the density measured by the context's most recent finished
+ * quantization (read back asynchronously, so no call waits for it; 1.0 before the first).
+ * crossover >= 1 disables the dense path, crossover <= 0 always prefers it.
+ */
+int dbp_set_crossover(dbp_ctx *ctx, float crossover);
 
 /* Elements per segment of the sparse structure (see dbp_sparse). */
 #define DBP_SEGMENT 1024

@@ -20,7 +20,7 @@ EXPORTED_SYMBOLS = [
     "dbp_last_device_status", "dbp_sparse_bytes", "nsd_quantize", "nsd_decode_dense",
     "dithered_linear_backward", "dithered_conv_backward", "dithered_linear_backward_host",
     "dithered_conv_backward_host", "dbp_relu_backward", "dbp_maxpool2x2_backward",
-    "dbp_profile_enable", "dbp_profile_read",
+    "dbp_profile_enable", "dbp_profile_read", "dbp_set_crossover",
 ]
 
 KERNEL_KINDS = ["statistics", "quantize", "weight_taps", "dx", "dw", "db", "decode", "glue"]
@@ -75,6 +75,7 @@ def load_library():
     lib.dithered_conv_backward_host.argtypes = [vp, vp, vp, vp, i32, ll, ll, ll, ll, ll, i32, i32,
                                                 i32, ull, f32, vp, vp, vp, u32,
                                                 ctypes.POINTER(f32), ctypes.POINTER(ll)]
+    lib.dbp_set_crossover.argtypes = [vp, f32]
     lib.dbp_profile_enable.argtypes = [vp, i32]
     lib.dbp_profile_read.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ll)]
     lib.dbp_relu_backward.argtypes = [vp, vp, vp, vp, ll]
@@ -139,6 +140,10 @@ class Context:
         _check(load_library().dbp_last_device_status(self._h, ctypes.byref(st), ctypes.byref(sat)),
                "dbp_last_device_status")
         return st.value, sat.value
+
+    def set_crossover(self, crossover: float):
+        """Density above which layers the dense tensor-core path supports use it."""
+        _check(load_library().dbp_set_crossover(self._h, float(crossover)), "dbp_set_crossover")
 
     def profile_enable(self, on: bool = True):
         _check(load_library().dbp_profile_enable(self._h, int(bool(on))), "dbp_profile_enable")

@@ -96,14 +96,50 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     if ((dW && !X) || (dX && !W)) return DBP_EINVAL;
     if (!aligned16(delta) || !aligned16(X) || !aligned16(W) || !aligned16(dW) || !aligned16(dX)) return DBP_EINVAL;
     if ((flags & DBP_FORCE_SPARSE) && (flags & DBP_FORCE_DENSE)) return DBP_EINVAL;
-    if (flags & DBP_FORCE_DENSE) return DBP_EUNSUPPORTED;   // no dense tensor-core path yet
+    const bool can_dense = tc_supported(s, io);
+    if ((flags & DBP_FORCE_DENSE) && !can_dense) return DBP_EUNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DBP_ECUDA;
     const long long numel = s.B * s.Cout * s.H * s.W;
     const float *delta_p = nullptr;
     const int8_t *codes = nullptr;
+    // pick up the density of the last finished quantization, if its read-back has landed
+    if (ctx->nnz_pending && cudaEventQuery(ctx->nnz_event) == cudaSuccess) {
+        ctx->density_estimate = static_cast<float>(static_cast<double>(*ctx->nnz_host) /
+                                                   static_cast<double>(ctx->nnz_host_numel));
+        ctx->nnz_pending = false;
+    }
+    cudaGetLastError();   // cudaErrorNotReady from the query is not an error
+    const bool dense = can_dense && !(flags & DBP_FORCE_SPARSE) &&
+                       ((flags & DBP_FORCE_DENSE) || ctx->density_estimate > ctx->crossover);
     int rc = quantize_for_products(ctx, delta, io, numel, seed, scale, delta_in, q_out, &delta_p, &codes);
     if (rc) return rc;
+    if (!ctx->nnz_pending && ctx->nnz_host && ctx->nnz_event) {
+        ctx->nnz_host_numel = numel;
+        if (cudaMemcpyAsync(ctx->nnz_host, &ctx->state->nnz, sizeof(unsigned long long), cudaMemcpyDeviceToHost,
+                            ctx->stream) == cudaSuccess &&
+            cudaEventRecord(ctx->nnz_event, ctx->stream) == cudaSuccess)
+            ctx->nnz_pending = true;
+    }
+    if (dense) {
+        if (dX) {
+            KernelTimer t(ctx, DBP_K_DX);
+            rc = launch_tc_dx(ctx, codes, W, delta_p, s, dX, (io == DBP_BF16) && !(flags & DBP_DX_F32),
+                              &ctx->state->tc_timeout);
+            if (rc) return rc;
+        }
+        if (dW) {
+            KernelTimer t(ctx, DBP_K_DW);
+            rc = launch_tc_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout);
+            if (rc) return rc;
+        }
+        if (db) {
+            KernelTimer t(ctx, DBP_K_DB);
+            rc = launch_bias_grad(ctx, codes, delta_p, s, db);
+            if (rc) return rc;
+        }
+        return DBP_OK;
+    }
     if (dX) {
         const size_t wb = sizeof(float) * static_cast<size_t>(s.Cout) * s.Cin * s.k * s.k;
         if ((rc = ws_reserve(ctx, ctx->w_taps, wb))) return rc;
@@ -168,7 +204,19 @@ int dbp_create(dbp_ctx **out, int device, void *cuda_stream) {
         dbp_destroy(ctx);
         return DBP_ENOMEM;
     }
+    if (cudaMallocHost(&ctx->nnz_host, sizeof(unsigned long long)) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->nnz_event, cudaEventDisableTiming) != cudaSuccess) {
+        cudaGetLastError();
+        dbp_destroy(ctx);
+        return DBP_ENOMEM;
+    }
     *out = ctx;
+    return DBP_OK;
+}
+
+int dbp_set_crossover(dbp_ctx *ctx, float crossover) {
+    if (!ctx || crossover != crossover) return DBP_EINVAL;
+    ctx->crossover = crossover;
     return DBP_OK;
 }
 
@@ -180,6 +228,8 @@ int dbp_destroy(dbp_ctx *ctx) {
     for (Workspace *w : all) if (w->ptr) cudaFree(w->ptr);
     for (Workspace &w : ctx->io) if (w.ptr) cudaFree(w.ptr);
     for (ProfSlot &p : ctx->prof) { cudaEventDestroy(p.begin); cudaEventDestroy(p.end); }
+    if (ctx->nnz_host) cudaFreeHost(ctx->nnz_host);
+    if (ctx->nnz_event) cudaEventDestroy(ctx->nnz_event);
     if (ctx->state) cudaFree(ctx->state);
     if (ctx->partials) cudaFree(ctx->partials);
     delete ctx;
@@ -202,6 +252,7 @@ const char *dbp_status_string(int status) {
         case DBP_ENONFINITE: return "non-finite value in delta";
         case DBP_ESATURATED: return "codes clipped to +-127";
         case DBP_ECAPACITY: return "buffer too small";
+        case DBP_ETIMEOUT: return "bounded device wait expired";
         default: return "unknown status";
     }
 }
@@ -213,10 +264,12 @@ int dbp_last_device_status(dbp_ctx *ctx, int *status, long long *saturated) {
     if (cudaMemcpyAsync(&h, ctx->state, sizeof(h), cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess ||
         cudaStreamSynchronize(ctx->stream) != cudaSuccess)
         return DBP_ECUDA;
-    if (status) *status = h.nonfinite ? DBP_ENONFINITE : (h.saturated ? DBP_ESATURATED : DBP_OK);
+    if (status)
+        *status = h.tc_timeout ? DBP_ETIMEOUT : h.nonfinite ? DBP_ENONFINITE : (h.saturated ? DBP_ESATURATED : DBP_OK);
     if (saturated) *saturated = static_cast<long long>(h.saturated);
-    if (h.nonfinite || h.saturated) {
+    if (h.nonfinite || h.saturated || h.tc_timeout) {
         if (cudaMemsetAsync(&ctx->state->nonfinite, 0, sizeof(int), ctx->stream) != cudaSuccess ||
+            cudaMemsetAsync(&ctx->state->tc_timeout, 0, sizeof(int), ctx->stream) != cudaSuccess ||
             cudaMemsetAsync(&ctx->state->saturated, 0, sizeof(unsigned long long), ctx->stream) != cudaSuccess)
             return DBP_ECUDA;
     }

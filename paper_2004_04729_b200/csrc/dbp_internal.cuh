@@ -19,7 +19,7 @@ struct DeviceState {
     float delta;                        // step size of the internal quantization
     int nonfinite;                      // set when delta_z held NaN/Inf
     unsigned int ticket;                // last-block election of the statistics kernel
-    int pad0;
+    int tc_timeout;                     // a bounded wait of a tensor-core kernel expired
     unsigned long long nnz;             // non-zero codes of the internal quantization
     unsigned long long saturated;       // clipped codes since the last report
 };
@@ -47,6 +47,12 @@ struct dbp_ctx {
     dbp::Workspace w_taps;              // fp32 weights as [Cout][k*k][Cin]
     dbp::Workspace sp_bitmap, sp_offsets, sp_values;  // internal dbp_sparse
     dbp::Workspace io[8];               // staging for the *_host entry points
+    float crossover = 0.03f;            // density above which the dense path is preferred
+    float density_estimate = 1.0f;      // density of the latest finished quantization
+    unsigned long long *nnz_host = nullptr;   // pinned: asynchronous read-back of nnz
+    long long nnz_host_numel = 0;
+    cudaEvent_t nnz_event = nullptr;
+    bool nnz_pending = false;
     bool profiling = false;
     std::vector<dbp::ProfSlot> prof;    // event pairs, reused after every read
     size_t prof_used = 0;
@@ -84,6 +90,12 @@ int launch_conv_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, int dtype,
                    const float *delta_p, const ConvShape &s, float *dW);
 int launch_conv_dw_streamed(dbp_ctx *ctx, const int8_t *codes, const void *X, int dtype,
                             const float *delta_p, const ConvShape &s, float *dW);
+// ---- tc_dense.cu
+bool tc_supported(const ConvShape &s, int io);
+int launch_tc_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *delta_p,
+                 const ConvShape &s, float *dW, int *err_flag);
+int launch_tc_dx(dbp_ctx *ctx, const int8_t *codes, const void *W, const float *delta_p,
+                 const ConvShape &s, void *dX, bool dx_bf16, int *err_flag);
 int launch_bias_grad(dbp_ctx *ctx, const int8_t *codes, const float *delta_p, const ConvShape &s,
                      float *db);
 int launch_relu_backward(dbp_ctx *ctx, const float *da, const uint8_t *mask, float *dz,

@@ -1,0 +1,115 @@
+"""The dense tensor-core path (bf16 linear / 1x1 layers) against the CPU oracle, and the
+density crossover that chooses between it and the sparse kernels. Same bars as the sparse
+path: codes bit-exact, dW and dX within 1e-5 (relative Frobenius and |err| <= 1e-5 sum|terms|);
+products of bf16 values are exact in fp32, only the accumulation order differs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as wl
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    import paper_2004_04729_b200 as dbp
+    c = dbp.Context(0)
+    yield c
+    c.close()
+
+
+def _t(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda().to(torch.bfloat16)
+
+
+def _run(ctx, L, flags):
+    import paper_2004_04729_b200 as dbp
+    d, X, W = _t(L.delta), _t(L.X), _t(L.W)
+    q = dbp.SparseGradient(d.numel())
+    fn = dbp.dithered_linear_backward if L.kind == "linear" else dbp.dithered_conv_backward
+    out = fn(ctx, d, X, W, L.seed, L.scale, q_out=q, need_db=True, flags=flags | dbp.DBP_DX_F32)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == (0, 0)
+    D = np.float32(q.delta.item())
+    codes, nnz, _ = oracle.nsd_codes(L.delta, L.seed, D)
+    assert np.array_equal(dbp.nsd_decode_dense(ctx, q).cpu().numpy().reshape(codes.shape), codes)
+    ofn = oracle.linear_backward if L.kind == "linear" else oracle.conv_backward
+    ref = ofn(codes, D, L.X, L.W, with_abs=True)
+    for key in ("dW", "dX", "db"):
+        got = out[key].double().cpu().numpy()
+        fro = np.linalg.norm(got - ref[key]) / max(np.linalg.norm(ref[key]), 1e-300)
+        assert fro <= TOL, (key, fro)
+        bound = TOL * ref["S_" + key] + 1e-30
+        assert np.all(np.abs(got - ref[key]) <= bound), (key, float((np.abs(got - ref[key]) / bound).max()))
+    return out
+
+
+@pytest.mark.parametrize("B,Ci,Co,H,W", [
+    (2, 64, 64, 16, 16),      # one k-stage, narrow N tile
+    (1, 256, 64, 56, 56),     # ResNet stage-1 reduce, positions % 8 == 0
+    (2, 64, 256, 28, 28),     # expand: K = 256 output channels over four stages for dX
+    (3, 512, 128, 14, 14),    # 196 positions per image: 4-element groups
+    (5, 128, 512, 7, 7),      # 49 positions per image: element-wise loads, ragged row tiles
+    (2, 72, 40, 5, 9),        # channel counts that fill neither tile
+    (1, 1024, 256, 14, 14),
+])
+def test_dense_path_conv1x1(ctx, B, Ci, Co, H, W):
+    import paper_2004_04729_b200 as dbp
+    L = wl.conv_layer(B, Ci, Co, H, W, 1, data_seed=B + Ci + Co, scale=5.0, dtype="bf16")
+    _run(ctx, L, dbp.DBP_FORCE_DENSE)
+
+
+@pytest.mark.parametrize("B,N,K", [(128, 300, 784), (256, 512, 2048), (70, 10, 512), (33, 100, 304)])
+def test_dense_path_linear(ctx, B, N, K):
+    import paper_2004_04729_b200 as dbp
+    L = wl.linear_layer(B, N, K, data_seed=N + K, scale=2.0, dtype="bf16")
+    if K % 8:
+        pytest.skip("dense path needs Cin % 8 == 0")
+    _run(ctx, L, dbp.DBP_FORCE_DENSE)
+
+
+def test_dense_and_sparse_paths_agree_and_unsupported_is_refused(ctx):
+    import paper_2004_04729_b200 as dbp
+    L = wl.conv_layer(2, 128, 128, 14, 14, 1, data_seed=3, scale=5.0, dtype="bf16")
+    a = _run(ctx, L, dbp.DBP_FORCE_DENSE)
+    b = _run(ctx, L, dbp.DBP_FORCE_SPARSE)
+    for key in ("dW", "dX"):
+        ref = b[key].double()
+        assert (a[key].double() - ref).norm() <= 2e-5 * ref.norm()
+    L3 = wl.conv_layer(1, 16, 16, 6, 6, 3, data_seed=4, dtype="bf16")
+    with pytest.raises(dbp.DbpError) as e:          # 3x3 has no dense path
+        dbp.dithered_conv_backward(ctx, _t(L3.delta), _t(L3.X), _t(L3.W), 0, 2.0, flags=dbp.DBP_FORCE_DENSE)
+    assert e.value.status == -2
+    Lf = wl.conv_layer(1, 16, 16, 6, 6, 1, data_seed=4)
+    with pytest.raises(dbp.DbpError) as e:          # fp32 operands have no dense path
+        dbp.dithered_conv_backward(ctx, torch.from_numpy(Lf.delta).cuda(), torch.from_numpy(Lf.X).cuda(),
+                                   torch.from_numpy(Lf.W).cuda(), 0, 2.0, flags=dbp.DBP_FORCE_DENSE)
+    assert e.value.status == -2
+
+
+def test_crossover_uses_the_measured_density(ctx):
+    """With crossover 0.5 a layer at ~10 % density switches to the sparse kernels once the
+    first call's density has been read back; with crossover 0 it stays dense. Both paths give
+    the same gradients, so only the kernel mix (profile counters) tells them apart."""
+    import paper_2004_04729_b200 as dbp
+    c2 = dbp.Context(0)
+    L = wl.conv_layer(2, 64, 64, 16, 16, 1, data_seed=9, scale=5.0, dtype="bf16")
+    d, X, W = _t(L.delta), _t(L.X), _t(L.W)
+    c2.set_crossover(0.5)
+    c2.profile_enable(True)
+    dbp.dithered_conv_backward(c2, d, X, W, 0, 5.0)          # estimate starts at 1.0 -> dense
+    torch.cuda.synchronize()
+    first = c2.profile_read()
+    assert first["weight_taps"][1] == 0
+    dbp.dithered_conv_backward(c2, d, X, W, 0, 5.0)          # now ~0.1 < 0.5 -> sparse
+    torch.cuda.synchronize()
+    second = c2.profile_read()
+    assert second["weight_taps"][1] == 1
+    c2.set_crossover(0.0)
+    dbp.dithered_conv_backward(c2, d, X, W, 0, 5.0)
+    torch.cuda.synchronize()
+    assert c2.profile_read()["weight_taps"][1] == 0
+    c2.close()

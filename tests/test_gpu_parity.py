@@ -146,7 +146,8 @@ def _layer_case(ctx, L, need_db=True, dx_f32=True):
     import paper_2004_04729_b200 as dbp
     d, X, W = _t(L.delta, L.dtype), _t(L.X, L.dtype), _t(L.W, L.dtype)
     q = dbp.SparseGradient(d.numel())
-    flags = dbp.DBP_DX_F32 if (L.dtype == "bf16" and dx_f32) else 0
+    # the sparse kernels are the subject here (the dense path has its own test file)
+    flags = dbp.DBP_FORCE_SPARSE | (dbp.DBP_DX_F32 if (L.dtype == "bf16" and dx_f32) else 0)
     fn = dbp.dithered_linear_backward if L.kind == "linear" else dbp.dithered_conv_backward
     out = fn(ctx, d, X, W, L.seed, L.scale, q_out=q, need_db=need_db, flags=flags)
     D = np.float32(q.delta.item())
