@@ -224,7 +224,8 @@ int dbp_destroy(dbp_ctx *ctx) {
     if (!ctx) return DBP_EINVAL;
     DeviceGuard guard(ctx->device);
     cudaStreamSynchronize(ctx->stream);
-    Workspace *all[] = {&ctx->dense_codes, &ctx->w_taps, &ctx->sp_bitmap, &ctx->sp_offsets, &ctx->sp_values};
+    Workspace *all[] = {&ctx->dense_codes, &ctx->w_taps, &ctx->sp_bitmap, &ctx->sp_offsets, &ctx->sp_values,
+                        &ctx->tc_partials};
     for (Workspace *w : all) if (w->ptr) cudaFree(w->ptr);
     for (Workspace &w : ctx->io) if (w.ptr) cudaFree(w.ptr);
     for (ProfSlot &p : ctx->prof) { cudaEventDestroy(p.begin); cudaEventDestroy(p.end); }

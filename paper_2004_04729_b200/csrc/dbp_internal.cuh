@@ -46,6 +46,7 @@ struct dbp_ctx {
     dbp::Workspace dense_codes;         // int8 per element of delta
     dbp::Workspace w_taps;              // fp32 weights as [Cout][k*k][Cin]
     dbp::Workspace sp_bitmap, sp_offsets, sp_values;  // internal dbp_sparse
+    dbp::Workspace tc_partials;         // split-K partial blocks of the dense dW kernel
     dbp::Workspace io[8];               // staging for the *_host entry points
     float crossover = 0.03f;            // density above which the dense path is preferred
     float density_estimate = 1.0f;      // density of the latest finished quantization

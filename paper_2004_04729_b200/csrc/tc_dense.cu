@@ -6,12 +6,13 @@
 //   dW[co][ci] = Delta * sum_r q[r,co] X[r,ci]      M = co, N = ci, K = rows r = (image, position)
 //   dX[r][ci]  = Delta * sum_co q[r,co] W[co,ci]    M = rows r,  N = ci, K = co
 //
-// Operands live in NCHW memory (positions contiguous), whose row pitch is in general not a
+// Operands live in NCHW memory (positions contiguous) whose row pitch is in general not a
 // multiple of 16 bytes and whose codes need conversion, so tiles are not fetched by TMA:
-// four producer warps load 8-element groups, convert, and store 16-byte chunks directly in
-// the 128-byte-swizzled canonical shared-memory layout that the MMA descriptors name. A fifth
-// warp issues the MMAs; mbarriers order producers, tensor core and epilogue. Every wait is
-// bounded: on expiry the kernel raises a flag in global memory and runs to its end.
+// four producer warps load 8-element groups (cp.async where no conversion is needed), convert,
+// and store 16-byte chunks directly in the 128-byte-swizzled canonical shared-memory layout
+// that the MMA descriptors name. A fifth warp issues the MMAs; mbarriers order producers,
+// tensor core and epilogue. Every wait is bounded: on expiry the kernel raises a flag in
+// global memory and runs to its end.
 #include "dbp_internal.cuh"
 
 namespace dbp {
@@ -19,10 +20,11 @@ namespace dbp {
 namespace {
 
 constexpr int kProducerWarps = 4;
-constexpr int kThreads = (kProducerWarps + 1) * 32;
-constexpr int kStages = 4;
-constexpr int kKT = 64;                     // K elements per stage (one 128-byte swizzled row)
-constexpr long long kWaitCycles = 1000000000ll;   // a wait gives up after this many SM clocks
+constexpr int kProducers = kProducerWarps * 32;
+constexpr int kThreads = kProducers + 32;
+constexpr int kMaxStages = 4;
+constexpr int kKT = 64;                             // K elements per stage (one 128-byte swizzled row)
+constexpr long long kWaitCycles = 1000000000ll;     // a wait gives up after this many SM clocks
 
 __device__ __forceinline__ unsigned smem_u32(const void *p) {
     return static_cast<unsigned>(__cvta_generic_to_shared(p));
@@ -32,6 +34,10 @@ __device__ __forceinline__ void mbar_init(unsigned long long *bar, int count) {
 }
 __device__ __forceinline__ void mbar_arrive(unsigned long long *bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// arrival that fires when this thread's earlier cp.async copies have landed
+__device__ __forceinline__ void mbar_arrive_on_cp_async(unsigned long long *bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 // Returns false when the phase did not complete within about half a second.
 __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity, int *err_flag) {
@@ -85,9 +91,13 @@ __device__ __forceinline__ void tmem_ld32(unsigned taddr, unsigned (&r)[32]) {
         : "r"(taddr));
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc, bool valid) {
+    const int n = valid ? 16 : 0;   // src-size 0: the 16 bytes are zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(n) : "memory");
+}
 
-// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1.
-// lbo/sbo in bytes. K-major operand: rows of 64 K-elements, 8-row groups sbo apart (lbo unused).
+// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1; lbo/sbo in bytes.
+// K-major operand: rows of 64 K-elements, 8-row groups sbo apart (lbo unused).
 // MN-major operand: rows (one per k) of 64 MN-elements, 8-row groups sbo apart, 64-element
 // MN groups lbo apart.
 __device__ __forceinline__ unsigned long long make_desc(unsigned smem_addr, unsigned lbo, unsigned sbo) {
@@ -105,160 +115,187 @@ __host__ __device__ constexpr unsigned make_idesc(int M, int N, bool a_mn_major,
            (static_cast<unsigned>(N >> 3) << 17) | (static_cast<unsigned>(M >> 4) << 24);
 }
 
-// ---- 8-element groups of a [image][channel][position] tensor along the flattened row index
-// r = image * P + position, for a fixed channel. `g` (1, 2, 4 or 8) divides P and the row
-// index of every group start, so a group never straddles two images and is g-element aligned.
-struct RowMap {
-    long long P;       // positions per image
-    long long C;       // channels of the tensor
-    long long rows;    // B * P
-    int g;
-};
-
-__device__ __forceinline__ uint4 load8_codes_as_bf16(const int8_t *codes, const RowMap &m, long long ch, long long r0) {
-    // eight consecutive rows r0..r0+7 of channel ch, int8 -> bf16 (exact)
-    unsigned short h[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) h[j] = 0;
-    if (m.g == 8) {
-        if (r0 < m.rows) {
-            const long long b = r0 / m.P, p = r0 - b * m.P;
-            const uint2 v = __ldg(reinterpret_cast<const uint2 *>(codes + (b * m.C + ch) * m.P + p));
-            const unsigned w[2] = {v.x, v.y};
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int c = static_cast<int8_t>((w[j >> 2] >> (8 * (j & 3))) & 0xff);
-                h[j] = __bfloat16_as_ushort(__int2bfloat16_rn(c));
-            }
-        }
-    } else {
-        for (int j0 = 0; j0 < 8; j0 += m.g) {
-            const long long r = r0 + j0;
-            if (r >= m.rows) break;
-            const long long b = r / m.P, p = r - b * m.P;
-            const int8_t *src = codes + (b * m.C + ch) * m.P + p;
-            for (int j = 0; j < m.g; ++j) h[j0 + j] = __bfloat16_as_ushort(__int2bfloat16_rn(static_cast<int>(__ldg(src + j))));
-        }
-    }
-    return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
-}
-
-__device__ __forceinline__ uint4 load8_bf16(const __nv_bfloat16 *x, const RowMap &m, long long ch, long long r0) {
-    if (m.g == 8) {
-        if (r0 >= m.rows) return make_uint4(0u, 0u, 0u, 0u);
-        const long long b = r0 / m.P, p = r0 - b * m.P;
-        return __ldg(reinterpret_cast<const uint4 *>(x + (b * m.C + ch) * m.P + p));
-    }
-    unsigned short h[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) h[j] = 0;
-    for (int j0 = 0; j0 < 8; j0 += m.g) {
-        const long long r = r0 + j0;
-        if (r >= m.rows) break;
-        const long long b = r / m.P, p = r - b * m.P;
-        const unsigned short *src = reinterpret_cast<const unsigned short *>(x + (b * m.C + ch) * m.P + p);
-        for (int j = 0; j < m.g; ++j) h[j0 + j] = __ldg(src + j);
-    }
-    return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
-}
-
 // byte offset of 16-byte chunk `chunk` (0..7) of row `row` inside a 128-byte-swizzled panel
 __device__ __forceinline__ unsigned swz(unsigned row, unsigned chunk) { return row * 128u + ((chunk ^ (row & 7u)) << 4); }
+
+// four int8 codes packed in a word -> two words of packed bf16 (exact).
+// byte ^ 0x80 = code + 128 as an unsigned byte; 0x4B0000xx read as a float is 2^23 + xx, so
+// subtracting 2^23 + 128 leaves the code as a float whose top 16 bits are its bf16 pattern.
+__device__ __forceinline__ void codes4_to_bf16(unsigned w, unsigned &lo, unsigned &hi) {
+    const unsigned x = w ^ 0x80808080u;
+    const float f0 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7650)) - 8388736.0f;
+    const float f1 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7651)) - 8388736.0f;
+    const float f2 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7652)) - 8388736.0f;
+    const float f3 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7653)) - 8388736.0f;
+    lo = __byte_perm(__float_as_uint(f0), __float_as_uint(f1), 0x7632);
+    hi = __byte_perm(__float_as_uint(f2), __float_as_uint(f3), 0x7632);
+}
+__device__ __forceinline__ unsigned short code_to_bf16(int c) {
+    return static_cast<unsigned short>(__float_as_uint(static_cast<float>(c)) >> 16);
+}
+
+// Row r of the flattened (image, position) index of a [B][C][P] tensor: walks eight consecutive
+// rows from (b, p) without divisions, for any P (P = 1 is a linear layer's [B][C] matrix).
+struct RowCursor {
+    long long b, p;
+    __device__ RowCursor(long long r, long long P) : b(r / P), p(r - (r / P) * P) {}
+};
+
+template <bool FAST>
+__device__ __forceinline__ uint4 load8_codes(const int8_t *codes, long long C, long long P, long long rows,
+                                             long long ch, long long r0, const RowCursor &cur) {
+    if (r0 >= rows) return make_uint4(0u, 0u, 0u, 0u);
+    if (FAST) {   // P % 8 == 0: the eight rows sit in one image, 8-byte aligned
+        const uint2 v = __ldg(reinterpret_cast<const uint2 *>(codes + (cur.b * C + ch) * P + cur.p));
+        uint4 o;
+        codes4_to_bf16(v.x, o.x, o.y);
+        codes4_to_bf16(v.y, o.z, o.w);
+        return o;
+    }
+    unsigned short h[8];
+    long long b = cur.b, pp = cur.p;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        h[j] = (r0 + j < rows) ? code_to_bf16(__ldg(codes + (b * C + ch) * P + pp)) : 0;
+        if (++pp == P) { pp = 0; ++b; }
+    }
+    return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+}
+
+__device__ __forceinline__ uint4 load8_bf16_slow(const __nv_bfloat16 *x, long long C, long long P, long long rows,
+                                                 long long ch, long long r0, const RowCursor &cur) {
+    if (r0 >= rows) return make_uint4(0u, 0u, 0u, 0u);
+    const unsigned short *src = reinterpret_cast<const unsigned short *>(x);
+    unsigned short h[8];
+    long long b = cur.b, pp = cur.p;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        h[j] = (r0 + j < rows) ? __ldg(src + (b * C + ch) * P + pp) : 0;
+        if (++pp == P) { pp = 0; ++b; }
+    }
+    return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+}
 
 struct TcParams {
     const int8_t *codes;          // [B][Cout][P]
     const __nv_bfloat16 *X;       // [B][Cin][P]      (dW)
     const __nv_bfloat16 *W;       // [Cout][Cin]      (dX)
     const float *delta_p;
-    float *dW;                    // [Cout][Cin]
+    float *partials;              // dW: [ksplit][Cout][Cin] partial sums (not yet scaled by Delta)
     void *dX;                     // [B][Cin][P], bf16 or fp32
     int dx_f32;
     int Cin, Cout;
     long long P, rows;
-    int g;                        // group size for row-wise loads
+    int stages;
     int ksplit;                   // dW: CTAs sharing one output tile
     long long kstages;            // dW: 64-row stages in total
+    long long per_split;          // dW: stages per CTA
     int *err_flag;
 };
 
 struct Pipe {
-    unsigned long long full[kStages], empty[kStages], acc;
+    unsigned long long full[kMaxStages], empty[kMaxStages], acc;
     unsigned tmem_base;
 };
 
+__device__ __forceinline__ void pipe_setup(Pipe &pipe, int stages, int full_count, int warp, int ncols) {
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) { mbar_init(&pipe.full[s], full_count); mbar_init(&pipe.empty[s], 1); }
+        mbar_init(&pipe.acc, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kProducerWarps) tmem_alloc(&pipe.tmem_base, ncols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+}
+
 // ---------------------------------------------------------------- dW: M = co, N = ci, K = rows
-template <int NT>
+// Both operands K-major: 128 (co) and NT (ci) rows of 64 consecutive flattened rows r.
+template <int NT, bool FAST>
 __global__ void __launch_bounds__(kThreads) tc_dw_kernel(const TcParams p) {
-    constexpr int A_BYTES = 128 * 128;          // 128 co rows x 64 k
-    constexpr int B_BYTES = NT * 128;           // NT ci rows x 64 k
+    constexpr int A_BYTES = 128 * 128;
+    constexpr int B_BYTES = NT * 128;
     constexpr int STAGE = A_BYTES + B_BYTES;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ Pipe pipe;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int co0 = blockIdx.x * 128, ci0 = blockIdx.y * NT;
-    // my share of the K stages
-    const long long per = (p.kstages + p.ksplit - 1) / p.ksplit;
-    const long long ks0 = blockIdx.z * per;
-    long long ks1 = ks0 + per;
+    const long long ks0 = blockIdx.z * p.per_split;
+    long long ks1 = ks0 + p.per_split;
     if (ks1 > p.kstages) ks1 = p.kstages;
     const int niter = ks1 > ks0 ? static_cast<int>(ks1 - ks0) : 0;
+    const int stages = p.stages;
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(&pipe.full[s], kProducerWarps); mbar_init(&pipe.empty[s], 1); }
-        mbar_init(&pipe.acc, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == kProducerWarps) tmem_alloc(&pipe.tmem_base, NT);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
+    pipe_setup(pipe, stages, FAST ? 2 * kProducers : kProducers, warp, NT);
     const unsigned tmem_d = pipe.tmem_base;
 
     if (warp < kProducerWarps) {
-        // ---------------- producers: chunk (row, c8) with c8 = tid % 8 fixed for the thread
-        const RowMap mq{p.P, p.Cout, p.rows, p.g}, mx{p.P, p.Cin, p.rows, p.g};
-        const int tid = threadIdx.x;           // 0..127
-        const int c8 = tid & 7, rsub = tid >> 3;   // 16 rows per pass
+        // ---------------- producers: chunk (row, c8); c8 = tid % 8 is fixed for the thread
+        const int tid = threadIdx.x;
+        const int c8 = tid & 7, rsub = tid >> 3;
         bool ok = true;
         for (int it = 0; it < niter && ok; ++it) {
-            const int s = it % kStages;
-            ok = mbar_wait(&pipe.empty[s], ((it / kStages) & 1) ^ 1, p.err_flag);
+            const int s = it % stages;
+            ok = mbar_wait(&pipe.empty[s], ((it / stages) & 1) ^ 1, p.err_flag);
             unsigned char *a_s = smem + s * STAGE, *b_s = a_s + A_BYTES;
             const long long r0 = (ks0 + it) * kKT + c8 * 8;
+            const RowCursor cur(r0 < p.rows ? r0 : 0, p.P);
+            if (FAST) {   // X needs no conversion: asynchronous 16-byte copies
+                const bool row_ok = r0 < p.rows;
+                const __nv_bfloat16 *src = p.X + (cur.b * p.Cin + ci0) * p.P + cur.p;
 #pragma unroll 4
-            for (int row = rsub; row < 128; row += 16) {
-                const int co = co0 + row;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (co < p.Cout) v = load8_codes_as_bf16(p.codes, mq, co, r0);
-                *reinterpret_cast<uint4 *>(a_s + swz(row, c8)) = v;
+                for (int row = rsub; row < NT; row += 16) {
+                    const bool v = row_ok && (ci0 + row < p.Cin);
+                    cp_async16(b_s + swz(row, c8), v ? src + row * p.P : p.X, v);
+                }
+                mbar_arrive_on_cp_async(&pipe.full[s]);
             }
-#pragma unroll 4
-            for (int row = rsub; row < NT; row += 16) {
-                const int ci = ci0 + row;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (ci < p.Cin) v = load8_bf16(p.X, mx, ci, r0);
-                *reinterpret_cast<uint4 *>(b_s + swz(row, c8)) = v;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {     // 4 loads in flight, then 4 stores
+                uint4 v[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int row = rsub + 16 * (half * 4 + i);
+                    const int co = co0 + row;
+                    v[i] = (co < p.Cout) ? load8_codes<FAST>(p.codes, p.Cout, p.P, p.rows, co, r0, cur)
+                                         : make_uint4(0u, 0u, 0u, 0u);
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    *reinterpret_cast<uint4 *>(a_s + swz(rsub + 16 * (half * 4 + i), c8)) = v[i];
+            }
+            if (!FAST) {
+#pragma unroll 2
+                for (int row = rsub; row < NT; row += 16) {
+                    const int ci = ci0 + row;
+                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                    if (ci < p.Cin) v = load8_bf16_slow(p.X, p.Cin, p.P, p.rows, ci, r0, cur);
+                    *reinterpret_cast<uint4 *>(b_s + swz(row, c8)) = v;
+                }
             }
             fence_async_proxy();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&pipe.full[s]);
+            mbar_arrive(&pipe.full[s]);
         }
-        // ---------------- epilogue: lanes = co rows, columns = ci
+        // ---------------- epilogue: lanes = co rows, columns = ci -> partial block of this split
         if (niter > 0 && mbar_wait(&pipe.acc, 0, p.err_flag)) {
             tc_fence_after();
-            const float delta = *p.delta_p;
             const int co = co0 + warp * 32 + lane;
+            float *dst_row = p.partials + (static_cast<long long>(blockIdx.z) * p.Cout + co) * p.Cin + ci0;
 #pragma unroll 1
             for (int c0 = 0; c0 < NT; c0 += 32) {
                 unsigned r[32];
                 tmem_ld32(tmem_d + (static_cast<unsigned>(warp * 32) << 16) + c0, r);
                 if (co < p.Cout) {
-                    float *dst = p.dW + static_cast<long long>(co) * p.Cin + ci0 + c0;
+                    if (ci0 + c0 + 32 <= p.Cin) {   // Cin % 8 == 0 and ci0 % 64 == 0: 16-byte aligned
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const float v = __uint_as_float(r[j]) * delta;
-                        if (ci0 + c0 + j < p.Cin && v != 0.f) atomicAdd(dst + j, v);
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<uint4 *>(dst_row + c0 + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (ci0 + c0 + j < p.Cin) dst_row[c0 + j] = __uint_as_float(r[j]);
                     }
                 }
             }
@@ -268,8 +305,9 @@ __global__ void __launch_bounds__(kThreads) tc_dw_kernel(const TcParams p) {
         constexpr unsigned idesc = make_idesc(128, NT, false, false);
         bool ok = true;
         for (int it = 0; it < niter && ok; ++it) {
-            const int s = it % kStages;
-            ok = mbar_wait(&pipe.full[s], (it / kStages) & 1, p.err_flag);
+            const int s = it % stages;
+            ok = mbar_wait(&pipe.full[s], (it / stages) & 1, p.err_flag);
+            fence_async_proxy();
             tc_fence_after();
             const unsigned a_addr = smem_u32(smem + s * STAGE), b_addr = a_addr + A_BYTES;
             const unsigned long long ad = make_desc(a_addr, 16, 1024), bd = make_desc(b_addr, 16, 1024);
@@ -288,10 +326,26 @@ __global__ void __launch_bounds__(kThreads) tc_dw_kernel(const TcParams p) {
     }
 }
 
+// dW = Delta * sum over splits of the partial blocks
+__global__ void __launch_bounds__(256) tc_dw_reduce_kernel(const float *__restrict__ partials, int ksplit,
+                                                           long long n, const float *__restrict__ delta_p,
+                                                           float *__restrict__ dW) {
+    const float delta = *delta_p;
+    for (long long i = (blockIdx.x * 256ll + threadIdx.x) * 4; i < n; i += gridDim.x * 1024ll) {
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s = 0; s < ksplit; ++s) {
+            const float4 v = __ldcs(reinterpret_cast<const float4 *>(partials + s * n + i));
+            a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+        }
+        *reinterpret_cast<float4 *>(dW + i) = make_float4(a.x * delta, a.y * delta, a.z * delta, a.w * delta);
+    }
+}
+
 // ---------------------------------------------------------------- dX: M = rows, N = ci, K = co
-template <int NT>
+// Both operands MN-major: k-rows (co) of 64 consecutive flattened rows r (A) / 64 ci (B).
+template <int NT, bool FAST>
 __global__ void __launch_bounds__(kThreads) tc_dx_kernel(const TcParams p) {
-    constexpr int A_BYTES = 2 * kKT * 128;      // two 64-row MN groups x 64 k-rows of 128 bytes
+    constexpr int A_BYTES = 2 * kKT * 128;
     constexpr int B_BYTES = (NT / 64) * kKT * 128;
     constexpr int STAGE = A_BYTES + B_BYTES;
     constexpr unsigned PANEL = kKT * 128;       // bytes between 64-element MN groups
@@ -302,85 +356,118 @@ __global__ void __launch_bounds__(kThreads) tc_dx_kernel(const TcParams p) {
     const long long row0 = static_cast<long long>(blockIdx.x) * 128;
     const int ci0 = blockIdx.y * NT;
     const int niter = (p.Cout + kKT - 1) / kKT;
+    const int stages = p.stages;
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(&pipe.full[s], kProducerWarps); mbar_init(&pipe.empty[s], 1); }
-        mbar_init(&pipe.acc, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == kProducerWarps) tmem_alloc(&pipe.tmem_base, NT);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
+    pipe_setup(pipe, stages, 2 * kProducers, warp, NT);
     const unsigned tmem_d = pipe.tmem_base;
 
     if (warp < kProducerWarps) {
-        const RowMap mq{p.P, p.Cout, p.rows, p.g};
         const int tid = threadIdx.x;
         const int c8 = tid & 7, ksub = tid >> 3;    // 16 k-rows per pass
+        // my two 8-row groups of the tile never change
+        const long long ra = row0 + c8 * 8, rb = ra + 64;
+        const RowCursor cura(ra < p.rows ? ra : 0, p.P), curb(rb < p.rows ? rb : 0, p.P);
         bool ok = true;
         for (int it = 0; it < niter && ok; ++it) {
-            const int s = it % kStages;
-            ok = mbar_wait(&pipe.empty[s], ((it / kStages) & 1) ^ 1, p.err_flag);
+            const int s = it % stages;
+            ok = mbar_wait(&pipe.empty[s], ((it / stages) & 1) ^ 1, p.err_flag);
             unsigned char *a_s = smem + s * STAGE, *b_s = a_s + A_BYTES;
-            // A = codes: k-row = co, 64-element MN groups of flattened rows
-#pragma unroll 2
-            for (int k = ksub; k < kKT; k += 16) {
-                const int co = it * kKT + k;
+            // B = W[co][ci]: k-row = co, 64-element groups of ci; no conversion: cp.async
 #pragma unroll
-                for (int grp = 0; grp < 2; ++grp) {
-                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                    if (co < p.Cout) v = load8_codes_as_bf16(p.codes, mq, co, row0 + grp * 64 + c8 * 8);
-                    *reinterpret_cast<uint4 *>(a_s + grp * PANEL + swz(k, c8)) = v;
-                }
-            }
-            // B = W[co][ci]: k-row = co, 64-element groups of ci
-#pragma unroll 2
-            for (int k = ksub; k < kKT; k += 16) {
+            for (int i = 0; i < kKT / 16; ++i) {
+                const int k = ksub + 16 * i;
                 const int co = it * kKT + k;
 #pragma unroll
                 for (int grp = 0; grp < NT / 64; ++grp) {
                     const int ci = ci0 + grp * 64 + c8 * 8;
-                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                    if (co < p.Cout && ci < p.Cin)     // Cin % 8 == 0 is required by the launcher
-                        v = __ldg(reinterpret_cast<const uint4 *>(p.W + static_cast<long long>(co) * p.Cin + ci));
-                    *reinterpret_cast<uint4 *>(b_s + grp * PANEL + swz(k, c8)) = v;
+                    const bool v = co < p.Cout && ci < p.Cin;     // Cin % 8 == 0
+                    cp_async16(b_s + grp * PANEL + swz(k, c8), v ? p.W + static_cast<long long>(co) * p.Cin + ci : p.W, v);
                 }
             }
+            mbar_arrive_on_cp_async(&pipe.full[s]);
+            // A = codes: k-row = co, two 64-element groups of flattened rows
+            uint4 va[kKT / 16], vb[kKT / 16];
+#pragma unroll
+            for (int i = 0; i < kKT / 16; ++i) {
+                const int co = it * kKT + ksub + 16 * i;
+                va[i] = vb[i] = make_uint4(0u, 0u, 0u, 0u);
+                if (co < p.Cout) {
+                    va[i] = load8_codes<FAST>(p.codes, p.Cout, p.P, p.rows, co, ra, cura);
+                    vb[i] = load8_codes<FAST>(p.codes, p.Cout, p.P, p.rows, co, rb, curb);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < kKT / 16; ++i) {
+                const int k = ksub + 16 * i;
+                *reinterpret_cast<uint4 *>(a_s + swz(k, c8)) = va[i];
+                *reinterpret_cast<uint4 *>(a_s + PANEL + swz(k, c8)) = vb[i];
+            }
             fence_async_proxy();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&pipe.full[s]);
+            mbar_arrive(&pipe.full[s]);
         }
-        // ---------------- epilogue: lanes = rows (image, position), columns = ci
+        // ---------------- epilogue: lanes = rows (image, position), columns = ci.
+        // Each warp turns its 32 rows x 32 columns block through a private shared-memory patch so
+        // that a lane stores 16 contiguous bytes of one channel row.
         if (mbar_wait(&pipe.acc, 0, p.err_flag)) {
             tc_fence_after();
             const float delta = *p.delta_p;
-            const long long r = row0 + warp * 32 + lane;
-            const bool row_ok = r < p.rows;
-            const long long b = row_ok ? r / p.P : 0, pp = row_ok ? r - b * p.P : 0;
-            const long long base = b * p.Cin * p.P + pp;
+            // all MMAs are complete: the stage buffers are free
+            constexpr int CS = 192;                          // bytes per column of the patch
+            unsigned char *patch = smem + warp * (32 * CS);
+            const int es = p.dx_f32 ? 4 : 2;
+            const int rows_per_lane = 16 / es;               // rows in one 16-byte store
+            const int lanes_per_col = 32 / rows_per_lane;
+            const int cols_per_pass = 32 / lanes_per_col;
+            const int rr = (lane % lanes_per_col) * rows_per_lane;
+            const long long r = row0 + warp * 32 + rr;       // first of my rows when storing
+            const long long rb_ = r < p.rows ? r / p.P : 0, rp_ = r < p.rows ? r - rb_ * p.P : 0;
 #pragma unroll 1
             for (int c0 = 0; c0 < NT; c0 += 32) {
                 unsigned v[32];
                 tmem_ld32(tmem_d + (static_cast<unsigned>(warp * 32) << 16) + c0, v);
-                if (row_ok) {
+                if (ci0 + c0 >= p.Cin) break;               // warp-uniform
+                if (p.dx_f32) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int ci = ci0 + c0 + j;
-                        if (ci >= p.Cin) break;
-                        const float f = __uint_as_float(v[j]) * delta;
-                        if (p.dx_f32) static_cast<float *>(p.dX)[base + ci * p.P] = f;
-                        else static_cast<__nv_bfloat16 *>(p.dX)[base + ci * p.P] = __float2bfloat16_rn(f);
+                    for (int j = 0; j < 32; ++j)
+                        *reinterpret_cast<float *>(patch + j * CS + lane * 4) = __uint_as_float(v[j]) * delta;
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        *reinterpret_cast<unsigned short *>(patch + j * CS + lane * 2) =
+                            __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(v[j]) * delta));
+                }
+                __syncwarp();
+                for (int cb = 0; cb < 32; cb += cols_per_pass) {
+                    const int j = cb + lane / lanes_per_col;
+                    const int ci = ci0 + c0 + j;
+                    if (ci < p.Cin && r < p.rows) {
+                        const uint4 val = *reinterpret_cast<const uint4 *>(patch + j * CS + rr * es);
+                        if (FAST) {      // the group sits in one image, 16-byte aligned
+                            unsigned char *dst = static_cast<unsigned char *>(p.dX) + ((rb_ * p.Cin + ci) * p.P + rp_) * es;
+                            *reinterpret_cast<uint4 *>(dst) = val;
+                        } else {
+                            long long b = rb_, pp = rp_;
+                            const unsigned w4[4] = {val.x, val.y, val.z, val.w};
+                            for (int e = 0; e < rows_per_lane && r + e < p.rows; ++e) {
+                                const long long o = (b * p.Cin + ci) * p.P + pp;
+                                if (p.dx_f32) static_cast<float *>(p.dX)[o] = __uint_as_float(w4[e]);
+                                else static_cast<unsigned short *>(p.dX)[o] =
+                                    static_cast<unsigned short>((w4[e >> 1] >> (16 * (e & 1))) & 0xffff);
+                                if (++pp == p.P) { pp = 0; ++b; }
+                            }
+                        }
                     }
                 }
+                __syncwarp();
             }
         }
     } else if (lane == 0) {
         constexpr unsigned idesc = make_idesc(128, NT, true, true);
         bool ok = true;
         for (int it = 0; it < niter && ok; ++it) {
-            const int s = it % kStages;
-            ok = mbar_wait(&pipe.full[s], (it / kStages) & 1, p.err_flag);
+            const int s = it % stages;
+            ok = mbar_wait(&pipe.full[s], (it / stages) & 1, p.err_flag);
+            fence_async_proxy();
             tc_fence_after();
             const unsigned a_addr = smem_u32(smem + s * STAGE), b_addr = a_addr + A_BYTES;
             const unsigned long long ad = make_desc(a_addr, PANEL, 1024), bd = make_desc(b_addr, PANEL, 1024);
@@ -399,12 +486,25 @@ __global__ void __launch_bounds__(kThreads) tc_dx_kernel(const TcParams p) {
     }
 }
 
-int pick_group(long long P) { return P % 8 == 0 ? 8 : P % 4 == 0 ? 4 : P % 2 == 0 ? 2 : 1; }
-
 template <typename K>
 int set_smem(K kern, size_t bytes) {
     return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes)) == cudaSuccess
                ? DBP_OK : DBP_ECUDA;
+}
+
+template <int NT, bool FAST>
+int run_dw(dbp_ctx *ctx, const TcParams &p, dim3 grid, size_t smem) {
+    int rc = set_smem(tc_dw_kernel<NT, FAST>, smem);
+    if (rc) return rc;
+    tc_dw_kernel<NT, FAST><<<grid, kThreads, smem, ctx->stream>>>(p);
+    return cuda_ok(cudaGetLastError());
+}
+template <int NT, bool FAST>
+int run_dx(dbp_ctx *ctx, const TcParams &p, dim3 grid, size_t smem) {
+    int rc = set_smem(tc_dx_kernel<NT, FAST>, smem);
+    if (rc) return rc;
+    tc_dx_kernel<NT, FAST><<<grid, kThreads, smem, ctx->stream>>>(p);
+    return cuda_ok(cudaGetLastError());
 }
 
 }  // namespace
@@ -416,25 +516,38 @@ bool tc_supported(const ConvShape &s, int io) {
 int launch_tc_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *delta_p,
                  const ConvShape &s, float *dW, int *err_flag) {
     TcParams p{};
-    p.codes = codes; p.X = static_cast<const __nv_bfloat16 *>(X); p.delta_p = delta_p; p.dW = dW;
+    p.codes = codes; p.X = static_cast<const __nv_bfloat16 *>(X); p.delta_p = delta_p;
     p.Cin = static_cast<int>(s.Cin); p.Cout = static_cast<int>(s.Cout);
-    p.P = s.H * s.W; p.rows = s.B * p.P; p.g = pick_group(p.P);
+    p.P = s.H * s.W; p.rows = s.B * p.P;
     p.kstages = (p.rows + kKT - 1) / kKT;
     p.err_flag = err_flag;
-    if (cudaMemsetAsync(dW, 0, sizeof(float) * s.Cout * s.Cin, ctx->stream) != cudaSuccess) return DBP_ECUDA;
     const int nt = s.Cin >= 256 ? 256 : s.Cin > 64 ? 128 : 64;
     const long long tiles = ((s.Cout + 127) / 128) * ((s.Cin + nt - 1) / nt);
-    long long split = (2LL * ctx->sm_count + tiles - 1) / tiles;
+    // split K so that every SM has a CTA, without empty splits
+    long long split = (ctx->sm_count + tiles - 1) / tiles;
     if (split > p.kstages) split = p.kstages;
     if (split < 1) split = 1;
+    p.per_split = (p.kstages + split - 1) / split;
+    split = (p.kstages + p.per_split - 1) / p.per_split;
     p.ksplit = static_cast<int>(split);
+    p.stages = p.per_split < kMaxStages ? static_cast<int>(p.per_split) : kMaxStages;
+    const size_t nw = static_cast<size_t>(s.Cout) * s.Cin;
+    int rc = ws_reserve(ctx, ctx->tc_partials, sizeof(float) * nw * split);
+    if (rc) return rc;
+    p.partials = static_cast<float *>(ctx->tc_partials.ptr);
     dim3 grid(static_cast<unsigned>((s.Cout + 127) / 128), static_cast<unsigned>((s.Cin + nt - 1) / nt),
               static_cast<unsigned>(split));
-    const size_t smem = static_cast<size_t>(kStages) * (128 * 128 + nt * 128) + 1024;
-    int rc;
-    if (nt == 256) { if ((rc = set_smem(tc_dw_kernel<256>, smem))) return rc; tc_dw_kernel<256><<<grid, kThreads, smem, ctx->stream>>>(p); }
-    else if (nt == 128) { if ((rc = set_smem(tc_dw_kernel<128>, smem))) return rc; tc_dw_kernel<128><<<grid, kThreads, smem, ctx->stream>>>(p); }
-    else { if ((rc = set_smem(tc_dw_kernel<64>, smem))) return rc; tc_dw_kernel<64><<<grid, kThreads, smem, ctx->stream>>>(p); }
+    const size_t smem = static_cast<size_t>(p.stages) * (128 * 128 + nt * 128) + 1024;
+    const bool fast = p.P % 8 == 0;
+    if (nt == 256) rc = fast ? run_dw<256, true>(ctx, p, grid, smem) : run_dw<256, false>(ctx, p, grid, smem);
+    else if (nt == 128) rc = fast ? run_dw<128, true>(ctx, p, grid, smem) : run_dw<128, false>(ctx, p, grid, smem);
+    else rc = fast ? run_dw<64, true>(ctx, p, grid, smem) : run_dw<64, false>(ctx, p, grid, smem);
+    if (rc) return rc;
+    long long blocks = (static_cast<long long>(nw) / 4 + 255) / 256;
+    if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
+    if (blocks < 1) blocks = 1;
+    tc_dw_reduce_kernel<<<static_cast<unsigned>(blocks), 256, 0, ctx->stream>>>(
+        p.partials, p.ksplit, static_cast<long long>(nw), delta_p, dW);   // Cout*Cin % 4 == 0 since Cin % 8 == 0
     return cuda_ok(cudaGetLastError());
 }
 
@@ -444,16 +557,20 @@ int launch_tc_dx(dbp_ctx *ctx, const int8_t *codes, const void *W, const float *
     p.codes = codes; p.W = static_cast<const __nv_bfloat16 *>(W); p.delta_p = delta_p; p.dX = dX;
     p.dx_f32 = dx_bf16 ? 0 : 1;
     p.Cin = static_cast<int>(s.Cin); p.Cout = static_cast<int>(s.Cout);
-    p.P = s.H * s.W; p.rows = s.B * p.P; p.g = pick_group(p.P);
+    p.P = s.H * s.W; p.rows = s.B * p.P;
     p.err_flag = err_flag;
-    const int nt = s.Cin >= 256 ? 256 : s.Cin > 64 ? 128 : 64;
+    const int niter = static_cast<int>((s.Cout + kKT - 1) / kKT);
+    p.stages = niter < kMaxStages ? niter : kMaxStages;
+    // narrower N tiles leave room for several CTAs per SM, which is what overlaps the load,
+    // MMA and store phases of different tiles
+    const int nt = s.Cin > 64 ? 128 : 64;
     dim3 grid(static_cast<unsigned>((p.rows + 127) / 128), static_cast<unsigned>((s.Cin + nt - 1) / nt));
-    const size_t smem = static_cast<size_t>(kStages) * (2 * kKT * 128 + (nt / 64) * kKT * 128) + 1024;
-    int rc;
-    if (nt == 256) { if ((rc = set_smem(tc_dx_kernel<256>, smem))) return rc; tc_dx_kernel<256><<<grid, kThreads, smem, ctx->stream>>>(p); }
-    else if (nt == 128) { if ((rc = set_smem(tc_dx_kernel<128>, smem))) return rc; tc_dx_kernel<128><<<grid, kThreads, smem, ctx->stream>>>(p); }
-    else { if ((rc = set_smem(tc_dx_kernel<64>, smem))) return rc; tc_dx_kernel<64><<<grid, kThreads, smem, ctx->stream>>>(p); }
-    return cuda_ok(cudaGetLastError());
+    size_t smem = static_cast<size_t>(p.stages) * (2 * kKT * 128 + (nt / 64) * kKT * 128);
+    if (smem < 4 * 32 * 192) smem = 4 * 32 * 192;
+    smem += 1024;
+    const bool fast = p.P % 8 == 0;
+    if (nt == 128) return fast ? run_dx<128, true>(ctx, p, grid, smem) : run_dx<128, false>(ctx, p, grid, smem);
+    return fast ? run_dx<64, true>(ctx, p, grid, smem) : run_dx<64, false>(ctx, p, grid, smem);
 }
 
 }  // namespace dbp
