@@ -49,7 +49,8 @@ typedef enum {
 /* flags for the backward calls */
 #define DBP_FORCE_SPARSE 1u /* always use the sparse gather kernels */
 #define DBP_FORCE_DENSE  2u /* always use the dense tensor-core path; DBP_EUNSUPPORTED where it
-                               does not exist (it covers bf16 linear and 1x1 layers, Cin % 8 == 0) */
+                               does not exist (it covers bf16 linear, 1x1 and 3x3 layers whose channel
+                               counts are multiples of 8) */
 #define DBP_DX_F32       4u /* with io = DBP_BF16: write dX as fp32 instead of bf16 */
 
 /*
@@ -117,7 +118,9 @@ typedef enum {
     DBP_K_DB = 5,         /* bias gradient */
     DBP_K_DECODE = 6,     /* sparse -> dense codes */
     DBP_K_GLUE = 7,       /* ReLU derivative / max-pool routing */
-    DBP_K_COUNT = 8
+    DBP_K_DX_DENSE = 8,   /* tensor-core input-gradient product */
+    DBP_K_DW_DENSE = 9,   /* tensor-core weight-gradient product (with its split-K reduction) */
+    DBP_K_COUNT = 10
 } dbp_kernel_kind;
 int dbp_profile_enable(dbp_ctx *ctx, int on);
 int dbp_profile_read(dbp_ctx *ctx, int kind, double *milliseconds, long long *launches);

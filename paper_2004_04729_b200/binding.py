@@ -23,7 +23,8 @@ EXPORTED_SYMBOLS = [
     "dbp_profile_enable", "dbp_profile_read", "dbp_set_crossover",
 ]
 
-KERNEL_KINDS = ["statistics", "quantize", "weight_taps", "dx", "dw", "db", "decode", "glue"]
+KERNEL_KINDS = ["statistics", "quantize", "weight_taps", "dx", "dw", "db", "decode", "glue",
+                "dx_dense", "dw_dense"]
 
 
 class DbpError(RuntimeError):

@@ -123,13 +123,13 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     }
     if (dense) {
         if (dX) {
-            KernelTimer t(ctx, DBP_K_DX);
+            KernelTimer t(ctx, DBP_K_DX_DENSE);
             rc = launch_tc_dx(ctx, codes, W, delta_p, s, dX, (io == DBP_BF16) && !(flags & DBP_DX_F32),
                               &ctx->state->tc_timeout);
             if (rc) return rc;
         }
         if (dW) {
-            KernelTimer t(ctx, DBP_K_DW);
+            KernelTimer t(ctx, DBP_K_DW_DENSE);
             rc = launch_tc_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout);
             if (rc) return rc;
         }
