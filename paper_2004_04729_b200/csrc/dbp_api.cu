@@ -96,7 +96,7 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     if ((dW && !X) || (dX && !W)) return DBP_EINVAL;
     if (!aligned16(delta) || !aligned16(X) || !aligned16(W) || !aligned16(dW) || !aligned16(dX)) return DBP_EINVAL;
     if ((flags & DBP_FORCE_SPARSE) && (flags & DBP_FORCE_DENSE)) return DBP_EINVAL;
-    const bool can_dense = tc_supported(s, io);
+    const bool can_dense = tc_supported(s, io) || tc3_supported(s, io);
     if ((flags & DBP_FORCE_DENSE) && !can_dense) return DBP_EUNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DBP_ECUDA;
@@ -124,13 +124,15 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     if (dense) {
         if (dX) {
             KernelTimer t(ctx, DBP_K_DX_DENSE);
-            rc = launch_tc_dx(ctx, codes, W, delta_p, s, dX, (io == DBP_BF16) && !(flags & DBP_DX_F32),
-                              &ctx->state->tc_timeout);
+            const bool dx_bf16 = (io == DBP_BF16) && !(flags & DBP_DX_F32);
+            rc = s.k == 3 ? launch_tc3_dx(ctx, codes, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout)
+                          : launch_tc_dx(ctx, codes, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout);
             if (rc) return rc;
         }
         if (dW) {
             KernelTimer t(ctx, DBP_K_DW_DENSE);
-            rc = launch_tc_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout);
+            rc = s.k == 3 ? launch_tc3_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout)
+                          : launch_tc_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout);
             if (rc) return rc;
         }
         if (db) {

@@ -97,6 +97,12 @@ int launch_tc_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *
                  const ConvShape &s, float *dW, int *err_flag);
 int launch_tc_dx(dbp_ctx *ctx, const int8_t *codes, const void *W, const float *delta_p,
                  const ConvShape &s, void *dX, bool dx_bf16, int *err_flag);
+// ---- tc_conv3x3.cu
+bool tc3_supported(const ConvShape &s, int io);
+int launch_tc3_dx(dbp_ctx *ctx, const int8_t *codes, const void *W, const float *delta_p,
+                  const ConvShape &s, void *dX, bool dx_bf16, int *err_flag);
+int launch_tc3_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *delta_p,
+                  const ConvShape &s, float *dW, int *err_flag);
 int launch_bias_grad(dbp_ctx *ctx, const int8_t *codes, const float *delta_p, const ConvShape &s,
                      float *db);
 int launch_relu_backward(dbp_ctx *ctx, const float *da, const uint8_t *mask, float *dz,

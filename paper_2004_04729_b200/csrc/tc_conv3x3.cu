@@ -1,0 +1,574 @@
+// Dense tensor-core path for the two backward products of 3x3 convolutions (stride 1, pad 1)
+// with bf16 operands. Each product is nine accumulating GEMMs, one per tap, in which the
+// operand that is shifted by the tap is always the quantized gradient: its int8 codes are
+// staged once per tile (with a halo) in shared memory, and for every tap a shifted, border-
+// masked copy is expanded to bf16 directly in the 128-byte-swizzled layout the MMA reads.
+// The dense operand (weights for dX, activations for dW) is copied unshifted by cp.async.
+//
+//   dX[ci][p]        = Delta sum_tap sum_co Wr[tap][ci][co] * q[co][p + s_tap]     (per image)
+//       M = ci (128 per accumulator, up to four accumulators), N = 128 positions, K = co
+//   dW[tap][co][ci]  = Delta sum_(b,p) X[ci][p] * q[co][p - s_tap]
+//       M = ci (128), N = 32 output channels per tap (nine accumulators), K = positions
+//
+// Eight producer warps build tiles, a ninth issues the MMAs. All waits are bounded.
+#include "tc_common.cuh"
+
+namespace dbp {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kProdWarps = 8;
+constexpr int kProd = kProdWarps * 32;
+constexpr int kThreads3 = kProd + 32;
+
+struct P3 {
+    const int8_t *codes;           // [B][Cout][H][W]
+    const __nv_bfloat16 *Wr;       // dX: weights as [tap][Cin][Cout]
+    const __nv_bfloat16 *X;        // dW: [B][Cin][H][W]
+    const float *delta_p;
+    void *dX;
+    float *partials;               // dW: [split][tap][Cout][Cin]
+    int dx_f32;
+    int B, Cin, Cout, H, W, P;
+    int tiles_per_img;             // dX: 128-position tiles per image; dW: 64-position stages per image
+    int raw_words;                 // 32-bit words per row of the staged code tile
+    int raw_pitch;                 // odd number of words between rows (bank-conflict free)
+    long long per_split, nstages;  // dW
+    int *err_flag;
+};
+
+// Eight consecutive code bytes of a staged row starting at byte offset `off`.
+__device__ __forceinline__ uint2 bytes8(const unsigned *row, int off) {
+    const int wi = off >> 2;
+    const unsigned sel = 0x3210u + 0x1111u * static_cast<unsigned>(off & 3);
+    const unsigned w0 = row[wi], w1 = row[wi + 1], w2 = row[wi + 2];
+    return make_uint2(__byte_perm(w0, w1, sel), __byte_perm(w1, w2, sel));
+}
+
+__device__ __forceinline__ uint4 expand8(uint2 c) {
+    uint4 o;
+    codes4_to_bf16(c.x, o.x, o.y);
+    codes4_to_bf16(c.y, o.z, o.w);
+    return o;
+}
+
+// One 32-bit word (four positions a..a+3 of plane `plane`) of the staged code tile; zero
+// outside [0, P). Planes start 4-byte aligned when P % 4 == 0.
+__device__ __forceinline__ unsigned load_code_word(const int8_t *plane, int a, int P, bool row_ok, bool aligned4) {
+    if (!row_ok || a + 3 < 0 || a >= P) return 0u;
+    if (aligned4 && a >= 0 && a + 3 < P) return __ldg(reinterpret_cast<const unsigned *>(plane + a));
+    unsigned w = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+        if (a + j >= 0 && a + j < P) w |= (static_cast<unsigned>(__ldg(plane + a + j)) & 0xffu) << (8 * j);
+    return w;
+}
+
+// byte masks (0xff = keep) for the eight positions n0..n0+7 of a tile starting at position p0:
+// .x/.y keep the positions whose column x allows a source at x+1 (x <= W-2); z/w at x-1 (x >= 1)
+__device__ __forceinline__ uint4 column_masks(int p0, int n0, int W) {
+    unsigned m[4] = {0, 0, 0, 0};
+    int x = (p0 + n0) % W;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        if (x <= W - 2) m[i >> 2] |= 0xffu << (8 * (i & 3));
+        if (x >= 1) m[2 + (i >> 2)] |= 0xffu << (8 * (i & 3));
+        if (++x == W) x = 0;
+    }
+    return make_uint4(m[0], m[1], m[2], m[3]);
+}
+
+struct Pipe3 {
+    unsigned long long a_full[4], a_empty[4], b_full[4], b_empty[4], acc;
+    unsigned tmem_base;
+};
+
+constexpr int kNA = 4;   // ring of dense-operand tiles
+constexpr int kRawMaxWords = 68;
+
+// ------------------------------------------------------------------------------------ dX
+template <int MT>
+__global__ void __launch_bounds__(kThreads3) tc3_dx_kernel(const P3 p) {
+    constexpr int NB = 3;                         // ring of shifted code tiles
+    constexpr int TILE = 16384;                   // 128 x 64 bf16
+    constexpr unsigned PANEL = 64 * 128;          // bytes between the two 64-position groups
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    unsigned char *a_s = smem;                            // kNA tiles [128 ci][64 co], K-major
+    unsigned char *b_s = a_s + kNA * TILE;                // NB tiles [64 co][128 positions], MN-major
+    unsigned *raw_s = reinterpret_cast<unsigned *>(b_s + NB * TILE);   // 2 x [64 rows][raw_pitch]
+    __shared__ Pipe3 pipe;
+    __shared__ uint4 masks[16];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = blockIdx.x / p.tiles_per_img;
+    const int p0 = (blockIdx.x - b * p.tiles_per_img) * 128;
+    const int ci_base = blockIdx.y * (MT * 128);
+    const int nchunks = (p.Cout + 63) / 64;
+    const int halo = p.W + 1;
+    const int a0 = ((p0 - halo) >> 2) << 2;       // position of byte 0 of a staged row (floor to 4)
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kNA; ++s) { mbar_init(&pipe.a_full[s], kProd); mbar_init(&pipe.a_empty[s], 1); }
+        for (int s = 0; s < NB; ++s) { mbar_init(&pipe.b_full[s], kProd); mbar_init(&pipe.b_empty[s], 1); }
+        mbar_init(&pipe.acc, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (threadIdx.x < 16) masks[threadIdx.x] = column_masks(p0, threadIdx.x * 8, p.W);
+    if (warp == kProdWarps) tmem_alloc(&pipe.tmem_base, MT * 128);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const unsigned tmem_d = pipe.tmem_base;
+
+    if (warp < kProdWarps) {
+        const bool aligned4 = (p.P & 3) == 0;
+        const int total_words = 64 * p.raw_words;
+        unsigned pre[17];                          // staged-tile words of the next chunk
+        auto fetch = [&](int c) {
+#pragma unroll
+            for (int i = 0; i < 17; ++i) {
+                const int idx = threadIdx.x + i * kProd;
+                unsigned w = 0;
+                if (idx < total_words) {
+                    const int row = idx / p.raw_words, wd = idx - row * p.raw_words;
+                    const int co = c * 64 + row;
+                    const int8_t *plane = p.codes + (static_cast<long long>(b) * p.Cout + co) * p.P;
+                    w = load_code_word(plane, a0 + 4 * wd, p.P, co < p.Cout, aligned4);
+                }
+                pre[i] = w;
+            }
+        };
+        fetch(0);
+        bool ok = true;
+        int ia = 0, ib = 0;
+        for (int c = 0; c < nchunks; ++c) {
+            unsigned *raw = raw_s + (c & 1) * (64 * p.raw_pitch);
+#pragma unroll
+            for (int i = 0; i < 17; ++i) {
+                const int idx = threadIdx.x + i * kProd;
+                if (idx < total_words) {
+                    const int row = idx / p.raw_words, wd = idx - row * p.raw_words;
+                    raw[row * p.raw_pitch + wd] = pre[i];
+                }
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(kProd) : "memory");
+            if (c + 1 < nchunks) fetch(c + 1);
+#pragma unroll 1
+            for (int tap = 0; tap < 9 && ok; ++tap, ++ib) {
+                const int ky = tap / 3, kx = tap - ky * 3;
+                const int shift = (1 - ky) * p.W + (1 - kx);
+                const int sb = ib % NB;
+                ok = mbar_wait(&pipe.b_empty[sb], ((ib / NB) & 1) ^ 1, p.err_flag);
+                unsigned char *bt = b_s + sb * TILE;
+                // 2 row groups x 16 chunks = 32 warp tasks; lanes = 32 consecutive co rows
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const int task = warp * 4 + t;
+                    const int ch = task & 15, row = (task >> 4) * 32 + lane;
+                    uint2 c8 = bytes8(raw + row * p.raw_pitch, p0 + ch * 8 + shift - a0);
+                    const uint4 m = masks[ch];
+                    if (kx == 0) { c8.x &= m.x; c8.y &= m.y; }
+                    if (kx == 2) { c8.x &= m.z; c8.y &= m.w; }
+                    *reinterpret_cast<uint4 *>(bt + (ch >> 3) * PANEL + swz(row, ch & 7)) = expand8(c8);
+                }
+                fence_async_proxy();
+                mbar_arrive(&pipe.b_full[sb]);
+                // weights of this tap and chunk: MT tiles [128 ci][64 co]
+                for (int m = 0; m < MT && ok; ++m, ++ia) {
+                    const int sa = ia % kNA;
+                    ok = mbar_wait(&pipe.a_empty[sa], ((ia / kNA) & 1) ^ 1, p.err_flag);
+                    unsigned char *at = a_s + sa * TILE;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int idx = threadIdx.x + i * kProd;      // 1024 chunks of 16 bytes
+                        const int row = idx >> 3, ch = idx & 7;
+                        const int ci = ci_base + m * 128 + row, co = c * 64 + ch * 8;
+                        const bool v = ci < p.Cin && co < p.Cout;      // Cout % 8 == 0
+                        cp_async16(at + swz(row, ch),
+                                   v ? p.Wr + (static_cast<long long>(tap) * p.Cin + ci) * p.Cout + co : p.Wr, v);
+                    }
+                    mbar_arrive_on_cp_async(&pipe.a_full[sa]);
+                }
+            }
+        }
+        // ---------------- epilogue: lanes = ci, columns = positions; warp w takes lane quarter
+        // w % 4 and column half w / 4
+        if (mbar_wait(&pipe.acc, 0, p.err_flag)) {
+            tc_fence_after();
+            const float delta = *p.delta_p;
+            const int q = warp & 3, half = warp >> 2;
+            const bool vec = (p.P & 7) == 0;
+            for (int m = 0; m < MT; ++m) {
+                const int ci = ci_base + m * 128 + q * 32 + lane;
+#pragma unroll 1
+                for (int cc = 0; cc < 2; ++cc) {
+                    const int n0 = half * 64 + cc * 32;
+                    unsigned v[32];
+                    tmem_ld32(tmem_d + (static_cast<unsigned>(q * 32) << 16) + m * 128 + n0, v);
+                    const long long base = (static_cast<long long>(b) * p.Cin + ci) * p.P + p0 + n0;
+                    const int nvalid = p.P - (p0 + n0);      // positions of this run inside the image
+                    if (ci >= p.Cin || nvalid <= 0) {
+                        // nothing to store for this lane / run
+                    } else if (p.dx_f32) {
+                        float *dst = static_cast<float *>(p.dX) + base;
+                        if (vec && nvalid >= 32) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4)
+                                *reinterpret_cast<float4 *>(dst + j) =
+                                    make_float4(__uint_as_float(v[j]) * delta, __uint_as_float(v[j + 1]) * delta,
+                                                __uint_as_float(v[j + 2]) * delta, __uint_as_float(v[j + 3]) * delta);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (j < nvalid) dst[j] = __uint_as_float(v[j]) * delta;
+                        }
+                    } else {
+                        __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.dX) + base;
+                        if (vec && nvalid >= 32) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 8) {
+                                unsigned w[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[j + 2 * e]) * delta,
+                                                                                   __uint_as_float(v[j + 2 * e + 1]) * delta);
+                                    w[e] = *reinterpret_cast<const unsigned *>(&h);
+                                }
+                                *reinterpret_cast<uint4 *>(dst + j) = make_uint4(w[0], w[1], w[2], w[3]);
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (j < nvalid) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]) * delta);
+                        }
+                    }
+                }
+            }
+        }
+    } else if (lane == 0) {
+        constexpr unsigned idesc = make_idesc(128, 128, false, true);
+        bool ok = true;
+        int ia = 0, ib = 0;
+        for (int c = 0; c < nchunks && ok; ++c) {
+            for (int tap = 0; tap < 9 && ok; ++tap, ++ib) {
+                const int sb = ib % NB;
+                ok = mbar_wait(&pipe.b_full[sb], (ib / NB) & 1, p.err_flag);
+                fence_async_proxy();
+                tc_fence_after();
+                const unsigned long long bd = make_desc(smem_u32(b_s + sb * TILE), PANEL, 1024);
+                for (int m = 0; m < MT && ok; ++m, ++ia) {
+                    const int sa = ia % kNA;
+                    ok = mbar_wait(&pipe.a_full[sa], (ia / kNA) & 1, p.err_flag);
+                    fence_async_proxy();
+                    tc_fence_after();
+                    const unsigned long long ad = make_desc(smem_u32(a_s + sa * TILE), 16, 1024);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        mma_bf16(tmem_d + m * 128, ad + 2 * k, bd + 128 * k, idesc, (c > 0 || tap > 0 || k > 0) ? 1u : 0u);
+                    mma_commit(&pipe.a_empty[sa]);
+                }
+                mma_commit(&pipe.b_empty[sb]);
+            }
+        }
+        mma_commit(&pipe.acc);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kProdWarps) {
+        __syncwarp();
+        tmem_dealloc(tmem_d, MT * 128);
+    }
+}
+
+// weights [Cout][Cin][3][3] -> [tap][Cin][Cout]
+__global__ void weight_rows_kernel(const __nv_bfloat16 *__restrict__ W, __nv_bfloat16 *__restrict__ out,
+                                   long long Cout, long long Cin) {
+    const long long n = Cout * Cin * 9;
+    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < n;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const long long co = i % Cout, ci = (i / Cout) % Cin, t = i / (Cout * Cin);
+        out[i] = W[(co * Cin + ci) * 9 + t];
+    }
+}
+
+// ------------------------------------------------------------------------------------ dW
+// One stage = 64 consecutive positions of one image. A = X tile [128 ci][64 positions] (native,
+// K-major), B_tap = shifted codes [32 co][64 positions] (K-major), nine accumulators of 32 columns.
+template <bool FASTX>
+__global__ void __launch_bounds__(kThreads3) tc3_dw_kernel(const P3 p) {
+    constexpr int NB = 2;
+    constexpr int A_TILE = 16384;                 // 128 x 64 bf16
+    constexpr int B_TAP = 32 * 128;               // 32 x 64 bf16
+    constexpr int B_STAGE = 9 * B_TAP;
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    unsigned char *a_s = smem;
+    unsigned char *b_s = a_s + kNA * A_TILE;
+    unsigned *raw_s = reinterpret_cast<unsigned *>(b_s + NB * B_STAGE);   // 2 x [32 rows][raw_pitch]
+    __shared__ Pipe3 pipe;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ci0 = blockIdx.x * 128, co0 = blockIdx.y * 32;
+    const long long s0 = blockIdx.z * p.per_split;
+    long long s1 = s0 + p.per_split;
+    if (s1 > p.nstages) s1 = p.nstages;
+    const int niter = s1 > s0 ? static_cast<int>(s1 - s0) : 0;
+    const int halo = p.W + 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kNA; ++s) { mbar_init(&pipe.a_full[s], kProd); mbar_init(&pipe.a_empty[s], 1); }
+        for (int s = 0; s < NB; ++s) { mbar_init(&pipe.b_full[s], kProd); mbar_init(&pipe.b_empty[s], 1); }
+        mbar_init(&pipe.acc, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kProdWarps) tmem_alloc(&pipe.tmem_base, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const unsigned tmem_d = pipe.tmem_base;
+
+    if (warp < kProdWarps) {
+        const bool aligned4 = (p.P & 3) == 0;
+        const int total_words = 32 * p.raw_words;
+        unsigned pre[9];
+        auto stage_origin = [&](long long st, int &bimg, int &k0) {
+            bimg = static_cast<int>(st / p.tiles_per_img);
+            k0 = static_cast<int>(st - static_cast<long long>(bimg) * p.tiles_per_img) * 64;
+        };
+        auto fetch = [&](long long st) {
+            int bimg, k0;
+            stage_origin(st, bimg, k0);
+            const int a0 = ((k0 - halo) >> 2) << 2;
+#pragma unroll
+            for (int i = 0; i < 9; ++i) {
+                const int idx = threadIdx.x + i * kProd;
+                unsigned w = 0;
+                if (idx < total_words) {
+                    const int row = idx / p.raw_words, wd = idx - row * p.raw_words;
+                    const int co = co0 + row;
+                    const int8_t *plane = p.codes + (static_cast<long long>(bimg) * p.Cout + co) * p.P;
+                    w = load_code_word(plane, a0 + 4 * wd, p.P, co < p.Cout, aligned4);
+                }
+                pre[i] = w;
+            }
+        };
+        if (niter > 0) fetch(s0);
+        bool ok = true;
+        for (int it = 0; it < niter; ++it) {
+            int bimg, k0;
+            stage_origin(s0 + it, bimg, k0);
+            const int a0 = ((k0 - halo) >> 2) << 2;
+            unsigned *raw = raw_s + (it & 1) * (32 * p.raw_pitch);
+#pragma unroll
+            for (int i = 0; i < 9; ++i) {
+                const int idx = threadIdx.x + i * kProd;
+                if (idx < total_words) {
+                    const int row = idx / p.raw_words, wd = idx - row * p.raw_words;
+                    raw[row * p.raw_pitch + wd] = pre[i];
+                }
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(kProd) : "memory");
+            if (it + 1 < niter) fetch(s0 + it + 1);
+            if (!ok) continue;       // a wait expired: keep the barrier count, skip the work
+            // ---- X tile: 128 ci rows x 8 chunks of 8 positions
+            const int sa = it % kNA;
+            ok = mbar_wait(&pipe.a_empty[sa], ((it / kNA) & 1) ^ 1, p.err_flag);
+            unsigned char *at = a_s + sa * A_TILE;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int idx = threadIdx.x + i * kProd;
+                const int row = idx >> 3, ch = idx & 7;
+                const int ci = ci0 + row, pp = k0 + ch * 8;
+                const __nv_bfloat16 *src = p.X + (static_cast<long long>(bimg) * p.Cin + ci) * p.P + pp;
+                if (FASTX) {     // P % 8 == 0: whole 16-byte groups, aligned
+                    const bool v = ci < p.Cin && pp < p.P;
+                    cp_async16(at + swz(row, ch), v ? src : p.X, v);
+                } else {
+                    unsigned short h[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        h[j] = (ci < p.Cin && pp + j < p.P) ? __ldg(reinterpret_cast<const unsigned short *>(src) + j) : 0;
+                    *reinterpret_cast<uint4 *>(at + swz(row, ch)) =
+                        make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+                }
+            }
+            if (FASTX) {
+                mbar_arrive_on_cp_async(&pipe.a_full[sa]);
+            } else {
+                fence_async_proxy();
+                mbar_arrive(&pipe.a_full[sa]);
+            }
+            // ---- nine shifted code tiles: 72 warp tasks (tap, chunk), lanes = 32 co rows
+            const int sb = it % NB;
+            ok = ok && mbar_wait(&pipe.b_empty[sb], ((it / NB) & 1) ^ 1, p.err_flag);
+            unsigned char *bt = b_s + sb * B_STAGE;
+#pragma unroll 1
+            for (int task = warp; task < 72; task += kProdWarps) {
+                const int tap = task >> 3, ch = task & 7;
+                const int ky = tap / 3, kx = tap - ky * 3;
+                // X[p + (ky-1) W + (kx-1)] pairs with q[p]; with p' the X position, q index is p' - s
+                const int shift = -((ky - 1) * p.W + (kx - 1));
+                uint2 c8 = bytes8(raw + lane * p.raw_pitch, k0 + ch * 8 + shift - a0);
+                // source column is x' - (kx-1): kx = 0 needs x' <= W-2, kx = 2 needs x' >= 1
+                const uint4 m = column_masks(k0, ch * 8, p.W);
+                if (kx == 0) { c8.x &= m.x; c8.y &= m.y; }
+                if (kx == 2) { c8.x &= m.z; c8.y &= m.w; }
+                *reinterpret_cast<uint4 *>(bt + tap * B_TAP + swz(lane, ch)) = expand8(c8);
+            }
+            fence_async_proxy();
+            mbar_arrive(&pipe.b_full[sb]);
+        }
+        // ---------------- epilogue: lanes = ci, columns = (tap, co); partials [split][tap][Cout][Cin]
+        if (niter > 0 && mbar_wait(&pipe.acc, 0, p.err_flag)) {
+            tc_fence_after();
+            const int q = warp & 3;
+            const int ci = ci0 + q * 32 + lane;
+            for (int tap = warp >> 2; tap < 9; tap += 2) {
+                unsigned v[32];
+                tmem_ld32(tmem_d + (static_cast<unsigned>(q * 32) << 16) + tap * 32, v);
+                if (ci < p.Cin) {
+                    float *dst = p.partials + ((static_cast<long long>(blockIdx.z) * 9 + tap) * p.Cout + co0) * p.Cin + ci;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (co0 + j < p.Cout) dst[static_cast<long long>(j) * p.Cin] = __uint_as_float(v[j]);
+                }
+            }
+        }
+    } else if (lane == 0) {
+        constexpr unsigned idesc = make_idesc(128, 32, false, false);
+        bool ok = true;
+        for (int it = 0; it < niter && ok; ++it) {
+            const int sa = it % kNA, sb = it % NB;
+            ok = mbar_wait(&pipe.a_full[sa], (it / kNA) & 1, p.err_flag);
+            ok = ok && mbar_wait(&pipe.b_full[sb], (it / NB) & 1, p.err_flag);
+            fence_async_proxy();
+            tc_fence_after();
+            const unsigned long long ad = make_desc(smem_u32(a_s + sa * A_TILE), 16, 1024);
+            const unsigned b_addr = smem_u32(b_s + sb * B_STAGE);
+            for (int tap = 0; tap < 9; ++tap) {
+                const unsigned long long bd = make_desc(b_addr + tap * B_TAP, 16, 1024);
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    mma_bf16(tmem_d + tap * 32, ad + 2 * k, bd + 2 * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
+            }
+            mma_commit(&pipe.a_empty[sa]);
+            mma_commit(&pipe.b_empty[sb]);
+        }
+        if (niter > 0) mma_commit(&pipe.acc);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kProdWarps) {
+        __syncwarp();
+        tmem_dealloc(tmem_d, 512);
+    }
+}
+
+// dW[co][ci][tap] = Delta * sum over splits of partials[split][tap][co][ci]
+__global__ void __launch_bounds__(256) tc3_dw_reduce_kernel(const float *__restrict__ partials, int nsplit,
+                                                            long long Cout, long long Cin,
+                                                            const float *__restrict__ delta_p, float *__restrict__ dW) {
+    const float delta = *delta_p;
+    const long long n = Cout * Cin, tot = n * 9;
+    for (long long i = blockIdx.x * 256ll + threadIdx.x; i < tot; i += gridDim.x * 256ll) {
+        const long long tap = i / n, rem = i - tap * n;      // rem = co * Cin + ci (coalesced reads)
+        float a = 0.f;
+        for (int s = 0; s < nsplit; ++s) a += __ldcs(partials + (static_cast<long long>(s) * 9 + tap) * n + rem);
+        dW[rem * 9 + tap] = a * delta;
+    }
+}
+
+int raw_geometry(int W, int span, int &words, int &pitch) {
+    // a staged row covers positions [floor4(start - (W+1)), start + span + (W+1)) plus slack for
+    // the three-word reads of bytes8
+    words = (span + 2 * (W + 1) + 3 + 3) / 4 + 2;
+    pitch = words | 1;
+    return words <= kRawMaxWords ? DBP_OK : DBP_EUNSUPPORTED;
+}
+
+template <typename K>
+int set_smem3(K kern, size_t bytes) {
+    return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes)) == cudaSuccess
+               ? DBP_OK : DBP_ECUDA;
+}
+
+}  // namespace
+
+bool tc3_supported(const ConvShape &s, int io) {
+    return io == DBP_BF16 && s.k == 3 && s.Cin % 8 == 0 && s.Cout % 8 == 0 && s.W <= 62 && s.H * s.W < (1 << 24);
+}
+
+int launch_tc3_dx(dbp_ctx *ctx, const int8_t *codes, const void *W, const float *delta_p,
+                  const ConvShape &s, void *dX, bool dx_bf16, int *err_flag) {
+    P3 p{};
+    p.codes = codes; p.delta_p = delta_p; p.dX = dX; p.dx_f32 = dx_bf16 ? 0 : 1;
+    p.B = static_cast<int>(s.B); p.Cin = static_cast<int>(s.Cin); p.Cout = static_cast<int>(s.Cout);
+    p.H = static_cast<int>(s.H); p.W = static_cast<int>(s.W); p.P = p.H * p.W;
+    p.tiles_per_img = (p.P + 127) / 128;
+    p.err_flag = err_flag;
+    int rc = raw_geometry(p.W, 128, p.raw_words, p.raw_pitch);
+    if (rc) return rc;
+    if (64 * p.raw_words > 17 * kProd) return DBP_EUNSUPPORTED;
+    const size_t wb = sizeof(__nv_bfloat16) * static_cast<size_t>(s.Cout) * s.Cin * 9;
+    if ((rc = ws_reserve(ctx, ctx->w_taps, wb))) return rc;
+    __nv_bfloat16 *wr = static_cast<__nv_bfloat16 *>(ctx->w_taps.ptr);
+    {
+        long long blocks = (static_cast<long long>(s.Cout) * s.Cin * 9 + 255) / 256;
+        if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
+        weight_rows_kernel<<<static_cast<unsigned>(blocks), 256, 0, ctx->stream>>>(
+            static_cast<const __nv_bfloat16 *>(W), wr, s.Cout, s.Cin);
+        if ((rc = cuda_ok(cudaGetLastError()))) return rc;
+    }
+    p.Wr = wr;
+    const int mt = s.Cin > 256 ? 4 : s.Cin > 128 ? 2 : 1;
+    dim3 grid(static_cast<unsigned>(s.B * p.tiles_per_img), static_cast<unsigned>((s.Cin + mt * 128 - 1) / (mt * 128)));
+    const size_t smem = static_cast<size_t>(kNA + 3) * 16384 + 2 * 64 * static_cast<size_t>(p.raw_pitch) * 4 + 1024;
+    if (mt == 4) { if ((rc = set_smem3(tc3_dx_kernel<4>, smem))) return rc; tc3_dx_kernel<4><<<grid, kThreads3, smem, ctx->stream>>>(p); }
+    else if (mt == 2) { if ((rc = set_smem3(tc3_dx_kernel<2>, smem))) return rc; tc3_dx_kernel<2><<<grid, kThreads3, smem, ctx->stream>>>(p); }
+    else { if ((rc = set_smem3(tc3_dx_kernel<1>, smem))) return rc; tc3_dx_kernel<1><<<grid, kThreads3, smem, ctx->stream>>>(p); }
+    return cuda_ok(cudaGetLastError());
+}
+
+int launch_tc3_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *delta_p,
+                  const ConvShape &s, float *dW, int *err_flag) {
+    P3 p{};
+    p.codes = codes; p.X = static_cast<const __nv_bfloat16 *>(X); p.delta_p = delta_p;
+    p.B = static_cast<int>(s.B); p.Cin = static_cast<int>(s.Cin); p.Cout = static_cast<int>(s.Cout);
+    p.H = static_cast<int>(s.H); p.W = static_cast<int>(s.W); p.P = p.H * p.W;
+    p.tiles_per_img = (p.P + 63) / 64;
+    p.nstages = static_cast<long long>(s.B) * p.tiles_per_img;
+    p.err_flag = err_flag;
+    int rc = raw_geometry(p.W, 64, p.raw_words, p.raw_pitch);
+    if (rc) return rc;
+    if (32 * p.raw_words > 9 * kProd) return DBP_EUNSUPPORTED;
+    const long long tiles = ((s.Cin + 127) / 128) * ((s.Cout + 31) / 32);
+    long long split = (ctx->sm_count + tiles - 1) / tiles;
+    if (split > p.nstages) split = p.nstages;
+    if (split < 1) split = 1;
+    p.per_split = (p.nstages + split - 1) / split;
+    split = (p.nstages + p.per_split - 1) / p.per_split;
+    const size_t nw = static_cast<size_t>(s.Cout) * s.Cin * 9;
+    if ((rc = ws_reserve(ctx, ctx->tc_partials, sizeof(float) * nw * split))) return rc;
+    p.partials = static_cast<float *>(ctx->tc_partials.ptr);
+    dim3 grid(static_cast<unsigned>((s.Cin + 127) / 128), static_cast<unsigned>((s.Cout + 31) / 32),
+              static_cast<unsigned>(split));
+    const size_t smem = static_cast<size_t>(kNA) * 16384 + 2 * 9 * 4096 + 2 * 32 * static_cast<size_t>(p.raw_pitch) * 4 + 1024;
+    if (p.P % 8 == 0) {
+        if ((rc = set_smem3(tc3_dw_kernel<true>, smem))) return rc;
+        tc3_dw_kernel<true><<<grid, kThreads3, smem, ctx->stream>>>(p);
+    } else {
+        if ((rc = set_smem3(tc3_dw_kernel<false>, smem))) return rc;
+        tc3_dw_kernel<false><<<grid, kThreads3, smem, ctx->stream>>>(p);
+    }
+    if ((rc = cuda_ok(cudaGetLastError()))) return rc;
+    long long blocks = (static_cast<long long>(nw) + 255) / 256;
+    if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
+    tc3_dw_reduce_kernel<<<static_cast<unsigned>(blocks), 256, 0, ctx->stream>>>(
+        p.partials, static_cast<int>(split), s.Cout, s.Cin, delta_p, dW);
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace dbp

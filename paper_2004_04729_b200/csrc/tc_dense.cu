@@ -13,7 +13,7 @@
 // that the MMA descriptors name. A fifth warp issues the MMAs; mbarriers order producers,
 // tensor core and epilogue. Every wait is bounded: on expiry the kernel raises a flag in
 // global memory and runs to its end.
-#include "dbp_internal.cuh"
+#include "tc_common.cuh"
 
 namespace dbp {
 
@@ -24,115 +24,8 @@ constexpr int kProducers = kProducerWarps * 32;
 constexpr int kThreads = kProducers + 32;
 constexpr int kMaxStages = 4;
 constexpr int kKT = 64;                             // K elements per stage (one 128-byte swizzled row)
-constexpr long long kWaitCycles = 1000000000ll;     // a wait gives up after this many SM clocks
 
-__device__ __forceinline__ unsigned smem_u32(const void *p) {
-    return static_cast<unsigned>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(unsigned long long *bar, int count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(unsigned long long *bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// arrival that fires when this thread's earlier cp.async copies have landed
-__device__ __forceinline__ void mbar_arrive_on_cp_async(unsigned long long *bar) {
-    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// Returns false when the phase did not complete within about half a second.
-__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity, int *err_flag) {
-    const unsigned addr = smem_u32(bar);
-    const long long t0 = clock64();
-    for (;;) {
-        unsigned done;
-        asm volatile(
-            "{\n\t.reg .pred P1;\n\t"
-            "mbarrier.test_wait.parity.shared::cta.b64 P1, [%1], %2;\n\t"
-            "selp.b32 %0, 1, 0, P1;\n\t}"
-            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
-        if (done) return true;
-        if (clock64() - t0 > kWaitCycles) break;
-        __nanosleep(20);
-    }
-    atomicExch(err_flag, 1);
-    return false;
-}
-__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(unsigned *dst_smem, int ncols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols));
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
-}
-__device__ __forceinline__ void tmem_dealloc(unsigned taddr, int ncols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols));
-}
-__device__ __forceinline__ void mma_bf16(unsigned tmem_d, unsigned long long adesc, unsigned long long bdesc,
-                                         unsigned idesc, unsigned accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void mma_commit(unsigned long long *bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(unsigned taddr, unsigned (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc, bool valid) {
-    const int n = valid ? 16 : 0;   // src-size 0: the 16 bytes are zero-filled
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(n) : "memory");
-}
-
-// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1; lbo/sbo in bytes.
-// K-major operand: rows of 64 K-elements, 8-row groups sbo apart (lbo unused).
-// MN-major operand: rows (one per k) of 64 MN-elements, 8-row groups sbo apart, 64-element
-// MN groups lbo apart.
-__device__ __forceinline__ unsigned long long make_desc(unsigned smem_addr, unsigned lbo, unsigned sbo) {
-    unsigned long long d = 0;
-    d |= static_cast<unsigned long long>((smem_addr & 0x3ffffu) >> 4);
-    d |= static_cast<unsigned long long>((lbo >> 4) & 0x3fffu) << 16;
-    d |= static_cast<unsigned long long>((sbo >> 4) & 0x3fffu) << 32;
-    d |= 1ull << 46;     // version
-    d |= 2ull << 61;     // SWIZZLE_128B
-    return d;
-}
-// Instruction descriptor: fp32 accumulate, bf16 x bf16.
-__host__ __device__ constexpr unsigned make_idesc(int M, int N, bool a_mn_major, bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn_major ? (1u << 15) : 0u) | (b_mn_major ? (1u << 16) : 0u) |
-           (static_cast<unsigned>(N >> 3) << 17) | (static_cast<unsigned>(M >> 4) << 24);
-}
-
-// byte offset of 16-byte chunk `chunk` (0..7) of row `row` inside a 128-byte-swizzled panel
-__device__ __forceinline__ unsigned swz(unsigned row, unsigned chunk) { return row * 128u + ((chunk ^ (row & 7u)) << 4); }
-
-// four int8 codes packed in a word -> two words of packed bf16 (exact).
-// byte ^ 0x80 = code + 128 as an unsigned byte; 0x4B0000xx read as a float is 2^23 + xx, so
-// subtracting 2^23 + 128 leaves the code as a float whose top 16 bits are its bf16 pattern.
-__device__ __forceinline__ void codes4_to_bf16(unsigned w, unsigned &lo, unsigned &hi) {
-    const unsigned x = w ^ 0x80808080u;
-    const float f0 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7650)) - 8388736.0f;
-    const float f1 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7651)) - 8388736.0f;
-    const float f2 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7652)) - 8388736.0f;
-    const float f3 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7653)) - 8388736.0f;
-    lo = __byte_perm(__float_as_uint(f0), __float_as_uint(f1), 0x7632);
-    hi = __byte_perm(__float_as_uint(f2), __float_as_uint(f3), 0x7632);
-}
-__device__ __forceinline__ unsigned short code_to_bf16(int c) {
-    return static_cast<unsigned short>(__float_as_uint(static_cast<float>(c)) >> 16);
-}
+using namespace tc;
 
 // Row r of the flattened (image, position) index of a [B][C][P] tensor: walks eight consecutive
 // rows from (b, p) without divisions, for any P (P = 1 is a linear layer's [B][C] matrix).

@@ -62,6 +62,22 @@ def test_dense_path_conv1x1(ctx, B, Ci, Co, H, W):
     _run(ctx, L, dbp.DBP_FORCE_DENSE)
 
 
+@pytest.mark.parametrize("B,Ci,Co,H,W", [
+    (2, 64, 64, 32, 32),      # config-3 shape at batch 2 (bf16)
+    (1, 64, 64, 56, 56),      # ResNet stage 1: 25 position tiles per image, last one half full
+    (2, 128, 128, 28, 28),
+    (2, 256, 256, 14, 14),    # two accumulators per CTA for dX; 196 positions: unaligned rows
+    (3, 512, 512, 7, 7),      # four accumulators; one ragged tile per image
+    (1, 72, 40, 9, 11),       # channel counts that fill no tile, odd width
+    (2, 16, 24, 3, 62),       # widest supported row
+    (2, 8, 8, 1, 1),          # a single position: every tap but the centre is masked
+])
+def test_dense_path_conv3x3(ctx, B, Ci, Co, H, W):
+    import paper_2004_04729_b200 as dbp
+    L = wl.conv_layer(B, Ci, Co, H, W, 3, data_seed=B + Ci + Co + H, scale=5.0 if Ci > 64 else 2.0, dtype="bf16")
+    _run(ctx, L, dbp.DBP_FORCE_DENSE)
+
+
 @pytest.mark.parametrize("B,N,K", [(128, 300, 784), (256, 512, 2048), (70, 10, 512), (33, 100, 304)])
 def test_dense_path_linear(ctx, B, N, K):
     import paper_2004_04729_b200 as dbp
@@ -79,8 +95,8 @@ def test_dense_and_sparse_paths_agree_and_unsupported_is_refused(ctx):
     for key in ("dW", "dX"):
         ref = b[key].double()
         assert (a[key].double() - ref).norm() <= 2e-5 * ref.norm()
-    L3 = wl.conv_layer(1, 16, 16, 6, 6, 3, data_seed=4, dtype="bf16")
-    with pytest.raises(dbp.DbpError) as e:          # 3x3 has no dense path
+    L3 = wl.conv_layer(1, 12, 16, 6, 6, 3, data_seed=4, dtype="bf16")
+    with pytest.raises(dbp.DbpError) as e:          # channel count not a multiple of 8
         dbp.dithered_conv_backward(ctx, _t(L3.delta), _t(L3.X), _t(L3.W), 0, 2.0, flags=dbp.DBP_FORCE_DENSE)
     assert e.value.status == -2
     Lf = wl.conv_layer(1, 16, 16, 6, 6, 1, data_seed=4)
