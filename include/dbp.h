@@ -209,6 +209,39 @@ int dbp_relu_backward(dbp_ctx *ctx, const float *delta_a, const uint8_t *mask, f
 int dbp_maxpool2x2_backward(dbp_ctx *ctx, const float *g, const int8_t *argmax, float *out,
                             long long planes, long long h, long long w);
 
+/*
+ * Step size without any allocation (the paper has no counterpart: this entry point exists
+ * for the way the library is embedded, not for the method).
+ *
+ * Every other call needs a dbp_ctx, and a context allocates: dbp_create and the first call
+ * of each size call cudaMalloc for the workspace. Some hosts cannot do that at the point
+ * where they need the step size -- a serving process whose device memory is handed out once
+ * at start-up and then frozen, a real-time loop that must not hit the implicit device
+ * synchronisation of cudaMalloc/cudaFree, a plug-in that runs inside someone else's memory
+ * budget. For them this call computes Delta = scale * std(delta) (Algorithm 1's first two
+ * lines, same arithmetic and same result as nsd_quantize's step) with no context and no
+ * allocation of any kind: the reduction's scratch is a fixed array of about 16 KB inside the
+ * library image, present on every GPU that loads the library until the process exits.
+ *
+ *   delta      : DEVICE pointer, numel elements of dtype (DBP_F32 / DBP_BF16), 16-byte aligned.
+ *   numel      : 1 ... DBP_NOALLOC_MAX_NUMEL; larger tensors return DBP_ECAPACITY and nothing
+ *                is enqueued.
+ *   scale      : s > 0.
+ *   delta_out  : DEVICE pointer to one float, written by the kernel.
+ *   cuda_stream: cudaStream_t to enqueue on (NULL = default stream); the call does not
+ *                synchronise. It runs on the CURRENT device.
+ *
+ * The first call on each device looks up the device address of the scratch array (a runtime
+ * query, no allocation); make that first call outside any stream capture.
+ * All calls on one device share the one scratch array, which keeps whatever the previous
+ * call left in it; the call resets the part that must start at zero. Two calls whose
+ * kernels can overlap on the same GPU (different streams, different threads) race on it:
+ * serialise them. Non-finite input gives Delta = 0.
+ */
+#define DBP_NOALLOC_MAX_NUMEL (1ll << 31)
+int nsd_step_size_noalloc(const void *delta, int dtype, long long numel, float scale,
+                          float *delta_out, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

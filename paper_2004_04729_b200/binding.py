@@ -20,7 +20,7 @@ EXPORTED_SYMBOLS = [
     "dbp_last_device_status", "dbp_sparse_bytes", "nsd_quantize", "nsd_decode_dense",
     "dithered_linear_backward", "dithered_conv_backward", "dithered_linear_backward_host",
     "dithered_conv_backward_host", "dbp_relu_backward", "dbp_maxpool2x2_backward",
-    "dbp_profile_enable", "dbp_profile_read", "dbp_set_crossover",
+    "dbp_profile_enable", "dbp_profile_read", "dbp_set_crossover", "nsd_step_size_noalloc",
 ]
 
 KERNEL_KINDS = ["statistics", "quantize", "weight_taps", "dx", "dw", "db", "decode", "glue",
@@ -77,6 +77,7 @@ def load_library():
                                                 i32, ull, f32, vp, vp, vp, u32,
                                                 ctypes.POINTER(f32), ctypes.POINTER(ll)]
     lib.dbp_set_crossover.argtypes = [vp, f32]
+    lib.nsd_step_size_noalloc.argtypes = [vp, i32, ll, f32, vp, vp]
     lib.dbp_profile_enable.argtypes = [vp, i32]
     lib.dbp_profile_read.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ll)]
     lib.dbp_relu_backward.argtypes = [vp, vp, vp, vp, ll]
@@ -308,6 +309,21 @@ def maxpool2x2_backward(ctx: Context, g: torch.Tensor, argmax_i8: torch.Tensor) 
     _check(load_library().dbp_maxpool2x2_backward(ctx._h, _ptr(g), _ptr(argmax_i8), _ptr(out),
                                                   B * C, h, w), "dbp_maxpool2x2_backward")
     return out
+
+
+def nsd_step_size_noalloc(delta: torch.Tensor, scale: float, out: torch.Tensor,
+                          stream: Optional[torch.cuda.Stream] = None, numel: Optional[int] = None) -> None:
+    """Delta = scale * std(delta) written to the one-element device tensor `out`, through the
+    library's allocation-free entry point: no Context, no workspace. The caller owns `delta`
+    and `out`; nothing is allocated here either. `numel` overrides delta.numel() (used to
+    probe the size limit without a large tensor)."""
+    _dev(delta, "delta"), _dev(out, "out")
+    if out.dtype != torch.float32 or out.numel() < 1:
+        raise ValueError("out must hold one float32")
+    s = stream if stream is not None else torch.cuda.current_stream()
+    _check(load_library().nsd_step_size_noalloc(
+        _ptr(delta), _dtype_code(delta), delta.numel() if numel is None else int(numel), float(scale),
+        _ptr(out), ctypes.c_void_p(s.cuda_stream)), "nsd_step_size_noalloc")
 
 
 def _splitmix64_output(seed: int, index: int) -> int:
