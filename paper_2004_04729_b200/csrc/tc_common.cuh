@@ -78,6 +78,14 @@ __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc, boo
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(n) : "memory");
 }
 
+// 4- or 8-byte asynchronous copy (zero-filled when !valid); both addresses aligned to the size
+template <int BYTES>
+__device__ __forceinline__ void cp_async_small(void *smem_dst, const void *gsrc, bool valid) {
+    static_assert(BYTES == 4 || BYTES == 8, "cp.async.ca copies 4, 8 or 16 bytes");
+    const int n = valid ? BYTES : 0;
+    asm volatile("cp.async.ca.shared.global [%0], [%1], %2, %3;" ::"r"(smem_u32(smem_dst)), "l"(gsrc), "n"(BYTES), "r"(n) : "memory");
+}
+
 // Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1; lbo/sbo in bytes.
 // K-major operand: rows of 64 K-elements, 8-row groups sbo apart (lbo unused).
 // MN-major operand: rows (one per k) of 64 MN-elements, 8-row groups sbo apart, 64-element
@@ -111,6 +119,13 @@ __device__ __forceinline__ void codes4_to_bf16(unsigned w, unsigned &lo, unsigne
     const float f3 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7653)) - 8388736.0f;
     lo = __byte_perm(__float_as_uint(f0), __float_as_uint(f1), 0x7632);
     hi = __byte_perm(__float_as_uint(f2), __float_as_uint(f3), 0x7632);
+}
+// eight int8 codes (two words) -> eight bf16 (one 16-byte chunk)
+__device__ __forceinline__ uint4 expand8(uint2 c) {
+    uint4 o;
+    codes4_to_bf16(c.x, o.x, o.y);
+    codes4_to_bf16(c.y, o.z, o.w);
+    return o;
 }
 __device__ __forceinline__ unsigned short code_to_bf16(int c) {
     return static_cast<unsigned short>(__float_as_uint(static_cast<float>(c)) >> 16);

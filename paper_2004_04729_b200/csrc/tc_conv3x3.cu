@@ -47,13 +47,6 @@ __device__ __forceinline__ uint2 bytes8(const unsigned *row, int off) {
     return make_uint2(__byte_perm(w0, w1, sel), __byte_perm(w1, w2, sel));
 }
 
-__device__ __forceinline__ uint4 expand8(uint2 c) {
-    uint4 o;
-    codes4_to_bf16(c.x, o.x, o.y);
-    codes4_to_bf16(c.y, o.z, o.w);
-    return o;
-}
-
 // One 32-bit word (four positions a..a+3 of plane `plane`) of the staged code tile; zero
 // outside [0, P). Planes start 4-byte aligned when P % 4 == 0.
 __device__ __forceinline__ unsigned load_code_word(const int8_t *plane, int a, int P, bool row_ok, bool aligned4) {

@@ -1,4 +1,5 @@
-// Dense tensor-core path for the two backward products of 1x1 convolutions and linear layers
+// Dense tensor-core path for 1x1 convolutions and linear layers: the input-gradient product
+// (the weight-gradient product lives in tc_dw1x1.cu).
 // with bf16 operands (the fallback above the density crossover): the int8 codes are expanded
 // to bf16 on the fly (exact: |q| <= 127) and the products run on the 5th-generation tensor
 // cores (tcgen05.mma, fp32 accumulators in tensor memory).
@@ -55,20 +56,6 @@ __device__ __forceinline__ uint4 load8_codes(const int8_t *codes, long long C, l
     return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
 }
 
-__device__ __forceinline__ uint4 load8_bf16_slow(const __nv_bfloat16 *x, long long C, long long P, long long rows,
-                                                 long long ch, long long r0, const RowCursor &cur) {
-    if (r0 >= rows) return make_uint4(0u, 0u, 0u, 0u);
-    const unsigned short *src = reinterpret_cast<const unsigned short *>(x);
-    unsigned short h[8];
-    long long b = cur.b, pp = cur.p;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        h[j] = (r0 + j < rows) ? __ldg(src + (b * C + ch) * P + pp) : 0;
-        if (++pp == P) { pp = 0; ++b; }
-    }
-    return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
-}
-
 struct TcParams {
     const int8_t *codes;          // [B][Cout][P]
     const __nv_bfloat16 *X;       // [B][Cin][P]      (dW)
@@ -101,137 +88,6 @@ __device__ __forceinline__ void pipe_setup(Pipe &pipe, int stages, int full_coun
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-}
-
-// ---------------------------------------------------------------- dW: M = co, N = ci, K = rows
-// Both operands K-major: 128 (co) and NT (ci) rows of 64 consecutive flattened rows r.
-template <int NT, bool FAST>
-__global__ void __launch_bounds__(kThreads) tc_dw_kernel(const TcParams p) {
-    constexpr int A_BYTES = 128 * 128;
-    constexpr int B_BYTES = NT * 128;
-    constexpr int STAGE = A_BYTES + B_BYTES;
-    extern __shared__ __align__(1024) unsigned char smem_raw[];
-    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    __shared__ Pipe pipe;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int co0 = blockIdx.x * 128, ci0 = blockIdx.y * NT;
-    const long long ks0 = blockIdx.z * p.per_split;
-    long long ks1 = ks0 + p.per_split;
-    if (ks1 > p.kstages) ks1 = p.kstages;
-    const int niter = ks1 > ks0 ? static_cast<int>(ks1 - ks0) : 0;
-    const int stages = p.stages;
-
-    pipe_setup(pipe, stages, FAST ? 2 * kProducers : kProducers, warp, NT);
-    const unsigned tmem_d = pipe.tmem_base;
-
-    if (warp < kProducerWarps) {
-        // ---------------- producers: chunk (row, c8); c8 = tid % 8 is fixed for the thread
-        const int tid = threadIdx.x;
-        const int c8 = tid & 7, rsub = tid >> 3;
-        bool ok = true;
-        for (int it = 0; it < niter && ok; ++it) {
-            const int s = it % stages;
-            ok = mbar_wait(&pipe.empty[s], ((it / stages) & 1) ^ 1, p.err_flag);
-            unsigned char *a_s = smem + s * STAGE, *b_s = a_s + A_BYTES;
-            const long long r0 = (ks0 + it) * kKT + c8 * 8;
-            const RowCursor cur(r0 < p.rows ? r0 : 0, p.P);
-            if (FAST) {   // X needs no conversion: asynchronous 16-byte copies
-                const bool row_ok = r0 < p.rows;
-                const __nv_bfloat16 *src = p.X + (cur.b * p.Cin + ci0) * p.P + cur.p;
-#pragma unroll 4
-                for (int row = rsub; row < NT; row += 16) {
-                    const bool v = row_ok && (ci0 + row < p.Cin);
-                    cp_async16(b_s + swz(row, c8), v ? src + row * p.P : p.X, v);
-                }
-                mbar_arrive_on_cp_async(&pipe.full[s]);
-            }
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {     // 4 loads in flight, then 4 stores
-                uint4 v[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int row = rsub + 16 * (half * 4 + i);
-                    const int co = co0 + row;
-                    v[i] = (co < p.Cout) ? load8_codes<FAST>(p.codes, p.Cout, p.P, p.rows, co, r0, cur)
-                                         : make_uint4(0u, 0u, 0u, 0u);
-                }
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    *reinterpret_cast<uint4 *>(a_s + swz(rsub + 16 * (half * 4 + i), c8)) = v[i];
-            }
-            if (!FAST) {
-#pragma unroll 2
-                for (int row = rsub; row < NT; row += 16) {
-                    const int ci = ci0 + row;
-                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                    if (ci < p.Cin) v = load8_bf16_slow(p.X, p.Cin, p.P, p.rows, ci, r0, cur);
-                    *reinterpret_cast<uint4 *>(b_s + swz(row, c8)) = v;
-                }
-            }
-            fence_async_proxy();
-            mbar_arrive(&pipe.full[s]);
-        }
-        // ---------------- epilogue: lanes = co rows, columns = ci -> partial block of this split
-        if (niter > 0 && mbar_wait(&pipe.acc, 0, p.err_flag)) {
-            tc_fence_after();
-            const int co = co0 + warp * 32 + lane;
-            float *dst_row = p.partials + (static_cast<long long>(blockIdx.z) * p.Cout + co) * p.Cin + ci0;
-#pragma unroll 1
-            for (int c0 = 0; c0 < NT; c0 += 32) {
-                unsigned r[32];
-                tmem_ld32(tmem_d + (static_cast<unsigned>(warp * 32) << 16) + c0, r);
-                if (co < p.Cout) {
-                    if (ci0 + c0 + 32 <= p.Cin) {   // Cin % 8 == 0 and ci0 % 64 == 0: 16-byte aligned
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4)
-                            *reinterpret_cast<uint4 *>(dst_row + c0 + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (ci0 + c0 + j < p.Cin) dst_row[c0 + j] = __uint_as_float(r[j]);
-                    }
-                }
-            }
-        }
-    } else if (lane == 0) {
-        // ---------------- MMA issuer
-        constexpr unsigned idesc = make_idesc(128, NT, false, false);
-        bool ok = true;
-        for (int it = 0; it < niter && ok; ++it) {
-            const int s = it % stages;
-            ok = mbar_wait(&pipe.full[s], (it / stages) & 1, p.err_flag);
-            fence_async_proxy();
-            tc_fence_after();
-            const unsigned a_addr = smem_u32(smem + s * STAGE), b_addr = a_addr + A_BYTES;
-            const unsigned long long ad = make_desc(a_addr, 16, 1024), bd = make_desc(b_addr, 16, 1024);
-#pragma unroll
-            for (int k = 0; k < kKT / 16; ++k)     // 32 bytes further along K per MMA
-                mma_bf16(tmem_d, ad + 2 * k, bd + 2 * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
-            mma_commit(&pipe.empty[s]);
-        }
-        if (niter > 0) mma_commit(&pipe.acc);
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == kProducerWarps) {
-        __syncwarp();
-        tmem_dealloc(tmem_d, NT);
-    }
-}
-
-// dW = Delta * sum over splits of the partial blocks
-__global__ void __launch_bounds__(256) tc_dw_reduce_kernel(const float *__restrict__ partials, int ksplit,
-                                                           long long n, const float *__restrict__ delta_p,
-                                                           float *__restrict__ dW) {
-    const float delta = *delta_p;
-    for (long long i = (blockIdx.x * 256ll + threadIdx.x) * 4; i < n; i += gridDim.x * 1024ll) {
-        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s = 0; s < ksplit; ++s) {
-            const float4 v = __ldcs(reinterpret_cast<const float4 *>(partials + s * n + i));
-            a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
-        }
-        *reinterpret_cast<float4 *>(dW + i) = make_float4(a.x * delta, a.y * delta, a.z * delta, a.w * delta);
-    }
 }
 
 // ---------------------------------------------------------------- dX: M = rows, N = ci, K = co
@@ -386,13 +242,6 @@ int set_smem(K kern, size_t bytes) {
 }
 
 template <int NT, bool FAST>
-int run_dw(dbp_ctx *ctx, const TcParams &p, dim3 grid, size_t smem) {
-    int rc = set_smem(tc_dw_kernel<NT, FAST>, smem);
-    if (rc) return rc;
-    tc_dw_kernel<NT, FAST><<<grid, kThreads, smem, ctx->stream>>>(p);
-    return cuda_ok(cudaGetLastError());
-}
-template <int NT, bool FAST>
 int run_dx(dbp_ctx *ctx, const TcParams &p, dim3 grid, size_t smem) {
     int rc = set_smem(tc_dx_kernel<NT, FAST>, smem);
     if (rc) return rc;
@@ -404,44 +253,6 @@ int run_dx(dbp_ctx *ctx, const TcParams &p, dim3 grid, size_t smem) {
 
 bool tc_supported(const ConvShape &s, int io) {
     return io == DBP_BF16 && s.k == 1 && s.Cin % 8 == 0;
-}
-
-int launch_tc_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *delta_p,
-                 const ConvShape &s, float *dW, int *err_flag) {
-    TcParams p{};
-    p.codes = codes; p.X = static_cast<const __nv_bfloat16 *>(X); p.delta_p = delta_p;
-    p.Cin = static_cast<int>(s.Cin); p.Cout = static_cast<int>(s.Cout);
-    p.P = s.H * s.W; p.rows = s.B * p.P;
-    p.kstages = (p.rows + kKT - 1) / kKT;
-    p.err_flag = err_flag;
-    const int nt = s.Cin >= 256 ? 256 : s.Cin > 64 ? 128 : 64;
-    const long long tiles = ((s.Cout + 127) / 128) * ((s.Cin + nt - 1) / nt);
-    // split K so that every SM has a CTA, without empty splits
-    long long split = (ctx->sm_count + tiles - 1) / tiles;
-    if (split > p.kstages) split = p.kstages;
-    if (split < 1) split = 1;
-    p.per_split = (p.kstages + split - 1) / split;
-    split = (p.kstages + p.per_split - 1) / p.per_split;
-    p.ksplit = static_cast<int>(split);
-    p.stages = p.per_split < kMaxStages ? static_cast<int>(p.per_split) : kMaxStages;
-    const size_t nw = static_cast<size_t>(s.Cout) * s.Cin;
-    int rc = ws_reserve(ctx, ctx->tc_partials, sizeof(float) * nw * split);
-    if (rc) return rc;
-    p.partials = static_cast<float *>(ctx->tc_partials.ptr);
-    dim3 grid(static_cast<unsigned>((s.Cout + 127) / 128), static_cast<unsigned>((s.Cin + nt - 1) / nt),
-              static_cast<unsigned>(split));
-    const size_t smem = static_cast<size_t>(p.stages) * (128 * 128 + nt * 128) + 1024;
-    const bool fast = p.P % 8 == 0;
-    if (nt == 256) rc = fast ? run_dw<256, true>(ctx, p, grid, smem) : run_dw<256, false>(ctx, p, grid, smem);
-    else if (nt == 128) rc = fast ? run_dw<128, true>(ctx, p, grid, smem) : run_dw<128, false>(ctx, p, grid, smem);
-    else rc = fast ? run_dw<64, true>(ctx, p, grid, smem) : run_dw<64, false>(ctx, p, grid, smem);
-    if (rc) return rc;
-    long long blocks = (static_cast<long long>(nw) / 4 + 255) / 256;
-    if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
-    if (blocks < 1) blocks = 1;
-    tc_dw_reduce_kernel<<<static_cast<unsigned>(blocks), 256, 0, ctx->stream>>>(
-        p.partials, p.ksplit, static_cast<long long>(nw), delta_p, dW);   // Cout*Cin % 4 == 0 since Cin % 8 == 0
-    return cuda_ok(cudaGetLastError());
 }
 
 int launch_tc_dx(dbp_ctx *ctx, const int8_t *codes, const void *W, const float *delta_p,

@@ -1,0 +1,281 @@
+// Dense tensor-core weight gradient of 1x1 convolutions and linear layers, bf16 operands:
+//   dW[co][ci] = Delta * sum_r q[r,co] X[r,ci],   r = (image, position) flattened
+//   M = co (128), N = ci (NT), K = rows in stages of 64; both operands K-major.
+//
+// The kernel is bound by HBM (every byte of X and of the codes is read once), so its pipeline
+// is built to keep many bytes in flight per SM: all global reads are cp.async copies issued
+// several stages ahead -- X straight into its 128-byte-swizzled operand tile, the int8 codes
+// into a raw staging tile -- and tracked by mbarriers; the eight producer warps then expand
+// the staged codes to bf16 from shared memory (no global latency on that path) while the next
+// stages' copies are already under way. A ninth warp issues the MMAs. K is split across CTAs;
+// partial blocks go to a workspace and a small kernel sums them and applies Delta.
+#include "tc_common.cuh"
+
+namespace dbp {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kPW = 8;
+constexpr int kP = kPW * 32;
+constexpr int kThreadsDw = kP + 32;
+constexpr int kMaxS = 4;
+constexpr int kKT = 64;
+
+struct DwP {
+    const int8_t *codes;          // [B][Cout][P]
+    const __nv_bfloat16 *X;       // [B][Cin][P]
+    float *partials;              // [ksplit][Cout][Cin]
+    int Cin, Cout;
+    long long P, rows;
+    int stages;
+    long long kstages, per_split;
+    int *err_flag;
+};
+
+struct PipeDw {
+    unsigned long long load_full[kMaxS], full[kMaxS], empty[kMaxS], acc;
+    unsigned tmem_base;
+};
+
+// G = rows per aligned, image-contained group: 8 (P % 8 == 0), 4 (P % 4 == 0) or 1 (any P).
+template <int NT, int G>
+__global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
+    constexpr int A_BYTES = 128 * 128;
+    constexpr int B_BYTES = NT * 128;
+    constexpr int RAW_BYTES = 128 * 64;
+    constexpr int STAGE = A_BYTES + B_BYTES + RAW_BYTES;
+    constexpr int NGRP = 8 / G;
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ PipeDw pipe;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int co0 = blockIdx.x * 128, ci0 = blockIdx.y * NT;
+    const long long ks0 = blockIdx.z * p.per_split;
+    long long ks1 = ks0 + p.per_split;
+    if (ks1 > p.kstages) ks1 = p.kstages;
+    const int niter = ks1 > ks0 ? static_cast<int>(ks1 - ks0) : 0;
+    const int S = p.stages, LA = S - 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(&pipe.load_full[s], kP);
+            mbar_init(&pipe.full[s], kP);
+            mbar_init(&pipe.empty[s], 1);
+        }
+        mbar_init(&pipe.acc, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kPW) tmem_alloc(&pipe.tmem_base, NT);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const unsigned tmem_d = pipe.tmem_base;
+
+    if (warp < kPW) {
+        const int tid = threadIdx.x;
+        const int c8 = tid & 7, rsub = tid >> 3;      // chunk column, first of my rows (stride 32)
+        bool ok = true;
+        // copies of local stage j: X chunks into the operand tile, code bytes into the raw tile
+        auto issue = [&](int j) {
+            const int s = j % S;
+            ok = ok && mbar_wait(&pipe.empty[s], ((j / S) & 1) ^ 1, p.err_flag);
+            unsigned char *st = smem + s * STAGE;
+            unsigned char *b_s = st + A_BYTES, *raw = b_s + B_BYTES;
+            const long long r0 = (ks0 + j) * kKT + c8 * 8;
+            long long gb[NGRP > 2 ? 1 : NGRP], gp[NGRP > 2 ? 1 : NGRP];
+            if (G > 1) {
+#pragma unroll
+                for (int g = 0; g < NGRP; ++g) {
+                    const long long r = r0 + g * G;
+                    gb[g] = r < p.rows ? r / p.P : -1;
+                    gp[g] = r < p.rows ? r - gb[g] * p.P : 0;
+                }
+#pragma unroll
+                for (int i = 0; i < NT / 32; ++i) {
+                    const int row = rsub + 32 * i, ci = ci0 + row;
+#pragma unroll
+                    for (int g = 0; g < NGRP; ++g) {
+                        const bool v = gb[g] >= 0 && ci < p.Cin;
+                        const __nv_bfloat16 *src = v ? p.X + (gb[g] * p.Cin + ci) * p.P + gp[g] : p.X;
+                        if (G == 8) cp_async16(b_s + swz(row, c8), src, v);
+                        else cp_async_small<8>(b_s + swz(row, c8) + g * 8, src, v);
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int row = rsub + 32 * i, co = co0 + row;
+#pragma unroll
+                    for (int g = 0; g < NGRP; ++g) {
+                        const bool v = gb[g] >= 0 && co < p.Cout;
+                        const int8_t *src = v ? p.codes + (gb[g] * p.Cout + co) * p.P + gp[g] : p.codes;
+                        if (G == 8) cp_async_small<8>(raw + row * 64 + c8 * 8, src, v);
+                        else cp_async_small<4>(raw + row * 64 + c8 * 8 + g * 4, src, v);
+                    }
+                }
+                mbar_arrive_on_cp_async(&pipe.load_full[s]);
+            } else {
+                // element-wise: walk the eight rows from (b, p)
+                const long long rr = r0 < p.rows ? r0 : 0;
+                const long long b0 = rr / p.P, q0 = rr - b0 * p.P;
+                const unsigned short *xs = reinterpret_cast<const unsigned short *>(p.X);
+                for (int i = 0; i < NT / 32; ++i) {
+                    const int row = rsub + 32 * i, ci = ci0 + row;
+                    unsigned short h[8];
+                    long long b = b0, pp = q0;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        h[e] = (r0 + e < p.rows && ci < p.Cin) ? __ldg(xs + (b * p.Cin + ci) * p.P + pp) : 0;
+                        if (++pp == p.P) { pp = 0; ++b; }
+                    }
+                    *reinterpret_cast<uint4 *>(b_s + swz(row, c8)) =
+                        make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+                }
+                for (int i = 0; i < 4; ++i) {
+                    const int row = rsub + 32 * i, co = co0 + row;
+                    unsigned w[2] = {0u, 0u};
+                    long long b = b0, pp = q0;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        if (r0 + e < p.rows && co < p.Cout)
+                            w[e >> 2] |= (static_cast<unsigned>(__ldg(p.codes + (b * p.Cout + co) * p.P + pp)) & 0xffu) << (8 * (e & 3));
+                        if (++pp == p.P) { pp = 0; ++b; }
+                    }
+                    *reinterpret_cast<uint2 *>(raw + row * 64 + c8 * 8) = make_uint2(w[0], w[1]);
+                }
+                mbar_arrive(&pipe.load_full[s]);
+            }
+        };
+        for (int j = 0; j < LA && j < niter; ++j) issue(j);
+        for (int it = 0; it < niter; ++it) {
+            if (it + LA < niter) issue(it + LA);
+            const int s = it % S;
+            ok = ok && mbar_wait(&pipe.load_full[s], (it / S) & 1, p.err_flag);
+            unsigned char *a_s = smem + s * STAGE, *raw = a_s + A_BYTES + B_BYTES;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int row = rsub + 32 * i;
+                const uint2 c = *reinterpret_cast<const uint2 *>(raw + row * 64 + c8 * 8);
+                *reinterpret_cast<uint4 *>(a_s + swz(row, c8)) = expand8(c);
+            }
+            fence_async_proxy();
+            mbar_arrive(&pipe.full[s]);
+        }
+        // ---------------- epilogue: lanes = co rows, columns = ci -> partial block of this split
+        if (niter > 0 && mbar_wait(&pipe.acc, 0, p.err_flag)) {
+            tc_fence_after();
+            const int q = warp & 3, half = warp >> 2;
+            const int co = co0 + q * 32 + lane;
+            float *dst_row = p.partials + (static_cast<long long>(blockIdx.z) * p.Cout + co) * p.Cin + ci0;
+#pragma unroll 1
+            for (int c0 = half * (NT / 2); c0 < (half + 1) * (NT / 2); c0 += 32) {
+                unsigned r[32];
+                tmem_ld32(tmem_d + (static_cast<unsigned>(q * 32) << 16) + c0, r);
+                if (co < p.Cout) {
+                    if (ci0 + c0 + 32 <= p.Cin) {   // Cin % 8 == 0, ci0 % 64 == 0: 16-byte aligned
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<uint4 *>(dst_row + c0 + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (ci0 + c0 + j < p.Cin) dst_row[c0 + j] = __uint_as_float(r[j]);
+                    }
+                }
+            }
+        }
+    } else if (lane == 0) {
+        constexpr unsigned idesc = make_idesc(128, NT, false, false);
+        bool ok = true;
+        for (int it = 0; it < niter && ok; ++it) {
+            const int s = it % S;
+            ok = mbar_wait(&pipe.full[s], (it / S) & 1, p.err_flag);
+            fence_async_proxy();
+            tc_fence_after();
+            const unsigned a_addr = smem_u32(smem + s * STAGE), b_addr = a_addr + A_BYTES;
+            const unsigned long long ad = make_desc(a_addr, 16, 1024), bd = make_desc(b_addr, 16, 1024);
+#pragma unroll
+            for (int k = 0; k < kKT / 16; ++k)
+                mma_bf16(tmem_d, ad + 2 * k, bd + 2 * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
+            mma_commit(&pipe.empty[s]);
+        }
+        if (niter > 0) mma_commit(&pipe.acc);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kPW) {
+        __syncwarp();
+        tmem_dealloc(tmem_d, NT);
+    }
+}
+
+// dW = Delta * sum over splits of the partial blocks
+__global__ void __launch_bounds__(256) tc_dw_sum_kernel(const float *__restrict__ partials, int ksplit,
+                                                        long long n, const float *__restrict__ delta_p,
+                                                        float *__restrict__ dW) {
+    const float delta = *delta_p;
+    for (long long i = (blockIdx.x * 256ll + threadIdx.x) * 4; i < n; i += gridDim.x * 1024ll) {
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s = 0; s < ksplit; ++s) {
+            const float4 v = __ldcs(reinterpret_cast<const float4 *>(partials + s * n + i));
+            a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+        }
+        *reinterpret_cast<float4 *>(dW + i) = make_float4(a.x * delta, a.y * delta, a.z * delta, a.w * delta);
+    }
+}
+
+template <int NT, int G>
+int run(dbp_ctx *ctx, const DwP &p, dim3 grid, size_t smem) {
+    if (cudaFuncSetAttribute(tc_dw_async_kernel<NT, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(smem)) != cudaSuccess)
+        return DBP_ECUDA;
+    tc_dw_async_kernel<NT, G><<<grid, kThreadsDw, smem, ctx->stream>>>(p);
+    return cuda_ok(cudaGetLastError());
+}
+
+template <int NT>
+int run_g(dbp_ctx *ctx, const DwP &p, dim3 grid, size_t smem) {
+    if (p.P % 8 == 0) return run<NT, 8>(ctx, p, grid, smem);
+    if (p.P % 4 == 0) return run<NT, 4>(ctx, p, grid, smem);
+    return run<NT, 1>(ctx, p, grid, smem);
+}
+
+}  // namespace
+
+int launch_tc_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *delta_p,
+                 const ConvShape &s, float *dW, int *err_flag) {
+    DwP p{};
+    p.codes = codes; p.X = static_cast<const __nv_bfloat16 *>(X);
+    p.Cin = static_cast<int>(s.Cin); p.Cout = static_cast<int>(s.Cout);
+    p.P = s.H * s.W; p.rows = s.B * p.P;
+    p.kstages = (p.rows + kKT - 1) / kKT;
+    p.err_flag = err_flag;
+    const int nt = s.Cin >= 256 ? 256 : s.Cin > 64 ? 128 : 64;
+    const long long tiles = ((s.Cout + 127) / 128) * ((s.Cin + nt - 1) / nt);
+    // split K so that every SM has a CTA, without empty splits
+    long long split = (ctx->sm_count + tiles - 1) / tiles;
+    if (split > p.kstages) split = p.kstages;
+    if (split < 1) split = 1;
+    p.per_split = (p.kstages + split - 1) / split;
+    split = (p.kstages + p.per_split - 1) / p.per_split;
+    const int max_s = nt == 256 ? 3 : kMaxS;
+    p.stages = p.per_split < max_s ? static_cast<int>(p.per_split) : max_s;
+    const size_t nw = static_cast<size_t>(s.Cout) * s.Cin;
+    int rc = ws_reserve(ctx, ctx->tc_partials, sizeof(float) * nw * split);
+    if (rc) return rc;
+    p.partials = static_cast<float *>(ctx->tc_partials.ptr);
+    dim3 grid(static_cast<unsigned>((s.Cout + 127) / 128), static_cast<unsigned>((s.Cin + nt - 1) / nt),
+              static_cast<unsigned>(split));
+    const size_t smem = static_cast<size_t>(p.stages) * (128 * 128 + nt * 128 + 128 * 64) + 1024;
+    rc = nt == 256 ? run_g<256>(ctx, p, grid, smem) : nt == 128 ? run_g<128>(ctx, p, grid, smem) : run_g<64>(ctx, p, grid, smem);
+    if (rc) return rc;
+    long long blocks = (static_cast<long long>(nw) / 4 + 255) / 256;
+    if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
+    if (blocks < 1) blocks = 1;
+    tc_dw_sum_kernel<<<static_cast<unsigned>(blocks), 256, 0, ctx->stream>>>(
+        p.partials, static_cast<int>(split), static_cast<long long>(nw), delta_p, dW);   // Cout*Cin % 4 == 0
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace dbp
