@@ -1,0 +1,280 @@
+// Dense tensor-core input gradient of 1x1 convolutions and linear layers, bf16 operands:
+//   dX[r][ci] = Delta * sum_co q[r,co] W[co,ci],   r = (image, position) flattened
+//   M = 128 rows r, N = ci (NT), K = co in stages of 64; both operands MN-major
+//   (a k-row holds 64 consecutive rows r / 64 consecutive input channels).
+//
+// Bound by HBM: the codes are read once and dX is written once. All global reads are cp.async
+// copies issued ahead of use (weights straight into their swizzled operand tile, code bytes
+// into a raw staging tile); eight producer warps expand the staged codes to bf16 from shared
+// memory; a ninth warp issues the MMAs. The accumulator leaves through per-warp shared-memory
+// patches so that each lane stores a contiguous run of positions of one channel.
+#include "tc_common.cuh"
+
+namespace dbp {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kPW = 8;
+constexpr int kP = kPW * 32;
+constexpr int kThreadsDx = kP + 32;
+constexpr int kMaxS = 4;
+constexpr int kKT = 64;
+constexpr int kPatchCol = 192;                 // bytes per column of an epilogue patch
+constexpr int kPatch = 32 * kPatchCol;         // one warp's 32 columns x 32 rows
+
+struct DxP {
+    const int8_t *codes;          // [B][Cout][P]
+    const __nv_bfloat16 *W;       // [Cout][Cin]
+    const float *delta_p;
+    void *dX;                     // [B][Cin][P], bf16 or fp32
+    int dx_f32;
+    int Cin, Cout;
+    long long P, rows;
+    int stages;
+    int *err_flag;
+};
+
+struct PipeDx {
+    unsigned long long load_full[kMaxS], full[kMaxS], empty[kMaxS], acc;
+    unsigned tmem_base;
+};
+
+template <int BYTES>
+__device__ __forceinline__ void store_bytes(void *dst, const unsigned char *src) {
+    if (BYTES == 16) *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
+    else if (BYTES == 8) *reinterpret_cast<uint2 *>(dst) = *reinterpret_cast<const uint2 *>(src);
+    else if (BYTES == 4) *reinterpret_cast<unsigned *>(dst) = *reinterpret_cast<const unsigned *>(src);
+    else *reinterpret_cast<unsigned short *>(dst) = *reinterpret_cast<const unsigned short *>(src);
+}
+
+// One warp's 32 rows x 32 columns patch -> global: a lane stores RL consecutive rows (one
+// aligned, image-contained group) of one column.
+template <int ES, int RL>
+__device__ __forceinline__ void store_patch(const unsigned char *patch, const DxP &p, int lane, long long row_first,
+                                            int ci_first) {
+    constexpr int LPC = 32 / RL;               // lanes per column
+    constexpr int CPP = 32 / LPC;              // columns per pass
+    const int rr = (lane % LPC) * RL;
+    const long long r = row_first + rr;
+    if (r >= p.rows) return;
+    const long long b = r / p.P, pp = r - b * p.P;
+    unsigned char *base = static_cast<unsigned char *>(p.dX) + ((b * p.Cin) * p.P + pp) * ES;
+#pragma unroll 4
+    for (int cb = 0; cb < 32; cb += CPP) {
+        const int j = cb + lane / LPC;
+        const int ci = ci_first + j;
+        if (ci < p.Cin) store_bytes<RL * ES>(base + static_cast<long long>(ci) * p.P * ES, patch + j * kPatchCol + rr * ES);
+    }
+}
+
+// G = rows per aligned, image-contained group: 8 (P % 8 == 0), 4 (P % 4 == 0) or 1 (any P).
+template <int NT, int G>
+__global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
+    constexpr int A_BYTES = 2 * kKT * 128;          // two 64-row groups x 64 k-rows
+    constexpr int B_BYTES = (NT / 64) * kKT * 128;
+    constexpr int RAW_BYTES = kKT * 128;            // 64 co x 128 rows, one byte each
+    constexpr int STAGE = A_BYTES + B_BYTES + RAW_BYTES;
+    constexpr unsigned PANEL = kKT * 128;
+    constexpr int NGRP = 8 / G;
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ PipeDx pipe;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long row0 = static_cast<long long>(blockIdx.x) * 128;
+    const int ci0 = blockIdx.y * NT;
+    const int niter = (p.Cout + kKT - 1) / kKT;
+    const int S = p.stages, LA = S - 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(&pipe.load_full[s], kP);
+            mbar_init(&pipe.full[s], kP);
+            mbar_init(&pipe.empty[s], 1);
+        }
+        mbar_init(&pipe.acc, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kPW) tmem_alloc(&pipe.tmem_base, NT);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const unsigned tmem_d = pipe.tmem_base;
+
+    if (warp < kPW) {
+        const int tid = threadIdx.x;
+        const int c16 = tid & 15, ksub = tid >> 4;     // my 8-row chunk of the tile, first k-row (stride 16)
+        // where my chunk's groups live: the same for every stage
+        const long long r0 = row0 + c16 * 8;
+        long long gbase[NGRP > 2 ? 1 : NGRP];          // offset of (image, position) in channel 0, or -1
+        if (G > 1) {
+#pragma unroll
+            for (int g = 0; g < NGRP; ++g) {
+                const long long r = r0 + g * G;
+                const long long b = r / p.P;
+                gbase[g] = r < p.rows ? b * p.Cout * p.P + (r - b * p.P) : -1;
+            }
+        }
+        const long long rr0 = r0 < p.rows ? r0 : 0;
+        const long long b0 = rr0 / p.P, q0 = rr0 - b0 * p.P;
+        bool ok = true;
+        auto issue = [&](int j) {
+            const int s = j % S;
+            ok = ok && mbar_wait(&pipe.empty[s], ((j / S) & 1) ^ 1, p.err_flag);
+            unsigned char *st = smem + s * STAGE;
+            unsigned char *b_s = st + A_BYTES, *raw = b_s + B_BYTES;
+            // weights: k-row = co, 64-channel groups; 64 x (NT/8) chunks of 16 bytes
+#pragma unroll
+            for (int i = 0; i < (kKT * NT / 8) / kP; ++i) {
+                const int idx = tid + i * kP;
+                const int k = idx / (NT / 8), cc = idx - k * (NT / 8);
+                const int co = j * kKT + k, ci = ci0 + cc * 8;
+                const bool v = co < p.Cout && ci < p.Cin;     // Cin % 8 == 0
+                cp_async16(b_s + (cc >> 3) * PANEL + swz(k, cc & 7), v ? p.W + static_cast<long long>(co) * p.Cin + ci : p.W, v);
+            }
+            // code bytes: k-row = co, my chunk of 8 rows
+            if (G > 1) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int k = ksub + 16 * i, co = j * kKT + k;
+#pragma unroll
+                    for (int g = 0; g < NGRP; ++g) {
+                        const bool v = gbase[g] >= 0 && co < p.Cout;
+                        const int8_t *src = v ? p.codes + gbase[g] + co * p.P : p.codes;
+                        if (G == 8) cp_async_small<8>(raw + k * 128 + c16 * 8, src, v);
+                        else cp_async_small<4>(raw + k * 128 + c16 * 8 + g * 4, src, v);
+                    }
+                }
+                mbar_arrive_on_cp_async(&pipe.load_full[s]);
+            } else {
+                for (int i = 0; i < 4; ++i) {
+                    const int k = ksub + 16 * i, co = j * kKT + k;
+                    unsigned w[2] = {0u, 0u};
+                    long long b = b0, pp = q0;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        if (r0 + e < p.rows && co < p.Cout)
+                            w[e >> 2] |= (static_cast<unsigned>(__ldg(p.codes + (b * p.Cout + co) * p.P + pp)) & 0xffu) << (8 * (e & 3));
+                        if (++pp == p.P) { pp = 0; ++b; }
+                    }
+                    *reinterpret_cast<uint2 *>(raw + k * 128 + c16 * 8) = make_uint2(w[0], w[1]);
+                }
+                // the weight copies above are still asynchronous: count them, then arrive
+                asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
+                mbar_arrive(&pipe.load_full[s]);
+            }
+        };
+        for (int j = 0; j < LA && j < niter; ++j) issue(j);
+        for (int it = 0; it < niter; ++it) {
+            if (it + LA < niter) issue(it + LA);
+            const int s = it % S;
+            ok = ok && mbar_wait(&pipe.load_full[s], (it / S) & 1, p.err_flag);
+            unsigned char *a_s = smem + s * STAGE, *raw = a_s + A_BYTES + B_BYTES;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int k = ksub + 16 * i;
+                const uint2 c = *reinterpret_cast<const uint2 *>(raw + k * 128 + c16 * 8);
+                *reinterpret_cast<uint4 *>(a_s + (c16 >> 3) * PANEL + swz(k, c16 & 7)) = expand8(c);
+            }
+            fence_async_proxy();
+            mbar_arrive(&pipe.full[s]);
+        }
+        // ---------------- epilogue: TMEM lanes = rows, columns = ci. Warp w: rows 32 (w % 4) ...,
+        // column half w / 4. All MMAs are complete, so the stage buffers hold the patches.
+        if (mbar_wait(&pipe.acc, 0, p.err_flag)) {
+            tc_fence_after();
+            const float delta = *p.delta_p;
+            const int q = warp & 3, half = warp >> 2;
+            unsigned char *patch = smem + warp * kPatch;
+            const long long row_first = row0 + q * 32;
+#pragma unroll 1
+            for (int c0 = half * (NT / 2); c0 < (half + 1) * (NT / 2); c0 += 32) {
+                unsigned v[32];
+                tmem_ld32(tmem_d + (static_cast<unsigned>(q * 32) << 16) + c0, v);
+                if (ci0 + c0 < p.Cin) {                       // warp-uniform
+                    if (p.dx_f32) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            *reinterpret_cast<float *>(patch + j * kPatchCol + lane * 4) = __uint_as_float(v[j]) * delta;
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            *reinterpret_cast<unsigned short *>(patch + j * kPatchCol + lane * 2) =
+                                __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(v[j]) * delta));
+                    }
+                    __syncwarp();
+                    if (p.dx_f32) store_patch<4, (G >= 4 ? 4 : 1)>(patch, p, lane, row_first, ci0 + c0);
+                    else store_patch<2, G>(patch, p, lane, row_first, ci0 + c0);
+                    __syncwarp();
+                }
+            }
+        }
+    } else if (lane == 0) {
+        constexpr unsigned idesc = make_idesc(128, NT, true, true);
+        bool ok = true;
+        for (int it = 0; it < niter && ok; ++it) {
+            const int s = it % S;
+            ok = mbar_wait(&pipe.full[s], (it / S) & 1, p.err_flag);
+            fence_async_proxy();
+            tc_fence_after();
+            const unsigned a_addr = smem_u32(smem + s * STAGE), b_addr = a_addr + A_BYTES;
+            const unsigned long long ad = make_desc(a_addr, PANEL, 1024), bd = make_desc(b_addr, PANEL, 1024);
+#pragma unroll
+            for (int k = 0; k < kKT / 16; ++k)     // 16 k-rows = two 1024-byte groups further per MMA
+                mma_bf16(tmem_d, ad + 128 * k, bd + 128 * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
+            mma_commit(&pipe.empty[s]);
+        }
+        mma_commit(&pipe.acc);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kPW) {
+        __syncwarp();
+        tmem_dealloc(tmem_d, NT);
+    }
+}
+
+template <int NT, int G>
+int run(dbp_ctx *ctx, const DxP &p, dim3 grid, size_t smem) {
+    if (cudaFuncSetAttribute(tc_dx_async_kernel<NT, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(smem)) != cudaSuccess)
+        return DBP_ECUDA;
+    tc_dx_async_kernel<NT, G><<<grid, kThreadsDx, smem, ctx->stream>>>(p);
+    return cuda_ok(cudaGetLastError());
+}
+
+template <int NT>
+int run_g(dbp_ctx *ctx, const DxP &p, dim3 grid, size_t smem) {
+    if (p.P % 8 == 0) return run<NT, 8>(ctx, p, grid, smem);
+    if (p.P % 4 == 0) return run<NT, 4>(ctx, p, grid, smem);
+    return run<NT, 1>(ctx, p, grid, smem);
+}
+
+}  // namespace
+
+bool tc_supported(const ConvShape &s, int io) {
+    return io == DBP_BF16 && s.k == 1 && s.Cin % 8 == 0;
+}
+
+int launch_tc_dx(dbp_ctx *ctx, const int8_t *codes, const void *W, const float *delta_p,
+                 const ConvShape &s, void *dX, bool dx_bf16, int *err_flag) {
+    DxP p{};
+    p.codes = codes; p.W = static_cast<const __nv_bfloat16 *>(W); p.delta_p = delta_p; p.dX = dX;
+    p.dx_f32 = dx_bf16 ? 0 : 1;
+    p.Cin = static_cast<int>(s.Cin); p.Cout = static_cast<int>(s.Cout);
+    p.P = s.H * s.W; p.rows = s.B * p.P;
+    p.err_flag = err_flag;
+    const int niter = static_cast<int>((s.Cout + kKT - 1) / kKT);
+    p.stages = niter < kMaxS ? niter : kMaxS;
+    // narrow N tiles leave room for several CTAs per SM, which overlaps the load, MMA and
+    // store phases of different tiles
+    const int nt = s.Cin > 64 ? 128 : 64;
+    dim3 grid(static_cast<unsigned>((p.rows + 127) / 128), static_cast<unsigned>((s.Cin + nt - 1) / nt));
+    size_t smem = static_cast<size_t>(p.stages) * (2 * kKT * 128 + (nt / 64) * kKT * 128 + kKT * 128);
+    if (smem < static_cast<size_t>(kPW) * kPatch) smem = static_cast<size_t>(kPW) * kPatch;
+    smem += 1024;
+    return nt == 128 ? run_g<128>(ctx, p, grid, smem) : run_g<64>(ctx, p, grid, smem);
+}
+
+}  // namespace dbp
