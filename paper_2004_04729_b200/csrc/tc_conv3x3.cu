@@ -118,21 +118,17 @@ __global__ void __launch_bounds__(kThreads3) tc3_dx_kernel(const P3 p) {
 
     if (warp < kProdWarps) {
         const bool aligned4 = (p.P & 3) == 0;
-        const int total_words = 64 * p.raw_words;
+        // staged code tile: 64 rows x raw_words words; thread t owns row t/4, words t%4 + 4 i
+        const int rrow = threadIdx.x >> 2, rw0 = threadIdx.x & 3;
+        const int nword = (p.raw_words - rw0 + 3) >> 2;          // my words in a row (<= 17)
+        const int8_t *img_base = p.codes + static_cast<long long>(b) * p.Cout * p.P;
         unsigned pre[17];                          // staged-tile words of the next chunk
         auto fetch = [&](int c) {
+            const int co = c * 64 + rrow;
+            const int8_t *plane = img_base + static_cast<long long>(co < p.Cout ? co : 0) * p.P;
 #pragma unroll
-            for (int i = 0; i < 17; ++i) {
-                const int idx = threadIdx.x + i * kProd;
-                unsigned w = 0;
-                if (idx < total_words) {
-                    const int row = idx / p.raw_words, wd = idx - row * p.raw_words;
-                    const int co = c * 64 + row;
-                    const int8_t *plane = p.codes + (static_cast<long long>(b) * p.Cout + co) * p.P;
-                    w = load_code_word(plane, a0 + 4 * wd, p.P, co < p.Cout, aligned4);
-                }
-                pre[i] = w;
-            }
+            for (int i = 0; i < 17; ++i)
+                pre[i] = (i < nword) ? load_code_word(plane, a0 + 4 * (rw0 + 4 * i), p.P, co < p.Cout, aligned4) : 0u;
         };
         fetch(0);
         bool ok = true;
@@ -140,13 +136,8 @@ __global__ void __launch_bounds__(kThreads3) tc3_dx_kernel(const P3 p) {
         for (int c = 0; c < nchunks; ++c) {
             unsigned *raw = raw_s + (c & 1) * (64 * p.raw_pitch);
 #pragma unroll
-            for (int i = 0; i < 17; ++i) {
-                const int idx = threadIdx.x + i * kProd;
-                if (idx < total_words) {
-                    const int row = idx / p.raw_words, wd = idx - row * p.raw_words;
-                    raw[row * p.raw_pitch + wd] = pre[i];
-                }
-            }
+            for (int i = 0; i < 17; ++i)
+                if (i < nword) raw[rrow * p.raw_pitch + rw0 + 4 * i] = pre[i];
             asm volatile("bar.sync 1, %0;" ::"n"(kProd) : "memory");
             if (c + 1 < nchunks) fetch(c + 1);
 #pragma unroll 1
@@ -325,94 +316,94 @@ __global__ void __launch_bounds__(kThreads3) tc3_dw_kernel(const P3 p) {
 
     if (warp < kProdWarps) {
         const bool aligned4 = (p.P & 3) == 0;
-        const int total_words = 32 * p.raw_words;
+        // staged code tile: 32 rows x raw_words words; thread t owns row t/8, words t%8 + 8 i
+        const int rrow = threadIdx.x >> 3, rw0 = threadIdx.x & 7;
+        const int nword = (p.raw_words - rw0 + 7) >> 3;         // my words in a row (<= 9)
+        const bool rrow_ok = co0 + rrow < p.Cout;
+        const int8_t *row_base = p.codes + static_cast<long long>(co0 + (rrow_ok ? rrow : 0)) * p.P;
+        const long long img_codes = static_cast<long long>(p.Cout) * p.P, img_x = static_cast<long long>(p.Cin) * p.P;
+        // X tile: my four 16-byte chunks are (row = t/8 + 32 i, chunk = t%8)
+        const int xch = threadIdx.x & 7;
+        // position of a stage: image and first position, advanced incrementally
+        int bimg = static_cast<int>(s0 / p.tiles_per_img);
+        int k0 = static_cast<int>(s0 - static_cast<long long>(bimg) * p.tiles_per_img) * 64;
+        int nb = bimg, nk0 = k0;                                 // the stage being prefetched
         unsigned pre[9];
-        auto stage_origin = [&](long long st, int &bimg, int &k0) {
-            bimg = static_cast<int>(st / p.tiles_per_img);
-            k0 = static_cast<int>(st - static_cast<long long>(bimg) * p.tiles_per_img) * 64;
-        };
-        auto fetch = [&](long long st) {
-            int bimg, k0;
-            stage_origin(st, bimg, k0);
-            const int a0 = ((k0 - halo) >> 2) << 2;
+        auto fetch = [&]() {
+            const int a0 = ((nk0 - halo) >> 2) << 2;
+            const int8_t *plane = row_base + nb * img_codes;
 #pragma unroll
-            for (int i = 0; i < 9; ++i) {
-                const int idx = threadIdx.x + i * kProd;
-                unsigned w = 0;
-                if (idx < total_words) {
-                    const int row = idx / p.raw_words, wd = idx - row * p.raw_words;
-                    const int co = co0 + row;
-                    const int8_t *plane = p.codes + (static_cast<long long>(bimg) * p.Cout + co) * p.P;
-                    w = load_code_word(plane, a0 + 4 * wd, p.P, co < p.Cout, aligned4);
-                }
-                pre[i] = w;
-            }
+            for (int i = 0; i < 9; ++i)
+                pre[i] = (i < nword) ? load_code_word(plane, a0 + 4 * (rw0 + 8 * i), p.P, rrow_ok, aligned4) : 0u;
         };
-        if (niter > 0) fetch(s0);
+        auto advance = [&](int &bb, int &kk) {
+            kk += 64;
+            if (kk >= p.tiles_per_img * 64) { kk = 0; ++bb; }
+        };
+        if (niter > 0) fetch();
         bool ok = true;
         for (int it = 0; it < niter; ++it) {
-            int bimg, k0;
-            stage_origin(s0 + it, bimg, k0);
             const int a0 = ((k0 - halo) >> 2) << 2;
             unsigned *raw = raw_s + (it & 1) * (32 * p.raw_pitch);
 #pragma unroll
-            for (int i = 0; i < 9; ++i) {
-                const int idx = threadIdx.x + i * kProd;
-                if (idx < total_words) {
-                    const int row = idx / p.raw_words, wd = idx - row * p.raw_words;
-                    raw[row * p.raw_pitch + wd] = pre[i];
-                }
-            }
+            for (int i = 0; i < 9; ++i)
+                if (i < nword) raw[rrow * p.raw_pitch + rw0 + 8 * i] = pre[i];
             asm volatile("bar.sync 1, %0;" ::"n"(kProd) : "memory");
-            if (it + 1 < niter) fetch(s0 + it + 1);
-            if (!ok) continue;       // a wait expired: keep the barrier count, skip the work
-            // ---- X tile: 128 ci rows x 8 chunks of 8 positions
-            const int sa = it % kNA;
-            ok = mbar_wait(&pipe.a_empty[sa], ((it / kNA) & 1) ^ 1, p.err_flag);
-            unsigned char *at = a_s + sa * A_TILE;
+            advance(nb, nk0);
+            if (it + 1 < niter) fetch();
+            if (ok) {
+                // ---- X tile: 128 ci rows x 8 chunks of 8 positions
+                const int sa = it % kNA;
+                ok = mbar_wait(&pipe.a_empty[sa], ((it / kNA) & 1) ^ 1, p.err_flag);
+                unsigned char *at = a_s + sa * A_TILE;
+                const int pp = k0 + xch * 8;
+                const __nv_bfloat16 *xsrc = p.X + bimg * img_x + pp;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int idx = threadIdx.x + i * kProd;
-                const int row = idx >> 3, ch = idx & 7;
-                const int ci = ci0 + row, pp = k0 + ch * 8;
-                const __nv_bfloat16 *src = p.X + (static_cast<long long>(bimg) * p.Cin + ci) * p.P + pp;
-                if (FASTX) {     // P % 8 == 0: whole 16-byte groups, aligned
-                    const bool v = ci < p.Cin && pp < p.P;
-                    cp_async16(at + swz(row, ch), v ? src : p.X, v);
-                } else {
-                    unsigned short h[8];
+                for (int i = 0; i < 4; ++i) {
+                    const int row = (threadIdx.x >> 3) + 32 * i;
+                    const int ci = ci0 + row;
+                    const __nv_bfloat16 *src = xsrc + static_cast<long long>(ci) * p.P;
+                    if (FASTX) {     // P % 8 == 0: whole 16-byte groups, aligned
+                        const bool v = ci < p.Cin && pp < p.P;
+                        cp_async16(at + swz(row, xch), v ? src : p.X, v);
+                    } else {
+                        unsigned short h[8];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        h[j] = (ci < p.Cin && pp + j < p.P) ? __ldg(reinterpret_cast<const unsigned short *>(src) + j) : 0;
-                    *reinterpret_cast<uint4 *>(at + swz(row, ch)) =
-                        make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+                        for (int j = 0; j < 8; ++j)
+                            h[j] = (ci < p.Cin && pp + j < p.P) ? __ldg(reinterpret_cast<const unsigned short *>(src) + j) : 0;
+                        *reinterpret_cast<uint4 *>(at + swz(row, xch)) =
+                            make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+                    }
                 }
-            }
-            if (FASTX) {
-                mbar_arrive_on_cp_async(&pipe.a_full[sa]);
-            } else {
-                fence_async_proxy();
-                mbar_arrive(&pipe.a_full[sa]);
-            }
-            // ---- nine shifted code tiles: 72 warp tasks (tap, chunk), lanes = 32 co rows
-            const int sb = it % NB;
-            ok = ok && mbar_wait(&pipe.b_empty[sb], ((it / NB) & 1) ^ 1, p.err_flag);
-            unsigned char *bt = b_s + sb * B_STAGE;
-#pragma unroll 1
-            for (int task = warp; task < 72; task += kProdWarps) {
-                const int tap = task >> 3, ch = task & 7;
-                const int ky = tap / 3, kx = tap - ky * 3;
-                // X[p + (ky-1) W + (kx-1)] pairs with q[p]; with p' the X position, q index is p' - s
-                const int shift = -((ky - 1) * p.W + (kx - 1));
-                uint2 c8 = bytes8(raw + lane * p.raw_pitch, k0 + ch * 8 + shift - a0);
+                if (FASTX) {
+                    mbar_arrive_on_cp_async(&pipe.a_full[sa]);
+                } else {
+                    fence_async_proxy();
+                    mbar_arrive(&pipe.a_full[sa]);
+                }
+                // ---- nine shifted code tiles; warp w builds chunk w of every tap, lanes = co rows
+                const int sb = it % NB;
+                ok = ok && mbar_wait(&pipe.b_empty[sb], ((it / NB) & 1) ^ 1, p.err_flag);
+                unsigned char *bt = b_s + sb * B_STAGE + swz(lane, warp);
+                const unsigned *rrow_s = raw + lane * p.raw_pitch;
+                const int off0 = k0 + warp * 8 - a0;
                 // source column is x' - (kx-1): kx = 0 needs x' <= W-2, kx = 2 needs x' >= 1
-                const uint4 m = column_masks(k0, ch * 8, p.W);
-                if (kx == 0) { c8.x &= m.x; c8.y &= m.y; }
-                if (kx == 2) { c8.x &= m.z; c8.y &= m.w; }
-                *reinterpret_cast<uint4 *>(bt + tap * B_TAP + swz(lane, ch)) = expand8(c8);
+                const uint4 m = column_masks(k0, warp * 8, p.W);
+#pragma unroll
+                for (int ky = 0; ky < 3; ++ky) {
+                    // X[p + (ky-1) W + (kx-1)] pairs with q[p]: with p' the X position, q index is p' - s
+                    const int offy = off0 - (ky - 1) * p.W;
+                    uint2 c0 = bytes8(rrow_s, offy + 1), c1 = bytes8(rrow_s, offy), c2 = bytes8(rrow_s, offy - 1);
+                    c0.x &= m.x; c0.y &= m.y;
+                    c2.x &= m.z; c2.y &= m.w;
+                    *reinterpret_cast<uint4 *>(bt + (ky * 3 + 0) * B_TAP) = expand8(c0);
+                    *reinterpret_cast<uint4 *>(bt + (ky * 3 + 1) * B_TAP) = expand8(c1);
+                    *reinterpret_cast<uint4 *>(bt + (ky * 3 + 2) * B_TAP) = expand8(c2);
+                }
+                fence_async_proxy();
+                mbar_arrive(&pipe.b_full[sb]);
             }
-            fence_async_proxy();
-            mbar_arrive(&pipe.b_full[sb]);
+            advance(bimg, k0);
         }
         // ---------------- epilogue: lanes = ci, columns = (tap, co); partials [split][tap][Cout][Cin]
         if (niter > 0 && mbar_wait(&pipe.acc, 0, p.err_flag)) {
