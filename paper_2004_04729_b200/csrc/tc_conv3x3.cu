@@ -281,7 +281,8 @@ __global__ void weight_rows_kernel(const __nv_bfloat16 *__restrict__ W, __nv_bfl
 // ------------------------------------------------------------------------------------ dW
 // One stage = 64 consecutive positions of one image. A = X tile [128 ci][64 positions] (native,
 // K-major), B_tap = shifted codes [32 co][64 positions] (K-major), nine accumulators of 32 columns.
-template <bool FASTX>
+// GX: positions per aligned group of X: 8 (P % 8 == 0), 4 (P % 4 == 0) or 1
+template <int GX>
 __global__ void __launch_bounds__(kThreads3) tc3_dw_kernel(const P3 p) {
     constexpr int NB = 2;
     constexpr int A_TILE = 16384;                 // 128 x 64 bf16
@@ -363,9 +364,13 @@ __global__ void __launch_bounds__(kThreads3) tc3_dw_kernel(const P3 p) {
                     const int row = (threadIdx.x >> 3) + 32 * i;
                     const int ci = ci0 + row;
                     const __nv_bfloat16 *src = xsrc + static_cast<long long>(ci) * p.P;
-                    if (FASTX) {     // P % 8 == 0: whole 16-byte groups, aligned
+                    if (GX == 8) {   // whole 16-byte groups, aligned
                         const bool v = ci < p.Cin && pp < p.P;
                         cp_async16(at + swz(row, xch), v ? src : p.X, v);
+                    } else if (GX == 4) {   // two aligned 8-byte halves, each inside the image or not
+                        const bool v0 = ci < p.Cin && pp < p.P, v1 = ci < p.Cin && pp + 4 < p.P;
+                        cp_async_small<8>(at + swz(row, xch), v0 ? src : p.X, v0);
+                        cp_async_small<8>(at + swz(row, xch) + 8, v1 ? src + 4 : p.X, v1);
                     } else {
                         unsigned short h[8];
 #pragma unroll
@@ -375,7 +380,7 @@ __global__ void __launch_bounds__(kThreads3) tc3_dw_kernel(const P3 p) {
                             make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
                     }
                 }
-                if (FASTX) {
+                if (GX > 1) {
                     mbar_arrive_on_cp_async(&pipe.a_full[sa]);
                 } else {
                     fence_async_proxy();
@@ -541,11 +546,14 @@ int launch_tc3_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float 
               static_cast<unsigned>(split));
     const size_t smem = static_cast<size_t>(kNA) * 16384 + 2 * 9 * 4096 + 2 * 32 * static_cast<size_t>(p.raw_pitch) * 4 + 1024;
     if (p.P % 8 == 0) {
-        if ((rc = set_smem3(tc3_dw_kernel<true>, smem))) return rc;
-        tc3_dw_kernel<true><<<grid, kThreads3, smem, ctx->stream>>>(p);
+        if ((rc = set_smem3(tc3_dw_kernel<8>, smem))) return rc;
+        tc3_dw_kernel<8><<<grid, kThreads3, smem, ctx->stream>>>(p);
+    } else if (p.P % 4 == 0) {
+        if ((rc = set_smem3(tc3_dw_kernel<4>, smem))) return rc;
+        tc3_dw_kernel<4><<<grid, kThreads3, smem, ctx->stream>>>(p);
     } else {
-        if ((rc = set_smem3(tc3_dw_kernel<false>, smem))) return rc;
-        tc3_dw_kernel<false><<<grid, kThreads3, smem, ctx->stream>>>(p);
+        if ((rc = set_smem3(tc3_dw_kernel<1>, smem))) return rc;
+        tc3_dw_kernel<1><<<grid, kThreads3, smem, ctx->stream>>>(p);
     }
     if ((rc = cuda_ok(cudaGetLastError()))) return rc;
     long long blocks = (static_cast<long long>(nw) + 255) / 256;

@@ -1,13 +1,14 @@
 // Dense tensor-core input gradient of 1x1 convolutions and linear layers, bf16 operands:
 //   dX[r][ci] = Delta * sum_co q[r,co] W[co,ci],   r = (image, position) flattened
-//   M = 128 rows r, N = ci (NT), K = co in stages of 64; both operands MN-major
-//   (a k-row holds 64 consecutive rows r / 64 consecutive input channels).
+//   M = 128 input channels, N = 128 rows r, K = co in stages of 64; both operands MN-major
+//   (a k-row holds 64 consecutive input channels / 64 consecutive rows r). With channels on
+//   the accumulator's lanes, a thread of the epilogue holds consecutive positions of one
+//   channel, which is how dX lies in memory.
 //
 // Bound by HBM: the codes are read once and dX is written once. All global reads are cp.async
 // copies issued ahead of use (weights straight into their swizzled operand tile, code bytes
 // into a raw staging tile); eight producer warps expand the staged codes to bf16 from shared
-// memory; a ninth warp issues the MMAs. The accumulator leaves through per-warp shared-memory
-// patches so that each lane stores a contiguous run of positions of one channel.
+// memory; a ninth warp issues the MMAs.
 #include "tc_common.cuh"
 
 namespace dbp {
@@ -21,8 +22,6 @@ constexpr int kP = kPW * 32;
 constexpr int kThreadsDx = kP + 32;
 constexpr int kMaxS = 4;
 constexpr int kKT = 64;
-constexpr int kPatchCol = 192;                 // bytes per column of an epilogue patch
-constexpr int kPatch = 32 * kPatchCol;         // one warp's 32 columns x 32 rows
 
 struct DxP {
     const int8_t *codes;          // [B][Cout][P]
@@ -41,38 +40,16 @@ struct PipeDx {
     unsigned tmem_base;
 };
 
-template <int BYTES>
-__device__ __forceinline__ void store_bytes(void *dst, const unsigned char *src) {
-    if (BYTES == 16) *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
-    else if (BYTES == 8) *reinterpret_cast<uint2 *>(dst) = *reinterpret_cast<const uint2 *>(src);
-    else if (BYTES == 4) *reinterpret_cast<unsigned *>(dst) = *reinterpret_cast<const unsigned *>(src);
-    else *reinterpret_cast<unsigned short *>(dst) = *reinterpret_cast<const unsigned short *>(src);
-}
-
-// One warp's 32 rows x 32 columns patch -> global: a lane stores RL consecutive rows (one
-// aligned, image-contained group) of one column.
-template <int ES, int RL>
-__device__ __forceinline__ void store_patch(const unsigned char *patch, const DxP &p, int lane, long long row_first,
-                                            int ci_first) {
-    constexpr int LPC = 32 / RL;               // lanes per column
-    constexpr int CPP = 32 / LPC;              // columns per pass
-    const int rr = (lane % LPC) * RL;
-    const long long r = row_first + rr;
-    if (r >= p.rows) return;
-    const long long b = r / p.P, pp = r - b * p.P;
-    unsigned char *base = static_cast<unsigned char *>(p.dX) + ((b * p.Cin) * p.P + pp) * ES;
-#pragma unroll 4
-    for (int cb = 0; cb < 32; cb += CPP) {
-        const int j = cb + lane / LPC;
-        const int ci = ci_first + j;
-        if (ci < p.Cin) store_bytes<RL * ES>(base + static_cast<long long>(ci) * p.P * ES, patch + j * kPatchCol + rr * ES);
-    }
+// 32-byte store (one full sector); dst 32-byte aligned
+__device__ __forceinline__ void st_global_v8(void *dst, const unsigned (&w)[8]) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+                 "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
 }
 
 // G = rows per aligned, image-contained group: 8 (P % 8 == 0), 4 (P % 4 == 0) or 1 (any P).
 template <int NT, int G>
 __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
-    constexpr int A_BYTES = 2 * kKT * 128;          // two 64-row groups x 64 k-rows
+    constexpr int A_BYTES = 2 * kKT * 128;          // codes: two 64-row groups x 64 k-rows
     constexpr int B_BYTES = (NT / 64) * kKT * 128;
     constexpr int RAW_BYTES = kKT * 128;            // 64 co x 128 rows, one byte each
     constexpr int STAGE = A_BYTES + B_BYTES + RAW_BYTES;
@@ -96,7 +73,7 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
         mbar_init(&pipe.acc, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == kPW) tmem_alloc(&pipe.tmem_base, NT);
+    if (warp == kPW) tmem_alloc(&pipe.tmem_base, 128);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -180,46 +157,100 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
             fence_async_proxy();
             mbar_arrive(&pipe.full[s]);
         }
-        // ---------------- epilogue: TMEM lanes = rows, columns = ci. Warp w: rows 32 (w % 4) ...,
-        // column half w / 4. All MMAs are complete, so the stage buffers hold the patches.
+        // ---------------- epilogue: TMEM lanes = input channels, columns = rows. Warp w takes lane
+        // quarter w % 4 and column half w / 4; a lane stores runs of consecutive positions.
         if (mbar_wait(&pipe.acc, 0, p.err_flag)) {
             tc_fence_after();
             const float delta = *p.delta_p;
             const int q = warp & 3, half = warp >> 2;
-            unsigned char *patch = smem + warp * kPatch;
-            const long long row_first = row0 + q * 32;
+            const int ci = ci0 + q * 32 + lane;
+            constexpr int RL = G >= 8 ? 8 : G;          // rows per store group
 #pragma unroll 1
-            for (int c0 = half * (NT / 2); c0 < (half + 1) * (NT / 2); c0 += 32) {
+            for (int c0 = half * 64; c0 < half * 64 + 64; c0 += 32) {
                 unsigned v[32];
                 tmem_ld32(tmem_d + (static_cast<unsigned>(q * 32) << 16) + c0, v);
-                if (ci0 + c0 < p.Cin) {                       // warp-uniform
-                    if (p.dx_f32) {
+                const long long rfirst = row0 + c0;
+                if (ci < p.Cin && rfirst < p.rows) {
+                    long long b = rfirst / p.P, pp = rfirst - b * p.P;
+                    if (G == 8 && (p.dx_f32 || (p.P & 15) == 0)) {
+                        // 32-byte stores: one full sector per lane and instruction
+                        constexpr int kStep32 = 0;
+                        (void)kStep32;
+                        const int step = p.dx_f32 ? 8 : 16;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            *reinterpret_cast<float *>(patch + j * kPatchCol + lane * 4) = __uint_as_float(v[j]) * delta;
+                        for (int j0 = 0; j0 < 32; j0 += 8) {
+                            if (!p.dx_f32 && (j0 & 8)) continue;        // bf16: 16 rows per store
+                            if (rfirst + j0 < p.rows) {
+                                const long long o = (b * p.Cin + ci) * p.P + pp;
+                                unsigned w[8];
+                                if (p.dx_f32) {
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) w[e] = __float_as_uint(__uint_as_float(v[j0 + e]) * delta);
+                                    st_global_v8(static_cast<float *>(p.dX) + o, w);
+                                } else {
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) {
+                                        const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[j0 + 2 * e]) * delta,
+                                                                                       __uint_as_float(v[(j0 + 2 * e + 1) & 31]) * delta);
+                                        w[e] = *reinterpret_cast<const unsigned *>(&h);
+                                    }
+                                    st_global_v8(static_cast<__nv_bfloat16 *>(p.dX) + o, w);
+                                }
+                            }
+                            pp += step;
+                            if (pp >= p.P) { pp -= p.P; ++b; }
+                        }
                     } else {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            *reinterpret_cast<unsigned short *>(patch + j * kPatchCol + lane * 2) =
-                                __bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(v[j]) * delta));
+                    for (int j0 = 0; j0 < 32; j0 += RL) {
+                        if (rfirst + j0 < p.rows) {
+                            const long long o = (b * p.Cin + ci) * p.P + pp;
+                            if (p.dx_f32) {
+                                float *dst = static_cast<float *>(p.dX) + o;
+                                if (RL >= 4) {
+#pragma unroll
+                                    for (int e = 0; e < RL; e += 4)
+                                        *reinterpret_cast<float4 *>(dst + e) =
+                                            make_float4(__uint_as_float(v[j0 + e]) * delta, __uint_as_float(v[j0 + e + 1]) * delta,
+                                                        __uint_as_float(v[j0 + e + 2]) * delta, __uint_as_float(v[j0 + e + 3]) * delta);
+                                } else {
+                                    dst[0] = __uint_as_float(v[j0]) * delta;
+                                }
+                            } else {
+                                __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.dX) + o;
+                                if (RL >= 4) {
+                                    unsigned w[RL / 2 > 0 ? RL / 2 : 1];
+#pragma unroll
+                                    for (int e = 0; e < RL / 2; ++e) {
+                                        const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[j0 + 2 * e]) * delta,
+                                                                                       __uint_as_float(v[j0 + 2 * e + 1]) * delta);
+                                        w[e] = *reinterpret_cast<const unsigned *>(&h);
+                                    }
+                                    if (RL == 8) *reinterpret_cast<uint4 *>(dst) = make_uint4(w[0], w[1], w[RL / 2 > 2 ? 2 : 0], w[RL / 2 > 3 ? 3 : 0]);
+                                    else *reinterpret_cast<uint2 *>(dst) = make_uint2(w[0], w[1]);
+                                } else {
+                                    dst[0] = __float2bfloat16_rn(__uint_as_float(v[j0]) * delta);
+                                }
+                            }
+                        }
+                        pp += RL;
+                        if (pp >= p.P) { pp -= p.P; ++b; }      // groups never straddle two images
                     }
-                    __syncwarp();
-                    if (p.dx_f32) store_patch<4, (G >= 4 ? 4 : 1)>(patch, p, lane, row_first, ci0 + c0);
-                    else store_patch<2, G>(patch, p, lane, row_first, ci0 + c0);
-                    __syncwarp();
+                    }
                 }
             }
         }
     } else if (lane == 0) {
-        constexpr unsigned idesc = make_idesc(128, NT, true, true);
+        constexpr unsigned idesc = make_idesc(128, 128, true, true);
         bool ok = true;
         for (int it = 0; it < niter && ok; ++it) {
             const int s = it % S;
             ok = mbar_wait(&pipe.full[s], (it / S) & 1, p.err_flag);
             fence_async_proxy();
             tc_fence_after();
-            const unsigned a_addr = smem_u32(smem + s * STAGE), b_addr = a_addr + A_BYTES;
-            const unsigned long long ad = make_desc(a_addr, PANEL, 1024), bd = make_desc(b_addr, PANEL, 1024);
+            const unsigned q_addr = smem_u32(smem + s * STAGE), w_addr = q_addr + A_BYTES;
+            // A = weights (M = channels), B = codes (N = rows)
+            const unsigned long long ad = make_desc(w_addr, PANEL, 1024), bd = make_desc(q_addr, PANEL, 1024);
 #pragma unroll
             for (int k = 0; k < kKT / 16; ++k)     // 16 k-rows = two 1024-byte groups further per MMA
                 mma_bf16(tmem_d, ad + 128 * k, bd + 128 * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
@@ -231,7 +262,7 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
     __syncthreads();
     if (warp == kPW) {
         __syncwarp();
-        tmem_dealloc(tmem_d, NT);
+        tmem_dealloc(tmem_d, 128);
     }
 }
 
@@ -267,14 +298,11 @@ int launch_tc_dx(dbp_ctx *ctx, const int8_t *codes, const void *W, const float *
     p.err_flag = err_flag;
     const int niter = static_cast<int>((s.Cout + kKT - 1) / kKT);
     p.stages = niter < kMaxS ? niter : kMaxS;
-    // narrow N tiles leave room for several CTAs per SM, which overlaps the load, MMA and
-    // store phases of different tiles
-    const int nt = s.Cin > 64 ? 128 : 64;
-    dim3 grid(static_cast<unsigned>((p.rows + 127) / 128), static_cast<unsigned>((s.Cin + nt - 1) / nt));
-    size_t smem = static_cast<size_t>(p.stages) * (2 * kKT * 128 + (nt / 64) * kKT * 128 + kKT * 128);
-    if (smem < static_cast<size_t>(kPW) * kPatch) smem = static_cast<size_t>(kPW) * kPatch;
-    smem += 1024;
-    return nt == 128 ? run_g<128>(ctx, p, grid, smem) : run_g<64>(ctx, p, grid, smem);
+    // one CTA: 128 rows x 128 channels; few stages leave room for several CTAs per SM, which
+    // overlaps the load, MMA and store phases of different tiles
+    dim3 grid(static_cast<unsigned>((p.rows + 127) / 128), static_cast<unsigned>((s.Cin + 127) / 128));
+    const size_t smem = static_cast<size_t>(p.stages) * (2 * kKT * 128 + 2 * kKT * 128 + kKT * 128) + 1024;
+    return run_g<128>(ctx, p, grid, smem);
 }
 
 }  // namespace dbp
