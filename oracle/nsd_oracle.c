@@ -75,7 +75,8 @@ int64_t oracle_nsd_codes(const float *x, int64_t n, uint64_t seed, float Delta,
         float t = fmaf(x[i], inv, u);          /* one rounding */
         float f = floorf(t);
         int q;
-        if (f > 127.0f) { q = 127; ++sat; }
+        if (isnan(t)) q = 0;                   /* Eq. (nsd) is undefined for NaN: no code */
+        else if (f > 127.0f) { q = 127; ++sat; }
         else if (f < -127.0f) { q = -127; ++sat; }
         else q = (int)f;
         codes[i] = (int8_t)q;

@@ -147,14 +147,16 @@ __device__ __forceinline__ float dither_from_bits(unsigned h) {
     return __uint_as_float(0x3f800000u | (h >> 9)) - 0.99999994f;
 }
 
-// q = floor(x / Delta + u) with one rounding, clipped to [-127, 127].
+// q = floor(x / Delta + u) with one rounding, clipped to [-127, 127]; NaN gives 0.
+// floor and the conversion to int are one round-down addition of 1.5 * 2^23 (exact for the
+// clamped range) and an integer subtraction.
 __device__ __forceinline__ int quantize_one(float x, float inv, float u, unsigned &sat) {
-    const float f = floorf(__fmaf_rn(x, inv, u));
-    int q;
-    if (f > 127.f) { q = 127; ++sat; }
-    else if (f < -127.f) { q = -127; ++sat; }
-    else q = __float2int_rz(f);
-    return q;
+    const float t = __fmaf_rn(x, inv, u);
+    const float tc = fminf(fmaxf(t, -127.f), 127.99999f);
+    const bool num = (t == t);
+    sat += (num && tc != t) ? 1u : 0u;
+    const int q = __float_as_int(__fadd_rd(tc, 12582912.0f)) - 0x4B400000;
+    return num ? q : 0;
 }
 
 // One warp owns one 1024-element segment at a time: ITER 128-bit loads per lane, codes
@@ -170,77 +172,102 @@ quantize_kernel(const T *__restrict__ x, long long n, unsigned long long seed,
     constexpr int EPT = Elem<T>::EPT;
     constexpr int ITER = kSegment / (32 * EPT);  // 8 (fp32) or 4 (bf16)
     constexpr int LPW = 32 / EPT;                // lanes that share one bitmap word
+    constexpr int NW = EPT / 4;                  // packed code words per lane and iteration
     __shared__ __align__(16) int8_t stage[kThreads / 32][kSegment];
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long nseg = (n + kSegment - 1) / kSegment;
     const long long nwarps = static_cast<long long>(gridDim.x) * (kThreads / 32);
+    const long long first = static_cast<long long>(blockIdx.x) * (kThreads / 32) + warp;
     const float delta = *delta_p;
     const bool live = (delta > 0.f) && (delta < __int_as_float(0x7f800000));
-    const float inv = live ? __fdiv_rn(1.0f, delta) : 0.f;
+    if (!live) {   // sigma = 0 or non-finite input: every code is 0
+        for (long long seg = first; seg < nseg; seg += nwarps) {
+            bitmap[seg * kWordsPerSegment + lane] = 0u;
+            offsets[seg * kWordsPerSegment + lane] = 0;
+            if (dense != nullptr) {
+                const long long e0 = seg * kSegment + lane * 32;
+                if (e0 + 32 <= n) {
+                    reinterpret_cast<uint4 *>(dense + e0)[0] = make_uint4(0u, 0u, 0u, 0u);
+                    reinterpret_cast<uint4 *>(dense + e0)[1] = make_uint4(0u, 0u, 0u, 0u);
+                } else {
+                    for (int j = 0; j < 32; ++j)
+                        if (e0 + j < n) dense[e0 + j] = 0;
+                }
+            }
+        }
+        return;
+    }
+    const float inv = __fdiv_rn(1.0f, delta);
     const int sub = lane % LPW;                  // my position inside the word
-    const unsigned below = (1u << (EPT * sub)) - 1u;
     unsigned long long nnz_local = 0ull;
     unsigned sat = 0;
 
-    for (long long seg = static_cast<long long>(blockIdx.x) * (kThreads / 32) + warp; seg < nseg; seg += nwarps) {
+    for (long long seg = first; seg < nseg; seg += nwarps) {
+        const bool full = (seg + 1) * kSegment <= n;
         unsigned running = 0, my_word = 0, my_off = 0;
 #pragma unroll
         for (int it = 0; it < ITER; ++it) {
             const long long e0 = seg * kSegment + it * (32 * EPT) + lane * EPT;
             float v[EPT];
-            if (e0 + EPT <= n) {
+            if (full || e0 + EPT <= n) {
                 Elem<T>::load(x + e0, v);
             } else {
 #pragma unroll
                 for (int j = 0; j < EPT; ++j) v[j] = (e0 + j < n) ? Elem<T>::one(x + e0 + j) : 0.f;
             }
-            int q[EPT];
+            unsigned pk[NW];
+#pragma unroll
+            for (int w = 0; w < NW; ++w) pk[w] = 0u;
             unsigned bits = 0;
             unsigned long long z = seed + (static_cast<unsigned long long>(e0 >> 1) + 1ull) * 0x9E3779B97F4A7C15ull;
 #pragma unroll
             for (int j = 0; j < EPT; j += 2) {
                 const unsigned long long r = splitmix64_mix(z);
                 z += 0x9E3779B97F4A7C15ull;
-                q[j] = live ? quantize_one(v[j], inv, dither_from_bits(static_cast<unsigned>(r)), sat) : 0;
-                q[j + 1] = live ? quantize_one(v[j + 1], inv, dither_from_bits(static_cast<unsigned>(r >> 32)), sat) : 0;
-                if (e0 + j >= n) q[j] = 0;
-                if (e0 + j + 1 >= n) q[j + 1] = 0;
-                bits |= (q[j] != 0 ? 1u : 0u) << j;
-                bits |= (q[j + 1] != 0 ? 1u : 0u) << (j + 1);
+                const int q0 = quantize_one(v[j], inv, dither_from_bits(static_cast<unsigned>(r)), sat);
+                const int q1 = quantize_one(v[j + 1], inv, dither_from_bits(static_cast<unsigned>(r >> 32)), sat);
+                pk[j >> 2] |= (static_cast<unsigned>(q0) & 0xffu) << (8 * (j & 3));
+                pk[j >> 2] |= (static_cast<unsigned>(q1) & 0xffu) << (8 * ((j + 1) & 3));
+                bits |= (q0 != 0 ? 1u : 0u) << j;
+                bits |= (q1 != 0 ? 1u : 0u) << (j + 1);
+            }
+            if (!full) {   // elements past the end carry no code (their x was read as 0 already)
+#pragma unroll
+                for (int j = 0; j < EPT; ++j)
+                    if (e0 + j >= n) { bits &= ~(1u << j); pk[j >> 2] &= ~(0xffu << (8 * (j & 3))); }
             }
             // bitmap word shared by LPW consecutive lanes
             unsigned word = bits << (EPT * sub);
 #pragma unroll
             for (int o = 1; o < LPW; o <<= 1) word |= __shfl_xor_sync(kFull, word, o);
-            const unsigned pc = __popc(word);
-            // exclusive prefix over the EPT words of this iteration
-            unsigned before = 0, total = 0;
-            const int my_w = lane / LPW;
+            // exclusive rank of my first code inside the segment: warp scan of the lane counts
+            const unsigned pc = __popc(bits);
+            unsigned incl = pc;
 #pragma unroll
-            for (int w = 0; w < EPT; ++w) {
-                const unsigned c = __shfl_sync(kFull, pc, w * LPW);
-                before += (w < my_w) ? c : 0u;
-                total += c;
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned up = __shfl_up_sync(kFull, incl, o);
+                if (lane >= o) incl += up;
             }
-            const unsigned word_off = running + before;
-            unsigned rank = word_off + __popc(word & below);
-#pragma unroll
-            for (int j = 0; j < EPT; ++j)
-                if (q[j] != 0) stage[warp][rank++] = static_cast<int8_t>(q[j]);
+            const unsigned total = __shfl_sync(kFull, incl, 31);
+            unsigned rank = running + incl - pc;
+            const unsigned word_off = rank;      // for a word's first lane: codes before the word
+            // non-zero codes to the staging line, in element order
+            unsigned b = bits;
+            while (b) {
+                const int j = __ffs(b) - 1;
+                b &= b - 1;
+                const unsigned wsel = (NW == 1 || j < 4) ? pk[0] : pk[NW - 1];
+                stage[warp][rank++] = static_cast<int8_t>((wsel >> (8 * (j & 3))) & 0xffu);
+            }
             if (dense != nullptr) {
-                if (e0 + EPT <= n) {
-                    unsigned pk[EPT / 4];
-#pragma unroll
-                    for (int j = 0; j < EPT; j += 4)
-                        pk[j / 4] = (q[j] & 0xff) | ((q[j + 1] & 0xff) << 8) | ((q[j + 2] & 0xff) << 16) |
-                                    (static_cast<unsigned>(q[j + 3] & 0xff) << 24);
+                if (full || e0 + EPT <= n) {
                     if (EPT == 4) *reinterpret_cast<unsigned *>(dense + e0) = pk[0];
-                    else *reinterpret_cast<uint2 *>(dense + e0) = make_uint2(pk[0], pk[EPT / 4 - 1]);
+                    else *reinterpret_cast<uint2 *>(dense + e0) = make_uint2(pk[0], pk[NW - 1]);
                 } else {
 #pragma unroll
                     for (int j = 0; j < EPT; ++j)
-                        if (e0 + j < n) dense[e0 + j] = static_cast<int8_t>(q[j]);
+                        if (e0 + j < n) dense[e0 + j] = static_cast<int8_t>((pk[j >> 2] >> (8 * (j & 3))) & 0xffu);
                 }
             }
             // lane (it*EPT + w) keeps word w of this iteration and its offset
