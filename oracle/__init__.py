@@ -8,7 +8,8 @@ Nothing here is imported by, or shares code with, the CUDA library or its bindin
 from .nsd import (splitmix64_at, dither_u, mean_std, step_size, nsd_codes,
                   nsd_codes_literal_f64, nsd_codes_exact_python, derive_layer_seed)
 from .products import (linear_backward, conv_backward, conv_forward,
-                       linear_backward_bruteforce, conv_backward_bruteforce)
+                       linear_backward_bruteforce, conv_backward_bruteforce,
+                       conv_dW_entry, conv_dX_entry)
 
 from .chain import relu_backward, maxpool2x2_backward, layer_backward, chain_backward
 
@@ -17,5 +18,5 @@ __all__ = [
     "splitmix64_at", "dither_u", "mean_std", "step_size", "nsd_codes",
     "nsd_codes_literal_f64", "nsd_codes_exact_python", "derive_layer_seed",
     "linear_backward", "conv_backward", "conv_forward",
-    "linear_backward_bruteforce", "conv_backward_bruteforce",
+    "linear_backward_bruteforce", "conv_backward_bruteforce", "conv_dW_entry", "conv_dX_entry",
 ]

@@ -143,3 +143,45 @@ def conv_backward_bruteforce(codes, Delta, X, W):
                                     dW[co, ci, ky, kx] += t * X[b, ci, yy, xx]
                                     dX[b, ci, yy, xx] += t * W[co, ci, ky, kx]
     return {"dW": dW, "dX": dX, "db": db}
+
+
+# ---- single outputs of the same definitions (for full-size tensors, where the whole product
+# ---- in fp64 would take minutes): each value is the defining sum written out for one index.
+
+def _shifted_dot(q, x, ky, kx, p):
+    """sum_{b,y,x} q[b,y,x] * x[b,y+ky-p,x+kx-p] with zero padding, and the sum of |terms|."""
+    B, H, Wd = q.shape
+    dy, dx = ky - p, kx - p
+    y0, y1 = max(0, -dy), min(H, H - dy)
+    x0, x1 = max(0, -dx), min(Wd, Wd - dx)
+    if y0 >= y1 or x0 >= x1:
+        return 0.0, 0.0
+    t = q[:, y0:y1, x0:x1] * x[:, y0 + dy:y1 + dy, x0 + dx:x1 + dx]
+    return float(t.sum()), float(np.abs(t).sum())
+
+
+def conv_dW_entry(codes, Delta, X, co, ci, ky, kx, k):
+    """(dW[co,ci,ky,kx], sum |terms|) from the definition for a k x k kernel, padding (k-1)/2;
+    codes [B,Co,H,W], X [B,Ci,H,W]."""
+    D = float(np.float32(Delta))
+    q = np.asarray(codes[:, co], dtype=np.float64) * D
+    x = np.asarray(X[:, ci], dtype=np.float64)
+    return _shifted_dot(q, x, ky, kx, (k - 1) // 2)
+
+
+def conv_dX_entry(codes, Delta, W, b, ci, y, x):
+    """(dX[b,ci,y,x], sum |terms|): sum_{co,ky,kx} delta~[b,co,y-ky+p,x-kx+p] W[co,ci,ky,kx]."""
+    D = float(np.float32(Delta))
+    Co, _, k, _ = W.shape
+    p = (k - 1) // 2
+    H, Wd = codes.shape[2], codes.shape[3]
+    tot = 0.0
+    tot_abs = 0.0
+    for ky in range(k):
+        for kx in range(k):
+            yy, xx = y - ky + p, x - kx + p
+            if 0 <= yy < H and 0 <= xx < Wd:
+                t = np.asarray(codes[b, :, yy, xx], dtype=np.float64) * D * np.asarray(W[:, ci, ky, kx], dtype=np.float64)
+                tot += float(t.sum())
+                tot_abs += float(np.abs(t).sum())
+    return tot, tot_abs

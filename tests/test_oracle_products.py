@@ -122,3 +122,17 @@ def test_small_step_limit_recovers_dense_products():
     o = oracle.linear_backward(c, D, L.X, L.W)
     dense = d.astype(np.float64).T @ L.X.astype(np.float64)
     assert np.abs(o["dW"] - dense).max() <= 8 * float(D) * np.abs(L.X).max()
+
+
+@pytest.mark.parametrize("k", [1, 3])
+def test_single_entry_routines_match_the_full_products(k):
+    c, D, X, Wt = _tiny_conv(B=3, Co=4, Ci=5, H=5, W=6, k=k, seed=21)
+    full = oracle.conv_backward(c, D, X, Wt, with_abs=True)
+    r = np.random.default_rng(0)
+    for _ in range(25):
+        co, ci, ky, kx = r.integers(4), r.integers(5), r.integers(k), r.integers(k)
+        v, s = oracle.conv_dW_entry(c, D, X, co, ci, ky, kx, k)
+        assert abs(v - full["dW"][co, ci, ky, kx]) < 1e-12 and abs(s - full["S_dW"][co, ci, ky, kx]) < 1e-12
+        b, y, x = r.integers(3), r.integers(5), r.integers(6)
+        v, s = oracle.conv_dX_entry(c, D, Wt, b, ci, y, x)
+        assert abs(v - full["dX"][b, ci, y, x]) < 1e-12 and abs(s - full["S_dX"][b, ci, y, x]) < 1e-12
