@@ -20,7 +20,7 @@ using namespace tc;
 constexpr int kPW = 8;
 constexpr int kP = kPW * 32;
 constexpr int kThreadsDw = kP + 32;
-constexpr int kMaxS = 4;
+constexpr int kMaxS = 5;
 constexpr int kKT = 64;
 
 struct DwP {
@@ -56,7 +56,10 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
     long long ks1 = ks0 + p.per_split;
     if (ks1 > p.kstages) ks1 = p.kstages;
     const int niter = ks1 > ks0 ? static_cast<int>(ks1 - ks0) : 0;
-    const int S = p.stages, LA = S - 1;
+    const int S = p.stages;
+    // copies run LA stages ahead; with LA = S - 2 a slot is refilled two MMAs after it was
+    // consumed, so producers never wait on the tensor core's latency
+    const int LA = S > 2 ? S - 2 : S - 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
@@ -77,42 +80,55 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
         const int tid = threadIdx.x;
         const int c8 = tid & 7, rsub = tid >> 3;      // chunk column, first of my rows (stride 32)
         bool ok = true;
-        // copies of local stage j: X chunks into the operand tile, code bytes into the raw tile
+        // Addresses are kept incremental: a thread's rows are 32 apart (constant pointer and
+        // shared-memory steps) and a stage advances every group by 64 flattened rows.
+        const long long xstep = 32 * p.P, cstep = 32 * p.P;
+        const unsigned b_off0 = swz(rsub, c8), raw_off0 = rsub * 64 + c8 * 8;
+        long long grow[NGRP > 2 ? 1 : NGRP], gb[NGRP > 2 ? 1 : NGRP], gp[NGRP > 2 ? 1 : NGRP];
+        if (G > 1) {
+#pragma unroll
+            for (int g = 0; g < NGRP; ++g) {
+                grow[g] = ks0 * kKT + c8 * 8 + g * G;
+                gb[g] = grow[g] / p.P;
+                gp[g] = grow[g] - gb[g] * p.P;
+            }
+        }
+        // copies of local stage j (called for j = 0, 1, 2, ... in order): X chunks into the
+        // operand tile, code bytes into the raw tile
         auto issue = [&](int j) {
             const int s = j % S;
             ok = ok && mbar_wait(&pipe.empty[s], ((j / S) & 1) ^ 1, p.err_flag);
             unsigned char *st = smem + s * STAGE;
             unsigned char *b_s = st + A_BYTES, *raw = b_s + B_BYTES;
             const long long r0 = (ks0 + j) * kKT + c8 * 8;
-            long long gb[NGRP > 2 ? 1 : NGRP], gp[NGRP > 2 ? 1 : NGRP];
             if (G > 1) {
 #pragma unroll
                 for (int g = 0; g < NGRP; ++g) {
-                    const long long r = r0 + g * G;
-                    gb[g] = r < p.rows ? r / p.P : -1;
-                    gp[g] = r < p.rows ? r - gb[g] * p.P : 0;
-                }
+                    const bool gv = grow[g] < p.rows;
+                    const __nv_bfloat16 *xs = p.X + (gb[g] * p.Cin + ci0 + rsub) * p.P + gp[g];
+                    unsigned char *xd = b_s + b_off0 + g * 8;
 #pragma unroll
-                for (int i = 0; i < NT / 32; ++i) {
-                    const int row = rsub + 32 * i, ci = ci0 + row;
-#pragma unroll
-                    for (int g = 0; g < NGRP; ++g) {
-                        const bool v = gb[g] >= 0 && ci < p.Cin;
-                        const __nv_bfloat16 *src = v ? p.X + (gb[g] * p.Cin + ci) * p.P + gp[g] : p.X;
-                        if (G == 8) cp_async16(b_s + swz(row, c8), src, v);
-                        else cp_async_small<8>(b_s + swz(row, c8) + g * 8, src, v);
+                    for (int i = 0; i < NT / 32; ++i) {
+                        const bool v = gv && (ci0 + rsub + 32 * i < p.Cin);
+                        if (G == 8) cp_async16(xd, v ? xs : p.X, v);
+                        else cp_async_small<8>(xd, v ? xs : p.X, v);
+                        xs += xstep;
+                        xd += 32 * 128;
                     }
-                }
+                    const int8_t *cs = p.codes + (gb[g] * p.Cout + co0 + rsub) * p.P + gp[g];
+                    unsigned char *cd = raw + raw_off0 + g * 4;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int row = rsub + 32 * i, co = co0 + row;
-#pragma unroll
-                    for (int g = 0; g < NGRP; ++g) {
-                        const bool v = gb[g] >= 0 && co < p.Cout;
-                        const int8_t *src = v ? p.codes + (gb[g] * p.Cout + co) * p.P + gp[g] : p.codes;
-                        if (G == 8) cp_async_small<8>(raw + row * 64 + c8 * 8, src, v);
-                        else cp_async_small<4>(raw + row * 64 + c8 * 8 + g * 4, src, v);
+                    for (int i = 0; i < 4; ++i) {
+                        const bool v = gv && (co0 + rsub + 32 * i < p.Cout);
+                        if (G == 8) cp_async_small<8>(cd, v ? cs : p.codes, v);
+                        else cp_async_small<4>(cd, v ? cs : p.codes, v);
+                        cs += cstep;
+                        cd += 32 * 64;
                     }
+                    // next stage: 64 rows further
+                    grow[g] += kKT;
+                    gp[g] += kKT;
+                    while (gp[g] >= p.P) { gp[g] -= p.P; ++gb[g]; }
                 }
                 mbar_arrive_on_cp_async(&pipe.load_full[s]);
             } else {
@@ -259,7 +275,7 @@ int launch_tc_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *
     if (split < 1) split = 1;
     p.per_split = (p.kstages + split - 1) / split;
     split = (p.kstages + p.per_split - 1) / p.per_split;
-    const int max_s = nt == 256 ? 3 : kMaxS;
+    const int max_s = nt == 256 ? 4 : kMaxS;
     p.stages = p.per_split < max_s ? static_cast<int>(p.per_split) : max_s;
     const size_t nw = static_cast<size_t>(s.Cout) * s.Cin;
     int rc = ws_reserve(ctx, ctx->tc_partials, sizeof(float) * nw * split);

@@ -20,7 +20,7 @@ using namespace tc;
 constexpr int kPW = 8;
 constexpr int kP = kPW * 32;
 constexpr int kThreadsDx = kP + 32;
-constexpr int kMaxS = 4;
+constexpr int kMaxS = 5;
 constexpr int kKT = 64;
 
 struct DxP {
@@ -62,7 +62,10 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
     const long long row0 = static_cast<long long>(blockIdx.x) * 128;
     const int ci0 = blockIdx.y * NT;
     const int niter = (p.Cout + kKT - 1) / kKT;
-    const int S = p.stages, LA = S - 1;
+    const int S = p.stages;
+    // copies run LA stages ahead; with LA = S - 2 a slot is refilled two MMAs after it was
+    // consumed, so producers never wait on the tensor core's latency
+    const int LA = S > 2 ? S - 2 : S - 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
@@ -101,26 +104,33 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
             ok = ok && mbar_wait(&pipe.empty[s], ((j / S) & 1) ^ 1, p.err_flag);
             unsigned char *st = smem + s * STAGE;
             unsigned char *b_s = st + A_BYTES, *raw = b_s + B_BYTES;
-            // weights: k-row = co, 64-channel groups; 64 x (NT/8) chunks of 16 bytes
+            // weights: k-row = co; my chunk column is c16 (8 channels), my k-rows ksub + 16 i.
+            // Pointers step by constants: 16 k-rows per i, 64 per stage.
+            {
+                const int ci = ci0 + c16 * 8;
+                const __nv_bfloat16 *ws = p.W + static_cast<long long>(j * kKT + ksub) * p.Cin + ci;
+                unsigned char *wd = b_s + (c16 >> 3) * PANEL + swz(ksub, c16 & 7);
 #pragma unroll
-            for (int i = 0; i < (kKT * NT / 8) / kP; ++i) {
-                const int idx = tid + i * kP;
-                const int k = idx / (NT / 8), cc = idx - k * (NT / 8);
-                const int co = j * kKT + k, ci = ci0 + cc * 8;
-                const bool v = co < p.Cout && ci < p.Cin;     // Cin % 8 == 0
-                cp_async16(b_s + (cc >> 3) * PANEL + swz(k, cc & 7), v ? p.W + static_cast<long long>(co) * p.Cin + ci : p.W, v);
+                for (int i = 0; i < 4; ++i) {
+                    const bool v = (j * kKT + ksub + 16 * i < p.Cout) && ci < p.Cin;     // Cin % 8 == 0
+                    cp_async16(wd, v ? ws : p.W, v);
+                    ws += 16 * static_cast<long long>(p.Cin);
+                    wd += 16 * 128;
+                }
             }
             // code bytes: k-row = co, my chunk of 8 rows
             if (G > 1) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int k = ksub + 16 * i, co = j * kKT + k;
+                for (int g = 0; g < NGRP; ++g) {
+                    const int8_t *cs = p.codes + gbase[g] + static_cast<long long>(j * kKT + ksub) * p.P;
+                    unsigned char *cd = raw + ksub * 128 + c16 * 8 + g * 4;
 #pragma unroll
-                    for (int g = 0; g < NGRP; ++g) {
-                        const bool v = gbase[g] >= 0 && co < p.Cout;
-                        const int8_t *src = v ? p.codes + gbase[g] + co * p.P : p.codes;
-                        if (G == 8) cp_async_small<8>(raw + k * 128 + c16 * 8, src, v);
-                        else cp_async_small<4>(raw + k * 128 + c16 * 8 + g * 4, src, v);
+                    for (int i = 0; i < 4; ++i) {
+                        const bool v = gbase[g] >= 0 && (j * kKT + ksub + 16 * i < p.Cout);
+                        if (G == 8) cp_async_small<8>(cd, v ? cs : p.codes, v);
+                        else cp_async_small<4>(cd, v ? cs : p.codes, v);
+                        cs += 16 * p.P;
+                        cd += 16 * 128;
                     }
                 }
                 mbar_arrive_on_cp_async(&pipe.load_full[s]);
