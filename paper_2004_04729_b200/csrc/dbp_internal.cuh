@@ -99,6 +99,9 @@ int launch_tc_dx(dbp_ctx *ctx, const int8_t *codes, const void *W, const float *
                  const ConvShape &s, void *dX, bool dx_bf16, int *err_flag);
 // ---- tc_conv3x3.cu
 bool tc3_supported(const ConvShape &s, int io);
+// row-shift variant of the 3x3 dX product; DBP_EUNSUPPORTED when the shape does not fit it
+int launch_tc3_dx_shift(dbp_ctx *ctx, const int8_t *codes, const void *W, const float *delta_p,
+                        const ConvShape &s, void *dX, bool dx_bf16, int *err_flag);
 int launch_tc3_dx(dbp_ctx *ctx, const int8_t *codes, const void *W, const float *delta_p,
                   const ConvShape &s, void *dX, bool dx_bf16, int *err_flag);
 int launch_tc3_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *delta_p,

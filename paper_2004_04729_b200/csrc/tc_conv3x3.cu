@@ -492,6 +492,10 @@ bool tc3_supported(const ConvShape &s, int io) {
 
 int launch_tc3_dx(dbp_ctx *ctx, const int8_t *codes, const void *W, const float *delta_p,
                   const ConvShape &s, void *dX, bool dx_bf16, int *err_flag) {
+    {
+        const int rc_shift = launch_tc3_dx_shift(ctx, codes, W, delta_p, s, dX, dx_bf16, err_flag);
+        if (rc_shift != DBP_EUNSUPPORTED) return rc_shift;
+    }
     P3 p{};
     p.codes = codes; p.delta_p = delta_p; p.dX = dX; p.dx_f32 = dx_bf16 ? 0 : 1;
     p.B = static_cast<int>(s.B); p.Cin = static_cast<int>(s.Cin); p.Cout = static_cast<int>(s.Cout);

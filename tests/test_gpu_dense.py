@@ -71,6 +71,10 @@ def test_dense_path_conv1x1(ctx, B, Ci, Co, H, W):
     (1, 72, 40, 9, 11),       # channel counts that fill no tile, odd width
     (2, 16, 24, 3, 62),       # widest supported row
     (2, 8, 8, 1, 1),          # a single position: every tap but the centre is masked
+    (2, 64, 192, 12, 12),     # row-shift dX kernel, 16-aligned planes, three stages
+    (3, 200, 128, 6, 6),      # row-shift dX kernel, slabs of 36 positions, ragged channel tile
+    (5, 64, 64, 5, 7),        # row-shift dX kernel, odd plane size: byte-aligned slabs
+    (240, 512, 64, 8, 8),     # row-shift dX kernel, four accumulators per CTA
 ])
 def test_dense_path_conv3x3(ctx, B, Ci, Co, H, W):
     import paper_2004_04729_b200 as dbp
@@ -85,6 +89,22 @@ def test_dense_path_linear(ctx, B, N, K):
     if K % 8:
         pytest.skip("dense path needs Cin % 8 == 0")
     _run(ctx, L, dbp.DBP_FORCE_DENSE)
+
+
+@pytest.mark.parametrize("B,Ci,Co,H,W,k", [
+    (2, 64, 64, 16, 16, 3), (2, 128, 128, 14, 14, 3), (3, 64, 128, 7, 7, 3), (2, 64, 128, 28, 28, 1),
+])
+def test_dense_bf16_dx_is_the_rounded_f32_dx(ctx, B, Ci, Co, H, W, k):
+    """The bf16 store path of dX rounds the same accumulators the fp32 store path writes."""
+    import paper_2004_04729_b200 as dbp
+    L = wl.conv_layer(B, Ci, Co, H, W, k, data_seed=7 + H, scale=5.0, dtype="bf16")
+    d, X, W_ = _t(L.delta), _t(L.X), _t(L.W)
+    a = dbp.dithered_conv_backward(ctx, d, X, W_, L.seed, L.scale, flags=dbp.DBP_FORCE_DENSE | dbp.DBP_DX_F32)
+    b = dbp.dithered_conv_backward(ctx, d, X, W_, L.seed, L.scale, flags=dbp.DBP_FORCE_DENSE)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == (0, 0)
+    assert b["dX"].dtype == torch.bfloat16 and a["dX"].dtype == torch.float32
+    assert torch.equal(a["dX"].to(torch.bfloat16), b["dX"])
 
 
 def test_dense_and_sparse_paths_agree_and_unsupported_is_refused(ctx):
