@@ -107,7 +107,9 @@ int dbp_last_device_status(dbp_ctx *ctx, int *status, long long *saturated);
  * the library launches is bracketed by CUDA events on the context's stream.
  * dbp_profile_read synchronises the stream and returns, for one kernel kind, the summed
  * device time in milliseconds and the number of launches since the previous read of that
- * kind (either output may be NULL).
+ * kind (either output may be NULL). The events themselves cost a few microseconds of stream
+ * time each, so dbp_profile_select can restrict the timing to some kinds: bit k of
+ * `kind_mask` set = launches of kind k are timed (default: all kinds).
  */
 typedef enum {
     DBP_K_STATISTICS = 0, /* sigma / Delta reduction */
@@ -123,6 +125,7 @@ typedef enum {
     DBP_K_COUNT = 10
 } dbp_kernel_kind;
 int dbp_profile_enable(dbp_ctx *ctx, int on);
+int dbp_profile_select(dbp_ctx *ctx, unsigned kind_mask);
 int dbp_profile_read(dbp_ctx *ctx, int kind, double *milliseconds, long long *launches);
 
 /* Bytes the caller must allocate for each array of a dbp_sparse over `numel` elements. */

@@ -20,7 +20,7 @@ EXPORTED_SYMBOLS = [
     "dbp_last_device_status", "dbp_sparse_bytes", "nsd_quantize", "nsd_decode_dense",
     "dithered_linear_backward", "dithered_conv_backward", "dithered_linear_backward_host",
     "dithered_conv_backward_host", "dbp_relu_backward", "dbp_maxpool2x2_backward",
-    "dbp_profile_enable", "dbp_profile_read", "dbp_set_crossover", "nsd_step_size_noalloc",
+    "dbp_profile_enable", "dbp_profile_select", "dbp_profile_read", "dbp_set_crossover", "nsd_step_size_noalloc",
 ]
 
 KERNEL_KINDS = ["statistics", "quantize", "weight_taps", "dx", "dw", "db", "decode", "glue",
@@ -79,6 +79,7 @@ def load_library():
     lib.dbp_set_crossover.argtypes = [vp, f32]
     lib.nsd_step_size_noalloc.argtypes = [vp, i32, ll, f32, vp, vp]
     lib.dbp_profile_enable.argtypes = [vp, i32]
+    lib.dbp_profile_select.argtypes = [vp, u32]
     lib.dbp_profile_read.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ll)]
     lib.dbp_relu_backward.argtypes = [vp, vp, vp, vp, ll]
     lib.dbp_maxpool2x2_backward.argtypes = [vp, vp, vp, vp, ll, ll, ll]
@@ -149,6 +150,11 @@ class Context:
 
     def profile_enable(self, on: bool = True):
         _check(load_library().dbp_profile_enable(self._h, int(bool(on))), "dbp_profile_enable")
+
+    def profile_select(self, kinds=None):
+        """Time only the named kernel kinds while profiling is on (None: all kinds)."""
+        mask = 0xFFFFFFFF if kinds is None else sum(1 << KERNEL_KINDS.index(k) for k in kinds)
+        _check(load_library().dbp_profile_select(self._h, mask), "dbp_profile_select")
 
     def profile_read(self):
         """{kernel kind: (milliseconds, launches)} since the previous read."""

@@ -103,8 +103,14 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     const long long numel = s.B * s.Cout * s.H * s.W;
     const float *delta_p = nullptr;
     const int8_t *codes = nullptr;
+    // While the stream is being captured into a CUDA graph the density read-back is left alone
+    // (an event recorded inside a capture cannot be queried): the choice of path is the one the
+    // last eager call would have made, and it is frozen into the graph.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(ctx->stream, &cap) != cudaSuccess) return DBP_ECUDA;
+    const bool capturing = cap != cudaStreamCaptureStatusNone;
     // pick up the density of the last finished quantization, if its read-back has landed
-    if (ctx->nnz_pending && cudaEventQuery(ctx->nnz_event) == cudaSuccess) {
+    if (!capturing && ctx->nnz_pending && cudaEventQuery(ctx->nnz_event) == cudaSuccess) {
         ctx->density_estimate = static_cast<float>(static_cast<double>(*ctx->nnz_host) /
                                                    static_cast<double>(ctx->nnz_host_numel));
         ctx->nnz_pending = false;
@@ -114,7 +120,7 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
                        ((flags & DBP_FORCE_DENSE) || ctx->density_estimate > ctx->crossover);
     int rc = quantize_for_products(ctx, delta, io, numel, seed, scale, delta_in, q_out, &delta_p, &codes);
     if (rc) return rc;
-    if (!ctx->nnz_pending && ctx->nnz_host && ctx->nnz_event) {
+    if (!capturing && !ctx->nnz_pending && ctx->nnz_host && ctx->nnz_event) {
         ctx->nnz_host_numel = numel;
         if (cudaMemcpyAsync(ctx->nnz_host, &ctx->state->nnz, sizeof(unsigned long long), cudaMemcpyDeviceToHost,
                             ctx->stream) == cudaSuccess &&
@@ -282,6 +288,12 @@ int dbp_last_device_status(dbp_ctx *ctx, int *status, long long *saturated) {
 int dbp_profile_enable(dbp_ctx *ctx, int on) {
     if (!ctx) return DBP_EINVAL;
     ctx->profiling = on != 0;
+    return DBP_OK;
+}
+
+int dbp_profile_select(dbp_ctx *ctx, unsigned kind_mask) {
+    if (!ctx) return DBP_EINVAL;
+    ctx->prof_mask = kind_mask;
     return DBP_OK;
 }
 

@@ -55,6 +55,7 @@ struct dbp_ctx {
     cudaEvent_t nnz_event = nullptr;
     bool nnz_pending = false;
     bool profiling = false;
+    unsigned prof_mask = 0xffffffffu;   // kinds that are timed while profiling is on
     std::vector<dbp::ProfSlot> prof;    // event pairs, reused after every read
     size_t prof_used = 0;
     double prof_ms[DBP_K_COUNT] = {0};
@@ -118,7 +119,7 @@ struct KernelTimer {
     dbp_ctx *ctx;
     ProfSlot *slot = nullptr;
     KernelTimer(dbp_ctx *c, int kind) : ctx(c) {
-        if (!c->profiling) return;
+        if (!c->profiling || !((c->prof_mask >> kind) & 1u)) return;
         if (c->prof_used == c->prof.size()) {
             ProfSlot s;
             if (cudaEventCreate(&s.begin) != cudaSuccess) return;

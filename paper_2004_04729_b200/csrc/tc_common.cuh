@@ -21,21 +21,25 @@ __device__ __forceinline__ void mbar_arrive(unsigned long long *bar) {
 __device__ __forceinline__ void mbar_arrive_on_cp_async(unsigned long long *bar) {
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// Returns false when the phase did not complete within about half a second.
+// Waits for the phase with the given parity. try_wait suspends the thread in hardware until the
+// phase completes or a short system time limit passes, so a waiter wakes as soon as the barrier
+// flips (a test_wait/nanosleep poll adds its sleep to every hand-over). Returns false, with the
+// error flag set, when the phase did not complete within about half a second.
+__device__ __forceinline__ bool mbar_try(unsigned addr, unsigned parity) {
+    unsigned done;
+    asm volatile(
+        "{\n\t.reg .pred P1;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, P1;\n\t}"
+        : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+    return done != 0;
+}
 __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity, int *err_flag) {
     const unsigned addr = smem_u32(bar);
+    if (mbar_try(addr, parity)) return true;
     const long long t0 = clock64();
-    for (;;) {
-        unsigned done;
-        asm volatile(
-            "{\n\t.reg .pred P1;\n\t"
-            "mbarrier.test_wait.parity.shared::cta.b64 P1, [%1], %2;\n\t"
-            "selp.b32 %0, 1, 0, P1;\n\t}"
-            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
-        if (done) return true;
-        if (clock64() - t0 > kWaitCycles) break;
-        __nanosleep(20);
-    }
+    while (clock64() - t0 <= kWaitCycles)
+        if (mbar_try(addr, parity)) return true;
     atomicExch(err_flag, 1);
     return false;
 }

@@ -456,17 +456,36 @@ __global__ void __launch_bounds__(kThreads3) tc3_dw_kernel(const P3 p) {
     }
 }
 
-// dW[co][ci][tap] = Delta * sum over splits of partials[split][tap][co][ci]
-__global__ void __launch_bounds__(256) tc3_dw_reduce_kernel(const float *__restrict__ partials, int nsplit,
+// dW[co][ci][tap] = Delta * sum over splits of partials[split][tap][co][ci]. A block spreads the
+// splits over its eight warps (lanes = 32 consecutive float4 of [tap][co][ci]) and combines the
+// eight partial sums in a fixed order.
+__global__ void __launch_bounds__(256) tc3_dw_reduce_kernel(const float4 *__restrict__ partials, int nsplit,
                                                             long long Cout, long long Cin,
                                                             const float *__restrict__ delta_p, float *__restrict__ dW) {
-    const float delta = *delta_p;
-    const long long n = Cout * Cin, tot = n * 9;
-    for (long long i = blockIdx.x * 256ll + threadIdx.x; i < tot; i += gridDim.x * 256ll) {
-        const long long tap = i / n, rem = i - tap * n;      // rem = co * Cin + ci (coalesced reads)
-        float a = 0.f;
-        for (int s = 0; s < nsplit; ++s) a += __ldcs(partials + (static_cast<long long>(s) * 9 + tap) * n + rem);
-        dW[rem * 9 + tap] = a * delta;
+    __shared__ float4 sh[8][32];
+    const long long n = Cout * Cin, tot4 = n * 9 / 4;            // Cin % 4 == 0
+    const int e = threadIdx.x & 31, sg = threadIdx.x >> 5;
+    const long long i4 = blockIdx.x * 32ll + e;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i4 < tot4) {
+#pragma unroll 4
+        for (int s = sg; s < nsplit; s += 8) {
+            const float4 v = __ldcs(partials + s * tot4 + i4);
+            a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+        }
+    }
+    sh[sg][e] = a;
+    __syncthreads();
+    if (sg == 0 && i4 < tot4) {
+#pragma unroll
+        for (int g = 1; g < 8; ++g) {
+            const float4 v = sh[g][e];
+            a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+        }
+        const float delta = *delta_p;
+        const long long i = i4 * 4, tap = i / n, rem = i - tap * n;      // rem = co * Cin + ci
+        float *dst = dW + rem * 9 + tap;
+        dst[0] = a.x * delta; dst[9] = a.y * delta; dst[18] = a.z * delta; dst[27] = a.w * delta;
     }
 }
 
@@ -560,10 +579,9 @@ int launch_tc3_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float 
         tc3_dw_kernel<1><<<grid, kThreads3, smem, ctx->stream>>>(p);
     }
     if ((rc = cuda_ok(cudaGetLastError()))) return rc;
-    long long blocks = (static_cast<long long>(nw) + 255) / 256;
-    if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
-    tc3_dw_reduce_kernel<<<static_cast<unsigned>(blocks), 256, 0, ctx->stream>>>(
-        p.partials, static_cast<int>(split), s.Cout, s.Cin, delta_p, dW);
+    const long long tot4 = static_cast<long long>(nw) / 4;
+    tc3_dw_reduce_kernel<<<static_cast<unsigned>((tot4 + 31) / 32), 256, 0, ctx->stream>>>(
+        reinterpret_cast<const float4 *>(p.partials), static_cast<int>(split), s.Cout, s.Cin, delta_p, dW);
     return cuda_ok(cudaGetLastError());
 }
 

@@ -5,9 +5,9 @@
 // The kernel is bound by HBM (every byte of X and of the codes is read once), so its pipeline
 // is built to keep many bytes in flight per SM: all global reads are cp.async copies issued
 // several stages ahead -- X straight into its 128-byte-swizzled operand tile, the int8 codes
-// into a raw staging tile -- and tracked by mbarriers; the eight producer warps then expand
+// into a raw staging tile -- and tracked by mbarriers; the producer warps then expand
 // the staged codes to bf16 from shared memory (no global latency on that path) while the next
-// stages' copies are already under way. A ninth warp issues the MMAs. K is split across CTAs;
+// stages' copies are already under way. One more warp issues the MMAs. K is split across CTAs;
 // partial blocks go to a workspace and a small kernel sums them and applies Delta.
 #include "tc_common.cuh"
 
@@ -19,6 +19,7 @@ using namespace tc;
 
 constexpr int kPW = 8;
 constexpr int kP = kPW * 32;
+constexpr int kRS = kP / 8;              // rows between two chunks of one producer thread
 constexpr int kThreadsDw = kP + 32;
 constexpr int kMaxS = 5;
 constexpr int kKT = 64;
@@ -78,11 +79,11 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
 
     if (warp < kPW) {
         const int tid = threadIdx.x;
-        const int c8 = tid & 7, rsub = tid >> 3;      // chunk column, first of my rows (stride 32)
+        const int c8 = tid & 7, rsub = tid >> 3;      // chunk column, first of my rows (stride kRS)
         bool ok = true;
-        // Addresses are kept incremental: a thread's rows are 32 apart (constant pointer and
+        // Addresses are kept incremental: a thread's rows are kRS apart (constant pointer and
         // shared-memory steps) and a stage advances every group by 64 flattened rows.
-        const long long xstep = 32 * p.P, cstep = 32 * p.P;
+        const long long xstep = kRS * p.P, cstep = kRS * p.P;
         const unsigned b_off0 = swz(rsub, c8), raw_off0 = rsub * 64 + c8 * 8;
         long long grow[NGRP > 2 ? 1 : NGRP], gb[NGRP > 2 ? 1 : NGRP], gp[NGRP > 2 ? 1 : NGRP];
         if (G > 1) {
@@ -108,22 +109,22 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
                     const __nv_bfloat16 *xs = p.X + (gb[g] * p.Cin + ci0 + rsub) * p.P + gp[g];
                     unsigned char *xd = b_s + b_off0 + g * 8;
 #pragma unroll
-                    for (int i = 0; i < NT / 32; ++i) {
-                        const bool v = gv && (ci0 + rsub + 32 * i < p.Cin);
+                    for (int i = 0; i < NT / kRS; ++i) {
+                        const bool v = gv && (ci0 + rsub + kRS * i < p.Cin);
                         if (G == 8) cp_async16(xd, v ? xs : p.X, v);
                         else cp_async_small<8>(xd, v ? xs : p.X, v);
                         xs += xstep;
-                        xd += 32 * 128;
+                        xd += kRS * 128;
                     }
                     const int8_t *cs = p.codes + (gb[g] * p.Cout + co0 + rsub) * p.P + gp[g];
                     unsigned char *cd = raw + raw_off0 + g * 4;
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const bool v = gv && (co0 + rsub + 32 * i < p.Cout);
+                    for (int i = 0; i < 128 / kRS; ++i) {
+                        const bool v = gv && (co0 + rsub + kRS * i < p.Cout);
                         if (G == 8) cp_async_small<8>(cd, v ? cs : p.codes, v);
                         else cp_async_small<4>(cd, v ? cs : p.codes, v);
                         cs += cstep;
-                        cd += 32 * 64;
+                        cd += kRS * 64;
                     }
                     // next stage: 64 rows further
                     grow[g] += kKT;
@@ -136,8 +137,8 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
                 const long long rr = r0 < p.rows ? r0 : 0;
                 const long long b0 = rr / p.P, q0 = rr - b0 * p.P;
                 const unsigned short *xs = reinterpret_cast<const unsigned short *>(p.X);
-                for (int i = 0; i < NT / 32; ++i) {
-                    const int row = rsub + 32 * i, ci = ci0 + row;
+                for (int i = 0; i < NT / kRS; ++i) {
+                    const int row = rsub + kRS * i, ci = ci0 + row;
                     unsigned short h[8];
                     long long b = b0, pp = q0;
 #pragma unroll
@@ -148,8 +149,8 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
                     *reinterpret_cast<uint4 *>(b_s + swz(row, c8)) =
                         make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
                 }
-                for (int i = 0; i < 4; ++i) {
-                    const int row = rsub + 32 * i, co = co0 + row;
+                for (int i = 0; i < 128 / kRS; ++i) {
+                    const int row = rsub + kRS * i, co = co0 + row;
                     unsigned w[2] = {0u, 0u};
                     long long b = b0, pp = q0;
 #pragma unroll
@@ -170,8 +171,8 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
             ok = ok && mbar_wait(&pipe.load_full[s], (it / S) & 1, p.err_flag);
             unsigned char *a_s = smem + s * STAGE, *raw = a_s + A_BYTES + B_BYTES;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int row = rsub + 32 * i;
+            for (int i = 0; i < 128 / kRS; ++i) {
+                const int row = rsub + kRS * i;
                 const uint2 c = *reinterpret_cast<const uint2 *>(raw + row * 64 + c8 * 8);
                 *reinterpret_cast<uint4 *>(a_s + swz(row, c8)) = expand8(c);
             }
@@ -181,11 +182,11 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
         // ---------------- epilogue: lanes = co rows, columns = ci -> partial block of this split
         if (niter > 0 && mbar_wait(&pipe.acc, 0, p.err_flag)) {
             tc_fence_after();
-            const int q = warp & 3, half = warp >> 2;
+            const int q = warp & 3, part = warp >> 2;      // lane quarter, first 32-column chunk
             const int co = co0 + q * 32 + lane;
             float *dst_row = p.partials + (static_cast<long long>(blockIdx.z) * p.Cout + co) * p.Cin + ci0;
 #pragma unroll 1
-            for (int c0 = half * (NT / 2); c0 < (half + 1) * (NT / 2); c0 += 32) {
+            for (int c0 = part * 32; c0 < NT; c0 += 32 * (kPW / 4)) {
                 unsigned r[32];
                 tmem_ld32(tmem_d + (static_cast<unsigned>(q * 32) << 16) + c0, r);
                 if (co < p.Cout) {
@@ -226,18 +227,33 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
     }
 }
 
-// dW = Delta * sum over splits of the partial blocks
-__global__ void __launch_bounds__(256) tc_dw_sum_kernel(const float *__restrict__ partials, int ksplit,
-                                                        long long n, const float *__restrict__ delta_p,
-                                                        float *__restrict__ dW) {
-    const float delta = *delta_p;
-    for (long long i = (blockIdx.x * 256ll + threadIdx.x) * 4; i < n; i += gridDim.x * 1024ll) {
-        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s = 0; s < ksplit; ++s) {
-            const float4 v = __ldcs(reinterpret_cast<const float4 *>(partials + s * n + i));
+// dW = Delta * sum over splits of the partial blocks. With few weights and many splits the sum
+// is a latency chain, so a block spreads the splits over its eight warps (lanes = 32 consecutive
+// float4 of the block) and combines the eight partial sums in a fixed order.
+__global__ void __launch_bounds__(256) tc_dw_sum_kernel(const float4 *__restrict__ partials, int ksplit,
+                                                        long long n4, const float *__restrict__ delta_p,
+                                                        float4 *__restrict__ dW) {
+    __shared__ float4 sh[8][32];
+    const int e = threadIdx.x & 31, sg = threadIdx.x >> 5;
+    const long long i4 = blockIdx.x * 32ll + e;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i4 < n4) {
+#pragma unroll 4
+        for (int s = sg; s < ksplit; s += 8) {
+            const float4 v = __ldcs(partials + s * n4 + i4);
             a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
         }
-        *reinterpret_cast<float4 *>(dW + i) = make_float4(a.x * delta, a.y * delta, a.z * delta, a.w * delta);
+    }
+    sh[sg][e] = a;
+    __syncthreads();
+    if (sg == 0 && i4 < n4) {
+#pragma unroll
+        for (int g = 1; g < 8; ++g) {
+            const float4 v = sh[g][e];
+            a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+        }
+        const float delta = *delta_p;
+        dW[i4] = make_float4(a.x * delta, a.y * delta, a.z * delta, a.w * delta);
     }
 }
 
@@ -286,11 +302,9 @@ int launch_tc_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *
     const size_t smem = static_cast<size_t>(p.stages) * (128 * 128 + nt * 128 + 128 * 64) + 1024;
     rc = nt == 256 ? run_g<256>(ctx, p, grid, smem) : nt == 128 ? run_g<128>(ctx, p, grid, smem) : run_g<64>(ctx, p, grid, smem);
     if (rc) return rc;
-    long long blocks = (static_cast<long long>(nw) / 4 + 255) / 256;
-    if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
-    if (blocks < 1) blocks = 1;
-    tc_dw_sum_kernel<<<static_cast<unsigned>(blocks), 256, 0, ctx->stream>>>(
-        p.partials, static_cast<int>(split), static_cast<long long>(nw), delta_p, dW);   // Cout*Cin % 4 == 0
+    const long long n4 = static_cast<long long>(nw) / 4;          // Cout * Cin % 4 == 0
+    tc_dw_sum_kernel<<<static_cast<unsigned>((n4 + 31) / 32), 256, 0, ctx->stream>>>(
+        reinterpret_cast<const float4 *>(p.partials), static_cast<int>(split), n4, delta_p, reinterpret_cast<float4 *>(dW));
     return cuda_ok(cudaGetLastError());
 }
 

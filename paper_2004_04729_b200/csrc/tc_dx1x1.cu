@@ -7,8 +7,8 @@
 //
 // Bound by HBM: the codes are read once and dX is written once. All global reads are cp.async
 // copies issued ahead of use (weights straight into their swizzled operand tile, code bytes
-// into a raw staging tile); eight producer warps expand the staged codes to bf16 from shared
-// memory; a ninth warp issues the MMAs.
+// into a raw staging tile); the producer warps expand the staged codes to bf16 from shared
+// memory; one more warp issues the MMAs.
 #include "tc_common.cuh"
 
 namespace dbp {
@@ -19,6 +19,7 @@ using namespace tc;
 
 constexpr int kPW = 8;
 constexpr int kP = kPW * 32;
+constexpr int kKS = kP / 16;             // k-rows between two chunks of one producer thread
 constexpr int kThreadsDx = kP + 32;
 constexpr int kMaxS = 5;
 constexpr int kKT = 64;
@@ -84,7 +85,7 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
 
     if (warp < kPW) {
         const int tid = threadIdx.x;
-        const int c16 = tid & 15, ksub = tid >> 4;     // my 8-row chunk of the tile, first k-row (stride 16)
+        const int c16 = tid & 15, ksub = tid >> 4;     // my 8-row chunk of the tile, first k-row (stride kKS)
         // where my chunk's groups live: the same for every stage
         const long long r0 = row0 + c16 * 8;
         long long gbase[NGRP > 2 ? 1 : NGRP];          // offset of (image, position) in channel 0, or -1
@@ -104,18 +105,18 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
             ok = ok && mbar_wait(&pipe.empty[s], ((j / S) & 1) ^ 1, p.err_flag);
             unsigned char *st = smem + s * STAGE;
             unsigned char *b_s = st + A_BYTES, *raw = b_s + B_BYTES;
-            // weights: k-row = co; my chunk column is c16 (8 channels), my k-rows ksub + 16 i.
-            // Pointers step by constants: 16 k-rows per i, 64 per stage.
+            // weights: k-row = co; my chunk column is c16 (8 channels), my k-rows ksub + kKS i.
+            // Pointers step by constants: kKS k-rows per i, 64 per stage.
             {
                 const int ci = ci0 + c16 * 8;
                 const __nv_bfloat16 *ws = p.W + static_cast<long long>(j * kKT + ksub) * p.Cin + ci;
                 unsigned char *wd = b_s + (c16 >> 3) * PANEL + swz(ksub, c16 & 7);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const bool v = (j * kKT + ksub + 16 * i < p.Cout) && ci < p.Cin;     // Cin % 8 == 0
+                for (int i = 0; i < kKT / kKS; ++i) {
+                    const bool v = (j * kKT + ksub + kKS * i < p.Cout) && ci < p.Cin;     // Cin % 8 == 0
                     cp_async16(wd, v ? ws : p.W, v);
-                    ws += 16 * static_cast<long long>(p.Cin);
-                    wd += 16 * 128;
+                    ws += kKS * static_cast<long long>(p.Cin);
+                    wd += kKS * 128;
                 }
             }
             // code bytes: k-row = co, my chunk of 8 rows
@@ -125,18 +126,18 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
                     const int8_t *cs = p.codes + gbase[g] + static_cast<long long>(j * kKT + ksub) * p.P;
                     unsigned char *cd = raw + ksub * 128 + c16 * 8 + g * 4;
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const bool v = gbase[g] >= 0 && (j * kKT + ksub + 16 * i < p.Cout);
+                    for (int i = 0; i < kKT / kKS; ++i) {
+                        const bool v = gbase[g] >= 0 && (j * kKT + ksub + kKS * i < p.Cout);
                         if (G == 8) cp_async_small<8>(cd, v ? cs : p.codes, v);
                         else cp_async_small<4>(cd, v ? cs : p.codes, v);
-                        cs += 16 * p.P;
-                        cd += 16 * 128;
+                        cs += kKS * p.P;
+                        cd += kKS * 128;
                     }
                 }
                 mbar_arrive_on_cp_async(&pipe.load_full[s]);
             } else {
-                for (int i = 0; i < 4; ++i) {
-                    const int k = ksub + 16 * i, co = j * kKT + k;
+                for (int i = 0; i < kKT / kKS; ++i) {
+                    const int k = ksub + kKS * i, co = j * kKT + k;
                     unsigned w[2] = {0u, 0u};
                     long long b = b0, pp = q0;
 #pragma unroll
@@ -159,8 +160,8 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
             ok = ok && mbar_wait(&pipe.load_full[s], (it / S) & 1, p.err_flag);
             unsigned char *a_s = smem + s * STAGE, *raw = a_s + A_BYTES + B_BYTES;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int k = ksub + 16 * i;
+            for (int i = 0; i < kKT / kKS; ++i) {
+                const int k = ksub + kKS * i;
                 const uint2 c = *reinterpret_cast<const uint2 *>(raw + k * 128 + c16 * 8);
                 *reinterpret_cast<uint4 *>(a_s + (c16 >> 3) * PANEL + swz(k, c16 & 7)) = expand8(c);
             }
@@ -168,15 +169,15 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
             mbar_arrive(&pipe.full[s]);
         }
         // ---------------- epilogue: TMEM lanes = input channels, columns = rows. Warp w takes lane
-        // quarter w % 4 and column half w / 4; a lane stores runs of consecutive positions.
+        // quarter w % 4 and the 32 columns w / 4; a lane stores runs of consecutive positions.
         if (mbar_wait(&pipe.acc, 0, p.err_flag)) {
             tc_fence_after();
             const float delta = *p.delta_p;
-            const int q = warp & 3, half = warp >> 2;
+            const int q = warp & 3, part = warp >> 2;
             const int ci = ci0 + q * 32 + lane;
             constexpr int RL = G >= 8 ? 8 : G;          // rows per store group
 #pragma unroll 1
-            for (int c0 = half * 64; c0 < half * 64 + 64; c0 += 32) {
+            for (int c0 = part * 32; c0 < 128; c0 += 32 * (kPW / 4)) {
                 unsigned v[32];
                 tmem_ld32(tmem_d + (static_cast<unsigned>(q * 32) << 16) + c0, v);
                 const long long rfirst = row0 + c0;
