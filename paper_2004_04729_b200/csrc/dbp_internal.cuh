@@ -105,6 +105,9 @@ int launch_tc3_dx_shift(dbp_ctx *ctx, const int8_t *codes, const void *W, const 
                         const ConvShape &s, void *dX, bool dx_bf16, int *err_flag);
 int launch_tc3_dx(dbp_ctx *ctx, const int8_t *codes, const void *W, const float *delta_p,
                   const ConvShape &s, void *dX, bool dx_bf16, int *err_flag);
+// row-shift variant of the 3x3 dW product: fills ctx->tc_partials and reports the split count
+int launch_tc3_dw_shift(dbp_ctx *ctx, const int8_t *codes, const void *X, const ConvShape &s,
+                        int *err_flag, long long *nsplit);
 int launch_tc3_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *delta_p,
                   const ConvShape &s, float *dW, int *err_flag);
 int launch_bias_grad(dbp_ctx *ctx, const int8_t *codes, const float *delta_p, const ConvShape &s,
@@ -135,6 +138,25 @@ struct KernelTimer {
         if (slot) cudaEventRecord(slot->end, ctx->stream);
     }
 };
+
+// Split of a K loop of `kunits` steps over CTAs when `tiles` output tiles exist and one CTA fits
+// per SM: the CTAs run in ceil(tiles * split / sms) waves of ceil(kunits / split) steps each, so
+// a split that spills a few CTAs into another wave doubles the time. Picks the split with the
+// fewest wave-steps (a CTA's fixed cost counted as two steps, a small charge per split for the
+// partial sums); *per_split receives the steps per CTA. The returned split has no empty part.
+inline long long choose_split(long long tiles, long long kunits, int sms, long long *per_split) {
+    long long best = 1, best_per = kunits;
+    double best_cost = 1e300;
+    const long long smax = kunits < 4ll * sms ? kunits : 4ll * sms;
+    for (long long want = 1; want <= smax; ++want) {
+        const long long per = (kunits + want - 1) / want, split = (kunits + per - 1) / per;
+        const long long waves = (tiles * split + sms - 1) / sms;
+        const double cost = static_cast<double>(waves) * static_cast<double>(per + 2) + 0.05 * static_cast<double>(split);
+        if (cost < best_cost) { best_cost = cost; best = split; best_per = per; }
+    }
+    *per_split = best_per;
+    return best;
+}
 
 inline int cuda_ok(cudaError_t e) { return e == cudaSuccess ? DBP_OK : DBP_ECUDA; }
 

@@ -17,6 +17,26 @@ __device__ __forceinline__ void mbar_init(unsigned long long *bar, int count) {
 __device__ __forceinline__ void mbar_arrive(unsigned long long *bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// One arrival for a whole warp: 256 threads arriving one by one on the same barrier word are
+// 256 serialized shared-memory atomics per hand-over; after __syncwarp the lanes' earlier
+// writes (and proxy fences) are ordered before lane 0's arrival.
+__device__ __forceinline__ void warp_arrive(unsigned long long *bar) {
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+}
+// cp.async groups: a thread closes a group after the copies of one stage and later waits until
+// at most `pending` newer groups are still in flight
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_pending(int pending) {
+    switch (pending) {
+        case 5: asm volatile("cp.async.wait_group 5;" ::: "memory"); break;
+        case 4: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
+        case 3: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+        case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
+        case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
+        default: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;   // fewer pending is always safe
+    }
+}
 // arrival that fires when this thread's earlier cp.async copies have landed
 __device__ __forceinline__ void mbar_arrive_on_cp_async(unsigned long long *bar) {
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -34,12 +54,24 @@ __device__ __forceinline__ bool mbar_try(unsigned addr, unsigned parity) {
         : "=r"(done) : "r"(addr), "r"(parity) : "memory");
     return done != 0;
 }
+__device__ __forceinline__ bool mbar_test(unsigned addr, unsigned parity) {
+    unsigned done;
+    asm volatile(
+        "{\n\t.reg .pred P1;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 P1, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, P1;\n\t}"
+        : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+    return done != 0;
+}
 __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity, int *err_flag) {
     const unsigned addr = smem_u32(bar);
-    if (mbar_try(addr, parity)) return true;
+    if (mbar_test(addr, parity)) return true;
     const long long t0 = clock64();
-    while (clock64() - t0 <= kWaitCycles)
-        if (mbar_try(addr, parity)) return true;
+    do {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_test(addr, parity)) return true;
+    } while (clock64() - t0 <= kWaitCycles);
     atomicExch(err_flag, 1);
     return false;
 }

@@ -544,8 +544,8 @@ int launch_tc3_dx(dbp_ctx *ctx, const int8_t *codes, const void *W, const float 
     return cuda_ok(cudaGetLastError());
 }
 
-int launch_tc3_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *delta_p,
-                  const ConvShape &s, float *dW, int *err_flag) {
+static int launch_tc3_dw_generic(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *delta_p,
+                                 const ConvShape &s, int *err_flag, long long *nsplit) {
     P3 p{};
     p.codes = codes; p.X = static_cast<const __nv_bfloat16 *>(X); p.delta_p = delta_p;
     p.B = static_cast<int>(s.B); p.Cin = static_cast<int>(s.Cin); p.Cout = static_cast<int>(s.Cout);
@@ -557,11 +557,7 @@ int launch_tc3_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float 
     if (rc) return rc;
     if (32 * p.raw_words > 9 * kProd) return DBP_EUNSUPPORTED;
     const long long tiles = ((s.Cin + 127) / 128) * ((s.Cout + 31) / 32);
-    long long split = (ctx->sm_count + tiles - 1) / tiles;
-    if (split > p.nstages) split = p.nstages;
-    if (split < 1) split = 1;
-    p.per_split = (p.nstages + split - 1) / split;
-    split = (p.nstages + p.per_split - 1) / p.per_split;
+    const long long split = choose_split(tiles, p.nstages, ctx->sm_count, &p.per_split);
     const size_t nw = static_cast<size_t>(s.Cout) * s.Cin * 9;
     if ((rc = ws_reserve(ctx, ctx->tc_partials, sizeof(float) * nw * split))) return rc;
     p.partials = static_cast<float *>(ctx->tc_partials.ptr);
@@ -578,10 +574,20 @@ int launch_tc3_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float 
         if ((rc = set_smem3(tc3_dw_kernel<1>, smem))) return rc;
         tc3_dw_kernel<1><<<grid, kThreads3, smem, ctx->stream>>>(p);
     }
-    if ((rc = cuda_ok(cudaGetLastError()))) return rc;
+    *nsplit = split;
+    return cuda_ok(cudaGetLastError());
+}
+
+int launch_tc3_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *delta_p,
+                  const ConvShape &s, float *dW, int *err_flag) {
+    const size_t nw = static_cast<size_t>(s.Cout) * s.Cin * 9;
+    long long split = 0;
+    int rc = launch_tc3_dw_shift(ctx, codes, X, s, err_flag, &split);
+    if (rc == DBP_EUNSUPPORTED) rc = launch_tc3_dw_generic(ctx, codes, X, delta_p, s, err_flag, &split);
+    if (rc) return rc;
     const long long tot4 = static_cast<long long>(nw) / 4;
     tc3_dw_reduce_kernel<<<static_cast<unsigned>((tot4 + 31) / 32), 256, 0, ctx->stream>>>(
-        reinterpret_cast<const float4 *>(p.partials), static_cast<int>(split), s.Cout, s.Cin, delta_p, dW);
+        reinterpret_cast<const float4 *>(ctx->tc_partials.ptr), static_cast<int>(split), s.Cout, s.Cin, delta_p, dW);
     return cuda_ok(cudaGetLastError());
 }
 

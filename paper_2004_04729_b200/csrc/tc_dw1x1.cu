@@ -5,7 +5,7 @@
 // The kernel is bound by HBM (every byte of X and of the codes is read once), so its pipeline
 // is built to keep many bytes in flight per SM: all global reads are cp.async copies issued
 // several stages ahead -- X straight into its 128-byte-swizzled operand tile, the int8 codes
-// into a raw staging tile -- and tracked by mbarriers; the producer warps then expand
+// into a raw staging tile -- and tracked by cp.async groups; the producer warps then expand
 // the staged codes to bf16 from shared memory (no global latency on that path) while the next
 // stages' copies are already under way. One more warp issues the MMAs. K is split across CTAs;
 // partial blocks go to a workspace and a small kernel sums them and applies Delta.
@@ -36,18 +36,23 @@ struct DwP {
 };
 
 struct PipeDw {
-    unsigned long long load_full[kMaxS], full[kMaxS], empty[kMaxS], acc;
+    unsigned long long full[kMaxS], empty[kMaxS], acc;
     unsigned tmem_base;
 };
 
 // G = rows per aligned, image-contained group: 8 (P % 8 == 0), 4 (P % 4 == 0) or 1 (any P).
+// G = 0 is the slab mode for small planes (9 <= P <= 64) of any alignment: a K stage is one
+// image (its P positions, zero-padded to 64); the [128 co][P] code block and the [NT ci][P]
+// activation block of an image are contiguous in memory, so both are staged by 16-byte
+// cp.async copies and re-laid into the operand tiles from shared memory.
 template <int NT, int G>
 __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
     constexpr int A_BYTES = 128 * 128;
     constexpr int B_BYTES = NT * 128;
     constexpr int RAW_BYTES = 128 * 64;
-    constexpr int STAGE = A_BYTES + B_BYTES + RAW_BYTES;
-    constexpr int NGRP = 8 / G;
+    constexpr int XRAW_BYTES = G == 0 ? NT * 128 : 0;       // slab mode: staged activations
+    constexpr int STAGE = A_BYTES + B_BYTES + RAW_BYTES + XRAW_BYTES;
+    constexpr int NGRP = G == 0 ? 1 : 8 / G;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ PipeDw pipe;
@@ -64,8 +69,7 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
-            mbar_init(&pipe.load_full[s], kP);
-            mbar_init(&pipe.full[s], kP);
+            mbar_init(&pipe.full[s], kPW);             // one arrival per producer warp
             mbar_init(&pipe.empty[s], 1);
         }
         mbar_init(&pipe.acc, 1);
@@ -102,7 +106,16 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
             unsigned char *st = smem + s * STAGE;
             unsigned char *b_s = st + A_BYTES, *raw = b_s + B_BYTES;
             const long long r0 = (ks0 + j) * kKT + c8 * 8;
-            if (G > 1) {
+            if (G == 0) {
+                const long long b = ks0 + j;                 // this stage's image
+                const int P = static_cast<int>(p.P);
+                const int nco = p.Cout - co0 < 128 ? p.Cout - co0 : 128, nci = p.Cin - ci0 < NT ? p.Cin - ci0 : NT;
+                const int8_t *cs = p.codes + (b * p.Cout + co0) * p.P;
+                for (int idx = tid; idx * 16 < nco * P; idx += kP) cp_async16(raw + idx * 16, cs + idx * 16, true);
+                const __nv_bfloat16 *xs = p.X + (b * p.Cin + ci0) * p.P;
+                unsigned char *rawx = raw + RAW_BYTES;
+                for (int idx = tid; idx * 8 < nci * P; idx += kP) cp_async16(rawx + idx * 16, xs + idx * 8, true);
+            } else if (G > 1) {
 #pragma unroll
                 for (int g = 0; g < NGRP; ++g) {
                     const bool gv = grow[g] < p.rows;
@@ -131,7 +144,6 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
                     gp[g] += kKT;
                     while (gp[g] >= p.P) { gp[g] -= p.P; ++gb[g]; }
                 }
-                mbar_arrive_on_cp_async(&pipe.load_full[s]);
             } else {
                 // element-wise: walk the eight rows from (b, p)
                 const long long rr = r0 < p.rows ? r0 : 0;
@@ -161,23 +173,75 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
                     }
                     *reinterpret_cast<uint2 *>(raw + row * 64 + c8 * 8) = make_uint2(w[0], w[1]);
                 }
-                mbar_arrive(&pipe.load_full[s]);
             }
         };
-        for (int j = 0; j < LA && j < niter; ++j) issue(j);
+        // every thread closes one cp.async group per stage (empty once the copies run out), so
+        // "at most LA groups pending" means the copies of stage `it` have landed
+        for (int j = 0; j < LA; ++j) {
+            if (j < niter) issue(j);
+            cp_async_commit();
+        }
         for (int it = 0; it < niter; ++it) {
             if (it + LA < niter) issue(it + LA);
+            cp_async_commit();
             const int s = it % S;
-            ok = ok && mbar_wait(&pipe.load_full[s], (it / S) & 1, p.err_flag);
+            cp_async_wait_pending(LA);
+            if (G == 0) asm volatile("bar.sync 1, %0;" ::"n"(kP) : "memory");   // slabs are read across threads
             unsigned char *a_s = smem + s * STAGE, *raw = a_s + A_BYTES + B_BYTES;
+            if (G == 0) {
+                // my chunk covers positions c8*8 .. c8*8+7 of the image; nv of them exist
+                const int P = static_cast<int>(p.P);
+                const int nv = P - c8 * 8 >= 8 ? 8 : (P - c8 * 8 > 0 ? P - c8 * 8 : 0);
+                const int nco = p.Cout - co0 < 128 ? p.Cout - co0 : 128, nci = p.Cin - ci0 < NT ? p.Cin - ci0 : NT;
+                // byte masks of the valid positions
+                const unsigned m0 = nv >= 4 ? 0xffffffffu : (nv > 0 ? (1u << (8 * nv)) - 1u : 0u);
+                const unsigned m1 = nv >= 8 ? 0xffffffffu : (nv > 4 ? (1u << (8 * (nv - 4))) - 1u : 0u);
+                const unsigned *rawc_w = reinterpret_cast<const unsigned *>(raw);
+#pragma unroll
+                for (int i = 0; i < 128 / kRS; ++i) {
+                    const int row = rsub + kRS * i;
+                    uint4 e = make_uint4(0u, 0u, 0u, 0u);
+                    if (row < nco && nv > 0) {
+                        // eight bytes from byte offset row * P + c8 * 8 (any alignment)
+                        const int off = row * P + c8 * 8, wi = off >> 2;
+                        const unsigned sel = 0x3210u + 0x1111u * static_cast<unsigned>(off & 3);
+                        const unsigned w0 = rawc_w[wi], w1 = rawc_w[wi + 1], w2 = rawc_w[wi + 2];
+                        e = expand8(make_uint2(__byte_perm(w0, w1, sel) & m0, __byte_perm(w1, w2, sel) & m1));
+                    }
+                    *reinterpret_cast<uint4 *>(a_s + swz(row, c8)) = e;
+                }
+                const unsigned *rawx_w = reinterpret_cast<const unsigned *>(raw + RAW_BYTES);
+                unsigned char *b_t = a_s + A_BYTES;
+                // 16-bit element masks for the four words of a chunk
+                const unsigned x0 = nv >= 2 ? 0xffffffffu : (nv == 1 ? 0xffffu : 0u);
+                const unsigned x1 = nv >= 4 ? 0xffffffffu : (nv == 3 ? 0xffffu : 0u);
+                const unsigned x2 = nv >= 6 ? 0xffffffffu : (nv == 5 ? 0xffffu : 0u);
+                const unsigned x3 = nv >= 8 ? 0xffffffffu : (nv == 7 ? 0xffffu : 0u);
+#pragma unroll
+                for (int i = 0; i < NT / kRS; ++i) {
+                    const int row = rsub + kRS * i;
+                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                    if (row < nci && nv > 0) {
+                        // eight bf16 from element offset row * P + c8 * 8 (2-byte aligned)
+                        const int off = row * P + c8 * 8, wi = off >> 1;
+                        const unsigned sh = (off & 1) * 16;
+                        const unsigned w0 = rawx_w[wi], w1 = rawx_w[wi + 1], w2 = rawx_w[wi + 2], w3 = rawx_w[wi + 3],
+                                       w4 = rawx_w[wi + 4];
+                        v = make_uint4(__funnelshift_r(w0, w1, sh) & x0, __funnelshift_r(w1, w2, sh) & x1,
+                                       __funnelshift_r(w2, w3, sh) & x2, __funnelshift_r(w3, w4, sh) & x3);
+                    }
+                    *reinterpret_cast<uint4 *>(b_t + swz(row, c8)) = v;
+                }
+            } else {
 #pragma unroll
             for (int i = 0; i < 128 / kRS; ++i) {
                 const int row = rsub + kRS * i;
                 const uint2 c = *reinterpret_cast<const uint2 *>(raw + row * 64 + c8 * 8);
                 *reinterpret_cast<uint4 *>(a_s + swz(row, c8)) = expand8(c);
             }
+            }
             fence_async_proxy();
-            mbar_arrive(&pipe.full[s]);
+            warp_arrive(&pipe.full[s]);
         }
         // ---------------- epilogue: lanes = co rows, columns = ci -> partial block of this split
         if (niter > 0 && mbar_wait(&pipe.acc, 0, p.err_flag)) {
@@ -267,7 +331,8 @@ int run(dbp_ctx *ctx, const DwP &p, dim3 grid, size_t smem) {
 }
 
 template <int NT>
-int run_g(dbp_ctx *ctx, const DwP &p, dim3 grid, size_t smem) {
+int run_g(dbp_ctx *ctx, const DwP &p, dim3 grid, size_t smem, bool slab) {
+    if (slab) return run<(NT > 128 ? 128 : NT), 0>(ctx, p, grid, smem);
     if (p.P % 8 == 0) return run<NT, 8>(ctx, p, grid, smem);
     if (p.P % 4 == 0) return run<NT, 4>(ctx, p, grid, smem);
     return run<NT, 1>(ctx, p, grid, smem);
@@ -281,17 +346,14 @@ int launch_tc_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *
     p.codes = codes; p.X = static_cast<const __nv_bfloat16 *>(X);
     p.Cin = static_cast<int>(s.Cin); p.Cout = static_cast<int>(s.Cout);
     p.P = s.H * s.W; p.rows = s.B * p.P;
-    p.kstages = (p.rows + kKT - 1) / kKT;
     p.err_flag = err_flag;
-    const int nt = s.Cin >= 256 ? 256 : s.Cin > 64 ? 128 : 64;
+    // small planes of awkward size: one image per K stage, staged as contiguous slabs
+    const bool slab = p.P % 4 != 0 && p.P >= 9 && p.P <= 64 && s.Cout % 16 == 0 && s.Cin % 8 == 0;
+    p.kstages = slab ? s.B : (p.rows + kKT - 1) / kKT;
+    const int nt = slab ? (s.Cin > 64 ? 128 : 64) : s.Cin >= 256 ? 256 : s.Cin > 64 ? 128 : 64;
     const long long tiles = ((s.Cout + 127) / 128) * ((s.Cin + nt - 1) / nt);
-    // split K so that every SM has a CTA, without empty splits
-    long long split = (ctx->sm_count + tiles - 1) / tiles;
-    if (split > p.kstages) split = p.kstages;
-    if (split < 1) split = 1;
-    p.per_split = (p.kstages + split - 1) / split;
-    split = (p.kstages + p.per_split - 1) / p.per_split;
-    const int max_s = nt == 256 ? 4 : kMaxS;
+    const long long split = choose_split(tiles, p.kstages, ctx->sm_count, &p.per_split);
+    const int max_s = (nt == 256 || slab) ? 4 : kMaxS;
     p.stages = p.per_split < max_s ? static_cast<int>(p.per_split) : max_s;
     const size_t nw = static_cast<size_t>(s.Cout) * s.Cin;
     int rc = ws_reserve(ctx, ctx->tc_partials, sizeof(float) * nw * split);
@@ -299,8 +361,9 @@ int launch_tc_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *
     p.partials = static_cast<float *>(ctx->tc_partials.ptr);
     dim3 grid(static_cast<unsigned>((s.Cout + 127) / 128), static_cast<unsigned>((s.Cin + nt - 1) / nt),
               static_cast<unsigned>(split));
-    const size_t smem = static_cast<size_t>(p.stages) * (128 * 128 + nt * 128 + 128 * 64) + 1024;
-    rc = nt == 256 ? run_g<256>(ctx, p, grid, smem) : nt == 128 ? run_g<128>(ctx, p, grid, smem) : run_g<64>(ctx, p, grid, smem);
+    const size_t smem = static_cast<size_t>(p.stages) * (128 * 128 + nt * 128 + 128 * 64 + (slab ? nt * 128 : 0)) + 1024 + 64;
+    rc = nt == 256 ? run_g<256>(ctx, p, grid, smem, slab) : nt == 128 ? run_g<128>(ctx, p, grid, smem, slab)
+                                                                      : run_g<64>(ctx, p, grid, smem, slab);
     if (rc) return rc;
     const long long n4 = static_cast<long long>(nw) / 4;          // Cout * Cin % 4 == 0
     tc_dw_sum_kernel<<<static_cast<unsigned>((n4 + 31) / 32), 256, 0, ctx->stream>>>(

@@ -37,7 +37,7 @@ struct DxP {
 };
 
 struct PipeDx {
-    unsigned long long load_full[kMaxS], full[kMaxS], empty[kMaxS], acc;
+    unsigned long long full[kMaxS], empty[kMaxS], acc;
     unsigned tmem_base;
 };
 
@@ -48,14 +48,18 @@ __device__ __forceinline__ void st_global_v8(void *dst, const unsigned (&w)[8]) 
 }
 
 // G = rows per aligned, image-contained group: 8 (P % 8 == 0), 4 (P % 4 == 0) or 1 (any P).
+// G = 0 is the slab mode for small planes (9 <= P <= 64) of any alignment: the [64 co][P] code
+// blocks of the images a row tile touches are contiguous in memory and are staged whole by
+// 16-byte cp.async copies; the expansion gathers its eight rows from them (a chunk of eight
+// rows crosses at most one image boundary).
 template <int NT, int G>
 __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
     constexpr int A_BYTES = 2 * kKT * 128;          // codes: two 64-row groups x 64 k-rows
     constexpr int B_BYTES = (NT / 64) * kKT * 128;
-    constexpr int RAW_BYTES = kKT * 128;            // 64 co x 128 rows, one byte each
+    constexpr int RAW_BYTES = G == 0 ? 2 * kKT * 128 : kKT * 128;   // 64 co x 128 rows, one byte each (slabs: up to twice that)
     constexpr int STAGE = A_BYTES + B_BYTES + RAW_BYTES;
     constexpr unsigned PANEL = kKT * 128;
-    constexpr int NGRP = 8 / G;
+    constexpr int NGRP = G == 0 ? 1 : 8 / G;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ PipeDx pipe;
@@ -70,8 +74,7 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
-            mbar_init(&pipe.load_full[s], kP);
-            mbar_init(&pipe.full[s], kP);
+            mbar_init(&pipe.full[s], kPW);             // one arrival per producer warp
             mbar_init(&pipe.empty[s], 1);
         }
         mbar_init(&pipe.acc, 1);
@@ -99,6 +102,32 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
         }
         const long long rr0 = r0 < p.rows ? r0 : 0;
         const long long b0 = rr0 / p.P, q0 = rr0 - b0 * p.P;
+        // slab mode: staged images img_lo .. img_lo + nimg - 1 as [image][64 co][P]; my copies are
+        // the 16-byte chunks tid + kP i; my chunk of eight rows starts at slab byte s_base (k-row 0)
+        // and continues in the next image after `split` rows
+        const int Pi = static_cast<int>(p.P);
+        const long long img_lo = row0 / p.P;
+        int s_dst[4], s_base = 0, split = 8, nvr = 0;
+        long long s_src[4];
+        if (G == 0) {
+            const long long last_row = (row0 + 127 < p.rows ? row0 + 127 : p.rows - 1);
+            const int nimg = static_cast<int>(last_row / p.P - img_lo) + 1;
+            const int per_img = 4 * Pi;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int idx = tid + kP * i;
+                s_dst[i] = -1;
+                s_src[i] = -1;
+                if (idx < nimg * per_img) {
+                    const int img = idx / per_img, k16 = idx - img * per_img;
+                    s_dst[i] = img * 64 * Pi + 16 * k16;
+                    s_src[i] = (img_lo + img) * p.Cout * p.P + 16 * k16;      // image exists: it holds a row of the tile
+                }
+            }
+            nvr = r0 < p.rows ? static_cast<int>(p.rows - r0 < 8 ? p.rows - r0 : 8) : 0;
+            s_base = static_cast<int>(b0 - img_lo) * 64 * Pi + static_cast<int>(q0);
+            split = Pi - static_cast<int>(q0) < 8 ? Pi - static_cast<int>(q0) : 8;
+        }
         bool ok = true;
         auto issue = [&](int j) {
             const int s = j % S;
@@ -120,7 +149,12 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
                 }
             }
             // code bytes: k-row = co, my chunk of 8 rows
-            if (G > 1) {
+            if (G == 0) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (s_dst[i] >= 0)
+                        cp_async16(raw + s_dst[i], p.codes + s_src[i] + static_cast<long long>(j) * kKT * p.P, true);
+            } else if (G > 1) {
 #pragma unroll
                 for (int g = 0; g < NGRP; ++g) {
                     const int8_t *cs = p.codes + gbase[g] + static_cast<long long>(j * kKT + ksub) * p.P;
@@ -134,7 +168,6 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
                         cd += kKS * 128;
                     }
                 }
-                mbar_arrive_on_cp_async(&pipe.load_full[s]);
             } else {
                 for (int i = 0; i < kKT / kKS; ++i) {
                     const int k = ksub + kKS * i, co = j * kKT + k;
@@ -148,25 +181,60 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
                     }
                     *reinterpret_cast<uint2 *>(raw + k * 128 + c16 * 8) = make_uint2(w[0], w[1]);
                 }
-                // the weight copies above are still asynchronous: count them, then arrive
-                asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
-                mbar_arrive(&pipe.load_full[s]);
             }
         };
-        for (int j = 0; j < LA && j < niter; ++j) issue(j);
+        // every thread closes one cp.async group per stage (empty once the copies run out), so
+        // "at most LA groups pending" means the copies of stage `it` have landed
+        for (int j = 0; j < LA; ++j) {
+            if (j < niter) issue(j);
+            cp_async_commit();
+        }
         for (int it = 0; it < niter; ++it) {
             if (it + LA < niter) issue(it + LA);
+            cp_async_commit();
             const int s = it % S;
-            ok = ok && mbar_wait(&pipe.load_full[s], (it / S) & 1, p.err_flag);
+            cp_async_wait_pending(LA);
+            if (G == 0) asm volatile("bar.sync 1, %0;" ::"n"(kP) : "memory");   // slabs are read across threads
             unsigned char *a_s = smem + s * STAGE, *raw = a_s + A_BYTES + B_BYTES;
+            if (G == 0) {
+                // byte e of my chunk is row r0 + e: before `split` it lies in image b0, after it in
+                // the next image, 63 P bytes further in the slab layout; rows beyond the end are zero
+                const unsigned long long keep = nvr >= 8 ? ~0ull : ((1ull << (8 * nvr)) - 1ull);
+                const unsigned long long first = split >= 8 ? ~0ull : ((1ull << (8 * split)) - 1ull);
+                const unsigned *raw_w = reinterpret_cast<const unsigned *>(raw);
+#pragma unroll
+                for (int i = 0; i < kKT / kKS; ++i) {
+                    const int k = ksub + kKS * i;
+                    uint4 e = make_uint4(0u, 0u, 0u, 0u);
+                    if (nvr > 0) {
+                        const int off = s_base + k * Pi, wi = off >> 2;
+                        const unsigned sel = 0x3210u + 0x1111u * static_cast<unsigned>(off & 3);
+                        const unsigned w0 = raw_w[wi], w1 = raw_w[wi + 1], w2 = raw_w[wi + 2];
+                        unsigned long long c = __byte_perm(w0, w1, sel) |
+                                               (static_cast<unsigned long long>(__byte_perm(w1, w2, sel)) << 32);
+                        if (split < nvr) {      // a row of the next image exists (and that image is staged)
+                            const int off2 = off + 63 * Pi, wj = off2 >> 2;
+                            const unsigned sel2 = 0x3210u + 0x1111u * static_cast<unsigned>(off2 & 3);
+                            const unsigned v0 = raw_w[wj], v1 = raw_w[wj + 1], v2 = raw_w[wj + 2];
+                            const unsigned long long c2 = __byte_perm(v0, v1, sel2) |
+                                                          (static_cast<unsigned long long>(__byte_perm(v1, v2, sel2)) << 32);
+                            c = (c & first) | (c2 & ~first);
+                        }
+                        c &= keep;
+                        e = expand8(make_uint2(static_cast<unsigned>(c), static_cast<unsigned>(c >> 32)));
+                    }
+                    *reinterpret_cast<uint4 *>(a_s + (c16 >> 3) * PANEL + swz(k, c16 & 7)) = e;
+                }
+            } else {
 #pragma unroll
             for (int i = 0; i < kKT / kKS; ++i) {
                 const int k = ksub + kKS * i;
                 const uint2 c = *reinterpret_cast<const uint2 *>(raw + k * 128 + c16 * 8);
                 *reinterpret_cast<uint4 *>(a_s + (c16 >> 3) * PANEL + swz(k, c16 & 7)) = expand8(c);
             }
+            }
             fence_async_proxy();
-            mbar_arrive(&pipe.full[s]);
+            warp_arrive(&pipe.full[s]);
         }
         // ---------------- epilogue: TMEM lanes = input channels, columns = rows. Warp w takes lane
         // quarter w % 4 and the 32 columns w / 4; a lane stores runs of consecutive positions.
@@ -175,7 +243,7 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
             const float delta = *p.delta_p;
             const int q = warp & 3, part = warp >> 2;
             const int ci = ci0 + q * 32 + lane;
-            constexpr int RL = G >= 8 ? 8 : G;          // rows per store group
+            constexpr int RL = G >= 8 ? 8 : (G == 0 ? 1 : G);          // rows per store group
 #pragma unroll 1
             for (int c0 = part * 32; c0 < 128; c0 += 32 * (kPW / 4)) {
                 unsigned v[32];
@@ -287,7 +355,8 @@ int run(dbp_ctx *ctx, const DxP &p, dim3 grid, size_t smem) {
 }
 
 template <int NT>
-int run_g(dbp_ctx *ctx, const DxP &p, dim3 grid, size_t smem) {
+int run_g(dbp_ctx *ctx, const DxP &p, dim3 grid, size_t smem, bool slab) {
+    if (slab) return run<NT, 0>(ctx, p, grid, smem);
     if (p.P % 8 == 0) return run<NT, 8>(ctx, p, grid, smem);
     if (p.P % 4 == 0) return run<NT, 4>(ctx, p, grid, smem);
     return run<NT, 1>(ctx, p, grid, smem);
@@ -308,12 +377,15 @@ int launch_tc_dx(dbp_ctx *ctx, const int8_t *codes, const void *W, const float *
     p.P = s.H * s.W; p.rows = s.B * p.P;
     p.err_flag = err_flag;
     const int niter = static_cast<int>((s.Cout + kKT - 1) / kKT);
-    p.stages = niter < kMaxS ? niter : kMaxS;
+    // small planes of awkward size: stage whole [64 co][P] blocks of the touched images
+    const bool slab = p.P % 4 != 0 && p.P >= 9 && p.P <= 64 && s.Cout % 64 == 0;
+    const int max_s = slab ? 4 : kMaxS;
+    p.stages = niter < max_s ? niter : max_s;
     // one CTA: 128 rows x 128 channels; few stages leave room for several CTAs per SM, which
     // overlaps the load, MMA and store phases of different tiles
     dim3 grid(static_cast<unsigned>((p.rows + 127) / 128), static_cast<unsigned>((s.Cin + 127) / 128));
-    const size_t smem = static_cast<size_t>(p.stages) * (2 * kKT * 128 + 2 * kKT * 128 + kKT * 128) + 1024;
-    return run_g<128>(ctx, p, grid, smem);
+    const size_t smem = static_cast<size_t>(p.stages) * (2 * kKT * 128 + 2 * kKT * 128 + (slab ? 2 : 1) * kKT * 128) + 1024 + 64;
+    return run_g<128>(ctx, p, grid, smem, slab);
 }
 
 }  // namespace dbp

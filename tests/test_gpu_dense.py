@@ -55,6 +55,10 @@ def _run(ctx, L, flags):
     (5, 128, 512, 7, 7),      # 49 positions per image: element-wise loads, ragged row tiles
     (2, 72, 40, 5, 9),        # channel counts that fill neither tile
     (1, 1024, 256, 14, 14),
+    (3, 64, 64, 3, 3),        # slab staging, smallest plane (9 positions): 15 images per row tile
+    (2, 136, 128, 8, 7),      # slab staging, 56 positions, ragged channel tile
+    (4, 64, 192, 9, 7),       # slab staging, 63 positions
+    (7, 2048, 512, 7, 7),     # ResNet stage-4 reduce at a small batch, rows end inside a tile
 ])
 def test_dense_path_conv1x1(ctx, B, Ci, Co, H, W):
     import paper_2004_04729_b200 as dbp
@@ -75,6 +79,8 @@ def test_dense_path_conv1x1(ctx, B, Ci, Co, H, W):
     (3, 200, 128, 6, 6),      # row-shift dX kernel, slabs of 36 positions, ragged channel tile
     (5, 64, 64, 5, 7),        # row-shift dX kernel, odd plane size: byte-aligned slabs
     (240, 512, 64, 8, 8),     # row-shift dX kernel, four accumulators per CTA
+    (2, 64, 32, 6, 4),        # row-shift dW kernel: 24 positions, 16-byte activation copies with slab-staged codes
+    (3, 136, 96, 20, 16),     # row-shift kernels: 320 positions = two segments per image, ragged channel tile
 ])
 def test_dense_path_conv3x3(ctx, B, Ci, Co, H, W):
     import paper_2004_04729_b200 as dbp
