@@ -89,20 +89,37 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
         // shared-memory steps) and a stage advances every group by 64 flattened rows.
         const long long xstep = kRS * p.P, cstep = kRS * p.P;
         const unsigned b_off0 = swz(rsub, c8), raw_off0 = rsub * 64 + c8 * 8;
-        long long grow[NGRP > 2 ? 1 : NGRP], gb[NGRP > 2 ? 1 : NGRP], gp[NGRP > 2 ? 1 : NGRP];
+        // Per group: flattened row, position inside its image and the source pointers of my first
+        // row, all advanced by 64 rows per stage (a pointer jumps by (C - 1) P when the group
+        // moves on to the next image). Row-exists masks and ring position are kept likewise, so a
+        // stage costs no division and no 64-bit multiply.
+        long long grow[NGRP > 2 ? 1 : NGRP], gp[NGRP > 2 ? 1 : NGRP];
+        const __nv_bfloat16 *xptr[NGRP > 2 ? 1 : NGRP];
+        const int8_t *cptr[NGRP > 2 ? 1 : NGRP];
+        unsigned xmask = 0, cmask = 0;
+        const long long xwrap = (p.Cin - 1) * p.P, cwrap = (p.Cout - 1) * p.P;
         if (G > 1) {
 #pragma unroll
             for (int g = 0; g < NGRP; ++g) {
                 grow[g] = ks0 * kKT + c8 * 8 + g * G;
-                gb[g] = grow[g] / p.P;
-                gp[g] = grow[g] - gb[g] * p.P;
+                const long long gb = grow[g] / p.P;
+                gp[g] = grow[g] - gb * p.P;
+                xptr[g] = p.X + (gb * p.Cin + ci0 + rsub) * p.P + gp[g];
+                cptr[g] = p.codes + (gb * p.Cout + co0 + rsub) * p.P + gp[g];
             }
+#pragma unroll
+            for (int i = 0; i < NT / kRS; ++i) xmask |= (ci0 + rsub + kRS * i < p.Cin ? 1u : 0u) << i;
+#pragma unroll
+            for (int i = 0; i < 128 / kRS; ++i) cmask |= (co0 + rsub + kRS * i < p.Cout ? 1u : 0u) << i;
         }
+        int is = 0;                 // ring slot of the next stage to fill
+        unsigned iparity = 1;       // parity to wait for on its empty barrier
         // copies of local stage j (called for j = 0, 1, 2, ... in order): X chunks into the
         // operand tile, code bytes into the raw tile
         auto issue = [&](int j) {
-            const int s = j % S;
-            ok = ok && mbar_wait(&pipe.empty[s], ((j / S) & 1) ^ 1, p.err_flag);
+            const int s = is;
+            ok = ok && mbar_wait(&pipe.empty[s], iparity, p.err_flag);
+            if (++is == S) { is = 0; iparity ^= 1u; }
             unsigned char *st = smem + s * STAGE;
             unsigned char *b_s = st + A_BYTES, *raw = b_s + B_BYTES;
             const long long r0 = (ks0 + j) * kKT + c8 * 8;
@@ -119,21 +136,21 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
 #pragma unroll
                 for (int g = 0; g < NGRP; ++g) {
                     const bool gv = grow[g] < p.rows;
-                    const __nv_bfloat16 *xs = p.X + (gb[g] * p.Cin + ci0 + rsub) * p.P + gp[g];
+                    const __nv_bfloat16 *xs = xptr[g];
                     unsigned char *xd = b_s + b_off0 + g * 8;
 #pragma unroll
                     for (int i = 0; i < NT / kRS; ++i) {
-                        const bool v = gv && (ci0 + rsub + kRS * i < p.Cin);
+                        const bool v = gv && ((xmask >> i) & 1u);
                         if (G == 8) cp_async16(xd, v ? xs : p.X, v);
                         else cp_async_small<8>(xd, v ? xs : p.X, v);
                         xs += xstep;
                         xd += kRS * 128;
                     }
-                    const int8_t *cs = p.codes + (gb[g] * p.Cout + co0 + rsub) * p.P + gp[g];
+                    const int8_t *cs = cptr[g];
                     unsigned char *cd = raw + raw_off0 + g * 4;
 #pragma unroll
                     for (int i = 0; i < 128 / kRS; ++i) {
-                        const bool v = gv && (co0 + rsub + kRS * i < p.Cout);
+                        const bool v = gv && ((cmask >> i) & 1u);
                         if (G == 8) cp_async_small<8>(cd, v ? cs : p.codes, v);
                         else cp_async_small<4>(cd, v ? cs : p.codes, v);
                         cs += cstep;
@@ -142,7 +159,9 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
                     // next stage: 64 rows further
                     grow[g] += kKT;
                     gp[g] += kKT;
-                    while (gp[g] >= p.P) { gp[g] -= p.P; ++gb[g]; }
+                    xptr[g] += kKT;
+                    cptr[g] += kKT;
+                    while (gp[g] >= p.P) { gp[g] -= p.P; xptr[g] += xwrap; cptr[g] += cwrap; }
                 }
             } else {
                 // element-wise: walk the eight rows from (b, p)
@@ -177,6 +196,7 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
         };
         // every thread closes one cp.async group per stage (empty once the copies run out), so
         // "at most LA groups pending" means the copies of stage `it` have landed
+        int cslot = 0;              // ring slot of the stage being expanded
         for (int j = 0; j < LA; ++j) {
             if (j < niter) issue(j);
             cp_async_commit();
@@ -184,7 +204,8 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
         for (int it = 0; it < niter; ++it) {
             if (it + LA < niter) issue(it + LA);
             cp_async_commit();
-            const int s = it % S;
+            const int s = cslot;
+            if (++cslot == S) cslot = 0;
             cp_async_wait_pending(LA);
             if (G == 0) asm volatile("bar.sync 1, %0;" ::"n"(kP) : "memory");   // slabs are read across threads
             unsigned char *a_s = smem + s * STAGE, *raw = a_s + A_BYTES + B_BYTES;
@@ -269,9 +290,10 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
     } else if (lane == 0) {
         constexpr unsigned idesc = make_idesc(128, NT, false, false);
         bool ok = true;
+        int s = 0;
+        unsigned parity = 0;
         for (int it = 0; it < niter && ok; ++it) {
-            const int s = it % S;
-            ok = mbar_wait(&pipe.full[s], (it / S) & 1, p.err_flag);
+            ok = mbar_wait(&pipe.full[s], parity, p.err_flag);
             fence_async_proxy();
             tc_fence_after();
             const unsigned a_addr = smem_u32(smem + s * STAGE), b_addr = a_addr + A_BYTES;
@@ -280,6 +302,7 @@ __global__ void __launch_bounds__(kThreadsDw) tc_dw_async_kernel(const DwP p) {
             for (int k = 0; k < kKT / 16; ++k)
                 mma_bf16(tmem_d, ad + 2 * k, bd + 2 * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
             mma_commit(&pipe.empty[s]);
+            if (++s == S) { s = 0; parity ^= 1u; }
         }
         if (niter > 0) mma_commit(&pipe.acc);
     }

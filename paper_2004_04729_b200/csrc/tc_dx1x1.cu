@@ -100,6 +100,11 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
                 gbase[g] = r < p.rows ? b * p.Cout * p.P + (r - b * p.P) : -1;
             }
         }
+        const int8_t *cptr[NGRP > 2 ? 1 : NGRP];
+        if (G > 1) {
+#pragma unroll
+            for (int g = 0; g < NGRP; ++g) cptr[g] = p.codes + (gbase[g] >= 0 ? gbase[g] : 0) + static_cast<long long>(ksub) * p.P;
+        }
         const long long rr0 = r0 < p.rows ? r0 : 0;
         const long long b0 = rr0 / p.P, q0 = rr0 - b0 * p.P;
         // slab mode: staged images img_lo .. img_lo + nimg - 1 as [image][64 co][P]; my copies are
@@ -129,24 +134,32 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
             split = Pi - static_cast<int>(q0) < 8 ? Pi - static_cast<int>(q0) : 8;
         }
         bool ok = true;
+        // ring position, weight pointer and first k-row of the next stage to fill: advanced per
+        // stage, so a stage costs no division and no 64-bit multiply
+        int is = 0, co_next = ksub;
+        unsigned iparity = 1;
+        const __nv_bfloat16 *wptr = p.W + static_cast<long long>(ksub) * p.Cin + ci0 + c16 * 8;
+        const bool wcol = ci0 + c16 * 8 < p.Cin;                 // Cin % 8 == 0
+        const long long wstep = kKS * static_cast<long long>(p.Cin), cstep = kKS * p.P;
         auto issue = [&](int j) {
-            const int s = j % S;
-            ok = ok && mbar_wait(&pipe.empty[s], ((j / S) & 1) ^ 1, p.err_flag);
+            const int s = is;
+            ok = ok && mbar_wait(&pipe.empty[s], iparity, p.err_flag);
+            if (++is == S) { is = 0; iparity ^= 1u; }
             unsigned char *st = smem + s * STAGE;
             unsigned char *b_s = st + A_BYTES, *raw = b_s + B_BYTES;
             // weights: k-row = co; my chunk column is c16 (8 channels), my k-rows ksub + kKS i.
             // Pointers step by constants: kKS k-rows per i, 64 per stage.
             {
-                const int ci = ci0 + c16 * 8;
-                const __nv_bfloat16 *ws = p.W + static_cast<long long>(j * kKT + ksub) * p.Cin + ci;
+                const __nv_bfloat16 *ws = wptr;
                 unsigned char *wd = b_s + (c16 >> 3) * PANEL + swz(ksub, c16 & 7);
 #pragma unroll
                 for (int i = 0; i < kKT / kKS; ++i) {
-                    const bool v = (j * kKT + ksub + kKS * i < p.Cout) && ci < p.Cin;     // Cin % 8 == 0
+                    const bool v = wcol && (co_next + kKS * i < p.Cout);
                     cp_async16(wd, v ? ws : p.W, v);
-                    ws += kKS * static_cast<long long>(p.Cin);
+                    ws += wstep;
                     wd += kKS * 128;
                 }
+                wptr += static_cast<long long>(kKT) * p.Cin;
             }
             // code bytes: k-row = co, my chunk of 8 rows
             if (G == 0) {
@@ -157,16 +170,17 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
             } else if (G > 1) {
 #pragma unroll
                 for (int g = 0; g < NGRP; ++g) {
-                    const int8_t *cs = p.codes + gbase[g] + static_cast<long long>(j * kKT + ksub) * p.P;
+                    const int8_t *cs = cptr[g];
                     unsigned char *cd = raw + ksub * 128 + c16 * 8 + g * 4;
 #pragma unroll
                     for (int i = 0; i < kKT / kKS; ++i) {
-                        const bool v = gbase[g] >= 0 && (j * kKT + ksub + kKS * i < p.Cout);
+                        const bool v = gbase[g] >= 0 && (co_next + kKS * i < p.Cout);
                         if (G == 8) cp_async_small<8>(cd, v ? cs : p.codes, v);
                         else cp_async_small<4>(cd, v ? cs : p.codes, v);
-                        cs += kKS * p.P;
+                        cs += cstep;
                         cd += kKS * 128;
                     }
+                    cptr[g] += static_cast<long long>(kKT) * p.P;
                 }
             } else {
                 for (int i = 0; i < kKT / kKS; ++i) {
@@ -182,9 +196,11 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
                     *reinterpret_cast<uint2 *>(raw + k * 128 + c16 * 8) = make_uint2(w[0], w[1]);
                 }
             }
+            co_next += kKT;
         };
         // every thread closes one cp.async group per stage (empty once the copies run out), so
         // "at most LA groups pending" means the copies of stage `it` have landed
+        int cslot = 0;              // ring slot of the stage being expanded
         for (int j = 0; j < LA; ++j) {
             if (j < niter) issue(j);
             cp_async_commit();
@@ -192,7 +208,8 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
         for (int it = 0; it < niter; ++it) {
             if (it + LA < niter) issue(it + LA);
             cp_async_commit();
-            const int s = it % S;
+            const int s = cslot;
+            if (++cslot == S) cslot = 0;
             cp_async_wait_pending(LA);
             if (G == 0) asm volatile("bar.sync 1, %0;" ::"n"(kP) : "memory");   // slabs are read across threads
             unsigned char *a_s = smem + s * STAGE, *raw = a_s + A_BYTES + B_BYTES;
@@ -322,9 +339,10 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
     } else if (lane == 0) {
         constexpr unsigned idesc = make_idesc(128, 128, true, true);
         bool ok = true;
+        int s = 0;
+        unsigned parity = 0;
         for (int it = 0; it < niter && ok; ++it) {
-            const int s = it % S;
-            ok = mbar_wait(&pipe.full[s], (it / S) & 1, p.err_flag);
+            ok = mbar_wait(&pipe.full[s], parity, p.err_flag);
             fence_async_proxy();
             tc_fence_after();
             const unsigned q_addr = smem_u32(smem + s * STAGE), w_addr = q_addr + A_BYTES;
@@ -334,6 +352,7 @@ __global__ void __launch_bounds__(kThreadsDx) tc_dx_async_kernel(const DxP p) {
             for (int k = 0; k < kKT / 16; ++k)     // 16 k-rows = two 1024-byte groups further per MMA
                 mma_bf16(tmem_d, ad + 128 * k, bd + 128 * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
             mma_commit(&pipe.empty[s]);
+            if (++s == S) { s = 0; parity ^= 1u; }
         }
         mma_commit(&pipe.acc);
     }
