@@ -191,6 +191,7 @@ def main():
     ap.add_argument("--config", type=int, default=5)
     ap.add_argument("--batch", type=int, default=0, help="override the config's batch size")
     ap.add_argument("--only", default="", help="config 5: comma-separated shape indices to run (profiling aid)")
+    ap.add_argument("--single", action="store_true", help="one instance of every shape (profiling aid)")
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--no-dense", action="store_true", help="skip the cuDNN/cuBLAS dense comparison")
     ap.add_argument("--no-e2e", action="store_true")
@@ -219,6 +220,9 @@ def main():
         keep = [int(t) for t in args.only.split(",")]
         specs = [specs[i] for i in keep]
         name += f" [only shapes {keep}]"
+    if args.single:
+        specs = [(make, 1) for make, _ in specs]
+        name += " [one instance per shape]"
     tdt = lambda L: torch.bfloat16 if L.dtype == "bf16" else torch.float32
     layers = []          # one entry per layer instance: (Layer, delta, X, W, dW, dX)
     hosts = []           # one entry per distinct shape: pinned host tensors

@@ -45,25 +45,15 @@ struct DeviceGuard {
 int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
                           unsigned long long seed, float scale, const float *delta_in,
                           dbp_sparse *q_out, const float **delta_p, const int8_t **codes) {
-    size_t bb, ob, vb;
-    int rc = dbp_sparse_bytes(numel, &bb, &ob, &vb);
-    if (rc) return rc;
+    int rc = DBP_OK;
     dbp_sparse sp;
+    sp.bitmap = nullptr; sp.offsets = nullptr; sp.values = nullptr; sp.delta = nullptr; sp.nnz = nullptr;
+    sp.numel = numel;
     if (q_out) {
         if (!q_out->bitmap || !q_out->offsets || !q_out->values || !q_out->delta || !q_out->nnz) return DBP_EINVAL;
         if (!aligned16(q_out->bitmap) || !aligned16(q_out->offsets) || !aligned16(q_out->values)) return DBP_EINVAL;
         q_out->numel = numel;
         sp = *q_out;
-    } else {
-        if ((rc = ws_reserve(ctx, ctx->sp_bitmap, bb)) || (rc = ws_reserve(ctx, ctx->sp_offsets, ob)) ||
-            (rc = ws_reserve(ctx, ctx->sp_values, vb)))
-            return rc;
-        sp.bitmap = static_cast<uint32_t *>(ctx->sp_bitmap.ptr);
-        sp.offsets = static_cast<uint16_t *>(ctx->sp_offsets.ptr);
-        sp.values = static_cast<int8_t *>(ctx->sp_values.ptr);
-        sp.delta = nullptr;
-        sp.nnz = nullptr;
-        sp.numel = numel;
     }
     if ((rc = ws_reserve(ctx, ctx->dense_codes, static_cast<size_t>(numel) + 16))) return rc;
     int8_t *dense = static_cast<int8_t *>(ctx->dense_codes.ptr);
@@ -75,8 +65,10 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
     if (rc) return rc;
     {
         KernelTimer t(ctx, DBP_K_QUANTIZE);
-        rc = launch_quantize(ctx, delta, dtype, numel, seed, &ctx->state->delta, sp.bitmap, sp.offsets,
-                             sp.values, dense, reinterpret_cast<unsigned long long *>(sp.nnz));
+        // the sparse structure is written only for a caller who asked for it
+        rc = q_out ? launch_quantize(ctx, delta, dtype, numel, seed, &ctx->state->delta, sp.bitmap, sp.offsets,
+                                     sp.values, dense, reinterpret_cast<unsigned long long *>(sp.nnz))
+                   : launch_quantize_dense(ctx, delta, dtype, numel, seed, &ctx->state->delta, dense);
     }
     if (rc) return rc;
     *delta_p = &ctx->state->delta;

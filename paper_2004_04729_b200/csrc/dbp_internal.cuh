@@ -73,6 +73,9 @@ int launch_quantize(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
                     unsigned long long seed, const float *delta_p, uint32_t *bitmap,
                     uint16_t *offsets, int8_t *values, int8_t *dense,
                     unsigned long long *nnz_out);
+// ---- nsd_dense.cu: the same codes, dense array only (no sparse structure)
+int launch_quantize_dense(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
+                          unsigned long long seed, const float *delta_p, int8_t *dense);
 int launch_decode(dbp_ctx *ctx, const uint32_t *bitmap, const uint16_t *offsets,
                   const int8_t *values, long long numel, int8_t *dense);
 

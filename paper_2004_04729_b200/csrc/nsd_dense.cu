@@ -1,0 +1,192 @@
+// NSD quantization for the product kernels (Section 3.1, Eq. (nsd)): the same codes as
+// quantize_kernel, written only as the dense array the dX / dW kernels read, without the
+// bitmap / offsets / packed-values structure. Used when the caller did not ask for the sparse
+// structure, so the pass costs one read of delta_z and one write of the codes.
+//
+// The common case (every |x / Delta + u| <= 127, no NaN) runs without clamping: the code's
+// two's-complement byte is the low byte of the round-down sum with 1.5 * 2^23. A vector that
+// holds a NaN or a value outside that range is redone element by element with the clipped,
+// counted decision.
+#include "dbp_internal.cuh"
+
+namespace dbp {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr unsigned kFull = 0xffffffffu;
+constexpr unsigned long long kGamma = 0x9E3779B97F4A7C15ull;
+
+__device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+// u = (2k+1) 2^-24, k = top 23 bits of h: the funnel shift builds 1 + k 2^-23 in one step
+__device__ __forceinline__ float dither(unsigned h) {
+    return __uint_as_float(__funnelshift_r(h, 0x7fu, 9)) - 0.99999994f;
+}
+// careful decision: clipped to [-127, 127], clipped codes counted, NaN gives 0
+__device__ __forceinline__ unsigned careful_byte(float x, float inv, float u, unsigned &sat) {
+    const float t = __fmaf_rn(x, inv, u);
+    const float tc = fminf(fmaxf(t, -127.f), 127.99999f);
+    const bool num = (t == t);
+    sat += (num && tc != t) ? 1u : 0u;
+    const unsigned q = __float_as_uint(__fadd_rd(tc, 12582912.0f)) & 0xffu;
+    return num ? q : 0u;
+}
+// number of non-zero bytes of a word
+__device__ __forceinline__ unsigned nonzero_bytes(unsigned w) {
+    return __popc((((w & 0x7f7f7f7fu) + 0x7f7f7f7fu) | w) & 0x80808080u);
+}
+
+// Codes of the V elements x[0..V) whose first element has the (even) linear index e0; packed
+// four to a word in element order. V is 4 or 8.
+template <int V>
+__device__ __forceinline__ void codes_of(const float (&x)[V], long long e0, unsigned long long seed,
+                                         float inv, unsigned (&pk)[V / 4], unsigned &sat) {
+    unsigned long long z = seed + (static_cast<unsigned long long>(e0 >> 1) + 1ull) * kGamma;
+    float u[V];
+#pragma unroll
+    for (int j = 0; j < V; j += 2) {
+        const unsigned long long r = mix64(z);
+        z += kGamma;
+        u[j] = dither(static_cast<unsigned>(r));
+        u[j + 1] = dither(static_cast<unsigned>(r >> 32));
+    }
+    unsigned b[V];
+    float amax = 0.f, sum = 0.f;
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+        const float t = __fmaf_rn(x[j], inv, u[j]);
+        amax = fmaxf(amax, fabsf(t));
+        sum += t;                                   // NaN iff some t is NaN (or +inf meets -inf)
+        b[j] = __float_as_uint(__fadd_rd(t, 12582912.0f));
+    }
+    if (!(amax <= 127.f) || sum != sum) {           // rare: clip, count, NaN
+#pragma unroll
+        for (int j = 0; j < V; ++j) b[j] = careful_byte(x[j], inv, u[j], sat);
+    }
+#pragma unroll
+    for (int w = 0; w < V / 4; ++w)
+        pk[w] = __byte_perm(__byte_perm(b[4 * w], b[4 * w + 1], 0x0040), __byte_perm(b[4 * w + 2], b[4 * w + 3], 0x0040), 0x5410);
+}
+
+template <typename T>
+struct Vec;
+template <>
+struct Vec<float> {
+    static constexpr int V = 4;
+    __device__ static void load(const float *p, float (&v)[4]) {
+        const float4 q = __ldg(reinterpret_cast<const float4 *>(p));
+        v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+    }
+    __device__ static float one(const float *p) { return __ldg(p); }
+    __device__ static void store(int8_t *d, const unsigned (&pk)[1]) { *reinterpret_cast<unsigned *>(d) = pk[0]; }
+};
+template <>
+struct Vec<__nv_bfloat16> {
+    static constexpr int V = 8;
+    __device__ static void load(const __nv_bfloat16 *p, float (&v)[8]) {
+        const uint4 q = __ldg(reinterpret_cast<const uint4 *>(p));
+        const unsigned w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[2 * i] = __uint_as_float(w[i] << 16);
+            v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    }
+    __device__ static float one(const __nv_bfloat16 *p) {
+        return __uint_as_float(static_cast<unsigned>(__ldg(reinterpret_cast<const unsigned short *>(p))) << 16);
+    }
+    __device__ static void store(int8_t *d, const unsigned (&pk)[2]) { *reinterpret_cast<uint2 *>(d) = make_uint2(pk[0], pk[1]); }
+};
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+quantize_dense_kernel(const T *__restrict__ x, long long n, unsigned long long seed,
+                      const float *__restrict__ delta_p, int8_t *__restrict__ dense,
+                      DeviceState *__restrict__ st) {
+    constexpr int V = Vec<T>::V;
+    const long long nvec = n / V;
+    const long long stride = static_cast<long long>(gridDim.x) * kThreads;
+    long long i = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x;
+    const float delta = *delta_p;
+    const bool live = (delta > 0.f) && (delta < __int_as_float(0x7f800000));
+    if (!live) {                                    // sigma = 0 or non-finite input: every code is 0
+        for (; i < nvec; i += stride) {
+            const unsigned zero[V / 4] = {};
+            Vec<T>::store(dense + i * V, zero);
+        }
+        if (blockIdx.x == 0 && threadIdx.x == 0)
+            for (long long e = nvec * V; e < n; ++e) dense[e] = 0;
+        return;
+    }
+    const float inv = __fdiv_rn(1.0f, delta);
+    unsigned nnz = 0, sat = 0;
+    // two vectors in flight per thread
+    for (; i + stride < nvec; i += 2 * stride) {
+        float a[V], b[V];
+        Vec<T>::load(x + i * V, a);
+        Vec<T>::load(x + (i + stride) * V, b);
+        unsigned pa[V / 4], pb[V / 4];
+        codes_of<V>(a, i * V, seed, inv, pa, sat);
+        codes_of<V>(b, (i + stride) * V, seed, inv, pb, sat);
+        Vec<T>::store(dense + i * V, pa);
+        Vec<T>::store(dense + (i + stride) * V, pb);
+#pragma unroll
+        for (int w = 0; w < V / 4; ++w) nnz += nonzero_bytes(pa[w]) + nonzero_bytes(pb[w]);
+    }
+    if (i < nvec) {
+        float a[V];
+        Vec<T>::load(x + i * V, a);
+        unsigned pa[V / 4];
+        codes_of<V>(a, i * V, seed, inv, pa, sat);
+        Vec<T>::store(dense + i * V, pa);
+#pragma unroll
+        for (int w = 0; w < V / 4; ++w) nnz += nonzero_bytes(pa[w]);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {      // the n % V last elements, one by one
+        for (long long e = nvec * V; e < n; ++e) {
+            const unsigned long long r = mix64(seed + (static_cast<unsigned long long>(e >> 1) + 1ull) * kGamma);
+            const float u = dither((e & 1) ? static_cast<unsigned>(r >> 32) : static_cast<unsigned>(r));
+            const unsigned q = careful_byte(Vec<T>::one(x + e), inv, u, sat);
+            dense[e] = static_cast<int8_t>(q);
+            nnz += q != 0u;
+        }
+    }
+    nnz = __reduce_add_sync(kFull, nnz);
+    sat = __reduce_add_sync(kFull, sat);
+    __shared__ unsigned s_nnz, s_sat;
+    if (threadIdx.x == 0) { s_nnz = 0; s_sat = 0; }
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) {
+        if (nnz) atomicAdd(&s_nnz, nnz);
+        if (sat) atomicAdd(&s_sat, sat);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (s_nnz) atomicAdd(&st->nnz, static_cast<unsigned long long>(s_nnz));
+        if (s_sat) atomicAdd(&st->saturated, static_cast<unsigned long long>(s_sat));
+    }
+}
+
+}  // namespace
+
+int launch_quantize_dense(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
+                          unsigned long long seed, const float *delta_p, int8_t *dense) {
+    const int v = dtype == DBP_F32 ? 4 : 8;
+    long long blocks = (numel / v + 2 * kThreads - 1) / (2 * kThreads);
+    if (blocks < 1) blocks = 1;
+    const long long cap = static_cast<long long>(ctx->sm_count) * 8;
+    if (blocks > cap) blocks = cap;
+    if (dtype == DBP_F32)
+        quantize_dense_kernel<float><<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(
+            static_cast<const float *>(delta), numel, seed, delta_p, dense, ctx->state);
+    else
+        quantize_dense_kernel<__nv_bfloat16><<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(
+            static_cast<const __nv_bfloat16 *>(delta), numel, seed, delta_p, dense, ctx->state);
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace dbp

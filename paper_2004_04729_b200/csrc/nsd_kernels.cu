@@ -62,7 +62,25 @@ statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ par
     const long long nvec = n / EPT;
     double d1 = 0.0, d2 = 0.0;
     const long long stride = static_cast<long long>(gridDim.x) * kThreads;
-    for (long long i = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x; i < nvec; i += stride) {
+    long long i = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x;
+    // four 128-bit loads in flight per thread
+    for (; i + 3 * stride < nvec; i += 4 * stride) {
+        float v[4][EPT];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) Elem<T>::load(x + (i + u * stride) * EPT, v[u]);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+            for (int j = 0; j < EPT; ++j) {
+                s1 += v[u][j];
+                s2 = fmaf(v[u][j], v[u][j], s2);
+            }
+            d1 += static_cast<double>(s1);
+            d2 += static_cast<double>(s2);
+        }
+    }
+    for (; i < nvec; i += stride) {
         float v[EPT];
         Elem<T>::load(x + i * EPT, v);
         float s1 = 0.f, s2 = 0.f;

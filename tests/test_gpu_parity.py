@@ -250,3 +250,34 @@ def test_host_entry_points_match_device_ones(ctx):
     assert nnz == rn
     _compare("dW", dW, ref["dW"], ref["S_dW"])
     _compare("dX", dX, ref["dX"], ref["S_dX"])
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B,N", [(1, 1), (3, 5), (7, 33), (64, 300), (129, 257)])
+def test_codes_of_the_internal_quantization(ctx, dtype, B, N):
+    """Without q_out the library quantizes into its own dense code array only. An identity
+    weight matrix makes dX = Delta * codes, so the codes (clipped ones and a NaN included) can
+    be compared with the oracle's bit for bit, and nnz / the clip count through the status."""
+    import paper_2004_04729_b200 as dbp
+    x = (wl.laplace(11, B, B * N, 3.0) * wl.bernoulli(11, N, B * N, 0.5)).astype(np.float32).reshape(B, N)
+    if B * N >= 15:
+        x.flat[3], x.flat[8], x.flat[14] = 500.0, -700.0, 127.5
+    if dtype == "bf16":
+        x = _t(x, "bf16").float().cpu().numpy()
+    eye = np.eye(N, dtype=np.float32)
+    step = torch.tensor([1.0], dtype=torch.float32, device="cuda")
+    ctx.last_device_status()
+    out = dbp.dithered_linear_backward(ctx, _t(x, dtype), _t(np.zeros((B, N), np.float32), dtype), _t(eye, dtype),
+                                       5, 0.0, delta_in=step, need_dW=False, flags=dbp.DBP_DX_F32 | dbp.DBP_FORCE_SPARSE)
+    ref, nnz, nsat = oracle.nsd_codes(x, 5, np.float32(1.0))
+    assert np.array_equal(out["dX"].cpu().numpy(), ref.astype(np.float32))
+    assert ctx.last_device_status() == ((-6, nsat) if nsat else (0, 0))
+    if B * N >= 15:
+        assert nsat == 2
+        x.flat[5] = np.nan                               # NaN with a given step size: code 0, others unchanged
+        out = dbp.dithered_linear_backward(ctx, _t(x, dtype), _t(np.zeros((B, N), np.float32), dtype), _t(eye, dtype),
+                                           5, 0.0, delta_in=step, need_dW=False, flags=dbp.DBP_DX_F32 | dbp.DBP_FORCE_SPARSE)
+        ref2 = ref.copy()
+        ref2.flat[5] = 0
+        assert np.array_equal(out["dX"].cpu().numpy(), ref2.astype(np.float32))
+        ctx.last_device_status()
