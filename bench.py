@@ -300,6 +300,13 @@ def main():
         ms = t.item()
     value = dense_flops * world / (ms * 1e-3) / 1e9
 
+    # host time to enqueue one step (the launch queue is empty and deep enough for one step)
+    barrier()
+    t0 = time.perf_counter()
+    step()
+    host_ms = (time.perf_counter() - t0) * 1e3
+    barrier()
+
     # non-zero work actually done (for the arithmetic roofline of the sparse products)
     nnz_flops = 0.0
     for (L, d, X, W, dW, dX) in layers:
@@ -430,7 +437,7 @@ def main():
         "data": "synthetic",
         "config": {"workload": name, "layers_per_step": len(layers), "l2": "inputs larger than L2 (distinct buffers per layer instance)"
                    if alg_bytes > 2.5e8 else "working set smaller than L2 (warm)", "nsd_density": density},
-        "clocks": clocks, "gpu_launches": launches, "e2e": e2e,
+        "clocks": clocks, "gpu_launches": launches, "host_enqueue_ms_per_step": host_ms, "e2e": e2e,
         "roofline": roof,
         "hbm_path": {"algorithmic_gb_per_step": alg_bytes / 1e9, "achieved_gbs": path_gbs,
                      "frac_of_measured_hbm": path_gbs / hbm_peak, "peak": hbm_peak, "peak_source": peak_src},

@@ -44,7 +44,9 @@ struct DeviceGuard {
 // context's dense code buffer, which the product kernels read.
 int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
                           unsigned long long seed, float scale, const float *delta_in,
-                          dbp_sparse *q_out, const float **delta_p, const int8_t **codes) {
+                          dbp_sparse *q_out, const float **delta_p, const int8_t **codes,
+                          bool want8 = true, long long planes_hw = 0, long long planes_pitch = 0,
+                          const void **codes16 = nullptr) {
     int rc = DBP_OK;
     dbp_sparse sp;
     sp.bitmap = nullptr; sp.offsets = nullptr; sp.values = nullptr; sp.delta = nullptr; sp.nnz = nullptr;
@@ -65,10 +67,25 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
     if (rc) return rc;
     {
         KernelTimer t(ctx, DBP_K_QUANTIZE);
-        // the sparse structure is written only for a caller who asked for it
-        rc = q_out ? launch_quantize(ctx, delta, dtype, numel, seed, &ctx->state->delta, sp.bitmap, sp.offsets,
-                                     sp.values, dense, reinterpret_cast<unsigned long long *>(sp.nnz))
-                   : launch_quantize_dense(ctx, delta, dtype, numel, seed, &ctx->state->delta, dense);
+        // the sparse structure is written only for a caller who asked for it; the bf16 planes
+        // of the TMA-fed kernels come from the dense kernel (a second pass when both are wanted)
+        void *p16 = nullptr;
+        if (codes16) {
+            const long long planes = numel / planes_hw;
+            if ((rc = ws_reserve(ctx, ctx->codes16, static_cast<size_t>(planes) * planes_pitch * 2 + 1024))) return rc;
+            p16 = ctx->codes16.ptr;
+            *codes16 = p16;
+        }
+        if (q_out) {
+            rc = launch_quantize(ctx, delta, dtype, numel, seed, &ctx->state->delta, sp.bitmap, sp.offsets,
+                                 sp.values, dense, reinterpret_cast<unsigned long long *>(sp.nnz));
+            if (!rc && p16)
+                rc = launch_quantize_dense(ctx, delta, dtype, numel, seed, &ctx->state->delta, nullptr, p16,
+                                           planes_hw, planes_pitch, false);
+        } else {
+            rc = launch_quantize_dense(ctx, delta, dtype, numel, seed, &ctx->state->delta, want8 ? dense : nullptr,
+                                       p16, planes_hw, planes_pitch, true);
+        }
     }
     if (rc) return rc;
     *delta_p = &ctx->state->delta;
@@ -110,7 +127,14 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     cudaGetLastError();   // cudaErrorNotReady from the query is not an error
     const bool dense = can_dense && !(flags & DBP_FORCE_SPARSE) &&
                        ((flags & DBP_FORCE_DENSE) || ctx->density_estimate > ctx->crossover);
-    int rc = quantize_for_products(ctx, delta, io, numel, seed, scale, delta_in, q_out, &delta_p, &codes);
+    // which dense kernels run: the TMA-fed ones read bf16 code planes, the others int8 codes
+    const bool dx_tma = dense && dX && tma_dx_supported(s, io);
+    const bool dw_tma = dense && dW && tma_dw_supported(s, io);
+    const bool any_tma = dx_tma || dw_tma;
+    const bool need8 = !dense || db || (dX && !dx_tma) || (dW && !dw_tma);
+    const void *codes16 = nullptr;
+    int rc = quantize_for_products(ctx, delta, io, numel, seed, scale, delta_in, q_out, &delta_p, &codes, need8,
+                                   s.H * s.W, any_tma ? tma_code_pitch(s) : 0, any_tma ? &codes16 : nullptr);
     if (rc) return rc;
     if (!capturing && !ctx->nnz_pending && ctx->nnz_host && ctx->nnz_event) {
         ctx->nnz_host_numel = numel;
@@ -123,14 +147,16 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
         if (dX) {
             KernelTimer t(ctx, DBP_K_DX_DENSE);
             const bool dx_bf16 = (io == DBP_BF16) && !(flags & DBP_DX_F32);
-            rc = s.k == 3 ? launch_tc3_dx(ctx, codes, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout)
-                          : launch_tc_dx(ctx, codes, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout);
+            rc = dx_tma ? launch_tma_dx(ctx, codes16, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout)
+                 : s.k == 3 ? launch_tc3_dx(ctx, codes, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout)
+                            : launch_tc_dx(ctx, codes, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout);
             if (rc) return rc;
         }
         if (dW) {
             KernelTimer t(ctx, DBP_K_DW_DENSE);
-            rc = s.k == 3 ? launch_tc3_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout)
-                          : launch_tc_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout);
+            rc = dw_tma ? launch_tma_dw(ctx, codes16, X, delta_p, s, dW, &ctx->state->tc_timeout)
+                 : s.k == 3 ? launch_tc3_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout)
+                            : launch_tc_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout);
             if (rc) return rc;
         }
         if (db) {
@@ -224,7 +250,7 @@ int dbp_destroy(dbp_ctx *ctx) {
     if (!ctx) return DBP_EINVAL;
     DeviceGuard guard(ctx->device);
     cudaStreamSynchronize(ctx->stream);
-    Workspace *all[] = {&ctx->dense_codes, &ctx->w_taps, &ctx->sp_bitmap, &ctx->sp_offsets, &ctx->sp_values,
+    Workspace *all[] = {&ctx->dense_codes, &ctx->codes16, &ctx->x_padded, &ctx->w_taps, &ctx->sp_bitmap, &ctx->sp_offsets, &ctx->sp_values,
                         &ctx->tc_partials};
     for (Workspace *w : all) if (w->ptr) cudaFree(w->ptr);
     for (Workspace &w : ctx->io) if (w.ptr) cudaFree(w.ptr);

@@ -44,6 +44,8 @@ struct dbp_ctx {
     double *partials = nullptr;         // device, statistics partial sums
     int partial_blocks = 0;
     dbp::Workspace dense_codes;         // int8 per element of delta
+    dbp::Workspace x_padded;            // activations copied to 16-byte aligned planes
+    dbp::Workspace codes16;             // bf16 code planes for the TMA-fed kernels
     dbp::Workspace w_taps;              // fp32 weights as [Cout][k*k][Cin]
     dbp::Workspace sp_bitmap, sp_offsets, sp_values;  // internal dbp_sparse
     dbp::Workspace tc_partials;         // split-K partial blocks of the dense dW kernel
@@ -74,8 +76,11 @@ int launch_quantize(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
                     uint16_t *offsets, int8_t *values, int8_t *dense,
                     unsigned long long *nnz_out);
 // ---- nsd_dense.cu: the same codes, dense array only (no sparse structure)
+// dense: int8 codes in delta's order (or null); planes_bf16: bf16 codes as [numel / hw][pitch]
+// (or null), pitch a multiple of 8
 int launch_quantize_dense(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
-                          unsigned long long seed, const float *delta_p, int8_t *dense);
+                          unsigned long long seed, const float *delta_p, int8_t *dense,
+                          void *planes_bf16, long long hw, long long pitch, bool count);
 int launch_decode(dbp_ctx *ctx, const uint32_t *bitmap, const uint16_t *offsets,
                   const int8_t *values, long long numel, int8_t *dense);
 
@@ -101,6 +106,19 @@ int launch_tc_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *
                  const ConvShape &s, float *dW, int *err_flag);
 int launch_tc_dx(dbp_ctx *ctx, const int8_t *codes, const void *W, const float *delta_p,
                  const ConvShape &s, void *dX, bool dx_bf16, int *err_flag);
+// ---- tma_dx.cu: 1x1 dX with TMA-fed operands; codes as bf16 planes [B*Cout][tma_code_pitch]
+bool tma_dx_supported(const ConvShape &s, int io);
+long long tma_code_pitch(const ConvShape &s);
+int launch_tma_dx(dbp_ctx *ctx, const void *codes_bf16, const void *W, const float *delta_p,
+                  const ConvShape &s, void *dX, bool dx_bf16, int *err_flag);
+// ---- tma_dw.cu: 1x1 dW with TMA-fed operands (same code planes)
+bool tma_dw_supported(const ConvShape &s, int io);
+int launch_tma_dw(dbp_ctx *ctx, const void *codes_bf16, const void *X, const float *delta_p,
+                  const ConvShape &s, float *dW, int *err_flag);
+// planes of H x W bf16 values -> rows of Wp values (multiple of 8), extra columns zero
+int launch_pad_planes(dbp_ctx *ctx, const void *in, void *out, long long planes, int H, int W, int Wp);
+// dW = Delta * sum of nsplit partial blocks of nw floats (nw % 4 == 0), fixed order
+int launch_dw_sum(dbp_ctx *ctx, const float *partials, int nsplit, long long nw, const float *delta_p, float *dW);
 // ---- tc_conv3x3.cu
 bool tc3_supported(const ConvShape &s, int io);
 // row-shift variant of the 3x3 dX product; DBP_EUNSUPPORTED when the shape does not fit it

@@ -72,6 +72,61 @@ __device__ __forceinline__ void codes_of(const float (&x)[V], long long e0, unsi
         pk[w] = __byte_perm(__byte_perm(b[4 * w], b[4 * w + 1], 0x0040), __byte_perm(b[4 * w + 2], b[4 * w + 3], 0x0040), 0x5410);
 }
 
+
+// four packed code bytes -> four bf16 (exact): byte ^ 0x80 is code + 128; 0x4B0000xx read as a
+// float is 2^23 + xx, so subtracting 2^23 + 128 leaves the code, whose top half is its bf16
+__device__ __forceinline__ void bytes4_to_bf16(unsigned w, unsigned &lo, unsigned &hi) {
+    const unsigned x = w ^ 0x80808080u;
+    const float f0 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7650)) - 8388736.0f;
+    const float f1 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7651)) - 8388736.0f;
+    const float f2 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7652)) - 8388736.0f;
+    const float f3 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7653)) - 8388736.0f;
+    lo = __byte_perm(__float_as_uint(f0), __float_as_uint(f1), 0x7632);
+    hi = __byte_perm(__float_as_uint(f2), __float_as_uint(f3), 0x7632);
+}
+
+// Where the codes go. dense8: one byte per element, same order as delta_z (may be null).
+// planes16: bf16 codes as [plane][pitch] with plane = e / hw (may be null); the pitch is a
+// multiple of 8 so that every plane starts on a 16-byte boundary.
+struct CodeSinks {
+    int8_t *dense8;
+    unsigned short *planes16;
+    long long hw, pitch;
+    int count;                    // add nnz / clipped counts to the context's counters
+};
+
+template <int V>
+__device__ __forceinline__ void store_codes(const CodeSinks &o, long long e0, const unsigned (&pk)[V / 4]) {
+    if (o.dense8 != nullptr) {
+        if (V == 4) *reinterpret_cast<unsigned *>(o.dense8 + e0) = pk[0];
+        else *reinterpret_cast<uint2 *>(o.dense8 + e0) = make_uint2(pk[0], pk[V / 4 - 1]);
+    }
+    if (o.planes16 != nullptr) {
+        unsigned h[V / 2];
+#pragma unroll
+        for (int w = 0; w < V / 4; ++w) bytes4_to_bf16(pk[w], h[2 * w], h[2 * w + 1]);
+        if (o.pitch == o.hw) {                      // planes are back to back: same order as delta_z
+            if (V == 4) *reinterpret_cast<uint2 *>(o.planes16 + e0) = make_uint2(h[0], h[1]);
+            else *reinterpret_cast<uint4 *>(o.planes16 + e0) = make_uint4(h[0], h[1], h[V / 2 - 2], h[V / 2 - 1]);
+        } else {
+            long long plane = e0 / o.hw, pp = e0 - plane * o.hw;
+#pragma unroll
+            for (int j = 0; j < V; ++j) {
+                o.planes16[plane * o.pitch + pp] = static_cast<unsigned short>(h[j >> 1] >> (16 * (j & 1)));
+                if (++pp == o.hw) { pp = 0; ++plane; }
+            }
+        }
+    }
+}
+__device__ __forceinline__ void store_code(const CodeSinks &o, long long e, unsigned byte) {
+    if (o.dense8 != nullptr) o.dense8[e] = static_cast<int8_t>(byte);
+    if (o.planes16 != nullptr) {
+        const long long plane = e / o.hw;
+        const float f = static_cast<float>(static_cast<int>(static_cast<signed char>(byte)));
+        o.planes16[plane * o.pitch + (e - plane * o.hw)] = static_cast<unsigned short>(__float_as_uint(f) >> 16);
+    }
+}
+
 template <typename T>
 struct Vec;
 template <>
@@ -82,7 +137,6 @@ struct Vec<float> {
         v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
     }
     __device__ static float one(const float *p) { return __ldg(p); }
-    __device__ static void store(int8_t *d, const unsigned (&pk)[1]) { *reinterpret_cast<unsigned *>(d) = pk[0]; }
 };
 template <>
 struct Vec<__nv_bfloat16> {
@@ -99,13 +153,12 @@ struct Vec<__nv_bfloat16> {
     __device__ static float one(const __nv_bfloat16 *p) {
         return __uint_as_float(static_cast<unsigned>(__ldg(reinterpret_cast<const unsigned short *>(p))) << 16);
     }
-    __device__ static void store(int8_t *d, const unsigned (&pk)[2]) { *reinterpret_cast<uint2 *>(d) = make_uint2(pk[0], pk[1]); }
 };
 
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
 quantize_dense_kernel(const T *__restrict__ x, long long n, unsigned long long seed,
-                      const float *__restrict__ delta_p, int8_t *__restrict__ dense,
+                      const float *__restrict__ delta_p, const CodeSinks out,
                       DeviceState *__restrict__ st) {
     constexpr int V = Vec<T>::V;
     const long long nvec = n / V;
@@ -116,10 +169,10 @@ quantize_dense_kernel(const T *__restrict__ x, long long n, unsigned long long s
     if (!live) {                                    // sigma = 0 or non-finite input: every code is 0
         for (; i < nvec; i += stride) {
             const unsigned zero[V / 4] = {};
-            Vec<T>::store(dense + i * V, zero);
+            store_codes<V>(out, i * V, zero);
         }
         if (blockIdx.x == 0 && threadIdx.x == 0)
-            for (long long e = nvec * V; e < n; ++e) dense[e] = 0;
+            for (long long e = nvec * V; e < n; ++e) store_code(out, e, 0u);
         return;
     }
     const float inv = __fdiv_rn(1.0f, delta);
@@ -132,8 +185,8 @@ quantize_dense_kernel(const T *__restrict__ x, long long n, unsigned long long s
         unsigned pa[V / 4], pb[V / 4];
         codes_of<V>(a, i * V, seed, inv, pa, sat);
         codes_of<V>(b, (i + stride) * V, seed, inv, pb, sat);
-        Vec<T>::store(dense + i * V, pa);
-        Vec<T>::store(dense + (i + stride) * V, pb);
+        store_codes<V>(out, i * V, pa);
+        store_codes<V>(out, (i + stride) * V, pb);
 #pragma unroll
         for (int w = 0; w < V / 4; ++w) nnz += nonzero_bytes(pa[w]) + nonzero_bytes(pb[w]);
     }
@@ -142,7 +195,7 @@ quantize_dense_kernel(const T *__restrict__ x, long long n, unsigned long long s
         Vec<T>::load(x + i * V, a);
         unsigned pa[V / 4];
         codes_of<V>(a, i * V, seed, inv, pa, sat);
-        Vec<T>::store(dense + i * V, pa);
+        store_codes<V>(out, i * V, pa);
 #pragma unroll
         for (int w = 0; w < V / 4; ++w) nnz += nonzero_bytes(pa[w]);
     }
@@ -151,7 +204,7 @@ quantize_dense_kernel(const T *__restrict__ x, long long n, unsigned long long s
             const unsigned long long r = mix64(seed + (static_cast<unsigned long long>(e >> 1) + 1ull) * kGamma);
             const float u = dither((e & 1) ? static_cast<unsigned>(r >> 32) : static_cast<unsigned>(r));
             const unsigned q = careful_byte(Vec<T>::one(x + e), inv, u, sat);
-            dense[e] = static_cast<int8_t>(q);
+            store_code(out, e, q);
             nnz += q != 0u;
         }
     }
@@ -165,7 +218,7 @@ quantize_dense_kernel(const T *__restrict__ x, long long n, unsigned long long s
         if (sat) atomicAdd(&s_sat, sat);
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (threadIdx.x == 0 && out.count) {
         if (s_nnz) atomicAdd(&st->nnz, static_cast<unsigned long long>(s_nnz));
         if (s_sat) atomicAdd(&st->saturated, static_cast<unsigned long long>(s_sat));
     }
@@ -174,18 +227,20 @@ quantize_dense_kernel(const T *__restrict__ x, long long n, unsigned long long s
 }  // namespace
 
 int launch_quantize_dense(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
-                          unsigned long long seed, const float *delta_p, int8_t *dense) {
+                          unsigned long long seed, const float *delta_p, int8_t *dense,
+                          void *planes_bf16, long long hw, long long pitch, bool count) {
     const int v = dtype == DBP_F32 ? 4 : 8;
     long long blocks = (numel / v + 2 * kThreads - 1) / (2 * kThreads);
     if (blocks < 1) blocks = 1;
     const long long cap = static_cast<long long>(ctx->sm_count) * 8;
     if (blocks > cap) blocks = cap;
+    CodeSinks out{dense, static_cast<unsigned short *>(planes_bf16), hw > 0 ? hw : 1, pitch > 0 ? pitch : 1, count ? 1 : 0};
     if (dtype == DBP_F32)
         quantize_dense_kernel<float><<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(
-            static_cast<const float *>(delta), numel, seed, delta_p, dense, ctx->state);
+            static_cast<const float *>(delta), numel, seed, delta_p, out, ctx->state);
     else
         quantize_dense_kernel<__nv_bfloat16><<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(
-            static_cast<const __nv_bfloat16 *>(delta), numel, seed, delta_p, dense, ctx->state);
+            static_cast<const __nv_bfloat16 *>(delta), numel, seed, delta_p, out, ctx->state);
     return cuda_ok(cudaGetLastError());
 }
 

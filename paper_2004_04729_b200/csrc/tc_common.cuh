@@ -170,3 +170,39 @@ __device__ __forceinline__ unsigned short code_to_bf16(int c) {
 
 }  // namespace tc
 }  // namespace dbp
+
+// ---------------------------------------------------------------- TMA (bulk tensor copies)
+#include <cuda.h>
+
+namespace dbp {
+namespace tc {
+
+// Arms a barrier with the byte count of the bulk copies that will complete on it (one arrival).
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Tiled loads of this GPU's own memory into this CTA's shared memory; completion is counted in
+// bytes on `bar`. The innermost coordinate times the element size must be a multiple of 16.
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c0, int c1, unsigned long long *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, int c0, int c1, int c2, unsigned long long *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap *map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+// Host: a bf16 tensor map with 128-byte swizzle. dims/box are in elements (innermost first),
+// strides in bytes for dimensions 1.. (multiples of 16); the box's innermost extent is 64
+// elements (128 bytes). Out-of-range elements read as zero. Returns false when the driver entry
+// point is missing or rejects the description.
+bool encode_map_bf16(CUtensorMap *map, const void *base, int rank, const unsigned long long *dims,
+                     const unsigned long long *strides_bytes, const unsigned *box);
+
+}  // namespace tc
+}  // namespace dbp

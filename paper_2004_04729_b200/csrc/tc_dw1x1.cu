@@ -394,4 +394,11 @@ int launch_tc_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *
     return cuda_ok(cudaGetLastError());
 }
 
+int launch_dw_sum(dbp_ctx *ctx, const float *partials, int nsplit, long long nw, const float *delta_p, float *dW) {
+    const long long n4 = nw / 4;
+    tc_dw_sum_kernel<<<static_cast<unsigned>((n4 + 31) / 32), 256, 0, ctx->stream>>>(
+        reinterpret_cast<const float4 *>(partials), nsplit, n4, delta_p, reinterpret_cast<float4 *>(dW));
+    return cuda_ok(cudaGetLastError());
+}
+
 }  // namespace dbp

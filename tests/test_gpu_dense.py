@@ -59,6 +59,9 @@ def _run(ctx, L, flags):
     (2, 136, 128, 8, 7),      # slab staging, 56 positions, ragged channel tile
     (4, 64, 192, 9, 7),       # slab staging, 63 positions
     (7, 2048, 512, 7, 7),     # ResNet stage-4 reduce at a small batch, rows end inside a tile
+    (4, 72, 320, 8, 8),       # two accumulators with a ragged second one, input channels fill no 16-group
+    (3, 264, 136, 12, 12),    # two input-channel tiles, the second nearly empty; 144 positions = 2.25 chunks
+    (2, 512, 256, 16, 8),     # two full accumulators, two full input-channel tiles
 ])
 def test_dense_path_conv1x1(ctx, B, Ci, Co, H, W):
     import paper_2004_04729_b200 as dbp
@@ -99,6 +102,8 @@ def test_dense_path_linear(ctx, B, N, K):
 
 @pytest.mark.parametrize("B,Ci,Co,H,W,k", [
     (2, 64, 64, 16, 16, 3), (2, 128, 128, 14, 14, 3), (3, 64, 128, 7, 7, 3), (2, 64, 128, 28, 28, 1),
+    (1, 256, 64, 56, 56, 1), (3, 512, 128, 14, 14, 1), (5, 128, 512, 7, 7, 1), (2, 72, 40, 5, 9, 1),
+    (2, 64, 64, 9, 9, 1), (2, 136, 128, 8, 8, 1), (3, 40, 64, 10, 10, 1),
 ])
 def test_dense_bf16_dx_is_the_rounded_f32_dx(ctx, B, Ci, Co, H, W, k):
     """The bf16 store path of dX rounds the same accumulators the fp32 store path writes."""
