@@ -108,6 +108,16 @@ __device__ __forceinline__ void store_codes(const CodeSinks &o, long long e0, co
         if (o.pitch == o.hw) {                      // planes are back to back: same order as delta_z
             if (V == 4) *reinterpret_cast<uint2 *>(o.planes16 + e0) = make_uint2(h[0], h[1]);
             else *reinterpret_cast<uint4 *>(o.planes16 + e0) = make_uint4(h[0], h[1], h[V / 2 - 2], h[V / 2 - 1]);
+        } else if ((o.hw & 3) == 0) {
+            // e0 and the plane size are multiples of 4: each group of four codes lies in one plane
+            // and starts on an 8-byte boundary there
+            long long plane = e0 / o.hw, pp = e0 - plane * o.hw;
+#pragma unroll
+            for (int g = 0; g < V / 4; ++g) {
+                *reinterpret_cast<uint2 *>(o.planes16 + plane * o.pitch + pp) = make_uint2(h[2 * g], h[2 * g + 1]);
+                pp += 4;
+                if (pp == o.hw) { pp = 0; ++plane; }
+            }
         } else {
             long long plane = e0 / o.hw, pp = e0 - plane * o.hw;
 #pragma unroll

@@ -236,8 +236,16 @@ pad_planes_kernel(const unsigned short *__restrict__ in, unsigned short *__restr
         const int x0 = static_cast<int>(g - row * groups_per_row) * 8;
         const unsigned short *src = in + row * W + x0;
         unsigned short v[8];
+        if ((W & 3) == 0 && x0 + 8 <= W) {          // rows start on 8-byte boundaries: two 8-byte loads
+            const uint2 a = __ldg(reinterpret_cast<const uint2 *>(src)), b = __ldg(reinterpret_cast<const uint2 *>(src + 4));
+            v[0] = static_cast<unsigned short>(a.x); v[1] = static_cast<unsigned short>(a.x >> 16);
+            v[2] = static_cast<unsigned short>(a.y); v[3] = static_cast<unsigned short>(a.y >> 16);
+            v[4] = static_cast<unsigned short>(b.x); v[5] = static_cast<unsigned short>(b.x >> 16);
+            v[6] = static_cast<unsigned short>(b.y); v[7] = static_cast<unsigned short>(b.y >> 16);
+        } else {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = (x0 + j < W) ? __ldg(src + j) : static_cast<unsigned short>(0);
+            for (int j = 0; j < 8; ++j) v[j] = (x0 + j < W) ? __ldg(src + j) : static_cast<unsigned short>(0);
+        }
         uint4 o;
         o.x = v[0] | (static_cast<unsigned>(v[1]) << 16);
         o.y = v[2] | (static_cast<unsigned>(v[3]) << 16);

@@ -104,6 +104,7 @@ def test_dense_path_linear(ctx, B, N, K):
     (2, 64, 64, 16, 16, 3), (2, 128, 128, 14, 14, 3), (3, 64, 128, 7, 7, 3), (2, 64, 128, 28, 28, 1),
     (1, 256, 64, 56, 56, 1), (3, 512, 128, 14, 14, 1), (5, 128, 512, 7, 7, 1), (2, 72, 40, 5, 9, 1),
     (2, 64, 64, 9, 9, 1), (2, 136, 128, 8, 8, 1), (3, 40, 64, 10, 10, 1),
+    (2, 64, 64, 28, 28, 3), (1, 64, 64, 56, 56, 3), (2, 72, 40, 9, 11, 3), (2, 16, 24, 3, 62, 3), (3, 136, 96, 20, 16, 3),
 ])
 def test_dense_bf16_dx_is_the_rounded_f32_dx(ctx, B, Ci, Co, H, W, k):
     """The bf16 store path of dX rounds the same accumulators the fp32 store path writes."""
