@@ -116,15 +116,24 @@ statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ par
         is_last = (t == gridDim.x - 1);
     }
     __syncthreads();
-    if (!is_last || warp != 0) return;
+    if (!is_last) return;
+    // the last block adds the partials: every thread a strided share (loads independent of one
+    // another), then warps and the block in a fixed order
     __threadfence();
     double a = 0.0, b = 0.0;
-    for (int blk = lane; blk < static_cast<int>(gridDim.x); blk += 32) {
+#pragma unroll 4
+    for (int blk = threadIdx.x; blk < static_cast<int>(gridDim.x); blk += kThreads) {
         a += __ldcg(partials + 2 * blk);
         b += __ldcg(partials + 2 * blk + 1);
     }
     a = warp_sum(a);
     b = warp_sum(b);
+    __syncthreads();                 // sh1/sh2 were read by thread 0 above
+    if (lane == 0) { sh1[warp] = a; sh2[warp] = b; }
+    __syncthreads();
+    if (warp != 0) return;
+    a = 0.0; b = 0.0;
+    for (int w = 0; w < kThreads / 32; ++w) { a += sh1[w]; b += sh2[w]; }
     if (lane == 0) {
         float delta = 0.f;
         if (!isfinite(a) || !isfinite(b)) {

@@ -50,12 +50,12 @@ namespace {
 
 using namespace tc;
 
-constexpr int kStages = 4;
+constexpr int kStages = 4;                       // most stages (one accumulator); three with two
 constexpr int kPanel = 64 * 128;                 // 64 k-rows x 128 bytes
-constexpr int kABytes = 2 * kPanel;              // 128 input channels
+constexpr int kABytes = 2 * kPanel;              // 128 input channels (one accumulator's weights)
 constexpr int kNChunks = 4;                      // chunks of 64 positions per tile
 constexpr int kBBytes = kNChunks * kPanel;
-constexpr int kStage = kABytes + kBBytes;        // 48 KB
+constexpr int kRing = kStages * (kABytes + kBBytes);   // bytes of the stage ring (3 x 64 KB = 4 x 48 KB)
 constexpr int kThreadsT = 192;
 constexpr int kAccCols = 256;
 constexpr int kStageOut = 32 * 128;               // one warp's staged chunk: 32 channels x 64 positions, bf16
@@ -68,6 +68,8 @@ struct DxT {
     int chunks_per_img;
     long long nchunks;            // B * chunks_per_img
     int ci_tiles, ksteps;
+    int nct;                      // 64-position chunks per tile (4, or fewer when that gives too few tiles)
+    int MA;                       // accumulators per tile: 1 (128 channels, two tiles in flight) or 2 (256 channels)
     long long ntiles;
     int *err_flag;
 };
@@ -83,6 +85,11 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ PipeT pipe;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // With two accumulators a tile is 256 channels: both share the stage's code tile, each has its
+    // own weight tile, and the two TMEM accumulators belong to one tile (no second tile in
+    // flight). With one accumulator tiles alternate between the two TMEM accumulators.
+    const int MA = p.MA, S = MA == 2 ? 3 : 4;
+    const int a_bytes = MA * kABytes, stage_bytes = a_bytes + kBBytes;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -109,9 +116,9 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
             unsigned parity = 1;                 // a fresh barrier passes a wait on the previous phase
             bool ok = true;
             for (long long t = blockIdx.x; t < p.ntiles && ok; t += gridDim.x) {
-                const int ci0 = static_cast<int>(t % p.ci_tiles) * 128;
-                const long long g0 = (t / p.ci_tiles) * kNChunks;
-                const int nch = static_cast<int>(p.nchunks - g0 < kNChunks ? p.nchunks - g0 : kNChunks);
+                const int ci0 = static_cast<int>(t % p.ci_tiles) * 128 * MA;
+                const long long g0 = (t / p.ci_tiles) * p.nct;
+                const int nch = static_cast<int>(p.nchunks - g0 < p.nct ? p.nchunks - g0 : p.nct);
                 int cb[kNChunks], cp[kNChunks];
                 for (int c = 0; c < nch; ++c) {
                     cb[c] = static_cast<int>((g0 + c) / p.chunks_per_img);
@@ -120,42 +127,48 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
                 for (int ks = 0; ks < p.ksteps && ok; ++ks) {
                     ok = mbar_wait(&pipe.empty[s], parity, p.err_flag);
                     if (!ok) break;
-                    unsigned char *st = smem + s * kStage;
-                    mbar_expect_tx(&pipe.full[s], static_cast<unsigned>((2 + nch) * kPanel));
-                    tma_load_2d(st, &map_w, ci0, ks * 64, &pipe.full[s]);
-                    tma_load_2d(st + kPanel, &map_w, ci0 + 64, ks * 64, &pipe.full[s]);
+                    unsigned char *st = smem + s * stage_bytes;
+                    mbar_expect_tx(&pipe.full[s], static_cast<unsigned>((2 * MA + nch) * kPanel));
+                    for (int h = 0; h < 2 * MA; ++h)
+                        tma_load_2d(st + h * kPanel, &map_w, ci0 + 64 * h, ks * 64, &pipe.full[s]);
                     for (int c = 0; c < nch; ++c)
-                        tma_load_3d(st + kABytes + c * kPanel, &map_q, cp[c], ks * 64, cb[c], &pipe.full[s]);
-                    if (++s == kStages) { s = 0; parity ^= 1u; }
+                        tma_load_3d(st + a_bytes + c * kPanel, &map_q, cp[c], ks * 64, cb[c], &pipe.full[s]);
+                    if (++s == S) { s = 0; parity ^= 1u; }
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr unsigned idesc = make_idesc(128, kAccCols, true, true);
+            const unsigned idesc = make_idesc(128, 64 * p.nct, true, true);
             int s = 0;
             unsigned parity = 0;
             bool ok = true;
             long long it = 0;
             for (long long t = blockIdx.x; t < p.ntiles && ok; t += gridDim.x, ++it) {
-                const int a = static_cast<int>(it & 1);
-                ok = mbar_wait(&pipe.acc_empty[a], ((it >> 1) & 1) ^ 1u, p.err_flag);
+                // accumulator slot(s) of this tile and how often they have been used before
+                const int slot0 = MA == 2 ? 0 : static_cast<int>(it & 1);
+                const unsigned uses = static_cast<unsigned>(MA == 2 ? it : (it >> 1));
+                for (int a = 0; a < MA && ok; ++a) ok = mbar_wait(&pipe.acc_empty[slot0 + a], (uses & 1u) ^ 1u, p.err_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const unsigned tmem_d = tmem_base + a * kAccCols;
                 for (int ks = 0; ks < p.ksteps; ++ks) {
                     ok = mbar_wait(&pipe.full[s], parity, p.err_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    const unsigned a_addr = smem_u32(smem + s * kStage);
-                    const unsigned long long ad = make_desc(a_addr, kPanel, 1024), bd = make_desc(a_addr + kABytes, kPanel, 1024);
+                    const unsigned a_addr = smem_u32(smem + s * stage_bytes);
+                    const unsigned long long bd = make_desc(a_addr + a_bytes, kPanel, 1024);
+                    for (int a = 0; a < MA; ++a) {
+                        const unsigned long long ad = make_desc(a_addr + a * kABytes, kPanel, 1024);
+                        const unsigned tmem_d = tmem_base + (slot0 + a) * kAccCols;
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)      // 16 k-rows = 2048 bytes further per MMA
-                        mma_bf16(tmem_d, ad + 128 * k, bd + 128 * k, idesc, (ks > 0 || k > 0) ? 1u : 0u);
+                        for (int k = 0; k < 4; ++k)      // 16 k-rows = 2048 bytes further per MMA
+                            mma_bf16(tmem_d, ad + 128 * k, bd + 128 * k, idesc, (ks > 0 || k > 0) ? 1u : 0u);
+                    }
                     mma_commit(&pipe.empty[s]);
-                    if (++s == kStages) { s = 0; parity ^= 1u; }
+                    if (++s == S) { s = 0; parity ^= 1u; }
                 }
-                if (ok) mma_commit(&pipe.acc_full[a]);
+                if (ok)
+                    for (int a = 0; a < MA; ++a) mma_commit(&pipe.acc_full[slot0 + a]);
             }
         }
     } else {
@@ -165,13 +178,17 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
         long long it = 0;
         const float delta = *p.delta_p;
         const int vw = (p.HW % 8 == 0) ? 8 : ((p.HW % 4 == 0) ? 4 : 1);
-        unsigned char *stage = smem + kStages * kStage + (warp - 2) * kStageOut;
+        unsigned char *stage = smem + kRing + (warp - 2) * kStageOut;
         for (long long t = blockIdx.x; t < p.ntiles && ok; t += gridDim.x, ++it) {
-            const int a = static_cast<int>(it & 1);
-            const int ci = static_cast<int>(t % p.ci_tiles) * 128 + q * 32 + lane;
-            const long long g0 = (t / p.ci_tiles) * kNChunks;
-            const int nch = static_cast<int>(p.nchunks - g0 < kNChunks ? p.nchunks - g0 : kNChunks);
-            ok = mbar_wait(&pipe.acc_full[a], (it >> 1) & 1, p.err_flag);
+          const int slot0 = MA == 2 ? 0 : static_cast<int>(it & 1);
+          const unsigned uses = static_cast<unsigned>(MA == 2 ? it : (it >> 1));
+          for (int am = 0; am < MA; ++am) {
+            const int a = slot0 + am;
+            const int ci_w = (static_cast<int>(t % p.ci_tiles) * MA + am) * 128 + q * 32;
+            const int ci = ci_w + lane;
+            const long long g0 = (t / p.ci_tiles) * p.nct;
+            const int nch = static_cast<int>(p.nchunks - g0 < p.nct ? p.nchunks - g0 : p.nct);
+            ok = mbar_wait(&pipe.acc_full[a], uses & 1u, p.err_flag);
             if (!ok) break;
             tc_fence_after();
             for (int c = 0; c < nch; ++c) {
@@ -230,7 +247,6 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
                     // staging block -> dX with lanes along the positions: full 128-byte rows, or, when
                     // the chunk is the whole plane, one contiguous run of 32 channels x HW positions
                     __syncwarp();
-                    const int ci_w = static_cast<int>(t % p.ci_tiles) * 128 + q * 32;
                     const int nrows = p.Cin - ci_w < 32 ? p.Cin - ci_w : 32;
                     __nv_bfloat16 *base = static_cast<__nv_bfloat16 *>(p.dX) + (b * p.Cin + ci_w) * p.HW + p0;
                     if (nrows > 0) {
@@ -275,6 +291,7 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
             }
             tc_fence_before();
             warp_arrive(&pipe.acc_empty[a]);
+          }
         }
     }
     tc_fence_before();
@@ -316,11 +333,17 @@ int launch_tma_dx(dbp_ctx *ctx, const void *codes_bf16, const void *W, const flo
     p.Cin = static_cast<int>(s.Cin); p.Cout = static_cast<int>(s.Cout); p.HW = static_cast<int>(HW);
     p.chunks_per_img = static_cast<int>((HW + 63) / 64);
     p.nchunks = s.B * p.chunks_per_img;
-    p.ci_tiles = static_cast<int>((s.Cin + 127) / 128);
     p.ksteps = static_cast<int>((s.Cout + 63) / 64);
-    p.ntiles = ((p.nchunks + kNChunks - 1) / kNChunks) * p.ci_tiles;
+    // Two accumulators halve the code traffic per MMA but leave half as many tiles and no second
+    // tile in flight: worth it for long reductions that still fill the GPU. Few tiles: narrower ones.
+    const long long ntile4 = (p.nchunks + kNChunks - 1) / kNChunks;
+    p.MA = (s.Cin >= 256 && p.ksteps >= 4 && ntile4 * ((s.Cin + 255) / 256) >= (ctx->sm_count * 3) / 4) ? 2 : 1;
+    p.ci_tiles = static_cast<int>((s.Cin + 128 * p.MA - 1) / (128 * p.MA));
+    p.nct = kNChunks;
+    while (p.nct > 1 && ((p.nchunks + p.nct - 1) / p.nct) * p.ci_tiles < (ctx->sm_count * 3) / 4) p.nct /= 2;
+    p.ntiles = ((p.nchunks + p.nct - 1) / p.nct) * p.ci_tiles;
     p.err_flag = err_flag;
-    const size_t smem = static_cast<size_t>(kStages) * kStage + 4 * kStageOut + 1024;
+    const size_t smem = static_cast<size_t>(kRing) + 4 * kStageOut + 1024;
     if (cudaFuncSetAttribute(tma_dx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
         return DBP_ECUDA;
     const long long grid = p.ntiles < ctx->sm_count ? p.ntiles : ctx->sm_count;
