@@ -4,11 +4,15 @@
 // tiled copies: a stage holds 64 output channels (the reduction index) of
 //   A = W rows  [64 co][128 ci]          (M = input channels, MN-major, two 64-channel panels)
 //   B = codes   [64 co][up to 256 p]     (N = positions, MN-major, one panel per 64-position chunk)
-// A CTA is persistent: warp 0 issues the copies, warp 1 the MMAs into one of two TMEM
-// accumulators, warps 2-5 drain the other accumulator (scale by Delta, convert, store), so the
-// stores of one tile overlap the copies and MMAs of the next. Positions are handled in chunks of
-// 64 that never cross an image; a tile is four consecutive chunks (they may belong to two
-// images). Rows past the tensor's edge are zero-filled by the copy engine.
+// A CTA is persistent: warp 0 issues the copies, warp 1 the MMAs, warps 2-5 drain an accumulator
+// (scale by Delta, convert, store through a shared-memory staging block so that global stores are
+// whole rows). TMEM holds two 256-column accumulators. With one accumulator per tile (128
+// channels) tiles alternate between them, so the stores of one tile overlap the copies and MMAs of
+// the next. With two per tile (256 channels; chosen for long reductions over many channels) both
+// accumulators share the stage's code tile, which halves the code traffic per MMA.
+// Positions are handled in chunks of 64 that never cross an image; a tile is up to four
+// consecutive chunks (they may belong to two images). Rows past the tensor's edge are zero-filled
+// by the copy engine.
 #include "tc_common.cuh"
 
 namespace dbp {
