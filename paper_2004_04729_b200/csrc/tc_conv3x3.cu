@@ -489,6 +489,40 @@ __global__ void __launch_bounds__(256) tc3_dw_reduce_kernel(const float4 *__rest
     }
 }
 
+// The same sum for large weight tensors and few splits: a block owns 128 consecutive (co, ci)
+// pairs, a warp one tap at a time (coalesced 512-byte reads of every split), and the block writes
+// its 128 x 9 results as one contiguous run instead of stores nine floats apart.
+__global__ void __launch_bounds__(256) tc3_dw_reduce_rows_kernel(const float4 *__restrict__ partials, int nsplit,
+                                                                 long long Cout, long long Cin,
+                                                                 const float *__restrict__ delta_p, float *__restrict__ dW) {
+    __shared__ float out[128 * 9];
+    const long long n = Cout * Cin, n4 = n / 4, tot4 = n4 * 9;   // Cin % 4 == 0
+    const int e = threadIdx.x & 31, sg = threadIdx.x >> 5;
+    const long long r4 = blockIdx.x * 32ll + e;                  // float4 index inside a tap's plane
+    const float delta = *delta_p;
+    for (int tap = sg; tap < 9; tap += 8) {
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (r4 < n4) {
+            const float4 *src = partials + tap * n4 + r4;
+#pragma unroll 4
+            for (int s = 0; s < nsplit; ++s) {
+                const float4 v = __ldcs(src + s * tot4);
+                a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+            }
+        }
+        out[(4 * e + 0) * 9 + tap] = a.x * delta;
+        out[(4 * e + 1) * 9 + tap] = a.y * delta;
+        out[(4 * e + 2) * 9 + tap] = a.z * delta;
+        out[(4 * e + 3) * 9 + tap] = a.w * delta;
+    }
+    __syncthreads();
+    const long long base = blockIdx.x * 128ll;                   // first (co, ci) pair of the block
+    const long long left = n - base;
+    const int cnt = static_cast<int>(left < 128 ? left : 128) * 9;   // a multiple of 4
+    float4 *dst = reinterpret_cast<float4 *>(dW + base * 9);
+    for (int i = threadIdx.x; i < cnt / 4; i += 256) dst[i] = reinterpret_cast<const float4 *>(out)[i];
+}
+
 int raw_geometry(int W, int span, int &words, int &pitch) {
     // a staged row covers positions [floor4(start - (W+1)), start + span + (W+1)) plus slack for
     // the three-word reads of bytes8
@@ -586,8 +620,13 @@ int launch_tc3_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float 
     if (rc == DBP_EUNSUPPORTED) rc = launch_tc3_dw_generic(ctx, codes, X, delta_p, s, err_flag, &split);
     if (rc) return rc;
     const long long tot4 = static_cast<long long>(nw) / 4;
-    tc3_dw_reduce_kernel<<<static_cast<unsigned>((tot4 + 31) / 32), 256, 0, ctx->stream>>>(
-        reinterpret_cast<const float4 *>(ctx->tc_partials.ptr), static_cast<int>(split), s.Cout, s.Cin, delta_p, dW);
+    const long long pairs = s.Cout * s.Cin;
+    if (split <= 32 && pairs >= 128 * 128)
+        tc3_dw_reduce_rows_kernel<<<static_cast<unsigned>((pairs + 127) / 128), 256, 0, ctx->stream>>>(
+            reinterpret_cast<const float4 *>(ctx->tc_partials.ptr), static_cast<int>(split), s.Cout, s.Cin, delta_p, dW);
+    else
+        tc3_dw_reduce_kernel<<<static_cast<unsigned>((tot4 + 31) / 32), 256, 0, ctx->stream>>>(
+            reinterpret_cast<const float4 *>(ctx->tc_partials.ptr), static_cast<int>(split), s.Cout, s.Cin, delta_p, dW);
     return cuda_ok(cudaGetLastError());
 }
 
