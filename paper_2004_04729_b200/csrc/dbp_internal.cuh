@@ -181,4 +181,30 @@ inline long long choose_split(long long tiles, long long kunits, int sms, long l
 
 inline int cuda_ok(cudaError_t e) { return e == cudaSuccess ? DBP_OK : DBP_ECUDA; }
 
+// Programmatic dependent launch: a kernel launched with launch_chained may become resident while
+// the kernel before it in the stream is still draining; it must call chain_wait() before it
+// touches global memory (the wait returns once the earlier kernel has completed and its writes
+// are visible), and chain_release() lets the kernel after it do the same. Both are no-ops for a
+// kernel launched the ordinary way.
+#ifdef __CUDACC__
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                  Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+#endif
+
 }  // namespace dbp

@@ -174,6 +174,8 @@ quantize_dense_kernel(const T *__restrict__ x, long long n, unsigned long long s
     const long long nvec = n / V;
     const long long stride = static_cast<long long>(gridDim.x) * kThreads;
     long long i = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x;
+    chain_wait();
+    chain_release();
     const float delta = *delta_p;
     const bool live = (delta > 0.f) && (delta < __int_as_float(0x7f800000));
     if (!live) {                                    // sigma = 0 or non-finite input: every code is 0
@@ -245,13 +247,14 @@ int launch_quantize_dense(dbp_ctx *ctx, const void *delta, int dtype, long long 
     const long long cap = static_cast<long long>(ctx->sm_count) * 8;
     if (blocks > cap) blocks = cap;
     CodeSinks out{dense, static_cast<unsigned short *>(planes_bf16), hw > 0 ? hw : 1, pitch > 0 ? pitch : 1, count ? 1 : 0};
+    cudaError_t e;
     if (dtype == DBP_F32)
-        quantize_dense_kernel<float><<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(
-            static_cast<const float *>(delta), numel, seed, delta_p, out, ctx->state);
+        e = launch_chained(quantize_dense_kernel<float>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
+                           static_cast<const float *>(delta), numel, seed, delta_p, out, ctx->state);
     else
-        quantize_dense_kernel<__nv_bfloat16><<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(
-            static_cast<const __nv_bfloat16 *>(delta), numel, seed, delta_p, out, ctx->state);
-    return cuda_ok(cudaGetLastError());
+        e = launch_chained(quantize_dense_kernel<__nv_bfloat16>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0,
+                           ctx->stream, static_cast<const __nv_bfloat16 *>(delta), numel, seed, delta_p, out, ctx->state);
+    return cuda_ok(e);
 }
 
 }  // namespace dbp

@@ -60,6 +60,8 @@ statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ par
                   unsigned long long *__restrict__ nnz_out) {
     constexpr int EPT = Elem<T>::EPT;
     const long long nvec = n / EPT;
+    chain_wait();
+    chain_release();
     double d1 = 0.0, d2 = 0.0;
     const long long stride = static_cast<long long>(gridDim.x) * kThreads;
     long long i = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x;
@@ -363,13 +365,14 @@ int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long nume
     long long blocks = (numel / ept + kThreads * 4 - 1) / (kThreads * 4);
     if (blocks < 1) blocks = 1;
     if (blocks > ctx->partial_blocks) blocks = ctx->partial_blocks;
+    cudaError_t e;
     if (dtype == DBP_F32)
-        statistics_kernel<float><<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(
-            static_cast<const float *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out);
+        e = launch_chained(statistics_kernel<float>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
+                           static_cast<const float *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out);
     else
-        statistics_kernel<__nv_bfloat16><<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(
-            static_cast<const __nv_bfloat16 *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out);
-    return cuda_ok(cudaGetLastError());
+        e = launch_chained(statistics_kernel<__nv_bfloat16>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
+                           static_cast<const __nv_bfloat16 *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out);
+    return cuda_ok(e);
 }
 
 int launch_quantize(dbp_ctx *ctx, const void *delta, int dtype, long long numel,

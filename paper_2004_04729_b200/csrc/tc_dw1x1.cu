@@ -323,6 +323,8 @@ __global__ void __launch_bounds__(256) tc_dw_sum_kernel(const float4 *__restrict
     __shared__ float4 sh[8][32];
     const int e = threadIdx.x & 31, sg = threadIdx.x >> 5;
     const long long i4 = blockIdx.x * 32ll + e;
+    chain_wait();
+    chain_release();
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
     if (i4 < n4) {
 #pragma unroll 4
@@ -396,9 +398,9 @@ int launch_tc_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *
 
 int launch_dw_sum(dbp_ctx *ctx, const float *partials, int nsplit, long long nw, const float *delta_p, float *dW) {
     const long long n4 = nw / 4;
-    tc_dw_sum_kernel<<<static_cast<unsigned>((n4 + 31) / 32), 256, 0, ctx->stream>>>(
-        reinterpret_cast<const float4 *>(partials), nsplit, n4, delta_p, reinterpret_cast<float4 *>(dW));
-    return cuda_ok(cudaGetLastError());
+    return cuda_ok(launch_chained(tc_dw_sum_kernel, dim3(static_cast<unsigned>((n4 + 31) / 32)), dim3(256), 0, ctx->stream,
+                                  reinterpret_cast<const float4 *>(partials), nsplit, n4, delta_p,
+                                  reinterpret_cast<float4 *>(dW)));
 }
 
 }  // namespace dbp

@@ -70,6 +70,8 @@ tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     __syncthreads();
     tc_fence_after();
     const unsigned tmem_base = pipe.tmem_base;
+    chain_wait();        // from here on the kernel reads what earlier kernels wrote
+    chain_release();
 
     if (warp == 0) {
         if (lane == 0) {
@@ -212,8 +214,9 @@ int launch_tma_dw(dbp_ctx *ctx, const void *codes_bf16, const void *X, const flo
     const size_t smem = static_cast<size_t>(p.stages) * (p.MA * kATile + kBMax) + 1024;
     if (cudaFuncSetAttribute(tma_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
         return DBP_ECUDA;
-    tma_dw_kernel<<<static_cast<unsigned>(tiles * nsplit), kThreadsW, smem, ctx->stream>>>(map_q, map_x, p);
-    if ((rc = cuda_ok(cudaGetLastError()))) return rc;
+    if ((rc = cuda_ok(launch_chained(tma_dw_kernel, dim3(static_cast<unsigned>(tiles * nsplit)), dim3(kThreadsW), smem,
+                                     ctx->stream, map_q, map_x, p))))
+        return rc;
     return launch_dw_sum(ctx, p.partials, p.nsplit, static_cast<long long>(nw), delta_p, dW);
 }
 
@@ -231,6 +234,8 @@ pad_planes_kernel(const unsigned short *__restrict__ in, unsigned short *__restr
                   int H, int W, int Wp) {
     const int groups_per_row = Wp / 8;
     const long long ngroups = planes * H * groups_per_row;
+    chain_wait();
+    chain_release();
     for (long long g = blockIdx.x * 256ll + threadIdx.x; g < ngroups; g += gridDim.x * 256ll) {
         const long long row = g / groups_per_row;           // (plane, y)
         const int x0 = static_cast<int>(g - row * groups_per_row) * 8;
@@ -263,9 +268,8 @@ int launch_pad_planes(dbp_ctx *ctx, const void *in, void *out, long long planes,
     const long long cap = static_cast<long long>(ctx->sm_count) * 16;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
-    pad_planes_kernel<<<static_cast<unsigned>(blocks), 256, 0, ctx->stream>>>(
-        static_cast<const unsigned short *>(in), static_cast<unsigned short *>(out), planes, H, W, Wp);
-    return cuda_ok(cudaGetLastError());
+    return cuda_ok(launch_chained(pad_planes_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, ctx->stream,
+                                  static_cast<const unsigned short *>(in), static_cast<unsigned short *>(out), planes, H, W, Wp));
 }
 
 }  // namespace dbp

@@ -113,6 +113,10 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
     __syncthreads();
     tc_fence_after();
     const unsigned tmem_base = pipe.tmem_base;
+    // everything above touched only this CTA's shared and tensor memory; what follows reads what
+    // earlier kernels wrote
+    chain_wait();
+    chain_release();
 
     if (warp == 0) {
         if (lane == 0) {
@@ -351,8 +355,8 @@ int launch_tma_dx(dbp_ctx *ctx, const void *codes_bf16, const void *W, const flo
     if (cudaFuncSetAttribute(tma_dx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
         return DBP_ECUDA;
     const long long grid = p.ntiles < ctx->sm_count ? p.ntiles : ctx->sm_count;
-    tma_dx_kernel<<<static_cast<unsigned>(grid), kThreadsT, smem, ctx->stream>>>(map_w, map_q, p);
-    return cuda_ok(cudaGetLastError());
+    return cuda_ok(launch_chained(tma_dx_kernel, dim3(static_cast<unsigned>(grid)), dim3(kThreadsT), smem, ctx->stream,
+                                  map_w, map_q, p));
 }
 
 }  // namespace dbp
