@@ -462,6 +462,8 @@ __global__ void __launch_bounds__(kThreads3) tc3_dw_kernel(const P3 p) {
 __global__ void __launch_bounds__(256) tc3_dw_reduce_kernel(const float4 *__restrict__ partials, int nsplit,
                                                             long long Cout, long long Cin,
                                                             const float *__restrict__ delta_p, float *__restrict__ dW) {
+    chain_wait();        // launched chained: earlier kernels' writes are visible from here on
+    chain_release();
     __shared__ float4 sh[8][32];
     const long long n = Cout * Cin, tot4 = n * 9 / 4;            // Cin % 4 == 0
     const int e = threadIdx.x & 31, sg = threadIdx.x >> 5;
@@ -495,6 +497,8 @@ __global__ void __launch_bounds__(256) tc3_dw_reduce_kernel(const float4 *__rest
 __global__ void __launch_bounds__(256) tc3_dw_reduce_rows_kernel(const float4 *__restrict__ partials, int nsplit,
                                                                  long long Cout, long long Cin,
                                                                  const float *__restrict__ delta_p, float *__restrict__ dW) {
+    chain_wait();        // launched chained: earlier kernels' writes are visible from here on
+    chain_release();
     __shared__ float out[128 * 9];
     const long long n = Cout * Cin, n4 = n / 4, tot4 = n4 * 9;   // Cin % 4 == 0
     const int e = threadIdx.x & 31, sg = threadIdx.x >> 5;
@@ -622,12 +626,12 @@ int launch_tc3_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float 
     const long long tot4 = static_cast<long long>(nw) / 4;
     const long long pairs = s.Cout * s.Cin;
     if (split <= 32 && pairs >= 128 * 128)
-        tc3_dw_reduce_rows_kernel<<<static_cast<unsigned>((pairs + 127) / 128), 256, 0, ctx->stream>>>(
-            reinterpret_cast<const float4 *>(ctx->tc_partials.ptr), static_cast<int>(split), s.Cout, s.Cin, delta_p, dW);
-    else
-        tc3_dw_reduce_kernel<<<static_cast<unsigned>((tot4 + 31) / 32), 256, 0, ctx->stream>>>(
-            reinterpret_cast<const float4 *>(ctx->tc_partials.ptr), static_cast<int>(split), s.Cout, s.Cin, delta_p, dW);
-    return cuda_ok(cudaGetLastError());
+        return cuda_ok(launch_chained(tc3_dw_reduce_rows_kernel, dim3(static_cast<unsigned>((pairs + 127) / 128)), dim3(256), 0,
+                                      ctx->stream, reinterpret_cast<const float4 *>(ctx->tc_partials.ptr),
+                                      static_cast<int>(split), s.Cout, s.Cin, delta_p, dW));
+    return cuda_ok(launch_chained(tc3_dw_reduce_kernel, dim3(static_cast<unsigned>((tot4 + 31) / 32)), dim3(256), 0, ctx->stream,
+                                  reinterpret_cast<const float4 *>(ctx->tc_partials.ptr), static_cast<int>(split), s.Cout,
+                                  s.Cin, delta_p, dW));
 }
 
 }  // namespace dbp

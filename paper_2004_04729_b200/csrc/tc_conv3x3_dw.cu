@@ -63,6 +63,8 @@ struct PipeW {
 // (any P <= 64). NP: 64-channel panels of the code operand (N = 64 NP output channels).
 template <int XM, int NP>
 __global__ void __launch_bounds__(kThreadsW) tc3_dw_shift_kernel(const Sw3P p) {
+    chain_wait();        // launched chained: earlier kernels' writes are visible from here on
+    chain_release();
     constexpr int N = 64 * NP;
     constexpr int TCOLS = NP == 2 ? 512 : 256;                         // three accumulators of N columns
     extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -367,7 +369,7 @@ int run_w(dbp_ctx *ctx, const Sw3P &p, dim3 grid, size_t smem) {
     if (cudaFuncSetAttribute(tc3_dw_shift_kernel<XM, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(smem)) != cudaSuccess)
         return DBP_ECUDA;
-    tc3_dw_shift_kernel<XM, NP><<<grid, kThreadsW, smem, ctx->stream>>>(p);
+    if (launch_chained(tc3_dw_shift_kernel<XM, NP>, grid, dim3(kThreadsW), smem, ctx->stream, p) != cudaSuccess) return DBP_ECUDA;
     return cuda_ok(cudaGetLastError());
 }
 template <int XM>

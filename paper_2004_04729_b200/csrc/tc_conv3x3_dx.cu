@@ -123,6 +123,8 @@ __device__ __forceinline__ void store_run(const Sx3P &p, const unsigned (&v)[32]
 
 template <int MT, int MODE>
 __global__ void __launch_bounds__(kThreadsS) tc3_dx_shift_kernel(const Sx3P p) {
+    chain_wait();        // launched chained: earlier kernels' writes are visible from here on
+    chain_release();
     constexpr bool SLAB = MODE != 0;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -328,6 +330,8 @@ __global__ void __launch_bounds__(kThreadsS) tc3_dx_shift_kernel(const Sx3P p) {
 // swizzled layout the MMA reads (zero beyond Cin); one thread per 16-byte chunk
 __global__ void __launch_bounds__(256) w_images_dx_kernel(const __nv_bfloat16 *__restrict__ W, __nv_bfloat16 *__restrict__ out,
                                                           int Cout, int Cin, int mt_pad, long long nchunks) {
+    chain_wait();        // launched chained: earlier kernels' writes are visible from here on
+    chain_release();
     const unsigned short *w = reinterpret_cast<const unsigned short *>(W);
     for (long long idx = blockIdx.x * 256ll + threadIdx.x; idx < nchunks; idx += gridDim.x * 256ll) {
         const long long img = idx >> 10;
@@ -351,7 +355,7 @@ int run_s(dbp_ctx *ctx, const Sx3P &p, dim3 grid, size_t smem) {
     if (cudaFuncSetAttribute(tc3_dx_shift_kernel<MT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(smem)) != cudaSuccess)
         return DBP_ECUDA;
-    tc3_dx_shift_kernel<MT, MODE><<<grid, kThreadsS, smem, ctx->stream>>>(p);
+    if (launch_chained(tc3_dx_shift_kernel<MT, MODE>, grid, dim3(kThreadsS), smem, ctx->stream, p) != cudaSuccess) return DBP_ECUDA;
     return cuda_ok(cudaGetLastError());
 }
 template <int MT>
@@ -415,9 +419,9 @@ int launch_tc3_dx_shift(dbp_ctx *ctx, const int8_t *codes, const void *W, const 
     {
         long long blocks = (nchunks + 255) / 256;
         if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
-        w_images_dx_kernel<<<static_cast<unsigned>(blocks), 256, 0, ctx->stream>>>(
-            static_cast<const __nv_bfloat16 *>(W), wimg, p.Cout, p.Cin, p.mt_pad, nchunks);
-        if ((rc = cuda_ok(cudaGetLastError()))) return rc;
+        if ((rc = cuda_ok(launch_chained(w_images_dx_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, ctx->stream,
+                                         static_cast<const __nv_bfloat16 *>(W), wimg, p.Cout, p.Cin, p.mt_pad, nchunks))))
+            return rc;
     }
     p.Wimg = wimg;
     dim3 grid(static_cast<unsigned>(tiles), static_cast<unsigned>(gy));
