@@ -4,7 +4,7 @@
 // tiled copies: a stage holds 64 output channels (the reduction index) of
 //   A = W rows  [64 co][128 ci]          (M = input channels, MN-major, two 64-channel panels)
 //   B = codes   [64 co][up to 256 p]     (N = positions, MN-major, one panel per 64-position chunk)
-// A CTA is persistent: warp 0 issues the copies, warp 1 the MMAs, warps 2-5 drain an accumulator
+// A CTA is persistent: warp 0 issues the copies, warp 1 the MMAs, warps 2-9 drain an accumulator
 // (scale by Delta, convert, store through a shared-memory staging block so that global stores are
 // whole rows). TMEM holds two 256-column accumulators. With one accumulator per tile (128
 // channels) tiles alternate between them, so the stores of one tile overlap the copies and MMAs of
@@ -60,7 +60,8 @@ constexpr int kABytes = 2 * kPanel;              // 128 input channels (one accu
 constexpr int kNChunks = 4;                      // chunks of 64 positions per tile
 constexpr int kBBytes = kNChunks * kPanel;
 constexpr int kRing = kStages * (kABytes + kBBytes);   // bytes of the stage ring (3 x 64 KB = 4 x 48 KB)
-constexpr int kThreadsT = 192;
+constexpr int kEpiWarps = 8;                      // two per TMEM lane quarter: even and odd chunks of a tile
+constexpr int kThreadsT = 64 + 32 * kEpiWarps;
 constexpr int kAccCols = 256;
 constexpr int kStageOut = 32 * 128;               // one warp's staged chunk: 32 channels x 64 positions, bf16
 
@@ -102,7 +103,7 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(&pipe.acc_full[a], 1);
-            mbar_init(&pipe.acc_empty[a], 4);
+            mbar_init(&pipe.acc_empty[a], kEpiWarps);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         tma_prefetch_desc(&map_w);
@@ -187,6 +188,7 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
         const float delta = *p.delta_p;
         const int vw = (p.HW % 8 == 0) ? 8 : ((p.HW % 4 == 0) ? 4 : 1);
         unsigned char *stage = smem + kRing + (warp - 2) * kStageOut;
+        const int part = (warp - 2) >> 2;          // which chunks of a tile this warp drains
         for (long long t = blockIdx.x; t < p.ntiles && ok; t += gridDim.x, ++it) {
           const int slot0 = MA == 2 ? 0 : static_cast<int>(it & 1);
           const unsigned uses = static_cast<unsigned>(MA == 2 ? it : (it >> 1));
@@ -199,7 +201,7 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
             ok = mbar_wait(&pipe.acc_full[a], uses & 1u, p.err_flag);
             if (!ok) break;
             tc_fence_after();
-            for (int c = 0; c < nch; ++c) {
+            for (int c = part; c < nch; c += kEpiWarps / 4) {
                 const long long b = (g0 + c) / p.chunks_per_img;
                 const int p0 = static_cast<int>((g0 + c) % p.chunks_per_img) * 64;
                 const int nv = p.HW - p0 < 64 ? p.HW - p0 : 64;           // valid positions of the chunk
@@ -351,7 +353,7 @@ int launch_tma_dx(dbp_ctx *ctx, const void *codes_bf16, const void *W, const flo
     while (p.nct > 1 && ((p.nchunks + p.nct - 1) / p.nct) * p.ci_tiles < (ctx->sm_count * 3) / 4) p.nct /= 2;
     p.ntiles = ((p.nchunks + p.nct - 1) / p.nct) * p.ci_tiles;
     p.err_flag = err_flag;
-    const size_t smem = static_cast<size_t>(kRing) + 4 * kStageOut + 1024;
+    const size_t smem = static_cast<size_t>(kRing) + kEpiWarps * kStageOut + 1024;
     if (cudaFuncSetAttribute(tma_dx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
         return DBP_ECUDA;
     const long long grid = p.ntiles < ctx->sm_count ? p.ntiles : ctx->sm_count;
