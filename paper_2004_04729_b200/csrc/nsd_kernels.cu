@@ -23,6 +23,12 @@ struct Elem<float> {
         v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
     }
     __device__ static float one(const float *p) { return __ldg(p); }
+    // read-once data: do not keep the line in L1
+    __device__ static void load_stream(const float *p, float (&v)[4]) {
+        unsigned a, b, c, d;
+        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "l"(p));
+        v[0] = __uint_as_float(a); v[1] = __uint_as_float(b); v[2] = __uint_as_float(c); v[3] = __uint_as_float(d);
+    }
 };
 
 template <>
@@ -39,6 +45,15 @@ struct Elem<__nv_bfloat16> {
     }
     __device__ static float one(const __nv_bfloat16 *p) {
         return __uint_as_float(static_cast<unsigned>(__ldg(reinterpret_cast<const unsigned short *>(p))) << 16);
+    }
+    __device__ static void load_stream(const __nv_bfloat16 *p, float (&v)[8]) {
+        unsigned w[4];
+        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "l"(p));
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[2 * i] = __uint_as_float(w[i] << 16);
+            v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
     }
 };
 
@@ -64,14 +79,17 @@ statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ par
     chain_release();
     double d1 = 0.0, d2 = 0.0;
     const long long stride = static_cast<long long>(gridDim.x) * kThreads;
-    long long i = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x;
-    // four 128-bit loads in flight per thread
-    for (; i + 3 * stride < nvec; i += 4 * stride) {
-        float v[4][EPT];
+    // whole tiles of kUnroll x kThreads 128-bit vectors, a block at a time: kUnroll loads in flight
+    // per thread, consecutive threads on consecutive vectors
+    constexpr int kUnroll = 8;
+    const long long tile = static_cast<long long>(kUnroll) * kThreads, ntile = nvec / tile;
+    for (long long t = blockIdx.x; t < ntile; t += gridDim.x) {
+        const T *p = x + (t * tile + threadIdx.x) * EPT;
+        float v[kUnroll][EPT];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) Elem<T>::load(x + (i + u * stride) * EPT, v[u]);
+        for (int u = 0; u < kUnroll; ++u) Elem<T>::load_stream(p + static_cast<long long>(u) * kThreads * EPT, v[u]);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < kUnroll; ++u) {
             float s1 = 0.f, s2 = 0.f;
 #pragma unroll
             for (int j = 0; j < EPT; ++j) {
@@ -82,6 +100,8 @@ statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ par
             d2 += static_cast<double>(s2);
         }
     }
+    // the vectors after the last whole tile
+    long long i = ntile * tile + static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x;
     for (; i < nvec; i += stride) {
         float v[EPT];
         Elem<T>::load(x + i * EPT, v);
@@ -362,7 +382,7 @@ int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long nume
         return cuda_ok(cudaGetLastError());
     }
     const int ept = dtype == DBP_F32 ? 4 : 8;
-    long long blocks = (numel / ept + kThreads * 4 - 1) / (kThreads * 4);
+    long long blocks = numel / ept / (kThreads * 8);          // one block per tile of eight vectors per thread
     if (blocks < 1) blocks = 1;
     if (blocks > ctx->partial_blocks) blocks = ctx->partial_blocks;
     cudaError_t e;
