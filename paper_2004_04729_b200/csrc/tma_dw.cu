@@ -20,6 +20,7 @@ using namespace tc;
 constexpr int kATile = 128 * 128;                // 128 rows x 64 bf16
 constexpr int kBMax = 256 * 128;
 constexpr int kThreadsW = 192;
+constexpr int kStageW = 32 * 128;                // one warp's staged 32 x 32 fp32 block
 
 struct DwT {
     float *partials;              // [nsplit][Cout][Cin]
@@ -120,25 +121,37 @@ tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             if (ok) mma_commit(&pipe.acc_full);
         }
     } else {
-        // epilogue: TMEM lane = output channel, column = input channel
+        // epilogue: TMEM lane = output channel, column = input channel. A warp's 32 x 32 block goes
+        // through a shared staging block (128-byte rows, 16-byte pieces XOR-swizzled by the row) so
+        // that the global stores are whole 128-byte rows of the partial block, four per instruction.
         const int q = warp & 3;
+        unsigned char *stage = smem + S * stage_bytes + (warp - 2) * kStageW;
         if (k1 > k0 && mbar_wait(&pipe.acc_full, 0, p.err_flag)) {
             tc_fence_after();
             for (int a = 0; a < p.MA; ++a) {
-                const int co = co0 + a * 128 + q * 32 + lane;
-                float *row = p.partials + (static_cast<long long>(split) * p.Cout + co) * p.Cin + ci0;
+                const int co_w = co0 + a * 128 + q * 32;                 // first output channel of this warp
+                const int nrows = p.Cout - co_w < 32 ? p.Cout - co_w : 32;
+                float *blk = p.partials + (static_cast<long long>(split) * p.Cout + co_w) * p.Cin + ci0;
 #pragma unroll 1
                 for (int c0 = 0; c0 < p.NT; c0 += 32) {
                     unsigned v[32];
                     tmem_ld32(tmem_base + (static_cast<unsigned>(q * 32) << 16) + a * p.NTp + c0, v);
-                    if (co < p.Cout) {
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4)
-                            if (c0 + j < p.NT && ci0 + c0 + j < p.Cin)
-                                *reinterpret_cast<float4 *>(row + c0 + j) =
-                                    make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
-                                                __uint_as_float(v[j + 3]));
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<uint4 *>(stage + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                            make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                    __syncwarp();
+                    const int ch = lane & 7;                              // my 16-byte piece: columns c0 + 4 ch ..
+                    if (c0 + 4 * ch < p.NT && ci0 + c0 + 4 * ch < p.Cin) {
+#pragma unroll
+                        for (int r0 = 0; r0 < 32; r0 += 4) {
+                            const int r = r0 + (lane >> 3);
+                            if (r < nrows)
+                                *reinterpret_cast<uint4 *>(blk + static_cast<long long>(r) * p.Cin + c0 + 4 * ch) =
+                                    *reinterpret_cast<const uint4 *>(stage + r * 128 + ((ch ^ (r & 7)) << 4));
+                        }
                     }
+                    __syncwarp();
                 }
             }
         }
@@ -211,7 +224,7 @@ int launch_tma_dw(dbp_ctx *ctx, const void *codes_bf16, const void *X, const flo
         const unsigned box[3] = {64, static_cast<unsigned>(p.NT), 1};
         if (!encode_map_bf16(&map_x, Xsrc, 3, dims, str, box)) return DBP_ECUDA;
     }
-    const size_t smem = static_cast<size_t>(p.stages) * (p.MA * kATile + kBMax) + 1024;
+    const size_t smem = static_cast<size_t>(p.stages) * (p.MA * kATile + kBMax) + 4 * kStageW + 1024;
     if (cudaFuncSetAttribute(tma_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
         return DBP_ECUDA;
     if ((rc = cuda_ok(launch_chained(tma_dw_kernel, dim3(static_cast<unsigned>(tiles * nsplit)), dim3(kThreadsW), smem,
