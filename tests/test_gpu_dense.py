@@ -161,3 +161,32 @@ def test_crossover_uses_the_measured_density(ctx):
     torch.cuda.synchronize()
     assert c2.profile_read()["weight_taps"][1] == 0
     c2.close()
+
+
+def test_back_to_back_calls_are_ordered(ctx):
+    """Two layers enqueued without a synchronisation in between, the second quantizing the dX of
+    the first (Eq. (qda) feeds the layer below): the second call's kernels may become resident
+    while the first call's are draining, but must not read dX before it is complete. Checked
+    layer by layer against the oracle, the oracle reading the CUDA path's own dX."""
+    import paper_2004_04729_b200 as dbp
+    L2 = wl.conv_layer(4, 128, 256, 14, 14, 1, data_seed=21, scale=5.0, dtype="bf16")   # upper layer: 128 -> 256
+    L1 = wl.conv_layer(4, 64, 128, 14, 14, 1, data_seed=22, scale=5.0, dtype="bf16")    # lower layer: 64 -> 128
+    d2, X2, W2 = _t(L2.delta), _t(L2.X), _t(L2.W)
+    X1, W1 = _t(L1.X), _t(L1.W)
+    for rep in range(3):                                  # repeated: the workspaces are reused every time
+        q2, q1 = dbp.SparseGradient(d2.numel()), dbp.SparseGradient(L1.delta.size)
+        o2 = dbp.dithered_conv_backward(ctx, d2, X2, W2, 7, 5.0, q_out=q2, flags=dbp.DBP_FORCE_DENSE)
+        o1 = dbp.dithered_conv_backward(ctx, o2["dX"], X1, W1, 8, 5.0, q_out=q1, flags=dbp.DBP_FORCE_DENSE | dbp.DBP_DX_F32)
+        torch.cuda.synchronize()
+        assert ctx.last_device_status() == (0, 0)
+        for (q, o, delta_np, X, W, seed, f32) in ((q2, o2, L2.delta, L2.X, L2.W, 7, False),
+                                                  (q1, o1, o2["dX"].float().cpu().numpy(), L1.X, L1.W, 8, True)):
+            D = np.float32(q.delta.item())
+            codes, nnz, _ = oracle.nsd_codes(delta_np, seed, D)
+            assert np.array_equal(dbp.nsd_decode_dense(ctx, q).cpu().numpy().reshape(codes.shape), codes)
+            ref = oracle.conv_backward(codes, D, X, W, with_abs=True)
+            got = o["dW"].double().cpu().numpy()
+            assert np.all(np.abs(got - ref["dW"]) <= TOL * ref["S_dW"] + 1e-30)
+            gx = o["dX"].double().cpu().numpy()
+            slack = 0.0 if f32 else 2.0 ** -8
+            assert np.all(np.abs(gx - ref["dX"]) <= slack * np.abs(ref["dX"]) + TOL * ref["S_dX"] + 1e-30)
