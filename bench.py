@@ -94,21 +94,29 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            self.rows.append((time.perf_counter(), [c.strip() for c in line.split(",")]))
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None, t_fallback=None):
+        """Samples taken inside [t_begin, t_end] (the timed region); when the region was shorter
+        than the sampling period, the samples since t_fallback (warm-up included) instead."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         time.sleep(0.15)
         self.proc.terminate()
-        sm = [float(r[0]) for r in self.rows if r and r[0].replace(".", "").isdigit()]
-        mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
+        window = "timed region"
+        rows = [r for t, r in self.rows if t_begin is None or (t_begin <= t <= t_end)]
+        if not rows and t_fallback is not None:
+            rows, window = [r for t, r in self.rows if t_fallback <= t <= t_end + 0.2], "warm-up and timed region"
+        if not rows:
+            rows, window = [r for _, r in self.rows], "whole run"
+        sm = [float(r[0]) for r in rows if r and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         reasons = [n for j, n in enumerate(names)
-                   if any(len(r) > 3 + j and r[3 + j].lower().startswith("active") for r in self.rows)]
+                   if any(len(r) > 3 + j and r[3 + j].lower().startswith("active") for r in rows)]
         return {"sm_mhz": statistics.median(sm) if sm else None,
                 "sm_max_mhz": max(mx) if mx else None, "reasons": reasons,
-                "samples": len(sm)}
+                "samples": len(sm), "window": window}
 
 
 # ------------------------------------------------------------------ CPU oracle arm
@@ -186,7 +194,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=5)
     ap.add_argument("--batch", type=int, default=0, help="override the config's batch size")
@@ -214,6 +222,9 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
     ctx = dbp.Context(local)
+    sampler = ClockSampler(local)       # nvidia-smi takes a while to deliver its first sample: start it now
+    if rank == 0:
+        sampler.start()
 
     specs, name = layer_specs(args.config, args.batch)
     if args.only:
@@ -271,6 +282,7 @@ def main():
     # and names the dominant kind. The events cost stream time, so the timed region brackets
     # only the dominant kind (its duration is what the roofline line uses).
     # The first warm-up step grows the context's workspaces (allocations) and is not profiled.
+    t_warm = time.perf_counter()
     step()
     barrier()
     ctx.profile_enable(True)
@@ -283,17 +295,16 @@ def main():
     prof_all = ctx.profile_read()
     top_kind = max(prof_all, key=lambda k: prof_all[k][0])
     ctx.profile_select([top_kind])
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    t_begin = time.perf_counter()
     e0.record()
     for _ in range(args.steps):
         step()
     e1.record()
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    t_end = time.perf_counter()
+    clocks = sampler.stop(t_begin, t_end, t_warm) if rank == 0 else None
     ms = e0.elapsed_time(e1) / args.steps
     prof_top = ctx.profile_read()
     ctx.profile_enable(False)
