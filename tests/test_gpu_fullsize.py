@@ -58,6 +58,21 @@ def test_config3_full_size(ctx):
     _full_size_case(ctx, wl.config3())           # B128, fp32: the sparse kernels
 
 
-@pytest.mark.parametrize("idx", [1, 2, 3, 10, 13, 14])
+@pytest.mark.parametrize("idx", [1, 2, 3, 9, 10, 11, 13, 14, 15])
 def test_config5_full_size_layers(ctx, idx):
     _full_size_case(ctx, wl.config5_layer(idx))  # B64, bf16: the path bench.py times
+
+
+@pytest.mark.parametrize("idx", [3, 9, 13, 15])
+def test_config5_full_size_bf16_dx_is_the_rounded_f32_dx(ctx, idx):
+    """bench.py stores dX as bf16: at full size (persistent CTAs over many tiles, one or two
+    accumulators per tile, padded small planes) those stores must be the fp32 results rounded."""
+    import paper_2004_04729_b200 as dbp
+    L = wl.config5_layer(idx)
+    d, X, W = (torch.from_numpy(a).to(torch.bfloat16).cuda() for a in (L.delta, L.X, L.W))
+    a = dbp.dithered_conv_backward(ctx, d, X, W, L.seed, L.scale, need_dW=False, flags=dbp.DBP_DX_F32)
+    b = dbp.dithered_conv_backward(ctx, d, X, W, L.seed, L.scale, need_dW=False)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == (0, 0)
+    assert b["dX"].dtype == torch.bfloat16
+    assert torch.equal(a["dX"].to(torch.bfloat16), b["dX"])
