@@ -91,7 +91,13 @@ typedef struct dbp_sparse {
 } dbp_sparse;
 
 /* Context. `device` is a CUDA ordinal; `cuda_stream` is a cudaStream_t (NULL = default
- * stream). The context owns its workspace and frees it in dbp_destroy. */
+ * stream). The context owns its workspace and frees it in dbp_destroy. The workspace grows
+ * (cudaMalloc, which synchronises the device) the first time a call needs more of it than any
+ * call before: the dense codes of delta (1 and/or 2 bytes per element), re-laid weights,
+ * activations copied to 16-byte aligned planes, the split-K partial blocks of dW. Calls of
+ * sizes seen before allocate nothing. Kernels of consecutive calls on one context may overlap at
+ * their edges (a kernel becomes resident while the one before it drains) but never read data
+ * before the kernel that writes it has completed. */
 int dbp_create(dbp_ctx **out, int device, void *cuda_stream);
 int dbp_destroy(dbp_ctx *ctx);
 int dbp_set_stream(dbp_ctx *ctx, void *cuda_stream);
