@@ -191,6 +191,23 @@ def run_reference(args):
 
 # ------------------------------------------------------------------ CUDA arm
 
+def max_over_ranks(value, device, world):
+    """The slowest rank's time: every rank runs the same step on its own shard, so the job's
+    step time is the maximum (the process group is NCCL on GPUs, gloo in the CPU tests)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.item()
+
+
+def job_throughput(flops_per_rank_step, world, ms_per_step):
+    """Whole-job dense-equivalent GFLOP/s: the work of all ranks over the slowest rank's time."""
+    return flops_per_rank_step * world / (ms_per_step * 1e-3) / 1e9
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -309,11 +326,8 @@ def main():
     prof_top = ctx.profile_read()
     ctx.profile_enable(False)
     ctx.profile_select(None)
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = t.item()
-    value = dense_flops * world / (ms * 1e-3) / 1e9
+    ms = max_over_ranks(ms, dev, world)
+    value = job_throughput(dense_flops, world, ms)
 
     # host time to enqueue one step (the launch queue is empty and deep enough for one step)
     barrier()
@@ -350,11 +364,8 @@ def main():
             host_step()
         barrier()
         dt = (time.perf_counter() - t0) / ksteps
-        if world > 1:
-            t = torch.tensor([dt], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = t.item()
-        e2e = {"value": dense_flops * world / dt / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+        dt = max_over_ranks(dt, dev, world)
+        e2e = {"value": job_throughput(dense_flops, world, dt * 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": dt * 1e3, "steps": ksteps}
 
     # ---- dense library backward on the same shapes (context, not the product path)
