@@ -152,6 +152,8 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
                             : launch_tc_dx(ctx, codes, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout);
             if (rc) return rc;
         }
+        if (ctx->hook_after_dx && cudaEventRecord(ctx->hook_after_dx, ctx->stream) != cudaSuccess) return DBP_ECUDA;
+        if (dW && ctx->hook_before_dw && cudaStreamWaitEvent(ctx->stream, ctx->hook_before_dw, 0) != cudaSuccess) return DBP_ECUDA;
         if (dW) {
             KernelTimer t(ctx, DBP_K_DW_DENSE);
             rc = dw_tma ? launch_tma_dw(ctx, codes16, X, delta_p, s, dW, &ctx->state->tc_timeout)
@@ -185,6 +187,8 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
         }
         if (rc) return rc;
     }
+    if (ctx->hook_after_dx && cudaEventRecord(ctx->hook_after_dx, ctx->stream) != cudaSuccess) return DBP_ECUDA;
+    if (dW && ctx->hook_before_dw && cudaStreamWaitEvent(ctx->stream, ctx->hook_before_dw, 0) != cudaSuccess) return DBP_ECUDA;
     if (dW) {
         KernelTimer t(ctx, DBP_K_DW);
         rc = launch_conv_dw_streamed(ctx, codes, X, io, delta_p, s, dW);
@@ -257,6 +261,10 @@ int dbp_destroy(dbp_ctx *ctx) {
     for (ProfSlot &p : ctx->prof) { cudaEventDestroy(p.begin); cudaEventDestroy(p.end); }
     if (ctx->nnz_host) cudaFreeHost(ctx->nnz_host);
     if (ctx->nnz_event) cudaEventDestroy(ctx->nnz_event);
+    if (ctx->copy_in) { cudaStreamSynchronize(ctx->copy_in); cudaStreamDestroy(ctx->copy_in); }
+    if (ctx->copy_out) { cudaStreamSynchronize(ctx->copy_out); cudaStreamDestroy(ctx->copy_out); }
+    if (ctx->ev_x_up) cudaEventDestroy(ctx->ev_x_up);
+    if (ctx->ev_dx_done) cudaEventDestroy(ctx->ev_dx_done);
     if (ctx->state) cudaFree(ctx->state);
     if (ctx->partials) cudaFree(ctx->partials);
     delete ctx;
@@ -416,19 +424,45 @@ static int host_backward(dbp_ctx *ctx, const void *delta, const void *X, const v
         (rc = ws_reserve(ctx, ctx->io[4], dX ? nx * dx_es : 16)) || (rc = ws_reserve(ctx, ctx->io[5], db ? s.Cout * 4 : 16)))
         return rc;
     cudaStream_t st = ctx->stream;
+    if (!ctx->copy_in) {
+        if (cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ctx->ev_x_up, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ctx->ev_dx_done, cudaEventDisableTiming) != cudaSuccess)
+            return DBP_ECUDA;
+    }
+    // delta and W go up on the context's stream (dX needs only them); X goes up beside them on
+    // its own stream and is waited for before the dW kernels; dX comes down on a third stream
+    // as soon as its kernel is done, while X is still going up and dW is being computed.
+    // Staging buffers are free here: the previous *_host call ended with every stream idle.
     if (cudaMemcpyAsync(ctx->io[0].ptr, delta, nd * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return DBP_ECUDA;
-    if (X && cudaMemcpyAsync(ctx->io[1].ptr, X, nx * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return DBP_ECUDA;
     if (W && cudaMemcpyAsync(ctx->io[2].ptr, W, nw * es, cudaMemcpyHostToDevice, st) != cudaSuccess) return DBP_ECUDA;
+    if (X) {
+        if (cudaMemcpyAsync(ctx->io[1].ptr, X, nx * es, cudaMemcpyHostToDevice, ctx->copy_in) != cudaSuccess ||
+            cudaEventRecord(ctx->ev_x_up, ctx->copy_in) != cudaSuccess)
+            return DBP_ECUDA;
+        ctx->hook_before_dw = ctx->ev_x_up;
+    }
+    if (dX) ctx->hook_after_dx = ctx->ev_dx_done;
     rc = conv_backward_impl(ctx, ctx->io[0].ptr, X ? ctx->io[1].ptr : nullptr, W ? ctx->io[2].ptr : nullptr, io, s,
                             seed, scale, nullptr, nullptr, dW ? static_cast<float *>(ctx->io[3].ptr) : nullptr,
                             dX ? ctx->io[4].ptr : nullptr, db ? static_cast<float *>(ctx->io[5].ptr) : nullptr, flags);
-    if (rc) return rc;
+    ctx->hook_before_dw = nullptr;
+    ctx->hook_after_dx = nullptr;
+    if (rc) {
+        cudaStreamSynchronize(ctx->copy_in);
+        return rc;
+    }
+    if (dX && (cudaStreamWaitEvent(ctx->copy_out, ctx->ev_dx_done, 0) != cudaSuccess ||
+               cudaMemcpyAsync(dX, ctx->io[4].ptr, nx * dx_es, cudaMemcpyDeviceToHost, ctx->copy_out) != cudaSuccess))
+        return DBP_ECUDA;
     if (dW && cudaMemcpyAsync(dW, ctx->io[3].ptr, nw * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DBP_ECUDA;
-    if (dX && cudaMemcpyAsync(dX, ctx->io[4].ptr, nx * dx_es, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DBP_ECUDA;
     if (db && cudaMemcpyAsync(db, ctx->io[5].ptr, s.Cout * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DBP_ECUDA;
     DeviceState h;
     if (cudaMemcpyAsync(&h, ctx->state, sizeof(h), cudaMemcpyDeviceToHost, st) != cudaSuccess) return DBP_ECUDA;
-    if (cudaStreamSynchronize(st) != cudaSuccess) return DBP_ECUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess || cudaStreamSynchronize(ctx->copy_out) != cudaSuccess ||
+        cudaStreamSynchronize(ctx->copy_in) != cudaSuccess)
+        return DBP_ECUDA;
     if (delta_out) *delta_out = h.delta;
     if (nnz_out) *nnz_out = static_cast<long long>(h.nnz);
     return DBP_OK;

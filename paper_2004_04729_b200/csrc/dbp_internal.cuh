@@ -50,6 +50,12 @@ struct dbp_ctx {
     dbp::Workspace sp_bitmap, sp_offsets, sp_values;  // internal dbp_sparse
     dbp::Workspace tc_partials;         // split-K partial blocks of the dense dW kernel
     dbp::Workspace io[8];               // staging for the *_host entry points
+    // *_host entry points: X goes up and dX comes down on streams of their own, so that the two
+    // directions of the host link work at the same time; the events order them against the
+    // kernels (dX done -> its read-back may start; X up -> the dW kernels may start)
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_x_up = nullptr, ev_dx_done = nullptr;
+    cudaEvent_t hook_after_dx = nullptr, hook_before_dw = nullptr;   // set only during a *_host call
     float crossover = 0.03f;            // density above which the dense path is preferred
     float density_estimate = 1.0f;      // density of the latest finished quantization
     unsigned long long *nnz_host = nullptr;   // pinned: asynchronous read-back of nnz
