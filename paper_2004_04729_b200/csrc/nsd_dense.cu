@@ -95,6 +95,19 @@ struct CodeSinks {
     int count;                    // add nnz / clipped counts to the context's counters
 };
 
+// plane = e / hw and the offset inside it; a 32-bit division when the index allows it (a 64-bit
+// one costs several times as many instructions)
+__device__ __forceinline__ void split_index(long long e, long long hw, long long &plane, long long &pp) {
+    if (((e | hw) >> 32) == 0) {
+        const unsigned q = static_cast<unsigned>(e) / static_cast<unsigned>(hw);
+        plane = q;
+        pp = static_cast<unsigned>(e) - q * static_cast<unsigned>(hw);
+    } else {
+        plane = e / hw;
+        pp = e - plane * hw;
+    }
+}
+
 template <int V>
 __device__ __forceinline__ void store_codes(const CodeSinks &o, long long e0, const unsigned (&pk)[V / 4]) {
     if (o.dense8 != nullptr) {
@@ -111,7 +124,8 @@ __device__ __forceinline__ void store_codes(const CodeSinks &o, long long e0, co
         } else if ((o.hw & 3) == 0) {
             // e0 and the plane size are multiples of 4: each group of four codes lies in one plane
             // and starts on an 8-byte boundary there
-            long long plane = e0 / o.hw, pp = e0 - plane * o.hw;
+            long long plane, pp;
+            split_index(e0, o.hw, plane, pp);
 #pragma unroll
             for (int g = 0; g < V / 4; ++g) {
                 *reinterpret_cast<uint2 *>(o.planes16 + plane * o.pitch + pp) = make_uint2(h[2 * g], h[2 * g + 1]);
@@ -119,7 +133,8 @@ __device__ __forceinline__ void store_codes(const CodeSinks &o, long long e0, co
                 if (pp == o.hw) { pp = 0; ++plane; }
             }
         } else {
-            long long plane = e0 / o.hw, pp = e0 - plane * o.hw;
+            long long plane, pp;
+            split_index(e0, o.hw, plane, pp);
 #pragma unroll
             for (int j = 0; j < V; ++j) {
                 o.planes16[plane * o.pitch + pp] = static_cast<unsigned short>(h[j >> 1] >> (16 * (j & 1)));
