@@ -44,6 +44,7 @@ struct Sx3P {
     int HL;                        // rows staged before the tile (>= W + 1)
     int RQ;                        // rows of one expanded copy (multiple of 8)
     int raw_bytes;                 // bytes of one staging buffer
+    int nq;                        // sets of the three expanded copies: 2 (expansion of a stage overlaps the MMAs of the one before) where they fit, else 1
     int nimg;                      // slab mode: images staged per tile
     int mt_pad;                    // 128-channel tiles the weight images provide
     int total;                     // B * HP
@@ -51,7 +52,7 @@ struct Sx3P {
 };
 
 struct PipeS {
-    unsigned long long raw_full[2], qt_full, qt_empty, a_full[kNA], a_empty[kNA], acc;
+    unsigned long long raw_full[2], qt_full[2], qt_empty[2], a_full[kNA], a_empty[kNA], acc;
     unsigned tmem_base;
 };
 
@@ -131,7 +132,7 @@ __global__ void __launch_bounds__(kThreadsS) tc3_dx_shift_kernel(const Sx3P p) {
     unsigned char *a_s = smem;                              // kNA weight tiles
     unsigned char *qt = a_s + kNA * kTile;                  // three copies of [RQ rows][64 co]
     const unsigned copy_bytes = static_cast<unsigned>(p.RQ) * 128u;
-    unsigned char *raw_s = qt + 3 * copy_bytes;             // two staging buffers
+    unsigned char *raw_s = qt + p.nq * 3 * copy_bytes;      // two staging buffers
     __shared__ PipeS pipe;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -142,8 +143,7 @@ __global__ void __launch_bounds__(kThreadsS) tc3_dx_shift_kernel(const Sx3P p) {
     if (threadIdx.x == 0) {
         mbar_init(&pipe.raw_full[0], kX);
         mbar_init(&pipe.raw_full[1], kX);
-        mbar_init(&pipe.qt_full, kX);
-        mbar_init(&pipe.qt_empty, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(&pipe.qt_full[b], kX); mbar_init(&pipe.qt_empty[b], 1); }
         for (int s = 0; s < kNA; ++s) { mbar_init(&pipe.a_full[s], 1); mbar_init(&pipe.a_empty[s], 1); }
         mbar_init(&pipe.acc, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -232,7 +232,9 @@ __global__ void __launch_bounds__(kThreadsS) tc3_dx_shift_kernel(const Sx3P p) {
         if (nch > 1) issue_raw(1);
         for (int c = 0; c < nch; ++c) {
             ok = ok && mbar_wait(&pipe.raw_full[c & 1], (c >> 1) & 1, p.err_flag);
-            if (c > 0) ok = ok && mbar_wait(&pipe.qt_empty, (c - 1) & 1, p.err_flag);
+            const int qb = p.nq == 2 ? (c & 1) : 0, qu = p.nq == 2 ? (c >> 1) : c;   // copy set and its earlier uses
+            if (qu > 0) ok = ok && mbar_wait(&pipe.qt_empty[qb], (qu - 1) & 1, p.err_flag);
+            unsigned char *qtb = qt + qb * 3 * copy_bytes;
             const unsigned char *raw = raw_s + (c & 1) * p.raw_bytes;
 #pragma unroll
             for (int pass = 0; pass < 4; ++pass) {
@@ -247,13 +249,13 @@ __global__ void __launch_bounds__(kThreadsS) tc3_dx_shift_kernel(const Sx3P p) {
                     }
                     const uint4 z = make_uint4(0u, 0u, 0u, 0u);
                     const unsigned o = swz(r, ch);
-                    *reinterpret_cast<uint4 *>(qt + copy_bytes + o) = e;
-                    *reinterpret_cast<uint4 *>(qt + o) = ((zmask >> pass) & 1u) ? z : e;
-                    *reinterpret_cast<uint4 *>(qt + 2 * copy_bytes + o) = ((zmask >> (4 + pass)) & 1u) ? z : e;
+                    *reinterpret_cast<uint4 *>(qtb + copy_bytes + o) = e;
+                    *reinterpret_cast<uint4 *>(qtb + o) = ((zmask >> pass) & 1u) ? z : e;
+                    *reinterpret_cast<uint4 *>(qtb + 2 * copy_bytes + o) = ((zmask >> (4 + pass)) & 1u) ? z : e;
                 }
             }
             fence_async_proxy();
-            mbar_arrive(&pipe.qt_full);
+            mbar_arrive(&pipe.qt_full[qb]);
             if (c + 2 < nch) {
                 asm volatile("bar.sync 1, %0;" ::"n"(kX) : "memory");   // everyone is done with this buffer
                 issue_raw(c + 2);
@@ -281,13 +283,14 @@ __global__ void __launch_bounds__(kThreadsS) tc3_dx_shift_kernel(const Sx3P p) {
             bool ok = true;
             int ia = 0;
             for (int c = 0; c < nch && ok; ++c) {
-                ok = mbar_wait(&pipe.qt_full, c & 1, p.err_flag);
+                const int qb = p.nq == 2 ? (c & 1) : 0, qu = p.nq == 2 ? (c >> 1) : c;
+                ok = mbar_wait(&pipe.qt_full[qb], qu & 1, p.err_flag);
                 fence_async_proxy();
                 tc_fence_after();
                 for (int tap = 0; tap < 9 && ok; ++tap) {
                     const int ky = tap / 3, kx = tap - ky * 3;
                     const int row = p.HL + (1 - ky) * p.W + (1 - kx);          // source row of the tile's row 0
-                    const unsigned long long bd = make_desc(qt_addr + kx * copy_bytes + row * 128, 16, 1024);
+                    const unsigned long long bd = make_desc(qt_addr + (qb * 3 + kx) * copy_bytes + row * 128, 16, 1024);
                     for (int m = 0; m < MT && ok; ++m, ++ia) {
                         const int sa = ia % kNA;
                         ok = mbar_wait(&pipe.a_full[sa], (ia / kNA) & 1, p.err_flag);
@@ -299,7 +302,7 @@ __global__ void __launch_bounds__(kThreadsS) tc3_dx_shift_kernel(const Sx3P p) {
                         mma_commit(&pipe.a_empty[sa]);
                     }
                 }
-                mma_commit(&pipe.qt_empty);
+                mma_commit(&pipe.qt_empty[qb]);
             }
             mma_commit(&pipe.acc);
         }
@@ -410,8 +413,10 @@ int launch_tc3_dx_shift(dbp_ctx *ctx, const int8_t *codes, const void *W, const 
         if (cand <= mt_total && static_cast<long long>(tiles) * ((mt_total + cand - 1) / cand) >= ctx->sm_count) { mt = cand; break; }
     const int gy = (mt_total + mt - 1) / mt;
     p.mt_pad = gy * mt;
-    const size_t smem = static_cast<size_t>(kNA) * kTile + 3 * static_cast<size_t>(p.RQ) * 128 + 2 * static_cast<size_t>(p.raw_bytes) + 1024;
-    if (smem > 227 * 1024) return DBP_EUNSUPPORTED;
+    const size_t smem1 = static_cast<size_t>(kNA) * kTile + 3 * static_cast<size_t>(p.RQ) * 128 + 2 * static_cast<size_t>(p.raw_bytes) + 1024;
+    if (smem1 > 227 * 1024) return DBP_EUNSUPPORTED;
+    p.nq = (p.Cout > 64 && smem1 + 3 * static_cast<size_t>(p.RQ) * 128 <= 226 * 1024) ? 2 : 1;
+    const size_t smem = smem1 + (p.nq - 1) * 3 * static_cast<size_t>(p.RQ) * 128;
     const long long nchunks = static_cast<long long>(p.Cout / 64) * 9 * p.mt_pad * 1024;
     int rc = ws_reserve(ctx, ctx->w_taps, static_cast<size_t>(nchunks) * 16);
     if (rc) return rc;
