@@ -407,10 +407,17 @@ int launch_tc3_dx_shift(dbp_ctx *ctx, const int8_t *codes, const void *W, const 
     }
     const int mt_total = static_cast<int>((s.Cin + 127) / 128);
     const int tiles = (p.total + 127) / 128;
-    // several accumulators per CTA save expansions, but only while every SM still has a CTA
+    // several accumulators per CTA share one expansion of the codes. A CTA costs about one unit for
+    // the expansion and one per accumulator, and the grid runs in waves of one CTA per SM: take the
+    // count with the least waves x cost (ties: fewer accumulators, more CTAs)
     int mt = 1;
-    for (int cand = 4; cand > 1; cand >>= 1)
-        if (cand <= mt_total && static_cast<long long>(tiles) * ((mt_total + cand - 1) / cand) >= ctx->sm_count) { mt = cand; break; }
+    long long best = -1;
+    for (int cand = 1; cand <= 4; cand <<= 1) {
+        if (cand > 1 && cand > mt_total) break;
+        const long long ctas = static_cast<long long>(tiles) * ((mt_total + cand - 1) / cand);
+        const long long cost = ((ctas + ctx->sm_count - 1) / ctx->sm_count) * (1 + cand);
+        if (best < 0 || cost < best) { best = cost; mt = cand; }
+    }
     const int gy = (mt_total + mt - 1) / mt;
     p.mt_pad = gy * mt;
     const size_t smem1 = static_cast<size_t>(kNA) * kTile + 3 * static_cast<size_t>(p.RQ) * 128 + 2 * static_cast<size_t>(p.raw_bytes) + 1024;
