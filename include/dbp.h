@@ -104,9 +104,19 @@ int dbp_set_stream(dbp_ctx *ctx, void *cuda_stream);
 const char *dbp_status_string(int status);
 
 /* Synchronises the stream, then reports the device-side condition of the calls since the
- * previous report (DBP_OK, DBP_ENONFINITE or DBP_ESATURATED) and the number of clipped
- * codes; both outputs may be NULL. Clears the record. */
+ * previous report (DBP_OK, DBP_ETIMEOUT, DBP_ENONFINITE or DBP_ESATURATED, the first that
+ * applies) and the number of clipped codes; both outputs may be NULL. Clears the record. */
 int dbp_last_device_status(dbp_ctx *ctx, int *status, long long *saturated);
+
+/*
+ * Self-test of the bounded device-side waits (no counterpart in the paper). Every wait inside
+ * the tensor-core kernels gives up after a clock budget, records DBP_ETIMEOUT for
+ * dbp_last_device_status and lets the kernel return. This call enqueues a one-warp kernel that
+ * runs the same wait, with a budget of `cycles` SM clocks (0 ... 10^8), on a barrier nothing
+ * ever arrives on: afterwards dbp_last_device_status reports DBP_ETIMEOUT once and the context
+ * keeps working. It touches no product kernel and no caller data.
+ */
+int dbp_selftest_bounded_wait(dbp_ctx *ctx, long long cycles);
 
 /*
  * Per-kernel device timing (a measurement aid, off by default). While enabled, every kernel
@@ -153,6 +163,22 @@ int dbp_sparse_bytes(long long numel, size_t *bitmap_bytes, size_t *offsets_byte
  */
 int nsd_quantize(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
                  unsigned long long seed, float scale, const float *delta_in, dbp_sparse *out);
+
+/*
+ * Step size and non-zero count of the context's most recent quantization (the one inside the
+ * latest nsd_quantize or dithered_*_backward call): Algorithm 1's Delta and the nnz of
+ * Eq. (nsd)'s codes, for callers that passed no dbp_sparse. HOST outputs (either may be NULL);
+ * the call synchronises the context's stream.
+ */
+int dbp_last_step(dbp_ctx *ctx, float *delta_out, long long *nnz_out);
+
+/*
+ * Seed of layer `layer` (0-based, forward order) of a network whose backward pass was given
+ * `seed`: every layer draws its own dither (Eq. (qdz) quantizes each layer's delta_z
+ * independently), so layer l uses output l of the SplitMix64 sequence started at `seed`.
+ * Pure host function; no context needed.
+ */
+unsigned long long dbp_layer_seed(unsigned long long seed, int layer);
 
 /* Expands a dbp_sparse to one int8 code per element (codes: numel bytes, device). */
 int nsd_decode_dense(dbp_ctx *ctx, const dbp_sparse *q, int8_t *codes);
@@ -228,7 +254,7 @@ int dbp_maxpool2x2_backward(dbp_ctx *ctx, const float *g, const int8_t *argmax, 
  * at start-up and then frozen, a real-time loop that must not hit the implicit device
  * synchronisation of cudaMalloc/cudaFree, a plug-in that runs inside someone else's memory
  * budget. For them this call computes Delta = scale * std(delta) (Algorithm 1's first two
- * lines, same arithmetic and same result as nsd_quantize's step) with no context and no
+ * lines; it agrees with nsd_quantize's Delta within 1e-6 relative) with no context and no
  * allocation of any kind: the reduction's scratch is a fixed array of about 16 KB inside the
  * library image, present on every GPU that loads the library until the process exits.
  *

@@ -21,6 +21,7 @@ EXPORTED_SYMBOLS = [
     "dithered_linear_backward", "dithered_conv_backward", "dithered_linear_backward_host",
     "dithered_conv_backward_host", "dbp_relu_backward", "dbp_maxpool2x2_backward",
     "dbp_profile_enable", "dbp_profile_select", "dbp_profile_read", "dbp_set_crossover", "nsd_step_size_noalloc",
+    "dbp_last_step", "dbp_layer_seed", "dbp_selftest_bounded_wait",
 ]
 
 KERNEL_KINDS = ["statistics", "quantize", "weight_taps", "dx", "dw", "db", "decode", "glue",
@@ -81,11 +82,15 @@ def load_library():
     lib.dbp_profile_enable.argtypes = [vp, i32]
     lib.dbp_profile_select.argtypes = [vp, u32]
     lib.dbp_profile_read.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ll)]
+    lib.dbp_selftest_bounded_wait.argtypes = [vp, ll]
+    lib.dbp_last_step.argtypes = [vp, ctypes.POINTER(f32), ctypes.POINTER(ll)]
+    lib.dbp_layer_seed.argtypes = [ull, i32]
     lib.dbp_relu_backward.argtypes = [vp, vp, vp, vp, ll]
     lib.dbp_maxpool2x2_backward.argtypes = [vp, vp, vp, vp, ll, ll, ll]
     for name in EXPORTED_SYMBOLS:
-        if name != "dbp_status_string":
+        if name not in ("dbp_status_string", "dbp_layer_seed"):
             getattr(lib, name).restype = i32
+    lib.dbp_layer_seed.restype = ull
     _lib = lib
     return lib
 
@@ -143,6 +148,17 @@ class Context:
         _check(load_library().dbp_last_device_status(self._h, ctypes.byref(st), ctypes.byref(sat)),
                "dbp_last_device_status")
         return st.value, sat.value
+
+    def last_step(self):
+        """(Delta, nnz) of the most recent quantization on this context (synchronises)."""
+        d, n = ctypes.c_float(), ctypes.c_longlong()
+        _check(load_library().dbp_last_step(self._h, ctypes.byref(d), ctypes.byref(n)), "dbp_last_step")
+        return d.value, n.value
+
+    def selftest_bounded_wait(self, cycles: int = 100000):
+        """Enqueues the library's wait self-test: a wait that nothing satisfies runs out after
+        `cycles` SM clocks and the next last_device_status() reports DBP_ETIMEOUT."""
+        _check(load_library().dbp_selftest_bounded_wait(self._h, int(cycles)), "dbp_selftest_bounded_wait")
 
     def set_crossover(self, crossover: float):
         """Density above which layers the dense tensor-core path supports use it."""
@@ -326,20 +342,19 @@ def nsd_step_size_noalloc(delta: torch.Tensor, scale: float, out: torch.Tensor,
     _dev(delta, "delta"), _dev(out, "out")
     if out.dtype != torch.float32 or out.numel() < 1:
         raise ValueError("out must hold one float32")
-    s = stream if stream is not None else torch.cuda.current_stream()
-    _check(load_library().nsd_step_size_noalloc(
-        _ptr(delta), _dtype_code(delta), delta.numel() if numel is None else int(numel), float(scale),
-        _ptr(out), ctypes.c_void_p(s.cuda_stream)), "nsd_step_size_noalloc")
+    if out.device != delta.device:
+        raise ValueError("delta and out must live on the same GPU")
+    # the C call runs on the current device with that device's scratch array
+    with torch.cuda.device(delta.device):
+        s = stream if stream is not None else torch.cuda.current_stream()
+        _check(load_library().nsd_step_size_noalloc(
+            _ptr(delta), _dtype_code(delta), delta.numel() if numel is None else int(numel), float(scale),
+            _ptr(out), ctypes.c_void_p(s.cuda_stream)), "nsd_step_size_noalloc")
 
 
-def _splitmix64_output(seed: int, index: int) -> int:
-    """Seed bookkeeping only: layer l of a network uses output l of the SplitMix64 sequence
-    started at the network seed (an integer hash of two integers; no tensor arithmetic)."""
-    m = (1 << 64) - 1
-    z = (seed + (index + 1) * 0x9E3779B97F4A7C15) & m
-    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & m
-    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & m
-    return z ^ (z >> 31)
+def layer_seed(seed: int, layer: int) -> int:
+    """Seed of layer `layer` of a network whose backward pass was given `seed` (C: dbp_layer_seed)."""
+    return int(load_library().dbp_layer_seed(int(seed) & (2 ** 64 - 1), int(layer)))
 
 
 def network_backward(ctx: Context, kinds, Xs, Ws, relu_masks, pool_argmax, delta_out, scale: float,
@@ -357,7 +372,7 @@ def network_backward(ctx: Context, kinds, Xs, Ws, relu_masks, pool_argmax, delta
         q = SparseGradient(dz.numel(), ctx.device)
         fn = dithered_linear_backward if kinds[l] == "linear" else dithered_conv_backward
         need_dx = l > 0 or first_layer_dX
-        r = fn(ctx, dz, Xs[l], Ws[l], _splitmix64_output(int(seed), l), scale, q_out=q,
+        r = fn(ctx, dz, Xs[l], Ws[l], layer_seed(seed, l), scale, q_out=q,
                need_dX=need_dx)
         r.update(Delta=q.delta, nnz=q.nnz)
         if keep_delta_z:

@@ -311,6 +311,13 @@ int dbp_last_device_status(dbp_ctx *ctx, int *status, long long *saturated) {
     return DBP_OK;
 }
 
+int dbp_selftest_bounded_wait(dbp_ctx *ctx, long long cycles) {
+    if (!ctx || cycles < 0 || cycles > 100000000ll) return DBP_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DBP_ECUDA;
+    return launch_bounded_wait_selftest(ctx, cycles);
+}
+
 int dbp_profile_enable(dbp_ctx *ctx, int on) {
     if (!ctx) return DBP_EINVAL;
     ctx->profiling = on != 0;
@@ -374,6 +381,26 @@ int nsd_quantize(dbp_ctx *ctx, const void *delta, int dtype, long long numel, un
     KernelTimer t(ctx, DBP_K_QUANTIZE);
     return launch_quantize(ctx, delta, dtype, numel, seed, &ctx->state->delta, out->bitmap, out->offsets,
                            out->values, nullptr, reinterpret_cast<unsigned long long *>(out->nnz));
+}
+
+int dbp_last_step(dbp_ctx *ctx, float *delta_out, long long *nnz_out) {
+    if (!ctx) return DBP_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DBP_ECUDA;
+    DeviceState h;
+    if (cudaMemcpyAsync(&h, ctx->state, sizeof(h), cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess ||
+        cudaStreamSynchronize(ctx->stream) != cudaSuccess)
+        return DBP_ECUDA;
+    if (delta_out) *delta_out = h.delta;
+    if (nnz_out) *nnz_out = static_cast<long long>(h.nnz);
+    return DBP_OK;
+}
+
+unsigned long long dbp_layer_seed(unsigned long long seed, int layer) {
+    unsigned long long z = seed + (static_cast<unsigned long long>(layer) + 1ull) * 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
 }
 
 int nsd_decode_dense(dbp_ctx *ctx, const dbp_sparse *q, int8_t *codes) {

@@ -144,6 +144,9 @@ int launch_relu_backward(dbp_ctx *ctx, const float *da, const uint8_t *mask, flo
 int launch_maxpool_backward(dbp_ctx *ctx, const float *g, const int8_t *argmax, float *out,
                             long long planes, long long h, long long w);
 
+// ---- selftest.cu
+int launch_bounded_wait_selftest(dbp_ctx *ctx, long long budget);
+
 // Brackets one kernel launch with events while profiling is on.
 struct KernelTimer {
     dbp_ctx *ctx;

@@ -64,10 +64,13 @@ __device__ __forceinline__ double warp_sum(double v) {
 }
 
 // ---------------------------------------------------------------- statistics (sigma, Delta)
-// Sum and sum of squares of every element: fp32 inside one 128-bit chunk, fp64 across
-// chunks, per-block partials combined in a fixed order by the last block to finish, so the
-// step size does not depend on scheduling. sigma is the population standard deviation about
-// the mean; Delta = scale * sigma rounded once to fp32.
+// Sum and sum of squares of every element's distance from a pivot (the tensor's first element):
+// fp32 inside one 128-bit chunk, fp64 across chunks, per-block partials combined in a fixed order
+// by the last block to finish, so the step size does not depend on scheduling. The variance is
+// shift-invariant, and with the pivot inside the data's range the moments stay of the order of
+// sigma: a constant tensor gives exactly 0 and a mean far from 0 costs no accuracy (raw moments
+// would cancel). sigma is the population standard deviation about the mean; Delta = scale * sigma
+// rounded once to fp32.
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
 statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ partials,
@@ -78,6 +81,7 @@ statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ par
     chain_wait();
     chain_release();
     double d1 = 0.0, d2 = 0.0;
+    const float pivot = Elem<T>::one(x);
     const long long stride = static_cast<long long>(gridDim.x) * kThreads;
     // whole tiles of kUnroll x kThreads 128-bit vectors, a block at a time: kUnroll loads in flight
     // per thread, consecutive threads on consecutive vectors
@@ -93,8 +97,9 @@ statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ par
             float s1 = 0.f, s2 = 0.f;
 #pragma unroll
             for (int j = 0; j < EPT; ++j) {
-                s1 += v[u][j];
-                s2 = fmaf(v[u][j], v[u][j], s2);
+                const float c = v[u][j] - pivot;
+                s1 += c;
+                s2 = fmaf(c, c, s2);
             }
             d1 += static_cast<double>(s1);
             d2 += static_cast<double>(s2);
@@ -108,17 +113,18 @@ statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ par
         float s1 = 0.f, s2 = 0.f;
 #pragma unroll
         for (int j = 0; j < EPT; ++j) {
-            s1 += v[j];
-            s2 = fmaf(v[j], v[j], s2);
+            const float c = v[j] - pivot;
+            s1 += c;
+            s2 = fmaf(c, c, s2);
         }
         d1 += static_cast<double>(s1);
         d2 += static_cast<double>(s2);
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         for (long long i = nvec * EPT; i < n; ++i) {
-            const float v = Elem<T>::one(x + i);
-            d1 += static_cast<double>(v);
-            d2 += static_cast<double>(v) * static_cast<double>(v);
+            const double c = static_cast<double>(Elem<T>::one(x + i)) - static_cast<double>(pivot);
+            d1 += c;
+            d2 += c * c;
         }
     }
     __shared__ double sh1[kThreads / 32], sh2[kThreads / 32];

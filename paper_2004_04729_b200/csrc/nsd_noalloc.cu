@@ -58,8 +58,10 @@ __device__ __forceinline__ double warp_sum(double v) {
     return v;
 }
 
-// Same arithmetic as the library's statistics step: fp32 inside a 128-bit chunk, fp64 across
-// chunks, block partials combined in a fixed order by the last block to finish.
+// Same arithmetic as the library's statistics step: moments of the distance from a pivot (the
+// first element; the variance does not depend on it, and a constant tensor gives exactly 0), fp32
+// inside a 128-bit chunk, fp64 across chunks, block partials combined in a fixed order by the last
+// block to finish.
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
 step_size_kernel(const T *__restrict__ x, long long n, float scale, Scratch *__restrict__ sc,
@@ -67,6 +69,7 @@ step_size_kernel(const T *__restrict__ x, long long n, float scale, Scratch *__r
     constexpr int EPT = Load<T>::EPT;
     const long long nvec = n / EPT;
     double d1 = 0.0, d2 = 0.0;
+    const float pivot = Load<T>::one(x);
     const long long stride = static_cast<long long>(gridDim.x) * kThreads;
     for (long long i = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x; i < nvec; i += stride) {
         float v[EPT];
@@ -74,17 +77,18 @@ step_size_kernel(const T *__restrict__ x, long long n, float scale, Scratch *__r
         float s1 = 0.f, s2 = 0.f;
 #pragma unroll
         for (int j = 0; j < EPT; ++j) {
-            s1 += v[j];
-            s2 = fmaf(v[j], v[j], s2);
+            const float c = v[j] - pivot;
+            s1 += c;
+            s2 = fmaf(c, c, s2);
         }
         d1 += static_cast<double>(s1);
         d2 += static_cast<double>(s2);
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         for (long long i = nvec * EPT; i < n; ++i) {
-            const float v = Load<T>::one(x + i);
-            d1 += static_cast<double>(v);
-            d2 += static_cast<double>(v) * static_cast<double>(v);
+            const double c = static_cast<double>(Load<T>::one(x + i)) - static_cast<double>(pivot);
+            d1 += c;
+            d2 += c * c;
         }
     }
     __shared__ double sh1[kThreads / 32], sh2[kThreads / 32];

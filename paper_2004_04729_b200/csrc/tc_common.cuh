@@ -63,7 +63,8 @@ __device__ __forceinline__ bool mbar_test(unsigned addr, unsigned parity) {
         : "=r"(done) : "r"(addr), "r"(parity) : "memory");
     return done != 0;
 }
-__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity, int *err_flag) {
+__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity, int *err_flag,
+                                          long long budget = kWaitCycles) {
     const unsigned addr = smem_u32(bar);
     if (mbar_test(addr, parity)) return true;
     const long long t0 = clock64();
@@ -71,7 +72,7 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned pari
 #pragma unroll 1
         for (int i = 0; i < 64; ++i)
             if (mbar_test(addr, parity)) return true;
-    } while (clock64() - t0 <= kWaitCycles);
+    } while (clock64() - t0 <= budget);
     atomicExch(err_flag, 1);
     return false;
 }

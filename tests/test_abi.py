@@ -12,7 +12,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def _declared_functions():
     text = open(os.path.join(ROOT, "include", "dbp.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    names = re.findall(r"^\s*(?:const\s+char\s*\*\s*|int\s+)(\w+)\s*\(", text, flags=re.M)
+    names = re.findall(r"^\s*(?:const\s+char\s*\*\s*|unsigned\s+long\s+long\s+|int\s+)(\w+)\s*\(", text, flags=re.M)
     return sorted(set(names))
 
 
@@ -41,6 +41,10 @@ def test_host_side_argument_checks_need_no_gpu():
     assert lib.dbp_sparse_bytes(1025, ctypes.byref(b), ctypes.byref(o), ctypes.byref(v)) == 0
     assert (b.value, o.value, v.value) == (2 * 32 * 4, 2 * 32 * 2, 2048)
     assert lib.dbp_destroy(None) == -1
+    # per-layer seeds: output l of the SplitMix64 sequence started at the seed (published vector:
+    # the first outputs for seed 0)
+    assert lib.dbp_layer_seed(0, 0) == 0xE220A8397B1DCDAF
+    assert lib.dbp_layer_seed(0, 1) == 0x6E789E6AA1B965F4
     assert lib.nsd_quantize(None, None, 0, 10, 0, 2.0, None, None) == -1
     # unsupported kernel size is refused before anything touches the device
     assert lib.dithered_conv_backward(None, None, None, None, 0, 1, 1, 1, 4, 4, 5, 1, 2, 0, 2.0,

@@ -58,9 +58,42 @@ def test_config3_full_size(ctx):
     _full_size_case(ctx, wl.config3())           # B128, fp32: the sparse kernels
 
 
-@pytest.mark.parametrize("idx", [1, 2, 3, 9, 10, 11, 13, 14, 15])
+@pytest.mark.parametrize("idx", range(16))
 def test_config5_full_size_layers(ctx, idx):
-    _full_size_case(ctx, wl.config5_layer(idx))  # B64, bf16: the path bench.py times
+    _full_size_case(ctx, wl.config5_layer(idx))  # B64, bf16: every shape of the set bench.py times
+
+
+@pytest.mark.parametrize("idx", range(16))
+def test_config5_full_size_as_bench_calls_it(ctx, idx, nsamples=32):
+    """The call `bench.py` times: no sparse structure asked for (the product-path quantizer
+    runs instead of the compacting one), default flags, dX stored as bf16. Delta and nnz come
+    back through dbp_last_step; the codes never leave the library, so the oracle's codes (given
+    the CUDA path's Delta) stand behind every sampled gradient entry.
+    Bars: nnz exact; dW within 1e-5 sum|terms|; dX = one bf16 rounding (2^-8 relative) on top."""
+    import paper_2004_04729_b200 as dbp
+    L = wl.config5_layer(idx)
+    d, X, W = (torch.from_numpy(a).to(torch.bfloat16).cuda() for a in (L.delta, L.X, L.W))
+    out = dbp.dithered_conv_backward(ctx, d, X, W, L.seed, L.scale)
+    D, nnz_gpu = ctx.last_step()
+    assert ctx.last_device_status() == (0, 0)
+    D = np.float32(D)
+    D_ref = oracle.step_size(L.delta, L.scale)
+    assert abs(float(D) - float(D_ref)) <= 1e-6 * float(D_ref)
+    codes, nnz, _ = oracle.nsd_codes(L.delta, L.seed, D)
+    assert nnz_gpu == nnz
+    assert out["dX"].dtype == torch.bfloat16
+    dW, dX = out["dW"].cpu().numpy(), out["dX"].float().cpu().numpy()
+    r = np.random.default_rng(321 + idx)
+    B, Co, H, Wd = codes.shape
+    Ci = L.X.shape[1]
+    pos = [(r.integers(B), r.integers(H), r.integers(Wd)) for _ in range(nsamples)]
+    pos += [(0, 0, 0), (B - 1, H - 1, Wd - 1), (B // 2, 0, Wd - 1), (1, H - 1, 0)]
+    for (b, y, x) in pos:
+        co, ci, ky, kx = r.integers(Co), r.integers(Ci), r.integers(L.k), r.integers(L.k)
+        v, sa = oracle.conv_dW_entry(codes, D, L.X, co, ci, ky, kx, L.k)
+        assert abs(float(dW[co, ci, ky, kx]) - v) <= TOL * sa + 1e-30, ("dW", co, ci, ky, kx)
+        v, sa = oracle.conv_dX_entry(codes, D, L.W, b, ci, y, x)
+        assert abs(float(dX[b, ci, y, x]) - v) <= 2.0 ** -8 * abs(v) + TOL * sa + 1e-30, ("dX", b, ci, y, x)
 
 
 @pytest.mark.parametrize("idx", [3, 9, 13, 15])

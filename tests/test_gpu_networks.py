@@ -80,6 +80,52 @@ def test_config4_vgg16_reduced_batch(ctx):
     _run_chain(ctx, c)
 
 
+def test_config4_vgg16_full_batch_sampled(ctx):
+    """Config 4 at its stated batch of 128. The full fp64 products would take many minutes, so
+    per layer (teacher-forced as above) the codes are compared in full and the gradients on
+    sampled entries, each computed by the oracle from the defining sum."""
+    import paper_2004_04729_b200 as dbp
+    c = wl.vgg_chain(batch=128, device="cuda")       # the forward pass only makes inputs
+    cu = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    Xs, Ws = [cu(a) for a in c.X], [cu(a) for a in c.W]
+    masks = [None if m is None else cu(m.astype(np.uint8)) for m in c.relu_mask]
+    pools = [cu(a) for a in c.pool_argmax]
+    res = dbp.network_backward(ctx, c.kinds, Xs, Ws, masks, pools, cu(c.delta_out), c.scale, 0,
+                               keep_delta_z=True)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status()[0] == 0
+    r = np.random.default_rng(4)
+    for l in range(len(c.kinds) - 1, -1, -1):
+        dz = res[l]["delta_z"].cpu().numpy()
+        D = np.float32(res[l]["Delta"].item())
+        D_ref = oracle.step_size(dz, c.scale)
+        assert abs(float(D) - float(D_ref)) <= 1e-6 * float(D_ref), l
+        codes, nnz, _ = oracle.nsd_codes(dz, oracle.derive_layer_seed(0, l), D)
+        got = dbp.nsd_decode_dense(ctx, res[l]["q"]).cpu().numpy().reshape(dz.shape)
+        assert np.array_equal(got, codes) and res[l]["nnz"].item() == nnz, l
+        dW = res[l]["dW"].cpu().numpy()
+        dX = None if res[l]["dX"] is None else res[l]["dX"].cpu().numpy()
+        if c.kinds[l] == "linear":
+            o = oracle.linear_backward(codes, D, c.X[l], c.W[l], with_abs=True)
+            assert np.all(np.abs(dW - o["dW"]) <= TOL * o["S_dW"] + 1e-30)
+            assert np.all(np.abs(dX - o["dX"]) <= TOL * o["S_dX"] + 1e-30)
+            continue
+        B, Co, H, Wd = codes.shape
+        Ci = c.X[l].shape[1]
+        for _ in range(12):
+            co, ci, ky, kx = r.integers(Co), r.integers(Ci), r.integers(3), r.integers(3)
+            v, sa = oracle.conv_dW_entry(codes, D, c.X[l], co, ci, ky, kx, 3)
+            assert abs(float(dW[co, ci, ky, kx]) - v) <= TOL * sa + 1e-30, (l, "dW", co, ci, ky, kx)
+            if dX is not None:
+                b, y, x = r.integers(B), r.integers(H), r.integers(Wd)
+                v, sa = oracle.conv_dX_entry(codes, D, c.W[l], b, ci, y, x)
+                assert abs(float(dX[b, ci, y, x]) - v) <= TOL * sa + 1e-30, (l, "dX", b, ci, y, x)
+        if dX is not None:
+            for (b, y, x) in ((0, 0, 0), (B - 1, H - 1, Wd - 1), (B // 2, 0, Wd - 1)):
+                v, sa = oracle.conv_dX_entry(codes, D, c.W[l], b, Ci - 1, y, x)
+                assert abs(float(dX[b, Ci - 1, y, x]) - v) <= TOL * sa + 1e-30, (l, "dX corner")
+
+
 def test_small_conv_pool_chain_other_seed(ctx):
     c = wl.vgg_chain(batch=3, cfg=[8, "M", 16, 16, "M"], hw=8, data_seed=77)
     _run_chain(ctx, c, seed=5)

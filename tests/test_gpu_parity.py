@@ -133,6 +133,43 @@ def test_nsd_degenerate_inputs(ctx):
     assert ctx.last_device_status() == (-6, nsat)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_step_size_is_shift_invariant(ctx, dtype):
+    """Algorithm 1's std is about the mean: a constant tensor whose value is not a binary
+    fraction has sigma = 0 exactly (Delta = 0, every code 0), and a mean of 100 sigma must not
+    cost accuracy (raw moments sum(x^2)/n - mean^2 would cancel on both)."""
+    import paper_2004_04729_b200 as dbp
+    for n in (3000, 70001, 1 << 20):
+        c = torch.full((n,), 0.1, device="cuda")
+        c = c.to(torch.bfloat16) if dtype == "bf16" else c
+        q = dbp.nsd_quantize(ctx, c, 0, 2.0)
+        assert q.delta.item() == 0 and q.nnz.item() == 0
+        assert not dbp.nsd_decode_dense(ctx, q).any()
+    assert ctx.last_device_status() == (0, 0)
+    if dtype == "f32":
+        # a bf16 tensor with this offset would hold almost no information about sigma
+        for n, seed in ((70001, 5), (1 << 20, 6)):
+            lap = wl.laplace(seed, 1, n, 1e-3)
+            d = (lap + 100.0 * lap.std()).astype(np.float32)
+            _nsd_case(ctx, d, 2.0, seed=seed, check_structure=False)
+            out = torch.zeros(1, device="cuda")
+            dbp.nsd_step_size_noalloc(_t(d), 2.0, out)
+            ref = float(oracle.step_size(d, 2.0))
+            assert abs(out.item() - ref) <= REL_DELTA * ref
+
+
+def test_bounded_wait_runs_out_and_is_reported(ctx):
+    """A device-side wait that nothing satisfies gives up after its clock budget: the kernel
+    returns, the status word says DBP_ETIMEOUT once, and the context keeps working."""
+    import paper_2004_04729_b200 as dbp
+    assert ctx.last_device_status() == (0, 0)
+    ctx.selftest_bounded_wait(100000)
+    assert ctx.last_device_status()[0] == -8
+    assert ctx.last_device_status() == (0, 0)            # cleared by the read
+    L = wl.config1()
+    _nsd_case(ctx, L.delta, 2.0, 0)                      # the context is still usable
+
+
 def _compare(name, got, ref, S):
     got = got.double().cpu().numpy()
     err = np.abs(got - ref)

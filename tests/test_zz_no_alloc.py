@@ -4,7 +4,7 @@ Hosts that may not allocate device memory when they call the library -- a server
 memory was handed out at start-up, a real-time loop that cannot afford cudaMalloc's implicit
 synchronisation -- get Delta = s * std(delta) from a call that owns no context and uses a
 fixed scratch array inside the library. This file checks that call against the regular
-`nsd_quantize` entry point, twice in a row (the scratch array keeps the previous call's
+`nsd_quantize` entry point and against the CPU oracle's step size, twice in a row (the scratch array keeps the previous call's
 contents, so the second call is the one that would show stale state), for both storage types,
 and that a tensor beyond the stated limit is refused before anything runs.
 
@@ -13,6 +13,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -36,16 +37,20 @@ def test_noalloc_step_matches_regular_entry_point_twice():
     ]
     for d, scale in cases:
         want = _reference_step(ctx, d, scale)
+        # the oracle sees the values the kernel sees (bf16 widens exactly to fp32)
+        exact = float(oracle.step_size(d.float().cpu().numpy(), scale))
         for _ in range(2):                       # two calls in a row on the shared scratch
             out.fill_(-1.0)
             dbp.nsd_step_size_noalloc(d, scale, out)
             torch.cuda.synchronize()
             got = float(out.item())
             assert want > 0 and abs(got - want) <= 1e-6 * want, (got, want)
-    # all-zero input: sigma = 0 is not an error
-    dbp.nsd_step_size_noalloc(torch.zeros(4096, device="cuda"), 2.0, out)
-    torch.cuda.synchronize()
-    assert out.item() == 0.0
+            assert abs(got - exact) <= 1e-6 * exact, (got, exact)
+    # sigma = 0 is not an error: all-zero input, and a constant that is no binary fraction
+    for value in (0.0, 0.1):
+        dbp.nsd_step_size_noalloc(torch.full((4099,), value, device="cuda"), 2.0, out)
+        torch.cuda.synchronize()
+        assert out.item() == 0.0
     ctx.close()
 
 
