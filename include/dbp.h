@@ -102,6 +102,10 @@ int dbp_create(dbp_ctx **out, int device, void *cuda_stream);
 int dbp_destroy(dbp_ctx *ctx);
 int dbp_set_stream(dbp_ctx *ctx, void *cuda_stream);
 const char *dbp_status_string(int status);
+/* Text of the most recent DBP_ECUDA on the calling thread: which step failed and the CUDA
+ * runtime's message (empty if none yet). The pointer stays valid; the text changes with the next
+ * failure on this thread. */
+const char *dbp_last_error(void);
 
 /* Synchronises the stream, then reports the device-side condition of the calls since the
  * previous report (DBP_OK, DBP_ETIMEOUT, DBP_ENONFINITE or DBP_ESATURATED, the first that
@@ -143,6 +147,21 @@ typedef enum {
 int dbp_profile_enable(dbp_ctx *ctx, int on);
 int dbp_profile_select(dbp_ctx *ctx, unsigned kind_mask);
 int dbp_profile_read(dbp_ctx *ctx, int kind, double *milliseconds, long long *launches);
+
+/*
+ * Where the TMA-fed 3x3 kernels' issuing threads stood still (a measurement aid). Each of those
+ * kernels has one thread that issues MMAs and one or two that issue copies; every time one of them
+ * waits on a barrier the SM clocks it waited are added to a counter, summed over all CTAs:
+ *   [0] MMA thread waiting for a code tile        [1] MMA thread waiting for weights / activations
+ *   [2] MMA thread waiting for a free accumulator [3] code-copy thread waiting for a free buffer
+ *   [4] weight/activation-copy thread waiting for a free buffer
+ *   [5] dX: epilogue thread 0 waiting for an accumulator; dW: clocks its additions into dW took
+ *   [6] lifetime of the MMA thread                [7] CTAs that reported
+ * dbp_wait_stats synchronises the stream, copies the DBP_WAIT_SLOTS counters to `out` (host) and
+ * clears them when `reset` is non-zero.
+ */
+#define DBP_WAIT_SLOTS 8
+int dbp_wait_stats(dbp_ctx *ctx, unsigned long long *out, int reset);
 
 /* Bytes the caller must allocate for each array of a dbp_sparse over `numel` elements. */
 int dbp_sparse_bytes(long long numel, size_t *bitmap_bytes, size_t *offsets_bytes,

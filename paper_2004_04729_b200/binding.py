@@ -21,7 +21,7 @@ EXPORTED_SYMBOLS = [
     "dithered_linear_backward", "dithered_conv_backward", "dithered_linear_backward_host",
     "dithered_conv_backward_host", "dbp_relu_backward", "dbp_maxpool2x2_backward",
     "dbp_profile_enable", "dbp_profile_select", "dbp_profile_read", "dbp_set_crossover", "nsd_step_size_noalloc",
-    "dbp_last_step", "dbp_layer_seed", "dbp_selftest_bounded_wait",
+    "dbp_last_step", "dbp_layer_seed", "dbp_selftest_bounded_wait", "dbp_last_error", "dbp_wait_stats",
 ]
 
 KERNEL_KINDS = ["statistics", "quantize", "weight_taps", "dx", "dw", "db", "decode", "glue",
@@ -31,7 +31,8 @@ KERNEL_KINDS = ["statistics", "quantize", "weight_taps", "dx", "dw", "db", "deco
 class DbpError(RuntimeError):
     def __init__(self, status, where):
         self.status = status
-        super().__init__(f"{where}: {_status_string(status)} ({status})")
+        detail = load_library().dbp_last_error().decode() if status == -3 else ""
+        super().__init__(f"{where}: {_status_string(status)} ({status})" + (f" [{detail}]" if detail else ""))
 
 
 class _Sparse(ctypes.Structure):
@@ -83,14 +84,17 @@ def load_library():
     lib.dbp_profile_select.argtypes = [vp, u32]
     lib.dbp_profile_read.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ll)]
     lib.dbp_selftest_bounded_wait.argtypes = [vp, ll]
+    lib.dbp_wait_stats.argtypes = [vp, ctypes.POINTER(ull), i32]
     lib.dbp_last_step.argtypes = [vp, ctypes.POINTER(f32), ctypes.POINTER(ll)]
     lib.dbp_layer_seed.argtypes = [ull, i32]
     lib.dbp_relu_backward.argtypes = [vp, vp, vp, vp, ll]
     lib.dbp_maxpool2x2_backward.argtypes = [vp, vp, vp, vp, ll, ll, ll]
     for name in EXPORTED_SYMBOLS:
-        if name not in ("dbp_status_string", "dbp_layer_seed"):
+        if name not in ("dbp_status_string", "dbp_layer_seed", "dbp_last_error"):
             getattr(lib, name).restype = i32
     lib.dbp_layer_seed.restype = ull
+    lib.dbp_last_error.argtypes = []
+    lib.dbp_last_error.restype = ctypes.c_char_p
     _lib = lib
     return lib
 
@@ -159,6 +163,12 @@ class Context:
         """Enqueues the library's wait self-test: a wait that nothing satisfies runs out after
         `cycles` SM clocks and the next last_device_status() reports DBP_ETIMEOUT."""
         _check(load_library().dbp_selftest_bounded_wait(self._h, int(cycles)), "dbp_selftest_bounded_wait")
+
+    def wait_stats(self, reset: bool = True):
+        """SM clocks the 3x3 kernels' issuing threads spent waiting, by cause (see dbp_wait_stats)."""
+        out = (ctypes.c_ulonglong * 8)()
+        _check(load_library().dbp_wait_stats(self._h, out, int(reset)), "dbp_wait_stats")
+        return list(out)
 
     def set_crossover(self, crossover: float):
         """Density above which layers the dense tensor-core path supports use it."""

@@ -3,7 +3,18 @@
 
 #include "dbp_internal.cuh"
 
+#include <cstdio>
+
 namespace dbp {
+
+namespace {
+thread_local char g_last_error[192] = "";
+}
+
+int fail_cuda(const char *what, cudaError_t e) {
+    std::snprintf(g_last_error, sizeof(g_last_error), "%s: %s", what, cudaGetErrorString(e));
+    return DBP_ECUDA;
+}
 
 int ws_reserve(dbp_ctx *ctx, Workspace &w, size_t bytes) {
     if (bytes <= w.bytes) return DBP_OK;
@@ -46,7 +57,8 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
                           unsigned long long seed, float scale, const float *delta_in,
                           dbp_sparse *q_out, const float **delta_p, const int8_t **codes,
                           bool want8 = true, long long planes_hw = 0, long long planes_pitch = 0,
-                          const void **codes16 = nullptr) {
+                          const void **codes16 = nullptr, const ConvShape *nhwc = nullptr,
+                          const void **codes_nhwc = nullptr) {
     int rc = DBP_OK;
     dbp_sparse sp;
     sp.bitmap = nullptr; sp.offsets = nullptr; sp.values = nullptr; sp.delta = nullptr; sp.nnz = nullptr;
@@ -76,12 +88,24 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
             p16 = ctx->codes16.ptr;
             *codes16 = p16;
         }
+        void *pn = nullptr;
+        if (nhwc) {
+            if ((rc = ws_reserve(ctx, ctx->codes_nhwc, static_cast<size_t>(numel) * 2 + 1024))) return rc;
+            pn = ctx->codes_nhwc.ptr;
+            *codes_nhwc = pn;
+        }
         if (q_out) {
             rc = launch_quantize(ctx, delta, dtype, numel, seed, &ctx->state->delta, sp.bitmap, sp.offsets,
                                  sp.values, dense, reinterpret_cast<unsigned long long *>(sp.nnz));
             if (!rc && p16)
                 rc = launch_quantize_dense(ctx, delta, dtype, numel, seed, &ctx->state->delta, nullptr, p16,
                                            planes_hw, planes_pitch, false);
+            if (!rc && pn)
+                rc = launch_quantize_nhwc(ctx, delta, dtype, nhwc->B, nhwc->Cout, nhwc->H * nhwc->W, seed,
+                                          &ctx->state->delta, pn, nullptr, false);
+        } else if (pn) {
+            rc = launch_quantize_nhwc(ctx, delta, dtype, nhwc->B, nhwc->Cout, nhwc->H * nhwc->W, seed,
+                                      &ctx->state->delta, pn, want8 ? dense : nullptr, true);
         } else {
             rc = launch_quantize_dense(ctx, delta, dtype, numel, seed, &ctx->state->delta, want8 ? dense : nullptr,
                                        p16, planes_hw, planes_pitch, true);
@@ -105,7 +129,7 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     if ((dW && !X) || (dX && !W)) return DBP_EINVAL;
     if (!aligned16(delta) || !aligned16(X) || !aligned16(W) || !aligned16(dW) || !aligned16(dX)) return DBP_EINVAL;
     if ((flags & DBP_FORCE_SPARSE) && (flags & DBP_FORCE_DENSE)) return DBP_EINVAL;
-    const bool can_dense = tc_supported(s, io) || tc3_supported(s, io);
+    const bool can_dense = tc_supported(s, io) || tc3_supported(s, io) || tc3_tma_supported(s, io);
     if ((flags & DBP_FORCE_DENSE) && !can_dense) return DBP_EUNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DBP_ECUDA;
@@ -131,10 +155,13 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     const bool dx_tma = dense && dX && tma_dx_supported(s, io);
     const bool dw_tma = dense && dW && tma_dw_supported(s, io);
     const bool any_tma = dx_tma || dw_tma;
-    const bool need8 = !dense || db || (dX && !dx_tma) || (dW && !dw_tma);
-    const void *codes16 = nullptr;
+    // 3x3 layers: the TMA-fed kernels read the codes position-major
+    const bool t3 = dense && (dX || dW) && tc3_tma_supported(s, io);
+    const bool need8 = !dense || db || (!t3 && ((dX && !dx_tma) || (dW && !dw_tma)));
+    const void *codes16 = nullptr, *codes_n = nullptr;
     int rc = quantize_for_products(ctx, delta, io, numel, seed, scale, delta_in, q_out, &delta_p, &codes, need8,
-                                   s.H * s.W, any_tma ? tma_code_pitch(s) : 0, any_tma ? &codes16 : nullptr);
+                                   s.H * s.W, any_tma ? tma_code_pitch(s) : 0, any_tma ? &codes16 : nullptr,
+                                   t3 ? &s : nullptr, t3 ? &codes_n : nullptr);
     if (rc) return rc;
     if (!capturing && !ctx->nnz_pending && ctx->nnz_host && ctx->nnz_event) {
         ctx->nnz_host_numel = numel;
@@ -148,6 +175,7 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
             KernelTimer t(ctx, DBP_K_DX_DENSE);
             const bool dx_bf16 = (io == DBP_BF16) && !(flags & DBP_DX_F32);
             rc = dx_tma ? launch_tma_dx(ctx, codes16, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout)
+                 : t3   ? launch_tc3_tma_dx(ctx, codes_n, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout)
                  : s.k == 3 ? launch_tc3_dx(ctx, codes, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout)
                             : launch_tc_dx(ctx, codes, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout);
             if (rc) return rc;
@@ -157,6 +185,7 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
         if (dW) {
             KernelTimer t(ctx, DBP_K_DW_DENSE);
             rc = dw_tma ? launch_tma_dw(ctx, codes16, X, delta_p, s, dW, &ctx->state->tc_timeout)
+                 : t3   ? launch_tc3_tma_dw(ctx, codes_n, X, delta_p, s, dW, &ctx->state->tc_timeout)
                  : s.k == 3 ? launch_tc3_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout)
                             : launch_tc_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout);
             if (rc) return rc;
@@ -227,7 +256,9 @@ int dbp_create(dbp_ctx **out, int device, void *cuda_stream) {
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) == cudaSuccess) ctx->sm_count = prop.multiProcessorCount;
     ctx->partial_blocks = ctx->sm_count * 8;
-    if (cudaMalloc(&ctx->state, sizeof(DeviceState)) != cudaSuccess ||
+    if (cudaMalloc(&ctx->wait_stats, sizeof(unsigned long long) * DBP_WAIT_SLOTS) != cudaSuccess ||
+        cudaMemset(ctx->wait_stats, 0, sizeof(unsigned long long) * DBP_WAIT_SLOTS) != cudaSuccess ||
+        cudaMalloc(&ctx->state, sizeof(DeviceState)) != cudaSuccess ||
         cudaMalloc(&ctx->partials, sizeof(double) * 2 * ctx->partial_blocks) != cudaSuccess ||
         cudaMemset(ctx->state, 0, sizeof(DeviceState)) != cudaSuccess) {
         cudaGetLastError();
@@ -244,6 +275,8 @@ int dbp_create(dbp_ctx **out, int device, void *cuda_stream) {
     return DBP_OK;
 }
 
+const char *dbp_last_error(void) { return g_last_error; }
+
 int dbp_set_crossover(dbp_ctx *ctx, float crossover) {
     if (!ctx || crossover != crossover) return DBP_EINVAL;
     ctx->crossover = crossover;
@@ -254,7 +287,7 @@ int dbp_destroy(dbp_ctx *ctx) {
     if (!ctx) return DBP_EINVAL;
     DeviceGuard guard(ctx->device);
     cudaStreamSynchronize(ctx->stream);
-    Workspace *all[] = {&ctx->dense_codes, &ctx->codes16, &ctx->x_padded, &ctx->w_taps, &ctx->sp_bitmap, &ctx->sp_offsets, &ctx->sp_values,
+    Workspace *all[] = {&ctx->dense_codes, &ctx->codes16, &ctx->codes_nhwc, &ctx->dw_acc, &ctx->x_padded, &ctx->w_taps, &ctx->sp_bitmap, &ctx->sp_offsets, &ctx->sp_values,
                         &ctx->tc_partials};
     for (Workspace *w : all) if (w->ptr) cudaFree(w->ptr);
     for (Workspace &w : ctx->io) if (w.ptr) cudaFree(w.ptr);
@@ -266,6 +299,7 @@ int dbp_destroy(dbp_ctx *ctx) {
     if (ctx->ev_x_up) cudaEventDestroy(ctx->ev_x_up);
     if (ctx->ev_dx_done) cudaEventDestroy(ctx->ev_dx_done);
     if (ctx->state) cudaFree(ctx->state);
+    if (ctx->wait_stats) cudaFree(ctx->wait_stats);
     if (ctx->partials) cudaFree(ctx->partials);
     delete ctx;
     return DBP_OK;
@@ -302,6 +336,7 @@ int dbp_last_device_status(dbp_ctx *ctx, int *status, long long *saturated) {
     if (status)
         *status = h.tc_timeout ? DBP_ETIMEOUT : h.nonfinite ? DBP_ENONFINITE : (h.saturated ? DBP_ESATURATED : DBP_OK);
     if (saturated) *saturated = static_cast<long long>(h.saturated);
+    if (h.tc_timeout) ctx->dw_acc_clean = false;        // a kernel gave up half way: its scratch may hold partial sums
     if (h.nonfinite || h.saturated || h.tc_timeout) {
         if (cudaMemsetAsync(&ctx->state->nonfinite, 0, sizeof(int), ctx->stream) != cudaSuccess ||
             cudaMemsetAsync(&ctx->state->tc_timeout, 0, sizeof(int), ctx->stream) != cudaSuccess ||
@@ -316,6 +351,18 @@ int dbp_selftest_bounded_wait(dbp_ctx *ctx, long long cycles) {
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DBP_ECUDA;
     return launch_bounded_wait_selftest(ctx, cycles);
+}
+
+int dbp_wait_stats(dbp_ctx *ctx, unsigned long long *out, int reset) {
+    if (!ctx || !out) return DBP_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DBP_ECUDA;
+    if (cudaMemcpyAsync(out, ctx->wait_stats, sizeof(unsigned long long) * DBP_WAIT_SLOTS, cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess ||
+        cudaStreamSynchronize(ctx->stream) != cudaSuccess)
+        return fail_cuda("reading the wait counters");
+    if (reset && cudaMemsetAsync(ctx->wait_stats, 0, sizeof(unsigned long long) * DBP_WAIT_SLOTS, ctx->stream) != cudaSuccess)
+        return fail_cuda("clearing the wait counters");
+    return DBP_OK;
 }
 
 int dbp_profile_enable(dbp_ctx *ctx, int on) {

@@ -42,6 +42,7 @@ struct dbp_ctx {
     int sm_count = 148;
     dbp::DeviceState *state = nullptr;  // device
     double *partials = nullptr;         // device, statistics partial sums
+    unsigned long long *wait_stats = nullptr;   // device, DBP_WAIT_SLOTS counters of SM clocks spent waiting
     int partial_blocks = 0;
     dbp::Workspace dense_codes;         // int8 per element of delta
     dbp::Workspace x_padded;            // activations copied to 16-byte aligned planes
@@ -49,6 +50,9 @@ struct dbp_ctx {
     dbp::Workspace w_taps;              // fp32 weights as [Cout][k*k][Cin]
     dbp::Workspace sp_bitmap, sp_offsets, sp_values;  // internal dbp_sparse
     dbp::Workspace tc_partials;         // split-K partial blocks of the dense dW kernel
+    dbp::Workspace codes_nhwc;          // bf16 codes [B][position][Cout] for the TMA-fed 3x3 kernels
+    dbp::Workspace dw_acc;              // fp32 [tap][Cout][Cin] that the 3x3 dW CTAs add into; zero between calls
+    bool dw_acc_clean = false;
     dbp::Workspace io[8];               // staging for the *_host entry points
     // *_host entry points: X goes up and dX comes down on streams of their own, so that the two
     // directions of the host link work at the same time; the events order them against the
@@ -87,6 +91,10 @@ int launch_quantize(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
 int launch_quantize_dense(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
                           unsigned long long seed, const float *delta_p, int8_t *dense,
                           void *planes_bf16, long long hw, long long pitch, bool count);
+// position-major bf16 codes [B][HW][C] for the TMA-fed 3x3 kernels (and int8 codes in delta's order
+// when dense8 is not null)
+int launch_quantize_nhwc(dbp_ctx *ctx, const void *delta, int dtype, long long B, long long C, long long HW,
+                         unsigned long long seed, const float *delta_p, void *codes_nhwc, int8_t *dense8, bool count);
 int launch_decode(dbp_ctx *ctx, const uint32_t *bitmap, const uint16_t *offsets,
                   const int8_t *values, long long numel, int8_t *dense);
 
@@ -137,6 +145,12 @@ int launch_tc3_dw_shift(dbp_ctx *ctx, const int8_t *codes, const void *X, const 
                         int *err_flag, long long *nsplit);
 int launch_tc3_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *delta_p,
                   const ConvShape &s, float *dW, int *err_flag);
+// ---- tc3_tma_dx.cu / tc3_tma_dw.cu: 3x3 products with TMA-fed operands; codes as bf16 [B][H*W][Cout]
+bool tc3_tma_supported(const ConvShape &s, int io);
+int launch_tc3_tma_dx(dbp_ctx *ctx, const void *codes_nhwc, const void *W, const float *delta_p,
+                      const ConvShape &s, void *dX, bool dx_bf16, int *err_flag);
+int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, const float *delta_p,
+                      const ConvShape &s, float *dW, int *err_flag);
 int launch_bias_grad(dbp_ctx *ctx, const int8_t *codes, const float *delta_p, const ConvShape &s,
                      float *db);
 int launch_relu_backward(dbp_ctx *ctx, const float *da, const uint8_t *mask, float *dz,
@@ -188,7 +202,12 @@ inline long long choose_split(long long tiles, long long kunits, int sms, long l
     return best;
 }
 
-inline int cuda_ok(cudaError_t e) { return e == cudaSuccess ? DBP_OK : DBP_ECUDA; }
+// Records where a CUDA call failed and what the runtime said (read back with dbp_last_error);
+// returns DBP_ECUDA.
+int fail_cuda(const char *what, cudaError_t e);
+inline int fail_cuda(const char *what) { return fail_cuda(what, cudaGetLastError()); }
+
+inline int cuda_ok(cudaError_t e) { return e == cudaSuccess ? DBP_OK : fail_cuda("launch", e); }
 
 // Programmatic dependent launch: a kernel launched with launch_chained may become resident while
 // the kernel before it in the stream is still draining; it must call chain_wait() before it

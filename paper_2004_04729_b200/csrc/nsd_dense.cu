@@ -251,6 +251,155 @@ quantize_dense_kernel(const T *__restrict__ x, long long n, unsigned long long s
     }
 }
 
+
+// ---------------------------------------------------------------- position-major bf16 codes
+// The same codes, written as bf16 in the order [image][position][channel] (the 3x3 tensor-core
+// kernels read this form: a row of 64 channels of one position is 128 contiguous bytes, so a
+// rectangular patch of positions with its halo is one tiled copy and a tap of the filter is a row
+// offset inside it). delta_z itself is [image][channel][position], so a block transposes tiles of
+// 64 channels x 64 positions through shared memory: rows of the input are read along the
+// positions, rows of the output are written along the channels. The dither of an element is
+// still keyed on its index in delta_z's own order.
+constexpr int kTC = 64, kTP = 64;                 // channels x positions per tile
+constexpr int kTileBytes = kTP * kTC * 2;
+
+// shared-memory byte offset of (position p, channel c) inside a tile: 128-byte rows, the
+// 16-byte pieces of a row permuted by the row's group of eight
+__device__ __forceinline__ unsigned tile_off(int p, int c) {
+    return static_cast<unsigned>(p) * 128u + (((static_cast<unsigned>(c) >> 3) ^ ((static_cast<unsigned>(p) >> 3) & 7u)) << 4) +
+           ((static_cast<unsigned>(c) & 7u) << 1);
+}
+
+// one element by itself (planes whose size is odd: the pair that shares a draw may straddle two
+// vectors); same decision as codes_of
+__device__ __forceinline__ unsigned code_single(float x, long long e, unsigned long long seed, float inv, unsigned &sat) {
+    const unsigned long long r = mix64(seed + (static_cast<unsigned long long>(e >> 1) + 1ull) * kGamma);
+    const float u = dither((e & 1) ? static_cast<unsigned>(r >> 32) : static_cast<unsigned>(r));
+    const float t = __fmaf_rn(x, inv, u);
+    if (fabsf(t) <= 127.f) return __float_as_uint(__fadd_rd(t, 12582912.0f)) & 0xffu;
+    return careful_byte(x, inv, u, sat);
+}
+__device__ __forceinline__ unsigned short byte_to_bf16(unsigned b) {
+    const float f = static_cast<float>(static_cast<int>(static_cast<signed char>(b)));
+    return static_cast<unsigned short>(__float_as_uint(f) >> 16);
+}
+
+template <typename T, int V>
+struct TileLoad;
+template <>
+struct TileLoad<__nv_bfloat16, 8> {
+    __device__ static void ld(const __nv_bfloat16 *p, float (&v)[8]) { Vec<__nv_bfloat16>::load(p, v); }
+};
+template <>
+struct TileLoad<__nv_bfloat16, 4> {
+    __device__ static void ld(const __nv_bfloat16 *p, float (&v)[4]) {
+        const uint2 q = __ldg(reinterpret_cast<const uint2 *>(p));
+        v[0] = __uint_as_float(q.x << 16); v[1] = __uint_as_float(q.x & 0xffff0000u);
+        v[2] = __uint_as_float(q.y << 16); v[3] = __uint_as_float(q.y & 0xffff0000u);
+    }
+};
+template <>
+struct TileLoad<float, 4> {
+    __device__ static void ld(const float *p, float (&v)[4]) { Vec<float>::load(p, v); }
+};
+
+// V: elements per load (plane size % V == 0), or 1 for element-wise loads (any plane size)
+template <typename T, int V>
+__global__ void __launch_bounds__(kThreads)
+quantize_nhwc_kernel(const T *__restrict__ x, int B, int C, int HW, unsigned long long seed,
+                     const float *__restrict__ delta_p, unsigned short *__restrict__ out,
+                     int8_t *__restrict__ dense8, DeviceState *__restrict__ st, int count) {
+    __shared__ __align__(16) unsigned char tile[2][kTileBytes];
+    constexpr int VV = (V > 1) ? V : 4;               // vector length of the vector path
+    chain_wait();
+    chain_release();
+    const float delta = *delta_p;
+    const bool live = (delta > 0.f) && (delta < __int_as_float(0x7f800000));
+    const float inv = live ? __fdiv_rn(1.0f, delta) : 0.f;
+    const int ct = (C + kTC - 1) / kTC, pt = (HW + kTP - 1) / kTP;
+    const long long ntiles = static_cast<long long>(B) * ct * pt;
+    unsigned nnz = 0, sat = 0;
+    int buf = 0;
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, buf ^= 1) {
+        const int b = static_cast<int>(t / (ct * pt));
+        const int rem = static_cast<int>(t - static_cast<long long>(b) * ct * pt);
+        const int c0 = (rem / pt) * kTC, p0 = (rem % pt) * kTP;
+        unsigned char *tl = tile[buf];
+        if (V > 1) {
+            constexpr int VPR = kTP / VV;            // vectors per channel row of the tile
+#pragma unroll
+            for (int i = 0; i < (kTC * VPR) / kThreads; ++i) {
+                const int v = threadIdx.x + kThreads * i;
+                const int c = v / VPR, pv = (v % VPR) * VV;
+                unsigned pk[VV / 4] = {};
+                const bool in = c0 + c < C && p0 + pv < HW;       // HW % V == 0: whole vectors
+                const long long e0 = (static_cast<long long>(b) * C + c0 + c) * HW + p0 + pv;
+                if (in && live) {
+                    float a[VV];
+                    TileLoad<T, VV>::ld(x + e0, a);
+                    codes_of<VV>(a, e0, seed, inv, pk, sat);
+                }
+                if (in && dense8 != nullptr) {
+                    if (VV == 4) *reinterpret_cast<unsigned *>(dense8 + e0) = pk[0];
+                    else *reinterpret_cast<uint2 *>(dense8 + e0) = make_uint2(pk[0], pk[VV / 4 - 1]);
+                }
+#pragma unroll
+                for (int w = 0; w < VV / 4; ++w) {
+                    nnz += nonzero_bytes(pk[w]);
+                    unsigned lo, hi;
+                    bytes4_to_bf16(pk[w], lo, hi);
+                    const int pp = pv + 4 * w;
+                    *reinterpret_cast<unsigned short *>(tl + tile_off(pp, c)) = static_cast<unsigned short>(lo);
+                    *reinterpret_cast<unsigned short *>(tl + tile_off(pp + 1, c)) = static_cast<unsigned short>(lo >> 16);
+                    *reinterpret_cast<unsigned short *>(tl + tile_off(pp + 2, c)) = static_cast<unsigned short>(hi);
+                    *reinterpret_cast<unsigned short *>(tl + tile_off(pp + 3, c)) = static_cast<unsigned short>(hi >> 16);
+                }
+            }
+        } else {
+#pragma unroll 4
+            for (int i = 0; i < (kTC * kTP) / kThreads; ++i) {
+                const int id = threadIdx.x + kThreads * i;
+                const int c = id / kTP, pp = id % kTP;
+                unsigned q = 0;
+                const bool in = c0 + c < C && p0 + pp < HW;
+                const long long e = (static_cast<long long>(b) * C + c0 + c) * HW + p0 + pp;
+                if (in && live) q = code_single(Vec<T>::one(x + e), e, seed, inv, sat);
+                if (in && dense8 != nullptr) dense8[e] = static_cast<int8_t>(q);
+                nnz += q != 0u;
+                *reinterpret_cast<unsigned short *>(tl + tile_off(pp, c)) = byte_to_bf16(q);
+            }
+        }
+        __syncthreads();
+        // rows of 64 channels (128 bytes) of one position each; eight lanes per row
+#pragma unroll
+        for (int i = 0; i < (kTP * 8) / kThreads; ++i) {
+            const int v = threadIdx.x + kThreads * i;
+            const int pp = v >> 3, ch = v & 7;
+            if (p0 + pp < HW && c0 + ch * 8 < C)
+                *reinterpret_cast<uint4 *>(out + (static_cast<long long>(b) * HW + p0 + pp) * C + c0 + ch * 8) =
+                    *reinterpret_cast<const uint4 *>(tl + tile_off(pp, ch * 8));
+        }
+        // the other buffer is written next; this one again only after the next barrier
+    }
+    nnz = __reduce_add_sync(kFull, nnz);
+    sat = __reduce_add_sync(kFull, sat);
+    if ((threadIdx.x & 31) == 0 && count) {
+        if (nnz) atomicAdd(&st->nnz, static_cast<unsigned long long>(nnz));
+        if (sat) atomicAdd(&st->saturated, static_cast<unsigned long long>(sat));
+    }
+}
+
+template <typename T, int V>
+cudaError_t run_nhwc(dbp_ctx *ctx, const void *delta, int B, int C, int HW, unsigned long long seed, const float *delta_p,
+                     void *out, int8_t *dense8, bool count) {
+    const long long ntiles = static_cast<long long>(B) * ((C + kTC - 1) / kTC) * ((HW + kTP - 1) / kTP);
+    long long blocks = ntiles < static_cast<long long>(ctx->sm_count) * 6 ? ntiles : static_cast<long long>(ctx->sm_count) * 6;
+    if (blocks < 1) blocks = 1;
+    return launch_chained(quantize_nhwc_kernel<T, V>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
+                          static_cast<const T *>(delta), B, C, HW, seed, delta_p, static_cast<unsigned short *>(out), dense8,
+                          ctx->state, count ? 1 : 0);
+}
+
 }  // namespace
 
 int launch_quantize_dense(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
@@ -269,6 +418,23 @@ int launch_quantize_dense(dbp_ctx *ctx, const void *delta, int dtype, long long 
     else
         e = launch_chained(quantize_dense_kernel<__nv_bfloat16>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0,
                            ctx->stream, static_cast<const __nv_bfloat16 *>(delta), numel, seed, delta_p, out, ctx->state);
+    return cuda_ok(e);
+}
+
+// delta_z [B][C][HW] -> bf16 codes [B][HW][C] (C % 8 == 0) and, when dense8 is not null, int8 codes
+// in delta_z's order
+int launch_quantize_nhwc(dbp_ctx *ctx, const void *delta, int dtype, long long B, long long C, long long HW,
+                         unsigned long long seed, const float *delta_p, void *codes_nhwc, int8_t *dense8, bool count) {
+    if (C % 8 != 0 || B * C * HW >= (1ll << 40) || HW >= (1ll << 30)) return DBP_EUNSUPPORTED;
+    const int b = static_cast<int>(B), c = static_cast<int>(C), hw = static_cast<int>(HW);
+    cudaError_t e;
+    if (dtype == DBP_F32)
+        e = hw % 4 == 0 ? run_nhwc<float, 4>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count)
+                        : run_nhwc<float, 1>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count);
+    else
+        e = hw % 8 == 0   ? run_nhwc<__nv_bfloat16, 8>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count)
+            : hw % 4 == 0 ? run_nhwc<__nv_bfloat16, 4>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count)
+                          : run_nhwc<__nv_bfloat16, 1>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count);
     return cuda_ok(e);
 }
 

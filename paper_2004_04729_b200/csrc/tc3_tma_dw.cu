@@ -1,0 +1,443 @@
+// Weight gradient of 3x3 convolutions (stride 1, pad 1) on the tensor cores, both operands brought
+// in by tiled copies (Eq. (qdw), "analogous for convolutional layers"):
+//   dW[co][ci][ky][kx] = Delta * sum_(b,j) X[b][ci][j] * q[b][co][j - (ky-1) W - (kx-1)]
+// with j a position of the image (row-major), the code taken as zero outside the image and where
+// the column x - (kx-1) leaves the row.
+//
+// The reduction index is the position. The activations lie [b][ci][position], so 64 consecutive
+// positions of 128 input channels are one K-major tile (A, M = input channels). The quantizer has
+// written the codes position-major, [b][position][co] in bf16, so a run of positions of 64 output
+// channels is one MN-major panel (B, N = output channels), one 128-byte row per position, and a
+// tap is only a different start row of that panel (the 128-byte swizzle is a function of the
+// shared-memory address). The copy engine zero-fills the rows before the first and after the last
+// position of the image, which is the padding above and below. Left/right padding cannot be a row
+// offset: a CTA handles ONE kernel column kx, and one warp zeroes, in the freshly copied panel, the
+// rows of image column 0 (kx = 0) or W-1 (kx = 2) before the MMAs read it.
+//
+// Per CTA: a range of segments (runs of up to 512 positions of one image, with a halo of W+1 rows
+// on either side), an output tile of 128 input channels x 64 or 128 output channels, the three
+// taps ky of its kx as three accumulators in tensor memory. With 64 output channels the taps ky = 1
+// and ky = 0 share one MMA of N = 128: its second 64-column group starts W rows further on.
+// Warp 0 copies code panels, warp 1 activation tiles, warp 2 issues the MMAs, warp 3 zeroes the
+// masked rows, warps 4-7 stage the accumulators in shared memory and the copy engine adds them into a
+// zero-initialised fp32 scratch [tap][co][ci] (the reduction over CTAs; the order of the additions,
+// hence the last bits of dW, can differ from run to run). A second kernel scales by Delta, writes
+// dW[co][ci][ky][kx] and puts the zeros back. Every wait is bounded.
+#include "tc_common.cuh"
+
+namespace dbp {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kThreadsW3 = 8 * 32;
+constexpr int kXTile = 16384;             // [128 ci][64 positions] bf16
+constexpr int kXS = 2;                    // 64-position stages per activation slot (one hand-over)
+constexpr int kXSlot = kXS * kXTile;
+constexpr int kMaxNX = 6;
+
+struct Dw3T {
+    int Cin, Cout, W, HW;
+    int SEG;                      // positions per segment (multiple of 64)
+    int segs_per_img;
+    long long nseg, per_split;
+    int nsplit;
+    int ci_tiles, co_tiles;
+    int rows_box, nload;          // a panel is copied as nload boxes of rows_box rows
+    int panel_bytes;              // multiple of 1024
+    int nx;                       // activation slots in flight
+    int stage_chunks;             // 32-column chunks of the accumulators that fit the shared memory at once
+    int *err_flag;
+    unsigned long long *stats;    // wait counters (may be null)
+};
+
+struct PipeW3 {
+    unsigned long long x_full[kMaxNX], x_empty[kMaxNX], q_full[2], q_ready[2], q_empty[2], acc;
+    unsigned tmem_base;
+};
+
+// NP: 64-channel panels of the code operand (N = 64 NP output channels per tap)
+template <int NP>
+__global__ void __launch_bounds__(kThreadsW3, 1)
+tc3_tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_x,
+                  const __grid_constant__ CUtensorMap map_acc, const Dw3T p) {
+    constexpr int TCOLS = NP == 2 ? 512 : 256;
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    unsigned char *x_s = smem;                                   // nx activation slots
+    unsigned char *q_s = x_s + p.nx * kXSlot;                    // 2 buffers x NP panels
+    const int qbuf_bytes = NP * p.panel_bytes;
+    __shared__ PipeW3 pipe;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // work item: (output tile, kernel column, range of segments)
+    const int split = blockIdx.x % p.nsplit;
+    int rest = blockIdx.x / p.nsplit;
+    const int kx = rest % 3;
+    rest /= 3;
+    const int ci0 = (rest % p.ci_tiles) * 128;
+    const int co0 = (rest / p.ci_tiles) * 64 * NP;
+    const long long g0 = split * p.per_split;
+    const long long g1 = g0 + p.per_split < p.nseg ? g0 + p.per_split : p.nseg;
+    const int halo = p.W + 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMaxNX; ++s) { mbar_init(&pipe.x_full[s], 1); mbar_init(&pipe.x_empty[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&pipe.q_full[s], 1); mbar_init(&pipe.q_ready[s], 1); mbar_init(&pipe.q_empty[s], 1); }
+        mbar_init(&pipe.acc, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tma_prefetch_desc(&map_q);
+        tma_prefetch_desc(&map_x);
+        tma_prefetch_desc(&map_acc);
+    }
+    if (warp == 2) tmem_alloc(&pipe.tmem_base, TCOLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const unsigned tmem_base = pipe.tmem_base;
+    chain_wait();        // from here on the kernel reads what earlier kernels wrote
+    chain_release();
+
+    // segment g: image, first position, number of 64-position stages
+    auto seg_of = [&](long long g, int &b, int &u0, int &ns) {
+        b = static_cast<int>(g / p.segs_per_img);
+        u0 = static_cast<int>(g - static_cast<long long>(b) * p.segs_per_img) * p.SEG;
+        const int left = p.HW - u0;
+        ns = ((left < p.SEG ? left : p.SEG) + 63) >> 6;
+    };
+    // The activation stages of this CTA are consecutive 64-position blocks of consecutive images; a
+    // slot holds kXS consecutive blocks of one image. A new slot starts at the CTA's first stage, at
+    // the first block of an image, and after kXS stages (copy and MMA threads follow the same rule).
+
+    if (warp == 0) {
+        if (lane == 0) {
+            bool ok = true;
+            const unsigned tx = static_cast<unsigned>(NP * p.nload * p.rows_box * 128);
+            int sg = 0;
+            long long waited = 0;
+            for (long long g = g0; g < g1 && ok; ++g, ++sg) {
+                int b, u0, ns;
+                seg_of(g, b, u0, ns);
+                const int buf = sg & 1;
+                ok = mbar_wait_timed(&pipe.q_empty[buf], ((sg >> 1) & 1) ^ 1, p.err_flag, waited);
+                if (!ok) break;
+                unsigned char *dst = q_s + buf * qbuf_bytes;
+                mbar_expect_tx(&pipe.q_full[buf], tx);
+#pragma unroll
+                for (int pn = 0; pn < NP; ++pn)
+                    for (int l = 0; l < p.nload; ++l)
+                        tma_load_3d(dst + pn * p.panel_bytes + l * p.rows_box * 128, &map_q, co0 + 64 * pn,
+                                    u0 - halo + l * p.rows_box, b, &pipe.q_full[buf]);
+            }
+            report_wait(p.stats, 3, waited);
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            bool ok = true;
+            int s = 0, j = kXS;                    // j: stages already in the current slot
+            unsigned parity = 1;
+            long long waited = 0;
+            for (long long g = g0; g < g1 && ok; ++g) {
+                int b, u0, ns;
+                seg_of(g, b, u0, ns);
+                for (int k = 0; k < ns; ++k) {
+                    const int blk = (u0 >> 6) + k;
+                    if (j == kXS || blk == 0) {
+                        ok = mbar_wait_timed(&pipe.x_empty[s], parity, p.err_flag, waited);
+                        if (!ok) break;
+                        unsigned char *dst = x_s + s * kXSlot;
+                        mbar_expect_tx(&pipe.x_full[s], kXSlot);
+                        // positions past the image's end read as zero (a block past its end is all zero)
+#pragma unroll
+                        for (int i = 0; i < kXS; ++i)
+                            tma_load_3d(dst + i * kXTile, &map_x, (blk + i) * 64, ci0, b, &pipe.x_full[s]);
+                        if (++s == p.nx) { s = 0; parity ^= 1u; }
+                        j = 0;
+                    }
+                    ++j;
+                }
+            }
+            report_wait(p.stats, 4, waited);
+        }
+    } else if (warp == 2) {
+        {   // the whole warp runs the loop (uniform control flow and operands); one elected lane issues
+            // tap ky reads the panel from row (2 - ky) W + (2 - kx) on. NP == 2: one MMA of N = 128 per tap
+            // (accumulator columns 128 ky ...). NP == 1: the three taps share ONE MMA of N = 192 whose
+            // 64-column groups start W rows apart (columns 0-63: ky = 2, 64-127: ky = 1, 128-191: ky = 0):
+            // an MMA instruction takes about a hundred clocks to issue however narrow it is.
+            constexpr unsigned idesc128 = make_idesc(128, 128, false, true), idesc192 = make_idesc(128, 192, false, true);
+            const unsigned r0 = static_cast<unsigned>((2 * p.W + 2 - kx) * 8), r1 = static_cast<unsigned>((p.W + 2 - kx) * 8),
+                           r2 = static_cast<unsigned>((2 - kx) * 8);     // start rows in 16-byte units
+            bool ok = true;
+            int slot = -1, j = kXS, sg = 0;
+            unsigned xpar = 0;
+            unsigned acc_on = 0u;
+            long long wq = 0, wx = 0;
+            const long long born = clock64();
+            for (long long g = g0; g < g1 && ok; ++g, ++sg) {
+                int b, u0, ns;
+                seg_of(g, b, u0, ns);
+                const int buf = sg & 1;
+                ok = __all_sync(0xffffffffu, mbar_wait_timed(&pipe.q_ready[buf], (sg >> 1) & 1, p.err_flag, wq));
+                if (!ok) break;
+                tc_fence_after();
+                const unsigned q_addr = smem_u32(q_s + buf * qbuf_bytes);
+                const unsigned long long bA = NP == 2 ? make_desc(q_addr, p.panel_bytes, 1024) + r0
+                                                      : make_desc(q_addr, p.W * 128, 1024) + r2;
+                const unsigned long long bB = make_desc(q_addr, p.panel_bytes, 1024) + r1;     // NP == 2 only
+                const unsigned long long bC = make_desc(q_addr, p.panel_bytes, 1024) + r2;     // NP == 2 only
+                for (int k = 0; k < ns && ok; ++k) {
+                    const int blk = (u0 >> 6) + k;
+                    if (j == kXS || blk == 0) {
+                        if (slot >= 0 && elect_one()) mma_commit(&pipe.x_empty[slot]);
+                        if (++slot == p.nx) { slot = 0; xpar ^= 1u; }
+                        ok = __all_sync(0xffffffffu, mbar_wait_timed(&pipe.x_full[slot], xpar, p.err_flag, wx));
+                        if (!ok) break;
+                        tc_fence_after();
+                        j = 0;
+                    }
+                    // the last stage of an image may hold fewer than 64 positions: skip the 16-position
+                    // slices that are entirely zero fill
+                    const int left = p.HW - (u0 + 64 * k);
+                    const int nk = left >= 64 ? 4 : (left + 15) >> 4;
+                    const unsigned long long ad = make_desc(smem_u32(x_s + slot * kXSlot + j * kXTile), 16, 1024);
+                    const unsigned radv = static_cast<unsigned>(64 * k * 8);
+                    if (elect_one())
+                    for (int kk = 0; kk < nk; ++kk) {
+                        const unsigned adv = radv + kk * 128;                 // 16 rows = 2048 bytes
+                        if (NP == 2) {
+                            mma_bf16(tmem_base, ad + 2 * kk, bA + adv, idesc128, acc_on);
+                            mma_bf16(tmem_base + 128, ad + 2 * kk, bB + adv, idesc128, acc_on);
+                            mma_bf16(tmem_base + 256, ad + 2 * kk, bC + adv, idesc128, acc_on);
+                        } else {
+                            mma_bf16(tmem_base, ad + 2 * kk, bA + adv, idesc192, acc_on);
+                        }
+                        acc_on = 1u;
+                    }
+                    acc_on = 1u;
+                    ++j;
+                }
+                if (ok && elect_one()) mma_commit(&pipe.q_empty[buf]);
+            }
+            if (ok && slot >= 0 && elect_one()) mma_commit(&pipe.x_empty[slot]);
+            if (ok && g1 > g0 && elect_one()) mma_commit(&pipe.acc);
+            if (lane == 0) {
+                report_wait(p.stats, 0, wq);
+                report_wait(p.stats, 1, wx);
+                report_wait(p.stats, 6, clock64() - born);
+                report_wait(p.stats, 7, 1);
+            }
+        }
+    } else if (warp == 3) {
+        // masked rows: image column 0 for kx = 0, W-1 for kx = 2 (generic-proxy writes, then a proxy
+        // fence so that the tensor core sees them)
+        bool ok = true;
+        int sg = 0;
+        const int zc = kx == 0 ? 0 : p.W - 1;
+        const int rows_total = p.nload * p.rows_box;
+        for (long long g = g0; g < g1 && ok; ++g, ++sg) {
+            int b, u0, ns;
+            seg_of(g, b, u0, ns);
+            const int buf = sg & 1;
+            ok = mbar_wait(&pipe.q_full[buf], (sg >> 1) & 1, p.err_flag);
+            if (!ok) break;
+            if (kx != 1) {
+                unsigned char *qb = q_s + buf * qbuf_bytes;
+                const int i_lo = u0 - halo;                       // image position of panel row 0
+                // first image position >= max(i_lo, 0) in column zc
+                const int start = i_lo > 0 ? i_lo : 0;
+                int i = start + ((zc - start % p.W) + p.W) % p.W;
+                const int sub = lane >> 3, chunk = lane & 7;      // four rows x eight 16-byte pieces per pass
+                i += sub * p.W;
+                for (; i < p.HW && i - i_lo < rows_total; i += 4 * p.W) {
+                    const int r = i - i_lo;
+#pragma unroll
+                    for (int pn = 0; pn < NP; ++pn)
+                        *reinterpret_cast<uint4 *>(qb + pn * p.panel_bytes + r * 128 + chunk * 16) = make_uint4(0u, 0u, 0u, 0u);
+                }
+                fence_async_proxy();
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&pipe.q_ready[buf]);
+        }
+    } else {
+        // epilogue: TMEM lane = input channel, column = (tap, output channel). Every buffer of the
+        // pipeline is free by now, so the accumulators are staged there as plain fp32 rows
+        // [column][128 ci] and one thread hands them to the copy engine, which adds them into the
+        // scratch [tap][co][ci] (rows of 512 bytes, 32 columns per request).
+        const int q = warp & 3, et = threadIdx.x - 128;
+        bool ok = g1 > g0 && mbar_wait(&pipe.acc, 0, p.err_flag);
+        {   // the same decision in all 128 threads (they meet at barriers below)
+            unsigned r;
+            asm volatile(
+                "{\n\t.reg .pred p, q;\n\t"
+                "setp.ne.b32 p, %1, 0;\n\t"
+                "bar.red.and.pred q, 1, 128, p;\n\t"
+                "selp.b32 %0, 1, 0, q;\n\t}"
+                : "=r"(r) : "r"(ok ? 1u : 0u) : "memory");
+            ok = r != 0;
+        }
+        if (ok) {
+            tc_fence_after();
+            const long long t_epi = clock64();
+            constexpr int nchunks = (NP == 2 ? 384 : 192) / 32;
+            float *stg = reinterpret_cast<float *>(smem);
+            for (int c0 = 0; c0 < nchunks; c0 += p.stage_chunks) {
+                const int nb = nchunks - c0 < p.stage_chunks ? nchunks - c0 : p.stage_chunks;
+                for (int i = 0; i < nb; ++i) {
+                    unsigned v[32];
+                    tmem_ld32(tmem_base + (static_cast<unsigned>(q * 32) << 16) + (c0 + i) * 32, v);
+                    float *dst = stg + i * 4096 + q * 32 + lane;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) dst[j * 128] = __uint_as_float(v[j]);
+                }
+                fence_async_proxy();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (et == 0) {
+                    for (int i = 0; i < nb; ++i) {
+                        const int c = c0 + i;
+                        int ky, col0;                           // tap and first output channel of these 32 columns
+                        if (NP == 2) { ky = c >> 2; col0 = (c & 3) * 32; }     // columns 0-127: ky = 0, 128-255: ky = 1, ...
+                        else { ky = 2 - (c >> 1); col0 = (c & 1) * 32; }       // columns 0-63: ky = 2, 64-127: ky = 1, 128-191: ky = 0
+                        // columns past Cout hold exact zeros (their codes were zero fill): adding them is harmless
+                        tma_reduce_add_2d(&map_acc, ci0, (ky * 3 + kx) * p.Cout + co0 + col0, stg + i * 4096);
+                    }
+                    bulk_commit();
+                    bulk_wait_read_all();
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+            }
+            if (et == 0) report_wait(p.stats, 5, clock64() - t_epi);     // how long handing over the sums took
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 2) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, TCOLS);
+    }
+}
+
+// dW[co][ci][tap] = Delta * acc[tap][co][ci]; the scratch goes back to zero for the next call.
+// A block takes 256 consecutive (co, ci) pairs: nine coalesced reads, a transposition through shared
+// memory, and the 256 x 9 results leave as one contiguous run.
+__global__ void __launch_bounds__(256)
+tc3_dw_finish_kernel(float *__restrict__ acc, const float *__restrict__ delta_p, float *__restrict__ dW, long long pairs) {
+    __shared__ float t_s[256 * 9];
+    chain_wait();
+    chain_release();
+    const float delta = *delta_p;
+    for (long long i0 = blockIdx.x * 256ll; i0 < pairs; i0 += gridDim.x * 256ll) {
+        const long long i = i0 + threadIdx.x;
+        if (i < pairs) {
+#pragma unroll
+            for (int t = 0; t < 9; ++t) {
+                t_s[threadIdx.x * 9 + t] = __ldcg(acc + t * pairs + i) * delta;
+                __stcg(acc + t * pairs + i, 0.f);
+            }
+        }
+        __syncthreads();
+        const long long left = pairs - i0;
+        const int n = static_cast<int>(left < 256 ? left : 256) * 9;
+        for (int k = threadIdx.x; k < n; k += 256) dW[i0 * 9 + k] = t_s[k];
+        __syncthreads();
+    }
+}
+
+int round_up(int v, int m) { return (v + m - 1) / m * m; }
+
+}  // namespace
+
+// DBP_EUNSUPPORTED: the shape does not fit (the caller uses another kernel)
+int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, const float *delta_p,
+                      const ConvShape &s, float *dW, int *err_flag) {
+    if (!tc3_tma_supported(s, DBP_BF16)) return DBP_EUNSUPPORTED;
+    const long long HW = s.H * s.W;
+    Dw3T p{};
+    p.Cin = static_cast<int>(s.Cin); p.Cout = static_cast<int>(s.Cout); p.W = static_cast<int>(s.W); p.HW = static_cast<int>(HW);
+    p.err_flag = err_flag;
+    p.stats = ctx->wait_stats;
+    const int NP = s.Cout > 64 ? 2 : 1;
+    p.ci_tiles = static_cast<int>((s.Cin + 127) / 128);
+    p.co_tiles = static_cast<int>((s.Cout + 64 * NP - 1) / (64 * NP));
+    // the longest segment whose two code buffers fit beside at least three activation slots
+    const size_t budget = 227 * 1024 - 2048;
+    const int seg_cap = static_cast<int>(HW < 512 ? (HW + 63) / 64 * 64 : 512);
+    size_t smem = 0;
+    for (int seg = seg_cap; seg >= 64; seg -= 64) {
+        const int rows = seg + 2 * (p.W + 1);
+        const int nload = (rows + 255) / 256, rows_box = (rows + nload - 1) / nload;
+        const int panel = round_up(nload * rows_box * 128, 1024);
+        const size_t fixed = 2 * static_cast<size_t>(NP) * panel + 1024;
+        if (fixed + 3 * kXSlot > budget) continue;
+        p.SEG = seg; p.nload = nload; p.rows_box = rows_box; p.panel_bytes = panel;
+        p.nx = static_cast<int>((budget - fixed) / kXSlot);
+        if (p.nx > kMaxNX) p.nx = kMaxNX;
+        smem = fixed + static_cast<size_t>(p.nx) * kXSlot;
+        break;
+    }
+    if (smem == 0) return DBP_EUNSUPPORTED;
+    p.segs_per_img = (p.HW + p.SEG - 1) / p.SEG;
+    p.nseg = s.B * p.segs_per_img;
+    const long long tiles = static_cast<long long>(p.ci_tiles) * p.co_tiles * 3;
+    const long long nsplit = choose_split(tiles, p.nseg, ctx->sm_count, &p.per_split);
+    p.nsplit = static_cast<int>(nsplit);
+    if (tiles * nsplit >= (1ll << 31)) return DBP_EUNSUPPORTED;
+    // fp32 scratch [9][Cout][Cin]: zero whenever no call is in flight
+    const size_t pairs = static_cast<size_t>(s.Cout) * s.Cin;
+    const size_t had = ctx->dw_acc.bytes;
+    int rc = ws_reserve(ctx, ctx->dw_acc, pairs * 9 * sizeof(float));
+    if (rc) return rc;
+    if (ctx->dw_acc.bytes != had || !ctx->dw_acc_clean) {
+        if (cudaMemsetAsync(ctx->dw_acc.ptr, 0, ctx->dw_acc.bytes, ctx->stream) != cudaSuccess) return fail_cuda("clearing the dW scratch");
+        ctx->dw_acc_clean = true;
+    }
+    float *acc = static_cast<float *>(ctx->dw_acc.ptr);
+    p.stage_chunks = static_cast<int>((smem - 1024) / 16384);
+    // activations whose planes do not start on 16-byte boundaries are first copied to padded planes
+    const void *Xsrc = X;
+    long long xpitch = HW;
+    if (HW % 8 != 0) {
+        xpitch = (HW + 7) / 8 * 8;
+        if ((rc = ws_reserve(ctx, ctx->x_padded, static_cast<size_t>(s.B) * s.Cin * xpitch * 2))) return rc;
+        if ((rc = launch_pad_planes(ctx, X, ctx->x_padded.ptr, s.B * s.Cin, 1, static_cast<int>(HW), static_cast<int>(xpitch))))
+            return rc;
+        Xsrc = ctx->x_padded.ptr;
+    }
+    CUtensorMap map_q, map_x, map_acc;
+    {
+        const unsigned long long dims[2] = {static_cast<unsigned long long>(s.Cin), static_cast<unsigned long long>(s.Cout) * 9};
+        const unsigned long long str[1] = {static_cast<unsigned long long>(s.Cin) * 4};
+        const unsigned box[2] = {128, 32};
+        if (!encode_map_f32_rows(&map_acc, acc, 2, dims, str, box)) return fail_cuda("tensor map of the dW scratch");
+    }
+    {
+        const unsigned long long dims[3] = {static_cast<unsigned long long>(s.Cout), static_cast<unsigned long long>(HW),
+                                            static_cast<unsigned long long>(s.B)};
+        const unsigned long long str[2] = {static_cast<unsigned long long>(s.Cout) * 2,
+                                           static_cast<unsigned long long>(s.Cout) * 2 * HW};
+        const unsigned box[3] = {64, static_cast<unsigned>(p.rows_box), 1};
+        if (!encode_map_bf16(&map_q, codes_nhwc, 3, dims, str, box)) return fail_cuda("tensor map of the code panels");
+    }
+    {
+        const unsigned long long dims[3] = {static_cast<unsigned long long>(HW), static_cast<unsigned long long>(s.Cin),
+                                            static_cast<unsigned long long>(s.B)};
+        const unsigned long long str[2] = {static_cast<unsigned long long>(xpitch) * 2,
+                                           static_cast<unsigned long long>(xpitch) * 2 * s.Cin};
+        const unsigned box[3] = {64, 128, 1};
+        if (!encode_map_bf16(&map_x, Xsrc, 3, dims, str, box)) return fail_cuda("tensor map of the activations");
+    }
+    auto kern = NP == 2 ? tc3_tma_dw_kernel<2> : tc3_tma_dw_kernel<1>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
+        return fail_cuda("shared memory size");
+    if ((rc = cuda_ok(launch_chained(kern, dim3(static_cast<unsigned>(tiles * nsplit)), dim3(kThreadsW3), smem,
+                                     ctx->stream, map_q, map_x, map_acc, p))))
+        return rc;
+    long long blocks = (static_cast<long long>(pairs) + 255) / 256;
+    if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
+    return cuda_ok(launch_chained(tc3_dw_finish_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, ctx->stream, acc,
+                                  delta_p, dW, static_cast<long long>(pairs)));
+}
+
+}  // namespace dbp

@@ -76,6 +76,30 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned pari
     atomicExch(err_flag, 1);
     return false;
 }
+// The same wait, with the SM clocks it took added to `waited` (a measurement aid: the single
+// threads that issue copies and MMAs report where they stood still).
+__device__ __forceinline__ bool mbar_wait_timed(unsigned long long *bar, unsigned parity, int *err_flag, long long &waited) {
+    if (mbar_test(smem_u32(bar), parity)) return true;
+    const long long t0 = clock64();
+    const bool ok = mbar_wait(bar, parity, err_flag);
+    waited += clock64() - t0;
+    return ok;
+}
+__device__ __forceinline__ void report_wait(unsigned long long *stats, int slot, long long cycles) {
+    if (stats != nullptr && cycles > 0) atomicAdd(stats + slot, static_cast<unsigned long long>(cycles));
+}
+// One lane of a converged warp: lets a whole warp run a loop with warp-uniform control flow and
+// operands (so that descriptor arithmetic can stay in uniform registers) while a single thread
+// issues the copy, MMA or commit.
+__device__ __forceinline__ bool elect_one() {
+    unsigned pred;
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "elect.sync _|P, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, P;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -204,6 +228,21 @@ __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap *map) {
 // point is missing or rejects the description.
 bool encode_map_bf16(CUtensorMap *map, const void *base, int rank, const unsigned long long *dims,
                      const unsigned long long *strides_bytes, const unsigned *box);
+// Host: an fp32 tensor map without swizzle (a box lands / leaves as plain rows of box[0] floats);
+// used for reductions into global memory.
+bool encode_map_f32_rows(CUtensorMap *map, const void *base, int rank, const unsigned long long *dims,
+                         const unsigned long long *strides_bytes, const unsigned *box);
+
+// Adds a box of fp32 values in shared memory (plain rows) into global memory through the copy
+// engine: the additions happen at the L2 with whole-line requests. Elements outside the tensor are
+// skipped. The issuing thread closes a group after its reductions and waits until the engine has
+// read the shared memory before that memory is reused (or the CTA exits).
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap *map, int c0, int c1, const void *src) {
+    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(map), "r"(c0), "r"(c1), "r"(smem_u32(src)) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
 }  // namespace tc
 }  // namespace dbp

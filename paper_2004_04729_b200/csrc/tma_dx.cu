@@ -19,8 +19,9 @@ namespace dbp {
 
 namespace tc {
 
-bool encode_map_bf16(CUtensorMap *map, const void *base, int rank, const unsigned long long *dims,
-                     const unsigned long long *strides_bytes, const unsigned *box) {
+namespace {
+bool encode_map(CUtensorMap *map, CUtensorMapDataType type, CUtensorMapSwizzle swizzle, const void *base, int rank,
+                const unsigned long long *dims, const unsigned long long *strides_bytes, const unsigned *box) {
     typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -43,9 +44,20 @@ bool encode_map_bf16(CUtensorMap *map, const void *base, int rank, const unsigne
         es[i] = 1;
         if (i > 0) gstr[i - 1] = strides_bytes[i - 1];
     }
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, static_cast<cuuint32_t>(rank), const_cast<void *>(base), gdim,
-              gstr, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return fn(map, type, static_cast<cuuint32_t>(rank), const_cast<void *>(base), gdim, gstr, bx, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+}  // namespace
+
+bool encode_map_bf16(CUtensorMap *map, const void *base, int rank, const unsigned long long *dims,
+                     const unsigned long long *strides_bytes, const unsigned *box) {
+    return encode_map(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B, base, rank, dims, strides_bytes, box);
+}
+
+bool encode_map_f32_rows(CUtensorMap *map, const void *base, int rank, const unsigned long long *dims,
+                         const unsigned long long *strides_bytes, const unsigned *box) {
+    return encode_map(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, CU_TENSOR_MAP_SWIZZLE_NONE, base, rank, dims, strides_bytes, box);
 }
 
 }  // namespace tc
