@@ -50,7 +50,7 @@ typedef enum {
 #define DBP_FORCE_SPARSE 1u /* always use the sparse gather kernels */
 #define DBP_FORCE_DENSE  2u /* always use the dense tensor-core path; DBP_EUNSUPPORTED where it
                                does not exist (it covers bf16 linear, 1x1 and 3x3 layers whose channel
-                               counts are multiples of 8) */
+                               counts are multiples of 8; 3x3 images up to 62 wide) */
 #define DBP_DX_F32       4u /* with io = DBP_BF16: write dX as fp32 instead of bf16 */
 
 /*

@@ -58,7 +58,7 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
                           dbp_sparse *q_out, const float **delta_p, const int8_t **codes,
                           bool want8 = true, long long planes_hw = 0, long long planes_pitch = 0,
                           const void **codes16 = nullptr, const ConvShape *nhwc = nullptr,
-                          const void **codes_nhwc = nullptr) {
+                          const void **codes_nhwc = nullptr, void *zero = nullptr, size_t zero_bytes = 0) {
     int rc = DBP_OK;
     dbp_sparse sp;
     sp.bitmap = nullptr; sp.offsets = nullptr; sp.values = nullptr; sp.delta = nullptr; sp.nnz = nullptr;
@@ -74,7 +74,7 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
     {
         KernelTimer t(ctx, DBP_K_STATISTICS);
         rc = launch_statistics(ctx, delta, dtype, numel, scale, delta_in, sp.delta,
-                               reinterpret_cast<unsigned long long *>(sp.nnz));
+                               reinterpret_cast<unsigned long long *>(sp.nnz), zero, zero_bytes);
     }
     if (rc) return rc;
     {
@@ -129,7 +129,7 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     if ((dW && !X) || (dX && !W)) return DBP_EINVAL;
     if (!aligned16(delta) || !aligned16(X) || !aligned16(W) || !aligned16(dW) || !aligned16(dX)) return DBP_EINVAL;
     if ((flags & DBP_FORCE_SPARSE) && (flags & DBP_FORCE_DENSE)) return DBP_EINVAL;
-    const bool can_dense = tc_supported(s, io) || tc3_supported(s, io) || tc3_tma_supported(s, io);
+    const bool can_dense = tc_supported(s, io) || tc3_tma_supported(s, io);
     if ((flags & DBP_FORCE_DENSE) && !can_dense) return DBP_EUNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DBP_ECUDA;
@@ -161,7 +161,9 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     const void *codes16 = nullptr, *codes_n = nullptr;
     int rc = quantize_for_products(ctx, delta, io, numel, seed, scale, delta_in, q_out, &delta_p, &codes, need8,
                                    s.H * s.W, any_tma ? tma_code_pitch(s) : 0, any_tma ? &codes16 : nullptr,
-                                   t3 ? &s : nullptr, t3 ? &codes_n : nullptr);
+                                   t3 ? &s : nullptr, t3 ? &codes_n : nullptr,
+                                   // the TMA-fed 1x1 dW kernel adds its partial sums into dW: cleared by the statistics kernel
+                                   dw_tma ? dW : nullptr, dw_tma ? sizeof(float) * static_cast<size_t>(s.Cout) * s.Cin : 0);
     if (rc) return rc;
     if (!capturing && !ctx->nnz_pending && ctx->nnz_host && ctx->nnz_event) {
         ctx->nnz_host_numel = numel;
@@ -176,8 +178,7 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
             const bool dx_bf16 = (io == DBP_BF16) && !(flags & DBP_DX_F32);
             rc = dx_tma ? launch_tma_dx(ctx, codes16, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout)
                  : t3   ? launch_tc3_tma_dx(ctx, codes_n, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout)
-                 : s.k == 3 ? launch_tc3_dx(ctx, codes, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout)
-                            : launch_tc_dx(ctx, codes, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout);
+                        : launch_tc_dx(ctx, codes, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout);
             if (rc) return rc;
         }
         if (ctx->hook_after_dx && cudaEventRecord(ctx->hook_after_dx, ctx->stream) != cudaSuccess) return DBP_ECUDA;
@@ -186,8 +187,7 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
             KernelTimer t(ctx, DBP_K_DW_DENSE);
             rc = dw_tma ? launch_tma_dw(ctx, codes16, X, delta_p, s, dW, &ctx->state->tc_timeout)
                  : t3   ? launch_tc3_tma_dw(ctx, codes_n, X, delta_p, s, dW, &ctx->state->tc_timeout)
-                 : s.k == 3 ? launch_tc3_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout)
-                            : launch_tc_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout);
+                        : launch_tc_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout);
             if (rc) return rc;
         }
         if (db) {

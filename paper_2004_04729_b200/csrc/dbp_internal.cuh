@@ -79,8 +79,10 @@ namespace dbp {
 int ws_reserve(dbp_ctx *ctx, Workspace &w, size_t bytes);
 
 // ---- nsd_kernels.cu
+// zero / zero_bytes: a buffer (16-byte aligned, a multiple of 16 bytes) that the same kernel clears
 int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long numel, float scale,
-                      const float *delta_in, float *delta_out, unsigned long long *nnz_out);
+                      const float *delta_in, float *delta_out, unsigned long long *nnz_out,
+                      void *zero = nullptr, size_t zero_bytes = 0);
 int launch_quantize(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
                     unsigned long long seed, const float *delta_p, uint32_t *bitmap,
                     uint16_t *offsets, int8_t *values, int8_t *dense,
@@ -133,18 +135,6 @@ int launch_tma_dw(dbp_ctx *ctx, const void *codes_bf16, const void *X, const flo
 int launch_pad_planes(dbp_ctx *ctx, const void *in, void *out, long long planes, int H, int W, int Wp);
 // dW = Delta * sum of nsplit partial blocks of nw floats (nw % 4 == 0), fixed order
 int launch_dw_sum(dbp_ctx *ctx, const float *partials, int nsplit, long long nw, const float *delta_p, float *dW);
-// ---- tc_conv3x3.cu
-bool tc3_supported(const ConvShape &s, int io);
-// row-shift variant of the 3x3 dX product; DBP_EUNSUPPORTED when the shape does not fit it
-int launch_tc3_dx_shift(dbp_ctx *ctx, const int8_t *codes, const void *W, const float *delta_p,
-                        const ConvShape &s, void *dX, bool dx_bf16, int *err_flag);
-int launch_tc3_dx(dbp_ctx *ctx, const int8_t *codes, const void *W, const float *delta_p,
-                  const ConvShape &s, void *dX, bool dx_bf16, int *err_flag);
-// row-shift variant of the 3x3 dW product: fills ctx->tc_partials and reports the split count
-int launch_tc3_dw_shift(dbp_ctx *ctx, const int8_t *codes, const void *X, const ConvShape &s,
-                        int *err_flag, long long *nsplit);
-int launch_tc3_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *delta_p,
-                  const ConvShape &s, float *dW, int *err_flag);
 // ---- tc3_tma_dx.cu / tc3_tma_dw.cu: 3x3 products with TMA-fed operands; codes as bf16 [B][H*W][Cout]
 bool tc3_tma_supported(const ConvShape &s, int io);
 int launch_tc3_tma_dx(dbp_ctx *ctx, const void *codes_nhwc, const void *W, const float *delta_p,

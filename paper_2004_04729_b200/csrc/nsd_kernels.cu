@@ -75,11 +75,15 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads)
 statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ partials,
                   DeviceState *__restrict__ st, float scale, float *__restrict__ delta_out,
-                  unsigned long long *__restrict__ nnz_out) {
+                  unsigned long long *__restrict__ nnz_out, uint4 *__restrict__ zero_ptr, long long zero_n16) {
     constexpr int EPT = Elem<T>::EPT;
     const long long nvec = n / EPT;
     chain_wait();
     chain_release();
+    // side job for the layer's weight-gradient kernel, which adds its partial sums into dW: clear it
+    for (long long i = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x; i < zero_n16;
+         i += static_cast<long long>(gridDim.x) * kThreads)
+        zero_ptr[i] = make_uint4(0u, 0u, 0u, 0u);
     double d1 = 0.0, d2 = 0.0;
     const float pivot = Elem<T>::one(x);
     const long long stride = static_cast<long long>(gridDim.x) * kThreads;
@@ -382,8 +386,11 @@ decode_kernel(const uint32_t *__restrict__ bitmap, const uint16_t *__restrict__ 
 }  // namespace
 
 int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long numel, float scale,
-                      const float *delta_in, float *delta_out, unsigned long long *nnz_out) {
+                      const float *delta_in, float *delta_out, unsigned long long *nnz_out, void *zero, size_t zero_bytes) {
+    uint4 *zp = static_cast<uint4 *>(zero);
+    const long long zn = zero ? static_cast<long long>(zero_bytes / 16) : 0;
     if (!(scale > 0.f)) {
+        if (zero && cudaMemsetAsync(zero, 0, zero_bytes, ctx->stream) != cudaSuccess) return fail_cuda("clearing dW");
         set_step_kernel<<<1, 1, 0, ctx->stream>>>(delta_in, ctx->state, delta_out, nnz_out);
         return cuda_ok(cudaGetLastError());
     }
@@ -394,10 +401,10 @@ int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long nume
     cudaError_t e;
     if (dtype == DBP_F32)
         e = launch_chained(statistics_kernel<float>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
-                           static_cast<const float *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out);
+                           static_cast<const float *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out, zp, zn);
     else
         e = launch_chained(statistics_kernel<__nv_bfloat16>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
-                           static_cast<const __nv_bfloat16 *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out);
+                           static_cast<const __nv_bfloat16 *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out, zp, zn);
     return cuda_ok(e);
 }
 

@@ -233,7 +233,11 @@ bool encode_map_bf16(CUtensorMap *map, const void *base, int rank, const unsigne
 bool encode_map_f32_rows(CUtensorMap *map, const void *base, int rank, const unsigned long long *dims,
                          const unsigned long long *strides_bytes, const unsigned *box);
 
-// Adds a box of fp32 values in shared memory (plain rows) into global memory through the copy
+// The same with 128-byte swizzle: the box's innermost extent is 32 floats.
+bool encode_map_f32_sw128(CUtensorMap *map, const void *base, int rank, const unsigned long long *dims,
+                          const unsigned long long *strides_bytes, const unsigned *box);
+
+// Adds a box of fp32 values in shared memory (plain rows, or swizzled as the tensor map says) into global memory through the copy
 // engine: the additions happen at the L2 with whole-line requests. Elements outside the tensor are
 // skipped. The issuing thread closes a group after its reductions and waits until the engine has
 // read the shared memory before that memory is reused (or the CTA exits).
@@ -243,6 +247,8 @@ __device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap *map, int c0
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// all but the three most recent groups of this thread have been read
+__device__ __forceinline__ void bulk_wait_read_but3() { asm volatile("cp.async.bulk.wait_group.read 3;" ::: "memory"); }
 
 }  // namespace tc
 }  // namespace dbp

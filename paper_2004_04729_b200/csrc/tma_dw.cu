@@ -6,9 +6,10 @@
 //   A = codes [128 co][64 p]   (one or two of them: MA accumulators share the activation tile)
 //   B = X     [NT ci][64 p]
 // The reduction over (image, 64-position chunk) is split over CTAs; a CTA accumulates its share in
-// TMEM and writes one fp32 partial block [split][Cout][Cin]; a second kernel adds the blocks in
-// a fixed order and scales by Delta. Warp 0 issues the copies, warp 1 the MMAs, warps 2-5 drain
-// the accumulators at the end. Positions past the end of a plane read as zero.
+// TMEM, scales it by Delta and has the copy engine add it into dW, which the layer's statistics
+// kernel has cleared (the order of these additions, hence the last bits of dW, can differ from run
+// to run). Warp 0 issues the copies, warp 1 the MMAs, warps 2-5 drain the accumulators at the end.
+// Positions past the end of a plane read as zero.
 #include "tc_common.cuh"
 
 namespace dbp {
@@ -23,7 +24,7 @@ constexpr int kThreadsW = 192;
 constexpr int kStageW = 32 * 128;                // one warp's staged 32 x 32 fp32 block
 
 struct DwT {
-    float *partials;              // [nsplit][Cout][Cin]
+    const float *delta_p;
     int Cin, Cout, HW;
     int cpi;                      // 64-position chunks per image
     long long nchunks;            // B * cpi
@@ -40,7 +41,8 @@ struct PipeW {
 };
 
 __global__ void __launch_bounds__(kThreadsW, 1)
-tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_x, const DwT p) {
+tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_x,
+              const __grid_constant__ CUtensorMap map_dw, const DwT p) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ PipeW pipe;
@@ -65,6 +67,7 @@ tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         tma_prefetch_desc(&map_q);
         tma_prefetch_desc(&map_x);
+        tma_prefetch_desc(&map_dw);
     }
     if (warp == 1) tmem_alloc(&pipe.tmem_base, p.tmem_cols);
     tc_fence_before();
@@ -121,39 +124,42 @@ tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             if (ok) mma_commit(&pipe.acc_full);
         }
     } else {
-        // epilogue: TMEM lane = output channel, column = input channel. A warp's 32 x 32 block goes
-        // through a shared staging block (128-byte rows, 16-byte pieces XOR-swizzled by the row) so
-        // that the global stores are whole 128-byte rows of the partial block, four per instruction.
+        // epilogue: TMEM lane = output channel, column = input channel. A warp's 32 x 32 block is scaled by
+        // Delta and staged in shared memory as 128-byte rows (16-byte pieces XOR-swizzled by the row, the
+        // layout the tensor map describes), then one lane asks the copy engine to add it into dW. The
+        // operand ring is free by now: each warp cycles through four 4 KB blocks of it.
         const int q = warp & 3;
-        unsigned char *stage = smem + S * stage_bytes + (warp - 2) * kStageW;
+        unsigned char *stage0 = smem + (warp - 2) * 4 * kStageW;
         if (k1 > k0 && mbar_wait(&pipe.acc_full, 0, p.err_flag)) {
             tc_fence_after();
+            const float delta = *p.delta_p;
+            int n = 0;
             for (int a = 0; a < p.MA; ++a) {
                 const int co_w = co0 + a * 128 + q * 32;                 // first output channel of this warp
-                const int nrows = p.Cout - co_w < 32 ? p.Cout - co_w : 32;
-                float *blk = p.partials + (static_cast<long long>(split) * p.Cout + co_w) * p.Cin + ci0;
 #pragma unroll 1
-                for (int c0 = 0; c0 < p.NT; c0 += 32) {
+                for (int c0 = 0; c0 < p.NT; c0 += 32, ++n) {
+                    unsigned char *stage = stage0 + (n & 3) * kStageW;
+                    if (n >= 4) {                                          // the engine must have read the block's last use
+                        if (lane == 0) bulk_wait_read_but3();
+                        __syncwarp();
+                    }
                     unsigned v[32];
                     tmem_ld32(tmem_base + (static_cast<unsigned>(q * 32) << 16) + a * p.NTp + c0, v);
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        *reinterpret_cast<uint4 *>(stage + lane * 128 + ((j ^ (lane & 7)) << 4)) =
-                            make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                        *reinterpret_cast<float4 *>(stage + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                            make_float4(__uint_as_float(v[4 * j]) * delta, __uint_as_float(v[4 * j + 1]) * delta,
+                                        __uint_as_float(v[4 * j + 2]) * delta, __uint_as_float(v[4 * j + 3]) * delta);
+                    fence_async_proxy();
                     __syncwarp();
-                    const int ch = lane & 7;                              // my 16-byte piece: columns c0 + 4 ch ..
-                    if (c0 + 4 * ch < p.NT && ci0 + c0 + 4 * ch < p.Cin) {
-#pragma unroll
-                        for (int r0 = 0; r0 < 32; r0 += 4) {
-                            const int r = r0 + (lane >> 3);
-                            if (r < nrows)
-                                *reinterpret_cast<uint4 *>(blk + static_cast<long long>(r) * p.Cin + c0 + 4 * ch) =
-                                    *reinterpret_cast<const uint4 *>(stage + r * 128 + ((ch ^ (r & 7)) << 4));
-                        }
+                    // rows past Cout and columns past Cin are skipped by the engine
+                    if (lane == 0) {
+                        if (co_w < p.Cout && ci0 + c0 < p.Cin) tma_reduce_add_2d(&map_dw, ci0 + c0, co_w, stage);
+                        bulk_commit();                 // a group per block, issued or not: the wait above counts groups
                     }
-                    __syncwarp();
                 }
             }
+            if (lane == 0) bulk_wait_read_all();
         }
     }
     tc_fence_before();
@@ -193,10 +199,8 @@ int launch_tma_dw(dbp_ctx *ctx, const void *codes_bf16, const void *X, const flo
     p.nsplit = static_cast<int>(nsplit);
     p.per_split = per;
     p.err_flag = err_flag;
-    const size_t nw = static_cast<size_t>(s.Cout) * s.Cin;
-    int rc = ws_reserve(ctx, ctx->tc_partials, nw * sizeof(float) * nsplit);
-    if (rc) return rc;
-    p.partials = static_cast<float *>(ctx->tc_partials.ptr);
+    p.delta_p = delta_p;
+    int rc = DBP_OK;
     // activations whose planes do not start on 16-byte boundaries are first copied to padded planes
     const void *Xsrc = X;
     long long xpitch = HW;
@@ -207,7 +211,13 @@ int launch_tma_dw(dbp_ctx *ctx, const void *codes_bf16, const void *X, const flo
             return rc;
         Xsrc = ctx->x_padded.ptr;
     }
-    CUtensorMap map_q, map_x;
+    CUtensorMap map_q, map_x, map_dw;
+    {
+        const unsigned long long dims[2] = {static_cast<unsigned long long>(s.Cin), static_cast<unsigned long long>(s.Cout)};
+        const unsigned long long str[1] = {static_cast<unsigned long long>(s.Cin) * 4};
+        const unsigned box[2] = {32, 32};
+        if (!encode_map_f32_sw128(&map_dw, dW, 2, dims, str, box)) return fail_cuda("tensor map of dW");
+    }
     {
         const unsigned long long dims[3] = {static_cast<unsigned long long>(HW), static_cast<unsigned long long>(s.Cout),
                                             static_cast<unsigned long long>(s.B)};
@@ -224,13 +234,12 @@ int launch_tma_dw(dbp_ctx *ctx, const void *codes_bf16, const void *X, const flo
         const unsigned box[3] = {64, static_cast<unsigned>(p.NT), 1};
         if (!encode_map_bf16(&map_x, Xsrc, 3, dims, str, box)) return DBP_ECUDA;
     }
-    const size_t smem = static_cast<size_t>(p.stages) * (p.MA * kATile + kBMax) + 4 * kStageW + 1024;
+    const size_t smem = static_cast<size_t>(p.stages) * (p.MA * kATile + kBMax) + 1024;       // >= 4 warps x 4 staging blocks
     if (cudaFuncSetAttribute(tma_dw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
         return DBP_ECUDA;
-    if ((rc = cuda_ok(launch_chained(tma_dw_kernel, dim3(static_cast<unsigned>(tiles * nsplit)), dim3(kThreadsW), smem,
-                                     ctx->stream, map_q, map_x, p))))
-        return rc;
-    return launch_dw_sum(ctx, p.partials, p.nsplit, static_cast<long long>(nw), delta_p, dW);
+    // dW has been cleared by this layer's statistics kernel
+    return cuda_ok(launch_chained(tma_dw_kernel, dim3(static_cast<unsigned>(tiles * nsplit)), dim3(kThreadsW), smem,
+                                  ctx->stream, map_q, map_x, map_dw, p));
 }
 
 }  // namespace dbp

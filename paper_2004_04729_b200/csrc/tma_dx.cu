@@ -55,6 +55,11 @@ bool encode_map_bf16(CUtensorMap *map, const void *base, int rank, const unsigne
     return encode_map(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B, base, rank, dims, strides_bytes, box);
 }
 
+bool encode_map_f32_sw128(CUtensorMap *map, const void *base, int rank, const unsigned long long *dims,
+                          const unsigned long long *strides_bytes, const unsigned *box) {
+    return encode_map(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, CU_TENSOR_MAP_SWIZZLE_128B, base, rank, dims, strides_bytes, box);
+}
+
 bool encode_map_f32_rows(CUtensorMap *map, const void *base, int rank, const unsigned long long *dims,
                          const unsigned long long *strides_bytes, const unsigned *box) {
     return encode_map(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, CU_TENSOR_MAP_SWIZZLE_NONE, base, rank, dims, strides_bytes, box);
