@@ -33,6 +33,7 @@ struct DwT {
     int NT, NTp, MA, stages;      // ci tile, its accumulator stride (multiple of 32), accumulators
     int tmem_cols;
     int *err_flag;
+    unsigned long long *stats;    // wait counters (may be null)
 };
 
 struct PipeW {
@@ -84,8 +85,9 @@ tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             long long b = k0 / p.cpi;
             int c = static_cast<int>(k0 - b * p.cpi);
             const unsigned bytes = static_cast<unsigned>(p.MA * kATile + p.NT * 128);
+            long long waited = 0;
             for (long long k = k0; k < k1; ++k) {
-                if (!mbar_wait(&pipe.empty[s], parity, p.err_flag)) break;
+                if (!mbar_wait_timed(&pipe.empty[s], parity, p.err_flag, waited)) break;
                 unsigned char *st = smem + s * stage_bytes;
                 mbar_expect_tx(&pipe.full[s], bytes);
                 for (int a = 0; a < p.MA; ++a)
@@ -94,16 +96,19 @@ tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 if (++c == p.cpi) { c = 0; ++b; }
                 if (++s == S) { s = 0; parity ^= 1u; }
             }
+            report_wait(p.stats, 3, waited);
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        {   // the whole warp runs the loop (uniform control flow and operands); one elected lane issues
             const unsigned idesc = make_idesc(128, p.NT, false, false);
             int s = 0;
             unsigned parity = 0;
             bool ok = true;
             int c = static_cast<int>(k0 % p.cpi);
+            long long wf = 0;
+            const long long born = clock64();
             for (long long k = k0; k < k1; ++k) {
-                ok = mbar_wait(&pipe.full[s], parity, p.err_flag);
+                ok = __all_sync(0xffffffffu, mbar_wait_timed(&pipe.full[s], parity, p.err_flag, wf));
                 if (!ok) break;
                 tc_fence_after();
                 // the last chunk of a plane may hold fewer than 64 positions: skip the 16-position
@@ -112,16 +117,23 @@ tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 const int nk = (valid + 15) >> 4;
                 const unsigned a_addr = smem_u32(smem + s * stage_bytes);
                 const unsigned long long bd = make_desc(a_addr + p.MA * kATile, 16, 1024);
-                for (int a = 0; a < p.MA; ++a) {
-                    const unsigned long long ad = make_desc(a_addr + a * kATile, 16, 1024);
-                    for (int kk = 0; kk < nk; ++kk)       // 16 positions = 32 bytes further per MMA
-                        mma_bf16(tmem_base + a * p.NTp, ad + 2 * kk, bd + 2 * kk, idesc, (k > k0 || kk > 0) ? 1u : 0u);
+                if (elect_one()) {
+                    for (int a = 0; a < p.MA; ++a) {
+                        const unsigned long long ad = make_desc(a_addr + a * kATile, 16, 1024);
+                        for (int kk = 0; kk < nk; ++kk)       // 16 positions = 32 bytes further per MMA
+                            mma_bf16(tmem_base + a * p.NTp, ad + 2 * kk, bd + 2 * kk, idesc, (k > k0 || kk > 0) ? 1u : 0u);
+                    }
+                    mma_commit(&pipe.empty[s]);
                 }
-                mma_commit(&pipe.empty[s]);
                 if (++c == p.cpi) c = 0;
                 if (++s == S) { s = 0; parity ^= 1u; }
             }
-            if (ok) mma_commit(&pipe.acc_full);
+            if (ok && elect_one()) mma_commit(&pipe.acc_full);
+            if (lane == 0) {
+                report_wait(p.stats, 1, wf);
+                report_wait(p.stats, 6, clock64() - born);
+                report_wait(p.stats, 7, 1);
+            }
         }
     } else {
         // epilogue: TMEM lane = output channel, column = input channel. A warp's 32 x 32 block is scaled by
@@ -132,6 +144,7 @@ tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         unsigned char *stage0 = smem + (warp - 2) * 4 * kStageW;
         if (k1 > k0 && mbar_wait(&pipe.acc_full, 0, p.err_flag)) {
             tc_fence_after();
+            const long long t_epi = clock64();
             const float delta = *p.delta_p;
             int n = 0;
             for (int a = 0; a < p.MA; ++a) {
@@ -160,6 +173,7 @@ tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 }
             }
             if (lane == 0) bulk_wait_read_all();
+            if (threadIdx.x == 64) report_wait(p.stats, 5, clock64() - t_epi);
         }
     }
     tc_fence_before();
@@ -199,6 +213,7 @@ int launch_tma_dw(dbp_ctx *ctx, const void *codes_bf16, const void *X, const flo
     p.nsplit = static_cast<int>(nsplit);
     p.per_split = per;
     p.err_flag = err_flag;
+    p.stats = ctx->wait_stats;
     p.delta_p = delta_p;
     int rc = DBP_OK;
     // activations whose planes do not start on 16-byte boundaries are first copied to padded planes

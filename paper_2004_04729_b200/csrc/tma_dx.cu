@@ -94,6 +94,7 @@ struct DxT {
     int MA;                       // accumulators per tile: 1 (128 channels, two tiles in flight) or 2 (256 channels)
     long long ntiles;
     int *err_flag;
+    unsigned long long *stats;    // wait counters (may be null)
 };
 
 struct PipeT {
@@ -137,64 +138,82 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
     chain_release();
 
     if (warp == 0) {
-        if (lane == 0) {
+        {   // the whole warp runs the loop (uniform control flow and operands); one elected lane issues
             int s = 0;
             unsigned parity = 1;                 // a fresh barrier passes a wait on the previous phase
             bool ok = true;
+            long long waited = 0;
             for (long long t = blockIdx.x; t < p.ntiles && ok; t += gridDim.x) {
                 const int ci0 = static_cast<int>(t % p.ci_tiles) * 128 * MA;
                 const long long g0 = (t / p.ci_tiles) * p.nct;
                 const int nch = static_cast<int>(p.nchunks - g0 < p.nct ? p.nchunks - g0 : p.nct);
-                int cb[kNChunks], cp[kNChunks];
-                for (int c = 0; c < nch; ++c) {
-                    cb[c] = static_cast<int>((g0 + c) / p.chunks_per_img);
-                    cp[c] = static_cast<int>((g0 + c) % p.chunks_per_img) * 64;
-                }
+                // the tile's chunks are consecutive: image and position of the first, then step and wrap
+                const int b0 = static_cast<int>(g0 / p.chunks_per_img);
+                const int c0 = static_cast<int>(g0 - static_cast<long long>(b0) * p.chunks_per_img);
+                const unsigned tx = static_cast<unsigned>((2 * MA + nch) * kPanel);
                 for (int ks = 0; ks < p.ksteps && ok; ++ks) {
-                    ok = mbar_wait(&pipe.empty[s], parity, p.err_flag);
+                    ok = __all_sync(0xffffffffu, mbar_wait_timed(&pipe.empty[s], parity, p.err_flag, waited));
                     if (!ok) break;
-                    unsigned char *st = smem + s * stage_bytes;
-                    mbar_expect_tx(&pipe.full[s], static_cast<unsigned>((2 * MA + nch) * kPanel));
-                    for (int h = 0; h < 2 * MA; ++h)
-                        tma_load_2d(st + h * kPanel, &map_w, ci0 + 64 * h, ks * 64, &pipe.full[s]);
-                    for (int c = 0; c < nch; ++c)
-                        tma_load_3d(st + a_bytes + c * kPanel, &map_q, cp[c], ks * 64, cb[c], &pipe.full[s]);
+                    if (elect_one()) {
+                        unsigned char *st = smem + s * stage_bytes;
+                        mbar_expect_tx(&pipe.full[s], tx);
+                        for (int h = 0; h < 2 * MA; ++h)
+                            tma_load_2d(st + h * kPanel, &map_w, ci0 + 64 * h, ks * 64, &pipe.full[s]);
+                        st += a_bytes;
+                        int b = b0, c = c0;
+                        for (int i = 0; i < nch; ++i, st += kPanel) {
+                            tma_load_3d(st, &map_q, c * 64, ks * 64, b, &pipe.full[s]);
+                            if (++c == p.chunks_per_img) { c = 0; ++b; }
+                        }
+                    }
                     if (++s == S) { s = 0; parity ^= 1u; }
                 }
             }
+            if (lane == 0) report_wait(p.stats, 3, waited);
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        {   // the whole warp runs the loop (uniform control flow and operands); one elected lane issues
             const unsigned idesc = make_idesc(128, 64 * p.nct, true, true);
             int s = 0;
             unsigned parity = 0;
             bool ok = true;
             long long it = 0;
+            long long wf = 0, wa = 0;
+            const long long born = clock64();
             for (long long t = blockIdx.x; t < p.ntiles && ok; t += gridDim.x, ++it) {
                 // accumulator slot(s) of this tile and how often they have been used before
                 const int slot0 = MA == 2 ? 0 : static_cast<int>(it & 1);
                 const unsigned uses = static_cast<unsigned>(MA == 2 ? it : (it >> 1));
-                for (int a = 0; a < MA && ok; ++a) ok = mbar_wait(&pipe.acc_empty[slot0 + a], (uses & 1u) ^ 1u, p.err_flag);
+                for (int a = 0; a < MA && ok; ++a)
+                    ok = __all_sync(0xffffffffu, mbar_wait_timed(&pipe.acc_empty[slot0 + a], (uses & 1u) ^ 1u, p.err_flag, wa));
                 if (!ok) break;
                 tc_fence_after();
                 for (int ks = 0; ks < p.ksteps; ++ks) {
-                    ok = mbar_wait(&pipe.full[s], parity, p.err_flag);
+                    ok = __all_sync(0xffffffffu, mbar_wait_timed(&pipe.full[s], parity, p.err_flag, wf));
                     if (!ok) break;
                     tc_fence_after();
                     const unsigned a_addr = smem_u32(smem + s * stage_bytes);
                     const unsigned long long bd = make_desc(a_addr + a_bytes, kPanel, 1024);
-                    for (int a = 0; a < MA; ++a) {
-                        const unsigned long long ad = make_desc(a_addr + a * kABytes, kPanel, 1024);
-                        const unsigned tmem_d = tmem_base + (slot0 + a) * kAccCols;
+                    if (elect_one()) {
+                        for (int a = 0; a < MA; ++a) {
+                            const unsigned long long ad = make_desc(a_addr + a * kABytes, kPanel, 1024);
+                            const unsigned tmem_d = tmem_base + (slot0 + a) * kAccCols;
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)      // 16 k-rows = 2048 bytes further per MMA
-                            mma_bf16(tmem_d, ad + 128 * k, bd + 128 * k, idesc, (ks > 0 || k > 0) ? 1u : 0u);
+                            for (int k = 0; k < 4; ++k)      // 16 k-rows = 2048 bytes further per MMA
+                                mma_bf16(tmem_d, ad + 128 * k, bd + 128 * k, idesc, (ks > 0 || k > 0) ? 1u : 0u);
+                        }
+                        mma_commit(&pipe.empty[s]);
                     }
-                    mma_commit(&pipe.empty[s]);
                     if (++s == S) { s = 0; parity ^= 1u; }
                 }
-                if (ok)
+                if (ok && elect_one())
                     for (int a = 0; a < MA; ++a) mma_commit(&pipe.acc_full[slot0 + a]);
+            }
+            if (lane == 0) {
+                report_wait(p.stats, 1, wf);
+                report_wait(p.stats, 2, wa);
+                report_wait(p.stats, 6, clock64() - born);
+                report_wait(p.stats, 7, 1);
             }
         }
     } else {
@@ -202,6 +221,7 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
         const int q = warp & 3;
         bool ok = true;
         long long it = 0;
+        long long we = 0;
         const float delta = *p.delta_p;
         const int vw = (p.HW % 8 == 0) ? 8 : ((p.HW % 4 == 0) ? 4 : 1);
         unsigned char *stage = smem + kRing + (warp - 2) * kStageOut;
@@ -215,7 +235,7 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
             const int ci = ci_w + lane;
             const long long g0 = (t / p.ci_tiles) * p.nct;
             const int nch = static_cast<int>(p.nchunks - g0 < p.nct ? p.nchunks - g0 : p.nct);
-            ok = mbar_wait(&pipe.acc_full[a], uses & 1u, p.err_flag);
+            ok = mbar_wait_timed(&pipe.acc_full[a], uses & 1u, p.err_flag, we);
             if (!ok) break;
             tc_fence_after();
             for (int c = part; c < nch; c += kEpiWarps / 4) {
@@ -320,6 +340,7 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
             warp_arrive(&pipe.acc_empty[a]);
           }
         }
+        if (threadIdx.x == 64) report_wait(p.stats, 5, we);
     }
     tc_fence_before();
     __syncthreads();
@@ -370,6 +391,7 @@ int launch_tma_dx(dbp_ctx *ctx, const void *codes_bf16, const void *W, const flo
     while (p.nct > 1 && ((p.nchunks + p.nct - 1) / p.nct) * p.ci_tiles < (ctx->sm_count * 3) / 4) p.nct /= 2;
     p.ntiles = ((p.nchunks + p.nct - 1) / p.nct) * p.ci_tiles;
     p.err_flag = err_flag;
+    p.stats = ctx->wait_stats;
     const size_t smem = static_cast<size_t>(kRing) + kEpiWarps * kStageOut + 1024;
     if (cudaFuncSetAttribute(tma_dx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
         return DBP_ECUDA;
