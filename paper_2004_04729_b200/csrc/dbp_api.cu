@@ -173,6 +173,12 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
             ctx->nnz_pending = true;
     }
     if (dense) {
+        // dX and dW read the same codes and nothing of each other: with both asked for, dW goes to the
+        // context's second stream, so that its CTAs start as SMs come free instead of after the last dX CTA
+        const bool forked = dX && dW && ctx->aux != nullptr;
+        if (forked && (cudaEventRecord(ctx->ev_fork, ctx->stream) != cudaSuccess ||
+                       cudaStreamWaitEvent(ctx->aux, ctx->ev_fork, 0) != cudaSuccess))
+            return fail_cuda("forking the dW stream");
         if (dX) {
             KernelTimer t(ctx, DBP_K_DX_DENSE);
             const bool dx_bf16 = (io == DBP_BF16) && !(flags & DBP_DX_F32);
@@ -182,14 +188,20 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
             if (rc) return rc;
         }
         if (ctx->hook_after_dx && cudaEventRecord(ctx->hook_after_dx, ctx->stream) != cudaSuccess) return DBP_ECUDA;
-        if (dW && ctx->hook_before_dw && cudaStreamWaitEvent(ctx->stream, ctx->hook_before_dw, 0) != cudaSuccess) return DBP_ECUDA;
-        if (dW) {
+        cudaStream_t caller = ctx->stream;
+        if (forked) ctx->stream = ctx->aux;          // the dW launchers enqueue on the context's stream
+        if (dW && ctx->hook_before_dw && cudaStreamWaitEvent(ctx->stream, ctx->hook_before_dw, 0) != cudaSuccess) rc = DBP_ECUDA;
+        if (dW && !rc) {
             KernelTimer t(ctx, DBP_K_DW_DENSE);
             rc = dw_tma ? launch_tma_dw(ctx, codes16, X, delta_p, s, dW, &ctx->state->tc_timeout)
                  : t3   ? launch_tc3_tma_dw(ctx, codes_n, X, delta_p, s, dW, &ctx->state->tc_timeout)
                         : launch_tc_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout);
-            if (rc) return rc;
         }
+        ctx->stream = caller;
+        if (forked && (cudaEventRecord(ctx->ev_join, ctx->aux) != cudaSuccess ||
+                       cudaStreamWaitEvent(caller, ctx->ev_join, 0) != cudaSuccess))
+            return fail_cuda("joining the dW stream");
+        if (rc) return rc;
         if (db) {
             KernelTimer t(ctx, DBP_K_DB);
             rc = launch_bias_grad(ctx, codes, delta_p, s, db);
@@ -265,7 +277,10 @@ int dbp_create(dbp_ctx **out, int device, void *cuda_stream) {
         dbp_destroy(ctx);
         return DBP_ENOMEM;
     }
-    if (cudaMallocHost(&ctx->nnz_host, sizeof(unsigned long long)) != cudaSuccess ||
+    if (cudaStreamCreateWithFlags(&ctx->aux, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+        cudaMallocHost(&ctx->nnz_host, sizeof(unsigned long long)) != cudaSuccess ||
         cudaEventCreateWithFlags(&ctx->nnz_event, cudaEventDisableTiming) != cudaSuccess) {
         cudaGetLastError();
         dbp_destroy(ctx);
@@ -294,6 +309,9 @@ int dbp_destroy(dbp_ctx *ctx) {
     for (ProfSlot &p : ctx->prof) { cudaEventDestroy(p.begin); cudaEventDestroy(p.end); }
     if (ctx->nnz_host) cudaFreeHost(ctx->nnz_host);
     if (ctx->nnz_event) cudaEventDestroy(ctx->nnz_event);
+    if (ctx->aux) { cudaStreamSynchronize(ctx->aux); cudaStreamDestroy(ctx->aux); }
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     if (ctx->copy_in) { cudaStreamSynchronize(ctx->copy_in); cudaStreamDestroy(ctx->copy_in); }
     if (ctx->copy_out) { cudaStreamSynchronize(ctx->copy_out); cudaStreamDestroy(ctx->copy_out); }
     if (ctx->ev_x_up) cudaEventDestroy(ctx->ev_x_up);

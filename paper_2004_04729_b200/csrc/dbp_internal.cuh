@@ -57,6 +57,10 @@ struct dbp_ctx {
     // *_host entry points: X goes up and dX comes down on streams of their own, so that the two
     // directions of the host link work at the same time; the events order them against the
     // kernels (dX done -> its read-back may start; X up -> the dW kernels may start)
+    // the dense dW kernels of a layer run beside its dX kernel on a stream of their own (they only
+    // share inputs): forked after the quantization, joined before the call returns to the caller's stream
+    cudaStream_t aux = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
     cudaEvent_t ev_x_up = nullptr, ev_dx_done = nullptr;
     cudaEvent_t hook_after_dx = nullptr, hook_before_dw = nullptr;   // set only during a *_host call
