@@ -271,24 +271,27 @@ def main():
     lib = dbp.load_library()
     import ctypes
 
+    ASYNC = dbp.DBP_DW_ASYNC        # dW of a layer may still run while the next layer is quantized; joined at the step's end
+
     def run_layer(L, d, X, W, dW, dX):
         code = 1 if L.dtype == "bf16" else 0
         if L.kind == "linear":
             B, N = d.shape
             rc = lib.dithered_linear_backward(ctx._h, d.data_ptr(), X.data_ptr(), W.data_ptr(), code,
                                               B, N, X.shape[1], L.seed, L.scale, None, None,
-                                              dW.data_ptr(), dX.data_ptr(), None, 0)
+                                              dW.data_ptr(), dX.data_ptr(), None, ASYNC)
         else:
             B, Co, H, Wd = d.shape
             rc = lib.dithered_conv_backward(ctx._h, d.data_ptr(), X.data_ptr(), W.data_ptr(), code,
                                             B, X.shape[1], Co, H, Wd, L.k, 1, (L.k - 1) // 2, L.seed,
-                                            L.scale, None, None, dW.data_ptr(), dX.data_ptr(), None, 0)
+                                            L.scale, None, None, dW.data_ptr(), dX.data_ptr(), None, ASYNC)
         if rc != 0:
             raise RuntimeError(f"library call failed on {L.name}: {rc}")
 
     def step():
         for item in layers:
             run_layer(*item)
+        ctx.join()                  # every dW of the step is ordered into the stream before the step ends
 
     def barrier():
         if world > 1:

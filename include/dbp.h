@@ -52,6 +52,13 @@ typedef enum {
                                does not exist (it covers bf16 linear, 1x1 and 3x3 layers whose channel
                                counts are multiples of 8; 3x3 images up to 62 wide) */
 #define DBP_DX_F32       4u /* with io = DBP_BF16: write dX as fp32 instead of bf16 */
+#define DBP_DW_ASYNC     8u /* dense path with both dW and dX asked for: the call returns with dX (and db)
+                               ordered on the context's stream as usual, while dW is still being computed on
+                               the context's second stream. dW (and the scratch it needs) is ordered into the
+                               context's stream by dbp_join, by dbp_last_device_status / dbp_last_step, or by
+                               dbp_destroy; until then the caller must not read dW nor overwrite X. This is the
+                               order a training step needs: the layer below depends on dX only, the weight
+                               gradients are needed by the optimizer at the end. */
 
 /*
  * Density crossover (Section 3.4: the sparse products cost O(p_nz m k n), a dense product
@@ -101,6 +108,9 @@ typedef struct dbp_sparse {
 int dbp_create(dbp_ctx **out, int device, void *cuda_stream);
 int dbp_destroy(dbp_ctx *ctx);
 int dbp_set_stream(dbp_ctx *ctx, void *cuda_stream);
+/* Makes the context's stream wait for every dW computation that earlier DBP_DW_ASYNC calls left
+ * running (a stream-ordered join: nothing blocks on the host). */
+int dbp_join(dbp_ctx *ctx);
 const char *dbp_status_string(int status);
 /* Text of the most recent DBP_ECUDA on the calling thread: which step failed and the CUDA
  * runtime's message (empty if none yet). The pointer stays valid; the text changes with the next

@@ -12,7 +12,7 @@ import torch
 HERE = os.path.dirname(os.path.abspath(__file__))
 
 DBP_F32, DBP_BF16 = 0, 1
-DBP_FORCE_SPARSE, DBP_FORCE_DENSE, DBP_DX_F32 = 1, 2, 4
+DBP_FORCE_SPARSE, DBP_FORCE_DENSE, DBP_DX_F32, DBP_DW_ASYNC = 1, 2, 4, 8
 DBP_SEGMENT = 1024
 
 EXPORTED_SYMBOLS = [
@@ -21,7 +21,7 @@ EXPORTED_SYMBOLS = [
     "dithered_linear_backward", "dithered_conv_backward", "dithered_linear_backward_host",
     "dithered_conv_backward_host", "dbp_relu_backward", "dbp_maxpool2x2_backward",
     "dbp_profile_enable", "dbp_profile_select", "dbp_profile_read", "dbp_set_crossover", "nsd_step_size_noalloc",
-    "dbp_last_step", "dbp_layer_seed", "dbp_selftest_bounded_wait", "dbp_last_error", "dbp_wait_stats",
+    "dbp_last_step", "dbp_layer_seed", "dbp_selftest_bounded_wait", "dbp_last_error", "dbp_wait_stats", "dbp_join",
 ]
 
 KERNEL_KINDS = ["statistics", "quantize", "weight_taps", "dx", "dw", "db", "decode", "glue",
@@ -84,6 +84,7 @@ def load_library():
     lib.dbp_profile_select.argtypes = [vp, u32]
     lib.dbp_profile_read.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ll)]
     lib.dbp_selftest_bounded_wait.argtypes = [vp, ll]
+    lib.dbp_join.argtypes = [vp]
     lib.dbp_wait_stats.argtypes = [vp, ctypes.POINTER(ull), i32]
     lib.dbp_last_step.argtypes = [vp, ctypes.POINTER(f32), ctypes.POINTER(ll)]
     lib.dbp_layer_seed.argtypes = [ull, i32]
@@ -169,6 +170,10 @@ class Context:
         out = (ctypes.c_ulonglong * 8)()
         _check(load_library().dbp_wait_stats(self._h, out, int(reset)), "dbp_wait_stats")
         return list(out)
+
+    def join(self):
+        """Orders every dW left running by DBP_DW_ASYNC calls into the context's stream."""
+        _check(load_library().dbp_join(self._h), "dbp_join")
 
     def set_crossover(self, crossover: float):
         """Density above which layers the dense tensor-core path supports use it."""

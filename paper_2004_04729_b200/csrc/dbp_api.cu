@@ -21,6 +21,7 @@ int ws_reserve(dbp_ctx *ctx, Workspace &w, size_t bytes) {
     // the stream may still be using the old block
     if (w.ptr) {
         if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return DBP_ECUDA;
+        if (ctx->aux && cudaStreamSynchronize(ctx->aux) != cudaSuccess) return DBP_ECUDA;
         cudaFree(w.ptr);
         w.ptr = nullptr;
         w.bytes = 0;
@@ -69,14 +70,22 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
         q_out->numel = numel;
         sp = *q_out;
     }
-    if ((rc = ws_reserve(ctx, ctx->dense_codes, static_cast<size_t>(numel) + 16))) return rc;
-    int8_t *dense = static_cast<int8_t *>(ctx->dense_codes.ptr);
+    const int k = ctx->code_set;
+    if ((rc = ws_reserve(ctx, ctx->dense_codes[k], static_cast<size_t>(numel) + 16))) return rc;
+    int8_t *dense = static_cast<int8_t *>(ctx->dense_codes[k].ptr);
     {
         KernelTimer t(ctx, DBP_K_STATISTICS);
-        rc = launch_statistics(ctx, delta, dtype, numel, scale, delta_in, sp.delta,
+        // without a caller's dbp_sparse the step size also goes to the set's own scalar: the product kernels
+        // read it there (the context's scalar is overwritten by the next call's statistics)
+        rc = launch_statistics(ctx, delta, dtype, numel, scale, delta_in, q_out ? sp.delta : ctx->delta_sets + k,
                                reinterpret_cast<unsigned long long *>(sp.nnz), zero, zero_bytes);
     }
     if (rc) return rc;
+    // the set's previous readers (an earlier call's dW kernels on the second stream) must be done
+    if (ctx->set_busy[k]) {
+        if (cudaStreamWaitEvent(ctx->stream, ctx->ev_set_free[k], 0) != cudaSuccess) return fail_cuda("waiting for the code buffers");
+        ctx->set_busy[k] = false;
+    }
     {
         KernelTimer t(ctx, DBP_K_QUANTIZE);
         // the sparse structure is written only for a caller who asked for it; the bf16 planes
@@ -84,14 +93,14 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
         void *p16 = nullptr;
         if (codes16) {
             const long long planes = numel / planes_hw;
-            if ((rc = ws_reserve(ctx, ctx->codes16, static_cast<size_t>(planes) * planes_pitch * 2 + 1024))) return rc;
-            p16 = ctx->codes16.ptr;
+            if ((rc = ws_reserve(ctx, ctx->codes16[k], static_cast<size_t>(planes) * planes_pitch * 2 + 1024))) return rc;
+            p16 = ctx->codes16[k].ptr;
             *codes16 = p16;
         }
         void *pn = nullptr;
         if (nhwc) {
-            if ((rc = ws_reserve(ctx, ctx->codes_nhwc, static_cast<size_t>(numel) * 2 + 1024))) return rc;
-            pn = ctx->codes_nhwc.ptr;
+            if ((rc = ws_reserve(ctx, ctx->codes_nhwc[k], static_cast<size_t>(numel) * 2 + 1024))) return rc;
+            pn = ctx->codes_nhwc[k].ptr;
             *codes_nhwc = pn;
         }
         if (q_out) {
@@ -112,7 +121,10 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
         }
     }
     if (rc) return rc;
-    *delta_p = &ctx->state->delta;
+    *delta_p = q_out ? &ctx->state->delta : ctx->delta_sets + k;
+    if (q_out && cudaMemcpyAsync(ctx->delta_sets + k, &ctx->state->delta, sizeof(float), cudaMemcpyDeviceToDevice, ctx->stream) != cudaSuccess)
+        return fail_cuda("copying the step size");
+    if (q_out) *delta_p = ctx->delta_sets + k;
     *codes = dense;
     return DBP_OK;
 }
@@ -155,6 +167,12 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     const bool dx_tma = dense && dX && tma_dx_supported(s, io);
     const bool dw_tma = dense && dW && tma_dw_supported(s, io);
     const bool any_tma = dx_tma || dw_tma;
+    // a call that does not itself fork its dW first orders the earlier calls' outstanding dW work into the
+    // stream: it may use the workspaces that work is still using
+    if (ctx->aux_pending && !(dense && dX && dW)) {
+        const int jr = dbp_join(ctx);
+        if (jr) return jr;
+    }
     // 3x3 layers: the TMA-fed kernels read the codes position-major
     const bool t3 = dense && (dX || dW) && tc3_tma_supported(s, io);
     const bool need8 = !dense || db || (!t3 && ((dX && !dx_tma) || (dW && !dw_tma)));
@@ -198,9 +216,19 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
                         : launch_tc_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout);
         }
         ctx->stream = caller;
-        if (forked && (cudaEventRecord(ctx->ev_join, ctx->aux) != cudaSuccess ||
-                       cudaStreamWaitEvent(caller, ctx->ev_join, 0) != cudaSuccess))
-            return fail_cuda("joining the dW stream");
+        if (forked) {
+            // the set's buffers are free once the dW kernels are done; with DBP_DW_ASYNC the caller's stream is
+            // ordered after them only by the next user of the set, by dbp_join or by a synchronising call
+            const int k = ctx->code_set;
+            if (cudaEventRecord(ctx->ev_set_free[k], ctx->aux) != cudaSuccess) return fail_cuda("recording the end of dW");
+            if ((flags & DBP_DW_ASYNC) && !rc) {
+                ctx->set_busy[k] = true;
+                ctx->aux_pending = true;
+                ctx->code_set = k ^ 1;
+            } else if (cudaStreamWaitEvent(caller, ctx->ev_set_free[k], 0) != cudaSuccess) {
+                return fail_cuda("joining the dW stream");
+            }
+        }
         if (rc) return rc;
         if (db) {
             KernelTimer t(ctx, DBP_K_DB);
@@ -280,6 +308,9 @@ int dbp_create(dbp_ctx **out, int device, void *cuda_stream) {
     if (cudaStreamCreateWithFlags(&ctx->aux, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_set_free[0], cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_set_free[1], cudaEventDisableTiming) != cudaSuccess ||
+        cudaMalloc(&ctx->delta_sets, 2 * sizeof(float)) != cudaSuccess ||
         cudaMallocHost(&ctx->nnz_host, sizeof(unsigned long long)) != cudaSuccess ||
         cudaEventCreateWithFlags(&ctx->nnz_event, cudaEventDisableTiming) != cudaSuccess) {
         cudaGetLastError();
@@ -292,6 +323,19 @@ int dbp_create(dbp_ctx **out, int device, void *cuda_stream) {
 
 const char *dbp_last_error(void) { return g_last_error; }
 
+int dbp_join(dbp_ctx *ctx) {
+    if (!ctx) return DBP_EINVAL;
+    if (!ctx->aux_pending) return DBP_OK;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DBP_ECUDA;
+    // everything enqueued on the second stream so far: one event, and the caller's stream waits for it
+    if (cudaEventRecord(ctx->ev_join, ctx->aux) != cudaSuccess || cudaStreamWaitEvent(ctx->stream, ctx->ev_join, 0) != cudaSuccess)
+        return fail_cuda("joining the dW stream");
+    ctx->aux_pending = false;
+    ctx->set_busy[0] = ctx->set_busy[1] = false;
+    return DBP_OK;
+}
+
 int dbp_set_crossover(dbp_ctx *ctx, float crossover) {
     if (!ctx || crossover != crossover) return DBP_EINVAL;
     ctx->crossover = crossover;
@@ -302,7 +346,9 @@ int dbp_destroy(dbp_ctx *ctx) {
     if (!ctx) return DBP_EINVAL;
     DeviceGuard guard(ctx->device);
     cudaStreamSynchronize(ctx->stream);
-    Workspace *all[] = {&ctx->dense_codes, &ctx->codes16, &ctx->codes_nhwc, &ctx->dw_acc, &ctx->x_padded, &ctx->w_taps, &ctx->sp_bitmap, &ctx->sp_offsets, &ctx->sp_values,
+    if (ctx->aux) cudaStreamSynchronize(ctx->aux);
+    Workspace *all[] = {&ctx->dense_codes[0], &ctx->dense_codes[1], &ctx->codes16[0], &ctx->codes16[1],
+                        &ctx->codes_nhwc[0], &ctx->codes_nhwc[1], &ctx->dw_acc, &ctx->x_padded, &ctx->w_taps, &ctx->sp_bitmap, &ctx->sp_offsets, &ctx->sp_values,
                         &ctx->tc_partials};
     for (Workspace *w : all) if (w->ptr) cudaFree(w->ptr);
     for (Workspace &w : ctx->io) if (w.ptr) cudaFree(w.ptr);
@@ -311,6 +357,8 @@ int dbp_destroy(dbp_ctx *ctx) {
     if (ctx->nnz_event) cudaEventDestroy(ctx->nnz_event);
     if (ctx->aux) { cudaStreamSynchronize(ctx->aux); cudaStreamDestroy(ctx->aux); }
     if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    for (cudaEvent_t e : ctx->ev_set_free) if (e) cudaEventDestroy(e);
+    if (ctx->delta_sets) cudaFree(ctx->delta_sets);
     if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     if (ctx->copy_in) { cudaStreamSynchronize(ctx->copy_in); cudaStreamDestroy(ctx->copy_in); }
     if (ctx->copy_out) { cudaStreamSynchronize(ctx->copy_out); cudaStreamDestroy(ctx->copy_out); }
@@ -325,6 +373,7 @@ int dbp_destroy(dbp_ctx *ctx) {
 
 int dbp_set_stream(dbp_ctx *ctx, void *cuda_stream) {
     if (!ctx) return DBP_EINVAL;
+    if (int jr = dbp_join(ctx)) return jr;           // outstanding dW work is ordered into the old stream
     ctx->stream = static_cast<cudaStream_t>(cuda_stream);
     return DBP_OK;
 }
@@ -346,6 +395,7 @@ const char *dbp_status_string(int status) {
 
 int dbp_last_device_status(dbp_ctx *ctx, int *status, long long *saturated) {
     if (!ctx) return DBP_EINVAL;
+    if (int jr = dbp_join(ctx)) return jr;
     DeviceGuard guard(ctx->device);
     DeviceState h;
     if (cudaMemcpyAsync(&h, ctx->state, sizeof(h), cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess ||
@@ -373,6 +423,7 @@ int dbp_selftest_bounded_wait(dbp_ctx *ctx, long long cycles) {
 
 int dbp_wait_stats(dbp_ctx *ctx, unsigned long long *out, int reset) {
     if (!ctx || !out) return DBP_EINVAL;
+    if (int jr = dbp_join(ctx)) return jr;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DBP_ECUDA;
     if (cudaMemcpyAsync(out, ctx->wait_stats, sizeof(unsigned long long) * DBP_WAIT_SLOTS, cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess ||
@@ -397,6 +448,7 @@ int dbp_profile_select(dbp_ctx *ctx, unsigned kind_mask) {
 
 int dbp_profile_read(dbp_ctx *ctx, int kind, double *milliseconds, long long *launches) {
     if (!ctx || kind < 0 || kind >= DBP_K_COUNT) return DBP_EINVAL;
+    if (int jr = dbp_join(ctx)) return jr;
     DeviceGuard guard(ctx->device);
     if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return DBP_ECUDA;
     for (size_t i = 0; i < ctx->prof_used; ++i) {
@@ -450,6 +502,7 @@ int nsd_quantize(dbp_ctx *ctx, const void *delta, int dtype, long long numel, un
 
 int dbp_last_step(dbp_ctx *ctx, float *delta_out, long long *nnz_out) {
     if (!ctx) return DBP_EINVAL;
+    if (int jr = dbp_join(ctx)) return jr;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DBP_ECUDA;
     DeviceState h;
@@ -538,7 +591,8 @@ static int host_backward(dbp_ctx *ctx, const void *delta, const void *X, const v
     if (dX) ctx->hook_after_dx = ctx->ev_dx_done;
     rc = conv_backward_impl(ctx, ctx->io[0].ptr, X ? ctx->io[1].ptr : nullptr, W ? ctx->io[2].ptr : nullptr, io, s,
                             seed, scale, nullptr, nullptr, dW ? static_cast<float *>(ctx->io[3].ptr) : nullptr,
-                            dX ? ctx->io[4].ptr : nullptr, db ? static_cast<float *>(ctx->io[5].ptr) : nullptr, flags);
+                            dX ? ctx->io[4].ptr : nullptr, db ? static_cast<float *>(ctx->io[5].ptr) : nullptr,
+                            flags & ~DBP_DW_ASYNC);      // the results are copied back right away
     ctx->hook_before_dw = nullptr;
     ctx->hook_after_dx = nullptr;
     if (rc) {

@@ -44,13 +44,20 @@ struct dbp_ctx {
     double *partials = nullptr;         // device, statistics partial sums
     unsigned long long *wait_stats = nullptr;   // device, DBP_WAIT_SLOTS counters of SM clocks spent waiting
     int partial_blocks = 0;
-    dbp::Workspace dense_codes;         // int8 per element of delta
+    // The codes of a layer exist in two sets of buffers used in turn: with DBP_DW_ASYNC the dW kernels of
+    // one call may still read their set while the next call's quantization writes the other one.
+    dbp::Workspace dense_codes[2];      // int8 per element of delta
     dbp::Workspace x_padded;            // activations copied to 16-byte aligned planes
-    dbp::Workspace codes16;             // bf16 code planes for the TMA-fed kernels
+    dbp::Workspace codes16[2];          // bf16 code planes for the TMA-fed kernels
     dbp::Workspace w_taps;              // fp32 weights as [Cout][k*k][Cin]
     dbp::Workspace sp_bitmap, sp_offsets, sp_values;  // internal dbp_sparse
     dbp::Workspace tc_partials;         // split-K partial blocks of the dense dW kernel
-    dbp::Workspace codes_nhwc;          // bf16 codes [B][position][Cout] for the TMA-fed 3x3 kernels
+    dbp::Workspace codes_nhwc[2];       // bf16 codes [B][position][Cout] for the TMA-fed 3x3 kernels
+    float *delta_sets = nullptr;        // device float[2]: the step size that belongs to each set
+    int code_set = 0;                   // the set the next call writes
+    cudaEvent_t ev_set_free[2] = {nullptr, nullptr};   // recorded on the dW stream after the set's last reader
+    bool set_busy[2] = {false, false};
+    bool aux_pending = false;           // dW work on the second stream that the caller's stream is not yet ordered after
     dbp::Workspace dw_acc;              // fp32 [tap][Cout][Cin] that the 3x3 dW CTAs add into; zero between calls
     bool dw_acc_clean = false;
     dbp::Workspace io[8];               // staging for the *_host entry points

@@ -190,3 +190,27 @@ def test_back_to_back_calls_are_ordered(ctx):
             gx = o["dX"].double().cpu().numpy()
             slack = 0.0 if f32 else 2.0 ** -8
             assert np.all(np.abs(gx - ref["dX"]) <= slack * np.abs(ref["dX"]) + TOL * ref["S_dX"] + 1e-30)
+
+
+def test_async_dw_matches_the_synchronous_call(ctx):
+    """DBP_DW_ASYNC: dW of a layer is still being computed on the context's second stream while the
+    next layers are quantized (their codes go to the other set of buffers). After dbp_join the
+    results are those of the synchronous calls: dX bit for bit, dW up to the order of the additions."""
+    import paper_2004_04729_b200 as dbp
+    shapes = [(2, 256, 64, 28, 28, 1), (2, 64, 64, 28, 28, 3), (3, 512, 128, 14, 14, 1), (3, 128, 128, 7, 7, 3),
+              (2, 64, 256, 28, 28, 1)]
+    layers = [wl.conv_layer(B, Ci, Co, H, W, k, data_seed=31 + i, scale=5.0, dtype="bf16")
+              for i, (B, Ci, Co, H, W, k) in enumerate(shapes)]
+    dev = [(_t(L.delta), _t(L.X), _t(L.W)) for L in layers]
+    ref = [dbp.dithered_conv_backward(ctx, d, X, W, L.seed, L.scale) for L, (d, X, W) in zip(layers, dev)]
+    torch.cuda.synchronize()
+    for _ in range(2):                                   # twice: both buffer sets get reused
+        out = [dbp.dithered_conv_backward(ctx, d, X, W, L.seed, L.scale, flags=dbp.DBP_DW_ASYNC)
+               for L, (d, X, W) in zip(layers, dev)]
+        ctx.join()
+        torch.cuda.synchronize()
+        assert ctx.last_device_status() == (0, 0)
+        for a, b in zip(ref, out):
+            assert torch.equal(a["dX"], b["dX"])
+            scale = a["dW"].abs().max().item()
+            assert (a["dW"] - b["dW"]).abs().max().item() <= 1e-5 * scale
