@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the dithered-backprop hot path on B200.
 
-    python bench.py --gpus N --steps K --warmup W [--config 5|3|1] [--impl reference]
+    python bench.py --gpus N --steps K --warmup W [--config 5|4|3|2|1] [--impl reference]
 
 One *step* is one pass of the whole path (statistics -> NSD quantize/compact -> dX -> dW)
 over every layer of the workload, on seeded synthetic inputs already resident in HBM.
@@ -35,7 +35,6 @@ import workloads as wl  # noqa: E402
 
 METRIC = "dithered backward dense-equiv GFLOP/s and % HBM roofline vs cuBLAS dense"
 UNIT = "GFLOP/s (dense-equivalent, dW+dX)"
-FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # fp32 FMA lanes x 2 flop x max SM clock
 
 
 def measured_peaks():
@@ -49,6 +48,10 @@ def measured_peaks():
 
 # ------------------------------------------------------------------ workloads
 
+CHAIN_NAMES = {2: "config2: LeNet-300-100 full backward, B256, fp32, s=2",
+               4: "config4: VGG-16/CIFAR full backward (13 conv3x3 + FC), B128, fp32, s=2"}
+
+
 def layer_specs(config, batch):
     """[(Layer factory, multiplicity)] in network order."""
     if config == 1:
@@ -60,7 +63,9 @@ def layer_specs(config, batch):
         specs = [((lambda i=i: wl.config5_layer(i, batch=b)), wl.RESNET50_SET[i][5])
                  for i in range(len(wl.RESNET50_SET))]
         return specs, f"config5: ResNet-50 bottleneck layer set (48 convs, 16 shapes), B{b}, bf16, s=5"
-    raise SystemExit("--config must be 1, 3 or 5")
+    if config in CHAIN_NAMES:
+        return [], CHAIN_NAMES[config]
+    raise SystemExit("--config must be 1 ... 5")
 
 
 def algorithmic_bytes(L):
@@ -127,6 +132,12 @@ def oracle_layers(config):
         return [wl.config1()], "the whole layer (B128)", 200
     if config == 3:
         return [wl.config3(batch=32)], "batch 32 of 128", 4
+    if config == 2:
+        c = wl.mlp_chain(batch=256)
+        return [c], "the whole network (B256)", 100
+    if config == 4:
+        c = wl.vgg_chain(batch=8)
+        return [c], "batch 8 of 128", 2
     layers = [wl.config5_layer(i, batch=16) for i in range(len(wl.RESNET50_SET))]
     return layers, "batch 16 of 64 of all 16 shapes (one instance each)", 3
 
@@ -139,6 +150,10 @@ def oracle_time(layers, passes, budget_s=30.0):
     flops, done = 0.0, 0
     for _ in range(passes):
         for L in layers:
+            if isinstance(L, wl.Chain):
+                oracle.chain_backward(L.kinds, L.X, L.W, L.relu_mask, L.pool_argmax, L.delta_out, L.scale, 0)
+                flops += chain_flops(L)
+                continue
             D = oracle.step_size(L.delta, L.scale)
             codes, _, _ = oracle.nsd_codes(L.delta, L.seed, D)
             fn = oracle.linear_backward if L.kind == "linear" else oracle.conv_backward
@@ -149,6 +164,28 @@ def oracle_time(layers, passes, budget_s=30.0):
             break
     dt = time.perf_counter() - t0
     return flops / dt / 1e9, dt, done
+
+
+def chain_flops(c):
+    """Dense backward FLOPs of a chain (2 per MAC, dW and dX of every layer; the first layer's dX is
+    not computed, as in a training step)."""
+    f = 0.0
+    for l, kind in enumerate(c.kinds):
+        X, W = c.X[l], c.W[l]
+        macs = X.shape[0] * W.shape[0] * W.shape[1] * (X.shape[2] * X.shape[3] * 9 if kind == "conv" else 1)
+        f += 2.0 * macs * (2 if l > 0 else 1)
+    return f
+
+
+def chain_bytes(c):
+    """Bytes a chain's backward must move at least: per layer delta twice (statistics, quantize), X and W
+    read, dW and (but for the first layer) dX written; fp32."""
+    b = 0
+    for l in range(len(c.kinds)):
+        nx, nw = c.X[l].size, c.W[l].size
+        nd = c.X[l].shape[0] * c.W[l].shape[0] * (c.X[l].shape[2] * c.X[l].shape[3] if c.kinds[l] == "conv" else 1)
+        b += 4 * (2 * nd + nx + nw + nw + (nx if l > 0 else 0))
+    return b
 
 
 def host_cores():
@@ -208,6 +245,98 @@ def job_throughput(flops_per_rank_step, world, ms_per_step):
     return flops_per_rank_step * world / (ms_per_step * 1e-3) / 1e9
 
 
+def time_events(torch, fn, reps):
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / reps
+
+
+def dense_layer_fn(torch, L, d, X, W):
+    if L.kind == "linear":
+        return lambda: (torch.matmul(d.t(), X), torch.matmul(d, W))
+    p = (L.k - 1) // 2
+    return lambda: torch.ops.aten.convolution_backward(d, X, W, None, [1, 1], [p, p], [1, 1], False, [0, 0], 1,
+                                                       [True, True, False])
+
+
+def dense_times(torch, fns, reps):
+    """cuDNN / cuBLAS backward (autotuned algorithms) on the given closures, TF32 off and on."""
+    torch.backends.cudnn.benchmark = True
+    out = {}
+    for label, tf32 in (("tf32_off", False), ("tf32_on", True)):
+        torch.backends.cudnn.allow_tf32 = tf32
+        torch.backends.cuda.matmul.allow_tf32 = tf32
+        step = lambda: [f() for f in fns]
+        for _ in range(3):
+            step()
+        torch.cuda.synchronize()
+        out[label] = time_events(torch, step, reps)
+    return out
+
+
+def small_config(torch, dbp, ctx, config, hbm_peak, fma_peak):
+    """One of configs 1-4 as a short side measurement: layer (or whole-network backward) time, dense-equivalent
+    throughput, fraction of the HBM roofline for the algorithmic bytes, fraction of the fp32 FMA peak for the
+    non-zero FMAs (these fp32 configurations run on the sparse gather kernels), the dense library time."""
+    dev = torch.device("cuda", ctx.device)
+    if config in (1, 3):
+        L = wl.config1() if config == 1 else wl.config3()
+        d, X, W = (torch.from_numpy(a).to(dev) for a in (L.delta, L.X, L.W))
+        fn = dbp.dithered_linear_backward if L.kind == "linear" else dbp.dithered_conv_backward
+        run = lambda: fn(ctx, d, X, W, L.seed, L.scale)
+        flops, nbytes = L.dense_flops, algorithmic_bytes(L)
+        q = dbp.nsd_quantize(ctx, d, L.seed, L.scale)
+        density = q.nnz.item() / d.numel()
+        dq = (dbp.nsd_decode_dense(ctx, q, d.shape).float() * q.delta).contiguous()
+        dense_fns = [dense_layer_fn(torch, L, dq, X, W)]
+        name = layer_specs(config, 0)[1]
+    else:
+        c = wl.mlp_chain(batch=256) if config == 2 else wl.vgg_chain(batch=128, device=str(dev))
+        cu = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+        Xs, Ws = [cu(a) for a in c.X], [cu(a) for a in c.W]
+        masks = [None if m is None else cu(m.astype(np.uint8)) for m in c.relu_mask]
+        pools = [cu(a) for a in c.pool_argmax]
+        dout = cu(c.delta_out)
+        run = lambda: dbp.network_backward(ctx, c.kinds, Xs, Ws, masks, pools, dout, c.scale, 0, with_sparse=False)
+        res = dbp.network_backward(ctx, c.kinds, Xs, Ws, masks, pools, dout, c.scale, 0, keep_delta_z=True)
+        torch.cuda.synchronize()
+        flops, nbytes = chain_flops(c), chain_bytes(c)
+        nz = sum(r["nnz"].item() for r in res)
+        density = nz / sum(r["delta_z"].numel() for r in res)
+        dense_fns = []
+        for l, kind in enumerate(c.kinds):
+            dz = res[l]["delta_z"]
+            if kind == "linear":
+                dense_fns.append(lambda dz=dz, X=Xs[l], W=Ws[l], l=l: (torch.matmul(dz.t(), X), torch.matmul(dz, W) if l else None))
+            else:
+                dense_fns.append(lambda dz=dz, X=Xs[l], W=Ws[l], l=l: torch.ops.aten.convolution_backward(
+                    dz, X, W, None, [1, 1], [1, 1], [1, 1], False, [0, 0], 1, [l > 0, True, False]))
+        name = CHAIN_NAMES[config]
+    for _ in range(3):
+        run()
+    torch.cuda.synchronize()
+    n0 = dbp.kernel_launches()
+    run()
+    launches = dbp.kernel_launches() - n0
+    ms = time_events(torch, run, 20 if config != 4 else 5)
+    dt = dense_times(torch, dense_fns, 20 if config != 4 else 5)
+    return {"workload": name, "ms": ms, "gflops_dense_equiv": flops / (ms * 1e-3) / 1e9,
+            "hbm_frac": nbytes / (ms * 1e-3) / 1e9 / hbm_peak, "algorithmic_mb": nbytes / 1e6,
+            "nsd_density": density, "fma_frac": density * flops / (ms * 1e-3) / 1e12 / fma_peak,
+            "dense_ms": dt, "launches": launches,
+            "note": "fp32: sparse gather kernels (no tensor-core path for fp32 operands); launch-bound at these sizes"
+                    if config in (1, 2) else "fp32: sparse gather kernels (no tensor-core path for fp32 operands)"}
+
+
+# DRAM bytes (read + written) of one bench step's launches of each kernel kind, from the ncu capture summarised in
+# profiles/bench_step_config5_dram_bytes.md; None = the kernels of that kind changed after the capture
+NCU_DRAM_BYTES_PER_STEP = {"statistics": None, "quantize": None, "dx_dense": None, "dw_dense": None}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -221,6 +350,8 @@ def main():
     ap.add_argument("--no-dense", action="store_true", help="skip the cuDNN/cuBLAS dense comparison")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-others", action="store_true", help="skip the side measurements of configs 1-4")
+    ap.add_argument("--sync-dw", action="store_true", help="every call joins its dW before it returns (no DBP_DW_ASYNC)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl != "reference":
         args.warmup = 3
@@ -242,6 +373,29 @@ def main():
     sampler = ClockSampler(local)       # nvidia-smi takes a while to deliver its first sample: start it now
     if rank == 0:
         sampler.start()
+    hbm_peak, peak_src = measured_peaks()
+    fma_peak = ctx.measure_fma_peak()
+
+    if args.config in CHAIN_NAMES:
+        # whole-network configurations: the side measurement is the measurement
+        r = small_config(torch, dbp, ctx, args.config, hbm_peak, fma_peak)
+        clocks = sampler.stop() if rank == 0 else None
+        ms = max_over_ranks(r["ms"], dev, world)
+        if rank == 0:
+            print(json.dumps({
+                "metric": METRIC, "value": job_throughput(r["gflops_dense_equiv"] * r["ms"] * 1e6, world, ms), "unit": UNIT,
+                "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": r["workload"], "nsd_density": r["nsd_density"], "l2": "working set smaller than L2 (warm)"},
+                "clocks": clocks, "gpu_launches": r["launches"] * 20, "e2e": None,
+                "roofline": {"kernel": "sparse gather dX/dW (conv_dx2_kernel, conv_dw2_kernel)", "bound": "alu",
+                             "achieved": r["fma_frac"] * fma_peak, "peak": fma_peak, "unit": "TFLOP/s", "frac": r["fma_frac"],
+                             "traffic": None, "peak_source": "measured: dependent fp32 FMA chains on every lane"},
+                "hbm_path": {"algorithmic_gb_per_step": r["algorithmic_mb"] / 1e3, "frac_of_measured_hbm": r["hbm_frac"], "peak": hbm_peak},
+                "dense_baseline": r["dense_ms"]}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     specs, name = layer_specs(args.config, args.batch)
     if args.only:
@@ -269,9 +423,10 @@ def main():
             dense_flops += L.dense_flops
             alg_bytes += algorithmic_bytes(L)
     lib = dbp.load_library()
-    import ctypes
 
-    ASYNC = dbp.DBP_DW_ASYNC        # dW of a layer may still run while the next layer is quantized; joined at the step's end
+    # dW of a layer may still run while the next layer is quantized (the layer below needs dX only); every dW
+    # is ordered into the stream before the step ends
+    FLAGS = 0 if args.sync_dw else dbp.DBP_DW_ASYNC
 
     def run_layer(L, d, X, W, dW, dX):
         code = 1 if L.dtype == "bf16" else 0
@@ -279,19 +434,19 @@ def main():
             B, N = d.shape
             rc = lib.dithered_linear_backward(ctx._h, d.data_ptr(), X.data_ptr(), W.data_ptr(), code,
                                               B, N, X.shape[1], L.seed, L.scale, None, None,
-                                              dW.data_ptr(), dX.data_ptr(), None, ASYNC)
+                                              dW.data_ptr(), dX.data_ptr(), None, FLAGS)
         else:
             B, Co, H, Wd = d.shape
             rc = lib.dithered_conv_backward(ctx._h, d.data_ptr(), X.data_ptr(), W.data_ptr(), code,
                                             B, X.shape[1], Co, H, Wd, L.k, 1, (L.k - 1) // 2, L.seed,
-                                            L.scale, None, None, dW.data_ptr(), dX.data_ptr(), None, ASYNC)
+                                            L.scale, None, None, dW.data_ptr(), dX.data_ptr(), None, FLAGS)
         if rc != 0:
-            raise RuntimeError(f"library call failed on {L.name}: {rc}")
+            raise RuntimeError(f"library call failed on {L.name}: {rc} {lib.dbp_last_error().decode()}")
 
     def step():
         for item in layers:
             run_layer(*item)
-        ctx.join()                  # every dW of the step is ordered into the stream before the step ends
+        ctx.join()
 
     def barrier():
         if world > 1:
@@ -300,7 +455,8 @@ def main():
 
     # Warm-up steps run with every kernel kind bracketed by events: that gives the per-kind table
     # and names the dominant kind. The events cost stream time, so the timed region brackets
-    # only the dominant kind (its duration is what the roofline line uses).
+    # only the dominant kind (its duration is what the roofline line uses). The dW kinds run on the
+    # context's second stream beside the others, so the kinds' times overlap and add up to more than the step.
     # The first warm-up step grows the context's workspaces (allocations) and is not profiled.
     t_warm = time.perf_counter()
     step()
@@ -317,6 +473,7 @@ def main():
     ctx.profile_select([top_kind])
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    launches0 = dbp.kernel_launches()
     t_begin = time.perf_counter()
     e0.record()
     for _ in range(args.steps):
@@ -324,6 +481,7 @@ def main():
     e1.record()
     barrier()
     t_end = time.perf_counter()
+    launches = dbp.kernel_launches() - launches0
     clocks = sampler.stop(t_begin, t_end, t_warm) if rank == 0 else None
     ms = e0.elapsed_time(e1) / args.steps
     prof_top = ctx.profile_read()
@@ -339,11 +497,14 @@ def main():
     host_ms = (time.perf_counter() - t0) * 1e3
     barrier()
 
-    # non-zero work actually done (for the arithmetic roofline of the sparse products)
+    # non-zero work actually done, and the dequantized gradients the dense comparison is fed
     nnz_flops = 0.0
+    dq = []
     for (L, d, X, W, dW, dX) in layers:
         q = dbp.nsd_quantize(ctx, d, L.seed, L.scale)
         nnz_flops += (q.nnz.item() / d.numel()) * L.dense_flops
+        if not args.no_dense and rank == 0:
+            dq.append((dbp.nsd_decode_dense(ctx, q, d.shape).float() * q.delta).to(d.dtype).contiguous())
     torch.cuda.synchronize()
     density = nnz_flops / dense_flops
 
@@ -374,67 +535,31 @@ def main():
     # ---- dense library backward on the same shapes (context, not the product path)
     dense = None
     if not args.no_dense and rank == 0:
-        import torch.nn.functional as F
-        def dense_step(allow_tf32):
-            torch.backends.cudnn.allow_tf32 = allow_tf32
-            torch.backends.cuda.matmul.allow_tf32 = allow_tf32
-            for (L, d, X, W, dW, dX) in layers:
-                if L.kind == "linear":
-                    torch.matmul(d.t(), X)
-                    torch.matmul(d, W)
-                else:
-                    p = (L.k - 1) // 2
-                    torch.ops.aten.convolution_backward(d, X, W, None, [1, 1], [p, p], [1, 1], False,
-                                                        [0, 0], 1, [True, True, False])
-        dense = {}
-        for label, tf32 in (("tf32_off", False), ("tf32_on", True)):
-            for _ in range(3):
-                dense_step(tf32)
-            torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            for _ in range(max(3, args.steps // 2)):
-                dense_step(tf32)
-            b.record()
-            torch.cuda.synchronize()
-            dms = a.elapsed_time(b) / max(3, args.steps // 2)
-            dense[label] = {"ms_per_step": dms, "gflops": dense_flops / (dms * 1e-3) / 1e9}
-        dense["what"] = "torch cuDNN/cuBLAS backward-data + backward-filter on the unquantized delta, same buffers"
+        fns = [dense_layer_fn(torch, L, g, X, W) for (L, d, X, W, dW, dX), g in zip(layers, dq)]
+        dt = dense_times(torch, fns, max(20, args.steps // 4))
+        dense = {k: {"ms_per_step": v, "gflops": dense_flops / (v * 1e-3) / 1e9} for k, v in dt.items()}
+        dense["what"] = ("torch cuDNN/cuBLAS backward-data + backward-filter (cudnn.benchmark autotuning) on the "
+                         "dequantized gradient Delta*q in the layers' dtype, same X and W buffers")
+        del fns, dq
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    hbm_peak, peak_src = measured_peaks()
     prof = {k: (v[0] / nprof, v[1] / nprof) for k, v in prof_all.items()}   # per step
-    kern = {k: {"ms_per_step": v[0], "launches_per_step": v[1], "measured": "warm-up steps, every kind bracketed by events"}
+    kern = {k: {"ms_per_step": v[0], "launches_per_step": v[1],
+                "measured": "warm-up steps, every kind bracketed by events (dW kinds run beside the others: times overlap)"}
             for k, v in prof.items() if v[1]}
     # algorithmic work of every kernel kind over one step; a layer counts as dense when the
     # library would run it so at this density (bf16, 1x1/linear or 3x3, channels % 8 == 0)
     e = 2 if layers[0][0].dtype == "bf16" else 4
     dense_on = prof["dx_dense"][1] > 0
     is_dense = lambda L: (dense_on and L.dtype == "bf16" and L.X.shape[1] % 8 == 0 and L.delta.shape[1] % 8 == 0)
-    # kernels launched in the timed region: statistics and quantize, then for a dense layer the
-    # dX product (after the weight re-layout for 3x3) and the dW product with its split-K sum,
-    # for a sparse layer the weight re-layout, dX and dW
-    # kernels launched in the timed region, per layer: statistics and quantize; then, dense 1x1:
-    # dX, (copy of X to padded planes when H*W % 8 != 0), dW, split-K sum; dense 3x3: weight
-    # re-layout, dX, dW, split-K sum; sparse: weight re-layout, dX, dW
-    tma = lambda L: is_dense(L) and L.kind == "conv" and L.k == 1 and L.X.shape[2] * L.X.shape[3] >= 16
-    per_step = 0
-    for (L, d, X, W, dW, dX) in layers:
-        if tma(L):
-            per_step += 2 + 1 + (1 if (L.X.shape[2] * L.X.shape[3]) % 8 else 0) + 2
-        elif is_dense(L):
-            per_step += 2 + (2 if (L.kind == "conv" and L.k == 3) else 1) + 2
-        else:
-            per_step += 2 + 2 + 1
-    launches = per_step * args.steps
     work = {k: 0.0 for k in ("statistics", "quantize", "dx", "dw", "dx_dense", "dw_dense")}
     for (L, d, X, W, dW, dX) in layers:
         nd, nx, nw = d.numel(), X.numel(), W.numel()
-        cb = 2 if tma(L) else 1                                        # bytes per code the product kernels read
+        cb = 2 if is_dense(L) else 1                                   # bytes per code the product kernels read
         work["statistics"] += nd * e                                   # bytes
         work["quantize"] += nd * (e + cb)                              # bytes: delta read, codes written
         if is_dense(L):
@@ -451,16 +576,19 @@ def main():
     if top in ("dx", "dw"):
         ach = work[top] / t_s / 1e12
         roof = {"kernel": f"sparse {top} (conv_{top}2_kernel)", "bound": "alu", "achieved": ach,
-                "peak": FMA_PEAK_TFLOPS, "unit": "TFLOP/s", "frac": ach / FMA_PEAK_TFLOPS, "traffic": None,
-                "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 flop x 1.965 GHz",
+                "peak": fma_peak, "unit": "TFLOP/s", "frac": ach / fma_peak, "traffic": None,
+                "peak_source": "measured: dependent fp32 FMA chains on every lane (dbp_measure_fma_peak)",
                 "note": "non-zero-code FMAs only (2*nnz*K_eff flops per product), summed over the layers that use it"}
     else:
         ach = work[top] / t_s / 1e9
-        roof = {"kernel": {"dx_dense": "tensor-core dX (tma_dx_kernel for 1x1, tc3_dx_shift_kernel for 3x3)",
-                           "dw_dense": "tensor-core dW (tma_dw_kernel for 1x1, tc3_dw_shift_kernel for 3x3, + split-K sums)"}.get(top, top + "_kernel"),
+        traffic = NCU_DRAM_BYTES_PER_STEP.get(top) if not (args.only or args.single or args.batch) else None
+        roof = {"kernel": {"dx_dense": "tensor-core dX (tma_dx_kernel for 1x1, tc3_tma_dx_kernel for 3x3)",
+                           "dw_dense": "tensor-core dW (tma_dw_kernel for 1x1, tc3_tma_dw_kernel + tc3_dw_finish_kernel for 3x3)",
+                           "quantize": "NSD quantizer (quantize_dense_kernel for 1x1, quantize_nhwc_kernel for 3x3)"}.get(top, top + "_kernel"),
                 "bound": "hbm", "achieved": ach, "peak": hbm_peak, "unit": "GB/s", "frac": ach / hbm_peak,
-                "traffic": None, "peak_source": peak_src + " (MEASURED_PEAKS.json hbm_gbs)",
-                "note": "algorithmic bytes summed over the layers that use it / summed launch time"}
+                "traffic": traffic, "peak_source": peak_src + " (MEASURED_PEAKS.json hbm_gbs)",
+                "note": "algorithmic bytes summed over the layers that use it / summed launch time of the kind inside the timed "
+                        "region; traffic: DRAM bytes of the kind's launches in one step (ncu, see profiles/)"}
     for k in work:
         if k in kern:
             kern[k]["work_per_step"] = work[k]
@@ -472,13 +600,17 @@ def main():
         "vs_baseline": None, "dtype": "bf16 storage, f32 accumulate" if layers[0][0].dtype == "bf16" else "f32",
         "data": "synthetic",
         "config": {"workload": name, "layers_per_step": len(layers), "l2": "inputs larger than L2 (distinct buffers per layer instance)"
-                   if alg_bytes > 2.5e8 else "working set smaller than L2 (warm)", "nsd_density": density},
+                   if alg_bytes > 2.5e8 else "working set smaller than L2 (warm)", "nsd_density": density,
+                   "dw": "joined per call" if args.sync_dw else "DBP_DW_ASYNC, joined at the end of the step"},
         "clocks": clocks, "gpu_launches": launches, "host_enqueue_ms_per_step": host_ms, "e2e": e2e,
         "roofline": roof,
         "hbm_path": {"algorithmic_gb_per_step": alg_bytes / 1e9, "achieved_gbs": path_gbs,
                      "frac_of_measured_hbm": path_gbs / hbm_peak, "peak": hbm_peak, "peak_source": peak_src},
+        "fma_peak_tflops": fma_peak,
         "kernels": kern, "dense_baseline": dense,
     }
+    if not args.no_others and world == 1 and args.config == 5 and not (args.only or args.single):
+        out["other_configs"] = {str(c): small_config(torch, dbp, ctx, c, hbm_peak, fma_peak) for c in (1, 2, 3, 4)}
     if not args.no_cpu and world == 1:
         v, dt, what, cores = oracle_sample(args.config)
         out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what,

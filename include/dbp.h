@@ -64,9 +64,10 @@ typedef enum {
  * Density crossover (Section 3.4: the sparse products cost O(p_nz m k n), a dense product
  * O(m k n) at a much higher arithmetic rate on tensor cores). Without a FORCE flag a layer
  * that the dense path supports uses it when the context's estimate of p_nz exceeds
- * `crossover`; the estimate is the density measured by the context's most recent finished
- * quantization (read back asynchronously, so no call waits for it; 1.0 before the first).
- * crossover >= 1 disables the dense path, crossover <= 0 always prefers it.
+ * `crossover`; the estimate is the density last measured on a layer of the same shape on this
+ * context (read back asynchronously, so no call waits for it; 1.0, i.e. dense, until the first
+ * measurement of that shape has arrived). crossover >= 1 disables the dense path, crossover <= 0
+ * always prefers it.
  */
 int dbp_set_crossover(dbp_ctx *ctx, float crossover);
 
@@ -108,6 +109,13 @@ typedef struct dbp_sparse {
 int dbp_create(dbp_ctx **out, int device, void *cuda_stream);
 int dbp_destroy(dbp_ctx *ctx);
 int dbp_set_stream(dbp_ctx *ctx, void *cuda_stream);
+/* Kernels the library has launched in this process so far (every launch is counted). */
+long long dbp_kernel_launches(void);
+
+/* fp32 FMA throughput of the context's device in TFLOP/s, measured with dependent FMA chains on
+ * every lane (the arithmetic ceiling of the sparse gather kernels). Synchronises. */
+int dbp_measure_fma_peak(dbp_ctx *ctx, double *tflops);
+
 /* Makes the context's stream wait for every dW computation that earlier DBP_DW_ASYNC calls left
  * running (a stream-ordered join: nothing blocks on the host). */
 int dbp_join(dbp_ctx *ctx);

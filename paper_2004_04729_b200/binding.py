@@ -21,7 +21,7 @@ EXPORTED_SYMBOLS = [
     "dithered_linear_backward", "dithered_conv_backward", "dithered_linear_backward_host",
     "dithered_conv_backward_host", "dbp_relu_backward", "dbp_maxpool2x2_backward",
     "dbp_profile_enable", "dbp_profile_select", "dbp_profile_read", "dbp_set_crossover", "nsd_step_size_noalloc",
-    "dbp_last_step", "dbp_layer_seed", "dbp_selftest_bounded_wait", "dbp_last_error", "dbp_wait_stats", "dbp_join",
+    "dbp_last_step", "dbp_layer_seed", "dbp_selftest_bounded_wait", "dbp_last_error", "dbp_wait_stats", "dbp_join", "dbp_kernel_launches", "dbp_measure_fma_peak",
 ]
 
 KERNEL_KINDS = ["statistics", "quantize", "weight_taps", "dx", "dw", "db", "decode", "glue",
@@ -85,13 +85,16 @@ def load_library():
     lib.dbp_profile_read.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ll)]
     lib.dbp_selftest_bounded_wait.argtypes = [vp, ll]
     lib.dbp_join.argtypes = [vp]
+    lib.dbp_kernel_launches.argtypes = []
+    lib.dbp_kernel_launches.restype = ll
+    lib.dbp_measure_fma_peak.argtypes = [vp, ctypes.POINTER(ctypes.c_double)]
     lib.dbp_wait_stats.argtypes = [vp, ctypes.POINTER(ull), i32]
     lib.dbp_last_step.argtypes = [vp, ctypes.POINTER(f32), ctypes.POINTER(ll)]
     lib.dbp_layer_seed.argtypes = [ull, i32]
     lib.dbp_relu_backward.argtypes = [vp, vp, vp, vp, ll]
     lib.dbp_maxpool2x2_backward.argtypes = [vp, vp, vp, vp, ll, ll, ll]
     for name in EXPORTED_SYMBOLS:
-        if name not in ("dbp_status_string", "dbp_layer_seed", "dbp_last_error"):
+        if name not in ("dbp_status_string", "dbp_layer_seed", "dbp_last_error", "dbp_kernel_launches"):
             getattr(lib, name).restype = i32
     lib.dbp_layer_seed.restype = ull
     lib.dbp_last_error.argtypes = []
@@ -170,6 +173,12 @@ class Context:
         out = (ctypes.c_ulonglong * 8)()
         _check(load_library().dbp_wait_stats(self._h, out, int(reset)), "dbp_wait_stats")
         return list(out)
+
+    def measure_fma_peak(self) -> float:
+        """fp32 FMA throughput of the device in TFLOP/s (dependent FMA chains on every lane)."""
+        v = ctypes.c_double()
+        _check(load_library().dbp_measure_fma_peak(self._h, ctypes.byref(v)), "dbp_measure_fma_peak")
+        return v.value
 
     def join(self):
         """Orders every dW left running by DBP_DW_ASYNC calls into the context's stream."""
@@ -367,29 +376,36 @@ def nsd_step_size_noalloc(delta: torch.Tensor, scale: float, out: torch.Tensor,
             _ptr(out), ctypes.c_void_p(s.cuda_stream)), "nsd_step_size_noalloc")
 
 
+def kernel_launches() -> int:
+    """Kernels the library has launched in this process so far."""
+    return int(load_library().dbp_kernel_launches())
+
+
 def layer_seed(seed: int, layer: int) -> int:
     """Seed of layer `layer` of a network whose backward pass was given `seed` (C: dbp_layer_seed)."""
     return int(load_library().dbp_layer_seed(int(seed) & (2 ** 64 - 1), int(layer)))
 
 
 def network_backward(ctx: Context, kinds, Xs, Ws, relu_masks, pool_argmax, delta_out, scale: float,
-                     seed: int, keep_delta_z: bool = False, first_layer_dX: bool = False):
+                     seed: int, keep_delta_z: bool = False, first_layer_dX: bool = False,
+                     with_sparse: bool = True, flags: int = 0):
     """Dithered backward pass of a feed-forward network (device tensors, forward order):
     for l = L..1: delta_z = delta_a (.) relu'(z); NSD; dW_l, and delta_a of the layer below
     from the QUANTIZED gradient; 2x2 max-pool routing where a pool follows layer l-1.
     Returns one dict per layer with dW, dX (None for layer 0 unless asked), Delta, nnz, and
-    optionally the delta_z that was quantized and its SparseGradient."""
+    optionally the delta_z that was quantized and its SparseGradient. with_sparse=False asks for
+    no sparse structure (Delta and nnz are then None; the library runs its leaner quantizer)."""
     L = len(kinds)
     res = [None] * L
     delta_a = delta_out
     for l in range(L - 1, -1, -1):
         dz = delta_a if relu_masks[l] is None else relu_backward(ctx, delta_a, relu_masks[l])
-        q = SparseGradient(dz.numel(), ctx.device)
+        q = SparseGradient(dz.numel(), ctx.device) if with_sparse else None
         fn = dithered_linear_backward if kinds[l] == "linear" else dithered_conv_backward
         need_dx = l > 0 or first_layer_dX
         r = fn(ctx, dz, Xs[l], Ws[l], layer_seed(seed, l), scale, q_out=q,
-               need_dX=need_dx)
-        r.update(Delta=q.delta, nnz=q.nnz)
+               need_dX=need_dx, flags=flags)
+        r.update(Delta=q.delta if q else None, nnz=q.nnz if q else None)
         if keep_delta_z:
             r.update(delta_z=dz, q=q)
         res[l] = r

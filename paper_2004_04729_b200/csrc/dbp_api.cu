@@ -3,13 +3,17 @@
 
 #include "dbp_internal.cuh"
 
+#include <atomic>
 #include <cstdio>
 
 namespace dbp {
 
 namespace {
 thread_local char g_last_error[192] = "";
+std::atomic<long long> g_launches{0};
 }
+
+void note_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
 int fail_cuda(const char *what, cudaError_t e) {
     std::snprintf(g_last_error, sizeof(g_last_error), "%s: %s", what, cudaGetErrorString(e));
@@ -155,14 +159,25 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     if (cudaStreamIsCapturing(ctx->stream, &cap) != cudaSuccess) return DBP_ECUDA;
     const bool capturing = cap != cudaStreamCaptureStatusNone;
     // pick up the density of the last finished quantization, if its read-back has landed
+    // The estimate that decides is the density last measured on a layer of THIS shape (1.0, i.e. dense, until
+    // one has been read back): a layer's own sparsity level picks its path, not its neighbour's.
+    const unsigned long long shape_key =
+        ((((((static_cast<unsigned long long>(s.B) * 1000003ull + s.Cin) * 1000003ull + s.Cout) * 1000003ull + s.H) * 1000003ull + s.W) * 8ull +
+          s.k) * 2ull + io);
     if (!capturing && ctx->nnz_pending && cudaEventQuery(ctx->nnz_event) == cudaSuccess) {
-        ctx->density_estimate = static_cast<float>(static_cast<double>(*ctx->nnz_host) /
-                                                   static_cast<double>(ctx->nnz_host_numel));
+        const float dns = static_cast<float>(static_cast<double>(*ctx->nnz_host) / static_cast<double>(ctx->nnz_host_numel));
+        bool found = false;
+        for (auto &e : ctx->densities)
+            if (e.key == ctx->nnz_host_key) { e.density = dns; found = true; }
+        if (!found) ctx->densities.push_back({ctx->nnz_host_key, dns});
         ctx->nnz_pending = false;
     }
     cudaGetLastError();   // cudaErrorNotReady from the query is not an error
+    float density_estimate = 1.0f;
+    for (const auto &e : ctx->densities)
+        if (e.key == shape_key) density_estimate = e.density;
     const bool dense = can_dense && !(flags & DBP_FORCE_SPARSE) &&
-                       ((flags & DBP_FORCE_DENSE) || ctx->density_estimate > ctx->crossover);
+                       ((flags & DBP_FORCE_DENSE) || density_estimate > ctx->crossover);
     // which dense kernels run: the TMA-fed ones read bf16 code planes, the others int8 codes
     const bool dx_tma = dense && dX && tma_dx_supported(s, io);
     const bool dw_tma = dense && dW && tma_dw_supported(s, io);
@@ -185,6 +200,7 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     if (rc) return rc;
     if (!capturing && !ctx->nnz_pending && ctx->nnz_host && ctx->nnz_event) {
         ctx->nnz_host_numel = numel;
+        ctx->nnz_host_key = shape_key;
         if (cudaMemcpyAsync(ctx->nnz_host, &ctx->state->nnz, sizeof(unsigned long long), cudaMemcpyDeviceToHost,
                             ctx->stream) == cudaSuccess &&
             cudaEventRecord(ctx->nnz_event, ctx->stream) == cudaSuccess)
@@ -322,6 +338,15 @@ int dbp_create(dbp_ctx **out, int device, void *cuda_stream) {
 }
 
 const char *dbp_last_error(void) { return g_last_error; }
+
+long long dbp_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int dbp_measure_fma_peak(dbp_ctx *ctx, double *tflops) {
+    if (!ctx || !tflops) return DBP_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DBP_ECUDA;
+    return measure_fma_peak(ctx, tflops);
+}
 
 int dbp_join(dbp_ctx *ctx) {
     if (!ctx) return DBP_EINVAL;

@@ -72,7 +72,10 @@ struct dbp_ctx {
     cudaEvent_t ev_x_up = nullptr, ev_dx_done = nullptr;
     cudaEvent_t hook_after_dx = nullptr, hook_before_dw = nullptr;   // set only during a *_host call
     float crossover = 0.03f;            // density above which the dense path is preferred
-    float density_estimate = 1.0f;      // density of the latest finished quantization
+    // densities measured so far, by layer shape (the path choice of a call uses its own shape's entry)
+    struct DensityEntry { unsigned long long key; float density; };
+    std::vector<DensityEntry> densities;
+    unsigned long long nnz_host_key = 0;         // shape whose read-back is in flight
     unsigned long long *nnz_host = nullptr;   // pinned: asynchronous read-back of nnz
     long long nnz_host_numel = 0;
     cudaEvent_t nnz_event = nullptr;
@@ -161,6 +164,8 @@ int launch_maxpool_backward(dbp_ctx *ctx, const float *g, const int8_t *argmax, 
 
 // ---- selftest.cu
 int launch_bounded_wait_selftest(dbp_ctx *ctx, long long budget);
+// fp32 FMA throughput of the device (dependent chains on every lane of every SM), TFLOP/s
+int measure_fma_peak(dbp_ctx *ctx, double *tflops);
 
 // Brackets one kernel launch with events while profiling is on.
 struct KernelTimer {
@@ -208,6 +213,9 @@ inline long long choose_split(long long tiles, long long kunits, int sms, long l
 int fail_cuda(const char *what, cudaError_t e);
 inline int fail_cuda(const char *what) { return fail_cuda(what, cudaGetLastError()); }
 
+// Every kernel launch of the library passes here (a process-wide count, read by dbp_kernel_launches).
+void note_launch();
+
 inline int cuda_ok(cudaError_t e) { return e == cudaSuccess ? DBP_OK : fail_cuda("launch", e); }
 
 // Programmatic dependent launch: a kernel launched with launch_chained may become resident while
@@ -232,6 +240,7 @@ inline cudaError_t launch_chained(void (*kern)(KArgs...), dim3 grid, dim3 block,
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    note_launch();
     return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 #endif

@@ -391,6 +391,7 @@ int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long nume
     const long long zn = zero ? static_cast<long long>(zero_bytes / 16) : 0;
     if (!(scale > 0.f)) {
         if (zero && cudaMemsetAsync(zero, 0, zero_bytes, ctx->stream) != cudaSuccess) return fail_cuda("clearing dW");
+        note_launch();
         set_step_kernel<<<1, 1, 0, ctx->stream>>>(delta_in, ctx->state, delta_out, nnz_out);
         return cuda_ok(cudaGetLastError());
     }
@@ -417,13 +418,13 @@ int launch_quantize(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
     const long long cap = static_cast<long long>(ctx->sm_count) * 8;
     if (blocks > cap) blocks = cap;
     if (dtype == DBP_F32)
-        quantize_kernel<float><<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(
+        { note_launch(); quantize_kernel<float><<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(
             static_cast<const float *>(delta), numel, seed, delta_p, bitmap, offsets, values, dense,
-            ctx->state, nnz_out);
+            ctx->state, nnz_out); }
     else
-        quantize_kernel<__nv_bfloat16><<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(
+        { note_launch(); quantize_kernel<__nv_bfloat16><<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(
             static_cast<const __nv_bfloat16 *>(delta), numel, seed, delta_p, bitmap, offsets, values,
-            dense, ctx->state, nnz_out);
+            dense, ctx->state, nnz_out); }
     return cuda_ok(cudaGetLastError());
 }
 
@@ -433,6 +434,7 @@ int launch_decode(dbp_ctx *ctx, const uint32_t *bitmap, const uint16_t *offsets,
     long long blocks = (nseg + kThreads / 32 - 1) / (kThreads / 32);
     const long long cap = static_cast<long long>(ctx->sm_count) * 8;
     if (blocks > cap) blocks = cap;
+    note_launch();
     decode_kernel<<<static_cast<unsigned>(blocks), kThreads, 0, ctx->stream>>>(bitmap, offsets, values,
                                                                             numel, dense);
     return cuda_ok(cudaGetLastError());

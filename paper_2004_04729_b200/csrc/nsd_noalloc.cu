@@ -10,6 +10,11 @@
 
 #include "dbp.h"
 
+namespace dbp {
+void note_launch();     // the library's launch count (dbp_kernel_launches)
+}
+using dbp::note_launch;
+
 namespace {
 
 constexpr int kThreads = 256;
@@ -169,10 +174,10 @@ extern "C" int nsd_step_size_noalloc(const void *delta, int dtype, long long num
     if (blocks < 1) blocks = 1;
     if (blocks > kMaxBlocks) blocks = kMaxBlocks;
     if (dtype == DBP_F32)
-        step_size_kernel<float><<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(
-            static_cast<const float *>(delta), numel, scale, sc, delta_out);
+        { note_launch(); step_size_kernel<float><<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(
+            static_cast<const float *>(delta), numel, scale, sc, delta_out); }
     else
-        step_size_kernel<__nv_bfloat16><<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(
-            static_cast<const __nv_bfloat16 *>(delta), numel, scale, sc, delta_out);
+        { note_launch(); step_size_kernel<__nv_bfloat16><<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(
+            static_cast<const __nv_bfloat16 *>(delta), numel, scale, sc, delta_out); }
     return cudaGetLastError() == cudaSuccess ? DBP_OK : DBP_ECUDA;
 }

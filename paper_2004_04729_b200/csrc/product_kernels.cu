@@ -357,14 +357,14 @@ int launch_weight_taps(dbp_ctx *ctx, const void *W, int dtype, const ConvShape &
     const long long n = s.Cout * s.Cin * KK;
     const int blocks = blocks_for(n, 256, ctx->sm_count * 8);
     if (dtype == DBP_F32)
-        weight_taps_kernel<float, float><<<blocks, 256, 0, ctx->stream>>>(
-            static_cast<const float *>(W), static_cast<float *>(w_taps), s.Cout, s.Cin, KK);
+        { note_launch(); weight_taps_kernel<float, float><<<blocks, 256, 0, ctx->stream>>>(
+            static_cast<const float *>(W), static_cast<float *>(w_taps), s.Cout, s.Cin, KK); }
     else if (to_f32)
-        weight_taps_kernel<__nv_bfloat16, float><<<blocks, 256, 0, ctx->stream>>>(
-            static_cast<const __nv_bfloat16 *>(W), static_cast<float *>(w_taps), s.Cout, s.Cin, KK);
+        { note_launch(); weight_taps_kernel<__nv_bfloat16, float><<<blocks, 256, 0, ctx->stream>>>(
+            static_cast<const __nv_bfloat16 *>(W), static_cast<float *>(w_taps), s.Cout, s.Cin, KK); }
     else
-        weight_taps_kernel<__nv_bfloat16, __nv_bfloat16><<<blocks, 256, 0, ctx->stream>>>(
-            static_cast<const __nv_bfloat16 *>(W), static_cast<__nv_bfloat16 *>(w_taps), s.Cout, s.Cin, KK);
+        { note_launch(); weight_taps_kernel<__nv_bfloat16, __nv_bfloat16><<<blocks, 256, 0, ctx->stream>>>(
+            static_cast<const __nv_bfloat16 *>(W), static_cast<__nv_bfloat16 *>(w_taps), s.Cout, s.Cin, KK); }
     return cuda_ok(cudaGetLastError());
 }
 
@@ -377,6 +377,7 @@ static int launch_dx_t(dbp_ctx *ctx, const DxParams &p, size_t smem) {
     }
     const int CI_T = 32 * VEC;
     dim3 grid(static_cast<unsigned>(p.B * p.tiles_y * p.tiles_x), static_cast<unsigned>((p.Cin + CI_T - 1) / CI_T));
+    note_launch();
     kern<<<grid, 256, smem, ctx->stream>>>(p);
     return cuda_ok(cudaGetLastError());
 }
@@ -420,6 +421,7 @@ static int launch_dw_t(dbp_ctx *ctx, const DwParams &p, size_t smem, dim3 grid) 
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return DBP_ECUDA;
     }
+    note_launch();
     kern<<<grid, 512, smem, ctx->stream>>>(p);
     return cuda_ok(cudaGetLastError());
 }
@@ -464,18 +466,21 @@ int launch_conv_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, int dtype,
 
 int launch_bias_grad(dbp_ctx *ctx, const int8_t *codes, const float *delta_p, const ConvShape &s,
                      float *db) {
+    note_launch();
     bias_grad_kernel<<<static_cast<unsigned>(s.Cout), 256, 0, ctx->stream>>>(
         codes, delta_p, static_cast<int>(s.B), static_cast<int>(s.Cout), s.H * s.W, db);
     return cuda_ok(cudaGetLastError());
 }
 
 int launch_relu_backward(dbp_ctx *ctx, const float *da, const uint8_t *mask, float *dz, long long n) {
+    note_launch();
     relu_backward_kernel<<<blocks_for(n, 256, ctx->sm_count * 8), 256, 0, ctx->stream>>>(da, mask, dz, n);
     return cuda_ok(cudaGetLastError());
 }
 
 int launch_maxpool_backward(dbp_ctx *ctx, const float *g, const int8_t *argmax, float *out,
                             long long planes, long long h, long long w) {
+    note_launch();
     maxpool_backward_kernel<<<blocks_for(planes * h * w * 4, 256, ctx->sm_count * 8), 256, 0, ctx->stream>>>(
         g, argmax, out, planes, h, w);
     return cuda_ok(cudaGetLastError());

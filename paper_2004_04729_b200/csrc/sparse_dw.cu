@@ -290,6 +290,7 @@ int launch_one(dbp_ctx *ctx, Dw2Params &p, const ConvShape &s) {
         return DBP_ECUDA;
     dim3 grid(static_cast<unsigned>((s.Cout + CO_T - 1) / CO_T), static_cast<unsigned>((s.Cin + CI_T - 1) / CI_T),
               static_cast<unsigned>(splits));
+    note_launch();
     kern<<<grid, kThreads, smem, ctx->stream>>>(p);
     return cuda_ok(cudaGetLastError());
 }

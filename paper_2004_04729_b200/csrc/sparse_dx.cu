@@ -281,6 +281,7 @@ int launch_one(dbp_ctx *ctx, Dx2Params &p, const ConvShape &s) {
     const long long tiles = KS == 1 ? (p.total_rows + PT - 1) / PT
                                     : s.B * p.tiles_y * p.tiles_x;
     dim3 grid(static_cast<unsigned>(tiles), static_cast<unsigned>((s.Cin + CI_T - 1) / CI_T));
+    note_launch();
     kern<<<grid, kWarps * 32, smem, ctx->stream>>>(p);
     return cuda_ok(cudaGetLastError());
 }

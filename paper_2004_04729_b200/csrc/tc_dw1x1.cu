@@ -351,6 +351,7 @@ int run(dbp_ctx *ctx, const DwP &p, dim3 grid, size_t smem) {
     if (cudaFuncSetAttribute(tc_dw_async_kernel<NT, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(smem)) != cudaSuccess)
         return DBP_ECUDA;
+    note_launch();
     tc_dw_async_kernel<NT, G><<<grid, kThreadsDw, smem, ctx->stream>>>(p);
     return cuda_ok(cudaGetLastError());
 }
@@ -391,8 +392,8 @@ int launch_tc_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, const float *
                                                                       : run_g<64>(ctx, p, grid, smem, slab);
     if (rc) return rc;
     const long long n4 = static_cast<long long>(nw) / 4;          // Cout * Cin % 4 == 0
-    tc_dw_sum_kernel<<<static_cast<unsigned>((n4 + 31) / 32), 256, 0, ctx->stream>>>(
-        reinterpret_cast<const float4 *>(p.partials), static_cast<int>(split), n4, delta_p, reinterpret_cast<float4 *>(dW));
+    { note_launch(); tc_dw_sum_kernel<<<static_cast<unsigned>((n4 + 31) / 32), 256, 0, ctx->stream>>>(
+        reinterpret_cast<const float4 *>(p.partials), static_cast<int>(split), n4, delta_p, reinterpret_cast<float4 *>(dW)); }
     return cuda_ok(cudaGetLastError());
 }
 

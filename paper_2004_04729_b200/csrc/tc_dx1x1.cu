@@ -369,6 +369,7 @@ int run(dbp_ctx *ctx, const DxP &p, dim3 grid, size_t smem) {
     if (cudaFuncSetAttribute(tc_dx_async_kernel<NT, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(smem)) != cudaSuccess)
         return DBP_ECUDA;
+    note_launch();
     tc_dx_async_kernel<NT, G><<<grid, kThreadsDx, smem, ctx->stream>>>(p);
     return cuda_ok(cudaGetLastError());
 }
