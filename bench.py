@@ -301,7 +301,11 @@ def small_config(torch, dbp, ctx, config, hbm_peak, fma_peak):
         masks = [None if m is None else cu(m.astype(np.uint8)) for m in c.relu_mask]
         pools = [cu(a) for a in c.pool_argmax]
         dout = cu(c.delta_out)
-        run = lambda: dbp.network_backward(ctx, c.kinds, Xs, Ws, masks, pools, dout, c.scale, 0, with_sparse=False)
+        def run():
+            # training order: a layer's dW may still run while the layer below is quantized; joined at the end
+            dbp.network_backward(ctx, c.kinds, Xs, Ws, masks, pools, dout, c.scale, 0, with_sparse=False,
+                                 flags=dbp.DBP_DW_ASYNC)
+            ctx.join()
         res = dbp.network_backward(ctx, c.kinds, Xs, Ws, masks, pools, dout, c.scale, 0, keep_delta_z=True)
         torch.cuda.synchronize()
         flops, nbytes = chain_flops(c), chain_bytes(c)

@@ -49,8 +49,9 @@ typedef enum {
 /* flags for the backward calls */
 #define DBP_FORCE_SPARSE 1u /* always use the sparse gather kernels */
 #define DBP_FORCE_DENSE  2u /* always use the dense tensor-core path; DBP_EUNSUPPORTED where it
-                               does not exist (it covers bf16 linear, 1x1 and 3x3 layers whose channel
-                               counts are multiples of 8; 3x3 images up to 62 wide) */
+                               does not exist (it covers bf16 linear and 1x1 layers and bf16 or fp32 3x3
+                               layers, channel counts multiples of 8, 3x3 images up to 62 wide; fp32
+                               operands enter the tensor cores as two bf16 pieces each) */
 #define DBP_DX_F32       4u /* with io = DBP_BF16: write dX as fp32 instead of bf16 */
 #define DBP_DW_ASYNC     8u /* dense path with both dW and dX asked for: the call returns with dX (and db)
                                ordered on the context's stream as usual, while dW is still being computed on

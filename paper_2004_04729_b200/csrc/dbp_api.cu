@@ -217,7 +217,7 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
             KernelTimer t(ctx, DBP_K_DX_DENSE);
             const bool dx_bf16 = (io == DBP_BF16) && !(flags & DBP_DX_F32);
             rc = dx_tma ? launch_tma_dx(ctx, codes16, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout)
-                 : t3   ? launch_tc3_tma_dx(ctx, codes_n, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout)
+                 : t3   ? launch_tc3_tma_dx(ctx, codes_n, W, io, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout)
                         : launch_tc_dx(ctx, codes, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout);
             if (rc) return rc;
         }
@@ -228,7 +228,7 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
         if (dW && !rc) {
             KernelTimer t(ctx, DBP_K_DW_DENSE);
             rc = dw_tma ? launch_tma_dw(ctx, codes16, X, delta_p, s, dW, &ctx->state->tc_timeout)
-                 : t3   ? launch_tc3_tma_dw(ctx, codes_n, X, delta_p, s, dW, &ctx->state->tc_timeout)
+                 : t3   ? launch_tc3_tma_dw(ctx, codes_n, X, io, delta_p, s, dW, &ctx->state->tc_timeout)
                         : launch_tc_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout);
         }
         ctx->stream = caller;

@@ -151,9 +151,10 @@ int launch_pad_planes(dbp_ctx *ctx, const void *in, void *out, long long planes,
 int launch_dw_sum(dbp_ctx *ctx, const float *partials, int nsplit, long long nw, const float *delta_p, float *dW);
 // ---- tc3_tma_dx.cu / tc3_tma_dw.cu: 3x3 products with TMA-fed operands; codes as bf16 [B][H*W][Cout]
 bool tc3_tma_supported(const ConvShape &s, int io);
-int launch_tc3_tma_dx(dbp_ctx *ctx, const void *codes_nhwc, const void *W, const float *delta_p,
+// io: the operands' type; fp32 weights / activations are split into two bf16 pieces on the way in
+int launch_tc3_tma_dx(dbp_ctx *ctx, const void *codes_nhwc, const void *W, int io, const float *delta_p,
                       const ConvShape &s, void *dX, bool dx_bf16, int *err_flag);
-int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, const float *delta_p,
+int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, int io, const float *delta_p,
                       const ConvShape &s, float *dW, int *err_flag);
 int launch_bias_grad(dbp_ctx *ctx, const int8_t *codes, const float *delta_p, const ConvShape &s,
                      float *db);

@@ -39,6 +39,7 @@ constexpr int kMaxNX = 6;
 
 struct Dw3T {
     int Cin, Cout, W, HW;
+    int code_batch;               // images of the code tensor (the activations may hold two pieces of every image, one after the other)
     int SEG;                      // positions per segment (multiple of 64)
     int segs_per_img;
     long long nseg, per_split;
@@ -128,7 +129,7 @@ tc3_tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 for (int pn = 0; pn < NP; ++pn)
                     for (int l = 0; l < p.nload; ++l)
                         tma_load_3d(dst + pn * p.panel_bytes + l * p.rows_box * 128, &map_q, co0 + 64 * pn,
-                                    u0 - halo + l * p.rows_box, b, &pipe.q_full[buf]);
+                                    u0 - halo + l * p.rows_box, b % p.code_batch, &pipe.q_full[buf]);
             }
             report_wait(p.stats, 3, waited);
         }
@@ -345,14 +346,37 @@ tc3_dw_finish_kernel(float *__restrict__ acc, const float *__restrict__ delta_p,
     }
 }
 
+// fp32 activations [planes][HW] -> two bf16 tensors of the same shape, one after the other, rows padded to
+// `pitch` (a multiple of 8): the values rounded to bf16 and what that rounding left over, rounded again.
+// The two pieces add up to the fp32 value to within 2^-18 of it.
+__global__ void __launch_bounds__(256)
+x_split_kernel(const float *__restrict__ X, __nv_bfloat16 *__restrict__ out, long long planes, int HW, int pitch) {
+    chain_wait();
+    chain_release();
+    const long long n = planes * pitch;
+    for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += gridDim.x * 256ll) {
+        const long long pl = i / pitch;
+        const int pp = static_cast<int>(i - pl * pitch);
+        __nv_bfloat16 hi = __float2bfloat16_rn(0.f), lo = hi;
+        if (pp < HW) {
+            const float x = __ldg(X + pl * HW + pp);
+            hi = __float2bfloat16_rn(x);
+            lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+        }
+        out[i] = hi;
+        out[n + i] = lo;
+    }
+}
+
 int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 }  // namespace
 
 // DBP_EUNSUPPORTED: the shape does not fit (the caller uses another kernel)
-int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, const float *delta_p,
+int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, int io, const float *delta_p,
                       const ConvShape &s, float *dW, int *err_flag) {
-    if (!tc3_tma_supported(s, DBP_BF16)) return DBP_EUNSUPPORTED;
+    if (!tc3_tma_supported(s, io)) return DBP_EUNSUPPORTED;
+    const int pieces = io == DBP_F32 ? 2 : 1;
     const long long HW = s.H * s.W;
     Dw3T p{};
     p.Cin = static_cast<int>(s.Cin); p.Cout = static_cast<int>(s.Cout); p.W = static_cast<int>(s.W); p.HW = static_cast<int>(HW);
@@ -379,7 +403,8 @@ int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, const
     }
     if (smem == 0) return DBP_EUNSUPPORTED;
     p.segs_per_img = (p.HW + p.SEG - 1) / p.SEG;
-    p.nseg = s.B * p.segs_per_img;
+    p.code_batch = static_cast<int>(s.B);
+    p.nseg = s.B * pieces * p.segs_per_img;
     const long long tiles = static_cast<long long>(p.ci_tiles) * p.co_tiles * 3;
     const long long nsplit = choose_split(tiles, p.nseg, ctx->sm_count, &p.per_split);
     p.nsplit = static_cast<int>(nsplit);
@@ -395,10 +420,22 @@ int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, const
     }
     float *acc = static_cast<float *>(ctx->dw_acc.ptr);
     p.stage_chunks = static_cast<int>((smem - 1024) / 16384);
-    // activations whose planes do not start on 16-byte boundaries are first copied to padded planes
+    // fp32 activations are split into two bf16 pieces (as if the batch were twice as long); bf16 ones whose
+    // planes do not start on 16-byte boundaries are first copied to padded planes
     const void *Xsrc = X;
     long long xpitch = HW;
-    if (HW % 8 != 0) {
+    if (io == DBP_F32) {
+        xpitch = (HW + 7) / 8 * 8;
+        const long long planes = s.B * s.Cin;
+        if ((rc = ws_reserve(ctx, ctx->x_padded, static_cast<size_t>(planes) * xpitch * 2 * 2))) return rc;
+        long long blocks = (planes * xpitch + 255) / 256;
+        if (blocks > ctx->sm_count * 16) blocks = ctx->sm_count * 16;
+        if ((rc = cuda_ok(launch_chained(x_split_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, ctx->stream,
+                                         static_cast<const float *>(X), static_cast<__nv_bfloat16 *>(ctx->x_padded.ptr), planes,
+                                         static_cast<int>(HW), static_cast<int>(xpitch)))))
+            return rc;
+        Xsrc = ctx->x_padded.ptr;
+    } else if (HW % 8 != 0) {
         xpitch = (HW + 7) / 8 * 8;
         if ((rc = ws_reserve(ctx, ctx->x_padded, static_cast<size_t>(s.B) * s.Cin * xpitch * 2))) return rc;
         if ((rc = launch_pad_planes(ctx, X, ctx->x_padded.ptr, s.B * s.Cin, 1, static_cast<int>(HW), static_cast<int>(xpitch))))
@@ -422,7 +459,7 @@ int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, const
     }
     {
         const unsigned long long dims[3] = {static_cast<unsigned long long>(HW), static_cast<unsigned long long>(s.Cin),
-                                            static_cast<unsigned long long>(s.B)};
+                                            static_cast<unsigned long long>(s.B) * pieces};
         const unsigned long long str[2] = {static_cast<unsigned long long>(xpitch) * 2,
                                            static_cast<unsigned long long>(xpitch) * 2 * s.Cin};
         const unsigned box[3] = {64, 128, 1};

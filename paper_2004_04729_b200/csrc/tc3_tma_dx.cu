@@ -53,7 +53,9 @@ struct Dx3T {
     int ci_tiles;
     long long pos_tiles, ntiles;
     int a_panels;                 // 64-channel panels of ci per weight tile (1 or 2)
-    int G;                        // taps per weight slot (one copy): 9, 3 or 1
+    int ntaps;                    // 9, or 18 for fp32 weights split into two bf16 pieces (taps 9-17: the low pieces)
+    int es;                       // bytes per element of dX (2 or 4)
+    int G;                        // taps per weight slot (one hand-over): 9, 3 or 1
     int w_slot;                   // bytes of a weight slot: G * a_panels * 8 KB
     int nq, nw;                   // ring sizes
     int resident;                 // the weights of all taps and co blocks stay in shared memory (one ci block)
@@ -136,7 +138,7 @@ tc3_tma_dx_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             y0 = 0;
         }
     };
-    const int slots_per_cb = 9 / p.G;
+    const int slots_per_cb = p.ntaps / p.G;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -181,7 +183,7 @@ tc3_tma_dx_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                                 tma_load_3d(dst, &map_w, ci0 + 64 * h, g * p.G + gg, c * 64, &pipe.w_full[s]);
                         if (++s == p.nw) { s = 0; parity ^= 1u; }
                     }
-                if (p.resident) break;             // one ci block: every tile uses the same weights
+                if (p.resident) break;             // one ci block: every tile uses the same weights (all slots are loaded now)
             }
             report_wait(p.stats, 4, waited);
         }
@@ -212,7 +214,7 @@ tc3_tma_dx_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     if (!ok) break;
                     tc_fence_after();
                     const unsigned long long bd0 = make_desc(smem_u32(q_s + qs * p.q_bytes), 16, 1024);
-                    int toff = tap_first, kx = 0;
+                    int toff = tap_first, kx = 0, ky = 0;
                     for (int g = 0; g < slots_per_cb && ok; ++g) {
                         ok = __all_sync(0xffffffffu, mbar_wait_timed(&pipe.w_full[ws], wpar, p.err_flag, ww));
                         if (!ok) break;
@@ -222,7 +224,14 @@ tc3_tma_dx_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         unsigned long long ad = make_desc(smem_u32(w_s + ws * p.w_slot), p.a_panels == 2 ? kWPanel : 0, 1024);
                         for (int gg = 0; gg < p.G; ++gg, ad += a_tap) {
                             const unsigned long long bd = bd0 + static_cast<unsigned>(toff);
-                            if (kx == 2) { kx = 0; toff += tap_wrap; } else { ++kx; toff -= 8; }
+                            if (kx == 2) {
+                                kx = 0;
+                                toff += tap_wrap;
+                                if (++ky == 3) { ky = 0; toff = tap_first; }      // the second piece's taps start over
+                            } else {
+                                ++kx;
+                                toff -= 8;
+                            }
                             if (elect_one()) {
 #pragma unroll
                                 for (int k = 0; k < 4; ++k)   // 16 co: 16 rows of A (2048 bytes), 32 bytes along a row of B
@@ -267,32 +276,26 @@ tc3_tma_dx_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             tc_fence_after();
             const int ci_l = q * 32 + lane, ci = ci0 + ci_l;
             const int rows_valid = p.H - y0 < p.Ht ? p.H - y0 : p.Ht;
-            // ---- phase A: accumulator -> staging block (bf16) or straight to dX (fp32)
+            // ---- phase A: accumulator -> staging block (rows of bf16 or fp32 values per channel)
             if (ci0 + q * 32 < p.Cin) {                              // warp-uniform: some of my 32 channels exist
                 unsigned char *row = stage + ci_l * p.pitch;
                 for (int chn = ch_lo; chn < ch_hi; ++chn) {
                     unsigned v[32];
                     tmem_ld32(tmem_base + (static_cast<unsigned>(q * 32) << 16) + slot * kAccCols + chn * 32, v);
                     const short *off = s_off + chn * 32;
-                    if (p.dx_f32) {
-                        if (ci < p.Cin) {
+                    // the 32 table entries of the chunk as four 16-byte loads
+                    const uint4 *tp = reinterpret_cast<const uint4 *>(off);
+                    const uint4 t0 = tp[0], t1 = tp[1], t2 = tp[2], t3 = tp[3];
+                    const unsigned tw[16] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w,
+                                             t2.x, t2.y, t2.z, t2.w, t3.x, t3.y, t3.z, t3.w};
+                    if (p.es == 4) {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) {
-                                const int o = off[j];
-                                if (o < 0) continue;
-                                const int img = o / p.run, within = o - img * p.run;
-                                if (within < rows_valid * p.W && b0 + img < p.B)
-                                    static_cast<float *>(p.dX)[(static_cast<long long>(b0 + img) * p.Cin + ci) * HW + y0 * p.W + within] =
-                                        __uint_as_float(v[j]) * delta;
-                            }
+                        for (int j = 0; j < 32; ++j) {
+                            const int o = static_cast<int>(static_cast<short>((tw[j >> 1] >> (16 * (j & 1))) & 0xffffu));
+                            if (o >= 0) *reinterpret_cast<float *>(row + 4 * o) = __uint_as_float(v[j]) * delta;
                         }
                     } else if (p.pairs) {
-                        // the 32 table entries of the chunk as four 16-byte loads; entry 2i tells where
-                        // columns 2i, 2i+1 go
-                        const uint4 *tp = reinterpret_cast<const uint4 *>(off);
-                        const uint4 t0 = tp[0], t1 = tp[1], t2 = tp[2], t3 = tp[3];
-                        const unsigned tw[16] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w,
-                                                 t2.x, t2.y, t2.z, t2.w, t3.x, t3.y, t3.z, t3.w};
+                        // entry 2i tells where columns 2i, 2i+1 go
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             const int o = static_cast<int>(static_cast<short>(tw[i] & 0xffffu));
@@ -302,7 +305,7 @@ tc3_tma_dx_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     } else {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
-                            const int o = off[j];
+                            const int o = static_cast<int>(static_cast<short>((tw[j >> 1] >> (16 * (j & 1))) & 0xffffu));
                             if (o >= 0) *reinterpret_cast<__nv_bfloat16 *>(row + 2 * o) = __float2bfloat16_rn(__uint_as_float(v[j]) * delta);
                         }
                     }
@@ -311,19 +314,20 @@ tc3_tma_dx_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             // the accumulator is free once every epilogue warp has read its part
             tc_fence_before();
             warp_arrive(&pipe.acc_empty[slot]);
-            if (p.dx_f32) continue;
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
             // ---- phase B: staging block -> dX, runs of consecutive positions per (image, channel)
             {
                 const int ncv = p.Cin - ci0 < 128 ? p.Cin - ci0 : 128;
                 const int len = rows_valid * p.W;                    // elements per run
-                __nv_bfloat16 *dst0 = static_cast<__nv_bfloat16 *>(p.dX);
+                unsigned char *dst0 = static_cast<unsigned char *>(p.dX);
+                const bool words = p.es == 4 || p.pairs;             // whole 32-bit words
+                const int nwords = p.es == 4 ? len : len >> 1;
                 for (int img = 0; img < p.nb && b0 + img < p.B; ++img) {
                     for (int r = et >> 5; r < ncv; r += kEpiThreads / 32) {
-                        const unsigned char *src = stage + r * p.pitch + 2 * img * p.run;
-                        __nv_bfloat16 *dst = dst0 + (static_cast<long long>(b0 + img) * p.Cin + ci0 + r) * HW + y0 * p.W;
-                        if (p.pairs) {
-                            for (int i = lane; i * 2 < len; i += 32)
+                        const unsigned char *src = stage + r * p.pitch + p.es * img * p.run;
+                        unsigned char *dst = dst0 + ((static_cast<long long>(b0 + img) * p.Cin + ci0 + r) * HW + y0 * p.W) * p.es;
+                        if (words) {
+                            for (int i = lane; i < nwords; i += 32)
                                 reinterpret_cast<unsigned *>(dst)[i] = reinterpret_cast<const unsigned *>(src)[i];
                         } else {
                             for (int i = lane; i < len; i += 32)
@@ -357,23 +361,44 @@ w_taps_bf16_kernel(const unsigned short *__restrict__ W, unsigned short *__restr
     }
 }
 
+// fp32 weights -> [Cout][18][Cin] bf16: taps 0-8 hold the values rounded to bf16, taps 9-17 what that
+// rounding left over, rounded to bf16 again. The sum of the two pieces differs from the fp32 value by
+// at most 2^-18 of it, and a code times a piece is exact in the fp32 accumulator.
+__global__ void __launch_bounds__(256)
+w_taps_split_kernel(const float *__restrict__ W, __nv_bfloat16 *__restrict__ out, long long Cout, long long Cin) {
+    chain_wait();
+    chain_release();
+    const long long n = Cout * Cin * 9;
+    for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += gridDim.x * 256ll) {
+        const long long ci = i % Cin, t = (i / Cin) % 9, co = i / (Cin * 9);
+        const float w = __ldg(W + (co * Cin + ci) * 9 + t);
+        const __nv_bfloat16 hi = __float2bfloat16_rn(w);
+        const __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(hi));
+        out[(co * 18 + t) * Cin + ci] = hi;
+        out[(co * 18 + 9 + t) * Cin + ci] = lo;
+    }
+}
+
 int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 }  // namespace
 
-// Shapes the TMA-fed 3x3 kernels take: bf16 operands, channel counts that keep every row of the
-// position-major codes, of the re-laid weights and of the activations on 16-byte boundaries.
+// Shapes the TMA-fed 3x3 kernels take: channel counts that keep every row of the position-major
+// codes, of the re-laid weights and of the activations on 16-byte boundaries. fp32 operands are
+// split into two bf16 pieces each (the codes are exact in bf16), so they take the same kernels.
 bool tc3_tma_supported(const ConvShape &s, int io) {
-    return io == DBP_BF16 && s.k == 3 && s.Cin % 8 == 0 && s.Cout % 8 == 0 && s.W >= 1 && s.W <= 62 && s.H <= 4096 &&
-           s.B * s.H * s.W < (1ll << 30);
+    return (io == DBP_BF16 || io == DBP_F32) && s.k == 3 && s.Cin % 8 == 0 && s.Cout % 8 == 0 && s.W >= 1 && s.W <= 62 &&
+           s.H <= 4096 && s.B * s.H * s.W < (1ll << 30);
 }
 
 // DBP_EUNSUPPORTED: the shape does not fit (the caller uses another kernel)
-int launch_tc3_tma_dx(dbp_ctx *ctx, const void *codes_nhwc, const void *W, const float *delta_p,
+int launch_tc3_tma_dx(dbp_ctx *ctx, const void *codes_nhwc, const void *W, int io, const float *delta_p,
                       const ConvShape &s, void *dX, bool dx_bf16, int *err_flag) {
-    if (!tc3_tma_supported(s, DBP_BF16)) return DBP_EUNSUPPORTED;
+    if (!tc3_tma_supported(s, io)) return DBP_EUNSUPPORTED;
     Dx3T p{};
     p.delta_p = delta_p; p.dX = dX; p.dx_f32 = dx_bf16 ? 0 : 1;
+    p.es = dx_bf16 ? 2 : 4;
+    p.ntaps = io == DBP_F32 ? 18 : 9;
     p.B = static_cast<int>(s.B); p.Cin = static_cast<int>(s.Cin); p.Cout = static_cast<int>(s.Cout);
     p.H = static_cast<int>(s.H); p.W = static_cast<int>(s.W); p.Wp = p.W + 2;
     p.err_flag = err_flag;
@@ -381,16 +406,29 @@ int launch_tc3_tma_dx(dbp_ctx *ctx, const void *codes_nhwc, const void *W, const
     p.ncb = (p.Cout + 63) / 64;
     p.ci_tiles = (p.Cin + 127) / 128;
     p.a_panels = p.Cin <= 64 ? 1 : 2;
+    const size_t tap_bytes = static_cast<size_t>(p.a_panels) * kWPanel;
+    const size_t budget = 227 * 1024 - 2048;
     // patch geometry: the cheapest of the candidates by (waves of one CTA per SM) x (columns per tile;
-    // a narrow MMA takes as long to issue as one of about 200 columns takes to run)
+    // a narrow MMA takes as long to issue as one of about 200 columns takes to run). A candidate must
+    // leave room for its two patch buffers, its staging block and at least three weight taps.
     const int sms = ctx->sm_count;
     int best_ht = 0, best_nb = 1;
     double best_cost = 1e300;
+    auto patch_bytes = [&](int ht, int nb, int n) {
+        const int img_rows = (ht + 2) * p.Wp, rows_read = n + 2 * p.Wp + 2;
+        return round_up((rows_read > img_rows * nb ? rows_read : img_rows * nb) * 128, 1024);
+    };
+    auto stage_pitch = [&](int ht, int nb) {
+        int pitch = round_up(nb * ht * p.W * p.es, 4);
+        if ((pitch / 4) % 2 == 0) pitch += 4;      // an odd number of words: see below
+        return pitch;
+    };
     auto consider = [&](int ht, int nb) {
         const int img_rows = (ht + 2) * p.Wp;
         const int last = (nb - 1) * img_rows + (ht - 1) * p.Wp + p.W - 1;     // last column that holds an output
         const int n = round_up(last + 1, 16);
         if (n > 256 || img_rows * nb > 1024) return;
+        if (2 * static_cast<size_t>(patch_bytes(ht, nb, n)) + 128 * static_cast<size_t>(stage_pitch(ht, nb)) + 1536 + 3 * tap_bytes > budget) return;
         const long long tiles = nb == 1 ? static_cast<long long>(p.B) * ((p.H + ht - 1) / ht) : (p.B + nb - 1) / nb;
         const long long waves = (tiles * p.ci_tiles + sms - 1) / sms;
         const double cost = static_cast<double>(waves) * ((n < 208 ? 208 : n) + 64);      // an MMA takes >= ~100 clocks to issue
@@ -408,30 +446,22 @@ int launch_tc3_tma_dx(dbp_ctx *ctx, const void *codes_nhwc, const void *W, const
     p.q_tx = p.img_rows * p.nb * 128;
     // the last tap of the last column reads row N - 1 + 2 Wp + 2; rows past the copied patch hold
     // stale data, which only reaches columns that are never stored
-    const int rows_read = p.N + 2 * p.Wp + 2;
-    p.q_bytes = round_up((rows_read > p.img_rows * p.nb ? rows_read : p.img_rows * p.nb) * 128, 1024);
+    p.q_bytes = patch_bytes(p.Ht, p.nb, p.N);
     p.run = p.Ht * p.W;
     // an odd number of 32-bit words per row: the 32 channels of a warp hit 32 different banks when
     // they stage the same position
-    p.pitch = round_up(p.nb * p.run * 2, 4);
-    if ((p.pitch / 4) % 2 == 0) p.pitch += 4;
+    p.pitch = stage_pitch(p.Ht, p.nb);
     p.pairs = p.W % 2 == 0 ? 1 : 0;
-    const size_t stage_bytes = dx_bf16 ? static_cast<size_t>(128) * p.pitch : 0;
-    const size_t budget = 227 * 1024 - 2048;
+    const size_t stage_bytes = static_cast<size_t>(128) * p.pitch;
     // Weights: a slot holds G taps and is handed over with one barrier (the hand-over, not the copy
     // instruction, is what costs time). With one ci block and room for all taps of all co blocks they
     // are loaded once and stay; otherwise they stream through a ring of slots.
-    const size_t tap_bytes = static_cast<size_t>(p.a_panels) * kWPanel;
     p.nq = kMaxQ;
-    size_t fixed = static_cast<size_t>(p.nq) * p.q_bytes + stage_bytes + 512 + 1024;
-    if (fixed + 3 * tap_bytes > budget) {
-        p.nq = 1;
-        fixed = static_cast<size_t>(p.q_bytes) + stage_bytes + 512 + 1024;
-        if (fixed + 3 * tap_bytes > budget) return DBP_EUNSUPPORTED;
-    }
+    const size_t fixed = static_cast<size_t>(p.nq) * p.q_bytes + stage_bytes + 512 + 1024;
     const size_t room = budget - fixed;
-    if (p.ci_tiles == 1 && p.ncb <= kMaxW && static_cast<size_t>(p.ncb) * 9 * tap_bytes <= room) {
-        p.resident = 1; p.G = 9; p.nw = p.ncb;
+    const int slots_all = p.ncb * (p.ntaps / 9);
+    if (p.ci_tiles == 1 && slots_all <= kMaxW && static_cast<size_t>(slots_all) * 9 * tap_bytes <= room) {
+        p.resident = 1; p.G = 9; p.nw = slots_all;
     } else if (room >= 2 * 3 * tap_bytes) {
         p.resident = 0; p.G = 3; p.nw = static_cast<int>(room / (3 * tap_bytes));
     } else {
@@ -442,16 +472,20 @@ int launch_tc3_tma_dx(dbp_ctx *ctx, const void *codes_nhwc, const void *W, const
     const size_t smem = fixed + static_cast<size_t>(p.nw) * p.w_slot;
 
     // re-laid weights
-    const size_t wb = sizeof(__nv_bfloat16) * static_cast<size_t>(s.Cout) * s.Cin * 9;
+    const size_t wb = sizeof(__nv_bfloat16) * static_cast<size_t>(s.Cout) * s.Cin * p.ntaps;
     int rc = ws_reserve(ctx, ctx->w_taps, wb);
     if (rc) return rc;
     {
         long long blocks = (static_cast<long long>(s.Cout) * s.Cin * 9 + 255) / 256;
         if (blocks > sms * 8) blocks = sms * 8;
-        if ((rc = cuda_ok(launch_chained(w_taps_bf16_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, ctx->stream,
-                                         static_cast<const unsigned short *>(W), static_cast<unsigned short *>(ctx->w_taps.ptr),
-                                         s.Cout, s.Cin))))
-            return rc;
+        if (io == DBP_F32)
+            rc = cuda_ok(launch_chained(w_taps_split_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, ctx->stream,
+                                        static_cast<const float *>(W), static_cast<__nv_bfloat16 *>(ctx->w_taps.ptr), s.Cout, s.Cin));
+        else
+            rc = cuda_ok(launch_chained(w_taps_bf16_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, ctx->stream,
+                                        static_cast<const unsigned short *>(W), static_cast<unsigned short *>(ctx->w_taps.ptr),
+                                        s.Cout, s.Cin));
+        if (rc) return rc;
     }
     CUtensorMap map_q, map_w;
     {
@@ -464,8 +498,10 @@ int launch_tc3_tma_dx(dbp_ctx *ctx, const void *codes_nhwc, const void *W, const
         if (!encode_map_bf16(&map_q, codes_nhwc, 4, dims, str, box)) return fail_cuda("tensor map of the code patches");
     }
     {
-        const unsigned long long dims[3] = {static_cast<unsigned long long>(s.Cin), 9ull, static_cast<unsigned long long>(s.Cout)};
-        const unsigned long long str[2] = {static_cast<unsigned long long>(s.Cin) * 2, static_cast<unsigned long long>(s.Cin) * 18};
+        const unsigned long long dims[3] = {static_cast<unsigned long long>(s.Cin), static_cast<unsigned long long>(p.ntaps),
+                                            static_cast<unsigned long long>(s.Cout)};
+        const unsigned long long str[2] = {static_cast<unsigned long long>(s.Cin) * 2,
+                                           static_cast<unsigned long long>(s.Cin) * 2 * p.ntaps};
         const unsigned box[3] = {64, 1, 64};
         if (!encode_map_bf16(&map_w, ctx->w_taps.ptr, 3, dims, str, box)) return fail_cuda("tensor map of the weights");
     }

@@ -25,9 +25,14 @@ def _t(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda().to(torch.bfloat16)
 
 
+def _f32(a):
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
+
+
 def _run(ctx, L, flags):
     import paper_2004_04729_b200 as dbp
-    d, X, W = _t(L.delta), _t(L.X), _t(L.W)
+    cast = _t if L.dtype == "bf16" else _f32
+    d, X, W = cast(L.delta), cast(L.X), cast(L.W)
     q = dbp.SparseGradient(d.numel())
     fn = dbp.dithered_linear_backward if L.kind == "linear" else dbp.dithered_conv_backward
     out = fn(ctx, d, X, W, L.seed, L.scale, q_out=q, need_db=True, flags=flags | dbp.DBP_DX_F32)
@@ -88,6 +93,23 @@ def test_dense_path_conv1x1(ctx, B, Ci, Co, H, W):
 def test_dense_path_conv3x3(ctx, B, Ci, Co, H, W):
     import paper_2004_04729_b200 as dbp
     L = wl.conv_layer(B, Ci, Co, H, W, 3, data_seed=B + Ci + Co + H, scale=5.0 if Ci > 64 else 2.0, dtype="bf16")
+    _run(ctx, L, dbp.DBP_FORCE_DENSE)
+
+
+@pytest.mark.parametrize("B,Ci,Co,H,W", [
+    (4, 64, 64, 32, 32),      # config-3 shape at batch 4: weights resident in shared memory (one ci block, 18 taps)
+    (2, 128, 128, 16, 16),    # config-4 stage 2
+    (2, 256, 256, 8, 8),      # two ci blocks: weights streamed
+    (3, 512, 512, 4, 4),      # several images per patch
+    (5, 512, 512, 2, 2),      # config-4 last stage: 4 positions per image
+    (2, 72, 40, 9, 11),       # channel counts that fill no tile, odd width (element-wise staging)
+    (2, 8, 16, 1, 1),         # a single position
+])
+def test_dense_path_conv3x3_fp32_operands(ctx, B, Ci, Co, H, W):
+    """fp32 layers on the tensor cores: weights and activations enter as two bf16 pieces each (the sum of the
+    pieces is within 2^-18 of the fp32 value, a code times a piece is exact), same bars as everywhere."""
+    import paper_2004_04729_b200 as dbp
+    L = wl.conv_layer(B, Ci, Co, H, W, 3, data_seed=B + Ci + Co + H, scale=2.0, dtype="f32")
     _run(ctx, L, dbp.DBP_FORCE_DENSE)
 
 
