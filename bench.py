@@ -336,6 +336,29 @@ def small_config(torch, dbp, ctx, config, hbm_peak, fma_peak):
                     if config in (1, 2) else "fp32: sparse gather kernels (no tensor-core path for fp32 operands)"}
 
 
+def crossover_sweep(torch, dbp, ctx):
+    """Sparse gather kernels against the tensor-core path as the gradient gets sparser (larger s): one 1x1,
+    one 3x3 and one linear shape, bf16. Prints one JSON line per (shape, s)."""
+    shapes = [("conv1x1 128->512 @28x28 B64", lambda s: wl.conv_layer(64, 128, 512, 28, 28, 1, data_seed=71, scale=s, dtype="bf16")),
+              ("conv3x3 128->128 @28x28 B64", lambda s: wl.conv_layer(64, 128, 128, 28, 28, 3, data_seed=72, scale=s, dtype="bf16")),
+              ("linear 2048->512 B256", lambda s: wl.linear_layer(256, 512, 2048, data_seed=73, scale=s, dtype="bf16"))]
+    for name, make in shapes:
+        for s in (2.0, 5.0, 10.0, 20.0, 40.0, 80.0):
+            L = make(s)
+            d, X, W = (torch.from_numpy(a).to(torch.bfloat16).cuda() for a in (L.delta, L.X, L.W))
+            fn = dbp.dithered_linear_backward if L.kind == "linear" else dbp.dithered_conv_backward
+            q = dbp.nsd_quantize(ctx, d, L.seed, L.scale)
+            dens = q.nnz.item() / d.numel()
+            row = {"shape": name, "s": s, "density": dens}
+            for label, flag in (("sparse_ms", dbp.DBP_FORCE_SPARSE), ("dense_ms", dbp.DBP_FORCE_DENSE)):
+                run = lambda: fn(ctx, d, X, W, L.seed, L.scale, flags=flag)
+                for _ in range(3):
+                    run()
+                torch.cuda.synchronize()
+                row[label] = time_events(torch, run, 10)
+            print(json.dumps(row))
+
+
 # DRAM bytes (read + written) of one bench step's launches of each kernel kind, from the ncu capture summarised in
 # profiles/bench_step_config5_dram_bytes.md; None = the kernels of that kind changed after the capture
 NCU_DRAM_BYTES_PER_STEP = {"statistics": None, "quantize": None, "dx_dense": None, "dw_dense": None}
@@ -355,6 +378,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-others", action="store_true", help="skip the side measurements of configs 1-4")
+    ap.add_argument("--crossover-sweep", action="store_true", help="time the sparse and the dense path against density and exit")
+    ap.add_argument("--force-sparse", action="store_true", help="gather kernels on every layer (profiling aid)")
+    ap.add_argument("--bf16", action="store_true", help="configs 1 and 3 with bf16 storage (profiling aid: the bf16 linear kernels)")
     ap.add_argument("--sync-dw", action="store_true", help="every call joins its dW before it returns (no DBP_DW_ASYNC)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl != "reference":
@@ -379,6 +405,10 @@ def main():
         sampler.start()
     hbm_peak, peak_src = measured_peaks()
     fma_peak = ctx.measure_fma_peak()
+    if args.crossover_sweep:
+        if rank == 0:
+            crossover_sweep(torch, dbp, ctx)
+        return
 
     if args.config in CHAIN_NAMES:
         # whole-network configurations: the side measurement is the measurement
@@ -402,6 +432,15 @@ def main():
         return
 
     specs, name = layer_specs(args.config, args.batch)
+    if args.bf16 and args.config in (1, 3):
+        def as_bf16(make):
+            def f():
+                L = make()
+                L.delta, L.X, L.W, L.dtype = wl.round_to_bf16(L.delta), wl.round_to_bf16(L.X), wl.round_to_bf16(L.W), "bf16"
+                return L
+            return f
+        specs = [(as_bf16(make), mult) for make, mult in specs]
+        name += " [bf16 storage]"
     if args.only:
         keep = [int(t) for t in args.only.split(",")]
         specs = [specs[i] for i in keep]
@@ -430,7 +469,9 @@ def main():
 
     # dW of a layer may still run while the next layer is quantized (the layer below needs dX only); every dW
     # is ordered into the stream before the step ends
-    FLAGS = 0 if args.sync_dw else dbp.DBP_DW_ASYNC
+    FLAGS = (0 if args.sync_dw else dbp.DBP_DW_ASYNC) | (dbp.DBP_FORCE_SPARSE if args.force_sparse else 0)
+    if args.force_sparse:
+        name += " [gather kernels forced]"
 
     def run_layer(L, d, X, W, dW, dX):
         code = 1 if L.dtype == "bf16" else 0

@@ -63,7 +63,7 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
                           dbp_sparse *q_out, const float **delta_p, const int8_t **codes,
                           bool want8 = true, long long planes_hw = 0, long long planes_pitch = 0,
                           const void **codes16 = nullptr, const ConvShape *nhwc = nullptr,
-                          const void **codes_nhwc = nullptr, void *zero = nullptr, size_t zero_bytes = 0) {
+                          const void **codes_nhwc = nullptr, const SideJobs &jobs = SideJobs()) {
     int rc = DBP_OK;
     dbp_sparse sp;
     sp.bitmap = nullptr; sp.offsets = nullptr; sp.values = nullptr; sp.delta = nullptr; sp.nnz = nullptr;
@@ -82,7 +82,7 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
         // without a caller's dbp_sparse the step size also goes to the set's own scalar: the product kernels
         // read it there (the context's scalar is overwritten by the next call's statistics)
         rc = launch_statistics(ctx, delta, dtype, numel, scale, delta_in, q_out ? sp.delta : ctx->delta_sets + k,
-                               reinterpret_cast<unsigned long long *>(sp.nnz), zero, zero_bytes);
+                               reinterpret_cast<unsigned long long *>(sp.nnz), jobs);
     }
     if (rc) return rc;
     // the set's previous readers (an earlier call's dW kernels on the second stream) must be done
@@ -177,7 +177,7 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     for (const auto &e : ctx->densities)
         if (e.key == shape_key) density_estimate = e.density;
     const bool dense = can_dense && !(flags & DBP_FORCE_SPARSE) &&
-                       ((flags & DBP_FORCE_DENSE) || density_estimate > ctx->crossover);
+                       ((flags & DBP_FORCE_DENSE) || ctx->crossover <= 0.f || density_estimate > ctx->crossover);
     // which dense kernels run: the TMA-fed ones read bf16 code planes, the others int8 codes
     const bool dx_tma = dense && dX && tma_dx_supported(s, io);
     const bool dw_tma = dense && dW && tma_dw_supported(s, io);
@@ -192,11 +192,20 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     const bool t3 = dense && (dX || dW) && tc3_tma_supported(s, io);
     const bool need8 = !dense || db || (!t3 && ((dX && !dx_tma) || (dW && !dw_tma)));
     const void *codes16 = nullptr, *codes_n = nullptr;
+    // what the statistics kernel does on the side: the TMA-fed 1x1 dW kernel adds its partial sums into dW, so dW
+    // is cleared; the 3x3 dX kernel reads the weights tap by tap, so they are re-laid
+    SideJobs jobs;
+    if (dw_tma) { jobs.zero = dW; jobs.zero_bytes = sizeof(float) * static_cast<size_t>(s.Cout) * s.Cin; }
+    const bool w_side = t3 && dX && scale > 0.f;
+    if (w_side) {
+        const int taps = io == DBP_F32 ? 18 : 9;
+        const int wr = ws_reserve(ctx, ctx->w_taps, sizeof(__nv_bfloat16) * static_cast<size_t>(s.Cout) * s.Cin * taps);
+        if (wr) return wr;
+        jobs.w_src = W; jobs.w_dst = ctx->w_taps.ptr; jobs.w_f32 = io == DBP_F32; jobs.Cout = s.Cout; jobs.Cin = s.Cin;
+    }
     int rc = quantize_for_products(ctx, delta, io, numel, seed, scale, delta_in, q_out, &delta_p, &codes, need8,
                                    s.H * s.W, any_tma ? tma_code_pitch(s) : 0, any_tma ? &codes16 : nullptr,
-                                   t3 ? &s : nullptr, t3 ? &codes_n : nullptr,
-                                   // the TMA-fed 1x1 dW kernel adds its partial sums into dW: cleared by the statistics kernel
-                                   dw_tma ? dW : nullptr, dw_tma ? sizeof(float) * static_cast<size_t>(s.Cout) * s.Cin : 0);
+                                   t3 ? &s : nullptr, t3 ? &codes_n : nullptr, jobs);
     if (rc) return rc;
     if (!capturing && !ctx->nnz_pending && ctx->nnz_host && ctx->nnz_event) {
         ctx->nnz_host_numel = numel;
@@ -217,7 +226,7 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
             KernelTimer t(ctx, DBP_K_DX_DENSE);
             const bool dx_bf16 = (io == DBP_BF16) && !(flags & DBP_DX_F32);
             rc = dx_tma ? launch_tma_dx(ctx, codes16, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout)
-                 : t3   ? launch_tc3_tma_dx(ctx, codes_n, W, io, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout)
+                 : t3   ? launch_tc3_tma_dx(ctx, codes_n, W, io, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout, w_side)
                         : launch_tc_dx(ctx, codes, W, delta_p, s, dX, dx_bf16, &ctx->state->tc_timeout);
             if (rc) return rc;
         }

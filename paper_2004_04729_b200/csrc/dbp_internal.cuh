@@ -71,7 +71,10 @@ struct dbp_ctx {
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
     cudaEvent_t ev_x_up = nullptr, ev_dx_done = nullptr;
     cudaEvent_t hook_after_dx = nullptr, hook_before_dw = nullptr;   // set only during a *_host call
-    float crossover = 0.03f;            // density above which the dense path is preferred
+    // density above which the dense path is preferred. Measured (sparse against dense time for a 1x1, a 3x3 and a
+    // linear layer, densities 22 % ... 0.6 %): the tensor-core path is 2.3x to 11x faster at every density, the gather
+    // kernels' time being mostly the scan of the dense codes; so wherever the dense path exists it is the default.
+    float crossover = 0.0f;
     // densities measured so far, by layer shape (the path choice of a call uses its own shape's entry)
     struct DensityEntry { unsigned long long key; float density; };
     std::vector<DensityEntry> densities;
@@ -93,10 +96,21 @@ namespace dbp {
 int ws_reserve(dbp_ctx *ctx, Workspace &w, size_t bytes);
 
 // ---- nsd_kernels.cu
-// zero / zero_bytes: a buffer (16-byte aligned, a multiple of 16 bytes) that the same kernel clears
+// Work the statistics kernel does on the side for the layer's product kernels (its blocks have time to spare
+// and this saves launches): clearing a buffer (16-byte aligned, a multiple of 16 bytes), and re-laying 3x3
+// weights [Cout][Cin][9] as [Cout][taps][Cin] bf16 (taps = 9 for bf16 weights; 18 for fp32 weights, split into
+// two bf16 pieces: taps 0-8 the rounded values, 9-17 what the rounding left over).
+struct SideJobs {
+    void *zero = nullptr;
+    size_t zero_bytes = 0;
+    const void *w_src = nullptr;       // null: no weights to re-lay
+    void *w_dst = nullptr;
+    int w_f32 = 0;
+    long long Cout = 0, Cin = 0;
+};
 int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long numel, float scale,
                       const float *delta_in, float *delta_out, unsigned long long *nnz_out,
-                      void *zero = nullptr, size_t zero_bytes = 0);
+                      const SideJobs &jobs = SideJobs());
 int launch_quantize(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
                     unsigned long long seed, const float *delta_p, uint32_t *bitmap,
                     uint16_t *offsets, int8_t *values, int8_t *dense,
@@ -152,8 +166,9 @@ int launch_dw_sum(dbp_ctx *ctx, const float *partials, int nsplit, long long nw,
 // ---- tc3_tma_dx.cu / tc3_tma_dw.cu: 3x3 products with TMA-fed operands; codes as bf16 [B][H*W][Cout]
 bool tc3_tma_supported(const ConvShape &s, int io);
 // io: the operands' type; fp32 weights / activations are split into two bf16 pieces on the way in
+// weights_ready: ctx->w_taps already holds the re-laid weights (the statistics kernel did it on the side)
 int launch_tc3_tma_dx(dbp_ctx *ctx, const void *codes_nhwc, const void *W, int io, const float *delta_p,
-                      const ConvShape &s, void *dX, bool dx_bf16, int *err_flag);
+                      const ConvShape &s, void *dX, bool dx_bf16, int *err_flag, bool weights_ready = false);
 int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, int io, const float *delta_p,
                       const ConvShape &s, float *dW, int *err_flag);
 int launch_bias_grad(dbp_ctx *ctx, const int8_t *codes, const float *delta_p, const ConvShape &s,

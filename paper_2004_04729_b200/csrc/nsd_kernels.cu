@@ -75,7 +75,8 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads)
 statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ partials,
                   DeviceState *__restrict__ st, float scale, float *__restrict__ delta_out,
-                  unsigned long long *__restrict__ nnz_out, uint4 *__restrict__ zero_ptr, long long zero_n16) {
+                  unsigned long long *__restrict__ nnz_out, uint4 *__restrict__ zero_ptr, long long zero_n16,
+                  const void *__restrict__ w_src, unsigned short *__restrict__ w_dst, int w_f32, long long w_cout, int w_cin) {
     constexpr int EPT = Elem<T>::EPT;
     const long long nvec = n / EPT;
     chain_wait();
@@ -84,6 +85,26 @@ statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ par
     for (long long i = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x; i < zero_n16;
          i += static_cast<long long>(gridDim.x) * kThreads)
         zero_ptr[i] = make_uint4(0u, 0u, 0u, 0u);
+    // side job for the layer's 3x3 input-gradient kernel: weights [co][ci][9] -> [co][tap][ci] bf16 (for fp32
+    // weights two pieces: taps 0-8 the values rounded to bf16, taps 9-17 the remainders rounded to bf16)
+    if (w_src != nullptr) {
+        const int per_co = 9 * w_cin, taps = w_f32 ? 18 : 9;
+        for (long long co = blockIdx.x; co < w_cout; co += gridDim.x) {
+            unsigned short *dst = w_dst + co * taps * w_cin;
+            for (int j = threadIdx.x; j < per_co; j += kThreads) {
+                const int t = j / w_cin, ci = j - t * w_cin;                 // writes run along ci
+                if (w_f32) {
+                    const float w = __ldg(static_cast<const float *>(w_src) + co * per_co + ci * 9 + t);
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(w);
+                    const __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(hi));
+                    dst[j] = *reinterpret_cast<const unsigned short *>(&hi);
+                    dst[per_co + j] = *reinterpret_cast<const unsigned short *>(&lo);
+                } else {
+                    dst[j] = __ldg(static_cast<const unsigned short *>(w_src) + co * per_co + ci * 9 + t);
+                }
+            }
+        }
+    }
     double d1 = 0.0, d2 = 0.0;
     const float pivot = Elem<T>::one(x);
     const long long stride = static_cast<long long>(gridDim.x) * kThreads;
@@ -386,11 +407,13 @@ decode_kernel(const uint32_t *__restrict__ bitmap, const uint16_t *__restrict__ 
 }  // namespace
 
 int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long numel, float scale,
-                      const float *delta_in, float *delta_out, unsigned long long *nnz_out, void *zero, size_t zero_bytes) {
-    uint4 *zp = static_cast<uint4 *>(zero);
-    const long long zn = zero ? static_cast<long long>(zero_bytes / 16) : 0;
-    if (!(scale > 0.f)) {
-        if (zero && cudaMemsetAsync(zero, 0, zero_bytes, ctx->stream) != cudaSuccess) return fail_cuda("clearing dW");
+                      const float *delta_in, float *delta_out, unsigned long long *nnz_out, const SideJobs &jobs) {
+    uint4 *zp = static_cast<uint4 *>(jobs.zero);
+    const long long zn = jobs.zero ? static_cast<long long>(jobs.zero_bytes / 16) : 0;
+    unsigned short *wd = static_cast<unsigned short *>(jobs.w_dst);
+    const int wci = static_cast<int>(jobs.Cin);
+    if (!(scale > 0.f)) {      // the step size is given: no statistics kernel, so no side jobs either (the caller sees to the weights)
+        if (jobs.zero && cudaMemsetAsync(jobs.zero, 0, jobs.zero_bytes, ctx->stream) != cudaSuccess) return fail_cuda("clearing dW");
         note_launch();
         set_step_kernel<<<1, 1, 0, ctx->stream>>>(delta_in, ctx->state, delta_out, nnz_out);
         return cuda_ok(cudaGetLastError());
@@ -402,10 +425,10 @@ int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long nume
     cudaError_t e;
     if (dtype == DBP_F32)
         e = launch_chained(statistics_kernel<float>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
-                           static_cast<const float *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out, zp, zn);
+                           static_cast<const float *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out, zp, zn, jobs.w_src, wd, jobs.w_f32, jobs.Cout, wci);
     else
         e = launch_chained(statistics_kernel<__nv_bfloat16>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
-                           static_cast<const __nv_bfloat16 *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out, zp, zn);
+                           static_cast<const __nv_bfloat16 *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out, zp, zn, jobs.w_src, wd, jobs.w_f32, jobs.Cout, wci);
     return cuda_ok(e);
 }
 

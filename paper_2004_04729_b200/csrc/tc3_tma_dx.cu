@@ -393,7 +393,7 @@ bool tc3_tma_supported(const ConvShape &s, int io) {
 
 // DBP_EUNSUPPORTED: the shape does not fit (the caller uses another kernel)
 int launch_tc3_tma_dx(dbp_ctx *ctx, const void *codes_nhwc, const void *W, int io, const float *delta_p,
-                      const ConvShape &s, void *dX, bool dx_bf16, int *err_flag) {
+                      const ConvShape &s, void *dX, bool dx_bf16, int *err_flag, bool weights_ready) {
     if (!tc3_tma_supported(s, io)) return DBP_EUNSUPPORTED;
     Dx3T p{};
     p.delta_p = delta_p; p.dX = dX; p.dx_f32 = dx_bf16 ? 0 : 1;
@@ -475,7 +475,7 @@ int launch_tc3_tma_dx(dbp_ctx *ctx, const void *codes_nhwc, const void *W, int i
     const size_t wb = sizeof(__nv_bfloat16) * static_cast<size_t>(s.Cout) * s.Cin * p.ntaps;
     int rc = ws_reserve(ctx, ctx->w_taps, wb);
     if (rc) return rc;
-    {
+    if (!weights_ready) {
         long long blocks = (static_cast<long long>(s.Cout) * s.Cin * 9 + 255) / 256;
         if (blocks > sms * 8) blocks = sms * 8;
         if (io == DBP_F32)
