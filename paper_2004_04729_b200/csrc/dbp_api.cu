@@ -145,7 +145,10 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     if ((dW && !X) || (dX && !W)) return DBP_EINVAL;
     if (!aligned16(delta) || !aligned16(X) || !aligned16(W) || !aligned16(dW) || !aligned16(dX)) return DBP_EINVAL;
     if ((flags & DBP_FORCE_SPARSE) && (flags & DBP_FORCE_DENSE)) return DBP_EINVAL;
-    const bool can_dense = tc_supported(s, io) || tc3_tma_supported(s, io);
+    // 3x3 on the tensor cores: both products, or (fp32, any Cin: a network's first layer) the weight gradient alone
+    const bool t3_full = tc3_tma_supported(s, io);
+    const bool t3_dw_only = !t3_full && dW && !dX && tc3_tma_dw_supported(s, io);
+    const bool can_dense = tc_supported(s, io) || t3_full || t3_dw_only;
     if ((flags & DBP_FORCE_DENSE) && !can_dense) return DBP_EUNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DBP_ECUDA;
@@ -189,7 +192,7 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
         if (jr) return jr;
     }
     // 3x3 layers: the TMA-fed kernels read the codes position-major
-    const bool t3 = dense && (dX || dW) && tc3_tma_supported(s, io);
+    const bool t3 = dense && (dX || dW) && (t3_full || t3_dw_only);
     const bool need8 = !dense || db || (!t3 && ((dX && !dx_tma) || (dW && !dw_tma)));
     const void *codes16 = nullptr, *codes_n = nullptr;
     // what the statistics kernel does on the side: the TMA-fed 1x1 dW kernel adds its partial sums into dW, so dW

@@ -165,6 +165,7 @@ int launch_pad_planes(dbp_ctx *ctx, const void *in, void *out, long long planes,
 int launch_dw_sum(dbp_ctx *ctx, const float *partials, int nsplit, long long nw, const float *delta_p, float *dW);
 // ---- tc3_tma_dx.cu / tc3_tma_dw.cu: 3x3 products with TMA-fed operands; codes as bf16 [B][H*W][Cout]
 bool tc3_tma_supported(const ConvShape &s, int io);
+bool tc3_tma_dw_supported(const ConvShape &s, int io);     // dW alone: also fp32 layers with any Cin
 // io: the operands' type; fp32 weights / activations are split into two bf16 pieces on the way in
 // weights_ready: ctx->w_taps already holds the re-laid weights (the statistics kernel did it on the side)
 int launch_tc3_tma_dx(dbp_ctx *ctx, const void *codes_nhwc, const void *W, int io, const float *delta_p,

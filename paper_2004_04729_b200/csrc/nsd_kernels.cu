@@ -421,6 +421,9 @@ int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long nume
     const int ept = dtype == DBP_F32 ? 4 : 8;
     long long blocks = numel / ept / (kThreads * 8);          // one block per tile of eight vectors per thread
     if (blocks < 1) blocks = 1;
+    // the side jobs want blocks of their own when the tensor is small (a block beyond the tensor's tiles adds zeros)
+    if (jobs.w_src != nullptr && blocks < jobs.Cout) blocks = jobs.Cout;
+    if (jobs.zero != nullptr && blocks < static_cast<long long>(jobs.zero_bytes / (16 * kThreads * 4))) blocks = static_cast<long long>(jobs.zero_bytes / (16 * kThreads * 4));
     if (blocks > ctx->partial_blocks) blocks = ctx->partial_blocks;
     cudaError_t e;
     if (dtype == DBP_F32)

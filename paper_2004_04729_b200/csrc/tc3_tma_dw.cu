@@ -320,46 +320,64 @@ tc3_tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     }
 }
 
-// dW[co][ci][tap] = Delta * acc[tap][co][ci]; the scratch goes back to zero for the next call.
-// A block takes 256 consecutive (co, ci) pairs: nine coalesced reads, a transposition through shared
-// memory, and the 256 x 9 results leave as one contiguous run.
-__global__ void __launch_bounds__(256)
-tc3_dw_finish_kernel(float *__restrict__ acc, const float *__restrict__ delta_p, float *__restrict__ dW, long long pairs) {
+// dW[co][ci][tap] = Delta * acc[tap][co][cip]; the scratch goes back to zero for the next call. The scratch
+// rows hold cin_pad >= Cin channels (activations whose channel count is no multiple of 8 were padded).
+// A block takes 256 consecutive (co, cip) pairs, four per thread: nine coalesced 16-byte reads, a
+// transposition through shared memory, and the results leave as contiguous runs.
+__global__ void __launch_bounds__(64)
+tc3_dw_finish_kernel(float *__restrict__ acc, const float *__restrict__ delta_p, float *__restrict__ dW, long long pairs,
+                     int cin, int cin_pad) {
     __shared__ float t_s[256 * 9];
     chain_wait();
     chain_release();
     const float delta = *delta_p;
     for (long long i0 = blockIdx.x * 256ll; i0 < pairs; i0 += gridDim.x * 256ll) {
-        const long long i = i0 + threadIdx.x;
+        const long long i = i0 + 4 * threadIdx.x;                 // pairs is a multiple of 8
         if (i < pairs) {
 #pragma unroll
             for (int t = 0; t < 9; ++t) {
-                t_s[threadIdx.x * 9 + t] = __ldcg(acc + t * pairs + i) * delta;
-                __stcg(acc + t * pairs + i, 0.f);
+                float4 *src = reinterpret_cast<float4 *>(acc + t * pairs + i);
+                const float4 v = __ldcg(src);
+                __stcg(src, make_float4(0.f, 0.f, 0.f, 0.f));
+                t_s[(4 * threadIdx.x + 0) * 9 + t] = v.x * delta;
+                t_s[(4 * threadIdx.x + 1) * 9 + t] = v.y * delta;
+                t_s[(4 * threadIdx.x + 2) * 9 + t] = v.z * delta;
+                t_s[(4 * threadIdx.x + 3) * 9 + t] = v.w * delta;
             }
         }
         __syncthreads();
         const long long left = pairs - i0;
-        const int n = static_cast<int>(left < 256 ? left : 256) * 9;
-        for (int k = threadIdx.x; k < n; k += 256) dW[i0 * 9 + k] = t_s[k];
+        const int np = static_cast<int>(left < 256 ? left : 256);
+        if (cin == cin_pad) {
+            for (int k = threadIdx.x; k < np * 9; k += 64) dW[i0 * 9 + k] = t_s[k];
+        } else {
+            for (int k = threadIdx.x; k < np * 9; k += 64) {
+                const long long pr = i0 + k / 9;
+                const long long co = pr / cin_pad;
+                const int ci = static_cast<int>(pr - co * cin_pad);
+                if (ci < cin) dW[(co * cin + ci) * 9 + k % 9] = t_s[k];
+            }
+        }
         __syncthreads();
     }
 }
 
-// fp32 activations [planes][HW] -> two bf16 tensors of the same shape, one after the other, rows padded to
-// `pitch` (a multiple of 8): the values rounded to bf16 and what that rounding left over, rounded again.
-// The two pieces add up to the fp32 value to within 2^-18 of it.
+// fp32 activations [B][Cin][HW] -> two bf16 tensors [B][cin_pad][pitch], one after the other: the values rounded
+// to bf16 and what that rounding left over, rounded again (the two pieces add up to the fp32 value to within
+// 2^-18 of it). Rows are padded to `pitch` (a multiple of 8) and channels to cin_pad (a multiple of 8) with zeros.
 __global__ void __launch_bounds__(256)
-x_split_kernel(const float *__restrict__ X, __nv_bfloat16 *__restrict__ out, long long planes, int HW, int pitch) {
+x_split_kernel(const float *__restrict__ X, __nv_bfloat16 *__restrict__ out, long long B, int Cin, int cin_pad, int HW, int pitch) {
     chain_wait();
     chain_release();
-    const long long n = planes * pitch;
+    const long long n = B * cin_pad * pitch;
     for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += gridDim.x * 256ll) {
         const long long pl = i / pitch;
         const int pp = static_cast<int>(i - pl * pitch);
+        const long long b = pl / cin_pad;
+        const int ci = static_cast<int>(pl - b * cin_pad);
         __nv_bfloat16 hi = __float2bfloat16_rn(0.f), lo = hi;
-        if (pp < HW) {
-            const float x = __ldg(X + pl * HW + pp);
+        if (pp < HW && ci < Cin) {
+            const float x = __ldg(X + (b * Cin + ci) * HW + pp);
             hi = __float2bfloat16_rn(x);
             lo = __float2bfloat16_rn(x - __bfloat162float(hi));
         }
@@ -375,15 +393,18 @@ int round_up(int v, int m) { return (v + m - 1) / m * m; }
 // DBP_EUNSUPPORTED: the shape does not fit (the caller uses another kernel)
 int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, int io, const float *delta_p,
                       const ConvShape &s, float *dW, int *err_flag) {
-    if (!tc3_tma_supported(s, io)) return DBP_EUNSUPPORTED;
+    if (!tc3_tma_dw_supported(s, io)) return DBP_EUNSUPPORTED;
     const int pieces = io == DBP_F32 ? 2 : 1;
+    // fp32 activations are re-written anyway (split into two bf16 pieces): their channels are padded to a
+    // multiple of 8 on the way, so any Cin works there
+    const long long cin_pad = io == DBP_F32 ? (s.Cin + 7) / 8 * 8 : s.Cin;
     const long long HW = s.H * s.W;
     Dw3T p{};
-    p.Cin = static_cast<int>(s.Cin); p.Cout = static_cast<int>(s.Cout); p.W = static_cast<int>(s.W); p.HW = static_cast<int>(HW);
+    p.Cin = static_cast<int>(cin_pad); p.Cout = static_cast<int>(s.Cout); p.W = static_cast<int>(s.W); p.HW = static_cast<int>(HW);
     p.err_flag = err_flag;
     p.stats = ctx->wait_stats;
     const int NP = s.Cout > 64 ? 2 : 1;
-    p.ci_tiles = static_cast<int>((s.Cin + 127) / 128);
+    p.ci_tiles = static_cast<int>((cin_pad + 127) / 128);
     p.co_tiles = static_cast<int>((s.Cout + 64 * NP - 1) / (64 * NP));
     // the longest segment whose two code buffers fit beside at least three activation slots
     const size_t budget = 227 * 1024 - 2048;
@@ -410,7 +431,7 @@ int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, int i
     p.nsplit = static_cast<int>(nsplit);
     if (tiles * nsplit >= (1ll << 31)) return DBP_EUNSUPPORTED;
     // fp32 scratch [9][Cout][Cin]: zero whenever no call is in flight
-    const size_t pairs = static_cast<size_t>(s.Cout) * s.Cin;
+    const size_t pairs = static_cast<size_t>(s.Cout) * cin_pad;
     const size_t had = ctx->dw_acc.bytes;
     int rc = ws_reserve(ctx, ctx->dw_acc, pairs * 9 * sizeof(float));
     if (rc) return rc;
@@ -426,13 +447,13 @@ int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, int i
     long long xpitch = HW;
     if (io == DBP_F32) {
         xpitch = (HW + 7) / 8 * 8;
-        const long long planes = s.B * s.Cin;
+        const long long planes = s.B * cin_pad;
         if ((rc = ws_reserve(ctx, ctx->x_padded, static_cast<size_t>(planes) * xpitch * 2 * 2))) return rc;
         long long blocks = (planes * xpitch + 255) / 256;
         if (blocks > ctx->sm_count * 16) blocks = ctx->sm_count * 16;
         if ((rc = cuda_ok(launch_chained(x_split_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, ctx->stream,
-                                         static_cast<const float *>(X), static_cast<__nv_bfloat16 *>(ctx->x_padded.ptr), planes,
-                                         static_cast<int>(HW), static_cast<int>(xpitch)))))
+                                         static_cast<const float *>(X), static_cast<__nv_bfloat16 *>(ctx->x_padded.ptr), s.B,
+                                         static_cast<int>(s.Cin), static_cast<int>(cin_pad), static_cast<int>(HW), static_cast<int>(xpitch)))))
             return rc;
         Xsrc = ctx->x_padded.ptr;
     } else if (HW % 8 != 0) {
@@ -444,8 +465,8 @@ int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, int i
     }
     CUtensorMap map_q, map_x, map_acc;
     {
-        const unsigned long long dims[2] = {static_cast<unsigned long long>(s.Cin), static_cast<unsigned long long>(s.Cout) * 9};
-        const unsigned long long str[1] = {static_cast<unsigned long long>(s.Cin) * 4};
+        const unsigned long long dims[2] = {static_cast<unsigned long long>(cin_pad), static_cast<unsigned long long>(s.Cout) * 9};
+        const unsigned long long str[1] = {static_cast<unsigned long long>(cin_pad) * 4};
         const unsigned box[2] = {128, 32};
         if (!encode_map_f32_rows(&map_acc, acc, 2, dims, str, box)) return fail_cuda("tensor map of the dW scratch");
     }
@@ -458,10 +479,10 @@ int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, int i
         if (!encode_map_bf16(&map_q, codes_nhwc, 3, dims, str, box)) return fail_cuda("tensor map of the code panels");
     }
     {
-        const unsigned long long dims[3] = {static_cast<unsigned long long>(HW), static_cast<unsigned long long>(s.Cin),
+        const unsigned long long dims[3] = {static_cast<unsigned long long>(HW), static_cast<unsigned long long>(cin_pad),
                                             static_cast<unsigned long long>(s.B) * pieces};
         const unsigned long long str[2] = {static_cast<unsigned long long>(xpitch) * 2,
-                                           static_cast<unsigned long long>(xpitch) * 2 * s.Cin};
+                                           static_cast<unsigned long long>(xpitch) * 2 * cin_pad};
         const unsigned box[3] = {64, 128, 1};
         if (!encode_map_bf16(&map_x, Xsrc, 3, dims, str, box)) return fail_cuda("tensor map of the activations");
     }
@@ -472,9 +493,9 @@ int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, int i
                                      ctx->stream, map_q, map_x, map_acc, p))))
         return rc;
     long long blocks = (static_cast<long long>(pairs) + 255) / 256;
-    if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
-    return cuda_ok(launch_chained(tc3_dw_finish_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, ctx->stream, acc,
-                                  delta_p, dW, static_cast<long long>(pairs)));
+    if (blocks > ctx->sm_count * 16) blocks = ctx->sm_count * 16;
+    return cuda_ok(launch_chained(tc3_dw_finish_kernel, dim3(static_cast<unsigned>(blocks)), dim3(64), 0, ctx->stream, acc,
+                                  delta_p, dW, static_cast<long long>(pairs), static_cast<int>(s.Cin), static_cast<int>(cin_pad)));
 }
 
 }  // namespace dbp

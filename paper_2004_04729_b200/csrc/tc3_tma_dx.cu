@@ -391,6 +391,15 @@ bool tc3_tma_supported(const ConvShape &s, int io) {
            s.H <= 4096 && s.B * s.H * s.W < (1ll << 30);
 }
 
+// The weight-gradient kernel alone also takes fp32 layers whose input channel count is no multiple of 8 (a
+// network's first layer): its activations are re-written channel-padded anyway.
+bool tc3_tma_dw_supported(const ConvShape &s, int io) {
+    if (tc3_tma_supported(s, io)) return true;
+    ConvShape t = s;
+    t.Cin = (s.Cin + 7) / 8 * 8;
+    return io == DBP_F32 && tc3_tma_supported(t, io);
+}
+
 // DBP_EUNSUPPORTED: the shape does not fit (the caller uses another kernel)
 int launch_tc3_tma_dx(dbp_ctx *ctx, const void *codes_nhwc, const void *W, int io, const float *delta_p,
                       const ConvShape &s, void *dX, bool dx_bf16, int *err_flag, bool weights_ready) {

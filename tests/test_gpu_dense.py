@@ -113,6 +113,25 @@ def test_dense_path_conv3x3_fp32_operands(ctx, B, Ci, Co, H, W):
     _run(ctx, L, dbp.DBP_FORCE_DENSE)
 
 
+@pytest.mark.parametrize("B,Ci,Co,H,W", [(4, 3, 64, 32, 32), (2, 5, 16, 7, 9), (3, 12, 8, 4, 4)])
+def test_dense_path_first_layer_dw_fp32(ctx, B, Ci, Co, H, W):
+    """A network's first layer (few input channels, no dX wanted): the fp32 weight gradient alone runs on the
+    tensor cores, the activations being padded to eight channels while they are split into bf16 pieces."""
+    import paper_2004_04729_b200 as dbp
+    L = wl.conv_layer(B, Ci, Co, H, W, 3, data_seed=5 + Ci, scale=2.0, dtype="f32")
+    d, X, Wt = _f32(L.delta), _f32(L.X), _f32(L.W)
+    q = dbp.SparseGradient(d.numel())
+    out = dbp.dithered_conv_backward(ctx, d, X, Wt, L.seed, L.scale, q_out=q, need_dX=False, flags=dbp.DBP_FORCE_DENSE)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == (0, 0)
+    D = np.float32(q.delta.item())
+    codes, nnz, _ = oracle.nsd_codes(L.delta, L.seed, D)
+    ref = oracle.conv_backward(codes, D, L.X, L.W, with_abs=True)
+    got = out["dW"].double().cpu().numpy()
+    assert np.linalg.norm(got - ref["dW"]) / np.linalg.norm(ref["dW"]) <= TOL
+    assert np.all(np.abs(got - ref["dW"]) <= TOL * ref["S_dW"] + 1e-30)
+
+
 @pytest.mark.parametrize("B,N,K", [(128, 300, 784), (256, 512, 2048), (70, 10, 512), (33, 100, 304)])
 def test_dense_path_linear(ctx, B, N, K):
     import paper_2004_04729_b200 as dbp
