@@ -314,23 +314,40 @@ __global__ void __launch_bounds__(256) bias_grad_kernel(const int8_t *__restrict
     }
 }
 
-__global__ void relu_backward_kernel(const float *__restrict__ da, const uint8_t *__restrict__ mask,
-                                     float *__restrict__ dz, long long n) {
-    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < n;
-         i += static_cast<long long>(gridDim.x) * blockDim.x)
-        dz[i] = mask[i] ? da[i] : 0.f;
+// delta_z = delta_a (.) f'(z), the derivative given as one byte per element; four elements per thread where
+// the size and the pointers allow
+__global__ void __launch_bounds__(256) relu_backward_kernel(const float *__restrict__ da, const uint8_t *__restrict__ mask,
+                                                            float *__restrict__ dz, long long n, int vec) {
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+    if (vec) {
+        const long long n4 = n >> 2;
+        for (; i < n4; i += stride) {
+            const float4 a = __ldg(reinterpret_cast<const float4 *>(da) + i);
+            const uchar4 m = __ldg(reinterpret_cast<const uchar4 *>(mask) + i);
+            reinterpret_cast<float4 *>(dz)[i] = make_float4(m.x ? a.x : 0.f, m.y ? a.y : 0.f, m.z ? a.z : 0.f, m.w ? a.w : 0.f);
+        }
+        return;
+    }
+    for (; i < n; i += stride) dz[i] = mask[i] ? da[i] : 0.f;
 }
 
-__global__ void maxpool_backward_kernel(const float *__restrict__ g, const int8_t *__restrict__ am,
-                                        float *__restrict__ out, long long planes, long long h,
-                                        long long w) {
-    const long long n = planes * h * w * 4;
+// Routing of a pooled gradient g [planes][h][w] to out [planes][2h][2w]: one thread per window, which writes
+// its four outputs (two pairs); argmax in {0,1,2,3} is the row-major position of the forward maximum
+__global__ void __launch_bounds__(256) maxpool_backward_kernel(const float *__restrict__ g, const int8_t *__restrict__ am,
+                                                               float *__restrict__ out, long long planes, int h, int w) {
+    const long long n = planes * h * w;
     for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < n;
          i += static_cast<long long>(gridDim.x) * blockDim.x) {
-        const long long X = i % (2 * w), Y = (i / (2 * w)) % (2 * h), pl = i / (4 * h * w);
-        const long long src = (pl * h + (Y >> 1)) * w + (X >> 1);
-        const int which = static_cast<int>((Y & 1) * 2 + (X & 1));
-        out[i] = (am[src] == which) ? g[src] : 0.f;
+        const long long row = i / w;                    // (plane, y)
+        const int x = static_cast<int>(i - row * w);
+        const long long pl = row / h;
+        const int y = static_cast<int>(row - pl * h);
+        const float v = __ldg(g + i);
+        const int which = am[i];
+        float *o = out + ((pl * 2 * h + 2 * y) * 2ll * w + 2 * x);
+        *reinterpret_cast<float2 *>(o) = make_float2(which == 0 ? v : 0.f, which == 1 ? v : 0.f);
+        *reinterpret_cast<float2 *>(o + 2 * w) = make_float2(which == 2 ? v : 0.f, which == 3 ? v : 0.f);
     }
 }
 
@@ -474,15 +491,17 @@ int launch_bias_grad(dbp_ctx *ctx, const int8_t *codes, const float *delta_p, co
 
 int launch_relu_backward(dbp_ctx *ctx, const float *da, const uint8_t *mask, float *dz, long long n) {
     note_launch();
-    relu_backward_kernel<<<blocks_for(n, 256, ctx->sm_count * 8), 256, 0, ctx->stream>>>(da, mask, dz, n);
+    const int vec = (n % 4 == 0) && ((reinterpret_cast<uintptr_t>(da) | reinterpret_cast<uintptr_t>(dz)) % 16 == 0) &&
+                    (reinterpret_cast<uintptr_t>(mask) % 4 == 0);
+    relu_backward_kernel<<<blocks_for(vec ? n / 4 : n, 256, ctx->sm_count * 8), 256, 0, ctx->stream>>>(da, mask, dz, n, vec);
     return cuda_ok(cudaGetLastError());
 }
 
 int launch_maxpool_backward(dbp_ctx *ctx, const float *g, const int8_t *argmax, float *out,
                             long long planes, long long h, long long w) {
     note_launch();
-    maxpool_backward_kernel<<<blocks_for(planes * h * w * 4, 256, ctx->sm_count * 8), 256, 0, ctx->stream>>>(
-        g, argmax, out, planes, h, w);
+    maxpool_backward_kernel<<<blocks_for(planes * h * w, 256, ctx->sm_count * 8), 256, 0, ctx->stream>>>(
+        g, argmax, out, planes, static_cast<int>(h), static_cast<int>(w));
     return cuda_ok(cudaGetLastError());
 }
 
