@@ -3,10 +3,10 @@
 // bitmap / offsets / packed-values structure. Used when the caller did not ask for the sparse
 // structure, so the pass costs one read of delta_z and one write of the codes.
 //
-// The common case (every |x / Delta + u| <= 127, no NaN) runs without clamping: the code's
-// two's-complement byte is the low byte of the round-down sum with 1.5 * 2^23. A vector that
-// holds a NaN or a value outside that range is redone element by element with the clipped,
-// counted decision.
+// The common case (every |x / Delta + u| <= 127, no NaN) runs without clamping or conversions:
+// the code is the round-down sum with 1.5 * 2^23, less that constant (a float holding a small
+// integer, whose upper half is its bf16). A vector that holds a NaN or a value outside that range
+// is redone element by element with the clipped, counted decision.
 #include "dbp_internal.cuh"
 
 namespace dbp {
@@ -14,6 +14,10 @@ namespace dbp {
 namespace {
 
 constexpr int kThreads = 256;
+#ifndef DBP_Q_BLOCKS_PER_SM
+#define DBP_Q_BLOCKS_PER_SM 4
+#endif
+constexpr int kBlocksPerSM = DBP_Q_BLOCKS_PER_SM;   // resident blocks the dense quantizer is compiled for
 constexpr unsigned kFull = 0xffffffffu;
 constexpr unsigned long long kGamma = 0x9E3779B97F4A7C15ull;
 
@@ -26,25 +30,26 @@ __device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
 __device__ __forceinline__ float dither(unsigned h) {
     return __uint_as_float(__funnelshift_r(h, 0x7fu, 9)) - 0.99999994f;
 }
-// careful decision: clipped to [-127, 127], clipped codes counted, NaN gives 0
-__device__ __forceinline__ unsigned careful_byte(float x, float inv, float u, unsigned &sat) {
+constexpr float kMagic = 12582912.0f;             // 1.5 * 2^23: a float in [2^23, 2^24) has unit spacing
+// careful decision: clipped to [-127, 127], clipped codes counted, NaN gives 0. Returns the bits of
+// kMagic + code (the low byte is the code's two's-complement byte).
+__device__ __forceinline__ unsigned careful_bits(float x, float inv, float u, unsigned &sat) {
     const float t = __fmaf_rn(x, inv, u);
     const float tc = fminf(fmaxf(t, -127.f), 127.99999f);
     const bool num = (t == t);
     sat += (num && tc != t) ? 1u : 0u;
-    const unsigned q = __float_as_uint(__fadd_rd(tc, 12582912.0f)) & 0xffu;
-    return num ? q : 0u;
+    return num ? __float_as_uint(__fadd_rd(tc, kMagic)) : __float_as_uint(kMagic);
 }
-// number of non-zero bytes of a word
-__device__ __forceinline__ unsigned nonzero_bytes(unsigned w) {
-    return __popc((((w & 0x7f7f7f7fu) + 0x7f7f7f7fu) | w) & 0x80808080u);
+__device__ __forceinline__ unsigned careful_byte(float x, float inv, float u, unsigned &sat) {
+    return careful_bits(x, inv, u, sat) & 0xffu;
 }
-
-// Codes of the V elements x[0..V) whose first element has the (even) linear index e0; packed
-// four to a word in element order. V is 4 or 8.
+// Codes of the V elements x[0..V) whose first element has the (even) linear index e0, as floats
+// (exact small integers). V is 4 or 8. The common case (every |t| <= 127, no NaN) is recognised by
+// the sum of the squares of t = x / Delta + u and needs no clamp: floor(t) is the round-down sum
+// with kMagic, less kMagic. The number of non-zero codes is added to nz (a float: exact below 2^24).
 template <int V>
 __device__ __forceinline__ void codes_of(const float (&x)[V], long long e0, unsigned long long seed,
-                                         float inv, unsigned (&pk)[V / 4], unsigned &sat) {
+                                         float inv, float (&f)[V], float &nz, unsigned &sat) {
     unsigned long long z = seed + (static_cast<unsigned long long>(e0 >> 1) + 1ull) * kGamma;
     float u[V];
 #pragma unroll
@@ -54,35 +59,36 @@ __device__ __forceinline__ void codes_of(const float (&x)[V], long long e0, unsi
         u[j] = dither(static_cast<unsigned>(r));
         u[j + 1] = dither(static_cast<unsigned>(r >> 32));
     }
-    unsigned b[V];
-    float amax = 0.f, sum = 0.f;
+    float s2 = 0.f;
 #pragma unroll
     for (int j = 0; j < V; ++j) {
         const float t = __fmaf_rn(x[j], inv, u[j]);
-        amax = fmaxf(amax, fabsf(t));
-        sum += t;                                   // NaN iff some t is NaN (or +inf meets -inf)
-        b[j] = __float_as_uint(__fadd_rd(t, 12582912.0f));
+        s2 = __fmaf_rn(t, t, s2);                   // NaN or inf if some t is; > 127^2 if some |t| > 127
+        f[j] = __fadd_rd(t, kMagic) - kMagic;
     }
-    if (!(amax <= 127.f) || sum != sum) {           // rare: clip, count, NaN
+    if (!(s2 <= 16128.f)) {                         // rare: clip, count, NaN
 #pragma unroll
-        for (int j = 0; j < V; ++j) b[j] = careful_byte(x[j], inv, u[j], sat);
+        for (int j = 0; j < V; ++j) f[j] = __uint_as_float(careful_bits(x[j], inv, u[j], sat)) - kMagic;
     }
+#pragma unroll
+    for (int j = 0; j < V; ++j) nz += __saturatef(f[j] * f[j]);
+}
+// the codes' bytes, four to a word in element order
+template <int V>
+__device__ __forceinline__ void pack_bytes(const float (&f)[V], unsigned (&pk)[V / 4]) {
+    unsigned b[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) b[j] = __float_as_uint(f[j] + kMagic);     // low byte: the code
 #pragma unroll
     for (int w = 0; w < V / 4; ++w)
         pk[w] = __byte_perm(__byte_perm(b[4 * w], b[4 * w + 1], 0x0040), __byte_perm(b[4 * w + 2], b[4 * w + 3], 0x0040), 0x5410);
 }
-
-
-// four packed code bytes -> four bf16 (exact): byte ^ 0x80 is code + 128; 0x4B0000xx read as a
-// float is 2^23 + xx, so subtracting 2^23 + 128 leaves the code, whose top half is its bf16
-__device__ __forceinline__ void bytes4_to_bf16(unsigned w, unsigned &lo, unsigned &hi) {
-    const unsigned x = w ^ 0x80808080u;
-    const float f0 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7650)) - 8388736.0f;
-    const float f1 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7651)) - 8388736.0f;
-    const float f2 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7652)) - 8388736.0f;
-    const float f3 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7653)) - 8388736.0f;
-    lo = __byte_perm(__float_as_uint(f0), __float_as_uint(f1), 0x7632);
-    hi = __byte_perm(__float_as_uint(f2), __float_as_uint(f3), 0x7632);
+// the codes as bf16, two to a word: an integer of at most 8 bits is exact in bf16, which is the
+// float's upper half
+template <int V>
+__device__ __forceinline__ void pack_bf16(const float (&f)[V], unsigned (&h)[V / 2]) {
+#pragma unroll
+    for (int j = 0; j < V / 2; ++j) h[j] = __byte_perm(__float_as_uint(f[2 * j]), __float_as_uint(f[2 * j + 1]), 0x7632);
 }
 
 // Where the codes go. dense8: one byte per element, same order as delta_z (may be null).
@@ -109,15 +115,16 @@ __device__ __forceinline__ void split_index(long long e, long long hw, long long
 }
 
 template <int V>
-__device__ __forceinline__ void store_codes(const CodeSinks &o, long long e0, const unsigned (&pk)[V / 4]) {
+__device__ __forceinline__ void store_codes(const CodeSinks &o, long long e0, const float (&f)[V]) {
     if (o.dense8 != nullptr) {
+        unsigned pk[V / 4];
+        pack_bytes<V>(f, pk);
         if (V == 4) *reinterpret_cast<unsigned *>(o.dense8 + e0) = pk[0];
         else *reinterpret_cast<uint2 *>(o.dense8 + e0) = make_uint2(pk[0], pk[V / 4 - 1]);
     }
     if (o.planes16 != nullptr) {
         unsigned h[V / 2];
-#pragma unroll
-        for (int w = 0; w < V / 4; ++w) bytes4_to_bf16(pk[w], h[2 * w], h[2 * w + 1]);
+        pack_bf16<V>(f, h);
         if (o.pitch == o.hw) {                      // planes are back to back: same order as delta_z
             if (V == 4) *reinterpret_cast<uint2 *>(o.planes16 + e0) = make_uint2(h[0], h[1]);
             else *reinterpret_cast<uint4 *>(o.planes16 + e0) = make_uint4(h[0], h[1], h[V / 2 - 2], h[V / 2 - 1]);
@@ -133,12 +140,26 @@ __device__ __forceinline__ void store_codes(const CodeSinks &o, long long e0, co
                 if (pp == o.hw) { pp = 0; ++plane; }
             }
         } else {
+            // odd plane sizes: code by code, or two at a time where the pair starts on an even offset
+            // of its plane and does not run over the plane's end
             long long plane, pp;
             split_index(e0, o.hw, plane, pp);
+            unsigned short *dst = o.planes16 + plane * o.pitch + pp;
+            long long left = o.hw - pp;                           // codes until the plane ends
+            const long long gap = o.pitch - o.hw;
 #pragma unroll
-            for (int j = 0; j < V; ++j) {
-                o.planes16[plane * o.pitch + pp] = static_cast<unsigned short>(h[j >> 1] >> (16 * (j & 1)));
-                if (++pp == o.hw) { pp = 0; ++plane; }
+            for (int j = 0; j < V; j += 2) {
+                if (left >= 2 && (reinterpret_cast<uintptr_t>(dst) & 3) == 0) {
+                    *reinterpret_cast<unsigned *>(dst) = h[j >> 1];
+                    dst += 2;
+                    left -= 2;
+                    if (left == 0) { left = o.hw; dst += gap; }
+                } else {
+                    *dst++ = static_cast<unsigned short>(h[j >> 1]);
+                    if (--left == 0) { left = o.hw; dst += gap; }
+                    *dst++ = static_cast<unsigned short>(h[j >> 1] >> 16);
+                    if (--left == 0) { left = o.hw; dst += gap; }
+                }
             }
         }
     }
@@ -181,7 +202,7 @@ struct Vec<__nv_bfloat16> {
 };
 
 template <typename T>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, kBlocksPerSM)
 quantize_dense_kernel(const T *__restrict__ x, long long n, unsigned long long seed,
                       const float *__restrict__ delta_p, const CodeSinks out,
                       DeviceState *__restrict__ st) {
@@ -195,7 +216,7 @@ quantize_dense_kernel(const T *__restrict__ x, long long n, unsigned long long s
     const bool live = (delta > 0.f) && (delta < __int_as_float(0x7f800000));
     if (!live) {                                    // sigma = 0 or non-finite input: every code is 0
         for (; i < nvec; i += stride) {
-            const unsigned zero[V / 4] = {};
+            const float zero[V] = {};
             store_codes<V>(out, i * V, zero);
         }
         if (blockIdx.x == 0 && threadIdx.x == 0)
@@ -204,28 +225,26 @@ quantize_dense_kernel(const T *__restrict__ x, long long n, unsigned long long s
     }
     const float inv = __fdiv_rn(1.0f, delta);
     unsigned nnz = 0, sat = 0;
+    float nz = 0.f;
     // two vectors in flight per thread
     for (; i + stride < nvec; i += 2 * stride) {
         float a[V], b[V];
         Vec<T>::load(x + i * V, a);
         Vec<T>::load(x + (i + stride) * V, b);
-        unsigned pa[V / 4], pb[V / 4];
-        codes_of<V>(a, i * V, seed, inv, pa, sat);
-        codes_of<V>(b, (i + stride) * V, seed, inv, pb, sat);
-        store_codes<V>(out, i * V, pa);
-        store_codes<V>(out, (i + stride) * V, pb);
-#pragma unroll
-        for (int w = 0; w < V / 4; ++w) nnz += nonzero_bytes(pa[w]) + nonzero_bytes(pb[w]);
+        float fa[V], fb[V];
+        codes_of<V>(a, i * V, seed, inv, fa, nz, sat);
+        codes_of<V>(b, (i + stride) * V, seed, inv, fb, nz, sat);
+        store_codes<V>(out, i * V, fa);
+        store_codes<V>(out, (i + stride) * V, fb);
     }
     if (i < nvec) {
         float a[V];
         Vec<T>::load(x + i * V, a);
-        unsigned pa[V / 4];
-        codes_of<V>(a, i * V, seed, inv, pa, sat);
-        store_codes<V>(out, i * V, pa);
-#pragma unroll
-        for (int w = 0; w < V / 4; ++w) nnz += nonzero_bytes(pa[w]);
+        float fa[V];
+        codes_of<V>(a, i * V, seed, inv, fa, nz, sat);
+        store_codes<V>(out, i * V, fa);
     }
+    nnz = static_cast<unsigned>(nz);                // a thread's share is far below 2^24 elements
     if (blockIdx.x == 0 && threadIdx.x == 0) {      // the n % V last elements, one by one
         for (long long e = nvec * V; e < n; ++e) {
             const unsigned long long r = mix64(seed + (static_cast<unsigned long long>(e >> 1) + 1ull) * kGamma);
@@ -271,17 +290,13 @@ __device__ __forceinline__ unsigned tile_off(int p, int c) {
 }
 
 // one element by itself (planes whose size is odd: the pair that shares a draw may straddle two
-// vectors); same decision as codes_of
-__device__ __forceinline__ unsigned code_single(float x, long long e, unsigned long long seed, float inv, unsigned &sat) {
+// vectors); same decision as codes_of. Returns the code as a float.
+__device__ __forceinline__ float code_single(float x, long long e, unsigned long long seed, float inv, unsigned &sat) {
     const unsigned long long r = mix64(seed + (static_cast<unsigned long long>(e >> 1) + 1ull) * kGamma);
     const float u = dither((e & 1) ? static_cast<unsigned>(r >> 32) : static_cast<unsigned>(r));
     const float t = __fmaf_rn(x, inv, u);
-    if (fabsf(t) <= 127.f) return __float_as_uint(__fadd_rd(t, 12582912.0f)) & 0xffu;
-    return careful_byte(x, inv, u, sat);
-}
-__device__ __forceinline__ unsigned short byte_to_bf16(unsigned b) {
-    const float f = static_cast<float>(static_cast<int>(static_cast<signed char>(b)));
-    return static_cast<unsigned short>(__float_as_uint(f) >> 16);
+    if (fabsf(t) <= 127.f) return __fadd_rd(t, kMagic) - kMagic;
+    return __uint_as_float(careful_bits(x, inv, u, sat)) - kMagic;
 }
 
 template <typename T, int V>
@@ -303,14 +318,27 @@ struct TileLoad<float, 4> {
     __device__ static void ld(const float *p, float (&v)[4]) { Vec<float>::load(p, v); }
 };
 
-// V: elements per load (plane size % V == 0), or 1 for element-wise loads (any plane size)
+template <int V>
+__device__ __forceinline__ void store_bytes(int8_t *dense8, long long e0, const float (&f)[V]) {
+    unsigned pk[V / 4];
+    pack_bytes<V>(f, pk);
+    if (V == 4) *reinterpret_cast<unsigned *>(dense8 + e0) = pk[0];
+    else *reinterpret_cast<uint2 *>(dense8 + e0) = make_uint2(pk[0], pk[V / 4 - 1]);
+}
+
+// V: elements per load (plane size % V == 0), or 1 for element-wise loads (any plane size).
+// Three ways to fill a tile. Planes smaller than a tile's 64 positions: the tile's 64 channels of one
+// image are one contiguous run of delta_z, read as whole vectors whatever the plane size. Otherwise,
+// plane size % V == 0: a thread takes the same V positions of two neighbouring channels and writes
+// the two codes of a position as one word. Otherwise element by element.
 template <typename T, int V>
 __global__ void __launch_bounds__(kThreads)
 quantize_nhwc_kernel(const T *__restrict__ x, int B, int C, int HW, unsigned long long seed,
                      const float *__restrict__ delta_p, unsigned short *__restrict__ out,
                      int8_t *__restrict__ dense8, DeviceState *__restrict__ st, int count) {
     __shared__ __align__(16) unsigned char tile[2][kTileBytes];
-    constexpr int VV = (V > 1) ? V : 4;               // vector length of the vector path
+    constexpr int VV = (V > 1) ? V : 4;               // vector length of the paired path
+    constexpr int VF = Vec<T>::V;                     // vector length of the contiguous path
     chain_wait();
     chain_release();
     const float delta = *delta_p;
@@ -318,55 +346,73 @@ quantize_nhwc_kernel(const T *__restrict__ x, int B, int C, int HW, unsigned lon
     const float inv = live ? __fdiv_rn(1.0f, delta) : 0.f;
     const int ct = (C + kTC - 1) / kTC, pt = (HW + kTP - 1) / kTP;
     const long long ntiles = static_cast<long long>(B) * ct * pt;
+    const bool flat = HW < kTP;
     unsigned nnz = 0, sat = 0;
+    float nz = 0.f;
     int buf = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, buf ^= 1) {
         const int b = static_cast<int>(t / (ct * pt));
         const int rem = static_cast<int>(t - static_cast<long long>(b) * ct * pt);
         const int c0 = (rem / pt) * kTC, p0 = (rem % pt) * kTP;
         unsigned char *tl = tile[buf];
-        if (V > 1) {
+        if (flat) {
+            // (b, c0 .. c0+63, every position): C % 8 == 0, so the run starts on a 16-byte boundary and on
+            // an even element, and holds a whole number of vectors
+            const int nch = C - c0 < kTC ? C - c0 : kTC;
+            const long long base = (static_cast<long long>(b) * C + c0) * HW;
+            const int nvec = nch * HW / VF;
+            for (int v = threadIdx.x; v < nvec; v += kThreads) {
+                float f[VF] = {};
+                if (live) {
+                    float a[VF];
+                    Vec<T>::load(x + base + v * VF, a);
+                    codes_of<VF>(a, base + v * VF, seed, inv, f, nz, sat);
+                }
+                if (dense8 != nullptr) store_bytes<VF>(dense8, base + v * VF, f);
+                int c = (v * VF) / HW, pp = v * VF - c * HW;
+#pragma unroll
+                for (int j = 0; j < VF; ++j) {
+                    *reinterpret_cast<unsigned short *>(tl + tile_off(pp, c)) = static_cast<unsigned short>(__float_as_uint(f[j]) >> 16);
+                    if (++pp == HW) { pp = 0; ++c; }
+                }
+            }
+        } else if (V > 1) {
             constexpr int VPR = kTP / VV;            // vectors per channel row of the tile
 #pragma unroll
-            for (int i = 0; i < (kTC * VPR) / kThreads; ++i) {
+            for (int i = 0; i < (kTC / 2 * VPR) / kThreads; ++i) {
                 const int v = threadIdx.x + kThreads * i;
-                const int c = v / VPR, pv = (v % VPR) * VV;
-                unsigned pk[VV / 4] = {};
-                const bool in = c0 + c < C && p0 + pv < HW;       // HW % V == 0: whole vectors
-                const long long e0 = (static_cast<long long>(b) * C + c0 + c) * HW + p0 + pv;
+                const int c = 2 * (v / VPR), pv = (v % VPR) * VV;
+                float f0[VV] = {}, f1[VV] = {};
+                const bool in = c0 + c < C && p0 + pv < HW;       // C is even, HW % V == 0: whole vectors, both channels
+                const long long e0 = (static_cast<long long>(b) * C + c0 + c) * HW + p0 + pv, e1 = e0 + HW;
                 if (in && live) {
-                    float a[VV];
-                    TileLoad<T, VV>::ld(x + e0, a);
-                    codes_of<VV>(a, e0, seed, inv, pk, sat);
+                    float a0[VV], a1[VV];
+                    TileLoad<T, VV>::ld(x + e0, a0);
+                    TileLoad<T, VV>::ld(x + e1, a1);
+                    codes_of<VV>(a0, e0, seed, inv, f0, nz, sat);
+                    codes_of<VV>(a1, e1, seed, inv, f1, nz, sat);
                 }
                 if (in && dense8 != nullptr) {
-                    if (VV == 4) *reinterpret_cast<unsigned *>(dense8 + e0) = pk[0];
-                    else *reinterpret_cast<uint2 *>(dense8 + e0) = make_uint2(pk[0], pk[VV / 4 - 1]);
+                    store_bytes<VV>(dense8, e0, f0);
+                    store_bytes<VV>(dense8, e1, f1);
                 }
 #pragma unroll
-                for (int w = 0; w < VV / 4; ++w) {
-                    nnz += nonzero_bytes(pk[w]);
-                    unsigned lo, hi;
-                    bytes4_to_bf16(pk[w], lo, hi);
-                    const int pp = pv + 4 * w;
-                    *reinterpret_cast<unsigned short *>(tl + tile_off(pp, c)) = static_cast<unsigned short>(lo);
-                    *reinterpret_cast<unsigned short *>(tl + tile_off(pp + 1, c)) = static_cast<unsigned short>(lo >> 16);
-                    *reinterpret_cast<unsigned short *>(tl + tile_off(pp + 2, c)) = static_cast<unsigned short>(hi);
-                    *reinterpret_cast<unsigned short *>(tl + tile_off(pp + 3, c)) = static_cast<unsigned short>(hi >> 16);
-                }
+                for (int j = 0; j < VV; ++j)
+                    *reinterpret_cast<unsigned *>(tl + tile_off(pv + j, c)) =
+                        __byte_perm(__float_as_uint(f0[j]), __float_as_uint(f1[j]), 0x7632);
             }
         } else {
 #pragma unroll 4
             for (int i = 0; i < (kTC * kTP) / kThreads; ++i) {
                 const int id = threadIdx.x + kThreads * i;
                 const int c = id / kTP, pp = id % kTP;
-                unsigned q = 0;
+                float f = 0.f;
                 const bool in = c0 + c < C && p0 + pp < HW;
                 const long long e = (static_cast<long long>(b) * C + c0 + c) * HW + p0 + pp;
-                if (in && live) q = code_single(Vec<T>::one(x + e), e, seed, inv, sat);
-                if (in && dense8 != nullptr) dense8[e] = static_cast<int8_t>(q);
-                nnz += q != 0u;
-                *reinterpret_cast<unsigned short *>(tl + tile_off(pp, c)) = byte_to_bf16(q);
+                if (in && live) f = code_single(Vec<T>::one(x + e), e, seed, inv, sat);
+                if (in && dense8 != nullptr) dense8[e] = static_cast<int8_t>(static_cast<int>(f));
+                nnz += f != 0.f;
+                *reinterpret_cast<unsigned short *>(tl + tile_off(pp, c)) = static_cast<unsigned short>(__float_as_uint(f) >> 16);
             }
         }
         __syncthreads();
@@ -381,6 +427,7 @@ quantize_nhwc_kernel(const T *__restrict__ x, int B, int C, int HW, unsigned lon
         }
         // the other buffer is written next; this one again only after the next barrier
     }
+    nnz += static_cast<unsigned>(nz);
     nnz = __reduce_add_sync(kFull, nnz);
     sat = __reduce_add_sync(kFull, sat);
     if ((threadIdx.x & 31) == 0 && count) {
@@ -408,7 +455,7 @@ int launch_quantize_dense(dbp_ctx *ctx, const void *delta, int dtype, long long 
     const int v = dtype == DBP_F32 ? 4 : 8;
     long long blocks = (numel / v + 2 * kThreads - 1) / (2 * kThreads);
     if (blocks < 1) blocks = 1;
-    const long long cap = static_cast<long long>(ctx->sm_count) * 8;
+    const long long cap = static_cast<long long>(ctx->sm_count) * kBlocksPerSM;
     if (blocks > cap) blocks = cap;
     CodeSinks out{dense, static_cast<unsigned short *>(planes_bf16), hw > 0 ? hw : 1, pitch > 0 ? pitch : 1, count ? 1 : 0};
     cudaError_t e;
