@@ -86,6 +86,7 @@ struct DxT {
     const float *delta_p;
     void *dX;                     // [B][Cin][HW], bf16 or fp32
     int dx_f32;
+    int tma_out;                  // bf16 dX whose rows are multiples of 16 bytes: chunks leave through the copy engine
     int Cin, Cout, HW;
     int chunks_per_img;
     long long nchunks;            // B * chunks_per_img
@@ -103,7 +104,8 @@ struct PipeT {
 };
 
 __global__ void __launch_bounds__(kThreadsT, 1)
-tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_q, const DxT p) {
+tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_q,
+              const __grid_constant__ CUtensorMap map_dx, const DxT p) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ PipeT pipe;
@@ -126,6 +128,7 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         tma_prefetch_desc(&map_w);
         tma_prefetch_desc(&map_q);
+        if (p.tma_out) tma_prefetch_desc(&map_dx);
     }
     if (warp == 1) tmem_alloc(&pipe.tmem_base, 2 * kAccCols);
     tc_fence_before();
@@ -241,6 +244,46 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
             for (int c = part; c < nch; c += kEpiWarps / 4) {
                 const long long b = (g0 + c) / p.chunks_per_img;
                 const int p0 = static_cast<int>((g0 + c) % p.chunks_per_img) * 64;
+                if (p.tma_out) {
+                    // the chunk's 32 channels x 64 positions: both halves out of TMEM, scaled and rounded, into the
+                    // staging block as swizzled 128-byte rows, then one tiled store (which skips what lies
+                    // outside the tensor). The block is free again once the previous store has read it.
+                    unsigned v0[32], v1[32];
+                    const unsigned taddr = tmem_base + (static_cast<unsigned>(q * 32) << 16) + a * kAccCols + c * 64;
+                    tmem_ld32(taddr, v0);
+                    tmem_ld32(taddr + 32, v1);
+                    if (lane == 0) bulk_wait_read_all();
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        unsigned w[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v0[8 * j + 2 * i]) * delta,
+                                                                           __uint_as_float(v0[8 * j + 2 * i + 1]) * delta);
+                            w[i] = *reinterpret_cast<const unsigned *>(&h);
+                        }
+                        *reinterpret_cast<uint4 *>(stage + lane * 128 + ((j ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        unsigned w[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v1[8 * j + 2 * i]) * delta,
+                                                                           __uint_as_float(v1[8 * j + 2 * i + 1]) * delta);
+                            w[i] = *reinterpret_cast<const unsigned *>(&h);
+                        }
+                        *reinterpret_cast<uint4 *>(stage + lane * 128 + (((4 + j) ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                    fence_async_proxy();
+                    __syncwarp();
+                    if (lane == 0 && ci_w < p.Cin) {
+                        tma_store_3d(&map_dx, p0, ci_w, static_cast<int>(b), stage);
+                        bulk_commit();
+                    }
+                    continue;
+                }
                 const int nv = p.HW - p0 < 64 ? p.HW - p0 : 64;           // valid positions of the chunk
                 const bool rows128 = nv == 64 && vw >= 4;                 // staged as swizzled 128-byte rows
 #pragma unroll 1
@@ -340,6 +383,7 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
             warp_arrive(&pipe.acc_empty[a]);
           }
         }
+        if (p.tma_out && lane == 0) bulk_wait_read_all();      // the staging block is read before the CTA goes
         if (threadIdx.x == 64) report_wait(p.stats, 5, we);
     }
     tc_fence_before();
@@ -378,6 +422,15 @@ int launch_tma_dx(dbp_ctx *ctx, const void *codes_bf16, const void *W, const flo
     }
     DxT p{};
     p.delta_p = delta_p; p.dX = dX; p.dx_f32 = dx_bf16 ? 0 : 1;
+    CUtensorMap map_dx = map_w;                  // a valid map when the store path is not used
+    p.tma_out = (dx_bf16 && HW % 8 == 0) ? 1 : 0;
+    if (p.tma_out) {
+        const unsigned long long dims[3] = {static_cast<unsigned long long>(HW), static_cast<unsigned long long>(s.Cin),
+                                            static_cast<unsigned long long>(s.B)};
+        const unsigned long long str[2] = {static_cast<unsigned long long>(HW) * 2, static_cast<unsigned long long>(HW) * 2 * s.Cin};
+        const unsigned box[3] = {64, 32, 1};
+        if (!encode_map_bf16(&map_dx, dX, 3, dims, str, box)) return DBP_ECUDA;
+    }
     p.Cin = static_cast<int>(s.Cin); p.Cout = static_cast<int>(s.Cout); p.HW = static_cast<int>(HW);
     p.chunks_per_img = static_cast<int>((HW + 63) / 64);
     p.nchunks = s.B * p.chunks_per_img;
@@ -397,7 +450,7 @@ int launch_tma_dx(dbp_ctx *ctx, const void *codes_bf16, const void *W, const flo
         return DBP_ECUDA;
     const long long grid = p.ntiles < ctx->sm_count ? p.ntiles : ctx->sm_count;
     return cuda_ok(launch_chained(tma_dx_kernel, dim3(static_cast<unsigned>(grid)), dim3(kThreadsT), smem, ctx->stream,
-                                  map_w, map_q, p));
+                                  map_w, map_q, map_dx, p));
 }
 
 }  // namespace dbp
