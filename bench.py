@@ -281,7 +281,8 @@ def dense_times(torch, fns, reps):
 def small_config(torch, dbp, ctx, config, hbm_peak, fma_peak):
     """One of configs 1-4 as a short side measurement: layer (or whole-network backward) time, dense-equivalent
     throughput, fraction of the HBM roofline for the algorithmic bytes, fraction of the fp32 FMA peak for the
-    non-zero FMAs (these fp32 configurations run on the sparse gather kernels), the dense library time."""
+    non-zero FMAs (meaningful for the linear layers, which run on the gather kernels; the fp32 3x3 convolutions run
+    on the tensor cores with operands split into two bf16 pieces), the dense library time."""
     dev = torch.device("cuda", ctx.device)
     if config in (1, 3):
         L = wl.config1() if config == 1 else wl.config3()
@@ -332,8 +333,9 @@ def small_config(torch, dbp, ctx, config, hbm_peak, fma_peak):
             "hbm_frac": nbytes / (ms * 1e-3) / 1e9 / hbm_peak, "algorithmic_mb": nbytes / 1e6,
             "nsd_density": density, "fma_frac": density * flops / (ms * 1e-3) / 1e12 / fma_peak,
             "dense_ms": dt, "launches": launches,
-            "note": "fp32: sparse gather kernels (no tensor-core path for fp32 operands); launch-bound at these sizes"
-                    if config in (1, 2) else "fp32: sparse gather kernels (no tensor-core path for fp32 operands)"}
+            "note": "fp32 linear layers: sparse gather kernels (no tensor-core path for fp32 linear operands); launch-bound at these sizes"
+                    if config in (1, 2) else "fp32 3x3 convolutions: tensor-core kernels, weights and activations split into two bf16 pieces "
+                                             "(codes are exact in bf16); fma_frac does not apply" + ("; the FC layer runs on the gather kernels" if config == 4 else "")}
 
 
 def crossover_sweep(torch, dbp, ctx):
@@ -473,24 +475,24 @@ def main():
     if args.force_sparse:
         name += " [gather kernels forced]"
 
-    def run_layer(L, d, X, W, dW, dX):
+    def run_layer(L, d, X, W, dW, dX, want_dw=True, want_dx=True):
         code = 1 if L.dtype == "bf16" else 0
+        pw, px = (dW.data_ptr() if want_dw else None), (dX.data_ptr() if want_dx else None)
         if L.kind == "linear":
             B, N = d.shape
             rc = lib.dithered_linear_backward(ctx._h, d.data_ptr(), X.data_ptr(), W.data_ptr(), code,
-                                              B, N, X.shape[1], L.seed, L.scale, None, None,
-                                              dW.data_ptr(), dX.data_ptr(), None, FLAGS)
+                                              B, N, X.shape[1], L.seed, L.scale, None, None, pw, px, None, FLAGS)
         else:
             B, Co, H, Wd = d.shape
             rc = lib.dithered_conv_backward(ctx._h, d.data_ptr(), X.data_ptr(), W.data_ptr(), code,
                                             B, X.shape[1], Co, H, Wd, L.k, 1, (L.k - 1) // 2, L.seed,
-                                            L.scale, None, None, dW.data_ptr(), dX.data_ptr(), None, FLAGS)
+                                            L.scale, None, None, pw, px, None, FLAGS)
         if rc != 0:
             raise RuntimeError(f"library call failed on {L.name}: {rc} {lib.dbp_last_error().decode()}")
 
-    def step():
+    def step(want_dw=True, want_dx=True):
         for item in layers:
-            run_layer(*item)
+            run_layer(*item, want_dw=want_dw, want_dx=want_dx)
         ctx.join()
 
     def barrier():
@@ -541,6 +543,23 @@ def main():
     step()
     host_ms = (time.perf_counter() - t0) * 1e3
     barrier()
+
+    # every kind by itself: one product per call, so nothing runs beside anything else (the quantization kinds
+    # are taken from the dX-only pass)
+    alone = {}
+    for want_dw, want_dx in ((False, True), (True, False)):
+        step(want_dw, want_dx)
+        barrier()
+        ctx.profile_enable(True)
+        ctx.profile_select(None)
+        ctx.profile_read()
+        for _ in range(3):
+            step(want_dw, want_dx)
+        barrier()
+        for k, v in ctx.profile_read().items():
+            if v[1] and k not in alone:
+                alone[k] = v[0] / 3
+        ctx.profile_enable(False)
 
     # non-zero work actually done, and the dequantized gradients the dense comparison is fed
     nnz_flops = 0.0
@@ -638,6 +657,11 @@ def main():
         if k in kern:
             kern[k]["work_per_step"] = work[k]
             kern[k]["unit"] = "flop" if k in ("dx", "dw") else "byte"
+    for k in kern:
+        if k in alone:
+            kern[k]["ms_per_step_alone"] = alone[k]
+            if k in work and kern[k].get("unit") == "byte":
+                kern[k]["frac_of_measured_hbm_alone"] = work[k] / (alone[k] * 1e-3) / 1e9 / hbm_peak
     path_gbs = alg_bytes / (ms * 1e-3) / 1e9
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -322,9 +322,10 @@ tc3_tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 
 // dW[co][ci][tap] = Delta * acc[tap][co][cip]; the scratch goes back to zero for the next call. The scratch
 // rows hold cin_pad >= Cin channels (activations whose channel count is no multiple of 8 were padded).
-// A block takes 256 consecutive (co, cip) pairs, four per thread: nine coalesced 16-byte reads, a
-// transposition through shared memory, and the results leave as contiguous runs.
-__global__ void __launch_bounds__(64)
+// A block takes 256 consecutive (co, cip) pairs, one per thread: nine coalesced reads (and the zeros written
+// back), a transposition through shared memory (row pitch 9 words: no bank conflicts either way), and the
+// results leave as one contiguous run.
+__global__ void __launch_bounds__(256)
 tc3_dw_finish_kernel(float *__restrict__ acc, const float *__restrict__ delta_p, float *__restrict__ dW, long long pairs,
                      int cin, int cin_pad) {
     __shared__ float t_s[256 * 9];
@@ -332,26 +333,24 @@ tc3_dw_finish_kernel(float *__restrict__ acc, const float *__restrict__ delta_p,
     chain_release();
     const float delta = *delta_p;
     for (long long i0 = blockIdx.x * 256ll; i0 < pairs; i0 += gridDim.x * 256ll) {
-        const long long i = i0 + 4 * threadIdx.x;                 // pairs is a multiple of 8
+        const long long i = i0 + threadIdx.x;
         if (i < pairs) {
+            float v[9];
+#pragma unroll
+            for (int t = 0; t < 9; ++t) v[t] = __ldcg(acc + t * pairs + i);
 #pragma unroll
             for (int t = 0; t < 9; ++t) {
-                float4 *src = reinterpret_cast<float4 *>(acc + t * pairs + i);
-                const float4 v = __ldcg(src);
-                __stcg(src, make_float4(0.f, 0.f, 0.f, 0.f));
-                t_s[(4 * threadIdx.x + 0) * 9 + t] = v.x * delta;
-                t_s[(4 * threadIdx.x + 1) * 9 + t] = v.y * delta;
-                t_s[(4 * threadIdx.x + 2) * 9 + t] = v.z * delta;
-                t_s[(4 * threadIdx.x + 3) * 9 + t] = v.w * delta;
+                __stcg(acc + t * pairs + i, 0.f);
+                t_s[threadIdx.x * 9 + t] = v[t] * delta;
             }
         }
         __syncthreads();
         const long long left = pairs - i0;
         const int np = static_cast<int>(left < 256 ? left : 256);
         if (cin == cin_pad) {
-            for (int k = threadIdx.x; k < np * 9; k += 64) dW[i0 * 9 + k] = t_s[k];
+            for (int k = threadIdx.x; k < np * 9; k += 256) dW[i0 * 9 + k] = t_s[k];
         } else {
-            for (int k = threadIdx.x; k < np * 9; k += 64) {
+            for (int k = threadIdx.x; k < np * 9; k += 256) {
                 const long long pr = i0 + k / 9;
                 const long long co = pr / cin_pad;
                 const int ci = static_cast<int>(pr - co * cin_pad);
@@ -494,7 +493,7 @@ int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, int i
         return rc;
     long long blocks = (static_cast<long long>(pairs) + 255) / 256;
     if (blocks > ctx->sm_count * 16) blocks = ctx->sm_count * 16;
-    return cuda_ok(launch_chained(tc3_dw_finish_kernel, dim3(static_cast<unsigned>(blocks)), dim3(64), 0, ctx->stream, acc,
+    return cuda_ok(launch_chained(tc3_dw_finish_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, ctx->stream, acc,
                                   delta_p, dW, static_cast<long long>(pairs), static_cast<int>(s.Cin), static_cast<int>(cin_pad)));
 }
 
