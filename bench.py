@@ -278,6 +278,15 @@ def dense_times(torch, fns, reps):
     return out
 
 
+def tensor_peak():
+    """Measured dense bf16 rate (TFLOP/s, burst) and where it comes from."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured (MEASURED_PEAKS.json bf16_tflops, burst)"
+    except (OSError, KeyError, ValueError):
+        return 1590.0, "fallback (an earlier measurement on this pool)"
+
+
 def small_config(torch, dbp, ctx, config, hbm_peak, fma_peak):
     """One of configs 1-4 as a short side measurement: layer (or whole-network backward) time, dense-equivalent
     throughput, fraction of the HBM roofline for the algorithmic bytes, fraction of the fp32 FMA peak for the
@@ -361,9 +370,9 @@ def crossover_sweep(torch, dbp, ctx):
             print(json.dumps(row))
 
 
-# DRAM bytes (read + written) of one bench step's launches of each kernel kind, from the ncu capture summarised in
-# profiles/bench_step_config5_dram_bytes.md; None = the kernels of that kind changed after the capture
-NCU_DRAM_BYTES_PER_STEP = {"statistics": None, "quantize": None, "dx_dense": None, "dw_dense": None}
+# DRAM bytes (read + written) of one config-5 bench step's launches of each kernel kind, from the ncu capture summarised
+# in profiles/bench_step_config5_launch_list.md; None = the kernels of that kind changed after the capture
+NCU_DRAM_BYTES_PER_STEP = {"statistics": 1156516096, "quantize": 1333905664, "dx_dense": 1311159808, "dw_dense": 2629937920}
 
 
 def main():
@@ -424,9 +433,16 @@ def main():
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": {"workload": r["workload"], "nsd_density": r["nsd_density"], "l2": "working set smaller than L2 (warm)"},
                 "clocks": clocks, "gpu_launches": r["launches"] * 20, "e2e": None,
-                "roofline": {"kernel": "sparse gather dX/dW (conv_dx2_kernel, conv_dw2_kernel)", "bound": "alu",
-                             "achieved": r["fma_frac"] * fma_peak, "peak": fma_peak, "unit": "TFLOP/s", "frac": r["fma_frac"],
-                             "traffic": None, "peak_source": "measured: dependent fp32 FMA chains on every lane"},
+                "roofline": ({"kernel": "sparse gather dX/dW (conv_dx2_kernel, conv_dw2_kernel)", "bound": "alu",
+                              "achieved": r["fma_frac"] * fma_peak, "peak": fma_peak, "unit": "TFLOP/s", "frac": r["fma_frac"],
+                              "traffic": None, "peak_source": "measured: dependent fp32 FMA chains on every lane"}
+                             if args.config == 2 else
+                             {"kernel": "tensor-core 3x3 dX/dW (tc3_tma_dx_kernel, tc3_tma_dw_kernel), fp32 operands as two bf16 pieces",
+                              "bound": "tensor", "achieved": r["gflops_dense_equiv"] / 1e3, "peak": tensor_peak()[0], "unit": "TFLOP/s",
+                              "frac": r["gflops_dense_equiv"] / 1e3 / tensor_peak()[0], "traffic": None,
+                              "peak_source": tensor_peak()[1],
+                              "note": "dense-equivalent flops of the whole backward pass (every kernel of it, not only the products) / its "
+                                      "time; the split operands cost two MMAs per dense-equivalent one"}),
                 "hbm_path": {"algorithmic_gb_per_step": r["algorithmic_mb"] / 1e3, "frac_of_measured_hbm": r["hbm_frac"], "peak": hbm_peak},
                 "dense_baseline": r["dense_ms"]}))
         if world > 1:
@@ -645,14 +661,21 @@ def main():
                 "note": "non-zero-code FMAs only (2*nnz*K_eff flops per product), summed over the layers that use it"}
     else:
         ach = work[top] / t_s / 1e9
-        traffic = NCU_DRAM_BYTES_PER_STEP.get(top) if not (args.only or args.single or args.batch) else None
+        # per launch, like the algorithmic bytes: a launch of a kind is one layer's use of it (48 per step)
+        per_step = NCU_DRAM_BYTES_PER_STEP.get(top) if (args.config == 5 and not (args.only or args.single or args.batch)) else None
+        n_launch = max(prof[top][1], 1)
+        traffic = None if per_step is None else per_step / n_launch
         roof = {"kernel": {"dx_dense": "tensor-core dX (tma_dx_kernel for 1x1, tc3_tma_dx_kernel for 3x3)",
                            "dw_dense": "tensor-core dW (tma_dw_kernel for 1x1, tc3_tma_dw_kernel + tc3_dw_finish_kernel for 3x3)",
                            "quantize": "NSD quantizer (quantize_dense_kernel for 1x1, quantize_nhwc_kernel for 3x3)"}.get(top, top + "_kernel"),
                 "bound": "hbm", "achieved": ach, "peak": hbm_peak, "unit": "GB/s", "frac": ach / hbm_peak,
-                "traffic": traffic, "peak_source": peak_src + " (MEASURED_PEAKS.json hbm_gbs)",
-                "note": "algorithmic bytes summed over the layers that use it / summed launch time of the kind inside the timed "
-                        "region; traffic: DRAM bytes of the kind's launches in one step (ncu, see profiles/)"}
+                "traffic": traffic, "algorithmic_bytes_per_launch": work[top] / n_launch, "launches_per_step": n_launch,
+                "peak_source": peak_src + " (MEASURED_PEAKS.json hbm_gbs)",
+                "note": "achieved = algorithmic bytes of the kind's launches / their summed duration inside the timed region "
+                        "(CUDA events on the stream they run on; the dW kinds run beside the other kernels, which share the "
+                        "SMs and the bandwidth with them: kernels[kind].frac_of_measured_hbm_alone is the same ratio with nothing "
+                        "else running); traffic: DRAM read+write bytes per launch from the committed ncu launch list "
+                        "(profiles/bench_step_config5_launch_list.md; write-back L2: a kernel's own write counters see little of its output)"}
     for k in work:
         if k in kern:
             kern[k]["work_per_step"] = work[k]
