@@ -162,7 +162,8 @@ typedef enum {
     DBP_K_GLUE = 7,       /* ReLU derivative / max-pool routing */
     DBP_K_DX_DENSE = 8,   /* tensor-core input-gradient product */
     DBP_K_DW_DENSE = 9,   /* tensor-core weight-gradient product (with its split-K reduction) */
-    DBP_K_COUNT = 10
+    DBP_K_FUSED = 10,     /* whole backward pass of a small fp32 linear layer in one launch */
+    DBP_K_COUNT = 11
 } dbp_kernel_kind;
 int dbp_profile_enable(dbp_ctx *ctx, int on);
 int dbp_profile_select(dbp_ctx *ctx, unsigned kind_mask);

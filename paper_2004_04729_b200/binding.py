@@ -25,7 +25,7 @@ EXPORTED_SYMBOLS = [
 ]
 
 KERNEL_KINDS = ["statistics", "quantize", "weight_taps", "dx", "dw", "db", "decode", "glue",
-                "dx_dense", "dw_dense"]
+                "dx_dense", "dw_dense", "fused"]
 
 
 class DbpError(RuntimeError):

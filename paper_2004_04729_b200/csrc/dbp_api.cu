@@ -155,6 +155,25 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     const long long numel = s.B * s.Cout * s.H * s.W;
     const float *delta_p = nullptr;
     const int8_t *codes = nullptr;
+    // small fp32 layers with one position per image (linear layers): everything in one launch
+    if (io == DBP_F32 && s.k == 1 && s.H == 1 && s.W == 1 && !q_out && (dW || dX) && (!db || dW) &&
+        !(flags & (DBP_FORCE_SPARSE | DBP_FORCE_DENSE)) && small_linear_fits(ctx, s.B, s.Cout, s.Cin, dW != nullptr, dX != nullptr)) {
+        if (ctx->aux_pending) {
+            const int jr = dbp_join(ctx);
+            if (jr) return jr;
+        }
+        // a *_host call: X is still on its way up on another stream, and dX is read back after an event
+        if (dW && ctx->hook_before_dw && cudaStreamWaitEvent(ctx->stream, ctx->hook_before_dw, 0) != cudaSuccess) return DBP_ECUDA;
+        int rc;
+        {
+            KernelTimer t(ctx, DBP_K_FUSED);
+            rc = launch_small_linear(ctx, static_cast<const float *>(delta), static_cast<const float *>(X),
+                                     static_cast<const float *>(W), s.B, s.Cout, s.Cin, seed, scale, delta_in, dW,
+                                     static_cast<float *>(dX), db, ctx->delta_sets ? ctx->delta_sets + ctx->code_set : nullptr);
+        }
+        if (!rc && ctx->hook_after_dx && cudaEventRecord(ctx->hook_after_dx, ctx->stream) != cudaSuccess) return DBP_ECUDA;
+        return rc;
+    }
     // While the stream is being captured into a CUDA graph the density read-back is left alone
     // (an event recorded inside a capture cannot be queried): the choice of path is the one the
     // last eager call would have made, and it is frozen into the graph.

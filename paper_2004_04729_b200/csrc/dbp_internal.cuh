@@ -128,6 +128,12 @@ int launch_quantize_nhwc(dbp_ctx *ctx, const void *delta, int dtype, long long B
 int launch_decode(dbp_ctx *ctx, const uint32_t *bitmap, const uint16_t *offsets,
                   const int8_t *values, long long numel, int8_t *dense);
 
+// ---- small_linear.cu: one launch for the whole backward pass of a small fp32 linear layer
+bool small_linear_fits(const dbp_ctx *ctx, long long B, long long N, long long K, bool want_dw, bool want_dx);
+int launch_small_linear(dbp_ctx *ctx, const float *delta, const float *X, const float *W, long long B, long long N,
+                        long long K, unsigned long long seed, float scale, const float *delta_in, float *dW, float *dX,
+                        float *db, float *delta_set);
+
 // ---- product_kernels.cu
 struct ConvShape {
     long long B, Cin, Cout, H, W;
