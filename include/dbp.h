@@ -232,6 +232,9 @@ int nsd_decode_dense(dbp_ctx *ctx, const dbp_sparse *q, int8_t *codes);
  * is of dtype `io` (fp32 with DBP_DX_F32). Any of dW, dX, db may be NULL (skipped).
  * q_out may be NULL; otherwise it receives the sparse structure (arrays sized for B*N).
  * Outputs are overwritten, not accumulated.
+ * fp32 layers with B*N <= 2^17, no q_out and no FORCE flag run as ONE kernel (statistics, dither,
+ * quantization and the products; profiling kind DBP_K_FUSED): same results to the same tolerances,
+ * Delta and nnz through dbp_last_step.
  */
 int dithered_linear_backward(dbp_ctx *ctx, const void *delta, const void *X, const void *W,
                              int io, long long B, long long N, long long K,
