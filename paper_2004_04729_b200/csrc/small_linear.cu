@@ -8,7 +8,12 @@
 //      every CTA adds in the same order, so all of them hold the same Delta without a grid barrier),
 //   2. quantizes the codes its tile needs as it loads them (the dither is a function of the seed and
 //      the element's index, so any CTA can produce any code),
-//   3. accumulates its tile with fp32 FMAs over the reduction index and scales by Delta once.
+//   3. accumulates its tile on the tensor cores and scales by Delta once: the codes are exact in bf16, the
+//      fp32 operand (X or W) is split into two bf16 pieces (the value rounded to bf16 and what that left
+//      over, rounded again: the pair is within 2^-18 of the value), so a k-step is two warp-level MMAs with
+//      fp32 accumulation. Warp-level MMAs (not the CTA-wide ones with accumulators in tensor memory)
+//      because the whole tile is a few hundred of them and nothing here can hide a tensor-memory
+//      allocation, a commit and a read-back.
 // The tiles whose column index is 0 see every element of delta_z exactly once: they count the
 // non-zero and the clipped codes, and the dW ones among them add up the bias gradient. The last CTA
 // to finish publishes Delta and nnz to the context.
@@ -20,7 +25,9 @@ namespace {
 
 constexpr int kThreads = 512;
 constexpr unsigned kFull = 0xffffffffu;
-constexpr int kRows = 64, kCols = 64, kRed = 32;      // output tile and reduction chunk
+constexpr int kRows = 64, kCols = 64, kRed = 64;      // output tile and reduction chunk
+constexpr int kPitch = 72;                            // halfwords per shared-memory row: a 16-byte multiple whose eight
+                                                      // consecutive rows fall into different 16-byte bank groups
 constexpr unsigned long long kGamma = 0x9E3779B97F4A7C15ull;
 
 __device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
@@ -40,6 +47,25 @@ __device__ __forceinline__ float code_of(float x, long long e, unsigned long lon
     const bool num = (t == t);
     sat += (num && tc != t) ? 1u : 0u;
     return num ? floorf(tc) : 0.f;
+}
+
+__device__ __forceinline__ unsigned smem_addr(const void *p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
+// four 8x8 matrices of 16-bit elements from shared memory: lane l gives the address of row l % 8 of matrix l / 8;
+// register m of lane (g, tig) receives elements (g, 2 tig) and (g, 2 tig + 1) of matrix m, or, transposed,
+// elements (2 tig, g) and (2 tig + 1, g)
+__device__ __forceinline__ void ldmatrix_x4(unsigned (&r)[4], unsigned addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(unsigned (&r)[4], unsigned addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// D += A (16 x 16, row-major fragments) * B (16 x 8, column-major fragments), bf16 in, fp32 accumulate
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const unsigned (&a)[4], unsigned b0, unsigned b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
 __device__ __forceinline__ double warp_sum(double v) {
@@ -64,8 +90,10 @@ struct SmallLinP {
 
 __global__ void __launch_bounds__(kThreads)
 small_linear_backward_kernel(const SmallLinP p) {
-    __shared__ float As[kRed][kRows + 1];     // codes, reduction index first
-    __shared__ float Bs[kRed][kCols];         // rows of X (dW) or W (dX)
+    // codes as bf16: dX tiles [row][reduction index], dW tiles [reduction index][row] (delta_z's own order either way)
+    __shared__ __align__(16) unsigned short As[64 * kPitch];
+    // rows of X (dW) or W (dX), [reduction index][column], as two bf16 pieces
+    __shared__ __align__(16) unsigned short Bh[kRed * kPitch], Bl[kRed * kPitch];
     __shared__ double red1[kThreads / 32], red2[kThreads / 32];
     __shared__ float db_s[kRows];
     __shared__ unsigned cnt_s[2];
@@ -143,23 +171,21 @@ small_linear_backward_kernel(const SmallLinP p) {
     if (tid < kRows) db_s[tid] = 0.f;
     if (tid < 2) cnt_s[tid] = 0u;
 
-    // element of delta_z for (reduction index r, output row): dW: delta[r][row] - consecutive threads along the
-    // rows; dX: delta[row][r] - consecutive threads along r. Either way four consecutive addresses per thread.
-    const int a_hi = is_dw ? tid >> 4 : tid >> 3;          // dW: r (0..31); dX: row (0..63)
-    const int a_lo = is_dw ? (tid & 15) * 4 : (tid & 7) * 4;   // dW: rows a_lo..+3; dX: r = a_lo..+3
-    const int b_r = tid >> 4, b_c = (tid & 15) * 4;        // row b_r of the chunk, columns b_c..+3
-    const int ty = tid >> 4, tx = tid & 15;                // outputs: rows 2ty, 2ty+1; columns 4tx..+3
+    // Loads of a chunk: eight consecutive elements of delta_z per thread (dX: row hi, reduction indices lo..lo+7;
+    // dW: reduction index hi, rows lo..lo+7) and eight consecutive columns of row hi of X or W.
+    const int hi = tid >> 3, lo = (tid & 7) * 8;
+    // warp tiling of the 64 x 64 tile: 16 rows x 16 columns per warp (two 16 x 8 accumulators)
+    const int wr = (warp >> 2) * 16, wc = (warp & 3) * 16;
+    const int g = lane >> 2, tig = lane & 3;
     float acc[2][4] = {};
-    float dbacc[4] = {};
+    float dbacc[8] = {};
     unsigned nnz = 0, sat = 0;
 
-    float a_reg[4];
-    float4 b_reg;
-    auto load_chunk = [&](long long r0) {
+    auto load_chunk = [&](long long r0, float (&a_reg)[8], float4 (&b_reg)[2]) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const long long r = r0 + (is_dw ? a_hi : a_lo + i);
-            const long long row = row0 + (is_dw ? a_lo + i : a_hi);
+        for (int i = 0; i < 8; ++i) {
+            const long long r = r0 + (is_dw ? hi : lo + i);
+            const long long row = row0 + (is_dw ? lo + i : hi);
             float q = 0.f;
             if (r < nred && row < nrows) {
                 const long long e = is_dw ? r * p.N + row : row * p.N + r;
@@ -168,69 +194,113 @@ small_linear_backward_kernel(const SmallLinP p) {
             }
             a_reg[i] = q;
         }
-        {
-            const long long r = r0 + b_r;
+        const long long r = r0 + hi;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            const long long c = k0 + lo + 4 * h;
             if (r < nred) {
-                const float *src = Bsrc + r * p.K + k0 + b_c;
+                const float *src = Bsrc + r * p.K + c;
                 if (p.vec4) {
-                    if (k0 + b_c < p.K) v = __ldg(reinterpret_cast<const float4 *>(src));
+                    if (c < p.K) v = __ldg(reinterpret_cast<const float4 *>(src));
                 } else {
-                    if (k0 + b_c + 0 < p.K) v.x = __ldg(src + 0);
-                    if (k0 + b_c + 1 < p.K) v.y = __ldg(src + 1);
-                    if (k0 + b_c + 2 < p.K) v.z = __ldg(src + 2);
-                    if (k0 + b_c + 3 < p.K) v.w = __ldg(src + 3);
+                    if (c + 0 < p.K) v.x = __ldg(src + 0);
+                    if (c + 1 < p.K) v.y = __ldg(src + 1);
+                    if (c + 2 < p.K) v.z = __ldg(src + 2);
+                    if (c + 3 < p.K) v.w = __ldg(src + 3);
                 }
             }
-            b_reg = v;
+            b_reg[h] = v;
+        }
+    };
+    // the addresses this lane hands to the 8x8-matrix loads (lane l: row l % 8 of matrix l / 8)
+    const int lm = lane >> 3, lr = lane & 7;
+    // A, four matrices: (rows 0-7, k 0-7), (rows 8-15, k 0-7), (rows 0-7, k 8-15), (rows 8-15, k 8-15);
+    // dW tiles hold them [k][row] and load them transposed
+    const unsigned a_base = smem_addr(As) + 2u * (is_dw ? static_cast<unsigned>(((lm >> 1) * 8 + lr) * kPitch + wr + (lm & 1) * 8)
+                                                        : static_cast<unsigned>((wr + (lm & 1) * 8 + lr) * kPitch + (lm >> 1) * 8));
+    const unsigned a_kstep = 2u * (is_dw ? 16u * kPitch : 16u);
+    // B, four matrices: (k 0-7, n 0-7), (k 8-15, n 0-7), (k 0-7, n 8-15), (k 8-15, n 8-15), stored [k][n]: transposed loads
+    const unsigned b_off = 2u * static_cast<unsigned>(((lm & 1) * 8 + lr) * kPitch + wc + (lm >> 1) * 8);
+    const unsigned bh_base = smem_addr(Bh) + b_off, bl_base = smem_addr(Bl) + b_off;
+
+    // one chunk: registers -> shared memory, the loads of the chunk after next, then the MMAs
+    auto step = [&](long long r0, float (&a_reg)[8], float4 (&b_reg)[2]) {
+        __syncthreads();                                 // the previous chunk has been used
+        {
+            // eight codes: small integers, exact in bf16 (the float's upper half)
+            unsigned c[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                c[i] = __byte_perm(__float_as_uint(a_reg[2 * i]), __float_as_uint(a_reg[2 * i + 1]), 0x7632);
+            *reinterpret_cast<uint4 *>(As + hi * kPitch + lo) = make_uint4(c[0], c[1], c[2], c[3]);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                nnz += a_reg[i] != 0.f;
+                dbacc[i] += a_reg[i];
+            }
+            const float v[8] = {b_reg[0].x, b_reg[0].y, b_reg[0].z, b_reg[0].w, b_reg[1].x, b_reg[1].y, b_reg[1].z, b_reg[1].w};
+            unsigned h2[4], l2[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const __nv_bfloat162 hh = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+                const float2 hf = __bfloat1622float2(hh);
+                const __nv_bfloat162 ll = __floats2bfloat162_rn(v[2 * i] - hf.x, v[2 * i + 1] - hf.y);
+                h2[i] = *reinterpret_cast<const unsigned *>(&hh);
+                l2[i] = *reinterpret_cast<const unsigned *>(&ll);
+            }
+            *reinterpret_cast<uint4 *>(Bh + hi * kPitch + lo) = make_uint4(h2[0], h2[1], h2[2], h2[3]);
+            *reinterpret_cast<uint4 *>(Bl + hi * kPitch + lo) = make_uint4(l2[0], l2[1], l2[2], l2[3]);
+        }
+        __syncthreads();
+        if (r0 + 2 * kRed < nred) load_chunk(r0 + 2 * kRed, a_reg, b_reg);   // in flight during this chunk's and the next one's MMAs
+#pragma unroll
+        for (int ks = 0; ks < kRed / 16; ++ks) {
+            unsigned a[4], bh[4], bl[4];
+            if (is_dw) ldmatrix_x4_trans(a, a_base + ks * a_kstep);
+            else ldmatrix_x4(a, a_base + ks * a_kstep);
+            ldmatrix_x4_trans(bh, bh_base + ks * 2u * 16u * kPitch);
+            ldmatrix_x4_trans(bl, bl_base + ks * 2u * 16u * kPitch);
+            mma_bf16_16816(acc[0], a, bh[0], bh[1]);
+            mma_bf16_16816(acc[0], a, bl[0], bl[1]);
+            mma_bf16_16816(acc[1], a, bh[2], bh[3]);
+            mma_bf16_16816(acc[1], a, bl[2], bl[3]);
         }
     };
 
-    load_chunk(0);
-    for (long long r0 = 0; r0 < nred; r0 += kRed) {
-        __syncthreads();                                 // the previous chunk has been used
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            if (is_dw) As[a_hi][a_lo + i] = a_reg[i];
-            else As[a_lo + i][a_hi] = a_reg[i];
-            nnz += a_reg[i] != 0.f;
-            dbacc[i] += a_reg[i];
-        }
-        *reinterpret_cast<float4 *>(&Bs[b_r][b_c]) = b_reg;
-        __syncthreads();
-        if (r0 + kRed < nred) load_chunk(r0 + kRed);     // in flight during the FMAs
-#pragma unroll
-        for (int r = 0; r < kRed; ++r) {
-            const float a0 = As[r][2 * ty], a1 = As[r][2 * ty + 1];
-            const float4 b = *reinterpret_cast<const float4 *>(&Bs[r][4 * tx]);
-            acc[0][0] = fmaf(a0, b.x, acc[0][0]); acc[0][1] = fmaf(a0, b.y, acc[0][1]);
-            acc[0][2] = fmaf(a0, b.z, acc[0][2]); acc[0][3] = fmaf(a0, b.w, acc[0][3]);
-            acc[1][0] = fmaf(a1, b.x, acc[1][0]); acc[1][1] = fmaf(a1, b.y, acc[1][1]);
-            acc[1][2] = fmaf(a1, b.z, acc[1][2]); acc[1][3] = fmaf(a1, b.w, acc[1][3]);
-        }
+    float a0[8], a1[8];
+    float4 b0[2], b1[2];
+    load_chunk(0, a0, b0);
+    if (kRed < nred) load_chunk(kRed, a1, b1);
+    for (long long r0 = 0; r0 < nred; r0 += 2 * kRed) {
+        step(r0, a0, b0);
+        if (r0 + kRed < nred) step(r0 + kRed, a1, b1);
     }
 
-    // ---- 3. the tile, scaled by Delta once
+    // ---- 3. the tile, scaled by Delta once: accumulator t holds rows g and g + 8, columns 2 tig, 2 tig + 1 of n-tile t
     float *out = is_dw ? p.dW : p.dX;
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const long long row = row0 + 2 * ty + i;
-        const long long col = k0 + 4 * tx;
-        if (row >= nrows || col >= p.K) continue;
-        float *dst = out + row * p.K + col;
-        if (p.vec4) {
-            *reinterpret_cast<float4 *>(dst) = make_float4(acc[i][0] * dscale, acc[i][1] * dscale, acc[i][2] * dscale, acc[i][3] * dscale);
-        } else {
+    for (int t = 0; t < 2; ++t) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-                if (col + c < p.K) dst[c] = acc[i][c] * dscale;
+        for (int h = 0; h < 2; ++h) {
+            const long long row = row0 + wr + g + 8 * h;
+            const long long col = k0 + wc + 8 * t + 2 * tig;
+            if (row >= nrows || col >= p.K) continue;
+            float *dst = out + row * p.K + col;
+            const float v0 = acc[t][2 * h] * dscale, v1 = acc[t][2 * h + 1] * dscale;
+            if ((p.K & 1) == 0) {
+                *reinterpret_cast<float2 *>(dst) = make_float2(v0, v1);
+            } else {
+                dst[0] = v0;
+                if (col + 1 < p.K) dst[1] = v1;
+            }
         }
     }
 
     // ---- 4. counts, bias gradient, and the step's scalars
-    if (do_db) {                                         // threads that share a_lo hold the same four rows
+    if (do_db) {                                         // threads that share lo hold the same eight rows
 #pragma unroll
-        for (int i = 0; i < 4; ++i) atomicAdd(&db_s[a_lo + i], dbacc[i]);   // small integers: exact in any order
+        for (int i = 0; i < 8; ++i) atomicAdd(&db_s[lo + i], dbacc[i]);     // small integers: exact in any order
     }
     nnz = __reduce_add_sync(kFull, nnz);
     sat = __reduce_add_sync(kFull, sat);
