@@ -377,7 +377,7 @@ def small_config(torch, dbp, ctx, config, hbm_peak, fma_peak):
             "hbm_frac": nbytes / (ms * 1e-3) / 1e9 / hbm_peak, "algorithmic_mb": nbytes / 1e6,
             "nsd_density": density, "fma_frac": density * flops / (ms * 1e-3) / 1e12 / fma_peak,
             "dense_ms": dt, "launches": launches,
-            "note": "fp32 linear layers: statistics, quantization and both products of a layer in one launch (small_linear_backward_kernel)"
+            "note": "fp32 linear layers: step size + codes, then both products on warp-level MMAs: two chained launches per layer (small_linear_*_kernel)"
                     if config in (1, 2) else "fp32 3x3 convolutions: tensor-core kernels, weights and activations split into two bf16 pieces "
                                              "(codes are exact in bf16); fma_frac does not apply" + ("; the FC layer runs on the gather kernels" if config == 4 else "")}
 
@@ -674,7 +674,7 @@ def main():
     work = {k: 0.0 for k in ("statistics", "quantize", "dx", "dw", "dx_dense", "dw_dense", "fused")}
     for (L, d, X, W, dW, dX) in layers:
         nd, nx, nw = d.numel(), X.numel(), W.numel()
-        if prof["fused"][1] > 0:                                       # one launch per layer: dense fp32 FMAs on the codes
+        if prof["fused"][1] > 0:                                       # two chained launches per layer: dense MMAs on the codes
             work["fused"] += L.dense_flops
             continue
         cb = 2 if is_dense(L) else 1                                   # bytes per code the product kernels read
@@ -693,11 +693,11 @@ def main():
         kern[top]["ms_per_step_timed_region"] = t_s * 1e3
     if top == "fused":
         ach = work[top] / t_s / 1e12
-        roof = {"kernel": "one-launch small linear backward (small_linear_backward_kernel)", "bound": "alu", "achieved": ach,
-                "peak": fma_peak, "unit": "TFLOP/s", "frac": ach / fma_peak, "traffic": None,
-                "peak_source": "measured: dependent fp32 FMA chains on every lane (dbp_measure_fma_peak)",
-                "note": "dense fp32 FMAs of both products on the quantized gradient (2 * 2 * B * N * K flops) / kernel time; at "
-                        "these sizes the kernel is bound by launch, the statistics pass and load latency, not by the FMA pipe"}
+        roof = {"kernel": "small linear backward (small_linear_quantize_kernel + small_linear_products_kernel)", "bound": "tensor",
+                "achieved": ach, "peak": tensor_peak()[0], "unit": "TFLOP/s", "frac": ach / tensor_peak()[0], "traffic": None,
+                "peak_source": tensor_peak()[1],
+                "note": "dense-equivalent flops of both products (2 * 2 * B * N * K) / time of the two launches; at these sizes they "
+                        "are bound by launch and load latency, not by the tensor pipe (warp-level MMAs, two bf16 pieces per fp32 operand)"}
     elif top in ("dx", "dw"):
         ach = work[top] / t_s / 1e12
         roof = {"kernel": f"sparse {top} (conv_{top}2_kernel)", "bound": "alu", "achieved": ach,

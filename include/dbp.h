@@ -162,7 +162,7 @@ typedef enum {
     DBP_K_GLUE = 7,       /* ReLU derivative / max-pool routing */
     DBP_K_DX_DENSE = 8,   /* tensor-core input-gradient product */
     DBP_K_DW_DENSE = 9,   /* tensor-core weight-gradient product (with its split-K reduction) */
-    DBP_K_FUSED = 10,     /* whole backward pass of a small fp32 linear layer in one launch */
+    DBP_K_FUSED = 10,     /* whole backward pass of a small fp32 linear layer (two chained launches) */
     DBP_K_COUNT = 11
 } dbp_kernel_kind;
 int dbp_profile_enable(dbp_ctx *ctx, int on);
@@ -232,8 +232,8 @@ int nsd_decode_dense(dbp_ctx *ctx, const dbp_sparse *q, int8_t *codes);
  * is of dtype `io` (fp32 with DBP_DX_F32). Any of dW, dX, db may be NULL (skipped).
  * q_out may be NULL; otherwise it receives the sparse structure (arrays sized for B*N).
  * Outputs are overwritten, not accumulated.
- * fp32 layers with B*N <= 2^17, no q_out and no FORCE flag run as ONE kernel (statistics, dither,
- * quantization and the products; profiling kind DBP_K_FUSED): same results to the same tolerances,
+ * fp32 layers with B*N <= 2^17, no q_out and no FORCE flag run as two chained kernels (statistics, dither
+ * and quantization; then the products; profiling kind DBP_K_FUSED): same results to the same tolerances,
  * Delta and nnz through dbp_last_step.
  */
 int dithered_linear_backward(dbp_ctx *ctx, const void *delta, const void *X, const void *W,

@@ -1,22 +1,23 @@
-// Backward pass of a small fp32 linear layer in one launch (Algorithm 1 with Eqs. (nsd), (qda), (qdw)):
-// step size, dither, quantization and both products.
+// Backward pass of a small fp32 linear layer in two chained launches (Algorithm 1 with Eqs. (nsd), (qda),
+// (qdw)) instead of five: step size + quantization, then both products.
 //
-// For gradients of a few tens of thousands of elements every separate kernel (statistics,
-// quantizer, dX, dW) is a handful of microseconds of work behind a launch and a dependent wait, and
-// the layer is bound by those. Here every CTA owns one 64 x 64 tile of dW or of dX and
-//   1. computes sigma and Delta = s * sigma over the whole tensor by itself (the tensor sits in L2;
-//      every CTA adds in the same order, so all of them hold the same Delta without a grid barrier),
-//   2. quantizes the codes its tile needs as it loads them (the dither is a function of the seed and
-//      the element's index, so any CTA can produce any code),
-//   3. accumulates its tile on the tensor cores and scales by Delta once: the codes are exact in bf16, the
-//      fp32 operand (X or W) is split into two bf16 pieces (the value rounded to bf16 and what that left
-//      over, rounded again: the pair is within 2^-18 of the value), so a k-step is two warp-level MMAs with
-//      fp32 accumulation. Warp-level MMAs (not the CTA-wide ones with accumulators in tensor memory)
-//      because the whole tile is a few hundred of them and nothing here can hide a tensor-memory
-//      allocation, a commit and a read-back.
-// The tiles whose column index is 0 see every element of delta_z exactly once: they count the
-// non-zero and the clipped codes, and the dW ones among them add up the bias gradient. The last CTA
-// to finish publishes Delta and nnz to the context.
+// For gradients of a few tens of thousands of elements every separate kernel (statistics, quantizer,
+// weight re-layout, dX, dW) is a handful of microseconds of work behind a launch and a dependent wait,
+// and the layer is bound by those.
+//   1. small_linear_quantize_kernel: every CTA computes sigma and Delta = s * sigma over the whole
+//      tensor by itself (the tensor sits in L2; every CTA adds in the same order, so all of them hold the
+//      same Delta and no grid-wide step separates statistics from quantization), then quantizes its own
+//      4096 elements into bf16 codes [B][N rounded up to 8] and counts the non-zero and clipped ones.
+//      The last CTA to finish publishes Delta and nnz.
+//   2. small_linear_products_kernel: every CTA owns one 64 x 64 tile of dW or of dX and accumulates it
+//      on the tensor cores: the codes are exact in bf16, the fp32 operand (X or W) is split into two
+//      bf16 pieces (the value rounded to bf16 and what that left over, rounded again: the pair is within
+//      2^-18 of the value), so a k-step is two warp-level MMAs with fp32 accumulation; Delta is applied
+//      once at the end. Warp-level MMAs (not the CTA-wide ones with accumulators in tensor memory)
+//      because a whole tile is a few hundred of them and nothing here can hide a tensor-memory
+//      allocation, a commit and a read-back. The dW tiles of column 0 add up the bias gradient.
+// The second kernel is launched with programmatic stream serialization: it becomes resident while the first
+// runs, loads its first tiles of X and W, and reads the codes as soon as the first one has finished.
 #include "dbp_internal.cuh"
 
 namespace dbp {
@@ -28,25 +29,18 @@ constexpr unsigned kFull = 0xffffffffu;
 constexpr int kRows = 64, kCols = 64, kRed = 64;      // output tile and reduction chunk
 constexpr int kPitch = 72;                            // halfwords per shared-memory row: a 16-byte multiple whose eight
                                                       // consecutive rows fall into different 16-byte bank groups
+constexpr int kQuantPerCta = kThreads * 8;            // elements a CTA of the first kernel quantizes
 constexpr unsigned long long kGamma = 0x9E3779B97F4A7C15ull;
+constexpr float kMagic = 12582912.0f;                 // 1.5 * 2^23: floats in [2^23, 2^24) have unit spacing
 
 __device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
     z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
     z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
     return z ^ (z >> 31);
 }
-
-// code of element e (Eq. (nsd)): q = floor(fma(x, 1 / Delta, u)), u = (2k+1) 2^-24 from the draw the
-// element shares with its neighbour; clipped to [-127, 127] (counted), NaN gives 0
-__device__ __forceinline__ float code_of(float x, long long e, unsigned long long seed, float inv, unsigned &sat) {
-    const unsigned long long r = mix64(seed + (static_cast<unsigned long long>(e >> 1) + 1ull) * kGamma);
-    const unsigned h = (e & 1) ? static_cast<unsigned>(r >> 32) : static_cast<unsigned>(r);
-    const float u = __uint_as_float(__funnelshift_r(h, 0x7fu, 9)) - 0.99999994f;
-    const float t = __fmaf_rn(x, inv, u);
-    const float tc = fminf(fmaxf(t, -127.f), 127.99999f);
-    const bool num = (t == t);
-    sat += (num && tc != t) ? 1u : 0u;
-    return num ? floorf(tc) : 0.f;
+// u = (2k+1) 2^-24, k = top 23 bits of h
+__device__ __forceinline__ float dither(unsigned h) {
+    return __uint_as_float(__funnelshift_r(h, 0x7fu, 9)) - 0.99999994f;
 }
 
 __device__ __forceinline__ unsigned smem_addr(const void *p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
@@ -78,32 +72,30 @@ struct SmallLinP {
     const float *delta, *X, *W;   // [B][N], [B][K], [N][K]
     const float *delta_in;        // used when scale <= 0
     float scale;
-    long long B, N, K;
+    long long B, N, K, Np;        // Np: N rounded up to 8, the row pitch of the codes
     unsigned long long seed;
     float *dW, *dX, *db;          // any may be null (not both products)
     DeviceState *st;
     float *delta_set;             // second place the step size goes to (may be null)
-    unsigned *slots;              // one count per counting CTA
-    int tiles_k, n_dw, n_dx, count_in_dx, n_count;
+    unsigned short *codes;        // bf16 [B][Np]
+    unsigned *slots;              // one non-zero count per CTA of the first kernel
+    int tiles_k, n_dw, n_dx;
     int vec4;                     // K % 4 == 0: 16-byte accesses along K
 };
 
+// ---------------------------------------------------------------- step size and codes
 __global__ void __launch_bounds__(kThreads)
-small_linear_backward_kernel(const SmallLinP p) {
-    // codes as bf16: dX tiles [row][reduction index], dW tiles [reduction index][row] (delta_z's own order either way)
-    __shared__ __align__(16) unsigned short As[64 * kPitch];
-    // rows of X (dW) or W (dX), [reduction index][column], as two bf16 pieces
-    __shared__ __align__(16) unsigned short Bh[kRed * kPitch], Bl[kRed * kPitch];
+small_linear_quantize_kernel(const SmallLinP p) {
     __shared__ double red1[kThreads / 32], red2[kThreads / 32];
-    __shared__ float db_s[kRows];
     __shared__ unsigned cnt_s[2];
     __shared__ bool is_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     chain_wait();
     chain_release();
     const long long n = p.B * p.N;
+    if (tid < 2) cnt_s[tid] = 0u;
 
-    // ---- 1. step size: shifted moments about the first element, fp32 inside a 16-byte load, fp64 across
+    // step size: shifted moments about the first element, fp32 inside a 16-byte load, fp64 across
     float delta;
     bool nonfinite = false;
     if (p.scale > 0.f) {
@@ -111,15 +103,16 @@ small_linear_backward_kernel(const SmallLinP p) {
         double d1 = 0.0, d2 = 0.0;
         const long long nvec = n / 4;
         const float4 *v4 = reinterpret_cast<const float4 *>(p.delta);
-        for (long long i0 = 0; i0 < nvec; i0 += kThreads * 8) {
-            float4 v[8];
+        constexpr int kU = 20;                          // loads in flight per thread: one round trip for 10 K vectors
+        for (long long i0 = 0; i0 < nvec; i0 += kThreads * kU) {
+            float4 v[kU];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+            for (int u = 0; u < kU; ++u) {
                 const long long i = i0 + u * kThreads + tid;
                 v[u] = i < nvec ? __ldg(v4 + i) : make_float4(pivot, pivot, pivot, pivot);
             }
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+            for (int u = 0; u < kU; ++u) {
                 const float c0 = v[u].x - pivot, c1 = v[u].y - pivot, c2 = v[u].z - pivot, c3 = v[u].w - pivot;
                 const float s1 = (c0 + c1) + (c2 + c3);
                 const float s2 = fmaf(c0, c0, fmaf(c1, c1, fmaf(c2, c2, c3 * c3)));
@@ -154,9 +147,88 @@ small_linear_backward_kernel(const SmallLinP p) {
     }
     const bool live = (delta > 0.f) && (delta < __int_as_float(0x7f800000));
     const float inv = live ? __fdiv_rn(1.0f, delta) : 0.f;
-    const float dscale = live ? delta : 0.f;             // what the outputs are scaled by
 
-    // ---- 2. this CTA's tile
+    // codes of this thread's eight consecutive elements (the first index is even: a pair shares a draw)
+    const long long e0 = static_cast<long long>(blockIdx.x) * kQuantPerCta + static_cast<long long>(tid) * 8;
+    unsigned nnz = 0, sat = 0;
+    if (e0 < n) {
+        float f[8];
+        unsigned long long z = p.seed + (static_cast<unsigned long long>(e0 >> 1) + 1ull) * kGamma;
+#pragma unroll
+        for (int j = 0; j < 8; j += 2) {
+            const unsigned long long r = mix64(z);
+            z += kGamma;
+            const float u[2] = {dither(static_cast<unsigned>(r)), dither(static_cast<unsigned>(r >> 32))};
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                float q = 0.f;
+                if (live && e0 + j + h < n) {
+                    const float t = __fmaf_rn(__ldg(p.delta + e0 + j + h), inv, u[h]);
+                    const float tc = fminf(fmaxf(t, -127.f), 127.99999f);      // clipped codes are counted, NaN gives 0
+                    const bool num = (t == t);
+                    sat += (num && tc != t) ? 1u : 0u;
+                    q = num ? __fadd_rd(tc, kMagic) - kMagic : 0.f;
+                }
+                f[j + h] = q;
+                nnz += q != 0.f;
+            }
+        }
+        // to [b][Np]: one division for the first element, then step and wrap; small integers are exact in
+        // bf16 (the float's upper half)
+        long long b = e0 / p.N;
+        long long j = e0 - b * p.N;
+        unsigned short *dst = p.codes + b * p.Np + j;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (e0 + i < n) *dst = static_cast<unsigned short>(__float_as_uint(f[i]) >> 16);
+            ++dst;
+            if (++j == p.N) { j = 0; dst += p.Np - p.N; }
+        }
+    }
+    nnz = __reduce_add_sync(kFull, nnz);
+    sat = __reduce_add_sync(kFull, sat);
+    __syncthreads();                                     // cnt_s is initialised (and red1 / red2 have been read)
+    if (lane == 0) {
+        if (nnz) atomicAdd(&cnt_s[0], nnz);
+        if (sat) atomicAdd(&cnt_s[1], sat);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        p.slots[blockIdx.x] = cnt_s[0];
+        if (cnt_s[1]) atomicAdd(&p.st->saturated, static_cast<unsigned long long>(cnt_s[1]));
+        __threadfence();
+        const unsigned ticket = atomicAdd(&p.st->ticket, 1u);
+        is_last = (ticket == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    unsigned long long total = 0;
+    for (int i = tid; i < static_cast<int>(gridDim.x); i += kThreads) total += __ldcg(p.slots + i);
+    const double tsum = warp_sum(static_cast<double>(total));   // counts below 2^53: exact
+    if (lane == 0) red1[warp] = tsum;
+    __syncthreads();
+    if (tid == 0) {
+        double all = 0.0;
+        for (int w = 0; w < kThreads / 32; ++w) all += red1[w];
+        p.st->nnz = static_cast<unsigned long long>(all);
+        p.st->delta = delta;
+        if (nonfinite) p.st->nonfinite = 1;
+        if (p.delta_set) *p.delta_set = delta;
+        p.st->ticket = 0u;
+    }
+}
+
+// ---------------------------------------------------------------- both products
+__global__ void __launch_bounds__(kThreads)
+small_linear_products_kernel(const SmallLinP p) {
+    // codes: dX tiles [row][reduction index], dW tiles [reduction index][row] (the order they are stored in either way)
+    __shared__ __align__(16) unsigned short As[64 * kPitch];
+    // rows of X (dW) or W (dX), [reduction index][column], as two bf16 pieces
+    __shared__ __align__(16) unsigned short Bh[kRed * kPitch], Bl[kRed * kPitch];
+    __shared__ float db_s[kRows];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
     const int t = blockIdx.x;
     const bool is_dw = t < p.n_dw;
     const int tt = is_dw ? t : t - p.n_dw;
@@ -166,34 +238,19 @@ small_linear_backward_kernel(const SmallLinP p) {
     const long long nrows = is_dw ? p.N : p.B;                       // output rows in all
     const long long nred = is_dw ? p.B : p.N;                        // reduction length
     const float *Bsrc = is_dw ? p.X : p.W;                           // [nred][K]
-    const bool counting = kt == 0 && (is_dw != (p.count_in_dx != 0));
     const bool do_db = is_dw && kt == 0 && p.db != nullptr;
     if (tid < kRows) db_s[tid] = 0.f;
-    if (tid < 2) cnt_s[tid] = 0u;
 
-    // Loads of a chunk: eight consecutive elements of delta_z per thread (dX: row hi, reduction indices lo..lo+7;
-    // dW: reduction index hi, rows lo..lo+7) and eight consecutive columns of row hi of X or W.
+    // Loads of a chunk: eight consecutive codes per thread, one 16-byte load (dX: row hi, reduction indices
+    // lo..lo+7; dW: reduction index hi, rows lo..lo+7), and eight consecutive columns of row hi of X or W.
     const int hi = tid >> 3, lo = (tid & 7) * 8;
     // warp tiling of the 64 x 64 tile: 16 rows x 16 columns per warp (two 16 x 8 accumulators)
     const int wr = (warp >> 2) * 16, wc = (warp & 3) * 16;
     const int g = lane >> 2, tig = lane & 3;
     float acc[2][4] = {};
     float dbacc[8] = {};
-    unsigned nnz = 0, sat = 0;
 
-    auto load_chunk = [&](long long r0, float (&a_reg)[8], float4 (&b_reg)[2]) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const long long r = r0 + (is_dw ? hi : lo + i);
-            const long long row = row0 + (is_dw ? lo + i : hi);
-            float q = 0.f;
-            if (r < nred && row < nrows) {
-                const long long e = is_dw ? r * p.N + row : row * p.N + r;
-                const float x = __ldg(p.delta + e);
-                if (live) q = code_of(x, e, p.seed, inv, sat);
-            }
-            a_reg[i] = q;
-        }
+    auto load_b = [&](long long r0, float4 (&b_reg)[2]) {
         const long long r = r0 + hi;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
@@ -213,6 +270,26 @@ small_linear_backward_kernel(const SmallLinP p) {
             b_reg[h] = v;
         }
     };
+    // codes outside the tensor (and the padding of a row) read as zero
+    auto load_a = [&](long long r0, uint4 &a_reg) {
+        const long long bb = is_dw ? r0 + hi : row0 + hi;            // image (row of delta_z)
+        const long long jj = is_dw ? row0 + lo : r0 + lo;            // first of eight output channels
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (bb < p.B && jj < p.N) {
+            v = __ldcg(reinterpret_cast<const uint4 *>(p.codes + bb * p.Np + jj));
+            const long long left = p.N - jj;                         // valid codes from jj on
+            if (left < 8) {
+                unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (2 * i >= left) w[i] = 0u;
+                    else if (2 * i + 1 >= left) w[i] &= 0xffffu;
+                }
+                v = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        }
+        a_reg = v;
+    };
     // the addresses this lane hands to the 8x8-matrix loads (lane l: row l % 8 of matrix l / 8)
     const int lm = lane >> 3, lr = lane & 7;
     // A, four matrices: (rows 0-7, k 0-7), (rows 8-15, k 0-7), (rows 0-7, k 8-15), (rows 8-15, k 8-15);
@@ -225,19 +302,17 @@ small_linear_backward_kernel(const SmallLinP p) {
     const unsigned bh_base = smem_addr(Bh) + b_off, bl_base = smem_addr(Bl) + b_off;
 
     // one chunk: registers -> shared memory, the loads of the chunk after next, then the MMAs
-    auto step = [&](long long r0, float (&a_reg)[8], float4 (&b_reg)[2]) {
+    auto step = [&](long long r0, uint4 &a_reg, float4 (&b_reg)[2]) {
         __syncthreads();                                 // the previous chunk has been used
         {
-            // eight codes: small integers, exact in bf16 (the float's upper half)
-            unsigned c[4];
+            *reinterpret_cast<uint4 *>(As + hi * kPitch + lo) = a_reg;
+            if (do_db) {
+                const unsigned w[4] = {a_reg.x, a_reg.y, a_reg.z, a_reg.w};
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                c[i] = __byte_perm(__float_as_uint(a_reg[2 * i]), __float_as_uint(a_reg[2 * i + 1]), 0x7632);
-            *reinterpret_cast<uint4 *>(As + hi * kPitch + lo) = make_uint4(c[0], c[1], c[2], c[3]);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                nnz += a_reg[i] != 0.f;
-                dbacc[i] += a_reg[i];
+                for (int i = 0; i < 4; ++i) {
+                    dbacc[2 * i] += __uint_as_float(w[i] << 16);
+                    dbacc[2 * i + 1] += __uint_as_float(w[i] & 0xffff0000u);
+                }
             }
             const float v[8] = {b_reg[0].x, b_reg[0].y, b_reg[0].z, b_reg[0].w, b_reg[1].x, b_reg[1].y, b_reg[1].z, b_reg[1].w};
             unsigned h2[4], l2[4];
@@ -253,7 +328,10 @@ small_linear_backward_kernel(const SmallLinP p) {
             *reinterpret_cast<uint4 *>(Bl + hi * kPitch + lo) = make_uint4(l2[0], l2[1], l2[2], l2[3]);
         }
         __syncthreads();
-        if (r0 + 2 * kRed < nred) load_chunk(r0 + 2 * kRed, a_reg, b_reg);   // in flight during this chunk's and the next one's MMAs
+        if (r0 + 2 * kRed < nred) {                      // in flight during this chunk's and the next one's MMAs
+            load_a(r0 + 2 * kRed, a_reg);
+            load_b(r0 + 2 * kRed, b_reg);
+        }
 #pragma unroll
         for (int ks = 0; ks < kRed / 16; ++ks) {
             unsigned a[4], bh[4], bl[4];
@@ -268,26 +346,33 @@ small_linear_backward_kernel(const SmallLinP p) {
         }
     };
 
-    float a0[8], a1[8];
+    uint4 a0, a1 = make_uint4(0u, 0u, 0u, 0u);
     float4 b0[2], b1[2];
-    load_chunk(0, a0, b0);
-    if (kRed < nred) load_chunk(kRed, a1, b1);
+    // X and W are inputs of the call: their first chunks are on their way before the first kernel is done
+    load_b(0, b0);
+    if (kRed < nred) load_b(kRed, b1);
+    chain_wait();
+    chain_release();
+    const float delta = __ldcg(&p.st->delta);
+    const float dscale = (delta > 0.f && delta < __int_as_float(0x7f800000)) ? delta : 0.f;
+    load_a(0, a0);
+    if (kRed < nred) load_a(kRed, a1);
     for (long long r0 = 0; r0 < nred; r0 += 2 * kRed) {
         step(r0, a0, b0);
         if (r0 + kRed < nred) step(r0 + kRed, a1, b1);
     }
 
-    // ---- 3. the tile, scaled by Delta once: accumulator t holds rows g and g + 8, columns 2 tig, 2 tig + 1 of n-tile t
+    // the tile, scaled by Delta once: accumulator t holds rows g and g + 8, columns 2 tig, 2 tig + 1 of n-tile t
     float *out = is_dw ? p.dW : p.dX;
 #pragma unroll
-    for (int t = 0; t < 2; ++t) {
+    for (int tn = 0; tn < 2; ++tn) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const long long row = row0 + wr + g + 8 * h;
-            const long long col = k0 + wc + 8 * t + 2 * tig;
+            const long long col = k0 + wc + 8 * tn + 2 * tig;
             if (row >= nrows || col >= p.K) continue;
             float *dst = out + row * p.K + col;
-            const float v0 = acc[t][2 * h] * dscale, v1 = acc[t][2 * h + 1] * dscale;
+            const float v0 = acc[tn][2 * h] * dscale, v1 = acc[tn][2 * h + 1] * dscale;
             if ((p.K & 1) == 0) {
                 *reinterpret_cast<float2 *>(dst) = make_float2(v0, v1);
             } else {
@@ -296,54 +381,18 @@ small_linear_backward_kernel(const SmallLinP p) {
             }
         }
     }
-
-    // ---- 4. counts, bias gradient, and the step's scalars
     if (do_db) {                                         // threads that share lo hold the same eight rows
 #pragma unroll
         for (int i = 0; i < 8; ++i) atomicAdd(&db_s[lo + i], dbacc[i]);     // small integers: exact in any order
-    }
-    nnz = __reduce_add_sync(kFull, nnz);
-    sat = __reduce_add_sync(kFull, sat);
-    if (lane == 0 && counting) {
-        atomicAdd(&cnt_s[0], nnz);
-        atomicAdd(&cnt_s[1], sat);
-    }
-    __syncthreads();
-    if (do_db && tid < kRows && row0 + tid < p.N) p.db[row0 + tid] = db_s[tid] * dscale;
-    if (tid == 0) {
-        if (counting) {
-            p.slots[rt] = cnt_s[0];
-            if (cnt_s[1]) atomicAdd(&p.st->saturated, static_cast<unsigned long long>(cnt_s[1]));
-        }
-        __threadfence();
-        const unsigned ticket = atomicAdd(&p.st->ticket, 1u);
-        is_last = (ticket == gridDim.x - 1);
-    }
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
-    unsigned long long total = 0;
-    for (int i = tid; i < p.n_count; i += kThreads) total += __ldcg(p.slots + i);
-    double tsum = warp_sum(static_cast<double>(total));   // counts below 2^53: exact
-    __syncthreads();
-    if (lane == 0) red1[warp] = tsum;
-    __syncthreads();
-    if (tid == 0) {
-        double all = 0.0;
-        for (int w = 0; w < kThreads / 32; ++w) all += red1[w];
-        p.st->nnz = static_cast<unsigned long long>(all);
-        p.st->delta = delta;
-        if (nonfinite) p.st->nonfinite = 1;
-        if (p.delta_set) *p.delta_set = delta;
-        p.st->ticket = 0u;
+        __syncthreads();
+        if (tid < kRows && row0 + tid < p.N) p.db[row0 + tid] = db_s[tid] * dscale;
     }
 }
 
 }  // namespace
 
-// Shapes the one-launch kernel takes: small enough that every CTA can read the whole gradient for its
-// statistics (the product of gradient size and CTA count bounds the L2 traffic of that), and few enough
-// counting CTAs for the context's scratch.
+// Shapes the two-launch path takes: small enough that every CTA of the first kernel can read the whole
+// gradient for its statistics (gradient size times CTA count is the L2 traffic of that: at most 32 x 2^17 elements).
 bool small_linear_fits(const dbp_ctx *ctx, long long B, long long N, long long K, bool want_dw, bool want_dx) {
     const long long n = B * N;
     if (n <= 0 || n > (1ll << 17) || K <= 0 || K > (1ll << 24)) return false;
@@ -351,9 +400,9 @@ bool small_linear_fits(const dbp_ctx *ctx, long long B, long long N, long long K
     const long long n_dw = want_dw ? ((N + kRows - 1) / kRows) * tiles_k : 0;
     const long long n_dx = want_dx ? ((B + kRows - 1) / kRows) * tiles_k : 0;
     const long long ctas = n_dw + n_dx;
-    if (ctas <= 0 || ctas > 65535 || n * ctas > (1ll << 25)) return false;
-    const long long n_count = want_dx ? (B + kRows - 1) / kRows : (N + kRows - 1) / kRows;
-    return n_count * static_cast<long long>(sizeof(unsigned)) <= static_cast<long long>(sizeof(double)) * 2 * ctx->partial_blocks;
+    if (ctas <= 0 || ctas > 65535) return false;
+    const long long qctas = (n + kQuantPerCta - 1) / kQuantPerCta;
+    return qctas * static_cast<long long>(sizeof(unsigned)) <= static_cast<long long>(sizeof(double)) * 2 * ctx->partial_blocks;
 }
 
 int launch_small_linear(dbp_ctx *ctx, const float *delta, const float *X, const float *W, long long B, long long N,
@@ -361,17 +410,21 @@ int launch_small_linear(dbp_ctx *ctx, const float *delta, const float *X, const 
                         float *db, float *delta_set) {
     SmallLinP p{};
     p.delta = delta; p.X = X; p.W = W; p.delta_in = delta_in; p.scale = scale;
-    p.B = B; p.N = N; p.K = K; p.seed = seed;
+    p.B = B; p.N = N; p.K = K; p.Np = (N + 7) / 8 * 8; p.seed = seed;
     p.dW = dW; p.dX = dX; p.db = dW ? db : nullptr;
     p.st = ctx->state; p.delta_set = delta_set;
+    const int k = ctx->code_set;
+    if (int rc = ws_reserve(ctx, ctx->codes16[k], static_cast<size_t>(B) * p.Np * 2 + 64)) return rc;
+    p.codes = static_cast<unsigned short *>(ctx->codes16[k].ptr);
     p.slots = reinterpret_cast<unsigned *>(ctx->partials);
     p.tiles_k = static_cast<int>((K + kCols - 1) / kCols);
     p.n_dw = dW ? static_cast<int>((N + kRows - 1) / kRows) * p.tiles_k : 0;
     p.n_dx = dX ? static_cast<int>((B + kRows - 1) / kRows) * p.tiles_k : 0;
-    p.count_in_dx = dX ? 1 : 0;
-    p.n_count = static_cast<int>(dX ? (B + kRows - 1) / kRows : (N + kRows - 1) / kRows);
     p.vec4 = (K % 4 == 0) ? 1 : 0;
-    return cuda_ok(launch_chained(small_linear_backward_kernel, dim3(static_cast<unsigned>(p.n_dw + p.n_dx)), dim3(kThreads), 0,
+    const long long n = B * N;
+    const unsigned qctas = static_cast<unsigned>((n + kQuantPerCta - 1) / kQuantPerCta);
+    if (int rc = cuda_ok(launch_chained(small_linear_quantize_kernel, dim3(qctas), dim3(kThreads), 0, ctx->stream, p))) return rc;
+    return cuda_ok(launch_chained(small_linear_products_kernel, dim3(static_cast<unsigned>(p.n_dw + p.n_dx)), dim3(kThreads), 0,
                                   ctx->stream, p));
 }
 

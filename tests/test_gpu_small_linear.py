@@ -1,4 +1,4 @@
-"""The one-launch backward pass of small fp32 linear layers (no caller's sparse structure) against the CPU
+"""The two-launch backward pass of small fp32 linear layers (no caller's sparse structure) against the CPU
 oracle: step size to 1e-6, the number of non-zero codes exactly (the oracle quantizes with the CUDA path's
 step size), dW, dX, db to 1e-5 (relative Frobenius and |err| <= 1e-5 sum|terms|). The codes themselves never
 leave the kernel; a wrong code shows in nnz and in the products."""
