@@ -364,24 +364,58 @@ tc3_dw_finish_kernel(float *__restrict__ acc, const float *__restrict__ delta_p,
 // fp32 activations [B][Cin][HW] -> two bf16 tensors [B][cin_pad][pitch], one after the other: the values rounded
 // to bf16 and what that rounding left over, rounded again (the two pieces add up to the fp32 value to within
 // 2^-18 of it). Rows are padded to `pitch` (a multiple of 8) and channels to cin_pad (a multiple of 8) with zeros.
+// A thread takes eight consecutive positions of one plane: two 16-byte loads where the plane allows it, one 16-byte
+// store per piece.
 __global__ void __launch_bounds__(256)
 x_split_kernel(const float *__restrict__ X, __nv_bfloat16 *__restrict__ out, long long B, int Cin, int cin_pad, int HW, int pitch) {
     chain_wait();
     chain_release();
-    const long long n = B * cin_pad * pitch;
-    for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += gridDim.x * 256ll) {
-        const long long pl = i / pitch;
-        const int pp = static_cast<int>(i - pl * pitch);
+    const int gpp = pitch / 8;                                   // groups of eight positions per plane
+    const long long planes = B * cin_pad, ngroups = planes * gpp;
+    const long long n = planes * pitch;
+    const bool vec = (HW % 4 == 0);
+    for (long long gi = blockIdx.x * 256ll + threadIdx.x; gi < ngroups; gi += gridDim.x * 256ll) {
+        long long pl;
+        int gq;
+        if ((ngroups >> 31) == 0) {                              // 32-bit divisions cost a fraction of 64-bit ones
+            const unsigned u = static_cast<unsigned>(gi);
+            pl = u / static_cast<unsigned>(gpp);
+            gq = static_cast<int>(u - static_cast<unsigned>(pl) * static_cast<unsigned>(gpp));
+        } else {
+            pl = gi / gpp;
+            gq = static_cast<int>(gi - pl * gpp);
+        }
         const long long b = pl / cin_pad;
         const int ci = static_cast<int>(pl - b * cin_pad);
-        __nv_bfloat16 hi = __float2bfloat16_rn(0.f), lo = hi;
-        if (pp < HW && ci < Cin) {
-            const float x = __ldg(X + (b * Cin + ci) * HW + pp);
-            hi = __float2bfloat16_rn(x);
-            lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+        const int pp0 = gq * 8;
+        float x[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        if (ci < Cin && pp0 < HW) {
+            const float *src = X + (b * Cin + ci) * HW + pp0;
+            if (vec) {
+                const float4 v0 = __ldg(reinterpret_cast<const float4 *>(src));
+                x[0] = v0.x; x[1] = v0.y; x[2] = v0.z; x[3] = v0.w;
+                if (pp0 + 4 < HW) {
+                    const float4 v1 = __ldg(reinterpret_cast<const float4 *>(src + 4));
+                    x[4] = v1.x; x[5] = v1.y; x[6] = v1.z; x[7] = v1.w;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (pp0 + i < HW) x[i] = __ldg(src + i);
+            }
         }
-        out[i] = hi;
-        out[n + i] = lo;
+        unsigned h[4], l[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __nv_bfloat162 hh = __floats2bfloat162_rn(x[2 * i], x[2 * i + 1]);
+            const float2 hf = __bfloat1622float2(hh);
+            const __nv_bfloat162 ll = __floats2bfloat162_rn(x[2 * i] - hf.x, x[2 * i + 1] - hf.y);
+            h[i] = *reinterpret_cast<const unsigned *>(&hh);
+            l[i] = *reinterpret_cast<const unsigned *>(&ll);
+        }
+        const long long o = pl * pitch + pp0;
+        *reinterpret_cast<uint4 *>(out + o) = make_uint4(h[0], h[1], h[2], h[3]);
+        *reinterpret_cast<uint4 *>(out + n + o) = make_uint4(l[0], l[1], l[2], l[3]);
     }
 }
 
@@ -448,7 +482,7 @@ int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, int i
         xpitch = (HW + 7) / 8 * 8;
         const long long planes = s.B * cin_pad;
         if ((rc = ws_reserve(ctx, ctx->x_padded, static_cast<size_t>(planes) * xpitch * 2 * 2))) return rc;
-        long long blocks = (planes * xpitch + 255) / 256;
+        long long blocks = (planes * (xpitch / 8) + 255) / 256;
         if (blocks > ctx->sm_count * 16) blocks = ctx->sm_count * 16;
         if ((rc = cuda_ok(launch_chained(x_split_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, ctx->stream,
                                          static_cast<const float *>(X), static_cast<__nv_bfloat16 *>(ctx->x_padded.ptr), s.B,
