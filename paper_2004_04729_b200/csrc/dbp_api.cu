@@ -63,7 +63,8 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
                           dbp_sparse *q_out, const float **delta_p, const int8_t **codes,
                           bool want8 = true, long long planes_hw = 0, long long planes_pitch = 0,
                           const void **codes16 = nullptr, const ConvShape *nhwc = nullptr,
-                          const void **codes_nhwc = nullptr, const SideJobs &jobs = SideJobs()) {
+                          const void **codes_nhwc = nullptr, const SideJobs &jobs = SideJobs(),
+                          int stack_g = 0, const void **codes_stack = nullptr) {
     int rc = DBP_OK;
     dbp_sparse sp;
     sp.bitmap = nullptr; sp.offsets = nullptr; sp.values = nullptr; sp.delta = nullptr; sp.nnz = nullptr;
@@ -107,6 +108,14 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
             pn = ctx->codes_nhwc[k].ptr;
             *codes_nhwc = pn;
         }
+        void *ps = nullptr;
+        if (nhwc && stack_g > 0 && codes_stack) {
+            // tall images of stack_g images each: (H + 1) W rows per image
+            const size_t rows = static_cast<size_t>(nhwc->B) * (nhwc->H + 1) * nhwc->W;
+            if ((rc = ws_reserve(ctx, ctx->codes_stack[k], rows * nhwc->Cout * 2 + 1024))) return rc;
+            ps = ctx->codes_stack[k].ptr;
+            *codes_stack = ps;
+        }
         if (q_out) {
             rc = launch_quantize(ctx, delta, dtype, numel, seed, &ctx->state->delta, sp.bitmap, sp.offsets,
                                  sp.values, dense, reinterpret_cast<unsigned long long *>(sp.nnz));
@@ -115,10 +124,10 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
                                            planes_hw, planes_pitch, false);
             if (!rc && pn)
                 rc = launch_quantize_nhwc(ctx, delta, dtype, nhwc->B, nhwc->Cout, nhwc->H * nhwc->W, seed,
-                                          &ctx->state->delta, pn, nullptr, false);
+                                          &ctx->state->delta, pn, nullptr, false, ps, static_cast<int>(nhwc->W), stack_g);
         } else if (pn) {
             rc = launch_quantize_nhwc(ctx, delta, dtype, nhwc->B, nhwc->Cout, nhwc->H * nhwc->W, seed,
-                                      &ctx->state->delta, pn, want8 ? dense : nullptr, true);
+                                      &ctx->state->delta, pn, want8 ? dense : nullptr, true, ps, static_cast<int>(nhwc->W), stack_g);
         } else {
             rc = launch_quantize_dense(ctx, delta, dtype, numel, seed, &ctx->state->delta, want8 ? dense : nullptr,
                                        p16, planes_hw, planes_pitch, true);
@@ -225,9 +234,12 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
         if (wr) return wr;
         jobs.w_src = W; jobs.w_dst = ctx->w_taps.ptr; jobs.w_f32 = io == DBP_F32; jobs.Cout = s.Cout; jobs.Cin = s.Cin;
     }
+    // tiny planes: the weight-gradient kernel reads the images stacked into tall ones
+    const int stack_g = (t3 && dW) ? tc3_stack_images(s, io) : 0;
+    const void *codes_st = nullptr;
     int rc = quantize_for_products(ctx, delta, io, numel, seed, scale, delta_in, q_out, &delta_p, &codes, need8,
                                    s.H * s.W, any_tma ? tma_code_pitch(s) : 0, any_tma ? &codes16 : nullptr,
-                                   t3 ? &s : nullptr, t3 ? &codes_n : nullptr, jobs);
+                                   t3 ? &s : nullptr, t3 ? &codes_n : nullptr, jobs, stack_g, &codes_st);
     if (rc) return rc;
     if (!capturing && !ctx->nnz_pending && ctx->nnz_host && ctx->nnz_event) {
         ctx->nnz_host_numel = numel;
@@ -259,6 +271,10 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
         if (dW && !rc) {
             KernelTimer t(ctx, DBP_K_DW_DENSE);
             rc = dw_tma ? launch_tma_dw(ctx, codes16, X, delta_p, s, dW, &ctx->state->tc_timeout)
+                 : (t3 && stack_g > 0)
+                     ? launch_tc3_tma_dw(ctx, codes_st, X, io, delta_p,
+                                         ConvShape{s.B / stack_g, s.Cin, s.Cout, static_cast<long long>(stack_g) * (s.H + 1), s.W, 3}, dW,
+                                         &ctx->state->tc_timeout, stack_g, static_cast<int>(s.H))
                  : t3   ? launch_tc3_tma_dw(ctx, codes_n, X, io, delta_p, s, dW, &ctx->state->tc_timeout)
                         : launch_tc_dw(ctx, codes, X, delta_p, s, dW, &ctx->state->tc_timeout);
         }
@@ -404,7 +420,7 @@ int dbp_destroy(dbp_ctx *ctx) {
     cudaStreamSynchronize(ctx->stream);
     if (ctx->aux) cudaStreamSynchronize(ctx->aux);
     Workspace *all[] = {&ctx->dense_codes[0], &ctx->dense_codes[1], &ctx->codes16[0], &ctx->codes16[1],
-                        &ctx->codes_nhwc[0], &ctx->codes_nhwc[1], &ctx->dw_acc, &ctx->x_padded, &ctx->w_taps, &ctx->sp_bitmap, &ctx->sp_offsets, &ctx->sp_values,
+                        &ctx->codes_nhwc[0], &ctx->codes_nhwc[1], &ctx->codes_stack[0], &ctx->codes_stack[1], &ctx->dw_acc, &ctx->x_padded, &ctx->w_taps, &ctx->sp_bitmap, &ctx->sp_offsets, &ctx->sp_values,
                         &ctx->tc_partials};
     for (Workspace *w : all) if (w->ptr) cudaFree(w->ptr);
     for (Workspace &w : ctx->io) if (w.ptr) cudaFree(w.ptr);

@@ -53,6 +53,7 @@ struct dbp_ctx {
     dbp::Workspace sp_bitmap, sp_offsets, sp_values;  // internal dbp_sparse
     dbp::Workspace tc_partials;         // split-K partial blocks of the dense dW kernel
     dbp::Workspace codes_nhwc[2];       // bf16 codes [B][position][Cout] for the TMA-fed 3x3 kernels
+    dbp::Workspace codes_stack[2];      // the same codes with G images stacked into one tall image (tiny planes, dW)
     float *delta_sets = nullptr;        // device float[2]: the step size that belongs to each set
     int code_set = 0;                   // the set the next call writes
     cudaEvent_t ev_set_free[2] = {nullptr, nullptr};   // recorded on the dW stream after the set's last reader
@@ -124,7 +125,8 @@ int launch_quantize_dense(dbp_ctx *ctx, const void *delta, int dtype, long long 
 // position-major bf16 codes [B][HW][C] for the TMA-fed 3x3 kernels (and int8 codes in delta's order
 // when dense8 is not null)
 int launch_quantize_nhwc(dbp_ctx *ctx, const void *delta, int dtype, long long B, long long C, long long HW,
-                         unsigned long long seed, const float *delta_p, void *codes_nhwc, int8_t *dense8, bool count);
+                         unsigned long long seed, const float *delta_p, void *codes_nhwc, int8_t *dense8, bool count,
+                         void *codes_stack = nullptr, int plane_w = 0, int stack_g = 0);
 int launch_decode(dbp_ctx *ctx, const uint32_t *bitmap, const uint16_t *offsets,
                   const int8_t *values, long long numel, int8_t *dense);
 
@@ -177,7 +179,10 @@ bool tc3_tma_dw_supported(const ConvShape &s, int io);     // dW alone: also fp3
 int launch_tc3_tma_dx(dbp_ctx *ctx, const void *codes_nhwc, const void *W, int io, const float *delta_p,
                       const ConvShape &s, void *dX, bool dx_bf16, int *err_flag, bool weights_ready = false);
 int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, int io, const float *delta_p,
-                      const ConvShape &s, float *dW, int *err_flag);
+                      const ConvShape &s, float *dW, int *err_flag, int stack_g = 0, int real_h = 0);
+// Planes of fewer than 64 positions: how many images of a batch to stack into one tall image (one zero row after
+// every image) for the weight-gradient kernel, whose work comes in segments of one image; 0: do not stack.
+int tc3_stack_images(const ConvShape &s, int io);
 int launch_bias_grad(dbp_ctx *ctx, const int8_t *codes, const float *delta_p, const ConvShape &s,
                      float *db);
 int launch_relu_backward(dbp_ctx *ctx, const float *da, const uint8_t *mask, float *dz,

@@ -335,7 +335,8 @@ template <typename T, int V>
 __global__ void __launch_bounds__(kThreads)
 quantize_nhwc_kernel(const T *__restrict__ x, int B, int C, int HW, unsigned long long seed,
                      const float *__restrict__ delta_p, unsigned short *__restrict__ out,
-                     int8_t *__restrict__ dense8, DeviceState *__restrict__ st, int count) {
+                     int8_t *__restrict__ dense8, DeviceState *__restrict__ st, int count,
+                     unsigned short *__restrict__ out_stack, int plane_w, int stack_g) {
     __shared__ __align__(16) unsigned char tile[2][kTileBytes];
     constexpr int VV = (V > 1) ? V : 4;               // vector length of the paired path
     constexpr int VF = Vec<T>::V;                     // vector length of the contiguous path
@@ -424,6 +425,13 @@ quantize_nhwc_kernel(const T *__restrict__ x, int B, int C, int HW, unsigned lon
             if (p0 + pp < HW && c0 + ch * 8 < C)
                 *reinterpret_cast<uint4 *>(out + (static_cast<long long>(b) * HW + p0 + pp) * C + c0 + ch * 8) =
                     *reinterpret_cast<const uint4 *>(tl + tile_off(pp, ch * 8));
+            // Second copy for the weight-gradient kernel of tiny planes: the images one below the other as tall
+            // images, a row of zeros after every image (what a tap that leaves an image must read).
+            if (out_stack != nullptr && pp < HW + plane_w && c0 + ch * 8 < C) {
+                const uint4 val = pp < HW ? *reinterpret_cast<const uint4 *>(tl + tile_off(pp, ch * 8)) : make_uint4(0u, 0u, 0u, 0u);
+                const long long row = static_cast<long long>(b) * (HW + plane_w) + pp;   // any number of images per tall image
+                *reinterpret_cast<uint4 *>(out_stack + row * C + c0 + ch * 8) = val;
+            }
         }
         // the other buffer is written next; this one again only after the next barrier
     }
@@ -438,13 +446,13 @@ quantize_nhwc_kernel(const T *__restrict__ x, int B, int C, int HW, unsigned lon
 
 template <typename T, int V>
 cudaError_t run_nhwc(dbp_ctx *ctx, const void *delta, int B, int C, int HW, unsigned long long seed, const float *delta_p,
-                     void *out, int8_t *dense8, bool count) {
+                     void *out, int8_t *dense8, bool count, void *out_stack, int plane_w, int stack_g) {
     const long long ntiles = static_cast<long long>(B) * ((C + kTC - 1) / kTC) * ((HW + kTP - 1) / kTP);
     long long blocks = ntiles < static_cast<long long>(ctx->sm_count) * 6 ? ntiles : static_cast<long long>(ctx->sm_count) * 6;
     if (blocks < 1) blocks = 1;
     return launch_chained(quantize_nhwc_kernel<T, V>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
                           static_cast<const T *>(delta), B, C, HW, seed, delta_p, static_cast<unsigned short *>(out), dense8,
-                          ctx->state, count ? 1 : 0);
+                          ctx->state, count ? 1 : 0, static_cast<unsigned short *>(out_stack), plane_w, stack_g);
 }
 
 }  // namespace
@@ -471,17 +479,21 @@ int launch_quantize_dense(dbp_ctx *ctx, const void *delta, int dtype, long long 
 // delta_z [B][C][HW] -> bf16 codes [B][HW][C] (C % 8 == 0) and, when dense8 is not null, int8 codes
 // in delta_z's order
 int launch_quantize_nhwc(dbp_ctx *ctx, const void *delta, int dtype, long long B, long long C, long long HW,
-                         unsigned long long seed, const float *delta_p, void *codes_nhwc, int8_t *dense8, bool count) {
+                         unsigned long long seed, const float *delta_p, void *codes_nhwc, int8_t *dense8, bool count,
+                         void *codes_stack, int plane_w, int stack_g) {
     if (C % 8 != 0 || B * C * HW >= (1ll << 40) || HW >= (1ll << 30)) return DBP_EUNSUPPORTED;
+    // the stacked copy is written by the path for planes smaller than a tile; the rows of image b start at
+    // b (HW + W) however many images make up a tall image: the stacking only adds the zero rows
+    if (codes_stack != nullptr && (HW >= kTP || plane_w <= 0 || stack_g <= 0 || HW + plane_w > kTP)) return DBP_EINVAL;
     const int b = static_cast<int>(B), c = static_cast<int>(C), hw = static_cast<int>(HW);
     cudaError_t e;
     if (dtype == DBP_F32)
-        e = hw % 4 == 0 ? run_nhwc<float, 4>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count)
-                        : run_nhwc<float, 1>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count);
+        e = hw % 4 == 0 ? run_nhwc<float, 4>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count, codes_stack, plane_w, stack_g)
+                        : run_nhwc<float, 1>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count, codes_stack, plane_w, stack_g);
     else
-        e = hw % 8 == 0   ? run_nhwc<__nv_bfloat16, 8>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count)
-            : hw % 4 == 0 ? run_nhwc<__nv_bfloat16, 4>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count)
-                          : run_nhwc<__nv_bfloat16, 1>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count);
+        e = hw % 8 == 0   ? run_nhwc<__nv_bfloat16, 8>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count, codes_stack, plane_w, stack_g)
+            : hw % 4 == 0 ? run_nhwc<__nv_bfloat16, 4>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count, codes_stack, plane_w, stack_g)
+                          : run_nhwc<__nv_bfloat16, 1>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count, codes_stack, plane_w, stack_g);
     return cuda_ok(e);
 }
 

@@ -419,14 +419,53 @@ x_split_kernel(const float *__restrict__ X, __nv_bfloat16 *__restrict__ out, lon
     }
 }
 
+// The same for tiny planes stacked into tall images (one row of zeros after every image): out is
+// [2][B / G][cin_pad][pitch] with G (H + 1) W positions per tall image; position q of tall image t is position
+// q % ((H + 1) W) of image t G + q / ((H + 1) W), or zero in the extra row and in the padding.
+__global__ void __launch_bounds__(256)
+x_split_stacked_kernel(const float *__restrict__ X, __nv_bfloat16 *__restrict__ out, long long Bt, int G, int Cin, int cin_pad,
+                       int HW, int W, int pitch) {
+    chain_wait();
+    chain_release();
+    const long long n = Bt * cin_pad * pitch;
+    const int per_img = HW + W;
+    for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += gridDim.x * 256ll) {
+        const long long pl = i / pitch;
+        const int q = static_cast<int>(i - pl * pitch);
+        const long long t = pl / cin_pad;
+        const int ci = static_cast<int>(pl - t * cin_pad);
+        const int g = q / per_img, r = q - g * per_img;
+        __nv_bfloat16 hi = __float2bfloat16_rn(0.f), lo = hi;
+        if (g < G && r < HW && ci < Cin) {
+            const float x = __ldg(X + ((t * G + g) * Cin + ci) * HW + r);
+            hi = __float2bfloat16_rn(x);
+            lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+        }
+        out[i] = hi;
+        out[n + i] = lo;
+    }
+}
+
 int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 }  // namespace
 
 // DBP_EUNSUPPORTED: the shape does not fit (the caller uses another kernel)
+int tc3_stack_images(const ConvShape &s, int io) {
+    const long long HW = s.H * s.W, per_img = HW + s.W;
+    if (io != DBP_F32 || s.k != 3 || HW >= 64 || per_img > 64 || s.B < 2) return 0;
+    // the largest divisor of the batch whose tall image stays within one segment of the kernel
+    for (long long g = s.B; g >= 2; --g)
+        if (s.B % g == 0 && g * per_img <= 320) return static_cast<int>(g);
+    return 0;
+}
+
+// stack_g > 0: `s` describes the tall images (B / G of them, G (H + 1) rows) and the codes are the stacked copy;
+// real_h is the height of one image
 int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, int io, const float *delta_p,
-                      const ConvShape &s, float *dW, int *err_flag) {
+                      const ConvShape &s, float *dW, int *err_flag, int stack_g, int real_h) {
     if (!tc3_tma_dw_supported(s, io)) return DBP_EUNSUPPORTED;
+    if (stack_g > 0 && io != DBP_F32) return DBP_EINVAL;
     const int pieces = io == DBP_F32 ? 2 : 1;
     // fp32 activations are re-written anyway (split into two bf16 pieces): their channels are padded to a
     // multiple of 8 on the way, so any Cin works there
@@ -484,10 +523,19 @@ int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, int i
         if ((rc = ws_reserve(ctx, ctx->x_padded, static_cast<size_t>(planes) * xpitch * 2 * 2))) return rc;
         long long blocks = (planes * (xpitch / 8) + 255) / 256;
         if (blocks > ctx->sm_count * 16) blocks = ctx->sm_count * 16;
-        if ((rc = cuda_ok(launch_chained(x_split_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, ctx->stream,
-                                         static_cast<const float *>(X), static_cast<__nv_bfloat16 *>(ctx->x_padded.ptr), s.B,
-                                         static_cast<int>(s.Cin), static_cast<int>(cin_pad), static_cast<int>(HW), static_cast<int>(xpitch)))))
-            return rc;
+        if (stack_g > 0) {
+            blocks = (planes * xpitch + 255) / 256;
+            if (blocks > ctx->sm_count * 16) blocks = ctx->sm_count * 16;
+            rc = cuda_ok(launch_chained(x_split_stacked_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, ctx->stream,
+                                        static_cast<const float *>(X), static_cast<__nv_bfloat16 *>(ctx->x_padded.ptr), s.B, stack_g,
+                                        static_cast<int>(s.Cin), static_cast<int>(cin_pad), static_cast<int>(real_h * s.W),
+                                        static_cast<int>(s.W), static_cast<int>(xpitch)));
+        } else {
+            rc = cuda_ok(launch_chained(x_split_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, ctx->stream,
+                                        static_cast<const float *>(X), static_cast<__nv_bfloat16 *>(ctx->x_padded.ptr), s.B,
+                                        static_cast<int>(s.Cin), static_cast<int>(cin_pad), static_cast<int>(HW), static_cast<int>(xpitch)));
+        }
+        if (rc) return rc;
         Xsrc = ctx->x_padded.ptr;
     } else if (HW % 8 != 0) {
         xpitch = (HW + 7) / 8 * 8;

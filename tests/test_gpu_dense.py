@@ -104,6 +104,11 @@ def test_dense_path_conv3x3(ctx, B, Ci, Co, H, W):
     (5, 512, 512, 2, 2),      # config-4 last stage: 4 positions per image
     (2, 72, 40, 9, 11),       # channel counts that fill no tile, odd width (element-wise staging)
     (2, 8, 16, 1, 1),         # a single position
+    (32, 64, 64, 4, 4),       # tiny planes, dW on images stacked 16 to a tall image (two tall images)
+    (128, 16, 24, 2, 2),      # 53 images of 6 rows each would be 318 rows: the largest divisor below is 32
+    (12, 8, 8, 3, 5),         # odd plane sizes stacked (12 images of 20 positions)
+    (7, 16, 16, 6, 6),        # a prime batch: 7 images in one tall image
+    (9, 8, 16, 7, 8),         # 56 + 8 = 64 positions with the extra row: the largest plane that is stacked
 ])
 def test_dense_path_conv3x3_fp32_operands(ctx, B, Ci, Co, H, W):
     """fp32 layers on the tensor cores: weights and activations enter as two bf16 pieces each (the sum of the
