@@ -276,6 +276,17 @@ int dithered_conv_backward_host(dbp_ctx *ctx, const void *delta, const void *X, 
                                 float *delta_out, long long *nnz_out);
 
 /*
+ * delta_z = delta_a (.) f'(z) folded into the next call (the elementwise step in front of Eq. (qdz)): `mask`
+ * (DEVICE, one byte per element of delta, non-zero where z > 0; must stay valid until that call's kernels have
+ * run) makes the next dithered_linear_backward / dithered_conv_backward on this context treat its `delta`
+ * argument as delta_a and quantize delta_a (.) mask. fp32 only (DBP_EUNSUPPORTED otherwise, at that call).
+ * Small linear layers apply the mask while they read delta_a (no extra pass, no delta_z in memory); other
+ * layers run the ReLU-derivative kernel into a workspace first. The setting is consumed by that one call.
+ * mask = NULL clears it.
+ */
+int dbp_set_relu_mask(dbp_ctx *ctx, const uint8_t *mask);
+
+/*
  * Elementwise steps between layers of a network's backward pass (Section 3, backward
  * equations): delta_z = delta_a (.) f'(z) for ReLU, with the derivative given as one byte
  * per element (0 or 1), and the 2x2 max-pool routing of a pooled gradient g [planes,h,w] to

@@ -21,7 +21,7 @@ EXPORTED_SYMBOLS = [
     "dithered_linear_backward", "dithered_conv_backward", "dithered_linear_backward_host",
     "dithered_conv_backward_host", "dbp_relu_backward", "dbp_maxpool2x2_backward",
     "dbp_profile_enable", "dbp_profile_select", "dbp_profile_read", "dbp_set_crossover", "nsd_step_size_noalloc",
-    "dbp_last_step", "dbp_layer_seed", "dbp_selftest_bounded_wait", "dbp_last_error", "dbp_wait_stats", "dbp_join", "dbp_kernel_launches", "dbp_measure_fma_peak",
+    "dbp_last_step", "dbp_layer_seed", "dbp_selftest_bounded_wait", "dbp_last_error", "dbp_wait_stats", "dbp_join", "dbp_kernel_launches", "dbp_measure_fma_peak", "dbp_set_relu_mask",
 ]
 
 KERNEL_KINDS = ["statistics", "quantize", "weight_taps", "dx", "dw", "db", "decode", "glue",
@@ -62,6 +62,7 @@ def load_library():
     lib.dbp_create.argtypes = [ctypes.POINTER(vp), i32, vp]
     lib.dbp_destroy.argtypes = [vp]
     lib.dbp_set_stream.argtypes = [vp, vp]
+    lib.dbp_set_relu_mask.argtypes = [vp, vp]
     lib.dbp_status_string.argtypes = [i32]
     lib.dbp_status_string.restype = ctypes.c_char_p
     lib.dbp_last_device_status.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(ll)]
@@ -156,6 +157,13 @@ class Context:
         _check(load_library().dbp_last_device_status(self._h, ctypes.byref(st), ctypes.byref(sat)),
                "dbp_last_device_status")
         return st.value, sat.value
+
+    def set_relu_mask(self, mask: Optional[torch.Tensor]):
+        """The next backward call on this context quantizes delta (.) mask (uint8, one byte per element, non-zero
+        where the forward pre-activation was positive); fp32 only. Consumed by that call."""
+        if mask is not None and not (mask.is_cuda and mask.is_contiguous() and mask.dtype == torch.uint8):
+            raise ValueError("mask must be a contiguous CUDA uint8 tensor")
+        _check(load_library().dbp_set_relu_mask(self._h, _ptr(mask)), "dbp_set_relu_mask")
 
     def last_step(self):
         """(Delta, nnz) of the most recent quantization on this context (synchronises)."""
@@ -399,7 +407,15 @@ def network_backward(ctx: Context, kinds, Xs, Ws, relu_masks, pool_argmax, delta
     res = [None] * L
     delta_a = delta_out
     for l in range(L - 1, -1, -1):
-        dz = delta_a if relu_masks[l] is None else relu_backward(ctx, delta_a, relu_masks[l])
+        # nobody asks for delta_z: the mask is folded into the call (small linear layers never write delta_z at all)
+        fold = relu_masks[l] is not None and not keep_delta_z and not with_sparse and delta_a.dtype == torch.float32
+        if fold:
+            if delta_a.numel() != relu_masks[l].numel():
+                raise ValueError("mask must have one byte per element of delta")
+            ctx.set_relu_mask(relu_masks[l])
+            dz = delta_a
+        else:
+            dz = delta_a if relu_masks[l] is None else relu_backward(ctx, delta_a, relu_masks[l])
         q = SparseGradient(dz.numel(), ctx.device) if with_sparse else None
         fn = dithered_linear_backward if kinds[l] == "linear" else dithered_conv_backward
         need_dx = l > 0 or first_layer_dX

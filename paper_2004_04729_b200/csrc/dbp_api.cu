@@ -147,6 +147,9 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
                        const float *delta_in, dbp_sparse *q_out, float *dW, void *dX, float *db,
                        unsigned flags) {
     if (!ctx || !delta) return DBP_EINVAL;
+    // a ReLU mask set for this call: consumed here whatever happens next
+    const uint8_t *mask = ctx->next_mask;
+    ctx->next_mask = nullptr;
     if (io != DBP_F32 && io != DBP_BF16) return DBP_EINVAL;
     if (s.B <= 0 || s.Cin <= 0 || s.Cout <= 0 || s.H <= 0 || s.W <= 0) return DBP_EINVAL;
     if (s.B > 65535 * 32 || s.Cin > (1 << 20) || s.Cout > (1 << 20) || s.H > 4096 || s.W > 4096) return DBP_EINVAL;
@@ -164,7 +167,8 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     const long long numel = s.B * s.Cout * s.H * s.W;
     const float *delta_p = nullptr;
     const int8_t *codes = nullptr;
-    // small fp32 layers with one position per image (linear layers): everything in one launch
+    if (mask && io != DBP_F32) return DBP_EUNSUPPORTED;
+    // small fp32 layers with one position per image (linear layers): two chained launches
     if (io == DBP_F32 && s.k == 1 && s.H == 1 && s.W == 1 && !q_out && (dW || dX) && (!db || dW) &&
         !(flags & (DBP_FORCE_SPARSE | DBP_FORCE_DENSE)) && small_linear_fits(ctx, s.B, s.Cout, s.Cin, dW != nullptr, dX != nullptr)) {
         if (ctx->aux_pending) {
@@ -178,10 +182,18 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
             KernelTimer t(ctx, DBP_K_FUSED);
             rc = launch_small_linear(ctx, static_cast<const float *>(delta), static_cast<const float *>(X),
                                      static_cast<const float *>(W), s.B, s.Cout, s.Cin, seed, scale, delta_in, dW,
-                                     static_cast<float *>(dX), db, ctx->delta_sets ? ctx->delta_sets + ctx->code_set : nullptr);
+                                     static_cast<float *>(dX), db, ctx->delta_sets ? ctx->delta_sets + ctx->code_set : nullptr, mask);
         }
         if (!rc && ctx->hook_after_dx && cudaEventRecord(ctx->hook_after_dx, ctx->stream) != cudaSuccess) return DBP_ECUDA;
         return rc;
+    }
+    if (mask) {      // every other path reads delta_z from memory: make it
+        const int wr = ws_reserve(ctx, ctx->dz_tmp, static_cast<size_t>(numel) * sizeof(float));
+        if (wr) return wr;
+        KernelTimer t(ctx, DBP_K_GLUE);
+        const int gr = launch_relu_backward(ctx, static_cast<const float *>(delta), mask, static_cast<float *>(ctx->dz_tmp.ptr), numel);
+        if (gr) return gr;
+        delta = ctx->dz_tmp.ptr;
     }
     // While the stream is being captured into a CUDA graph the density read-back is left alone
     // (an event recorded inside a capture cannot be queried): the choice of path is the one the
@@ -420,7 +432,7 @@ int dbp_destroy(dbp_ctx *ctx) {
     cudaStreamSynchronize(ctx->stream);
     if (ctx->aux) cudaStreamSynchronize(ctx->aux);
     Workspace *all[] = {&ctx->dense_codes[0], &ctx->dense_codes[1], &ctx->codes16[0], &ctx->codes16[1],
-                        &ctx->codes_nhwc[0], &ctx->codes_nhwc[1], &ctx->codes_stack[0], &ctx->codes_stack[1], &ctx->dw_acc, &ctx->x_padded, &ctx->w_taps, &ctx->sp_bitmap, &ctx->sp_offsets, &ctx->sp_values,
+                        &ctx->codes_nhwc[0], &ctx->codes_nhwc[1], &ctx->codes_stack[0], &ctx->codes_stack[1], &ctx->dz_tmp, &ctx->dw_acc, &ctx->x_padded, &ctx->w_taps, &ctx->sp_bitmap, &ctx->sp_offsets, &ctx->sp_values,
                         &ctx->tc_partials};
     for (Workspace *w : all) if (w->ptr) cudaFree(w->ptr);
     for (Workspace &w : ctx->io) if (w.ptr) cudaFree(w.ptr);
@@ -704,6 +716,12 @@ int dithered_conv_backward_host(dbp_ctx *ctx, const void *delta, const void *X, 
     if (!(scale > 0.f)) return DBP_EINVAL;
     ConvShape s{B, Cin, Cout, H, Wd, k};
     return host_backward(ctx, delta, X, W, io, s, seed, scale, dW, dX, db, flags, delta_out, nnz_out);
+}
+
+int dbp_set_relu_mask(dbp_ctx *ctx, const uint8_t *mask) {
+    if (!ctx) return DBP_EINVAL;
+    ctx->next_mask = mask;
+    return DBP_OK;
 }
 
 int dbp_relu_backward(dbp_ctx *ctx, const float *delta_a, const uint8_t *mask, float *delta_z, long long numel) {

@@ -53,6 +53,8 @@ struct dbp_ctx {
     dbp::Workspace sp_bitmap, sp_offsets, sp_values;  // internal dbp_sparse
     dbp::Workspace tc_partials;         // split-K partial blocks of the dense dW kernel
     dbp::Workspace codes_nhwc[2];       // bf16 codes [B][position][Cout] for the TMA-fed 3x3 kernels
+    const uint8_t *next_mask = nullptr; // ReLU mask for the next backward call (dbp_set_relu_mask)
+    dbp::Workspace dz_tmp;              // delta_z = delta_a (.) mask when that call cannot fold the mask into its loads
     dbp::Workspace codes_stack[2];      // the same codes with G images stacked into one tall image (tiny planes, dW)
     float *delta_sets = nullptr;        // device float[2]: the step size that belongs to each set
     int code_set = 0;                   // the set the next call writes
@@ -134,7 +136,7 @@ int launch_decode(dbp_ctx *ctx, const uint32_t *bitmap, const uint16_t *offsets,
 bool small_linear_fits(const dbp_ctx *ctx, long long B, long long N, long long K, bool want_dw, bool want_dx);
 int launch_small_linear(dbp_ctx *ctx, const float *delta, const float *X, const float *W, long long B, long long N,
                         long long K, unsigned long long seed, float scale, const float *delta_in, float *dW, float *dX,
-                        float *db, float *delta_set);
+                        float *db, float *delta_set, const uint8_t *mask = nullptr);
 
 // ---- product_kernels.cu
 struct ConvShape {

@@ -70,6 +70,7 @@ __device__ __forceinline__ double warp_sum(double v) {
 
 struct SmallLinP {
     const float *delta, *X, *W;   // [B][N], [B][K], [N][K]
+    const uint8_t *mask;          // not null: delta is delta_a and the gradient is delta_a where mask != 0, else 0
     const float *delta_in;        // used when scale <= 0
     float scale;
     long long B, N, K, Np;        // Np: N rounded up to 8, the row pitch of the codes
@@ -99,7 +100,9 @@ small_linear_quantize_kernel(const SmallLinP p) {
     float delta;
     bool nonfinite = false;
     if (p.scale > 0.f) {
-        const float pivot = __ldg(p.delta);
+        const bool masked = p.mask != nullptr;
+        const float pivot = (!masked || __ldg(p.mask)) ? __ldg(p.delta) : 0.f;
+        const uchar4 *m4 = reinterpret_cast<const uchar4 *>(p.mask);
         double d1 = 0.0, d2 = 0.0;
         const long long nvec = n / 4;
         const float4 *v4 = reinterpret_cast<const float4 *>(p.delta);
@@ -110,6 +113,11 @@ small_linear_quantize_kernel(const SmallLinP p) {
             for (int u = 0; u < kU; ++u) {
                 const long long i = i0 + u * kThreads + tid;
                 v[u] = i < nvec ? __ldg(v4 + i) : make_float4(pivot, pivot, pivot, pivot);
+                if (masked && i < nvec) {
+                    const uchar4 m = __ldg(m4 + i);
+                    v[u].x = m.x ? v[u].x : 0.f; v[u].y = m.y ? v[u].y : 0.f;
+                    v[u].z = m.z ? v[u].z : 0.f; v[u].w = m.w ? v[u].w : 0.f;
+                }
             }
 #pragma unroll
             for (int u = 0; u < kU; ++u) {
@@ -122,7 +130,8 @@ small_linear_quantize_kernel(const SmallLinP p) {
         }
         if (tid == 0)
             for (long long i = nvec * 4; i < n; ++i) {
-                const double c = static_cast<double>(__ldg(p.delta + i)) - static_cast<double>(pivot);
+                const float xi = (!masked || __ldg(p.mask + i)) ? __ldg(p.delta + i) : 0.f;
+                const double c = static_cast<double>(xi) - static_cast<double>(pivot);
                 d1 += c;
                 d2 += c * c;
             }
@@ -163,7 +172,8 @@ small_linear_quantize_kernel(const SmallLinP p) {
             for (int h = 0; h < 2; ++h) {
                 float q = 0.f;
                 if (live && e0 + j + h < n) {
-                    const float t = __fmaf_rn(__ldg(p.delta + e0 + j + h), inv, u[h]);
+                    const float xe = (p.mask == nullptr || __ldg(p.mask + e0 + j + h)) ? __ldg(p.delta + e0 + j + h) : 0.f;
+                    const float t = __fmaf_rn(xe, inv, u[h]);
                     const float tc = fminf(fmaxf(t, -127.f), 127.99999f);      // clipped codes are counted, NaN gives 0
                     const bool num = (t == t);
                     sat += (num && tc != t) ? 1u : 0u;
@@ -407,9 +417,9 @@ bool small_linear_fits(const dbp_ctx *ctx, long long B, long long N, long long K
 
 int launch_small_linear(dbp_ctx *ctx, const float *delta, const float *X, const float *W, long long B, long long N,
                         long long K, unsigned long long seed, float scale, const float *delta_in, float *dW, float *dX,
-                        float *db, float *delta_set) {
+                        float *db, float *delta_set, const uint8_t *mask) {
     SmallLinP p{};
-    p.delta = delta; p.X = X; p.W = W; p.delta_in = delta_in; p.scale = scale;
+    p.delta = delta; p.X = X; p.W = W; p.delta_in = delta_in; p.scale = scale; p.mask = mask;
     p.B = B; p.N = N; p.K = K; p.Np = (N + 7) / 8 * 8; p.seed = seed;
     p.dW = dW; p.dX = dX; p.db = dW ? db : nullptr;
     p.st = ctx->state; p.delta_set = delta_set;

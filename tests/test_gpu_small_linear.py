@@ -125,3 +125,57 @@ def test_larger_layers_and_a_callers_structure_take_the_general_path(ctx):
     pr = ctx.profile_read()
     ctx.profile_enable(False)
     assert pr["fused"][1] == 0 and pr["statistics"][1] == 2
+
+
+def test_relu_mask_folded_into_the_call(ctx):
+    """dbp_set_relu_mask: the next call quantizes delta_a (.) mask. A small linear layer applies the mask while it
+    reads delta_a; a convolution runs the ReLU-derivative kernel first. Either way the results are those of the
+    call on delta_z = delta_a (.) mask, and the setting lasts for one call."""
+    import paper_2004_04729_b200 as dbp
+    rng = np.random.default_rng(12)
+    L = wl.linear_layer(96, 52, 136, data_seed=901, scale=2.0, seed=3)
+    mask = (rng.random(L.delta.shape) < 0.6).astype(np.uint8)
+    dz = (L.delta * mask).astype(np.float32)
+    d, X, W, m = _cu(L.delta), _cu(L.X), _cu(L.W), torch.from_numpy(mask).cuda()
+    ctx.set_relu_mask(m)
+    out = _fused_was_used(ctx, lambda: dbp.dithered_linear_backward(ctx, d, X, W, L.seed, L.scale, need_db=True))
+    D, nnz = ctx.last_step()
+    D = np.float32(D)
+    want = oracle.step_size(dz, L.scale)
+    assert abs(float(D) - float(want)) <= 1e-6 * float(want)
+    codes, onnz, _ = oracle.nsd_codes(dz, L.seed, D)
+    assert nnz == onnz
+    _check_products(out, oracle.linear_backward(codes, D, L.X, L.W, with_abs=True), ("dW", "dX", "db"))
+    # consumed: the same call again quantizes delta itself
+    dbp.dithered_linear_backward(ctx, d, X, W, L.seed, L.scale)
+    _, nnz2 = ctx.last_step()
+    assert nnz2 == oracle.nsd_codes(L.delta, L.seed, np.float32(ctx.last_step()[0]))[1] and nnz2 != nnz
+    # a convolution: bit-identical to the two-step form
+    C = wl.conv_layer(4, 16, 24, 8, 8, 3, data_seed=902, scale=2.0)
+    cm = (rng.random(C.delta.shape) < 0.5).astype(np.uint8)
+    cd, cX, cW, cmask = _cu(C.delta), _cu(C.X), _cu(C.W), torch.from_numpy(cm).cuda()
+    ref = dbp.dithered_conv_backward(ctx, dbp.relu_backward(ctx, cd, cmask), cX, cW, C.seed, C.scale)
+    ref_step = ctx.last_step()
+    ctx.set_relu_mask(cmask)
+    got = dbp.dithered_conv_backward(ctx, cd, cX, cW, C.seed, C.scale)
+    assert ctx.last_step() == ref_step
+    assert torch.equal(got["dX"], ref["dX"])
+    assert (got["dW"] - ref["dW"]).abs().max().item() <= 1e-5 * ref["dW"].abs().max().item()
+
+
+def test_network_backward_without_delta_z_matches_the_step_by_step_form(ctx):
+    """LeNet-300-100 chain: with nobody asking for delta_z or the sparse structure the masks are folded into the
+    calls; the gradients are those of the step-by-step form (dW to the tolerance: other kernels add in another order)."""
+    import paper_2004_04729_b200 as dbp
+    c = wl.mlp_chain(batch=64)
+    cu = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    Xs, Ws = [cu(a) for a in c.X], [cu(a) for a in c.W]
+    masks = [None if mk is None else cu(mk.astype(np.uint8)) for mk in c.relu_mask]
+    pools = [cu(a) for a in c.pool_argmax]
+    dout = cu(c.delta_out)
+    ref = dbp.network_backward(ctx, c.kinds, Xs, Ws, masks, pools, dout, c.scale, 0, keep_delta_z=True)
+    got = dbp.network_backward(ctx, c.kinds, Xs, Ws, masks, pools, dout, c.scale, 0, with_sparse=False)
+    torch.cuda.synchronize()
+    for a, b in zip(ref, got):
+        scale = a["dW"].abs().max().item()
+        assert (a["dW"] - b["dW"]).abs().max().item() <= 2e-5 * scale
