@@ -407,7 +407,7 @@ def crossover_sweep(torch, dbp, ctx):
 
 # DRAM bytes (read + written) of one config-5 bench step's launches of each kernel kind, from the ncu capture summarised
 # in profiles/bench_step_config5_launch_list.md; None = the kernels of that kind changed after the capture
-NCU_DRAM_BYTES_PER_STEP = {"statistics": 1156516096, "quantize": 1333905664, "dx_dense": 1311159808, "dw_dense": 2629937920}
+NCU_DRAM_BYTES_PER_STEP = {"statistics": 1156897536, "quantize": 1334064128, "dx_dense": 1311867136, "dw_dense": 2630283776}
 
 
 def main():
