@@ -331,7 +331,7 @@ __device__ __forceinline__ void store_bytes(int8_t *dense8, long long e0, const 
 // image are one contiguous run of delta_z, read as whole vectors whatever the plane size. Otherwise,
 // plane size % V == 0: a thread takes the same V positions of two neighbouring channels and writes
 // the two codes of a position as one word. Otherwise element by element.
-template <typename T, int V>
+template <typename T, int V, bool STACK>
 __global__ void __launch_bounds__(kThreads)
 quantize_nhwc_kernel(const T *__restrict__ x, int B, int C, int HW, unsigned long long seed,
                      const float *__restrict__ delta_p, unsigned short *__restrict__ out,
@@ -427,7 +427,7 @@ quantize_nhwc_kernel(const T *__restrict__ x, int B, int C, int HW, unsigned lon
                     *reinterpret_cast<const uint4 *>(tl + tile_off(pp, ch * 8));
             // Second copy for the weight-gradient kernel of tiny planes: the images one below the other as tall
             // images, a row of zeros after every image (what a tap that leaves an image must read).
-            if (out_stack != nullptr && pp < HW + plane_w && c0 + ch * 8 < C) {
+            if (STACK && pp < HW + plane_w && c0 + ch * 8 < C) {
                 const uint4 val = pp < HW ? *reinterpret_cast<const uint4 *>(tl + tile_off(pp, ch * 8)) : make_uint4(0u, 0u, 0u, 0u);
                 const long long row = static_cast<long long>(b) * (HW + plane_w) + pp;   // any number of images per tall image
                 *reinterpret_cast<uint4 *>(out_stack + row * C + c0 + ch * 8) = val;
@@ -450,9 +450,13 @@ cudaError_t run_nhwc(dbp_ctx *ctx, const void *delta, int B, int C, int HW, unsi
     const long long ntiles = static_cast<long long>(B) * ((C + kTC - 1) / kTC) * ((HW + kTP - 1) / kTP);
     long long blocks = ntiles < static_cast<long long>(ctx->sm_count) * 6 ? ntiles : static_cast<long long>(ctx->sm_count) * 6;
     if (blocks < 1) blocks = 1;
-    return launch_chained(quantize_nhwc_kernel<T, V>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
+    if (out_stack != nullptr)
+        return launch_chained(quantize_nhwc_kernel<T, V, true>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
+                              static_cast<const T *>(delta), B, C, HW, seed, delta_p, static_cast<unsigned short *>(out), dense8,
+                              ctx->state, count ? 1 : 0, static_cast<unsigned short *>(out_stack), plane_w, stack_g);
+    return launch_chained(quantize_nhwc_kernel<T, V, false>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
                           static_cast<const T *>(delta), B, C, HW, seed, delta_p, static_cast<unsigned short *>(out), dense8,
-                          ctx->state, count ? 1 : 0, static_cast<unsigned short *>(out_stack), plane_w, stack_g);
+                          ctx->state, count ? 1 : 0, static_cast<unsigned short *>(nullptr), 0, 0);
 }
 
 }  // namespace
