@@ -8,7 +8,7 @@
 //      tensor by itself (the tensor sits in L2; every CTA adds in the same order, so all of them hold the
 //      same Delta and no grid-wide step separates statistics from quantization), then quantizes its own
 //      4096 elements into bf16 codes [B][N rounded up to 8] and counts the non-zero and clipped ones.
-//      The last CTA to finish publishes Delta and nnz.
+//      The first CTA publishes Delta; the second kernel adds up the counts.
 //   2. small_linear_products_kernel: every CTA owns one 64 x 64 tile of dW or of dX and accumulates it
 //      on the tensor cores: the codes are exact in bf16, the fp32 operand (X or W) is split into two
 //      bf16 pieces (the value rounded to bf16 and what that left over, rounded again: the pair is within
@@ -80,7 +80,7 @@ struct SmallLinP {
     float *delta_set;             // second place the step size goes to (may be null)
     unsigned short *codes;        // bf16 [B][Np]
     unsigned *slots;              // one non-zero count per CTA of the first kernel
-    int tiles_k, n_dw, n_dx;
+    int tiles_k, n_dw, n_dx, n_qctas;
     int vec4;                     // K % 4 == 0: 16-byte accesses along K
 };
 
@@ -89,7 +89,6 @@ __global__ void __launch_bounds__(kThreads)
 small_linear_quantize_kernel(const SmallLinP p) {
     __shared__ double red1[kThreads / 32], red2[kThreads / 32];
     __shared__ unsigned cnt_s[2];
-    __shared__ bool is_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     chain_wait();
     chain_release();
@@ -203,29 +202,16 @@ small_linear_quantize_kernel(const SmallLinP p) {
         if (sat) atomicAdd(&cnt_s[1], sat);
     }
     __syncthreads();
+    // Every CTA holds the same Delta, so the first one publishes it; the counts of the CTAs are added up by the
+    // products kernel, which runs when all of them are done (no election of a last CTA, no extra round trips here).
     if (tid == 0) {
         p.slots[blockIdx.x] = cnt_s[0];
         if (cnt_s[1]) atomicAdd(&p.st->saturated, static_cast<unsigned long long>(cnt_s[1]));
-        __threadfence();
-        const unsigned ticket = atomicAdd(&p.st->ticket, 1u);
-        is_last = (ticket == gridDim.x - 1);
-    }
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
-    unsigned long long total = 0;
-    for (int i = tid; i < static_cast<int>(gridDim.x); i += kThreads) total += __ldcg(p.slots + i);
-    const double tsum = warp_sum(static_cast<double>(total));   // counts below 2^53: exact
-    if (lane == 0) red1[warp] = tsum;
-    __syncthreads();
-    if (tid == 0) {
-        double all = 0.0;
-        for (int w = 0; w < kThreads / 32; ++w) all += red1[w];
-        p.st->nnz = static_cast<unsigned long long>(all);
-        p.st->delta = delta;
-        if (nonfinite) p.st->nonfinite = 1;
-        if (p.delta_set) *p.delta_set = delta;
-        p.st->ticket = 0u;
+        if (blockIdx.x == 0) {
+            p.st->delta = delta;
+            if (nonfinite) p.st->nonfinite = 1;
+            if (p.delta_set) *p.delta_set = delta;
+        }
     }
 }
 
@@ -365,6 +351,13 @@ small_linear_products_kernel(const SmallLinP p) {
     chain_release();
     const float delta = __ldcg(&p.st->delta);
     const float dscale = (delta > 0.f && delta < __int_as_float(0x7f800000)) ? delta : 0.f;
+    if (blockIdx.x == 0 && warp == 0) {                  // nnz of the step: the first kernel's per-CTA counts
+        unsigned long long total = 0;
+        for (int i = lane; i < p.n_qctas; i += 32) total += __ldcg(p.slots + i);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(kFull, total, o);
+        if (lane == 0) p.st->nnz = total;
+    }
     load_a(0, a0);
     if (kRed < nred) load_a(kRed, a1);
     for (long long r0 = 0; r0 < nred; r0 += 2 * kRed) {
@@ -433,6 +426,7 @@ int launch_small_linear(dbp_ctx *ctx, const float *delta, const float *X, const 
     p.vec4 = (K % 4 == 0) ? 1 : 0;
     const long long n = B * N;
     const unsigned qctas = static_cast<unsigned>((n + kQuantPerCta - 1) / kQuantPerCta);
+    p.n_qctas = static_cast<int>(qctas);
     if (int rc = cuda_ok(launch_chained(small_linear_quantize_kernel, dim3(qctas), dim3(kThreads), 0, ctx->stream, p))) return rc;
     return cuda_ok(launch_chained(small_linear_products_kernel, dim3(static_cast<unsigned>(p.n_dw + p.n_dx)), dim3(kThreads), 0,
                                   ctx->stream, p));
