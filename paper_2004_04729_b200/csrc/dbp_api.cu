@@ -4,6 +4,7 @@
 #include "dbp_internal.cuh"
 
 #include <atomic>
+#include <cstdlib>
 #include <cstdio>
 
 namespace dbp {
@@ -78,6 +79,14 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
     const int k = ctx->code_set;
     if ((rc = ws_reserve(ctx, ctx->dense_codes[k], static_cast<size_t>(numel) + 16))) return rc;
     int8_t *dense = static_cast<int8_t *>(ctx->dense_codes[k].ptr);
+    // The set's previous readers (an earlier call's dW kernels on the second stream) must be done before its step
+    // size and its codes are written again. The wait stands in front of the statistics kernel, where the stream
+    // already holds the previous call's fork event: stream operations between two kernels stop their programmatic
+    // overlap, so they are kept at one boundary per call.
+    if (ctx->set_busy[k]) {
+        if (cudaStreamWaitEvent(ctx->stream, ctx->ev_set_free[k], 0) != cudaSuccess) return fail_cuda("waiting for the code buffers");
+        ctx->set_busy[k] = false;
+    }
     {
         KernelTimer t(ctx, DBP_K_STATISTICS);
         // without a caller's dbp_sparse the step size also goes to the set's own scalar: the product kernels
@@ -86,11 +95,6 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
                                reinterpret_cast<unsigned long long *>(sp.nnz), jobs);
     }
     if (rc) return rc;
-    // the set's previous readers (an earlier call's dW kernels on the second stream) must be done
-    if (ctx->set_busy[k]) {
-        if (cudaStreamWaitEvent(ctx->stream, ctx->ev_set_free[k], 0) != cudaSuccess) return fail_cuda("waiting for the code buffers");
-        ctx->set_busy[k] = false;
-    }
     {
         KernelTimer t(ctx, DBP_K_QUANTIZE);
         // the sparse structure is written only for a caller who asked for it; the bf16 planes
@@ -265,6 +269,8 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
         // dX and dW read the same codes and nothing of each other: with both asked for, dW goes to the
         // context's second stream, so that its CTAs start as SMs come free instead of after the last dX CTA
         const bool forked = dX && dW && ctx->aux != nullptr;
+        // (forking after the dX kernel instead, which would keep the quantizer -> dX boundary free of stream
+        // operations, measured slower: dW then starts a kernel later and meets the next layer's dX)
         if (forked && (cudaEventRecord(ctx->ev_fork, ctx->stream) != cudaSuccess ||
                        cudaStreamWaitEvent(ctx->aux, ctx->ev_fork, 0) != cudaSuccess))
             return fail_cuda("forking the dW stream");
