@@ -304,6 +304,44 @@ def dense_times(torch, fns, reps):
     return out
 
 
+def per_shape_table(torch, layers, run_layer, ctx, dq, hbm_peak, no_dense):
+    """One row per distinct layer shape: time per layer of the whole backward (statistics, quantization, dX, dW)
+    with the instances of the shape run back to back on their own buffers, as in the step (dW of one instance may
+    run beside the next instance; joined after the last), the dense library's time for the same layers, and the
+    layer's algorithmic bytes against the measured bandwidth."""
+    groups = {}
+    for idx, item in enumerate(layers):
+        groups.setdefault(item[0].name, []).append(idx)
+    torch.backends.cudnn.benchmark = True
+    torch.backends.cudnn.allow_tf32 = False
+    torch.backends.cuda.matmul.allow_tf32 = False
+    rows = []
+    for name, idxs in groups.items():
+        L = layers[idxs[0]][0]
+        def ours():
+            for i in idxs:
+                run_layer(*layers[i])
+            ctx.join()
+        for _ in range(3):
+            ours()
+        torch.cuda.synchronize()
+        ms = time_events(torch, ours, 20) / len(idxs)
+        row = {"shape": name, "instances": len(idxs), "ms": ms, "algorithmic_mb": algorithmic_bytes(L) / 1e6,
+               "frac_of_measured_hbm": algorithmic_bytes(L) / (ms * 1e-3) / 1e9 / hbm_peak,
+               "tflops_dense_equiv": L.dense_flops / (ms * 1e-3) / 1e12}
+        if not no_dense and dq is not None:
+            fns = [dense_layer_fn(torch, layers[i][0], dq[i], layers[i][2], layers[i][3]) for i in idxs]
+            def dense():
+                for f in fns:
+                    f()
+            for _ in range(3):
+                dense()
+            torch.cuda.synchronize()
+            row["dense_ms"] = time_events(torch, dense, 20) / len(idxs)
+        rows.append(row)
+    return rows
+
+
 def tensor_peak():
     """Measured dense bf16 rate (TFLOP/s, burst) and where it comes from."""
     try:
@@ -649,13 +687,14 @@ def main():
 
     # ---- dense library backward on the same shapes (context, not the product path)
     dense = None
+    dq_by_layer = dq if (not args.no_dense and rank == 0) else None
     if not args.no_dense and rank == 0:
         fns = [dense_layer_fn(torch, L, g, X, W) for (L, d, X, W, dW, dX), g in zip(layers, dq)]
         dt = dense_times(torch, fns, max(20, args.steps // 4))
         dense = {k: {"ms_per_step": v, "gflops": dense_flops / (v * 1e-3) / 1e9} for k, v in dt.items()}
         dense["what"] = ("torch cuDNN/cuBLAS backward-data + backward-filter (cudnn.benchmark autotuning) on the "
                          "dequantized gradient Delta*q in the layers' dtype, same X and W buffers")
-        del fns, dq
+        del fns
 
     if rank != 0:
         if world > 1:
@@ -748,6 +787,7 @@ def main():
     }
     if not args.no_others and world == 1 and args.config == 5 and not (args.only or args.single):
         out["other_configs"] = {str(c): small_config(torch, dbp, ctx, c, hbm_peak, fma_peak) for c in (1, 2, 3, 4)}
+        out["per_shape"] = per_shape_table(torch, layers, run_layer, ctx, dq_by_layer, hbm_peak, args.no_dense)
     if not args.no_cpu and world == 1:
         v, dt, what, cores = oracle_sample(args.config)
         out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what,
