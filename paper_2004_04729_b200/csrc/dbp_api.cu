@@ -257,7 +257,8 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
                                    s.H * s.W, any_tma ? tma_code_pitch(s) : 0, any_tma ? &codes16 : nullptr,
                                    t3 ? &s : nullptr, t3 ? &codes_n : nullptr, jobs, stack_g, &codes_st);
     if (rc) return rc;
-    if (!capturing && !ctx->nnz_pending && ctx->nnz_host && ctx->nnz_event) {
+    // (the density decides nothing while the threshold is 0: no read-back then, one stream operation less)
+    if (!capturing && ctx->crossover > 0.f && !ctx->nnz_pending && ctx->nnz_host && ctx->nnz_event) {
         ctx->nnz_host_numel = numel;
         ctx->nnz_host_key = shape_key;
         if (cudaMemcpyAsync(ctx->nnz_host, &ctx->state->nnz, sizeof(unsigned long long), cudaMemcpyDeviceToHost,
