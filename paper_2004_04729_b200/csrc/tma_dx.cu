@@ -93,7 +93,8 @@ struct DxT {
     int ci_tiles, ksteps;
     int nct;                      // 64-position chunks per tile (4, or fewer when that gives too few tiles)
     int MA;                       // accumulators per tile: 1 (128 channels, two tiles in flight) or 2 (256 channels)
-    long long ntiles;
+    long long ntiles;             // tiles are taken from the last one down: the quantizer has just written the codes front to
+                                  // back, so the end of a tensor larger than the L2 is what is still there
     int *err_flag;
     unsigned long long *stats;    // wait counters (may be null)
 };
@@ -147,8 +148,9 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
             bool ok = true;
             long long waited = 0;
             for (long long t = blockIdx.x; t < p.ntiles && ok; t += gridDim.x) {
-                const int ci0 = static_cast<int>(t % p.ci_tiles) * 128 * MA;
-                const long long g0 = (t / p.ci_tiles) * p.nct;
+                const long long tr = p.ntiles - 1 - t;            // last positions first: see DxT::ntiles
+                const int ci0 = static_cast<int>(tr % p.ci_tiles) * 128 * MA;
+                const long long g0 = (tr / p.ci_tiles) * p.nct;
                 const int nch = static_cast<int>(p.nchunks - g0 < p.nct ? p.nchunks - g0 : p.nct);
                 // the tile's chunks are consecutive: image and position of the first, then step and wrap
                 const int b0 = static_cast<int>(g0 / p.chunks_per_img);
@@ -234,9 +236,10 @@ tma_dx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
           const unsigned uses = static_cast<unsigned>(MA == 2 ? it : (it >> 1));
           for (int am = 0; am < MA; ++am) {
             const int a = slot0 + am;
-            const int ci_w = (static_cast<int>(t % p.ci_tiles) * MA + am) * 128 + q * 32;
+            const long long tr = p.ntiles - 1 - t;
+            const int ci_w = (static_cast<int>(tr % p.ci_tiles) * MA + am) * 128 + q * 32;
             const int ci = ci_w + lane;
-            const long long g0 = (t / p.ci_tiles) * p.nct;
+            const long long g0 = (tr / p.ci_tiles) * p.nct;
             const int nch = static_cast<int>(p.nchunks - g0 < p.nct ? p.nchunks - g0 : p.nct);
             ok = mbar_wait_timed(&pipe.acc_full[a], uses & 1u, p.err_flag, we);
             if (!ok) break;
