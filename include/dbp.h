@@ -280,8 +280,9 @@ int dithered_conv_backward_host(dbp_ctx *ctx, const void *delta, const void *X, 
  * (DEVICE, one byte per element of delta, non-zero where z > 0; must stay valid until that call's kernels have
  * run) makes the next dithered_linear_backward / dithered_conv_backward on this context treat its `delta`
  * argument as delta_a and quantize delta_a (.) mask. fp32 only (DBP_EUNSUPPORTED otherwise, at that call).
- * Small linear layers apply the mask while they read delta_a (no extra pass, no delta_z in memory); other
- * layers run the ReLU-derivative kernel into a workspace first. The setting is consumed by that one call.
+ * Small linear layers and fp32 3x3 layers on the tensor-core kernels apply the mask while they read delta_a
+ * (no extra pass, no delta_z in memory; the mask must then start on a 4-byte boundary, else the next form is
+ * taken); other layers run the ReLU-derivative kernel into a workspace first. The setting is consumed by that one call.
  * mask = NULL clears it.
  */
 int dbp_set_relu_mask(dbp_ctx *ctx, const uint8_t *mask);

@@ -65,7 +65,7 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
                           bool want8 = true, long long planes_hw = 0, long long planes_pitch = 0,
                           const void **codes16 = nullptr, const ConvShape *nhwc = nullptr,
                           const void **codes_nhwc = nullptr, const SideJobs &jobs = SideJobs(),
-                          int stack_g = 0, const void **codes_stack = nullptr) {
+                          int stack_g = 0, const void **codes_stack = nullptr, const uint8_t *mask = nullptr) {
     int rc = DBP_OK;
     dbp_sparse sp;
     sp.bitmap = nullptr; sp.offsets = nullptr; sp.values = nullptr; sp.delta = nullptr; sp.nnz = nullptr;
@@ -92,7 +92,7 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
         // without a caller's dbp_sparse the step size also goes to the set's own scalar: the product kernels
         // read it there (the context's scalar is overwritten by the next call's statistics)
         rc = launch_statistics(ctx, delta, dtype, numel, scale, delta_in, q_out ? sp.delta : ctx->delta_sets + k,
-                               reinterpret_cast<unsigned long long *>(sp.nnz), jobs);
+                               reinterpret_cast<unsigned long long *>(sp.nnz), jobs, mask);
     }
     if (rc) return rc;
     {
@@ -131,7 +131,7 @@ int quantize_for_products(dbp_ctx *ctx, const void *delta, int dtype, long long 
                                           &ctx->state->delta, pn, nullptr, false, ps, static_cast<int>(nhwc->W), stack_g);
         } else if (pn) {
             rc = launch_quantize_nhwc(ctx, delta, dtype, nhwc->B, nhwc->Cout, nhwc->H * nhwc->W, seed,
-                                      &ctx->state->delta, pn, want8 ? dense : nullptr, true, ps, static_cast<int>(nhwc->W), stack_g);
+                                      &ctx->state->delta, pn, want8 ? dense : nullptr, true, ps, static_cast<int>(nhwc->W), stack_g, mask);
         } else {
             rc = launch_quantize_dense(ctx, delta, dtype, numel, seed, &ctx->state->delta, want8 ? dense : nullptr,
                                        p16, planes_hw, planes_pitch, true);
@@ -173,7 +173,8 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     const int8_t *codes = nullptr;
     if (mask && io != DBP_F32) return DBP_EUNSUPPORTED;
     // small fp32 layers with one position per image (linear layers): two chained launches
-    if (io == DBP_F32 && s.k == 1 && s.H == 1 && s.W == 1 && !q_out && (dW || dX) && (!db || dW) &&
+    const bool mask_vec = mask == nullptr || (reinterpret_cast<uintptr_t>(mask) & 3) == 0;    // masks are read four bytes at a time
+    if (io == DBP_F32 && s.k == 1 && s.H == 1 && s.W == 1 && !q_out && (dW || dX) && (!db || dW) && mask_vec &&
         !(flags & (DBP_FORCE_SPARSE | DBP_FORCE_DENSE)) && small_linear_fits(ctx, s.B, s.Cout, s.Cin, dW != nullptr, dX != nullptr)) {
         if (ctx->aux_pending) {
             const int jr = dbp_join(ctx);
@@ -190,14 +191,6 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
         }
         if (!rc && ctx->hook_after_dx && cudaEventRecord(ctx->hook_after_dx, ctx->stream) != cudaSuccess) return DBP_ECUDA;
         return rc;
-    }
-    if (mask) {      // every other path reads delta_z from memory: make it
-        const int wr = ws_reserve(ctx, ctx->dz_tmp, static_cast<size_t>(numel) * sizeof(float));
-        if (wr) return wr;
-        KernelTimer t(ctx, DBP_K_GLUE);
-        const int gr = launch_relu_backward(ctx, static_cast<const float *>(delta), mask, static_cast<float *>(ctx->dz_tmp.ptr), numel);
-        if (gr) return gr;
-        delta = ctx->dz_tmp.ptr;
     }
     // While the stream is being captured into a CUDA graph the density read-back is left alone
     // (an event recorded inside a capture cannot be queried): the choice of path is the one the
@@ -237,6 +230,18 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     }
     // 3x3 layers: the TMA-fed kernels read the codes position-major
     const bool t3 = dense && (dX || dW) && (t3_full || t3_dw_only);
+    // fp32 3x3 layers on the tensor-core kernels apply the mask while they read delta_a (statistics and the
+    // position-major quantizer); with a caller's sparse structure, or on any other path, delta_z is made first
+    const bool fold3 = mask && mask_vec && io == DBP_F32 && !q_out && t3;
+    const uint8_t *mask_q = fold3 ? mask : nullptr;
+    if (mask && !fold3) {      // every other path reads delta_z from memory: make it
+        const int wr = ws_reserve(ctx, ctx->dz_tmp, static_cast<size_t>(numel) * sizeof(float));
+        if (wr) return wr;
+        KernelTimer t(ctx, DBP_K_GLUE);
+        const int gr = launch_relu_backward(ctx, static_cast<const float *>(delta), mask, static_cast<float *>(ctx->dz_tmp.ptr), numel);
+        if (gr) return gr;
+        delta = ctx->dz_tmp.ptr;
+    }
     const bool need8 = !dense || db || (!t3 && ((dX && !dx_tma) || (dW && !dw_tma)));
     const void *codes16 = nullptr, *codes_n = nullptr;
     // what the statistics kernel does on the side: the TMA-fed 1x1 dW kernel adds its partial sums into dW, so dW
@@ -255,7 +260,7 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     const void *codes_st = nullptr;
     int rc = quantize_for_products(ctx, delta, io, numel, seed, scale, delta_in, q_out, &delta_p, &codes, need8,
                                    s.H * s.W, any_tma ? tma_code_pitch(s) : 0, any_tma ? &codes16 : nullptr,
-                                   t3 ? &s : nullptr, t3 ? &codes_n : nullptr, jobs, stack_g, &codes_st);
+                                   t3 ? &s : nullptr, t3 ? &codes_n : nullptr, jobs, stack_g, &codes_st, t3 ? mask_q : nullptr);
     if (rc) return rc;
     // (the density decides nothing while the threshold is 0: no read-back then, one stream operation less)
     if (!capturing && ctx->crossover > 0.f && !ctx->nnz_pending && ctx->nnz_host && ctx->nnz_event) {

@@ -113,7 +113,7 @@ struct SideJobs {
 };
 int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long numel, float scale,
                       const float *delta_in, float *delta_out, unsigned long long *nnz_out,
-                      const SideJobs &jobs = SideJobs());
+                      const SideJobs &jobs = SideJobs(), const uint8_t *mask = nullptr);
 int launch_quantize(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
                     unsigned long long seed, const float *delta_p, uint32_t *bitmap,
                     uint16_t *offsets, int8_t *values, int8_t *dense,
@@ -128,7 +128,7 @@ int launch_quantize_dense(dbp_ctx *ctx, const void *delta, int dtype, long long 
 // when dense8 is not null)
 int launch_quantize_nhwc(dbp_ctx *ctx, const void *delta, int dtype, long long B, long long C, long long HW,
                          unsigned long long seed, const float *delta_p, void *codes_nhwc, int8_t *dense8, bool count,
-                         void *codes_stack = nullptr, int plane_w = 0, int stack_g = 0);
+                         void *codes_stack = nullptr, int plane_w = 0, int stack_g = 0, const uint8_t *mask = nullptr);
 int launch_decode(dbp_ctx *ctx, const uint32_t *bitmap, const uint16_t *offsets,
                   const int8_t *values, long long numel, int8_t *dense);
 

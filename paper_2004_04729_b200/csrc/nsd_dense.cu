@@ -331,12 +331,23 @@ __device__ __forceinline__ void store_bytes(int8_t *dense8, long long e0, const 
 // image are one contiguous run of delta_z, read as whole vectors whatever the plane size. Otherwise,
 // plane size % V == 0: a thread takes the same V positions of two neighbouring channels and writes
 // the two codes of a position as one word. Otherwise element by element.
-template <typename T, int V, bool STACK>
+// mask (fp32 tensors only, may be null): x is delta_a and the gradient is delta_a where mask != 0, else 0
+__device__ __forceinline__ void apply_mask(const unsigned char *mask, long long e, float (&v)[4]) {
+    if (mask != nullptr) {
+        const uchar4 m = __ldg(reinterpret_cast<const uchar4 *>(mask + e));
+        v[0] = m.x ? v[0] : 0.f; v[1] = m.y ? v[1] : 0.f; v[2] = m.z ? v[2] : 0.f; v[3] = m.w ? v[3] : 0.f;
+    }
+}
+__device__ __forceinline__ void apply_mask(const unsigned char *, long long, float (&)[8]) {}
+
+template <typename T, int V, bool STACK, bool MASKED>
 __global__ void __launch_bounds__(kThreads)
 quantize_nhwc_kernel(const T *__restrict__ x, int B, int C, int HW, unsigned long long seed,
                      const float *__restrict__ delta_p, unsigned short *__restrict__ out,
                      int8_t *__restrict__ dense8, DeviceState *__restrict__ st, int count,
-                     unsigned short *__restrict__ out_stack, int plane_w, int stack_g) {
+                     unsigned short *__restrict__ out_stack, int plane_w, int stack_g,
+                     const unsigned char *__restrict__ mask_in) {
+    const unsigned char *mask = MASKED ? mask_in : nullptr;
     __shared__ __align__(16) unsigned char tile[2][kTileBytes];
     constexpr int VV = (V > 1) ? V : 4;               // vector length of the paired path
     constexpr int VF = Vec<T>::V;                     // vector length of the contiguous path
@@ -367,6 +378,7 @@ quantize_nhwc_kernel(const T *__restrict__ x, int B, int C, int HW, unsigned lon
                 if (live) {
                     float a[VF];
                     Vec<T>::load(x + base + v * VF, a);
+                    apply_mask(mask, base + v * VF, a);
                     codes_of<VF>(a, base + v * VF, seed, inv, f, nz, sat);
                 }
                 if (dense8 != nullptr) store_bytes<VF>(dense8, base + v * VF, f);
@@ -390,6 +402,8 @@ quantize_nhwc_kernel(const T *__restrict__ x, int B, int C, int HW, unsigned lon
                     float a0[VV], a1[VV];
                     TileLoad<T, VV>::ld(x + e0, a0);
                     TileLoad<T, VV>::ld(x + e1, a1);
+                    apply_mask(mask, e0, a0);
+                    apply_mask(mask, e1, a1);
                     codes_of<VV>(a0, e0, seed, inv, f0, nz, sat);
                     codes_of<VV>(a1, e1, seed, inv, f1, nz, sat);
                 }
@@ -410,7 +424,7 @@ quantize_nhwc_kernel(const T *__restrict__ x, int B, int C, int HW, unsigned lon
                 float f = 0.f;
                 const bool in = c0 + c < C && p0 + pp < HW;
                 const long long e = (static_cast<long long>(b) * C + c0 + c) * HW + p0 + pp;
-                if (in && live) f = code_single(Vec<T>::one(x + e), e, seed, inv, sat);
+                if (in && live) f = code_single((mask == nullptr || __ldg(mask + e)) ? Vec<T>::one(x + e) : 0.f, e, seed, inv, sat);
                 if (in && dense8 != nullptr) dense8[e] = static_cast<int8_t>(static_cast<int>(f));
                 nnz += f != 0.f;
                 *reinterpret_cast<unsigned short *>(tl + tile_off(pp, c)) = static_cast<unsigned short>(__float_as_uint(f) >> 16);
@@ -446,17 +460,20 @@ quantize_nhwc_kernel(const T *__restrict__ x, int B, int C, int HW, unsigned lon
 
 template <typename T, int V>
 cudaError_t run_nhwc(dbp_ctx *ctx, const void *delta, int B, int C, int HW, unsigned long long seed, const float *delta_p,
-                     void *out, int8_t *dense8, bool count, void *out_stack, int plane_w, int stack_g) {
+                     void *out, int8_t *dense8, bool count, void *out_stack, int plane_w, int stack_g, const uint8_t *mask) {
     const long long ntiles = static_cast<long long>(B) * ((C + kTC - 1) / kTC) * ((HW + kTP - 1) / kTP);
     long long blocks = ntiles < static_cast<long long>(ctx->sm_count) * 6 ? ntiles : static_cast<long long>(ctx->sm_count) * 6;
     if (blocks < 1) blocks = 1;
-    if (out_stack != nullptr)
-        return launch_chained(quantize_nhwc_kernel<T, V, true>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
+    const unsigned char *m = static_cast<const unsigned char *>(mask);
+    auto go = [&](auto kern, unsigned short *stack) {
+        return launch_chained(kern, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
                               static_cast<const T *>(delta), B, C, HW, seed, delta_p, static_cast<unsigned short *>(out), dense8,
-                              ctx->state, count ? 1 : 0, static_cast<unsigned short *>(out_stack), plane_w, stack_g);
-    return launch_chained(quantize_nhwc_kernel<T, V, false>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
-                          static_cast<const T *>(delta), B, C, HW, seed, delta_p, static_cast<unsigned short *>(out), dense8,
-                          ctx->state, count ? 1 : 0, static_cast<unsigned short *>(nullptr), 0, 0);
+                              ctx->state, count ? 1 : 0, stack, stack ? plane_w : 0, stack ? stack_g : 0, m);
+    };
+    unsigned short *st = static_cast<unsigned short *>(out_stack);
+    if (mask != nullptr)      // fp32 only (checked by the caller)
+        return st ? go(quantize_nhwc_kernel<T, V, true, true>, st) : go(quantize_nhwc_kernel<T, V, false, true>, st);
+    return st ? go(quantize_nhwc_kernel<T, V, true, false>, st) : go(quantize_nhwc_kernel<T, V, false, false>, st);
 }
 
 }  // namespace
@@ -484,20 +501,21 @@ int launch_quantize_dense(dbp_ctx *ctx, const void *delta, int dtype, long long 
 // in delta_z's order
 int launch_quantize_nhwc(dbp_ctx *ctx, const void *delta, int dtype, long long B, long long C, long long HW,
                          unsigned long long seed, const float *delta_p, void *codes_nhwc, int8_t *dense8, bool count,
-                         void *codes_stack, int plane_w, int stack_g) {
+                         void *codes_stack, int plane_w, int stack_g, const uint8_t *mask) {
     if (C % 8 != 0 || B * C * HW >= (1ll << 40) || HW >= (1ll << 30)) return DBP_EUNSUPPORTED;
+    if (mask != nullptr && dtype != DBP_F32) return DBP_EUNSUPPORTED;
     // the stacked copy is written by the path for planes smaller than a tile; the rows of image b start at
     // b (HW + W) however many images make up a tall image: the stacking only adds the zero rows
     if (codes_stack != nullptr && (HW >= kTP || plane_w <= 0 || stack_g <= 0 || HW + plane_w > kTP)) return DBP_EINVAL;
     const int b = static_cast<int>(B), c = static_cast<int>(C), hw = static_cast<int>(HW);
     cudaError_t e;
     if (dtype == DBP_F32)
-        e = hw % 4 == 0 ? run_nhwc<float, 4>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count, codes_stack, plane_w, stack_g)
-                        : run_nhwc<float, 1>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count, codes_stack, plane_w, stack_g);
+        e = hw % 4 == 0 ? run_nhwc<float, 4>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count, codes_stack, plane_w, stack_g, mask)
+                        : run_nhwc<float, 1>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count, codes_stack, plane_w, stack_g, mask);
     else
-        e = hw % 8 == 0   ? run_nhwc<__nv_bfloat16, 8>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count, codes_stack, plane_w, stack_g)
-            : hw % 4 == 0 ? run_nhwc<__nv_bfloat16, 4>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count, codes_stack, plane_w, stack_g)
-                          : run_nhwc<__nv_bfloat16, 1>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count, codes_stack, plane_w, stack_g);
+        e = hw % 8 == 0   ? run_nhwc<__nv_bfloat16, 8>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count, codes_stack, plane_w, stack_g, mask)
+            : hw % 4 == 0 ? run_nhwc<__nv_bfloat16, 4>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count, codes_stack, plane_w, stack_g, mask)
+                          : run_nhwc<__nv_bfloat16, 1>(ctx, delta, b, c, hw, seed, delta_p, codes_nhwc, dense8, count, codes_stack, plane_w, stack_g, mask);
     return cuda_ok(e);
 }
 

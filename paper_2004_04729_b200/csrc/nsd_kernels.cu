@@ -71,12 +71,25 @@ __device__ __forceinline__ double warp_sum(double v) {
 // sigma: a constant tensor gives exactly 0 and a mean far from 0 costs no accuracy (raw moments
 // would cancel). sigma is the population standard deviation about the mean; Delta = scale * sigma
 // rounded once to fp32.
-template <typename T>
+// MASKED (fp32 only): the tensor is delta_a and the statistics are those of delta_a where mask != 0, else 0 (the
+// ReLU derivative folded into the read; one byte per element).
+template <bool MASKED>
+__device__ __forceinline__ void mask4(const unsigned char *mask, long long e, float (&v)[4]) {
+    if (MASKED) {
+        const uchar4 m = __ldg(reinterpret_cast<const uchar4 *>(mask + e));
+        v[0] = m.x ? v[0] : 0.f; v[1] = m.y ? v[1] : 0.f; v[2] = m.z ? v[2] : 0.f; v[3] = m.w ? v[3] : 0.f;
+    }
+}
+template <bool MASKED>
+__device__ __forceinline__ void mask4(const unsigned char *, long long, float (&)[8]) {}   // bf16 tensors take no mask
+
+template <typename T, bool MASKED = false>
 __global__ void __launch_bounds__(kThreads)
 statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ partials,
                   DeviceState *__restrict__ st, float scale, float *__restrict__ delta_out,
                   unsigned long long *__restrict__ nnz_out, uint4 *__restrict__ zero_ptr, long long zero_n16,
-                  const void *__restrict__ w_src, unsigned short *__restrict__ w_dst, int w_f32, long long w_cout, int w_cin) {
+                  const void *__restrict__ w_src, unsigned short *__restrict__ w_dst, int w_f32, long long w_cout, int w_cin,
+                  const unsigned char *__restrict__ mask) {
     constexpr int EPT = Elem<T>::EPT;
     const long long nvec = n / EPT;
     chain_wait();
@@ -106,7 +119,7 @@ statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ par
         }
     }
     double d1 = 0.0, d2 = 0.0;
-    const float pivot = Elem<T>::one(x);
+    const float pivot = (!MASKED || __ldg(mask)) ? Elem<T>::one(x) : 0.f;
     const long long stride = static_cast<long long>(gridDim.x) * kThreads;
     // whole tiles of kUnroll x kThreads 128-bit vectors, a block at a time: kUnroll loads in flight
     // per thread, consecutive threads on consecutive vectors
@@ -117,6 +130,8 @@ statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ par
         float v[kUnroll][EPT];
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) Elem<T>::load_stream(p + static_cast<long long>(u) * kThreads * EPT, v[u]);
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) mask4<MASKED>(mask, (t * tile + threadIdx.x + static_cast<long long>(u) * kThreads) * EPT, v[u]);
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
             float s1 = 0.f, s2 = 0.f;
@@ -135,6 +150,7 @@ statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ par
     for (; i < nvec; i += stride) {
         float v[EPT];
         Elem<T>::load(x + i * EPT, v);
+        mask4<MASKED>(mask, i * EPT, v);
         float s1 = 0.f, s2 = 0.f;
 #pragma unroll
         for (int j = 0; j < EPT; ++j) {
@@ -147,7 +163,8 @@ statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ par
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         for (long long i = nvec * EPT; i < n; ++i) {
-            const double c = static_cast<double>(Elem<T>::one(x + i)) - static_cast<double>(pivot);
+            const float xi = (!MASKED || __ldg(mask + i)) ? Elem<T>::one(x + i) : 0.f;
+            const double c = static_cast<double>(xi) - static_cast<double>(pivot);
             d1 += c;
             d2 += c * c;
         }
@@ -407,7 +424,9 @@ decode_kernel(const uint32_t *__restrict__ bitmap, const uint16_t *__restrict__ 
 }  // namespace
 
 int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long numel, float scale,
-                      const float *delta_in, float *delta_out, unsigned long long *nnz_out, const SideJobs &jobs) {
+                      const float *delta_in, float *delta_out, unsigned long long *nnz_out, const SideJobs &jobs,
+                      const uint8_t *mask) {
+    if (mask != nullptr && dtype != DBP_F32) return DBP_EUNSUPPORTED;
     uint4 *zp = static_cast<uint4 *>(jobs.zero);
     const long long zn = jobs.zero ? static_cast<long long>(jobs.zero_bytes / 16) : 0;
     unsigned short *wd = static_cast<unsigned short *>(jobs.w_dst);
@@ -426,12 +445,17 @@ int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long nume
     if (jobs.zero != nullptr && blocks < static_cast<long long>(jobs.zero_bytes / (16 * kThreads * 4))) blocks = static_cast<long long>(jobs.zero_bytes / (16 * kThreads * 4));
     if (blocks > ctx->partial_blocks) blocks = ctx->partial_blocks;
     cudaError_t e;
-    if (dtype == DBP_F32)
-        e = launch_chained(statistics_kernel<float>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
-                           static_cast<const float *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out, zp, zn, jobs.w_src, wd, jobs.w_f32, jobs.Cout, wci);
+    const unsigned char *nomask = nullptr;
+    if (dtype == DBP_F32 && mask != nullptr)
+        e = launch_chained(statistics_kernel<float, true>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
+                           static_cast<const float *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out, zp, zn, jobs.w_src, wd, jobs.w_f32, jobs.Cout, wci,
+                           static_cast<const unsigned char *>(mask));
+    else if (dtype == DBP_F32)
+        e = launch_chained(statistics_kernel<float, false>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
+                           static_cast<const float *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out, zp, zn, jobs.w_src, wd, jobs.w_f32, jobs.Cout, wci, nomask);
     else
-        e = launch_chained(statistics_kernel<__nv_bfloat16>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
-                           static_cast<const __nv_bfloat16 *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out, zp, zn, jobs.w_src, wd, jobs.w_f32, jobs.Cout, wci);
+        e = launch_chained(statistics_kernel<__nv_bfloat16, false>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
+                           static_cast<const __nv_bfloat16 *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out, zp, zn, jobs.w_src, wd, jobs.w_f32, jobs.Cout, wci, nomask);
     return cuda_ok(e);
 }
 

@@ -150,17 +150,25 @@ def test_relu_mask_folded_into_the_call(ctx):
     dbp.dithered_linear_backward(ctx, d, X, W, L.seed, L.scale)
     _, nnz2 = ctx.last_step()
     assert nnz2 == oracle.nsd_codes(L.delta, L.seed, np.float32(ctx.last_step()[0]))[1] and nnz2 != nnz
-    # a convolution: bit-identical to the two-step form
-    C = wl.conv_layer(4, 16, 24, 8, 8, 3, data_seed=902, scale=2.0)
-    cm = (rng.random(C.delta.shape) < 0.5).astype(np.uint8)
-    cd, cX, cW, cmask = _cu(C.delta), _cu(C.X), _cu(C.W), torch.from_numpy(cm).cuda()
-    ref = dbp.dithered_conv_backward(ctx, dbp.relu_backward(ctx, cd, cmask), cX, cW, C.seed, C.scale)
-    ref_step = ctx.last_step()
-    ctx.set_relu_mask(cmask)
-    got = dbp.dithered_conv_backward(ctx, cd, cX, cW, C.seed, C.scale)
-    assert ctx.last_step() == ref_step
-    assert torch.equal(got["dX"], ref["dX"])
-    assert (got["dW"] - ref["dW"]).abs().max().item() <= 1e-5 * ref["dW"].abs().max().item()
+    # convolutions: bit-identical to the two-step form. fp32 3x3 layers on the tensor-core kernels apply the mask
+    # in the statistics kernel and in the quantizer (planes of 64 positions and more, tiny planes with stacked
+    # images, odd plane sizes); a 1x1 layer runs the ReLU-derivative kernel first.
+    for (B, Ci, Co, H, W, k) in ((4, 16, 24, 8, 8, 3), (32, 16, 16, 4, 4, 3), (3, 8, 8, 5, 7, 3), (2, 8, 16, 9, 9, 3), (4, 16, 8, 6, 6, 1)):
+        C = wl.conv_layer(B, Ci, Co, H, W, k, data_seed=902 + H, scale=2.0)
+        cm = (rng.random(C.delta.shape) < 0.5).astype(np.uint8)
+        cd, cX, cW, cmask = _cu(C.delta), _cu(C.X), _cu(C.W), torch.from_numpy(cm).cuda()
+        ref = dbp.dithered_conv_backward(ctx, dbp.relu_backward(ctx, cd, cmask), cX, cW, C.seed, C.scale, need_db=True)
+        ref_step = ctx.last_step()
+        ctx.set_relu_mask(cmask)
+        got = dbp.dithered_conv_backward(ctx, cd, cX, cW, C.seed, C.scale, need_db=True)
+        assert ctx.last_step() == ref_step, (B, Ci, Co, H, W, k)
+        assert torch.equal(got["dX"], ref["dX"]) and torch.equal(got["db"], ref["db"])
+        assert (got["dW"] - ref["dW"]).abs().max().item() <= 1e-5 * ref["dW"].abs().max().item()
+    # the oracle on delta_z for one of them
+    dz = (C.delta * cm).astype(np.float32)
+    D = np.float32(ref_step[0])
+    codes, onnz, _ = oracle.nsd_codes(dz, C.seed, D)
+    assert onnz == ref_step[1]
 
 
 def test_network_backward_without_delta_z_matches_the_step_by_step_form(ctx):
