@@ -476,12 +476,91 @@ cudaError_t run_nhwc(dbp_ctx *ctx, const void *delta, int B, int C, int HW, unsi
     return st ? go(quantize_nhwc_kernel<T, V, true, false>, st) : go(quantize_nhwc_kernel<T, V, false, false>, st);
 }
 
+// ---------------------------------------------------------------- bf16 planes of odd sizes
+// Planes whose size is no multiple of 4 (7 x 7, 9 x 9, ...) written at a pitch that is a multiple of 8: the codes
+// of eight consecutive elements then belong to unaligned places of one or two planes. A block takes a run of
+// whole planes (a multiple of eight of them, so that the run starts on a 16-byte boundary and on an even
+// element), quantizes it with whole-vector loads as everywhere, places the codes in shared memory at their pitch,
+// and the run leaves as one contiguous copy (the padding of a plane is never read by anybody).
+constexpr int kOddMaxSmem = 12 * 1024;            // bytes of the staged run (planes x pitch bf16)
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+quantize_planes_odd_kernel(const T *__restrict__ x, long long nplanes, int hw, int pitch, int planes_per_run,
+                           unsigned long long seed, const float *__restrict__ delta_p, unsigned short *__restrict__ out,
+                           int8_t *__restrict__ dense8, DeviceState *__restrict__ st, int count) {
+    constexpr int V = Vec<T>::V;
+    __shared__ __align__(16) unsigned short run_s[kOddMaxSmem / 2];
+    chain_wait();
+    chain_release();
+    const float delta = *delta_p;
+    const bool live = (delta > 0.f) && (delta < __int_as_float(0x7f800000));
+    const float inv = live ? __fdiv_rn(1.0f, delta) : 0.f;
+    const long long nruns = (nplanes + planes_per_run - 1) / planes_per_run;
+    unsigned sat = 0;
+    float nz = 0.f;
+    for (long long r = blockIdx.x; r < nruns; r += gridDim.x) {
+        const long long pl0 = r * planes_per_run;
+        const int np = static_cast<int>(nplanes - pl0 < planes_per_run ? nplanes - pl0 : planes_per_run);   // a multiple of 8
+        const long long e_base = pl0 * hw;
+        const int nvec = np * hw / V;
+        for (int v = threadIdx.x; v < nvec; v += kThreads) {
+            float f[V] = {};
+            const long long e0 = e_base + static_cast<long long>(v) * V;
+            if (live) {
+                float a[V];
+                Vec<T>::load(x + e0, a);
+                codes_of<V>(a, e0, seed, inv, f, nz, sat);
+            }
+            if (dense8 != nullptr) store_bytes<V>(dense8, e0, f);
+            int pl = (v * V) / hw, pp = v * V - pl * hw;
+#pragma unroll
+            for (int j = 0; j < V; ++j) {
+                run_s[pl * pitch + pp] = static_cast<unsigned short>(__float_as_uint(f[j]) >> 16);
+                if (++pp == hw) { pp = 0; ++pl; }
+            }
+        }
+        __syncthreads();
+        const int n16 = np * pitch / 8;
+        uint4 *dst = reinterpret_cast<uint4 *>(out + pl0 * pitch);
+        for (int i = threadIdx.x; i < n16; i += kThreads) dst[i] = reinterpret_cast<const uint4 *>(run_s)[i];
+        __syncthreads();
+    }
+    unsigned nnz = static_cast<unsigned>(nz);
+    nnz = __reduce_add_sync(kFull, nnz);
+    sat = __reduce_add_sync(kFull, sat);
+    if ((threadIdx.x & 31) == 0 && count) {
+        if (nnz) atomicAdd(&st->nnz, static_cast<unsigned long long>(nnz));
+        if (sat) atomicAdd(&st->saturated, static_cast<unsigned long long>(sat));
+    }
+}
+
 }  // namespace
 
 int launch_quantize_dense(dbp_ctx *ctx, const void *delta, int dtype, long long numel,
                           unsigned long long seed, const float *delta_p, int8_t *dense,
                           void *planes_bf16, long long hw, long long pitch, bool count) {
     const int v = dtype == DBP_F32 ? 4 : 8;
+    // odd plane sizes at a padded pitch: whole runs of planes through shared memory
+    if (planes_bf16 != nullptr && hw > 0 && pitch != hw && (hw & 3) != 0 && numel % hw == 0 && (numel / hw) % 8 == 0 &&
+        8 * pitch * 2 <= kOddMaxSmem && hw < (1 << 20)) {
+        const long long nplanes = numel / hw;
+        int per_run = static_cast<int>(kOddMaxSmem / 2 / pitch / 8 * 8);          // planes per run: a multiple of 8
+        const long long want = (4096 + 8 * hw - 1) / (8 * hw) * 8;               // about 4096 elements a run
+        if (per_run > want) per_run = static_cast<int>(want);
+        long long nruns = (nplanes + per_run - 1) / per_run;
+        long long blocks = nruns < static_cast<long long>(ctx->sm_count) * 8 ? nruns : static_cast<long long>(ctx->sm_count) * 8;
+        cudaError_t e;
+        if (dtype == DBP_F32)
+            e = launch_chained(quantize_planes_odd_kernel<float>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
+                               static_cast<const float *>(delta), nplanes, static_cast<int>(hw), static_cast<int>(pitch), per_run, seed,
+                               delta_p, static_cast<unsigned short *>(planes_bf16), dense, ctx->state, count ? 1 : 0);
+        else
+            e = launch_chained(quantize_planes_odd_kernel<__nv_bfloat16>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
+                               static_cast<const __nv_bfloat16 *>(delta), nplanes, static_cast<int>(hw), static_cast<int>(pitch), per_run,
+                               seed, delta_p, static_cast<unsigned short *>(planes_bf16), dense, ctx->state, count ? 1 : 0);
+        return cuda_ok(e);
+    }
     long long blocks = (numel / v + 2 * kThreads - 1) / (2 * kThreads);
     if (blocks < 1) blocks = 1;
     const long long cap = static_cast<long long>(ctx->sm_count) * kBlocksPerSM;
