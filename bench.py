@@ -445,7 +445,7 @@ def crossover_sweep(torch, dbp, ctx):
 
 # DRAM bytes (read + written) of one config-5 bench step's launches of each kernel kind, from the ncu capture summarised
 # in profiles/bench_step_config5_launch_list.md; None = the kernels of that kind changed after the capture
-NCU_DRAM_BYTES_PER_STEP = {"statistics": 1156897536, "quantize": 1334064128, "dx_dense": 1311867136, "dw_dense": 2630283776}
+NCU_DRAM_BYTES_PER_STEP = {"statistics": 1156103424, "quantize": 1331695616, "dx_dense": 1309135360, "dw_dense": 2629219840}
 
 
 def main():
@@ -751,7 +751,7 @@ def main():
         traffic = None if per_step is None else per_step / n_launch
         roof = {"kernel": {"dx_dense": "tensor-core dX (tma_dx_kernel for 1x1, tc3_tma_dx_kernel for 3x3)",
                            "dw_dense": "tensor-core dW (tma_dw_kernel for 1x1, tc3_tma_dw_kernel + tc3_dw_finish_kernel for 3x3)",
-                           "quantize": "NSD quantizer (quantize_dense_kernel for 1x1, quantize_nhwc_kernel for 3x3)"}.get(top, top + "_kernel"),
+                           "quantize": "NSD quantizer (quantize_dense_kernel / quantize_planes_odd_kernel for 1x1, quantize_nhwc_kernel for 3x3)"}.get(top, top + "_kernel"),
                 "bound": "hbm", "achieved": ach, "peak": hbm_peak, "unit": "GB/s", "frac": ach / hbm_peak,
                 "traffic": traffic, "algorithmic_bytes_per_launch": work[top] / n_launch, "launches_per_step": n_launch,
                 "peak_source": peak_src + " (MEASURED_PEAKS.json hbm_gbs)",
