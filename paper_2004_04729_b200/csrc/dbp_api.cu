@@ -173,7 +173,23 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     const int8_t *codes = nullptr;
     if (mask && io != DBP_F32) return DBP_EUNSUPPORTED;
     // small fp32 layers with one position per image (linear layers): two chained launches
-    const bool mask_vec = mask == nullptr || (reinterpret_cast<uintptr_t>(mask) & 3) == 0;    // masks are read four bytes at a time
+    // Masks are read four bytes at a time where they are folded into a kernel's loads. One that does not start on
+    // a 4-byte boundary is applied by the ReLU-derivative kernel here and now, and the call goes on without it.
+    if (mask != nullptr && (reinterpret_cast<uintptr_t>(mask) & 3) != 0) {
+        const long long n0 = numel;
+        if (ctx->aux_pending) {
+            const int jr = dbp_join(ctx);
+            if (jr) return jr;
+        }
+        const int wr = ws_reserve(ctx, ctx->dz_tmp, static_cast<size_t>(n0) * sizeof(float));
+        if (wr) return wr;
+        KernelTimer t(ctx, DBP_K_GLUE);
+        const int gr = launch_relu_backward(ctx, static_cast<const float *>(delta), mask, static_cast<float *>(ctx->dz_tmp.ptr), n0);
+        if (gr) return gr;
+        delta = ctx->dz_tmp.ptr;
+        mask = nullptr;
+    }
+    const bool mask_vec = true;
     if (io == DBP_F32 && s.k == 1 && s.H == 1 && s.W == 1 && !q_out && (dW || dX) && (!db || dW) && mask_vec &&
         !(flags & (DBP_FORCE_SPARSE | DBP_FORCE_DENSE)) && small_linear_fits(ctx, s.B, s.Cout, s.Cin, dW != nullptr, dX != nullptr)) {
         if (ctx->aux_pending) {

@@ -189,3 +189,31 @@ def test_network_backward_without_delta_z_matches_the_step_by_step_form(ctx, net
     for a, b in zip(ref, got):
         num = (a["dW"] - b["dW"]).norm().item()
         assert num <= 2e-5 * a["dW"].norm().item(), (net, num / a["dW"].norm().item())
+
+
+def test_relu_mask_corner_cases(ctx):
+    """A mask that does not start on a 4-byte boundary takes the form with a separate ReLU-derivative pass (same
+    results); bf16 tensors refuse a mask, and the refused call still consumes it."""
+    import paper_2004_04729_b200 as dbp
+    rng = np.random.default_rng(5)
+    L = wl.linear_layer(40, 24, 56, data_seed=950, scale=2.0, seed=1)
+    mask = (rng.random(L.delta.shape) < 0.5).astype(np.uint8)
+    d, X, W = _cu(L.delta), _cu(L.X), _cu(L.W)
+    store = torch.zeros(mask.size + 1, dtype=torch.uint8, device="cuda")
+    store[1:] = torch.from_numpy(mask.ravel()).cuda()
+    odd = store[1:].view(mask.shape)                     # one byte past an aligned address
+    assert odd.data_ptr() % 4 == 1 and odd.is_contiguous()
+    ctx.set_relu_mask(torch.from_numpy(mask).cuda())
+    ref = dbp.dithered_linear_backward(ctx, d, X, W, L.seed, L.scale)
+    ref_step = ctx.last_step()
+    ctx.set_relu_mask(odd)
+    got = dbp.dithered_linear_backward(ctx, d, X, W, L.seed, L.scale)
+    assert ctx.last_step() == ref_step
+    assert torch.equal(got["dX"], ref["dX"]) and torch.equal(got["dW"], ref["dW"])
+    db16, X16, W16 = (t.to(torch.bfloat16) for t in (d, X, W))
+    ctx.set_relu_mask(odd)
+    with pytest.raises(dbp.DbpError):
+        dbp.dithered_linear_backward(ctx, db16, X16, W16, L.seed, L.scale)
+    out = dbp.dithered_linear_backward(ctx, db16, X16, W16, L.seed, L.scale)     # the mask is gone
+    torch.cuda.synchronize()
+    assert out["dW"].isfinite().all()
