@@ -9,7 +9,8 @@ from .nsd import (splitmix64_at, dither_u, mean_std, step_size, nsd_codes,
                   nsd_codes_literal_f64, nsd_codes_exact_python, derive_layer_seed)
 from .products import (linear_backward, conv_backward, conv_forward,
                        linear_backward_bruteforce, conv_backward_bruteforce,
-                       conv_dW_entry, conv_dX_entry)
+                       conv_dW_entry, conv_dX_entry, strided_out_size, conv_forward_strided,
+                       conv_backward_strided, conv_backward_strided_bruteforce)
 
 from .chain import relu_backward, maxpool2x2_backward, layer_backward, chain_backward
 
@@ -19,4 +20,5 @@ __all__ = [
     "nsd_codes_literal_f64", "nsd_codes_exact_python", "derive_layer_seed",
     "linear_backward", "conv_backward", "conv_forward",
     "linear_backward_bruteforce", "conv_backward_bruteforce", "conv_dW_entry", "conv_dX_entry",
+    "strided_out_size", "conv_forward_strided", "conv_backward_strided", "conv_backward_strided_bruteforce",
 ]

@@ -185,3 +185,94 @@ def conv_dX_entry(codes, Delta, W, b, ci, y, x):
                 tot += float(t.sum())
                 tot_abs += float(np.abs(t).sum())
     return tot, tot_abs
+
+
+# ---- strided convolution (the down-sampling layers of residual networks): the same
+# ---- definitions with the input sampled every `stride` positions,
+#   z[b,co,y,x]      = sum_{ci,ky,kx} W[co,ci,ky,kx] X[b,ci,s*y+ky-p,s*x+kx-p],  p = (k-1)/2,
+#   Ho = (H + 2p - k) // s + 1,  Wo likewise,
+#   dW[co,ci,ky,kx]  = sum_{b,y,x} delta~[b,co,y,x] X[b,ci,s*y+ky-p,s*x+kx-p]
+#   dX[b,ci,y',x']   = sum over the (co,ky,kx,y,x) with s*y+ky-p = y', s*x+kx-p = x' of
+#                      delta~[b,co,y,x] W[co,ci,ky,kx]
+
+def strided_out_size(H, k, stride):
+    return (H + 2 * ((k - 1) // 2) - k) // stride + 1
+
+
+def conv_forward_strided(X, W, stride):
+    X = np.asarray(X, dtype=np.float64)
+    W = np.asarray(W, dtype=np.float64)
+    B, Ci, H, Wd = X.shape
+    Co, _, k, _ = W.shape
+    p, s = (k - 1) // 2, int(stride)
+    Ho, Wo = strided_out_size(H, k, s), strided_out_size(Wd, k, s)
+    Xp = _pad_hw(X, p)
+    z = np.zeros((B, Co, Ho, Wo))
+    for ky in range(k):
+        for kx in range(k):
+            xs = Xp[:, :, ky:ky + s * (Ho - 1) + 1:s, kx:kx + s * (Wo - 1) + 1:s]
+            z += np.einsum("bchw,oc->bohw", xs, W[:, :, ky, kx], optimize=True)
+    return z
+
+
+def conv_backward_strided(codes, Delta, X, W, stride, with_abs=False):
+    """codes [B,Co,Ho,Wo], X [B,Ci,H,W], W [Co,Ci,k,k] -> dict(dW, dX, db) in fp64."""
+    d = _dq(codes, Delta)
+    X = np.asarray(X, dtype=np.float64)
+    W = np.asarray(W, dtype=np.float64)
+    B, Co, Ho, Wo = d.shape
+    _, Ci, H, Wd = X.shape
+    k = W.shape[2]
+    p, s = (k - 1) // 2, int(stride)
+    assert W.shape == (Co, Ci, k, k) and k % 2 == 1
+    assert Ho == strided_out_size(H, k, s) and Wo == strided_out_size(Wd, k, s)
+
+    def both(dd, XX, WW):
+        Xp = _pad_hw(XX, p)
+        dXp = np.zeros_like(Xp)
+        dW = np.zeros((Co, Ci, k, k))
+        for ky in range(k):
+            for kx in range(k):
+                ys = slice(ky, ky + s * (Ho - 1) + 1, s)      # padded rows s*y + ky
+                xs = slice(kx, kx + s * (Wo - 1) + 1, s)
+                dW[:, :, ky, kx] = np.einsum("bohw,bchw->oc", dd, Xp[:, :, ys, xs], optimize=True)
+                dXp[:, :, ys, xs] += np.einsum("bohw,oc->bchw", dd, WW[:, :, ky, kx], optimize=True)
+        return dW, dXp[:, :, p:p + H, p:p + Wd]
+
+    dW, dX = both(d, X, W)
+    out = {"dW": dW, "dX": dX, "db": d.sum(axis=(0, 2, 3))}
+    if with_abs:
+        sW, sX = both(np.abs(d), np.abs(X), np.abs(W))
+        out["S_dW"], out["S_dX"] = sW, sX
+        out["S_db"] = np.abs(d).sum(axis=(0, 2, 3))
+    return out
+
+
+def conv_backward_strided_bruteforce(codes, Delta, X, W, stride):
+    D = float(np.float32(Delta))
+    codes = np.asarray(codes)
+    X = np.asarray(X, dtype=np.float64)
+    W = np.asarray(W, dtype=np.float64)
+    B, Co, Ho, Wo = codes.shape
+    _, Ci, H, Wd = X.shape
+    k = W.shape[2]
+    p, s = (k - 1) // 2, int(stride)
+    dW = np.zeros((Co, Ci, k, k))
+    dX = np.zeros((B, Ci, H, Wd))
+    db = np.zeros(Co)
+    for b in range(B):
+        for co in range(Co):
+            for y in range(Ho):
+                for x in range(Wo):
+                    t = float(codes[b, co, y, x]) * D
+                    if t == 0.0:
+                        continue
+                    db[co] += t
+                    for ci in range(Ci):
+                        for ky in range(k):
+                            for kx in range(k):
+                                yy, xx = s * y + ky - p, s * x + kx - p
+                                if 0 <= yy < H and 0 <= xx < Wd:
+                                    dW[co, ci, ky, kx] += t * X[b, ci, yy, xx]
+                                    dX[b, ci, yy, xx] += t * W[co, ci, ky, kx]
+    return {"dW": dW, "dX": dX, "db": db}
