@@ -37,7 +37,7 @@ typedef enum { DBP_F32 = 0, DBP_BF16 = 1 } dbp_dtype;
 typedef enum {
     DBP_OK = 0,
     DBP_EINVAL = -1,        /* null / misaligned pointer, non-positive size, bad enum */
-    DBP_EUNSUPPORTED = -2,  /* kernel size, stride or padding outside {1x1, 3x3; 1; (k-1)/2} */
+    DBP_EUNSUPPORTED = -2,  /* kernel size, stride or padding outside {1x1, 3x3; 1, 2; (k-1)/2} */
     DBP_ECUDA = -3,         /* a CUDA runtime call failed */
     DBP_ENOMEM = -4,        /* workspace allocation failed */
     DBP_ENONFINITE = -5,    /* device: delta holds NaN or Inf (all codes were set to 0) */
@@ -244,11 +244,18 @@ int dithered_linear_backward(dbp_ctx *ctx, const void *delta, const void *X, con
 
 /*
  * The same for a convolution layer ("analogous for convolutional layers", Section 3):
- * cross-correlation, NCHW, square kernel k in {1, 3}, stride 1, zero padding (k-1)/2.
- * delta [B,Cout,H,W], X [B,Cin,H,W], W [Cout,Cin,k,k]:
+ * cross-correlation, NCHW, square kernel k in {1, 3}, stride 1 or 2, zero padding (k-1)/2.
+ * H and Wd are the height and width of X. Stride 1: delta [B,Cout,H,W], X [B,Cin,H,W], W [Cout,Cin,k,k]:
  *     dX[b,ci,y,x]     = Delta sum_{co,ky,kx} q[b,co,y-ky+p,x-kx+p] W[co,ci,ky,kx]
  *     dW[co,ci,ky,kx]  = Delta sum_{b,y,x}    q[b,co,y,x] X[b,ci,y+ky-p,x+kx-p]
  *     db[co]           = Delta sum_{b,y,x}    q[b,co,y,x]
+ * Stride 2 (the down-sampling layers of residual networks; H and Wd even, else DBP_EUNSUPPORTED):
+ * delta [B,Cout,H/2,W/2] is the gradient at the layer's own output positions, X and dX stay [B,Cin,H,W]:
+ *     dW[co,ci,ky,kx]  = Delta sum_{b,y,x} q[b,co,y,x] X[b,ci,2y+ky-p,2x+kx-p]
+ *     dX[b,ci,y',x']   = Delta sum of q[b,co,y,x] W[co,ci,ky,kx] over the (co,ky,kx,y,x) with 2y+ky-p = y', 2x+kx-p = x'
+ * computed as the stride-1 layer on the four phase images of X (layout kernels on the context's stream around
+ * the same quantizer and product kernels; workspaces of the size of X, dX and 4x the weights). Such a call always
+ * joins its weight-gradient kernels before it returns (DBP_DW_ASYNC is ignored). q_out describes delta as given.
  * Other k, stride or pad return DBP_EUNSUPPORTED.
  */
 int dithered_conv_backward(dbp_ctx *ctx, const void *delta, const void *X, const void *W,

@@ -295,11 +295,14 @@ def dithered_conv_backward(ctx: Context, delta, X, W, seed: int, scale: float, *
                            delta_in=None, q_out: Optional[SparseGradient] = None,
                            need_dW=True, need_dX=True, need_db=False, flags: int = 0,
                            stride: int = 1, pad: Optional[int] = None):
-    """delta [B,Cout,H,W], X [B,Cin,H,W], W [Cout,Cin,k,k] (NCHW) -> dict(dW, dX, db)."""
+    """delta [B,Cout,H/stride,W/stride], X [B,Cin,H,W], W [Cout,Cin,k,k] (NCHW) -> dict(dW, dX, db)."""
     _dev(delta, "delta"), _dev(X, "X"), _dev(W, "W")
-    B, Co, H, Wd = delta.shape
+    B, Co = delta.shape[:2]
     Ci, k = X.shape[1], W.shape[2]
-    assert X.shape == (B, Ci, H, Wd) and W.shape == (Co, Ci, k, k)
+    H, Wd = X.shape[2], X.shape[3]
+    if stride not in (1, 2) or X.shape[0] != B or W.shape != (Co, Ci, k, k) or \
+            (H % stride, Wd % stride) != (0, 0) or tuple(delta.shape[2:]) != (H // stride, Wd // stride):
+        raise ValueError("shapes of delta, X and W do not belong to one layer")
     assert X.dtype == delta.dtype == W.dtype
     pad = (k - 1) // 2 if pad is None else pad
     dev = delta.device
@@ -337,14 +340,17 @@ def dithered_linear_backward_host(ctx: Context, delta, X, W, seed, scale, dW, dX
 
 
 def dithered_conv_backward_host(ctx: Context, delta, X, W, seed, scale, dW, dX, db=None,
-                                flags: int = 0):
+                                flags: int = 0, stride: int = 1):
     for n, t in (("delta", delta), ("X", X), ("W", W), ("dW", dW), ("dX", dX), ("db", db)):
         _host(t, n)
-    B, Co, H, Wd = delta.shape
+    B, Co = delta.shape[:2]
     Ci, k = X.shape[1], W.shape[2]
+    H, Wd = X.shape[2], X.shape[3]
+    if tuple(delta.shape[2:]) != (H // stride, Wd // stride):
+        raise ValueError("shapes of delta and X do not belong to one layer")
     d, nnz = ctypes.c_float(), ctypes.c_longlong()
     _check(load_library().dithered_conv_backward_host(
-        ctx._h, _ptr(delta), _ptr(X), _ptr(W), _dtype_code(delta), B, Ci, Co, H, Wd, k, 1,
+        ctx._h, _ptr(delta), _ptr(X), _ptr(W), _dtype_code(delta), B, Ci, Co, H, Wd, k, int(stride),
         (k - 1) // 2, int(seed) & (2 ** 64 - 1), float(scale), _ptr(dW), _ptr(dX), _ptr(db),
         int(flags), ctypes.byref(d), ctypes.byref(nnz)), "dithered_conv_backward_host")
     return d.value, nnz.value

@@ -375,6 +375,78 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     return DBP_OK;
 }
 
+// A stride-2 layer (k = 1 or 3, pad (k-1)/2, even H and W) as the stride-1 layer on the phase images of X
+// (strided_conv.cu): delta is that layer's own gradient [B][Cout][H/2][W/2] and is quantized as it is; X, W, dX
+// and dW pass through layout kernels on the context's stream. The weight-gradient kernels of such a call are
+// always joined before it returns (the workspaces they read are reused by the next strided call).
+int conv_backward_stride2(dbp_ctx *ctx, const void *delta, const void *X, const void *W, int io, const ConvShape &s,
+                          unsigned long long seed, float scale, const float *delta_in, dbp_sparse *q_out, float *dW,
+                          void *dX, float *db, unsigned flags) {
+    if (!ctx || !delta) return DBP_EINVAL;
+    const uint8_t *mask = ctx->next_mask;
+    ctx->next_mask = nullptr;
+    if (io != DBP_F32 && io != DBP_BF16) return DBP_EINVAL;
+    if (s.B <= 0 || s.Cin <= 0 || s.Cout <= 0 || s.H <= 0 || s.W <= 0 || s.H > 8192 || s.W > 8192) return DBP_EINVAL;
+    if ((s.H & 1) || (s.W & 1)) return DBP_EUNSUPPORTED;
+    if ((dW && !X) || (dX && !W)) return DBP_EINVAL;
+    if (!aligned16(X) || !aligned16(W) || !aligned16(dW) || !aligned16(dX)) return DBP_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return DBP_ECUDA;
+    const int phases = s.k == 1 ? 1 : 4;
+    const int Ho = static_cast<int>(s.H / 2), Wo = static_cast<int>(s.W / 2);
+    const ConvShape in{s.B, s.Cin * phases, s.Cout, Ho, Wo, s.k};
+    const size_t es = elem_size(io);
+    const bool dx_f32 = io == DBP_F32 || (flags & DBP_DX_F32);
+    const size_t nxp = static_cast<size_t>(in.B) * in.Cin * Ho * Wo, nwp = static_cast<size_t>(in.Cout) * in.Cin * s.k * s.k;
+    int rc;
+    if (dW && (rc = ws_reserve(ctx, ctx->s2_x, nxp * es))) return rc;
+    if (dX && (rc = ws_reserve(ctx, ctx->s2_dx, nxp * (dx_f32 ? 4 : 2)))) return rc;
+    if (dX && s.k == 3 && (rc = ws_reserve(ctx, ctx->s2_w, nwp * es))) return rc;
+    if (dW && s.k == 3 && (rc = ws_reserve(ctx, ctx->s2_dw, nwp * sizeof(float)))) return rc;
+    // a *_host call: X is still on its way up on another stream, and dX is read back after an event
+    cudaEvent_t after_dx = ctx->hook_after_dx;
+    ctx->hook_after_dx = nullptr;
+    if (dW) {
+        if (ctx->hook_before_dw && cudaStreamWaitEvent(ctx->stream, ctx->hook_before_dw, 0) != cudaSuccess) return DBP_ECUDA;
+        ctx->hook_before_dw = nullptr;
+        KernelTimer t(ctx, DBP_K_GLUE);
+        if ((rc = launch_phases_of(ctx, X, ctx->s2_x.ptr, io, s.B, s.Cin, static_cast<int>(s.H), static_cast<int>(s.W), phases))) return rc;
+    }
+    if (dX && s.k == 3) {
+        KernelTimer t(ctx, DBP_K_GLUE);
+        if ((rc = launch_phase_weights(ctx, W, ctx->s2_w.ptr, io, s.Cout, s.Cin))) return rc;
+    }
+    ctx->next_mask = mask;
+    rc = conv_backward_impl(ctx, delta, dW ? ctx->s2_x.ptr : nullptr, dX ? (s.k == 3 ? ctx->s2_w.ptr : W) : nullptr, io, in,
+                            seed, scale, delta_in, q_out,
+                            dW ? (s.k == 3 ? static_cast<float *>(ctx->s2_dw.ptr) : dW) : nullptr,
+                            dX ? ctx->s2_dx.ptr : nullptr, db, flags & ~DBP_DW_ASYNC);
+    if (rc) return rc;
+    if (dX) {
+        KernelTimer t(ctx, DBP_K_GLUE);
+        if ((rc = launch_from_phases(ctx, ctx->s2_dx.ptr, dX, dx_f32 ? 1 : 0, s.B, s.Cin, static_cast<int>(s.H),
+                                     static_cast<int>(s.W), phases)))
+            return rc;
+        if (after_dx && cudaEventRecord(after_dx, ctx->stream) != cudaSuccess) return DBP_ECUDA;
+    }
+    if (dW && s.k == 3) {
+        KernelTimer t(ctx, DBP_K_GLUE);
+        if ((rc = launch_strided_dw(ctx, static_cast<const float *>(ctx->s2_dw.ptr), dW, s.Cout, s.Cin))) return rc;
+    }
+    return DBP_OK;
+}
+
+bool conv_form_supported(int k, int stride, int pad) {
+    return (k == 1 || k == 3) && (stride == 1 || stride == 2) && pad == (k - 1) / 2;
+}
+
+int conv_backward_any(dbp_ctx *ctx, const void *delta, const void *X, const void *W, int io, const ConvShape &s,
+                      int stride, unsigned long long seed, float scale, const float *delta_in, dbp_sparse *q_out,
+                      float *dW, void *dX, float *db, unsigned flags) {
+    return stride == 2 ? conv_backward_stride2(ctx, delta, X, W, io, s, seed, scale, delta_in, q_out, dW, dX, db, flags)
+                       : conv_backward_impl(ctx, delta, X, W, io, s, seed, scale, delta_in, q_out, dW, dX, db, flags);
+}
+
 }  // namespace
 }  // namespace dbp
 
@@ -460,7 +532,7 @@ int dbp_destroy(dbp_ctx *ctx) {
     cudaStreamSynchronize(ctx->stream);
     if (ctx->aux) cudaStreamSynchronize(ctx->aux);
     Workspace *all[] = {&ctx->dense_codes[0], &ctx->dense_codes[1], &ctx->codes16[0], &ctx->codes16[1],
-                        &ctx->codes_nhwc[0], &ctx->codes_nhwc[1], &ctx->codes_stack[0], &ctx->codes_stack[1], &ctx->dz_tmp, &ctx->dw_acc, &ctx->x_padded, &ctx->w_taps, &ctx->sp_bitmap, &ctx->sp_offsets, &ctx->sp_values,
+                        &ctx->codes_nhwc[0], &ctx->codes_nhwc[1], &ctx->codes_stack[0], &ctx->codes_stack[1], &ctx->dz_tmp, &ctx->s2_x, &ctx->s2_w, &ctx->s2_dx, &ctx->s2_dw, &ctx->dw_acc, &ctx->x_padded, &ctx->w_taps, &ctx->sp_bitmap, &ctx->sp_offsets, &ctx->sp_values,
                         &ctx->tc_partials};
     for (Workspace *w : all) if (w->ptr) cudaFree(w->ptr);
     for (Workspace &w : ctx->io) if (w.ptr) cudaFree(w.ptr);
@@ -656,14 +728,14 @@ int dithered_conv_backward(dbp_ctx *ctx, const void *delta, const void *X, const
                            int stride, int pad, unsigned long long seed, float scale,
                            const float *delta_in, dbp_sparse *q_out, float *dW, void *dX, float *db,
                            unsigned flags) {
-    if ((k != 1 && k != 3) || stride != 1 || pad != (k - 1) / 2) return DBP_EUNSUPPORTED;
+    if (!conv_form_supported(k, stride, pad)) return DBP_EUNSUPPORTED;
     ConvShape s{B, Cin, Cout, H, Wd, k};
-    return conv_backward_impl(ctx, delta, X, W, io, s, seed, scale, delta_in, q_out, dW, dX, db, flags);
+    return conv_backward_any(ctx, delta, X, W, io, s, stride, seed, scale, delta_in, q_out, dW, dX, db, flags);
 }
 
 static int host_backward(dbp_ctx *ctx, const void *delta, const void *X, const void *W, int io,
                          const ConvShape &s, unsigned long long seed, float scale, float *dW, void *dX,
-                         float *db, unsigned flags, float *delta_out, long long *nnz_out) {
+                         float *db, unsigned flags, float *delta_out, long long *nnz_out, int stride = 1) {
     if (!ctx || !delta) return DBP_EINVAL;
     if (io != DBP_F32 && io != DBP_BF16) return DBP_EINVAL;
     if (s.B <= 0 || s.Cin <= 0 || s.Cout <= 0 || s.H <= 0 || s.W <= 0) return DBP_EINVAL;
@@ -671,7 +743,7 @@ static int host_backward(dbp_ctx *ctx, const void *delta, const void *X, const v
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return DBP_ECUDA;
     const size_t es = elem_size(io);
-    const size_t nd = static_cast<size_t>(s.B) * s.Cout * s.H * s.W;
+    const size_t nd = static_cast<size_t>(s.B) * s.Cout * (s.H / stride) * (s.W / stride);   // delta: the layer's output positions
     const size_t nx = static_cast<size_t>(s.B) * s.Cin * s.H * s.W;
     const size_t nw = static_cast<size_t>(s.Cout) * s.Cin * s.k * s.k;
     const size_t dx_es = (io == DBP_BF16 && !(flags & DBP_DX_F32)) ? 2 : 4;
@@ -701,7 +773,7 @@ static int host_backward(dbp_ctx *ctx, const void *delta, const void *X, const v
         ctx->hook_before_dw = ctx->ev_x_up;
     }
     if (dX) ctx->hook_after_dx = ctx->ev_dx_done;
-    rc = conv_backward_impl(ctx, ctx->io[0].ptr, X ? ctx->io[1].ptr : nullptr, W ? ctx->io[2].ptr : nullptr, io, s,
+    rc = conv_backward_any(ctx, ctx->io[0].ptr, X ? ctx->io[1].ptr : nullptr, W ? ctx->io[2].ptr : nullptr, io, s, stride,
                             seed, scale, nullptr, nullptr, dW ? static_cast<float *>(ctx->io[3].ptr) : nullptr,
                             dX ? ctx->io[4].ptr : nullptr, db ? static_cast<float *>(ctx->io[5].ptr) : nullptr,
                             flags & ~DBP_DW_ASYNC);      // the results are copied back right away
@@ -740,10 +812,11 @@ int dithered_conv_backward_host(dbp_ctx *ctx, const void *delta, const void *X, 
                                 int k, int stride, int pad, unsigned long long seed, float scale,
                                 float *dW, void *dX, float *db, unsigned flags, float *delta_out,
                                 long long *nnz_out) {
-    if ((k != 1 && k != 3) || stride != 1 || pad != (k - 1) / 2) return DBP_EUNSUPPORTED;
+    if (!conv_form_supported(k, stride, pad)) return DBP_EUNSUPPORTED;
+    if (stride == 2 && ((H & 1) || (Wd & 1))) return DBP_EUNSUPPORTED;
     if (!(scale > 0.f)) return DBP_EINVAL;
     ConvShape s{B, Cin, Cout, H, Wd, k};
-    return host_backward(ctx, delta, X, W, io, s, seed, scale, dW, dX, db, flags, delta_out, nnz_out);
+    return host_backward(ctx, delta, X, W, io, s, seed, scale, dW, dX, db, flags, delta_out, nnz_out, stride);
 }
 
 int dbp_set_relu_mask(dbp_ctx *ctx, const uint8_t *mask) {

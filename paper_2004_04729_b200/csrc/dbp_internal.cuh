@@ -56,6 +56,7 @@ struct dbp_ctx {
     const uint8_t *next_mask = nullptr; // ReLU mask for the next backward call (dbp_set_relu_mask)
     dbp::Workspace dz_tmp;              // delta_z = delta_a (.) mask when that call cannot fold the mask into its loads
     dbp::Workspace codes_stack[2];      // the same codes with G images stacked into one tall image (tiny planes, dW)
+    dbp::Workspace s2_x, s2_w, s2_dx, s2_dw;   // stride-2 layers: phase images of X, phase weights, and the two products in that layout
     float *delta_sets = nullptr;        // device float[2]: the step size that belongs to each set
     int code_set = 0;                   // the set the next call writes
     cudaEvent_t ev_set_free[2] = {nullptr, nullptr};   // recorded on the dW stream after the set's last reader
@@ -191,6 +192,13 @@ int launch_relu_backward(dbp_ctx *ctx, const float *da, const uint8_t *mask, flo
                          long long n);
 int launch_maxpool_backward(dbp_ctx *ctx, const float *g, const int8_t *argmax, float *out,
                             long long planes, long long h, long long w);
+
+// ---- strided_conv.cu: layout changes around a stride-2 layer run as a stride-1 layer on the input's phase images
+// (phases = 4: all four, channel (py*2+px)*Cin + ci; phases = 1: the even rows and columns only)
+int launch_phases_of(dbp_ctx *ctx, const void *X, void *Xp, int io, long long B, long long Cin, int H, int W, int phases);
+int launch_from_phases(dbp_ctx *ctx, const void *dXp, void *dX, int f32, long long B, long long Cin, int H, int W, int phases);
+int launch_phase_weights(dbp_ctx *ctx, const void *W, void *Wp, int io, long long Cout, long long Cin);
+int launch_strided_dw(dbp_ctx *ctx, const float *dWp, float *dW, long long Cout, long long Cin);
 
 // ---- selftest.cu
 int launch_bounded_wait_selftest(dbp_ctx *ctx, long long budget);

@@ -76,7 +76,7 @@ def round_to_bf16(a) -> np.ndarray:
 @dataclass
 class Layer:
     """One layer's backward inputs. kind 'linear': delta [B,N], X [B,K], W [N,K].
-    kind 'conv': delta [B,Cout,H,W], X [B,Cin,H,W], W [Cout,Cin,k,k] (NCHW, stride 1,
+    kind 'conv': delta [B,Cout,H/stride,W/stride], X [B,Cin,H,W], W [Cout,Cin,k,k] (NCHW,
     pad (k-1)/2). Arrays are fp32; with dtype 'bf16' their values are bf16-representable."""
     name: str
     kind: str
@@ -87,6 +87,7 @@ class Layer:
     seed: int = 0
     dtype: str = "f32"
     k: int = 1
+    stride: int = 1
 
     @property
     def dense_flops(self) -> float:
@@ -113,16 +114,18 @@ def linear_layer(B, N, K, *, data_seed, b_laplace=1e-3, keep=0.5, scale=2.0, see
 
 
 def conv_layer(B, Cin, Cout, H, Wd, k, *, data_seed, b_laplace=1e-4, keep=0.5, scale=2.0,
-               seed=0, dtype="f32", name=None) -> Layer:
+               seed=0, dtype="f32", name=None, stride=1) -> Layer:
     nX = B * Cin * H * Wd
     X = np.maximum(normal(data_seed, 1, nX), 0.0).reshape(B, Cin, H, Wd)   # post-ReLU
     W = normal(data_seed, 2, Cout * Cin * k * k, sigma=(2.0 / (Cin * k * k)) ** 0.5)
     W = W.reshape(Cout, Cin, k, k)                                          # He init
-    nd = B * Cout * H * Wd
+    Ho, Wo = H // stride, Wd // stride                                      # even H, W for stride 2
+    nd = B * Cout * Ho * Wo
     d = laplace(data_seed, 3, nd, b=b_laplace) * bernoulli(data_seed, 4, nd, keep)
-    return Layer(name or f"conv{k}x{k}_B{B}_{Cin}to{Cout}_{H}x{Wd}", "conv",
-                 _cast(d.reshape(B, Cout, H, Wd), dtype), _cast(X, dtype), _cast(W, dtype),
-                 scale, seed, dtype, k)
+    tag = f"_s{stride}" if stride != 1 else ""
+    return Layer(name or f"conv{k}x{k}{tag}_B{B}_{Cin}to{Cout}_{H}x{Wd}", "conv",
+                 _cast(d.reshape(B, Cout, Ho, Wo), dtype), _cast(X, dtype), _cast(W, dtype),
+                 scale, seed, dtype, k, stride)
 
 
 def config1(batch=128) -> Layer:
@@ -151,6 +154,21 @@ RESNET50_SET = [
     ("s4_reduce_first", 1024, 512, 14, 1, 1), ("s4_reduce", 2048, 512, 7, 1, 2),
     ("s4_conv3x3", 512, 512, 7, 3, 3), ("s4_expand", 512, 2048, 7, 1, 3),
 ]
+
+
+# The stride-2 layers of the same network (torchvision's placement: the stride sits on the 3x3 layer of a
+# stage's first block and on its 1x1 shortcut projection): (name, Cin, Cout, input HW, k).
+RESNET50_STRIDED = [
+    ("s2_conv3x3_down", 128, 128, 56, 3), ("s2_shortcut", 256, 512, 56, 1),
+    ("s3_conv3x3_down", 256, 256, 28, 3), ("s3_shortcut", 512, 1024, 28, 1),
+    ("s4_conv3x3_down", 512, 512, 14, 3), ("s4_shortcut", 1024, 2048, 14, 1),
+]
+
+
+def resnet50_strided_layer(idx, batch=64, scale=5.0, dtype="bf16") -> Layer:
+    name, ci, co, hw, k = RESNET50_STRIDED[idx]
+    return conv_layer(batch, ci, co, hw, hw, k, data_seed=2005 + 16 * idx, b_laplace=1e-4,
+                      scale=scale, dtype=dtype, name=name, stride=2)
 
 
 def config5_layer(idx, batch=64, scale=5.0, dtype="bf16") -> Layer:
