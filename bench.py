@@ -342,6 +342,54 @@ def per_shape_table(torch, layers, run_layer, ctx, dq, hbm_peak, no_dense):
     return rows
 
 
+def strided_table(torch, dbp, ctx, hbm_peak, no_dense, batch):
+    """The stride-2 layers of the same network (a side measurement, not part of the step): time per layer of the
+    whole backward through the library's stride-2 form, the dense library's strided backward on the dequantized
+    gradient, and the layer's algorithmic bytes against the measured bandwidth. Two instances of each shape on
+    their own buffers, run in turn."""
+    dev = torch.device("cuda", ctx.device)
+    torch.backends.cudnn.benchmark = True
+    torch.backends.cudnn.allow_tf32 = False
+    torch.backends.cuda.matmul.allow_tf32 = False
+    rows = []
+    for idx in range(len(wl.RESNET50_STRIDED)):
+        L = wl.resnet50_strided_layer(idx, batch=batch)
+        sets = []
+        for _ in range(2):
+            d, X, W = (torch.from_numpy(a).to(dev).to(torch.bfloat16) for a in (L.delta, L.X, L.W))
+            sets.append((d, X, W))
+        def ours():
+            for d, X, W in sets:
+                dbp.dithered_conv_backward(ctx, d, X, W, L.seed, L.scale, stride=2)
+        for _ in range(3):
+            ours()
+        torch.cuda.synchronize()
+        ms = time_events(torch, ours, 10) / len(sets)
+        q = dbp.nsd_quantize(ctx, sets[0][0], L.seed, L.scale)
+        row = {"shape": L.name, "k": L.k, "ms": ms, "algorithmic_mb": algorithmic_bytes(L) / 1e6,
+               "frac_of_measured_hbm": algorithmic_bytes(L) / (ms * 1e-3) / 1e9 / hbm_peak,
+               "tflops_dense_equiv": L.dense_flops / (ms * 1e-3) / 1e12, "nsd_density": q.nnz.item() / sets[0][0].numel()}
+        if not no_dense:
+            p = (L.k - 1) // 2
+            fns = []
+            for d, X, W in sets:
+                g = (dbp.nsd_decode_dense(ctx, dbp.nsd_quantize(ctx, d, L.seed, L.scale), d.shape).float() * q.delta).to(d.dtype).contiguous()
+                fns.append(lambda g=g, X=X, W=W: torch.ops.aten.convolution_backward(
+                    g, X, W, None, [2, 2], [p, p], [1, 1], False, [0, 0], 1, [True, True, False]))
+            def dense():
+                for f in fns:
+                    f()
+            for _ in range(3):
+                dense()
+            torch.cuda.synchronize()
+            row["dense_ms"] = time_events(torch, dense, 10) / len(sets)
+            del fns
+        rows.append(row)
+        del sets
+        torch.cuda.empty_cache()
+    return rows
+
+
 def tensor_peak():
     """Measured dense bf16 rate (TFLOP/s, burst) and where it comes from."""
     try:
@@ -788,6 +836,7 @@ def main():
     if not args.no_others and world == 1 and args.config == 5 and not (args.only or args.single):
         out["other_configs"] = {str(c): small_config(torch, dbp, ctx, c, hbm_peak, fma_peak) for c in (1, 2, 3, 4)}
         out["per_shape"] = per_shape_table(torch, layers, run_layer, ctx, dq_by_layer, hbm_peak, args.no_dense)
+        out["strided_layers"] = strided_table(torch, dbp, ctx, hbm_peak, args.no_dense, layers[0][0].delta.shape[0])
     if not args.no_cpu and world == 1:
         v, dt, what, cores = oracle_sample(args.config)
         out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what,

@@ -417,10 +417,12 @@ int conv_backward_stride2(dbp_ctx *ctx, const void *delta, const void *X, const 
         if ((rc = launch_phase_weights(ctx, W, ctx->s2_w.ptr, io, s.Cout, s.Cin))) return rc;
     }
     ctx->next_mask = mask;
+    ctx->phase_cin = s.k == 3 ? static_cast<int>(s.Cin) : 0;      // the 3x3 tensor-core kernels skip the taps that are zero by construction
     rc = conv_backward_impl(ctx, delta, dW ? ctx->s2_x.ptr : nullptr, dX ? (s.k == 3 ? ctx->s2_w.ptr : W) : nullptr, io, in,
                             seed, scale, delta_in, q_out,
                             dW ? (s.k == 3 ? static_cast<float *>(ctx->s2_dw.ptr) : dW) : nullptr,
                             dX ? ctx->s2_dx.ptr : nullptr, db, flags & ~DBP_DW_ASYNC);
+    ctx->phase_cin = 0;
     if (rc) return rc;
     if (dX) {
         KernelTimer t(ctx, DBP_K_GLUE);

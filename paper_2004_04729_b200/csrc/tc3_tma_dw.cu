@@ -49,6 +49,10 @@ struct Dw3T {
     int panel_bytes;              // multiple of 1024
     int nx;                       // activation slots in flight
     int stage_chunks;             // 32-column chunks of the accumulators that fit the shared memory at once
+    int phase_tiles;              // > 0: a stride-2 layer on phase images, this many 128-channel tiles per phase (phase
+                                  // ph = 2 py + px holds channels ph * 128 * phase_tiles ...). Only the taps with
+                                  // ky in {1} (py = 0) or {0, 1} (py = 1), kx likewise, are wanted: the work items of
+                                  // the other kernel columns do not exist and the other rows' MMAs are left out
     int *err_flag;
     unsigned long long *stats;    // wait counters (may be null)
 };
@@ -75,10 +79,26 @@ tc3_tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     // work item: (output tile, kernel column, range of segments)
     const int split = blockIdx.x % p.nsplit;
     int rest = blockIdx.x / p.nsplit;
-    const int kx = rest % 3;
-    rest /= 3;
-    const int ci0 = (rest % p.ci_tiles) * 128;
-    const int co0 = (rest / p.ci_tiles) * 64 * NP;
+    int kx, ci_t, co_t, live_lo = 0, live_hi = 3;       // rows ky in [live_lo, live_hi) are accumulated (NP == 2)
+    if (p.phase_tiles > 0) {
+        // per output-channel tile: the phases in order, one kernel column (kx = 1) per channel tile of a phase with
+        // px = 0, two (kx = 0, 1) with px = 1
+        const int tp = p.phase_tiles, per_co = 6 * tp;
+        co_t = rest / per_co;
+        int r = rest - co_t * per_co;
+        const int py = r / (3 * tp);
+        r -= py * 3 * tp;
+        if (r < tp) { ci_t = 2 * py * tp + r; kx = 1; }
+        else { r -= tp; ci_t = (2 * py + 1) * tp + (r >> 1); kx = r & 1; }
+        if (NP == 2) { live_lo = py ? 0 : 1; live_hi = 2; }
+    } else {
+        kx = rest % 3;
+        rest /= 3;
+        ci_t = rest % p.ci_tiles;
+        co_t = rest / p.ci_tiles;
+    }
+    const int ci0 = ci_t * 128;
+    const int co0 = co_t * 64 * NP;
     const long long g0 = split * p.per_split;
     const long long g1 = g0 + p.per_split < p.nseg ? g0 + p.per_split : p.nseg;
     const int halo = p.W + 1;
@@ -208,9 +228,9 @@ tc3_tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     for (int kk = 0; kk < nk; ++kk) {
                         const unsigned adv = radv + kk * 128;                 // 16 rows = 2048 bytes
                         if (NP == 2) {
-                            mma_bf16(tmem_base, ad + 2 * kk, bA + adv, idesc128, acc_on);
+                            if (live_lo == 0) mma_bf16(tmem_base, ad + 2 * kk, bA + adv, idesc128, acc_on);
                             mma_bf16(tmem_base + 128, ad + 2 * kk, bB + adv, idesc128, acc_on);
-                            mma_bf16(tmem_base + 256, ad + 2 * kk, bC + adv, idesc128, acc_on);
+                            if (live_hi == 3) mma_bf16(tmem_base + 256, ad + 2 * kk, bC + adv, idesc128, acc_on);
                         } else {
                             mma_bf16(tmem_base, ad + 2 * kk, bA + adv, idesc192, acc_on);
                         }
@@ -282,9 +302,10 @@ tc3_tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         if (ok) {
             tc_fence_after();
             const long long t_epi = clock64();
-            constexpr int nchunks = (NP == 2 ? 384 : 192) / 32;
+            // NP == 2: four chunks per row ky, only the accumulated rows are handed over
+            const int nchunks = NP == 2 ? 4 * live_hi : 192 / 32;
             float *stg = reinterpret_cast<float *>(smem);
-            for (int c0 = 0; c0 < nchunks; c0 += p.stage_chunks) {
+            for (int c0 = NP == 2 ? 4 * live_lo : 0; c0 < nchunks; c0 += p.stage_chunks) {
                 const int nb = nchunks - c0 < p.stage_chunks ? nchunks - c0 : p.stage_chunks;
                 for (int i = 0; i < nb; ++i) {
                     unsigned v[32];
@@ -498,7 +519,12 @@ int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, int i
     p.segs_per_img = (p.HW + p.SEG - 1) / p.SEG;
     p.code_batch = static_cast<int>(s.B);
     p.nseg = s.B * pieces * p.segs_per_img;
-    const long long tiles = static_cast<long long>(p.ci_tiles) * p.co_tiles * 3;
+    // a stride-2 layer on phase images whose phases are whole channel tiles: 6 of the 12 (phase, kernel column)
+    // pairs carry taps of the strided layer
+    p.phase_tiles = (ctx->phase_cin > 0 && ctx->phase_cin % 128 == 0 && cin_pad == 4ll * ctx->phase_cin && stack_g == 0)
+                        ? ctx->phase_cin / 128 : 0;
+    const long long tiles = p.phase_tiles > 0 ? static_cast<long long>(p.co_tiles) * 6 * p.phase_tiles
+                                              : static_cast<long long>(p.ci_tiles) * p.co_tiles * 3;
     const long long nsplit = choose_split(tiles, p.nseg, ctx->sm_count, &p.per_split);
     p.nsplit = static_cast<int>(nsplit);
     if (tiles * nsplit >= (1ll << 31)) return DBP_EUNSUPPORTED;

@@ -62,6 +62,9 @@ struct Dx3T {
     int run;                      // Ht * W: staged positions per image
     int pitch;                    // bytes per channel row of the staging block (an odd number of words)
     int pairs;                    // W even: columns are staged two at a time
+    int phase_cin;                // > 0: the layer is a stride-2 layer on phase images (channel block ph * phase_cin ...
+                                  // holds phase ph = 2 py + px); a phase's weights are zero outside the taps
+                                  // ky in {1} (py = 0) or {0, 1} (py = 1), kx likewise, and those taps are skipped
     int *err_flag;
     unsigned long long *stats;    // wait counters (may be null)
 };
@@ -208,6 +211,12 @@ tc3_tma_dx_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tc_fence_after();
                 const unsigned tmem_d = tmem_base + slot * kAccCols;
                 unsigned acc_on = 0u;
+                int live_y = 7, live_x = 7;                // bit t: taps with coordinate t carry non-zero weights
+                if (p.phase_cin > 0) {
+                    const int ph = static_cast<int>(t % p.ci_tiles) * 128 / p.phase_cin;
+                    live_y = (ph & 2) ? 3 : 2;
+                    live_x = (ph & 1) ? 3 : 2;
+                }
                 if (p.resident) { ws = 0; wpar = 0; }      // completed barriers stay passable on parity 0
                 for (int c = 0; c < p.ncb && ok; ++c) {
                     ok = __all_sync(0xffffffffu, mbar_wait_timed(&pipe.q_full[qs], qpar, p.err_flag, wq));
@@ -224,6 +233,7 @@ tc3_tma_dx_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         unsigned long long ad = make_desc(smem_u32(w_s + ws * p.w_slot), p.a_panels == 2 ? kWPanel : 0, 1024);
                         for (int gg = 0; gg < p.G; ++gg, ad += a_tap) {
                             const unsigned long long bd = bd0 + static_cast<unsigned>(toff);
+                            const bool live = ((live_y >> ky) & 1) && ((live_x >> kx) & 1);
                             if (kx == 2) {
                                 kx = 0;
                                 toff += tap_wrap;
@@ -232,6 +242,7 @@ tc3_tma_dx_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                                 ++kx;
                                 toff -= 8;
                             }
+                            if (!live) continue;
                             if (elect_one()) {
 #pragma unroll
                                 for (int k = 0; k < 4; ++k)   // 16 co: 16 rows of A (2048 bytes), 32 bytes along a row of B
@@ -412,6 +423,7 @@ int launch_tc3_tma_dx(dbp_ctx *ctx, const void *codes_nhwc, const void *W, int i
     p.H = static_cast<int>(s.H); p.W = static_cast<int>(s.W); p.Wp = p.W + 2;
     p.err_flag = err_flag;
     p.stats = ctx->wait_stats;
+    p.phase_cin = (ctx->phase_cin > 0 && ctx->phase_cin % 128 == 0 && s.Cin == 4ll * ctx->phase_cin) ? ctx->phase_cin : 0;
     p.ncb = (p.Cout + 63) / 64;
     p.ci_tiles = (p.Cin + 127) / 128;
     p.a_panels = p.Cin <= 64 ? 1 : 2;

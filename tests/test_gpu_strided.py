@@ -59,6 +59,8 @@ def _run(ctx, L, tol, flags=0):
     (1, 128, 128, 56, 56, 3),    # ResNet stage-2 down-sampling 3x3
     (2, 256, 256, 28, 28, 3),
     (2, 512, 512, 14, 14, 3),    # 7x7 outputs
+    (2, 128, 64, 20, 20, 3),     # whole channel tiles per phase, one 64-channel code panel
+    (3, 384, 192, 8, 12, 3),     # three channel tiles per phase, ragged output-channel tile
     (2, 3, 8, 10, 6, 3),         # 12 phase channels: off the tensor-core kernels
     (2, 64, 128, 16, 16, 1),
     (1, 256, 512, 56, 56, 1),    # ResNet stage-2 shortcut projection
@@ -75,6 +77,9 @@ def test_stride2_bf16(ctx, B, Ci, Co, H, W, k):
     (2, 16, 16, 8, 8, 3),
     (2, 64, 64, 32, 32, 3),
     (3, 24, 40, 12, 20, 3),
+    (2, 128, 64, 16, 16, 3),     # whole channel tiles per phase (the kernels skip the taps that are zero by construction)
+    (1, 128, 128, 24, 24, 3),
+    (4, 128, 128, 8, 8, 3),      # 4x4 outputs: images stacked for the weight gradient
     (2, 3, 8, 10, 6, 3),
     (2, 64, 128, 16, 16, 1),
     (2, 20, 12, 6, 10, 1),
