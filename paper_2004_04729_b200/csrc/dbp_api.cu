@@ -418,11 +418,14 @@ int conv_backward_stride2(dbp_ctx *ctx, const void *delta, const void *X, const 
     }
     ctx->next_mask = mask;
     ctx->phase_cin = s.k == 3 ? static_cast<int>(s.Cin) : 0;      // the 3x3 tensor-core kernels skip the taps that are zero by construction
+    ctx->phase_dw_out = (s.k == 3 && dW) ? dW : nullptr;
+    ctx->phase_dw_done = false;
     rc = conv_backward_impl(ctx, delta, dW ? ctx->s2_x.ptr : nullptr, dX ? (s.k == 3 ? ctx->s2_w.ptr : W) : nullptr, io, in,
                             seed, scale, delta_in, q_out,
                             dW ? (s.k == 3 ? static_cast<float *>(ctx->s2_dw.ptr) : dW) : nullptr,
                             dX ? ctx->s2_dx.ptr : nullptr, db, flags & ~DBP_DW_ASYNC);
     ctx->phase_cin = 0;
+    ctx->phase_dw_out = nullptr;
     if (rc) return rc;
     if (dX) {
         KernelTimer t(ctx, DBP_K_GLUE);
@@ -431,7 +434,7 @@ int conv_backward_stride2(dbp_ctx *ctx, const void *delta, const void *X, const 
             return rc;
         if (after_dx && cudaEventRecord(after_dx, ctx->stream) != cudaSuccess) return DBP_ECUDA;
     }
-    if (dW && s.k == 3) {
+    if (dW && s.k == 3 && !ctx->phase_dw_done) {
         KernelTimer t(ctx, DBP_K_GLUE);
         if ((rc = launch_strided_dw(ctx, static_cast<const float *>(ctx->s2_dw.ptr), dW, s.Cout, s.Cin))) return rc;
     }

@@ -56,6 +56,8 @@ struct dbp_ctx {
     const uint8_t *next_mask = nullptr; // ReLU mask for the next backward call (dbp_set_relu_mask)
     dbp::Workspace dz_tmp;              // delta_z = delta_a (.) mask when that call cannot fold the mask into its loads
     dbp::Workspace codes_stack[2];      // the same codes with G images stacked into one tall image (tiny planes, dW)
+    float *phase_dw_out = nullptr;      // that layer's dW: the 3x3 weight-gradient kernels write it directly when they run in phase mode ...
+    bool phase_dw_done = false;         // ... and say so here
     int phase_cin = 0;                  // > 0 while a stride-2 3x3 layer runs as a stride-1 layer on phase images: its own channel count
     dbp::Workspace s2_x, s2_w, s2_dx, s2_dw;   // stride-2 layers: phase images of X, phase weights, and the two products in that layout
     float *delta_sets = nullptr;        // device float[2]: the step size that belongs to each set

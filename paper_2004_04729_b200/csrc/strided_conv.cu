@@ -26,60 +26,84 @@ inline int blocks_of(long long n, int threads, int cap) {
     return static_cast<int>(b < cap ? b : cap);
 }
 
-template <typename T> struct Pair;
-template <> struct Pair<float> { using type = float2; };
-template <> struct Pair<__nv_bfloat16> { using type = __nv_bfloat162; };
+// NP pairs of neighbouring columns as one vector
+template <typename T, int NP> struct Cols;
+template <> struct Cols<float, 1> { using vec = float2; using half = float; };
+template <> struct Cols<float, 2> { using vec = float4; using half = float2; };
+template <> struct Cols<__nv_bfloat16, 1> { using vec = unsigned; using half = unsigned short; };
+template <> struct Cols<__nv_bfloat16, 2> { using vec = uint2; using half = unsigned; };
 
-// X [planes][H][W] -> X' [b][phase][ci][H/2][W/2], one thread per pair of neighbouring input columns (an aligned
-// 2-element load; W is even). phases = 1 keeps the (0,0) phase only.
-template <typename T>
-__global__ void __launch_bounds__(256) phases_of_kernel(const T *__restrict__ X, T *__restrict__ Xp, long long B,
-                                                        long long Cin, int H, int W, int phases) {
-    using P = typename Pair<T>::type;
-    const int Ho = H / 2, Wo = W / 2;
-    const long long rows = phases == 1 ? Ho : H;                  // input rows visited per plane
-    const long long n = B * Cin * rows * Wo;
-    for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += gridDim.x * 256ll) {
-        const int xo = static_cast<int>(i % Wo);
-        const long long r = i / Wo;
-        const int yr = static_cast<int>(r % rows);
-        const long long plane = r / rows;                         // b * Cin + ci
-        const long long b = plane / Cin, ci = plane - b * Cin;
-        const int y = phases == 1 ? 2 * yr : yr;
-        const int py = y & 1, yo = y >> 1;
-        const P v = *reinterpret_cast<const P *>(X + (plane * H + y) * W + 2 * xo);
-        const long long o0 = (((b * phases + (phases == 1 ? 0 : py * 2)) * Cin + ci) * Ho + yo) * Wo + xo;
-        Xp[o0] = v.x;
-        if (phases != 1) Xp[o0 + Cin * Ho * Wo] = v.y;
+// even-numbered and odd-numbered elements of a vector of 2 NP columns
+__device__ __forceinline__ void split_cols(const float2 v, float &e, float &o) { e = v.x; o = v.y; }
+__device__ __forceinline__ void split_cols(const float4 v, float2 &e, float2 &o) { e = make_float2(v.x, v.z); o = make_float2(v.y, v.w); }
+__device__ __forceinline__ void split_cols(const unsigned v, unsigned short &e, unsigned short &o) {
+    e = static_cast<unsigned short>(v & 0xffffu); o = static_cast<unsigned short>(v >> 16);
+}
+__device__ __forceinline__ void split_cols(const uint2 v, unsigned &e, unsigned &o) {
+    e = __byte_perm(v.x, v.y, 0x5410); o = __byte_perm(v.x, v.y, 0x7632);
+}
+__device__ __forceinline__ float2 join_cols(const float e, const float o) { return make_float2(e, o); }
+__device__ __forceinline__ float4 join_cols(const float2 e, const float2 o) { return make_float4(e.x, o.x, e.y, o.y); }
+__device__ __forceinline__ unsigned join_cols(const unsigned short e, const unsigned short o) {
+    return static_cast<unsigned>(e) | (static_cast<unsigned>(o) << 16);
+}
+__device__ __forceinline__ uint2 join_cols(const unsigned e, const unsigned o) {
+    return make_uint2(__byte_perm(e, o, 0x5410), __byte_perm(e, o, 0x7632));
+}
+
+// X [planes][H][W] -> X' [b][phase][ci][H/2][W/2]. One thread per run of 2 NP neighbouring input columns (one aligned
+// vector load; W is a multiple of 2 NP): the even columns go to phase (py, 0), the odd ones to (py, 1), NP elements
+// each. phases = 1 keeps the (0,0) phase only (even rows, even columns). Index arithmetic in 32 bits (the host
+// checks that the number of runs fits).
+template <typename T, int NP>
+__global__ void __launch_bounds__(256) phases_of_kernel(const T *__restrict__ X, T *__restrict__ Xp, unsigned planes,
+                                                        unsigned Cin, unsigned H, unsigned W, int phases) {
+    using V = typename Cols<T, NP>::vec;
+    using Hf = typename Cols<T, NP>::half;
+    const unsigned Ho = H / 2, Wo = W / 2, Wq = Wo / NP;
+    const unsigned rows = phases == 1 ? Ho : H;                   // input rows visited per plane
+    const unsigned n = planes * rows * Wq;
+    const size_t phase_stride = static_cast<size_t>(Cin) * Ho * Wo;
+    for (unsigned i = blockIdx.x * 256u + threadIdx.x; i < n; i += gridDim.x * 256u) {
+        const unsigned r = i / Wq, xq = i - r * Wq;
+        const unsigned plane = r / rows, yr = r - plane * rows;   // plane = b * Cin + ci
+        const unsigned b = plane / Cin, ci = plane - b * Cin;
+        const unsigned y = phases == 1 ? 2 * yr : yr;
+        const unsigned py = y & 1, yo = y >> 1;
+        const V v = *reinterpret_cast<const V *>(X + (static_cast<size_t>(plane) * H + y) * W + 2 * NP * xq);
+        Hf e, o;
+        split_cols(v, e, o);
+        T *dst = Xp + ((static_cast<size_t>(b) * phases + (phases == 1 ? 0 : py * 2)) * Cin + ci) * Ho * Wo +
+                 static_cast<size_t>(yo) * Wo + NP * xq;
+        *reinterpret_cast<Hf *>(dst) = e;
+        if (phases != 1) *reinterpret_cast<Hf *>(dst + phase_stride) = o;
     }
 }
 
-// dX' [b][phase][ci][H/2][W/2] -> dX [b][ci][H][W], one thread per pair of neighbouring output columns;
+// dX' [b][phase][ci][H/2][W/2] -> dX [b][ci][H][W], one thread per run of 2 NP neighbouring output columns;
 // phases = 1: only even rows and columns receive a value, the rest is zero.
-template <typename T>
-__global__ void __launch_bounds__(256) from_phases_kernel(const T *__restrict__ dXp, T *__restrict__ dX, long long B,
-                                                          long long Cin, int H, int W, int phases) {
-    using P = typename Pair<T>::type;
-    const int Ho = H / 2, Wo = W / 2;
-    const long long n = B * Cin * H * Wo;
-    for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += gridDim.x * 256ll) {
-        const int xo = static_cast<int>(i % Wo);
-        const long long r = i / Wo;
-        const int y = static_cast<int>(r % H);
-        const long long plane = r / H;
-        const long long b = plane / Cin, ci = plane - b * Cin;
-        const int py = y & 1, yo = y >> 1;
-        P v;
-        v.x = static_cast<T>(0.f);
-        v.y = static_cast<T>(0.f);
+template <typename T, int NP>
+__global__ void __launch_bounds__(256) from_phases_kernel(const T *__restrict__ dXp, T *__restrict__ dX, unsigned planes,
+                                                          unsigned Cin, unsigned H, unsigned W, int phases) {
+    using V = typename Cols<T, NP>::vec;
+    using Hf = typename Cols<T, NP>::half;
+    const unsigned Ho = H / 2, Wo = W / 2, Wq = Wo / NP;
+    const unsigned n = planes * H * Wq;
+    const size_t phase_stride = static_cast<size_t>(Cin) * Ho * Wo;
+    for (unsigned i = blockIdx.x * 256u + threadIdx.x; i < n; i += gridDim.x * 256u) {
+        const unsigned r = i / Wq, xq = i - r * Wq;
+        const unsigned plane = r / H, y = r - plane * H;
+        const unsigned b = plane / Cin, ci = plane - b * Cin;
+        const unsigned py = y & 1, yo = y >> 1;
+        Hf e = Hf(), o = Hf();                                     // zero bits are zero values in both types
         if (phases != 1) {
-            const long long o0 = (((b * 4 + py * 2) * Cin + ci) * Ho + yo) * Wo + xo;
-            v.x = dXp[o0];
-            v.y = dXp[o0 + Cin * Ho * Wo];
+            const T *src = dXp + ((static_cast<size_t>(b) * 4 + py * 2) * Cin + ci) * Ho * Wo + static_cast<size_t>(yo) * Wo + NP * xq;
+            e = *reinterpret_cast<const Hf *>(src);
+            o = *reinterpret_cast<const Hf *>(src + phase_stride);
         } else if (py == 0) {
-            v.x = dXp[((b * Cin + ci) * Ho + yo) * Wo + xo];
+            e = *reinterpret_cast<const Hf *>(dXp + (static_cast<size_t>(plane) * Ho + yo) * Wo + NP * xq);
         }
-        *reinterpret_cast<P *>(dX + (plane * H + y) * W + 2 * xo) = v;
+        *reinterpret_cast<V *>(dX + (static_cast<size_t>(plane) * H + y) * W + 2 * NP * xq) = join_cols(e, o);
     }
 }
 
@@ -88,30 +112,29 @@ __device__ __forceinline__ int strided_tap(int phase_bit, int t) {
     return phase_bit ? (t == 0 ? 0 : (t == 1 ? 2 : -1)) : (t == 1 ? 1 : -1);
 }
 
-// W [Cout][Cin][3][3] -> W' [Cout][4 Cin][3][3]
-template <typename T>
-__global__ void __launch_bounds__(256) phase_weights_kernel(const T *__restrict__ W, T *__restrict__ Wp, long long Cout,
-                                                            long long Cin) {
-    const long long n = Cout * 4 * Cin * 9;
-    for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += gridDim.x * 256ll) {
-        const int t = static_cast<int>(i % 9);
-        const long long r = i / 9;
-        const long long cp = r % (4 * Cin), co = r / (4 * Cin);
+// W [Cout][Cin][3][3] -> W' [Cout][4 Cin][3][3]  (I: index type, 32 bits where the element count allows)
+template <typename T, typename I>
+__global__ void __launch_bounds__(256) phase_weights_kernel(const T *__restrict__ W, T *__restrict__ Wp, I Cout, I Cin) {
+    const I n = Cout * 4 * Cin * 9;
+    for (I i = blockIdx.x * I(256) + threadIdx.x; i < n; i += gridDim.x * I(256)) {
+        const I r = i / 9;
+        const int t = static_cast<int>(i - r * 9);
+        const I co = r / (4 * Cin), cp = r - co * 4 * Cin;
         const int ph = static_cast<int>(cp / Cin);
-        const long long ci = cp - ph * Cin;
+        const I ci = cp - ph * Cin;
         const int ky = strided_tap(ph >> 1, t / 3), kx = strided_tap(ph & 1, t % 3);
         Wp[i] = (ky >= 0 && kx >= 0) ? W[(co * Cin + ci) * 9 + ky * 3 + kx] : static_cast<T>(0.f);
     }
 }
 
 // dW' [Cout][4 Cin][3][3] -> dW [Cout][Cin][3][3]: the nine places that hold the strided layer's taps
-__global__ void __launch_bounds__(256) strided_dw_kernel(const float *__restrict__ dWp, float *__restrict__ dW,
-                                                         long long Cout, long long Cin) {
-    const long long n = Cout * Cin * 9;
-    for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += gridDim.x * 256ll) {
-        const int t = static_cast<int>(i % 9);
-        const long long r = i / 9;
-        const long long ci = r % Cin, co = r / Cin;
+template <typename I>
+__global__ void __launch_bounds__(256) strided_dw_kernel(const float *__restrict__ dWp, float *__restrict__ dW, I Cout, I Cin) {
+    const I n = Cout * Cin * 9;
+    for (I i = blockIdx.x * I(256) + threadIdx.x; i < n; i += gridDim.x * I(256)) {
+        const I r = i / 9;
+        const int t = static_cast<int>(i - r * 9);
+        const I co = r / Cin, ci = r - co * Cin;
         const int ky = t / 3, kx = t % 3;
         // ky = 0 -> (odd phase, tap 0); 1 -> (even phase, tap 1); 2 -> (odd phase, tap 1)
         const int py = ky != 1, ty = ky == 0 ? 0 : 1;
@@ -122,45 +145,75 @@ __global__ void __launch_bounds__(256) strided_dw_kernel(const float *__restrict
 
 }  // namespace
 
+// runs of columns that the layout kernels index with 32 bits
+static bool fits32(long long n) { return n < (1ll << 31); }
+
 int launch_phases_of(dbp_ctx *ctx, const void *X, void *Xp, int io, long long B, long long Cin, int H, int W, int phases) {
-    const long long n = B * Cin * (phases == 1 ? H / 2 : H) * (W / 2);
+    const int np = W % 4 == 0 ? 2 : 1;
+    const long long n = B * Cin * (phases == 1 ? H / 2 : H) * (W / 2 / np);
+    if (!fits32(B * Cin * H * (W / 2))) return DBP_EUNSUPPORTED;
     const int g = blocks_of(n, 256, ctx->sm_count * 16);
+    const unsigned planes = static_cast<unsigned>(B * Cin), c = static_cast<unsigned>(Cin), h = H, w = W;
     note_launch();
-    if (io == DBP_F32)
-        phases_of_kernel<float><<<g, 256, 0, ctx->stream>>>(static_cast<const float *>(X), static_cast<float *>(Xp), B, Cin, H, W, phases);
-    else
-        phases_of_kernel<__nv_bfloat16><<<g, 256, 0, ctx->stream>>>(static_cast<const __nv_bfloat16 *>(X),
-                                                                    static_cast<__nv_bfloat16 *>(Xp), B, Cin, H, W, phases);
+    if (io == DBP_F32) {
+        const float *in = static_cast<const float *>(X);
+        float *out = static_cast<float *>(Xp);
+        if (np == 2) phases_of_kernel<float, 2><<<g, 256, 0, ctx->stream>>>(in, out, planes, c, h, w, phases);
+        else phases_of_kernel<float, 1><<<g, 256, 0, ctx->stream>>>(in, out, planes, c, h, w, phases);
+    } else {
+        const __nv_bfloat16 *in = static_cast<const __nv_bfloat16 *>(X);
+        __nv_bfloat16 *out = static_cast<__nv_bfloat16 *>(Xp);
+        if (np == 2) phases_of_kernel<__nv_bfloat16, 2><<<g, 256, 0, ctx->stream>>>(in, out, planes, c, h, w, phases);
+        else phases_of_kernel<__nv_bfloat16, 1><<<g, 256, 0, ctx->stream>>>(in, out, planes, c, h, w, phases);
+    }
     return cuda_ok(cudaGetLastError());
 }
 
 int launch_from_phases(dbp_ctx *ctx, const void *dXp, void *dX, int f32, long long B, long long Cin, int H, int W, int phases) {
-    const long long n = B * Cin * H * (W / 2);
+    const int np = W % 4 == 0 ? 2 : 1;
+    const long long n = B * Cin * H * (W / 2 / np);
+    if (!fits32(B * Cin * H * (W / 2))) return DBP_EUNSUPPORTED;
     const int g = blocks_of(n, 256, ctx->sm_count * 16);
+    const unsigned planes = static_cast<unsigned>(B * Cin), c = static_cast<unsigned>(Cin), h = H, w = W;
     note_launch();
-    if (f32)
-        from_phases_kernel<float><<<g, 256, 0, ctx->stream>>>(static_cast<const float *>(dXp), static_cast<float *>(dX), B, Cin, H, W, phases);
-    else
-        from_phases_kernel<__nv_bfloat16><<<g, 256, 0, ctx->stream>>>(static_cast<const __nv_bfloat16 *>(dXp),
-                                                                      static_cast<__nv_bfloat16 *>(dX), B, Cin, H, W, phases);
+    if (f32) {
+        const float *in = static_cast<const float *>(dXp);
+        float *out = static_cast<float *>(dX);
+        if (np == 2) from_phases_kernel<float, 2><<<g, 256, 0, ctx->stream>>>(in, out, planes, c, h, w, phases);
+        else from_phases_kernel<float, 1><<<g, 256, 0, ctx->stream>>>(in, out, planes, c, h, w, phases);
+    } else {
+        const __nv_bfloat16 *in = static_cast<const __nv_bfloat16 *>(dXp);
+        __nv_bfloat16 *out = static_cast<__nv_bfloat16 *>(dX);
+        if (np == 2) from_phases_kernel<__nv_bfloat16, 2><<<g, 256, 0, ctx->stream>>>(in, out, planes, c, h, w, phases);
+        else from_phases_kernel<__nv_bfloat16, 1><<<g, 256, 0, ctx->stream>>>(in, out, planes, c, h, w, phases);
+    }
     return cuda_ok(cudaGetLastError());
 }
 
 int launch_phase_weights(dbp_ctx *ctx, const void *W, void *Wp, int io, long long Cout, long long Cin) {
-    const int g = blocks_of(Cout * 4 * Cin * 9, 256, ctx->sm_count * 16);
+    const long long n = Cout * 4 * Cin * 9;
+    const int g = blocks_of(n, 256, ctx->sm_count * 16);
     note_launch();
-    if (io == DBP_F32)
-        phase_weights_kernel<float><<<g, 256, 0, ctx->stream>>>(static_cast<const float *>(W), static_cast<float *>(Wp), Cout, Cin);
-    else
-        phase_weights_kernel<__nv_bfloat16><<<g, 256, 0, ctx->stream>>>(static_cast<const __nv_bfloat16 *>(W),
-                                                                        static_cast<__nv_bfloat16 *>(Wp), Cout, Cin);
+    if (io == DBP_F32) {
+        const float *in = static_cast<const float *>(W);
+        float *out = static_cast<float *>(Wp);
+        if (fits32(n)) phase_weights_kernel<float, unsigned><<<g, 256, 0, ctx->stream>>>(in, out, static_cast<unsigned>(Cout), static_cast<unsigned>(Cin));
+        else phase_weights_kernel<float, long long><<<g, 256, 0, ctx->stream>>>(in, out, Cout, Cin);
+    } else {
+        const __nv_bfloat16 *in = static_cast<const __nv_bfloat16 *>(W);
+        __nv_bfloat16 *out = static_cast<__nv_bfloat16 *>(Wp);
+        if (fits32(n)) phase_weights_kernel<__nv_bfloat16, unsigned><<<g, 256, 0, ctx->stream>>>(in, out, static_cast<unsigned>(Cout), static_cast<unsigned>(Cin));
+        else phase_weights_kernel<__nv_bfloat16, long long><<<g, 256, 0, ctx->stream>>>(in, out, Cout, Cin);
+    }
     return cuda_ok(cudaGetLastError());
 }
 
 int launch_strided_dw(dbp_ctx *ctx, const float *dWp, float *dW, long long Cout, long long Cin) {
-    const int g = blocks_of(Cout * Cin * 9, 256, ctx->sm_count * 16);
+    const long long n = Cout * Cin * 9;
+    const int g = blocks_of(n, 256, ctx->sm_count * 16);
     note_launch();
-    strided_dw_kernel<<<g, 256, 0, ctx->stream>>>(dWp, dW, Cout, Cin);
+    if (fits32(4 * n)) strided_dw_kernel<unsigned><<<g, 256, 0, ctx->stream>>>(dWp, dW, static_cast<unsigned>(Cout), static_cast<unsigned>(Cin));
+    else strided_dw_kernel<long long><<<g, 256, 0, ctx->stream>>>(dWp, dW, Cout, Cin);
     return cuda_ok(cudaGetLastError());
 }
 

@@ -80,6 +80,7 @@ tc3_tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const int split = blockIdx.x % p.nsplit;
     int rest = blockIdx.x / p.nsplit;
     int kx, ci_t, co_t, live_lo = 0, live_hi = 3;       // rows ky in [live_lo, live_hi) are accumulated (NP == 2)
+    int c_lo = 0, c_hi = (NP == 2 ? 384 : 192) / 32;    // 32-column chunks of the accumulators that are handed over
     if (p.phase_tiles > 0) {
         // per output-channel tile: the phases in order, one kernel column (kx = 1) per channel tile of a phase with
         // px = 0, two (kx = 0, 1) with px = 1
@@ -90,7 +91,9 @@ tc3_tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         r -= py * 3 * tp;
         if (r < tp) { ci_t = 2 * py * tp + r; kx = 1; }
         else { r -= tp; ci_t = (2 * py + 1) * tp + (r >> 1); kx = r & 1; }
-        if (NP == 2) { live_lo = py ? 0 : 1; live_hi = 2; }
+        // NP == 2: columns 0-127 are ky = 0, 128-255 ky = 1, 256-383 ky = 2; NP == 1: 0-63 ky = 2, 64-127 ky = 1, 128-191 ky = 0
+        if (NP == 2) { live_lo = py ? 0 : 1; live_hi = 2; c_lo = 4 * live_lo; c_hi = 8; }
+        else { c_lo = 2; c_hi = py ? 6 : 4; }
     } else {
         kx = rest % 3;
         rest /= 3;
@@ -302,10 +305,9 @@ tc3_tma_dw_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         if (ok) {
             tc_fence_after();
             const long long t_epi = clock64();
-            // NP == 2: four chunks per row ky, only the accumulated rows are handed over
-            const int nchunks = NP == 2 ? 4 * live_hi : 192 / 32;
+            const int nchunks = c_hi;                  // only the rows the layer wants are handed over
             float *stg = reinterpret_cast<float *>(smem);
-            for (int c0 = NP == 2 ? 4 * live_lo : 0; c0 < nchunks; c0 += p.stage_chunks) {
+            for (int c0 = c_lo; c0 < nchunks; c0 += p.stage_chunks) {
                 const int nb = nchunks - c0 < p.stage_chunks ? nchunks - c0 : p.stage_chunks;
                 for (int i = 0; i < nb; ++i) {
                     unsigned v[32];
@@ -378,6 +380,45 @@ tc3_dw_finish_kernel(float *__restrict__ acc, const float *__restrict__ delta_p,
                 if (ci < cin) dW[(co * cin + ci) * 9 + k % 9] = t_s[k];
             }
         }
+        __syncthreads();
+    }
+}
+
+// The same for a stride-2 layer run on phase images (scratch rows of 4 cin channels, phase ph = 2 py + px at channels
+// ph * cin ...): the strided layer's tap (ky, kx) of (co, ci) is tap (ty, tx) of channel ph * cin + ci with
+// ky = 0 -> (py, ty) = (1, 0), 1 -> (0, 1), 2 -> (1, 1), kx likewise; the other scratch entries were never touched.
+// dW[co][ci][ky][kx] is written directly, one (co, ci) pair per thread.
+__global__ void __launch_bounds__(256)
+tc3_dw_finish_phases_kernel(float *__restrict__ acc, const float *__restrict__ delta_p, float *__restrict__ dW, int cout, int cin) {
+    __shared__ float t_s[256 * 9];
+    chain_wait();
+    chain_release();
+    const float delta = *delta_p;
+    const long long pairs = static_cast<long long>(cout) * cin, pairs4 = 4 * pairs;
+    for (long long i0 = blockIdx.x * 256ll; i0 < pairs; i0 += gridDim.x * 256ll) {
+        const long long i = i0 + threadIdx.x;
+        if (i < pairs) {
+            const long long co = i / cin, ci = i - co * cin;
+            float *base = acc + co * 4 * cin + ci;
+            float v[9];
+#pragma unroll
+            for (int t = 0; t < 9; ++t) {
+                const int ky = t / 3, kx = t % 3;
+                const int ph = (ky != 1) * 2 + (kx != 1), tp = (ky == 0 ? 0 : 1) * 3 + (kx == 0 ? 0 : 1);
+                v[t] = __ldcg(base + tp * pairs4 + static_cast<long long>(ph) * cin);
+            }
+#pragma unroll
+            for (int t = 0; t < 9; ++t) {
+                const int ky = t / 3, kx = t % 3;
+                const int ph = (ky != 1) * 2 + (kx != 1), tp = (ky == 0 ? 0 : 1) * 3 + (kx == 0 ? 0 : 1);
+                __stcg(base + tp * pairs4 + static_cast<long long>(ph) * cin, 0.f);
+                t_s[threadIdx.x * 9 + t] = v[t] * delta;
+            }
+        }
+        __syncthreads();
+        const long long left = pairs - i0;
+        const int np = static_cast<int>(left < 256 ? left : 256);
+        for (int k = threadIdx.x; k < np * 9; k += 256) dW[i0 * 9 + k] = t_s[k];
         __syncthreads();
     }
 }
@@ -599,6 +640,14 @@ int launch_tc3_tma_dw(dbp_ctx *ctx, const void *codes_nhwc, const void *X, int i
     if ((rc = cuda_ok(launch_chained(kern, dim3(static_cast<unsigned>(tiles * nsplit)), dim3(kThreadsW3), smem,
                                      ctx->stream, map_q, map_x, map_acc, p))))
         return rc;
+    if (p.phase_tiles > 0 && ctx->phase_dw_out != nullptr) {
+        // the strided layer's own weight gradient, straight from the scratch
+        long long blocks = (static_cast<long long>(pairs / 4) + 255) / 256;
+        if (blocks > ctx->sm_count * 16) blocks = ctx->sm_count * 16;
+        ctx->phase_dw_done = true;
+        return cuda_ok(launch_chained(tc3_dw_finish_phases_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, ctx->stream,
+                                      acc, delta_p, ctx->phase_dw_out, static_cast<int>(s.Cout), ctx->phase_cin));
+    }
     long long blocks = (static_cast<long long>(pairs) + 255) / 256;
     if (blocks > ctx->sm_count * 16) blocks = ctx->sm_count * 16;
     return cuda_ok(launch_chained(tc3_dw_finish_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, ctx->stream, acc,

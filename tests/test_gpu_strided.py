@@ -160,3 +160,21 @@ def test_stride2_rejects_what_it_cannot_do(ctx):
     rc = lib.dithered_conv_backward(ctx._h, d.data_ptr(), X.data_ptr(), W.data_ptr(), dbp.binding._dtype_code(d),
                                     1, 8, 8, 6, 8, 3, 3, 1, 0, 2.0, None, None, None, None, None, 0)
     assert rc == -2
+
+
+def test_stride2_leaves_the_weight_gradient_scratch_clean(ctx):
+    """A strided 3x3 layer and a plain one share the weight-gradient scratch: whatever one leaves there would show
+    up in the other's dW. Alternate them (both widths of the code operand) and compare with each layer run alone."""
+    import paper_2004_04729_b200 as dbp
+    fro = lambda a, b: float((a.double() - b.double()).norm() / b.double().norm())
+    for co in (64, 128):
+        S = wl.conv_layer(2, 128, co, 16, 16, 3, data_seed=41 + co, scale=5.0, dtype="bf16", stride=2)
+        P = wl.conv_layer(2, 512, co, 8, 8, 3, data_seed=43 + co, scale=5.0, dtype="bf16")
+        s_in = [_dev(a, "bf16") for a in (S.delta, S.X, S.W)]
+        p_in = [_dev(a, "bf16") for a in (P.delta, P.X, P.W)]
+        plain_alone = dbp.dithered_conv_backward(ctx, *p_in, 1, 5.0)["dW"].clone()
+        strided_alone = dbp.dithered_conv_backward(ctx, *s_in, 1, 5.0, stride=2)["dW"].clone()
+        for _ in range(2):
+            a = dbp.dithered_conv_backward(ctx, *s_in, 1, 5.0, stride=2)["dW"]
+            b = dbp.dithered_conv_backward(ctx, *p_in, 1, 5.0)["dW"]
+            assert fro(a, strided_alone) <= 1e-5 and fro(b, plain_alone) <= 1e-5
