@@ -513,6 +513,7 @@ def main():
     ap.add_argument("--crossover-sweep", action="store_true", help="time the sparse and the dense path against density and exit")
     ap.add_argument("--force-sparse", action="store_true", help="gather kernels on every layer (profiling aid)")
     ap.add_argument("--bf16", action="store_true", help="configs 1 and 3 with bf16 storage (profiling aid: the bf16 linear kernels)")
+    ap.add_argument("--strided-only", action="store_true", help="time the stride-2 layers of the network and exit (profiling aid)")
     ap.add_argument("--sync-dw", action="store_true", help="every call joins its dW before it returns (no DBP_DW_ASYNC)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl != "reference":
@@ -540,6 +541,10 @@ def main():
     if args.crossover_sweep:
         if rank == 0:
             crossover_sweep(torch, dbp, ctx)
+        return
+    if args.strided_only:
+        if rank == 0:
+            print(json.dumps({"strided_layers": strided_table(torch, dbp, ctx, hbm_peak, args.no_dense, args.batch or 64)}))
         return
 
     if args.config in CHAIN_NAMES:
