@@ -271,6 +271,19 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
         if (wr) return wr;
         jobs.w_src = W; jobs.w_dst = ctx->w_taps.ptr; jobs.w_f32 = io == DBP_F32; jobs.Cout = s.Cout; jobs.Cin = s.Cin;
     }
+    // a stride-2 layer run on phase images: W is a workspace for the phase weights that nobody has written yet.
+    // The re-laying side job makes its tap-major copy straight from the layer's own weights; any other path reads
+    // the phase weights themselves, which are made here
+    if (ctx->phase_w_src != nullptr && dX) {
+        if (w_side && ctx->phase_cin > 0 && s.Cin == 4ll * ctx->phase_cin) {
+            jobs.w_src = ctx->phase_w_src;
+            jobs.phase_cin = ctx->phase_cin;
+        } else {
+            KernelTimer t(ctx, DBP_K_GLUE);
+            const int pr = launch_phase_weights(ctx, ctx->phase_w_src, const_cast<void *>(W), io, s.Cout, s.Cin / 4);
+            if (pr) return pr;
+        }
+    }
     // tiny planes: the weight-gradient kernel reads the images stacked into tall ones
     const int stack_g = (t3 && dW) ? tc3_stack_images(s, io) : 0;
     const void *codes_st = nullptr;
@@ -412,13 +425,10 @@ int conv_backward_stride2(dbp_ctx *ctx, const void *delta, const void *X, const 
         KernelTimer t(ctx, DBP_K_GLUE);
         if ((rc = launch_phases_of(ctx, X, ctx->s2_x.ptr, io, s.B, s.Cin, static_cast<int>(s.H), static_cast<int>(s.W), phases))) return rc;
     }
-    if (dX && s.k == 3) {
-        KernelTimer t(ctx, DBP_K_GLUE);
-        if ((rc = launch_phase_weights(ctx, W, ctx->s2_w.ptr, io, s.Cout, s.Cin))) return rc;
-    }
     ctx->next_mask = mask;
     ctx->phase_cin = s.k == 3 ? static_cast<int>(s.Cin) : 0;      // the 3x3 tensor-core kernels skip the taps that are zero by construction
     ctx->phase_dw_out = (s.k == 3 && dW) ? dW : nullptr;
+    ctx->phase_w_src = (s.k == 3 && dX) ? W : nullptr;            // the phase weights are made inside, in the form the path wants
     ctx->phase_dw_done = false;
     rc = conv_backward_impl(ctx, delta, dW ? ctx->s2_x.ptr : nullptr, dX ? (s.k == 3 ? ctx->s2_w.ptr : W) : nullptr, io, in,
                             seed, scale, delta_in, q_out,
@@ -426,6 +436,7 @@ int conv_backward_stride2(dbp_ctx *ctx, const void *delta, const void *X, const 
                             dX ? ctx->s2_dx.ptr : nullptr, db, flags & ~DBP_DW_ASYNC);
     ctx->phase_cin = 0;
     ctx->phase_dw_out = nullptr;
+    ctx->phase_w_src = nullptr;
     if (rc) return rc;
     if (dX) {
         KernelTimer t(ctx, DBP_K_GLUE);

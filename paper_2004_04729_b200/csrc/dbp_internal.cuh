@@ -56,6 +56,7 @@ struct dbp_ctx {
     const uint8_t *next_mask = nullptr; // ReLU mask for the next backward call (dbp_set_relu_mask)
     dbp::Workspace dz_tmp;              // delta_z = delta_a (.) mask when that call cannot fold the mask into its loads
     dbp::Workspace codes_stack[2];      // the same codes with G images stacked into one tall image (tiny planes, dW)
+    const void *phase_w_src = nullptr;  // that layer's own weights: its W argument is a workspace for the phase weights, not yet written
     float *phase_dw_out = nullptr;      // that layer's dW: the 3x3 weight-gradient kernels write it directly when they run in phase mode ...
     bool phase_dw_done = false;         // ... and say so here
     int phase_cin = 0;                  // > 0 while a stride-2 3x3 layer runs as a stride-1 layer on phase images: its own channel count
@@ -114,6 +115,7 @@ struct SideJobs {
     void *w_dst = nullptr;
     int w_f32 = 0;
     long long Cout = 0, Cin = 0;
+    int phase_cin = 0;                 // > 0: w_src holds a stride-2 layer's own weights [Cout][phase_cin][9], Cin = 4 phase_cin
 };
 int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long numel, float scale,
                       const float *delta_in, float *delta_out, unsigned long long *nnz_out,

@@ -89,7 +89,7 @@ statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ par
                   DeviceState *__restrict__ st, float scale, float *__restrict__ delta_out,
                   unsigned long long *__restrict__ nnz_out, uint4 *__restrict__ zero_ptr, long long zero_n16,
                   const void *__restrict__ w_src, unsigned short *__restrict__ w_dst, int w_f32, long long w_cout, int w_cin,
-                  const unsigned char *__restrict__ mask) {
+                  const unsigned char *__restrict__ mask, int w_phase_cin) {
     constexpr int EPT = Elem<T>::EPT;
     const long long nvec = n / EPT;
     chain_wait();
@@ -99,21 +99,52 @@ statistics_kernel(const T *__restrict__ x, long long n, double *__restrict__ par
          i += static_cast<long long>(gridDim.x) * kThreads)
         zero_ptr[i] = make_uint4(0u, 0u, 0u, 0u);
     // side job for the layer's 3x3 input-gradient kernel: weights [co][ci][9] -> [co][tap][ci] bf16 (for fp32
-    // weights two pieces: taps 0-8 the values rounded to bf16, taps 9-17 the remainders rounded to bf16)
+    // weights two pieces: taps 0-8 the values rounded to bf16, taps 9-17 the remainders rounded to bf16).
+    // w_phase_cin > 0: the layer is a stride-2 layer run on the four phase images of its input; w_src holds that
+    // layer's own weights [co][w_phase_cin][9] and channel ph * w_phase_cin + c of the re-laid weights is phase
+    // ph = 2 py + px of channel c, whose tap (ty, tx) is the strided layer's tap ky = 0 for (py, ty) = (1, 0),
+    // 1 for (0, 1), 2 for (1, 1), kx likewise, and zero for every other pair.
     if (w_src != nullptr) {
         const int per_co = 9 * w_cin, taps = w_f32 ? 18 : 9;
         for (long long co = blockIdx.x; co < w_cout; co += gridDim.x) {
             unsigned short *dst = w_dst + co * taps * w_cin;
-            for (int j = threadIdx.x; j < per_co; j += kThreads) {
-                const int t = j / w_cin, ci = j - t * w_cin;                 // writes run along ci
+            // a thread takes one channel and all nine taps: nine independent loads, then stores that run along ci
+            for (int ci = threadIdx.x; ci < w_cin; ci += kThreads) {
+                int ph = 0;
+                long long base = (co * w_cin + ci) * 9;
+                if (w_phase_cin > 0) {
+                    ph = ci / w_phase_cin;
+                    base = (co * w_phase_cin + (ci - ph * w_phase_cin)) * 9;
+                }
+                int k[9];                                                  // source tap, or -1 for a zero weight
+#pragma unroll
+                for (int t = 0; t < 9; ++t) {
+                    const int ty = t / 3, tx = t % 3;
+                    k[t] = t;
+                    if (w_phase_cin > 0) {
+                        const int ky = (ph & 2) ? (ty == 0 ? 0 : (ty == 1 ? 2 : -1)) : (ty == 1 ? 1 : -1);
+                        const int kx = (ph & 1) ? (tx == 0 ? 0 : (tx == 1 ? 2 : -1)) : (tx == 1 ? 1 : -1);
+                        k[t] = (ky >= 0 && kx >= 0) ? ky * 3 + kx : -1;
+                    }
+                }
                 if (w_f32) {
-                    const float w = __ldg(static_cast<const float *>(w_src) + co * per_co + ci * 9 + t);
-                    const __nv_bfloat16 hi = __float2bfloat16_rn(w);
-                    const __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(hi));
-                    dst[j] = *reinterpret_cast<const unsigned short *>(&hi);
-                    dst[per_co + j] = *reinterpret_cast<const unsigned short *>(&lo);
+                    float w[9];
+#pragma unroll
+                    for (int t = 0; t < 9; ++t) w[t] = k[t] >= 0 ? __ldg(static_cast<const float *>(w_src) + base + k[t]) : 0.f;
+#pragma unroll
+                    for (int t = 0; t < 9; ++t) {
+                        const __nv_bfloat16 hi = __float2bfloat16_rn(w[t]);
+                        const __nv_bfloat16 lo = __float2bfloat16_rn(w[t] - __bfloat162float(hi));
+                        dst[t * w_cin + ci] = *reinterpret_cast<const unsigned short *>(&hi);
+                        dst[per_co + t * w_cin + ci] = *reinterpret_cast<const unsigned short *>(&lo);
+                    }
                 } else {
-                    dst[j] = __ldg(static_cast<const unsigned short *>(w_src) + co * per_co + ci * 9 + t);
+                    unsigned short w[9];
+#pragma unroll
+                    for (int t = 0; t < 9; ++t)
+                        w[t] = k[t] >= 0 ? __ldg(static_cast<const unsigned short *>(w_src) + base + k[t]) : static_cast<unsigned short>(0);
+#pragma unroll
+                    for (int t = 0; t < 9; ++t) dst[t * w_cin + ci] = w[t];
                 }
             }
         }
@@ -449,13 +480,13 @@ int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long nume
     if (dtype == DBP_F32 && mask != nullptr)
         e = launch_chained(statistics_kernel<float, true>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
                            static_cast<const float *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out, zp, zn, jobs.w_src, wd, jobs.w_f32, jobs.Cout, wci,
-                           static_cast<const unsigned char *>(mask));
+                           static_cast<const unsigned char *>(mask), jobs.phase_cin);
     else if (dtype == DBP_F32)
         e = launch_chained(statistics_kernel<float, false>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
-                           static_cast<const float *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out, zp, zn, jobs.w_src, wd, jobs.w_f32, jobs.Cout, wci, nomask);
+                           static_cast<const float *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out, zp, zn, jobs.w_src, wd, jobs.w_f32, jobs.Cout, wci, nomask, jobs.phase_cin);
     else
         e = launch_chained(statistics_kernel<__nv_bfloat16, false>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, ctx->stream,
-                           static_cast<const __nv_bfloat16 *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out, zp, zn, jobs.w_src, wd, jobs.w_f32, jobs.Cout, wci, nomask);
+                           static_cast<const __nv_bfloat16 *>(delta), numel, ctx->partials, ctx->state, scale, delta_out, nnz_out, zp, zn, jobs.w_src, wd, jobs.w_f32, jobs.Cout, wci, nomask, jobs.phase_cin);
     return cuda_ok(e);
 }
 

@@ -178,3 +178,17 @@ def test_stride2_leaves_the_weight_gradient_scratch_clean(ctx):
             a = dbp.dithered_conv_backward(ctx, *s_in, 1, 5.0, stride=2)["dW"]
             b = dbp.dithered_conv_backward(ctx, *p_in, 1, 5.0)["dW"]
             assert fro(a, strided_alone) <= 1e-5 and fro(b, plain_alone) <= 1e-5
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_stride2_with_a_given_step_size(ctx, dtype):
+    """scale <= 0 and a device step size: no statistics kernel runs, so the weights take the other route."""
+    import paper_2004_04729_b200 as dbp
+    L = wl.conv_layer(2, 128, 64, 16, 16, 3, data_seed=51, scale=2.0, dtype=dtype, stride=2)
+    d, X, W = (_dev(a, dtype) for a in (L.delta, L.X, L.W))
+    D = np.float32(2.0 * oracle.mean_std(L.delta)[1])
+    step = torch.tensor([float(D)], dtype=torch.float32, device="cuda")
+    out = dbp.dithered_conv_backward(ctx, d, X, W, 6, 0.0, delta_in=step, need_db=True, stride=2, flags=dbp.DBP_DX_F32)
+    torch.cuda.synchronize()
+    codes, _, _ = oracle.nsd_codes(L.delta, 6, D)
+    _check(out, oracle.conv_backward_strided(codes, D, L.X, L.W, 2, with_abs=True), 1e-5)
