@@ -37,7 +37,7 @@ typedef enum { DBP_F32 = 0, DBP_BF16 = 1 } dbp_dtype;
 typedef enum {
     DBP_OK = 0,
     DBP_EINVAL = -1,        /* null / misaligned pointer, non-positive size, bad enum */
-    DBP_EUNSUPPORTED = -2,  /* kernel size, stride or padding outside {1x1, 3x3; 1, 2; (k-1)/2} */
+    DBP_EUNSUPPORTED = -2,  /* kernel size, stride or padding outside {1x1, 3x3; 1, 2; (k-1)/2} and {5x5; 1; 2} */
     DBP_ECUDA = -3,         /* a CUDA runtime call failed */
     DBP_ENOMEM = -4,        /* workspace allocation failed */
     DBP_ENONFINITE = -5,    /* device: delta holds NaN or Inf (all codes were set to 0) */
@@ -244,7 +244,8 @@ int dithered_linear_backward(dbp_ctx *ctx, const void *delta, const void *X, con
 
 /*
  * The same for a convolution layer ("analogous for convolutional layers", Section 3):
- * cross-correlation, NCHW, square kernel k in {1, 3}, stride 1 or 2, zero padding (k-1)/2.
+ * cross-correlation, NCHW, square kernel k in {1, 3}, stride 1 or 2, zero padding (k-1)/2; also k = 5 with
+ * stride 1 and padding 2 (the 5x5 layers of LeNet-5-like networks; these run on the gather kernels only).
  * H and Wd are the height and width of X. Stride 1: delta [B,Cout,H,W], X [B,Cin,H,W], W [Cout,Cin,k,k]:
  *     dX[b,ci,y,x]     = Delta sum_{co,ky,kx} q[b,co,y-ky+p,x-kx+p] W[co,ci,ky,kx]
  *     dW[co,ci,ky,kx]  = Delta sum_{b,y,x}    q[b,co,y,x] X[b,ci,y+ky-p,x+kx-p]

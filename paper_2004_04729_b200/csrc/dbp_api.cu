@@ -359,7 +359,7 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
         void *wt = ctx->w_taps.ptr;
         const bool dx_bf16 = (io == DBP_BF16) && !(flags & DBP_DX_F32);
         // streamed kernel: weight rows must be 16-byte multiples; otherwise the generic one
-        const bool streamed = (s.Cin * static_cast<long long>(elem_size(io))) % 16 == 0;
+        const bool streamed = s.k != 5 && (s.Cin * static_cast<long long>(elem_size(io))) % 16 == 0;
         {
             KernelTimer t(ctx, DBP_K_WEIGHT_TAPS);
             rc = launch_weight_taps(ctx, W, io, s, wt, !streamed);
@@ -376,7 +376,7 @@ int conv_backward_impl(dbp_ctx *ctx, const void *delta, const void *X, const voi
     if (dW && ctx->hook_before_dw && cudaStreamWaitEvent(ctx->stream, ctx->hook_before_dw, 0) != cudaSuccess) return DBP_ECUDA;
     if (dW) {
         KernelTimer t(ctx, DBP_K_DW);
-        rc = launch_conv_dw_streamed(ctx, codes, X, io, delta_p, s, dW);
+        rc = s.k == 5 ? DBP_EUNSUPPORTED : launch_conv_dw_streamed(ctx, codes, X, io, delta_p, s, dW);
         if (rc == DBP_EUNSUPPORTED) rc = launch_conv_dw(ctx, codes, X, io, delta_p, s, dW);
         if (rc) return rc;
     }
@@ -453,7 +453,7 @@ int conv_backward_stride2(dbp_ctx *ctx, const void *delta, const void *X, const 
 }
 
 bool conv_form_supported(int k, int stride, int pad) {
-    return (k == 1 || k == 3) && (stride == 1 || stride == 2) && pad == (k - 1) / 2;
+    return ((k == 1 || k == 3) && (stride == 1 || stride == 2) && pad == (k - 1) / 2) || (k == 5 && stride == 1 && pad == 2);
 }
 
 int conv_backward_any(dbp_ctx *ctx, const void *delta, const void *X, const void *W, int io, const ConvShape &s,

@@ -3,7 +3,7 @@
 // Section 3.4), Delta is applied once per output, accumulation is fp32.
 //
 // A linear layer is the 1x1 convolution with H = W = 1 (the memory layouts coincide), so one
-// pair of kernels covers linear, 1x1 and 3x3.
+// pair of kernels covers linear, 1x1, 3x3 and 5x5 (the 5x5 layers of LeNet-5-like networks run here only).
 #include "dbp_internal.cuh"
 
 namespace dbp {
@@ -427,6 +427,7 @@ int launch_conv_dx(dbp_ctx *ctx, const int8_t *codes, const float *w_taps, const
 #define DBP_DX(KS, VEC)                                                                         \
     (dx_bf16 ? launch_dx_t<KS, VEC, __nv_bfloat16>(ctx, p, smem) : launch_dx_t<KS, VEC, float>(ctx, p, smem))
     if (s.k == 1) return vec == 4 ? DBP_DX(1, 4) : vec == 2 ? DBP_DX(1, 2) : DBP_DX(1, 1);
+    if (s.k == 5) return vec == 4 ? DBP_DX(5, 4) : vec == 2 ? DBP_DX(5, 2) : DBP_DX(5, 1);
     return vec == 4 ? DBP_DX(3, 4) : vec == 2 ? DBP_DX(3, 2) : DBP_DX(3, 1);
 #undef DBP_DX
 }
@@ -449,7 +450,8 @@ int launch_conv_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, int dtype,
     p.codes = codes; p.X = X; p.delta_p = delta_p; p.dW = dW;
     p.B = static_cast<int>(s.B); p.Cin = static_cast<int>(s.Cin); p.Cout = static_cast<int>(s.Cout);
     p.H = static_cast<int>(s.H); p.W = static_cast<int>(s.W);
-    const int ci_t = s.Cin <= 64 ? 64 : 128;
+    // 5x5: 25 taps x 4 channels of accumulators per thread leave no room for a second output channel per group
+    const int ci_t = (s.Cin <= 64 || s.k == 5) ? 64 : 128;
     const int pad = (s.k - 1) / 2;
     int max_pos = 128;
     size_t smem = 0;
@@ -477,6 +479,7 @@ int launch_conv_dw(dbp_ctx *ctx, const int8_t *codes, const void *X, int dtype,
     (dtype == DBP_F32 ? launch_dw_t<KS, CT, float>(ctx, p, smem, grid)                       \
                       : launch_dw_t<KS, CT, __nv_bfloat16>(ctx, p, smem, grid))
     if (s.k == 1) return ci_t == 64 ? DBP_DW(1, 64) : DBP_DW(1, 128);
+    if (s.k == 5) return DBP_DW(5, 64);
     return ci_t == 64 ? DBP_DW(3, 64) : DBP_DW(3, 128);
 #undef DBP_DW
 }

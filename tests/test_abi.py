@@ -47,7 +47,7 @@ def test_host_side_argument_checks_need_no_gpu():
     assert lib.dbp_layer_seed(0, 1) == 0x6E789E6AA1B965F4
     assert lib.nsd_quantize(None, None, 0, 10, 0, 2.0, None, None) == -1
     # unsupported kernel size is refused before anything touches the device
-    assert lib.dithered_conv_backward(None, None, None, None, 0, 1, 1, 1, 4, 4, 5, 1, 2, 0, 2.0,
+    assert lib.dithered_conv_backward(None, None, None, None, 0, 1, 1, 1, 4, 4, 7, 1, 3, 0, 2.0,
                                       None, None, None, None, None, 0) == -2
 
 

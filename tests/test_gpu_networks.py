@@ -129,3 +129,10 @@ def test_config4_vgg16_full_batch_sampled(ctx):
 def test_small_conv_pool_chain_other_seed(ctx):
     c = wl.vgg_chain(batch=3, cfg=[8, "M", 16, 16, "M"], hw=8, data_seed=77)
     _run_chain(ctx, c, seed=5)
+
+
+def test_lenet5_like_chain_with_5x5_kernels(ctx):
+    """conv5x5(1->6) - pool - conv5x5(6->16) - pool - classifier on 32x32 inputs (same padding): the whole
+    backward pass layer by layer against the oracle."""
+    c = wl.vgg_chain(batch=8, cfg=[6, "M", 16, "M"], hw=32, in_ch=1, data_seed=55, k=5, name="lenet5_like")
+    _run_chain(ctx, c, seed=5)

@@ -192,3 +192,29 @@ def test_stride2_with_a_given_step_size(ctx, dtype):
     torch.cuda.synchronize()
     codes, _, _ = oracle.nsd_codes(L.delta, 6, D)
     _check(out, oracle.conv_backward_strided(codes, D, L.X, L.W, 2, with_abs=True), 1e-5)
+
+
+@pytest.mark.parametrize("B,Ci,Co,H,W,dtype", [
+    (4, 1, 6, 32, 32, "f32"),        # LeNet-5 C1 (same padding)
+    (4, 6, 16, 14, 14, "f32"),       # LeNet-5 C3
+    (2, 3, 64, 32, 32, "f32"),       # an AlexNet-for-CIFAR first layer
+    (2, 64, 192, 8, 8, "f32"),
+    (3, 10, 7, 5, 9, "f32"),         # planes smaller than the kernel's reach in one direction
+    (2, 16, 24, 12, 12, "bf16"),
+    (1, 128, 40, 7, 7, "bf16"),
+])
+def test_5x5_layers(ctx, B, Ci, Co, H, W, dtype):
+    """5x5 kernels (stride 1, padding 2) against the oracle's definition: codes bit-exact, products within 1e-5."""
+    import paper_2004_04729_b200 as dbp
+    L = wl.conv_layer(B, Ci, Co, H, W, 5, data_seed=3 * B + Ci + Co, scale=2.0, dtype=dtype)
+    d, X, W_ = (_dev(a, dtype) for a in (L.delta, L.X, L.W))
+    q = dbp.SparseGradient(d.numel())
+    out = dbp.dithered_conv_backward(ctx, d, X, W_, 8, 2.0, q_out=q, need_db=True, flags=dbp.DBP_DX_F32)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == (0, 0)
+    D = np.float32(q.delta.item())
+    codes, nnz, _ = oracle.nsd_codes(L.delta, 8, D)
+    assert np.array_equal(dbp.nsd_decode_dense(ctx, q).cpu().numpy().reshape(codes.shape), codes)
+    _check(out, oracle.conv_backward(codes, D, L.X, L.W, with_abs=True), 1e-5)
+    with pytest.raises(dbp.DbpError):
+        dbp.dithered_conv_backward(ctx, d, X, W_, 8, 2.0, flags=dbp.DBP_FORCE_DENSE)

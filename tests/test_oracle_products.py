@@ -33,7 +33,7 @@ def test_linear_matches_bruteforce():
     assert a["dW"].shape == W.shape and a["dX"].shape == X.shape
 
 
-@pytest.mark.parametrize("k,H,W", [(3, 4, 5), (1, 3, 4), (3, 1, 1), (3, 2, 7)])
+@pytest.mark.parametrize("k,H,W", [(3, 4, 5), (1, 3, 4), (3, 1, 1), (3, 2, 7), (5, 6, 5), (5, 2, 3)])
 def test_conv_matches_bruteforce(k, H, W):
     c, D, X, Wt = _tiny_conv(k=k, H=H, W=W, seed=k + H)
     a, b = oracle.conv_backward(c, D, X, Wt), oracle.conv_backward_bruteforce(c, D, X, Wt)
@@ -41,7 +41,7 @@ def test_conv_matches_bruteforce(k, H, W):
         np.testing.assert_allclose(a[key], b[key], rtol=0, atol=1e-13)
 
 
-@pytest.mark.parametrize("k", [1, 3])
+@pytest.mark.parametrize("k", [1, 3, 5])
 def test_conv_matches_library_autograd(k):
     c, D, X, Wt = _tiny_conv(B=3, Co=4, Ci=5, H=6, W=7, k=k, seed=5)
     Xt = torch.tensor(X, dtype=torch.float64, requires_grad=True)

@@ -234,8 +234,8 @@ VGG16_CIFAR = [64, 64, "M", 128, 128, "M", 256, 256, 256, "M", 512, 512, 512, "M
 
 
 def vgg_chain(batch=128, cfg=None, hw=32, in_ch=3, classes=10, *, data_seed=1004,
-              scale=2.0, device="cpu") -> Chain:
-    """VGG-16 (CIFAR variant, no batch-norm): 3x3 convs + ReLU, 2x2 max-pool after each
+              scale=2.0, device="cpu", k=3, name="vgg16_cifar") -> Chain:
+    """VGG-16 (CIFAR variant, no batch-norm): k x k convs (3x3 unless asked) + ReLU, 2x2 max-pool after each
     stage, one fully-connected classifier; He-initialised weights, N(0,1) input, random
     labels. The forward pass runs through torch (on `device`) -- it only makes inputs."""
     import torch
@@ -248,9 +248,9 @@ def vgg_chain(batch=128, cfg=None, hw=32, in_ch=3, classes=10, *, data_seed=1004
     i = 0
     while i < len(cfg):
         co = cfg[i]
-        W = normal(data_seed, 10 + li, co * c * 9, sigma=(2.0 / (c * 9)) ** 0.5)
-        W = torch.from_numpy(W.reshape(co, c, 3, 3).astype(np.float32)).to(device)
-        z = F.conv2d(a, W, padding=1)
+        W = normal(data_seed, 10 + li, co * c * k * k, sigma=(2.0 / (c * k * k)) ** 0.5)
+        W = torch.from_numpy(W.reshape(co, c, k, k).astype(np.float32)).to(device)
+        z = F.conv2d(a, W, padding=(k - 1) // 2)
         kinds.append("conv")
         Xs.append(a.cpu().numpy())
         Ws.append(W.cpu().numpy())
@@ -279,6 +279,6 @@ def vgg_chain(batch=128, cfg=None, hw=32, in_ch=3, classes=10, *, data_seed=1004
     masks.append(None)
     pools.append(None)
     labels = (uniform01(data_seed, 2, batch) * classes).astype(np.int64) % classes
-    return Chain("vgg16_cifar", kinds, Xs, Ws, masks, pools,
+    return Chain(name, kinds, Xs, Ws, masks, pools,
                  _softmax_minus_onehot(logits.cpu().numpy(), labels), scale,
                  extra={"feat_shape": tuple(a.shape)})
