@@ -441,3 +441,28 @@ def network_backward(ctx: Context, kinds, Xs, Ws, relu_masks, pool_argmax, delta
                 g = maxpool2x2_backward(ctx, g, pool_argmax[l - 1])
             delta_a = g
     return res
+
+
+def average_weight_gradients(grads, group=None) -> None:
+    """The exchange step of the data-parallel form (Section 3.6): every rank's weight gradients are replaced, in
+    place, by their mean over the ranks of `group` (the parameter server's average followed by its broadcast, as
+    one all-reduce). `grads`: this rank's dW tensors (fp32, one device). They travel as one flat bucket, so the
+    collective's launch cost is paid once per step, not once per layer. With one rank it does nothing.
+    Plumbing only: `torch.distributed` (NCCL between GPUs) moves and adds the data."""
+    import torch.distributed as dist
+    grads = [g for g in grads if g is not None]
+    if not grads or not dist.is_available() or not dist.is_initialized():
+        return
+    world = dist.get_world_size(group)
+    if world == 1:
+        return
+    if any(g.dtype != torch.float32 or g.device != grads[0].device for g in grads):
+        raise ValueError("weight gradients must be float32 tensors on one device")
+    bucket = torch.cat([g.reshape(-1) for g in grads])
+    dist.all_reduce(bucket, op=dist.ReduceOp.SUM, group=group)
+    bucket.div_(world)
+    off = 0
+    for g in grads:
+        n = g.numel()
+        g.copy_(bucket[off:off + n].view_as(g))
+        off += n
