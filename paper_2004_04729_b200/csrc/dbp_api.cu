@@ -401,6 +401,7 @@ int conv_backward_stride2(dbp_ctx *ctx, const void *delta, const void *X, const 
     if (io != DBP_F32 && io != DBP_BF16) return DBP_EINVAL;
     if (s.B <= 0 || s.Cin <= 0 || s.Cout <= 0 || s.H <= 0 || s.W <= 0 || s.H > 8192 || s.W > 8192) return DBP_EINVAL;
     if ((s.H & 1) || (s.W & 1)) return DBP_EUNSUPPORTED;
+    if (s.B * s.Cin * s.H * (s.W / 2) >= (1ll << 31)) return DBP_EUNSUPPORTED;      // the layout kernels index in 32 bits
     if ((dW && !X) || (dX && !W)) return DBP_EINVAL;
     if (!aligned16(X) || !aligned16(W) || !aligned16(dW) || !aligned16(dX)) return DBP_EINVAL;
     DeviceGuard guard(ctx->device);

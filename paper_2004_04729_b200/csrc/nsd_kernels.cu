@@ -454,6 +454,8 @@ decode_kernel(const uint32_t *__restrict__ bitmap, const uint16_t *__restrict__ 
 
 }  // namespace
 
+constexpr int kStatBlocksPerSM = 2;
+
 int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long numel, float scale,
                       const float *delta_in, float *delta_out, unsigned long long *nnz_out, const SideJobs &jobs,
                       const uint8_t *mask) {
@@ -475,6 +477,11 @@ int launch_statistics(dbp_ctx *ctx, const void *delta, int dtype, long long nume
     if (jobs.w_src != nullptr && blocks < jobs.Cout) blocks = jobs.Cout;
     if (jobs.zero != nullptr && blocks < static_cast<long long>(jobs.zero_bytes / (16 * kThreads * 4))) blocks = static_cast<long long>(jobs.zero_bytes / (16 * kThreads * 4));
     if (blocks > ctx->partial_blocks) blocks = ctx->partial_blocks;
+    // two resident blocks per SM, each walking several tiles, finish sooner than one block per tile: fewer partial
+    // sums for the last block to add and fewer tickets (measured on the ResNet-50 layer set: 0.70 against 0.73 ms
+    // per step for 48 layers; one block per SM: 0.76). The weight re-laying side job wants one block per output channel.
+    if (jobs.w_src == nullptr && blocks > static_cast<long long>(ctx->sm_count) * kStatBlocksPerSM)
+        blocks = static_cast<long long>(ctx->sm_count) * kStatBlocksPerSM;
     cudaError_t e;
     const unsigned char *nomask = nullptr;
     if (dtype == DBP_F32 && mask != nullptr)
